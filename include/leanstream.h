@@ -1,0 +1,214 @@
+/*
+ * leanstream.h -- C ABI of the B200 (sm_100a) speculate-and-refine sparse FFN decode library.
+ *
+ * One FFN layer of a decoder at batch 1 (small batches allowed) is executed the way Section 2.1 of the
+ * LeanStream paper describes: a predictor scores the layer's hidden neurons from a residual feature
+ * (speculate), the selected neurons are computed in K priority-ordered stages (Eq. 1), and after every stage the
+ * partial residual feature (Eq. 2) re-scores the neurons of the next layer (refine).  Weights of layers that do
+ * not fit in HBM live in pinned host memory and are served through an HBM neuron cache (Section 3.3.3, cache
+ * eviction task; Section 4.3, cache miss ratio).
+ *
+ * Conventions
+ *  - Every function returns an int32_t status: LS_OK (0) or a negative LS_ERR_* code; ls_last_error() gives a
+ *    text for the calling thread's last failure.  Nothing throws, aborts or traps.
+ *  - Pointers named d_* and every pointer inside ls_selection / ls_step_trace are DEVICE pointers owned by the
+ *    caller; the library neither frees nor keeps them after the call has been enqueued.  Pointers inside
+ *    ls_layer_desc are HOST pointers read only during ls_layer_create().
+ *  - `stream` arguments carry a cudaStream_t (0 = the legacy default stream).  Work is enqueued asynchronously;
+ *    argument validation is synchronous.  Calls on layers with a cache (cache_rows > 0) synchronise with the host
+ *    to issue the miss copies and must not be made during stream capture; calls on fully resident layers never
+ *    synchronise or allocate and may be captured in a CUDA graph.
+ *  - A layer handle is not thread safe: one call at a time per layer; per-layer scratch is reused by every call.
+ *  - Neuron i of a layer owns gate row i, up row i and down-projection row i (column i of the paper's W_gate /
+ *    W_up, row i of W_down).  Index lists are int32, masks hold neuron i at bit (i & 31) of word (i >> 5).
+ */
+#ifndef LEANSTREAM_H_
+#define LEANSTREAM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define LS_OK 0
+#define LS_ERR_INVALID (-1)  /* bad argument (null pointer, size out of range, unsupported combination) */
+#define LS_ERR_NOMEM (-2)    /* host or device allocation failed */
+#define LS_ERR_CUDA (-3)     /* a CUDA runtime call failed; ls_last_error() has the CUDA message */
+#define LS_ERR_STATE (-4)    /* call not valid for this layer (e.g. cache call on a resident layer) */
+#define LS_ERR_CAPACITY (-5) /* wanted + protected neurons exceed the cache capacity, or a list exceeds its cap */
+#define LS_ERR_TIMEOUT (-6)  /* a bounded wait for miss copies gave up */
+
+#define LS_ACT_RELU 0
+#define LS_WDTYPE_BF16 0
+#define LS_WDTYPE_FP16 1
+#define LS_NORM_RMS 0
+#define LS_NORM_NONE 1
+
+typedef struct ls_layer ls_layer;
+
+/*
+ * Problem statement of one FFN layer: the operands of Eq. 1 plus the layer's neuron predictor.
+ *   act(h W_gate) * (h W_up) W_down with act = ReLU (the sparsity source of Section 2.1); gated = 0 gives the
+ *   two-matrix form act(h W_fc1 + b) W_fc2 + b_down.  h = rmsnorm(x) without gain (norm = LS_NORM_RMS) or h = x.
+ *   Predictor (Section 3.3.3: projection of the feature, then the scorer): s = pred_b^T (pred_a^T h) + pred_c.
+ * All weight matrices are 16-bit (wdtype), row-major, HOST memory, copied by ls_layer_create():
+ *   w_gate, w_up, w_down_t: [d_ff][d_model] (w_down_t is neuron-major, i.e. the transposed down projection);
+ *   pred_a: [d_model][pred_rank];  pred_b: [pred_rank][d_ff];  b_gate, pred_c: float [d_ff] or NULL (zeros);
+ *   b_down: float [d_model] or NULL.  d_model and pred_rank must be multiples of 8; d_model <= 16384.
+ * cache_rows = 0 keeps every neuron in HBM.  cache_rows > 0 keeps the weights in library-owned pinned host memory
+ *   and gives the layer an HBM cache of that many neuron bundles (gate, up, down rows of one neuron).
+ * max_batch (default 1 when 0, at most 8) and max_sel (default d_ff when 0) size the per-layer scratch: the largest
+ *   batch and the longest selection list any call will pass.
+ */
+typedef struct {
+  uint32_t struct_size; /* sizeof(ls_layer_desc), checked */
+  int32_t device;       /* CUDA device ordinal */
+  int32_t d_model, d_ff;
+  int32_t gated, act, wdtype, norm;
+  float norm_eps;
+  int32_t pred_rank;
+  const void *w_gate, *w_up, *w_down_t;
+  const float *b_gate, *b_down;
+  const void *pred_a, *pred_b;
+  const float *pred_c;
+  int64_t cache_rows;
+  int32_t max_batch, max_sel;
+} ls_layer_desc;
+
+/* Creates a layer on desc->device (weights uploaded before return).  *out is owned by the library until
+ * ls_layer_destroy().  Errors: LS_ERR_INVALID (shape/flags), LS_ERR_NOMEM, LS_ERR_CUDA; *out is NULL on failure. */
+int32_t ls_layer_create(const ls_layer_desc *desc, ls_layer **out);
+/* Waits for the layer's own streams, frees everything the layer owns.  NULL is accepted. */
+int32_t ls_layer_destroy(ls_layer *layer);
+
+/*
+ * A selection of neurons (caller-allocated device buffers).
+ *   scores: [d_ff] priority of every neuron (batch > 1: max over the batch), fp64; NULL = not wanted.
+ *   mask:   [ceil(d_ff/32)] membership bitmask; NULL = not wanted.
+ *   idx:    [cap] the selected neurons in RANK ORDER (highest priority first; equal scores: lower index first),
+ *           so that stage c of K is the slice [c*m, min(count,(c+1)*m)), m = ceil(count/K).
+ *   count:  [1] number of selected neurons (k at batch 1, size of the union otherwise).
+ */
+typedef struct {
+  double *scores;
+  uint32_t *mask;
+  int32_t *idx;
+  int32_t *count;
+  int32_t cap;
+} ls_selection;
+
+/*
+ * Speculate (Section 2.1, Fig. 2; Section 3.3.3 neuron-activation prediction): scores every neuron of `layer`
+ * from d_feature [batch][d_model] (float, un-normalised residual-like feature; the library applies the layer's
+ * norm), accumulating in fp64, and selects per token the k best under the total order (score descending, index
+ * ascending; NaN ranks last, -0 equals +0); batch > 1 returns the union ordered by the per-neuron maximum score.
+ * The layer keeps the priorities as its cache-retention priorities.  0 <= k <= d_ff; out->idx and out->count are
+ * required and out->cap >= min(batch*k, d_ff).  Errors: LS_ERR_INVALID; device-side problems (a list longer than
+ * its cap) are reported through ls_layer_status().
+ */
+int32_t ls_predict(ls_layer *layer, const float *d_feature, int32_t batch, int32_t k, ls_selection *out,
+                   void *stream);
+
+/*
+ * Optional validation outputs of ls_sparse_ffn_step (device pointers, each may be NULL).
+ *   xtilde:        [n_chunks+1][batch][d_model] partial residual features x~^(j), j = 0..K (Eq. 2)
+ *   refine_masks:  [n_chunks+1][ceil(d_ff_next/32)] refined sets C^(j) for the next layer
+ *   refine_counts: [n_chunks+1] their sizes
+ *   survive_mask:  [ceil(d_ff/32)] selected neurons whose activation is nonzero for some token
+ *   exec_idx:      [count] the order in which the selected neurons were executed (differs from the rank order
+ *                  only on cached layers: residents first, then misses, each in rank order)
+ */
+typedef struct {
+  float *xtilde;
+  uint32_t *refine_masks;
+  int32_t *refine_counts;
+  uint32_t *survive_mask;
+  int32_t *exec_idx;
+} ls_step_trace;
+
+/*
+ * One layer's speculate-and-refine step (Section 2.1, Eq. 1 and Eq. 2; Section 3.2.2 permutation-invariant
+ * execution): h = norm(x); the neurons listed in `sel` (rank order, *sel->count of them) run in n_chunks stages;
+ * stage c adds dm^(c) = sum_i a_i W_down[i] over its neurons with a_i = relu(w_gate[i].h + b_i) * (w_up[i].h),
+ * reading down rows only where a_i != 0; x~^(0) = x (+ b_down), x~^(j) = x~^(j-1) + dm^(j); d_x_out = x~^(K).
+ * When `next` is given, every x~^(j), j = 0..K, is scored by next's predictor and the top k_next set C^(j) is
+ * formed; C^(K) is returned in sel_next (required when next != NULL) and next's retention priorities are updated
+ * at each stage.  When `next` has a cache, the first ceil(count_j (j+1)/(K+1)) ranks of C^(j), j < K, are reserved
+ * in it (miss copies start on next's copy stream).  When `layer` has a cache, the whole selection is reserved
+ * first, residents run before misses, and the stages that need copied rows wait for them on `stream`.
+ * d_x, d_x_out: float [batch][d_model]; d_x_out may alias d_x.  next may equal layer.
+ * Errors: LS_ERR_INVALID, LS_ERR_CAPACITY (cached layer: selection larger than the cache), LS_ERR_CUDA.
+ */
+int32_t ls_sparse_ffn_step(ls_layer *layer, ls_layer *next, const float *d_x, float *d_x_out, int32_t batch,
+                           const ls_selection *sel, int32_t n_chunks, int32_t k_next, ls_selection *sel_next,
+                           ls_step_trace *trace, void *stream);
+
+/*
+ * HBM neuron cache (Section 3.3.3 cache-eviction task; Section 4.3 cache miss ratio).  Residency is logical: a
+ * neuron is resident once a slot is assigned to it; its bytes arrive on the layer's copy stream and consumers
+ * wait for the copy event.  All three calls return LS_ERR_STATE on a layer created with cache_rows = 0.
+ *
+ * ls_cache_lookup: d_slot[j] = slot of neuron d_idx[j] or -1 (miss); *d_nhit = number of residents.  n <= max_sel.
+ *
+ * ls_cache_reserve: makes the first `admit_ranks` entries (< 0: all) of want->idx resident.  The new resident set
+ *   is the cache_rows best of (residents + wanted) under the key (wanted or protected first, then retention
+ *   priority descending, then index ascending); the rest are evicted and their slots given to the misses, whose
+ *   bundles are copied from pinned host memory with cudaMemcpyAsync on the layer's copy stream.  When
+ *   want->scores is given it first replaces the layer's retention priorities.  d_protect_mask (nullable) marks
+ *   neurons that must not be evicted.  *h_nmiss (nullable, HOST) receives the number of misses.  Synchronises
+ *   `stream` with the host.  LS_ERR_CAPACITY if wanted + protected exceed cache_rows (nothing changes).
+ *
+ * ls_cache_evict: evicts lowest-priority unprotected residents until at least min_free slots are free (fewer when
+ *   only protected ones remain); d_evicted (nullable, [cache_rows]) and d_nevicted (nullable) receive them.
+ */
+int32_t ls_cache_lookup(ls_layer *layer, const int32_t *d_idx, int32_t n, int32_t *d_slot, int32_t *d_nhit,
+                        void *stream);
+int32_t ls_cache_reserve(ls_layer *layer, const ls_selection *want, int32_t admit_ranks,
+                         const uint32_t *d_protect_mask, int32_t *h_nmiss, void *stream);
+int32_t ls_cache_evict(ls_layer *layer, int32_t min_free, const uint32_t *d_protect_mask, int32_t *d_evicted,
+                       int32_t *d_nevicted, void *stream);
+/* d_resident_mask [ceil(d_ff/32)] <- current logical resident set (for parity checks). */
+int32_t ls_cache_snapshot(ls_layer *layer, uint32_t *d_resident_mask, void *stream);
+/* Makes `stream` wait until every miss copy issued so far for this layer has landed. */
+int32_t ls_cache_wait(ls_layer *layer, void *stream);
+
+typedef struct {
+  int64_t hits, misses, evictions; /* counted over reserve calls (wanted entries found / not found resident) */
+  int64_t h2d_bytes;               /* bytes copied from pinned host memory into cache slots */
+  int64_t h2d_copies;              /* number of cudaMemcpyAsync calls issued for them */
+  int64_t resident;                /* current number of resident neurons */
+} ls_cache_stats_t;
+/* Host-side counters (no synchronisation needed; they are updated when a reserve call returns). */
+int32_t ls_cache_stats(ls_layer *layer, ls_cache_stats_t *host_out);
+
+/* Reads and clears the layer's device-side status word (0 = no problem seen by any kernel since the last read;
+ * otherwise the first LS_ERR_* code a kernel recorded, e.g. an out-of-range neuron index, which kernels skip
+ * rather than dereference).  Synchronises the device. */
+int32_t ls_layer_status(ls_layer *layer, int32_t *host_status);
+
+/*
+ * Kernel timing for roofline accounting (no counterpart in the paper).  While enabled (process-wide, off by default)
+ * the launches of the named kernel groups are bracketed by CUDA events on the stream they are launched on; not valid
+ * during stream capture.  ls_timing_read() waits for the recorded events of one group, returns their number and summed
+ * duration in milliseconds, and forgets them.
+ */
+#define LS_TIMED_GATEUP 0  /* gate/up gather-GEMV + activation of one stage */
+#define LS_TIMED_DOWN 1    /* sparse down projection of one stage */
+#define LS_TIMED_PREDICT 2 /* latent + scores + top-k of one predictor evaluation */
+#define LS_TIMED_FUSED 3   /* the fused per-layer step kernel */
+int32_t ls_timing_enable(int32_t on);
+int32_t ls_timing_read(int32_t kind, int64_t *launches, double *total_ms);
+
+/* Number of kernels launched by this library in the calling process since load (for launch accounting). */
+int64_t ls_kernel_launches(void);
+/* Copies the calling thread's last error text (NUL terminated, truncated to n) and returns its length. */
+size_t ls_last_error(char *buf, size_t n);
+/* Library ABI version (major * 1000 + minor). */
+int32_t ls_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LEANSTREAM_H_ */

@@ -1,0 +1,578 @@
+// Host side of the C ABI declared in include/leanstream.h: handles, argument checks, launches.
+#include "../../include/leanstream.h"
+
+#include <atomic>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "ls_cache.cuh"
+#include "ls_kernels.cuh"
+
+namespace {
+
+thread_local std::string g_err;
+std::atomic<int64_t> g_launches{0};
+
+int32_t fail(int32_t code, const char* fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof buf, fmt, ap);
+  va_end(ap);
+  g_err = buf;
+  return code;
+}
+
+#define LS_CUDA(call)                                                                         \
+  do {                                                                                        \
+    cudaError_t e_ = (call);                                                                  \
+    if (e_ != cudaSuccess) return fail(LS_ERR_CUDA, "%s: %s", #call, cudaGetErrorString(e_)); \
+  } while (0)
+
+#define LS_LAUNCHED()                                                                                   \
+  do {                                                                                                  \
+    g_launches.fetch_add(1, std::memory_order_relaxed);                                                 \
+    cudaError_t e_ = cudaPeekAtLastError();                                                             \
+    if (e_ != cudaSuccess) return fail(LS_ERR_CUDA, "kernel launch (%s:%d): %s", __FILE__, __LINE__,    \
+                                       cudaGetErrorString(e_));                                        \
+  } while (0)
+
+// Optional per-kernel timing with CUDA events on the launching stream (roofline accounting; off by default).
+struct TimedLaunch { int kind; cudaEvent_t a, b; };
+std::atomic<int> g_timing{0};
+std::mutex g_timing_mu;
+std::vector<TimedLaunch> g_timed;
+
+struct KernelTimer {
+  cudaStream_t st;
+  TimedLaunch t{};
+  bool on;
+  KernelTimer(int kind, cudaStream_t s) : st(s), on(g_timing.load(std::memory_order_relaxed) != 0) {
+    if (!on) return;
+    t.kind = kind;
+    if (cudaEventCreate(&t.a) != cudaSuccess || cudaEventCreate(&t.b) != cudaSuccess) { on = false; return; }
+    cudaEventRecord(t.a, st);
+  }
+  ~KernelTimer() {
+    if (!on) return;
+    cudaEventRecord(t.b, st);
+    std::lock_guard<std::mutex> lk(g_timing_mu);
+    g_timed.push_back(t);
+  }
+};
+
+struct DeviceGuard {
+  int prev = -1;
+  explicit DeviceGuard(int dev) {
+    cudaGetDevice(&prev);
+    if (prev != dev) cudaSetDevice(dev);
+  }
+  ~DeviceGuard() {
+    int cur = -1;
+    cudaGetDevice(&cur);
+    if (prev >= 0 && cur != prev) cudaSetDevice(prev);
+  }
+};
+
+}  // namespace
+
+struct ls_layer {
+  int device = 0;
+  int d = 0, F = 0, gated = 1, act = 0, wd = 0, norm = 0, r = 0;
+  float eps = 1e-5f;
+  int n_mat = 3;
+  int max_batch = 1, max_sel = 0;
+  int nwords = 0;
+  int sm_count = 148;
+  int64_t cache_rows = 0;  // 0: resident
+  int64_t nslots = 0;
+
+  // weights (device)
+  uint16_t* bundles = nullptr;  // [nslots][n_mat][d]
+  float* b_gate = nullptr;
+  float* b_down = nullptr;
+  uint16_t* pred_at = nullptr;  // [r][d]
+  uint16_t* pred_bt = nullptr;  // [F][r]
+  float* pred_c = nullptr;
+
+  // scratch (device)
+  double* z = nullptr;       // [max_batch][r]
+  double* sumsq = nullptr;   // [max_batch]
+  double* scores = nullptr;  // [max_batch][F] (batch > 1 only)
+  double* prio = nullptr;    // [F] latest priorities (retention priorities of the cache)
+  unsigned long long* cand_key = nullptr;  // [F]
+  int32_t* cand_idx = nullptr;             // [F]
+  uint32_t* umask = nullptr;               // [nwords] union mask (batch > 1)
+  int32_t* tmp_idx = nullptr;              // [max_sel] refined list of a stage j < K
+  int32_t* tmp_count = nullptr;            // [1]
+  uint32_t* tmp_mask = nullptr;            // [nwords]
+  float* xin = nullptr;                    // [max_batch][d]
+  float* xt = nullptr;                     // [max_batch][d] current partial residual feature
+  float* actv = nullptr;                   // [max_batch][max_sel]
+  float* ypart = nullptr;                  // [down_splits][max_batch][d]
+  uint32_t* survive = nullptr;             // [nwords]
+  int* status = nullptr;                   // [1]
+  int down_splits = 0;
+
+  ls::CacheState cache;  // residency tables, pinned backing store, copy stream
+};
+
+namespace {
+
+template <typename T>
+int32_t dalloc(T** p, size_t n) {
+  *p = nullptr;
+  if (n == 0) n = 1;
+  cudaError_t e = cudaMalloc(reinterpret_cast<void**>(p), n * sizeof(T));
+  if (e != cudaSuccess) return fail(e == cudaErrorMemoryAllocation ? LS_ERR_NOMEM : LS_ERR_CUDA, "cudaMalloc(%zu bytes): %s",
+                                    n * sizeof(T), cudaGetErrorString(e));
+  return LS_OK;
+}
+
+#define LS_TRY(expr)              \
+  do {                            \
+    int32_t rc_ = (expr);         \
+    if (rc_ != LS_OK) return rc_; \
+  } while (0)
+
+void free_layer(ls_layer* L) {
+  if (!L) return;
+  ls::cache_destroy(L->cache);
+  cudaFree(L->bundles); cudaFree(L->b_gate); cudaFree(L->b_down); cudaFree(L->pred_at); cudaFree(L->pred_bt);
+  cudaFree(L->pred_c); cudaFree(L->z); cudaFree(L->sumsq); cudaFree(L->scores); cudaFree(L->prio); cudaFree(L->cand_key);
+  cudaFree(L->cand_idx); cudaFree(L->umask); cudaFree(L->tmp_idx); cudaFree(L->tmp_count); cudaFree(L->tmp_mask);
+  cudaFree(L->xin); cudaFree(L->xt); cudaFree(L->actv); cudaFree(L->ypart); cudaFree(L->survive); cudaFree(L->status);
+  delete L;
+}
+
+int32_t upload_f32(float** dst, const float* src, size_t n) {
+  LS_TRY(dalloc(dst, n));
+  if (src) LS_CUDA(cudaMemcpy(*dst, src, n * sizeof(float), cudaMemcpyHostToDevice));
+  else LS_CUDA(cudaMemset(*dst, 0, n * sizeof(float)));
+  return LS_OK;
+}
+
+// [rows][cols] 16-bit host matrix -> transposed [cols][rows] on the device
+int32_t upload_transposed16(uint16_t** dst, const void* src, int rows, int cols) {
+  std::vector<uint16_t> t;
+  try { t.resize((size_t)rows * cols); } catch (const std::bad_alloc&) { return fail(LS_ERR_NOMEM, "host staging buffer"); }
+  const uint16_t* s = static_cast<const uint16_t*>(src);
+  for (int i = 0; i < rows; ++i)
+    for (int j = 0; j < cols; ++j) t[(size_t)j * rows + i] = s[(size_t)i * cols + j];
+  LS_TRY(dalloc(dst, t.size()));
+  LS_CUDA(cudaMemcpy(*dst, t.data(), t.size() * 2, cudaMemcpyHostToDevice));
+  return LS_OK;
+}
+
+int32_t create_impl(const ls_layer_desc* D, ls_layer* L) {
+  L->device = D->device; L->d = D->d_model; L->F = D->d_ff; L->gated = D->gated ? 1 : 0; L->act = D->act;
+  L->wd = D->wdtype; L->norm = D->norm; L->eps = D->norm_eps; L->r = D->pred_rank; L->n_mat = L->gated ? 3 : 2;
+  L->max_batch = D->max_batch > 0 ? D->max_batch : 1;
+  L->max_sel = D->max_sel > 0 ? D->max_sel : D->d_ff;
+  L->nwords = (L->F + 31) / 32;
+  L->cache_rows = D->cache_rows;
+  L->nslots = D->cache_rows > 0 ? D->cache_rows : L->F;
+  cudaDeviceProp prop;
+  LS_CUDA(cudaGetDeviceProperties(&prop, D->device));
+  L->sm_count = prop.multiProcessorCount;
+  const size_t d = L->d, F = L->F, row_bytes = d * 2, bundle_bytes = row_bytes * L->n_mat;
+
+  LS_TRY(dalloc(&L->bundles, (size_t)L->nslots * L->n_mat * d));
+  const void* mats[3] = {D->w_gate, L->gated ? D->w_up : D->w_down_t, D->w_down_t};
+  if (L->cache_rows == 0) {
+    for (int m = 0; m < L->n_mat; ++m)
+      LS_CUDA(cudaMemcpy2D(reinterpret_cast<char*>(L->bundles) + m * row_bytes, bundle_bytes, mats[m], row_bytes, row_bytes, F,
+                           cudaMemcpyHostToDevice));
+  } else {
+    LS_TRY(ls::cache_create(L->cache, (int)F, (int)L->cache_rows, bundle_bytes, L->max_sel, g_err));
+    char* hb = static_cast<char*>(L->cache.h_bundles);
+    for (int m = 0; m < L->n_mat; ++m) {
+      const char* src = static_cast<const char*>(mats[m]);
+      for (size_t i = 0; i < F; ++i) memcpy(hb + i * bundle_bytes + m * row_bytes, src + i * row_bytes, row_bytes);
+    }
+  }
+  LS_TRY(upload_f32(&L->b_gate, D->b_gate, F));
+  if (D->b_down) LS_TRY(upload_f32(&L->b_down, D->b_down, d));
+  LS_TRY(upload_transposed16(&L->pred_at, D->pred_a, (int)d, L->r));
+  LS_TRY(upload_transposed16(&L->pred_bt, D->pred_b, L->r, (int)F));
+  LS_TRY(upload_f32(&L->pred_c, D->pred_c, F));
+
+  const size_t MB = L->max_batch;
+  LS_TRY(dalloc(&L->z, MB * L->r));
+  LS_TRY(dalloc(&L->sumsq, MB));
+  LS_TRY(dalloc(&L->scores, MB > 1 ? MB * F : 1));
+  LS_TRY(dalloc(&L->prio, F));
+  LS_TRY(dalloc(&L->cand_key, F));
+  LS_TRY(dalloc(&L->cand_idx, F));
+  LS_TRY(dalloc(&L->umask, (size_t)L->nwords));
+  LS_TRY(dalloc(&L->tmp_idx, (size_t)L->max_sel));
+  LS_TRY(dalloc(&L->tmp_count, 1));
+  LS_TRY(dalloc(&L->tmp_mask, (size_t)L->nwords));
+  LS_TRY(dalloc(&L->xin, MB * d));
+  LS_TRY(dalloc(&L->xt, MB * d));
+  LS_TRY(dalloc(&L->actv, MB * L->max_sel));
+  L->down_splits = L->sm_count;
+  LS_TRY(dalloc(&L->ypart, (size_t)L->down_splits * MB * d));
+  LS_TRY(dalloc(&L->survive, (size_t)L->nwords));
+  LS_TRY(dalloc(&L->status, 1));
+  LS_CUDA(cudaMemset(L->status, 0, sizeof(int)));
+  LS_CUDA(cudaMemset(L->prio, 0xff, F * sizeof(double)));  // NaN: ranks last until a prediction sets it
+
+  // opt in to the large dynamic shared memory the kernels may ask for
+  const int big = 200 * 1024;
+  LS_CUDA(cudaFuncSetAttribute(ls::ls_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, big));
+  LS_CUDA(cudaFuncSetAttribute(ls::ls_scores_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024));
+  LS_CUDA(cudaFuncSetAttribute(ls::ls_scores_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024));
+#define LS_ATTR_GU(WD, BT) \
+  LS_CUDA(cudaFuncSetAttribute(ls::ls_gateup_kernel<WD, BT>, cudaFuncAttributeMaxDynamicSharedMemorySize, big))
+  LS_ATTR_GU(0, 1); LS_ATTR_GU(0, 4); LS_ATTR_GU(0, 8); LS_ATTR_GU(1, 1); LS_ATTR_GU(1, 4); LS_ATTR_GU(1, 8);
+#undef LS_ATTR_GU
+  LS_CUDA(cudaDeviceSynchronize());
+  return LS_OK;
+}
+
+// ---- speculate / refine: latent -> scores -> top-k (-> union for batch > 1) ------------------------------------------
+int32_t predict_impl(ls_layer* L, const float* d_feature, int B, int k, double* scores_user, uint32_t* mask_out,
+                     int32_t* idx_out, int32_t* count_out, int cap, cudaStream_t st) {
+  const int d = L->d, r = L->r, F = L->F;
+  KernelTimer timer(LS_TIMED_PREDICT, st);
+  {
+    const int wpb = 8, grid = (r + wpb - 1) / wpb;
+    if (L->wd == 0) ls::ls_latent_kernel<0><<<grid, 256, 0, st>>>(L->pred_at, d_feature, d, r, B, L->z, L->sumsq);
+    else ls::ls_latent_kernel<1><<<grid, 256, 0, st>>>(L->pred_at, d_feature, d, r, B, L->z, L->sumsq);
+    LS_LAUNCHED();
+  }
+  {
+    const int grid = std::min((F + 7) / 8, L->sm_count * 8);
+    const size_t sm = (size_t)B * r * sizeof(double);
+    if (L->wd == 0)
+      ls::ls_scores_kernel<0><<<grid, 256, sm, st>>>(L->pred_bt, L->pred_c, L->z, L->sumsq, d, r, F, B, L->norm, L->eps, L->scores,
+                                                     L->prio, scores_user);
+    else
+      ls::ls_scores_kernel<1><<<grid, 256, sm, st>>>(L->pred_bt, L->pred_c, L->z, L->sumsq, d, r, F, B, L->norm, L->eps, L->scores,
+                                                     L->prio, scores_user);
+    LS_LAUNCHED();
+  }
+  const size_t tsm = ls::topk_kernel_smem(F);
+  if (B == 1) {
+    ls::ls_topk_kernel<<<1, ls::TK_THREADS, tsm, st>>>(L->prio, F, k, nullptr, idx_out, cap, mask_out, 0, count_out, L->cand_key,
+                                                       L->cand_idx, L->status);
+    LS_LAUNCHED();
+  } else {
+    ls::ls_fill_u32_kernel<<<1, 256, 0, st>>>(L->umask, 0u, L->nwords);
+    LS_LAUNCHED();
+    for (int b = 0; b < B; ++b) {
+      ls::ls_topk_kernel<<<1, ls::TK_THREADS, tsm, st>>>(L->scores + (size_t)b * F, F, k, nullptr, nullptr, 0, L->umask, 1, nullptr,
+                                                         L->cand_key, L->cand_idx, L->status);
+      LS_LAUNCHED();
+    }
+    ls::ls_topk_kernel<<<1, ls::TK_THREADS, tsm, st>>>(L->prio, F, F, L->umask, idx_out, cap, mask_out, 0, count_out, L->cand_key,
+                                                       L->cand_idx, L->status);
+    LS_LAUNCHED();
+  }
+  return LS_OK;
+}
+
+template <int WD, int BT>
+int32_t launch_stage(ls_layer* L, int B, const int32_t* exec_idx, const int32_t* count_ptr, int sel_cap, int K, int c,
+                     cudaStream_t st) {
+  const int d = L->d;
+  const int32_t* slot_of = L->cache_rows > 0 ? L->cache.d_slot_of : nullptr;
+  const int per_stage = (sel_cap + K - 1) / K;
+  {
+    KernelTimer timer(LS_TIMED_GATEUP, st);
+    const int grid = std::max(1, std::min((per_stage + 7) / 8, L->sm_count * 4));
+    const size_t sm = (size_t)B * d * sizeof(float);
+    ls::ls_gateup_kernel<WD, BT><<<grid, 256, sm, st>>>(L->bundles, L->n_mat, L->gated, slot_of, L->b_gate, L->xin, B, d, L->norm,
+                                                        L->eps, exec_idx, count_ptr, K, c, L->F, L->actv, L->max_sel, L->survive,
+                                                        L->status);
+    LS_LAUNCHED();
+  }
+  {
+    KernelTimer timer(LS_TIMED_DOWN, st);
+    const int tiles = (d / 8 + 255) / 256;
+    const int splits = std::max(1, std::min(L->down_splits, std::max(1, L->sm_count / tiles)));
+    dim3 grid(tiles, splits);
+    ls::ls_down_kernel<WD, BT><<<grid, 256, 0, st>>>(L->bundles, L->n_mat, slot_of, exec_idx, count_ptr, K, c, L->actv, L->max_sel, B,
+                                                     d, L->F, L->ypart);
+    LS_LAUNCHED();
+    return splits;
+  }
+}
+
+int32_t launch_stage_dispatch(ls_layer* L, int B, const int32_t* exec_idx, const int32_t* count_ptr, int sel_cap, int K, int c,
+                              cudaStream_t st) {
+#define LS_STAGE(WD, BT) return launch_stage<WD, BT>(L, B, exec_idx, count_ptr, sel_cap, K, c, st)
+  if (L->wd == 0) {
+    if (B == 1) LS_STAGE(0, 1);
+    if (B <= 4) LS_STAGE(0, 4);
+    LS_STAGE(0, 8);
+  } else {
+    if (B == 1) LS_STAGE(1, 1);
+    if (B <= 4) LS_STAGE(1, 4);
+    LS_STAGE(1, 8);
+  }
+#undef LS_STAGE
+}
+
+int32_t check_layer_call(ls_layer* L, int batch, const char* what) {
+  if (!L) return fail(LS_ERR_INVALID, "%s: layer is NULL", what);
+  if (batch < 1 || batch > L->max_batch) return fail(LS_ERR_INVALID, "%s: batch %d outside [1, max_batch=%d]", what, batch, L->max_batch);
+  return LS_OK;
+}
+
+}  // namespace
+
+// =====================================================================================================================
+extern "C" {
+
+int32_t ls_version(void) { return 1000; }
+
+size_t ls_last_error(char* buf, size_t n) {
+  if (buf && n > 0) {
+    const size_t m = std::min(n - 1, g_err.size());
+    memcpy(buf, g_err.data(), m);
+    buf[m] = 0;
+  }
+  return g_err.size();
+}
+
+int64_t ls_kernel_launches(void) { return g_launches.load(); }
+
+int32_t ls_timing_enable(int32_t on) {
+  g_timing.store(on ? 1 : 0);
+  return LS_OK;
+}
+
+int32_t ls_timing_read(int32_t kind, int64_t* launches, double* total_ms) {
+  if (!launches || !total_ms) return fail(LS_ERR_INVALID, "ls_timing_read: NULL argument");
+  std::lock_guard<std::mutex> lk(g_timing_mu);
+  *launches = 0;
+  *total_ms = 0.0;
+  std::vector<TimedLaunch> keep;
+  for (const TimedLaunch& t : g_timed) {
+    if (t.kind != kind) { keep.push_back(t); continue; }
+    float ms = 0.f;
+    cudaError_t e = cudaEventSynchronize(t.b);
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, t.a, t.b);
+    cudaEventDestroy(t.a);
+    cudaEventDestroy(t.b);
+    if (e != cudaSuccess) return fail(LS_ERR_CUDA, "ls_timing_read: %s", cudaGetErrorString(e));
+    *launches += 1;
+    *total_ms += ms;
+  }
+  g_timed.swap(keep);
+  return LS_OK;
+}
+
+int32_t ls_layer_create(const ls_layer_desc* D, ls_layer** out) {
+  if (out) *out = nullptr;
+  if (!D || !out) return fail(LS_ERR_INVALID, "ls_layer_create: NULL argument");
+  if (D->struct_size != sizeof(ls_layer_desc))
+    return fail(LS_ERR_INVALID, "ls_layer_create: struct_size %u, expected %zu", D->struct_size, sizeof(ls_layer_desc));
+  if (D->d_model < 8 || D->d_model % 8 || D->d_model > 16384) return fail(LS_ERR_INVALID, "d_model must be a multiple of 8 in [8, 16384]");
+  if (D->d_ff < 1 || D->d_ff > 32768) return fail(LS_ERR_INVALID, "d_ff must be in [1, 32768]");
+  if (D->pred_rank < 8 || D->pred_rank % 8 || D->pred_rank > 1024) return fail(LS_ERR_INVALID, "pred_rank must be a multiple of 8 in [8, 1024]");
+  if (D->act != LS_ACT_RELU) return fail(LS_ERR_INVALID, "only LS_ACT_RELU is implemented");
+  if (D->wdtype != LS_WDTYPE_BF16 && D->wdtype != LS_WDTYPE_FP16) return fail(LS_ERR_INVALID, "unknown wdtype");
+  if (D->norm != LS_NORM_RMS && D->norm != LS_NORM_NONE) return fail(LS_ERR_INVALID, "unknown norm");
+  if (!D->w_gate || !D->w_down_t || (D->gated && !D->w_up) || !D->pred_a || !D->pred_b)
+    return fail(LS_ERR_INVALID, "ls_layer_create: missing weight pointer");
+  if (D->cache_rows < 0 || D->cache_rows > D->d_ff) return fail(LS_ERR_INVALID, "cache_rows must be in [0, d_ff]");
+  if (D->max_batch < 0 || D->max_batch > 8) return fail(LS_ERR_INVALID, "max_batch must be in [0, 8]");
+  if (D->max_sel < 0 || D->max_sel > D->d_ff) return fail(LS_ERR_INVALID, "max_sel must be in [0, d_ff]");
+  const int mb = D->max_batch > 0 ? D->max_batch : 1;
+  if ((size_t)mb * D->d_model * 4 > 192 * 1024) return fail(LS_ERR_INVALID, "max_batch * d_model * 4 bytes must fit in 192 KB of shared memory");
+  int ndev = 0;
+  LS_CUDA(cudaGetDeviceCount(&ndev));
+  if (D->device < 0 || D->device >= ndev) return fail(LS_ERR_INVALID, "device %d out of range", D->device);
+  DeviceGuard guard(D->device);
+  ls_layer* L = new (std::nothrow) ls_layer();
+  if (!L) return fail(LS_ERR_NOMEM, "host allocation");
+  const int32_t rc = create_impl(D, L);
+  if (rc != LS_OK) {
+    const std::string keep = g_err;
+    free_layer(L);
+    cudaGetLastError();
+    g_err = keep;
+    return rc;
+  }
+  *out = L;
+  return LS_OK;
+}
+
+int32_t ls_layer_destroy(ls_layer* L) {
+  if (!L) return LS_OK;
+  DeviceGuard guard(L->device);
+  cudaDeviceSynchronize();
+  free_layer(L);
+  return LS_OK;
+}
+
+int32_t ls_layer_status(ls_layer* L, int32_t* host_status) {
+  if (!L || !host_status) return fail(LS_ERR_INVALID, "ls_layer_status: NULL argument");
+  DeviceGuard guard(L->device);
+  LS_CUDA(cudaDeviceSynchronize());
+  LS_CUDA(cudaMemcpy(host_status, L->status, sizeof(int), cudaMemcpyDeviceToHost));
+  LS_CUDA(cudaMemset(L->status, 0, sizeof(int)));
+  return LS_OK;
+}
+
+int32_t ls_predict(ls_layer* L, const float* d_feature, int32_t batch, int32_t k, ls_selection* out, void* stream) {
+  LS_TRY(check_layer_call(L, batch, "ls_predict"));
+  if (!d_feature || !out || !out->idx || !out->count) return fail(LS_ERR_INVALID, "ls_predict: feature, out->idx and out->count are required");
+  if (k < 0 || k > L->F) return fail(LS_ERR_INVALID, "ls_predict: k %d outside [0, d_ff]", k);
+  const long need = std::min<long>((long)batch * k, L->F);
+  if (out->cap < need) return fail(LS_ERR_INVALID, "ls_predict: out->cap %d < %ld", out->cap, need);
+  DeviceGuard guard(L->device);
+  return predict_impl(L, d_feature, batch, k, out->scores, out->mask, out->idx, out->count, out->cap, (cudaStream_t)stream);
+}
+
+int32_t ls_sparse_ffn_step(ls_layer* L, ls_layer* next, const float* d_x, float* d_x_out, int32_t batch, const ls_selection* sel,
+                           int32_t K, int32_t k_next, ls_selection* sel_next, ls_step_trace* trace, void* stream) {
+  LS_TRY(check_layer_call(L, batch, "ls_sparse_ffn_step"));
+  if (!d_x || !d_x_out || !sel || !sel->idx || !sel->count) return fail(LS_ERR_INVALID, "ls_sparse_ffn_step: x, x_out, sel->idx, sel->count are required");
+  if (K < 1 || K > 4096) return fail(LS_ERR_INVALID, "ls_sparse_ffn_step: n_chunks %d outside [1, 4096]", K);
+  if (sel->cap < 0 || sel->cap > L->max_sel) return fail(LS_ERR_INVALID, "ls_sparse_ffn_step: sel->cap %d outside [0, max_sel=%d]", sel->cap, L->max_sel);
+  if (next) {
+    if (next->d != L->d) return fail(LS_ERR_INVALID, "ls_sparse_ffn_step: next layer has a different d_model");
+    if (next->device != L->device) return fail(LS_ERR_INVALID, "ls_sparse_ffn_step: next layer is on another device");
+    if (batch > next->max_batch) return fail(LS_ERR_INVALID, "ls_sparse_ffn_step: batch exceeds next->max_batch");
+    if (!sel_next || !sel_next->idx || !sel_next->count) return fail(LS_ERR_INVALID, "ls_sparse_ffn_step: sel_next->idx and ->count are required with next");
+    if (k_next < 0 || k_next > next->F) return fail(LS_ERR_INVALID, "ls_sparse_ffn_step: k_next outside [0, d_ff_next]");
+    const long need = std::min<long>((long)batch * k_next, next->F);
+    if (sel_next->cap < need || need > next->max_sel) return fail(LS_ERR_INVALID, "ls_sparse_ffn_step: sel_next->cap or next->max_sel below %ld", need);
+  }
+  DeviceGuard guard(L->device);
+  cudaStream_t st = (cudaStream_t)stream;
+  const int d = L->d, B = batch;
+  const size_t bd = (size_t)B * d;
+  ls_step_trace tr{};
+  if (trace) tr = *trace;
+
+  ls::ls_step_init_kernel<<<std::min(64, (int)((bd + 255) / 256)), 256, 0, st>>>(d_x, L->b_down, L->xin, L->xt, tr.xtilde, B, d,
+                                                                               L->survive, L->nwords, nullptr);
+  LS_LAUNCHED();
+
+  const int32_t* exec_idx = sel->idx;
+  int first_miss_stage = K;
+  if (L->cache_rows > 0) {
+    // reserve the whole selection; residents run first, misses after (in the order their copies were issued)
+    int32_t nmiss = 0;
+    LS_TRY(ls::cache_reserve(L->cache, L->prio, L->F, sel->idx, sel->count, -1, 0, 0, sel->cap, nullptr, L->bundles, L->status, st,
+                             &nmiss, g_err, g_launches));
+    exec_idx = L->cache.d_exec_idx;
+    // stages made of residents only may start before the copies have landed
+    const int count = L->cache.last_nhit + L->cache.last_nmiss;
+    const int m = count > 0 ? (count + K - 1) / K : 1;
+    first_miss_stage = nmiss > 0 ? L->cache.last_nhit / m : K;
+  }
+  if (tr.exec_idx) {
+    ls::ls_copy_u32_kernel<<<8, 256, 0, st>>>(reinterpret_cast<const uint32_t*>(exec_idx), reinterpret_cast<uint32_t*>(tr.exec_idx),
+                                              sel->cap);
+    LS_LAUNCHED();
+  }
+
+  auto refine = [&](int j) -> int32_t {
+    if (!next) return LS_OK;
+    const bool last = (j == K);
+    uint32_t* mask_out = tr.refine_masks ? tr.refine_masks + (size_t)j * next->nwords : (last ? sel_next->mask : nullptr);
+    int32_t* idx_out = last ? sel_next->idx : next->tmp_idx;
+    int32_t* cnt_out = last ? sel_next->count : next->tmp_count;
+    const int cap = last ? sel_next->cap : next->max_sel;
+    LS_TRY(predict_impl(next, L->xt, B, k_next, last ? sel_next->scores : nullptr, mask_out, idx_out, cnt_out, cap, st));
+    if (last && tr.refine_masks && sel_next->mask) {
+      ls::ls_copy_u32_kernel<<<4, 256, 0, st>>>(mask_out, sel_next->mask, next->nwords);
+      LS_LAUNCHED();
+    }
+    if (tr.refine_counts) {
+      ls::ls_copy_u32_kernel<<<1, 32, 0, st>>>(reinterpret_cast<const uint32_t*>(cnt_out),
+                                               reinterpret_cast<uint32_t*>(tr.refine_counts + j), 1);
+      LS_LAUNCHED();
+    }
+    if (!last && next->cache_rows > 0 && next != L) {
+      // fetch rule: the first ceil(count (j+1)/(K+1)) ranks of C^(j) are admitted
+      int32_t nmiss = 0;
+      LS_TRY(ls::cache_reserve(next->cache, next->prio, next->F, idx_out, cnt_out, 0, j + 1, K + 1, next->max_sel, nullptr,
+                               next->bundles, next->status, st, &nmiss, g_err, g_launches));
+    }
+    return LS_OK;
+  };
+
+  LS_TRY(refine(0));
+  for (int c = 0; c < K; ++c) {
+    if (c == first_miss_stage) LS_TRY(ls::cache_wait(L->cache, st, g_err));
+    const int32_t splits = launch_stage_dispatch(L, B, exec_idx, sel->count, sel->cap, K, c, st);
+    if (splits < 0) return splits;
+    const bool last = (c + 1 == K);
+    ls::ls_stage_finalize_kernel<<<std::min(64, (int)((bd + 255) / 256)), 256, 0, st>>>(
+        L->ypart, splits, B, d, L->xt, tr.xtilde ? tr.xtilde + (size_t)(c + 1) * bd : nullptr, last ? d_x_out : nullptr);
+    LS_LAUNCHED();
+    LS_TRY(refine(c + 1));
+  }
+  if (tr.survive_mask) {
+    ls::ls_copy_u32_kernel<<<4, 256, 0, st>>>(L->survive, tr.survive_mask, L->nwords);
+    LS_LAUNCHED();
+  }
+  return LS_OK;
+}
+
+// ---- cache entry points ---------------------------------------------------------------------------------------------
+int32_t ls_cache_lookup(ls_layer* L, const int32_t* d_idx, int32_t n, int32_t* d_slot, int32_t* d_nhit, void* stream) {
+  if (!L || !d_idx || !d_slot) return fail(LS_ERR_INVALID, "ls_cache_lookup: NULL argument");
+  if (L->cache_rows == 0) return fail(LS_ERR_STATE, "ls_cache_lookup: layer has no cache");
+  if (n < 0 || n > L->max_sel) return fail(LS_ERR_INVALID, "ls_cache_lookup: n outside [0, max_sel]");
+  DeviceGuard guard(L->device);
+  return ls::cache_lookup(L->cache, L->F, d_idx, n, d_slot, d_nhit, L->status, (cudaStream_t)stream, g_err, g_launches);
+}
+
+int32_t ls_cache_reserve(ls_layer* L, const ls_selection* want, int32_t admit_ranks, const uint32_t* d_protect_mask, int32_t* h_nmiss,
+                         void* stream) {
+  if (!L || !want || !want->idx || !want->count) return fail(LS_ERR_INVALID, "ls_cache_reserve: NULL argument");
+  if (L->cache_rows == 0) return fail(LS_ERR_STATE, "ls_cache_reserve: layer has no cache");
+  if (want->cap < 0 || want->cap > L->max_sel) return fail(LS_ERR_INVALID, "ls_cache_reserve: want->cap outside [0, max_sel]");
+  DeviceGuard guard(L->device);
+  cudaStream_t st = (cudaStream_t)stream;
+  if (want->scores) LS_CUDA(cudaMemcpyAsync(L->prio, want->scores, (size_t)L->F * sizeof(double), cudaMemcpyDeviceToDevice, st));
+  return ls::cache_reserve(L->cache, L->prio, L->F, want->idx, want->count, admit_ranks < 0 ? -1 : admit_ranks, 0, 0, want->cap,
+                           d_protect_mask, L->bundles, L->status, st, h_nmiss, g_err, g_launches);
+}
+
+int32_t ls_cache_evict(ls_layer* L, int32_t min_free, const uint32_t* d_protect_mask, int32_t* d_evicted, int32_t* d_nevicted,
+                       void* stream) {
+  if (!L) return fail(LS_ERR_INVALID, "ls_cache_evict: NULL layer");
+  if (L->cache_rows == 0) return fail(LS_ERR_STATE, "ls_cache_evict: layer has no cache");
+  if (min_free < 0 || min_free > L->cache_rows) return fail(LS_ERR_INVALID, "ls_cache_evict: min_free outside [0, cache_rows]");
+  DeviceGuard guard(L->device);
+  return ls::cache_evict(L->cache, L->prio, L->F, min_free, d_protect_mask, d_evicted, d_nevicted, L->status, (cudaStream_t)stream,
+                         g_err, g_launches);
+}
+
+int32_t ls_cache_snapshot(ls_layer* L, uint32_t* d_resident_mask, void* stream) {
+  if (!L || !d_resident_mask) return fail(LS_ERR_INVALID, "ls_cache_snapshot: NULL argument");
+  if (L->cache_rows == 0) return fail(LS_ERR_STATE, "ls_cache_snapshot: layer has no cache");
+  DeviceGuard guard(L->device);
+  return ls::cache_snapshot(L->cache, L->F, d_resident_mask, (cudaStream_t)stream, g_err, g_launches);
+}
+
+int32_t ls_cache_wait(ls_layer* L, void* stream) {
+  if (!L) return fail(LS_ERR_INVALID, "ls_cache_wait: NULL layer");
+  if (L->cache_rows == 0) return fail(LS_ERR_STATE, "ls_cache_wait: layer has no cache");
+  DeviceGuard guard(L->device);
+  return ls::cache_wait(L->cache, (cudaStream_t)stream, g_err);
+}
+
+int32_t ls_cache_stats(ls_layer* L, ls_cache_stats_t* out) {
+  if (!L || !out) return fail(LS_ERR_INVALID, "ls_cache_stats: NULL argument");
+  if (L->cache_rows == 0) return fail(LS_ERR_STATE, "ls_cache_stats: layer has no cache");
+  out->hits = L->cache.hits; out->misses = L->cache.misses; out->evictions = L->cache.evictions;
+  out->h2d_bytes = L->cache.h2d_bytes; out->h2d_copies = L->cache.h2d_copies; out->resident = L->cache.resident;
+  return LS_OK;
+}
+
+}  // extern "C"
