@@ -226,6 +226,8 @@ int32_t create_impl(const ls_layer_desc* D, ls_layer* L) {
   // opt in to the large dynamic shared memory the kernels may ask for
   const int big = 200 * 1024;
   LS_CUDA(cudaFuncSetAttribute(ls::ls_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, big));
+  LS_CUDA(cudaFuncSetAttribute(ls::ls_cache_reserve_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, big));
+  LS_CUDA(cudaFuncSetAttribute(ls::ls_cache_evict_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, big));
   LS_CUDA(cudaFuncSetAttribute(ls::ls_scores_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024));
   LS_CUDA(cudaFuncSetAttribute(ls::ls_scores_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024));
 #define LS_ATTR_GU(WD, BT) \

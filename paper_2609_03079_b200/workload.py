@@ -30,6 +30,10 @@ from typing import Dict, List, Optional
 
 import numpy as np
 
+import threading
+
+_EIGH_LOCK = threading.Lock()
+
 T_GATE, T_UP, T_DOWN, T_PRED_NOISE, T_TOKENS = 0, 1, 2, 3, 4
 
 WEIGHT_STD = 0.02
@@ -165,7 +169,8 @@ def _svd_predictor(w_gate_f32: np.ndarray, rank: int, seed: int, layer: int, wdt
     else:
         torch.backends.cuda.matmul.allow_tf32 = False
     G = W.T @ W
-    evals, evecs = torch.linalg.eigh(G)
+    with _EIGH_LOCK:  # torch initialises its linear-algebra backend lazily and not thread-safely
+        evals, evecs = torch.linalg.eigh(G)
     V = evecs[:, -rank:].flip(1).contiguous()  # [d, r], descending singular value
     Bt = (W @ V).float().cpu().numpy()  # [F, r]
     A = V.float().cpu().numpy()

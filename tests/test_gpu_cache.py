@@ -91,7 +91,7 @@ def test_reserve_prefix_protect_capacity_and_evict():
     # wanted + protected beyond the capacity: refused, nothing changes
     before = snapshot(gl)
     with pytest.raises(ls.LeanStreamError) as e:
-        ls.ls_cache_reserve(gl, sel, admit_ranks=60, protect_mask=dev_tensor(protect.view(np.int32)))
+        ls.ls_cache_reserve(gl, sel, admit_ranks=100, protect_mask=dev_tensor(protect.view(np.int32)))
     assert e.value.code == ls.LS_ERR_CAPACITY
     assert snapshot(gl) == before
     assert ls.ls_layer_status(gl) == ls.LS_ERR_CAPACITY
