@@ -189,6 +189,16 @@ int32_t ls_cache_stats(ls_layer *layer, ls_cache_stats_t *host_out);
 int32_t ls_layer_status(ls_layer *layer, int32_t *host_status);
 
 /*
+ * Process-wide options (no counterpart in the paper).  LS_OPT_FUSED (default 1): steps that qualify (batch 1, layer and
+ * next layer fully resident, n_chunks <= 16, shared memory fits) run as ONE cooperative kernel per layer in which
+ * streaming and refinement overlap; 0 forces the stage-by-stage kernels, which compute the same thing.  With the fused
+ * kernel the partial outputs of different SMs are combined with floating-point atomics, so the low bits of x~^(j) may
+ * differ between two runs; the selected sets are always the exact top-k of the features that were actually produced.
+ */
+#define LS_OPT_FUSED 1
+int32_t ls_set_option(int32_t option, int32_t value);
+
+/*
  * Kernel timing for roofline accounting (no counterpart in the paper).  While enabled (process-wide, off by default)
  * the launches of the named kernel groups are bracketed by CUDA events on the stream they are launched on; not valid
  * during stream capture.  ls_timing_read() waits for the recorded events of one group, returns their number and summed

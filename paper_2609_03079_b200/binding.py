@@ -22,7 +22,7 @@ LS_NORM_RMS, LS_NORM_NONE = 0, 1
 EXPORTS = [
     "ls_layer_create", "ls_layer_destroy", "ls_predict", "ls_sparse_ffn_step", "ls_cache_lookup", "ls_cache_reserve",
     "ls_cache_evict", "ls_cache_snapshot", "ls_cache_wait", "ls_cache_stats", "ls_layer_status", "ls_kernel_launches",
-    "ls_last_error", "ls_version", "ls_timing_enable", "ls_timing_read",
+    "ls_last_error", "ls_version", "ls_timing_enable", "ls_timing_read", "ls_set_option",
 ]
 
 
@@ -82,6 +82,7 @@ def lib() -> C.CDLL:
         L.ls_cache_wait.argtypes = [C.c_void_p, C.c_void_p]
         L.ls_cache_stats.argtypes = [C.c_void_p, C.POINTER(ls_cache_stats_t)]
         L.ls_layer_status.argtypes = [C.c_void_p, C.POINTER(C.c_int32)]
+        L.ls_set_option.argtypes = [C.c_int32, C.c_int32]
         L.ls_timing_enable.argtypes = [C.c_int32]
         L.ls_timing_read.argtypes = [C.c_int32, C.POINTER(C.c_int64), C.POINTER(C.c_double)]
         L.ls_kernel_launches.restype = C.c_int64
@@ -293,3 +294,10 @@ def ls_timing_read(kind: int):
     n, ms = C.c_int64(0), C.c_double(0.0)
     _check(lib().ls_timing_read(kind, C.byref(n), C.byref(ms)))
     return n.value, ms.value
+
+
+LS_OPT_FUSED = 1
+
+
+def ls_set_option(option: int, value: int) -> None:
+    _check(lib().ls_set_option(option, value))

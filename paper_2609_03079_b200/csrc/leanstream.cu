@@ -11,12 +11,14 @@
 #include <vector>
 
 #include "ls_cache.cuh"
+#include "ls_fused.cuh"
 #include "ls_kernels.cuh"
 
 namespace {
 
 thread_local std::string g_err;
 std::atomic<int64_t> g_launches{0};
+std::atomic<int> g_opt_fused{1};
 
 int32_t fail(int32_t code, const char* fmt, ...) {
   char buf[512];
@@ -119,6 +121,18 @@ struct ls_layer {
   int* status = nullptr;                   // [1]
   int down_splits = 0;
 
+  // scratch of the fused per-layer kernel (see ls_fused.cuh for the zero-on-entry invariants)
+  float* fz_dacc = nullptr;           // [FZ_MAXK][d]
+  unsigned* fz_ctr = nullptr;         // stage_done[FZ_MAXK], fin, bar_count, bar_gen
+  double* fz_z = nullptr;             // [2][r] + sumsq[2] + range[2]
+  unsigned* fz_cnt = nullptr;         // [3][FZ_CNT_STRIDE]
+  unsigned long long* fz_bkey = nullptr;  // [3][FZ_NB * FZ_CAPB]
+  int32_t* fz_bidx = nullptr;
+  unsigned long long* fz_okey = nullptr;  // [3][F]
+  int32_t* fz_oidx = nullptr;
+  int32_t* fz_obin = nullptr;
+  unsigned long long* fz_range_obs = nullptr;  // [2]
+
   ls::CacheState cache;  // residency tables, pinned backing store, copy stream
 };
 
@@ -146,6 +160,8 @@ void free_layer(ls_layer* L) {
   cudaFree(L->bundles); cudaFree(L->b_gate); cudaFree(L->b_down); cudaFree(L->pred_at); cudaFree(L->pred_bt);
   cudaFree(L->pred_c); cudaFree(L->z); cudaFree(L->sumsq); cudaFree(L->scores); cudaFree(L->prio); cudaFree(L->cand_key);
   cudaFree(L->cand_idx); cudaFree(L->umask); cudaFree(L->tmp_idx); cudaFree(L->tmp_count); cudaFree(L->tmp_mask);
+  cudaFree(L->fz_dacc); cudaFree(L->fz_ctr); cudaFree(L->fz_z); cudaFree(L->fz_cnt); cudaFree(L->fz_bkey); cudaFree(L->fz_bidx);
+  cudaFree(L->fz_okey); cudaFree(L->fz_oidx); cudaFree(L->fz_obin); cudaFree(L->fz_range_obs);
   cudaFree(L->xin); cudaFree(L->xt); cudaFree(L->actv); cudaFree(L->ypart); cudaFree(L->survive); cudaFree(L->status);
   delete L;
 }
@@ -223,6 +239,26 @@ int32_t create_impl(const ls_layer_desc* D, ls_layer* L) {
   LS_CUDA(cudaMemset(L->status, 0, sizeof(int)));
   LS_CUDA(cudaMemset(L->prio, 0xff, F * sizeof(double)));  // NaN: ranks last until a prediction sets it
 
+  if (L->cache_rows == 0) {
+    LS_TRY(dalloc(&L->fz_dacc, (size_t)ls::FZ_MAXK * d));
+    LS_TRY(dalloc(&L->fz_ctr, (size_t)ls::FZ_MAXK + 8));
+    LS_TRY(dalloc(&L->fz_z, (size_t)2 * L->r + 8));
+    LS_TRY(dalloc(&L->fz_cnt, (size_t)3 * ls::FZ_CNT_STRIDE));
+    LS_TRY(dalloc(&L->fz_bkey, (size_t)3 * ls::FZ_NB * ls::FZ_CAPB));
+    LS_TRY(dalloc(&L->fz_bidx, (size_t)3 * ls::FZ_NB * ls::FZ_CAPB));
+    LS_TRY(dalloc(&L->fz_okey, 3 * F));
+    LS_TRY(dalloc(&L->fz_oidx, 3 * F));
+    LS_TRY(dalloc(&L->fz_obin, 3 * F));
+    LS_TRY(dalloc(&L->fz_range_obs, 2));
+    LS_CUDA(cudaMemset(L->fz_dacc, 0, (size_t)ls::FZ_MAXK * d * sizeof(float)));
+    LS_CUDA(cudaMemset(L->fz_ctr, 0, ((size_t)ls::FZ_MAXK + 8) * sizeof(unsigned)));
+    LS_CUDA(cudaMemset(L->fz_cnt, 0, (size_t)3 * ls::FZ_CNT_STRIDE * sizeof(unsigned)));
+    const double zr[8] = {0, 0, 0, 0, -1.0, 1.0, 0, 0};  // sumsq[2] unused slots, range = [-1, 1] until a launch observes one
+    LS_CUDA(cudaMemset(L->fz_z, 0, ((size_t)2 * L->r + 8) * sizeof(double)));
+    LS_CUDA(cudaMemcpy(L->fz_z + 2 * L->r, zr, sizeof zr, cudaMemcpyHostToDevice));
+    const unsigned long long ro[2] = {0xffffffffffffffffULL, 0ULL};
+    LS_CUDA(cudaMemcpy(L->fz_range_obs, ro, sizeof ro, cudaMemcpyHostToDevice));
+  }
   // opt in to the large dynamic shared memory the kernels may ask for
   const int big = 200 * 1024;
   LS_CUDA(cudaFuncSetAttribute(ls::ls_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, big));
@@ -234,8 +270,78 @@ int32_t create_impl(const ls_layer_desc* D, ls_layer* L) {
   LS_CUDA(cudaFuncSetAttribute(ls::ls_gateup_kernel<WD, BT>, cudaFuncAttributeMaxDynamicSharedMemorySize, big))
   LS_ATTR_GU(0, 1); LS_ATTR_GU(0, 4); LS_ATTR_GU(0, 8); LS_ATTR_GU(1, 1); LS_ATTR_GU(1, 4); LS_ATTR_GU(1, 8);
 #undef LS_ATTR_GU
+#define LS_ATTR_FZ(WD, CPT) \
+  LS_CUDA(cudaFuncSetAttribute(ls::ls_fused_step_kernel<WD, CPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024))
+  LS_ATTR_FZ(0, 1); LS_ATTR_FZ(0, 2); LS_ATTR_FZ(0, 3); LS_ATTR_FZ(0, 4);
+  LS_ATTR_FZ(1, 1); LS_ATTR_FZ(1, 2); LS_ATTR_FZ(1, 3); LS_ATTR_FZ(1, 4);
+#undef LS_ATTR_FZ
   LS_CUDA(cudaDeviceSynchronize());
   return LS_OK;
+}
+
+// ---- the fused per-layer kernel: eligibility and launch ---------------------------------------------------------------
+bool fused_eligible(const ls_layer* L, const ls_layer* next, int batch, int K) {
+  if (!g_opt_fused.load(std::memory_order_relaxed)) return false;
+  if (batch != 1 || L->cache_rows != 0 || (next && next->cache_rows != 0)) return false;
+  if (K > ls::FZ_MAXK) return false;
+  if ((L->d >> 3) > ls::FZ_STREAM_THREADS * 4) return false;
+  const ls::FusedSmemLayout lay = ls::fused_layout(L->d, L->gated ? 2 : 1, next ? next->r : 0, next ? next->F : 0, L->sm_count, next ? 1 : 0);
+  if (lay.total > 226 * 1024) return false;
+  if (next && lay.per > 4096) return false;
+  return true;
+}
+
+template <int WD>
+int32_t launch_fused_cpt(int cpt, const ls::FusedArgs& a, int grid, size_t smem, cudaStream_t st) {
+  void* params[] = {const_cast<ls::FusedArgs*>(&a)};
+  const void* fn = nullptr;
+  switch (cpt) {
+    case 1: fn = (const void*)ls::ls_fused_step_kernel<WD, 1>; break;
+    case 2: fn = (const void*)ls::ls_fused_step_kernel<WD, 2>; break;
+    case 3: fn = (const void*)ls::ls_fused_step_kernel<WD, 3>; break;
+    default: fn = (const void*)ls::ls_fused_step_kernel<WD, 4>; break;
+  }
+  KernelTimer timer(LS_TIMED_FUSED, st);
+  LS_CUDA(cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(ls::FZ_THREADS), params, smem, st));
+  LS_LAUNCHED();
+  return LS_OK;
+}
+
+int32_t fused_step(ls_layer* L, ls_layer* next, const float* d_x, float* d_x_out, const ls_selection* sel, int K, int k_next,
+                   ls_selection* sel_next, const ls_step_trace& tr, cudaStream_t st) {
+  ls::FusedArgs a{};
+  a.bundles = L->bundles; a.n_mat = L->n_mat; a.gated = L->gated; a.b_gate = L->b_gate; a.b_down = L->b_down;
+  a.d = L->d; a.F = L->F; a.norm = L->norm; a.eps = L->eps;
+  a.x = d_x; a.x_out = d_x_out;
+  a.sel_idx = sel->idx; a.sel_count = sel->count; a.sel_cap = sel->cap; a.K = K;
+  a.dacc = L->fz_dacc; a.stage_done = L->fz_ctr; a.fin = L->fz_ctr + ls::FZ_MAXK;
+  a.bar_count = L->fz_ctr + ls::FZ_MAXK + 1; a.bar_gen = L->fz_ctr + ls::FZ_MAXK + 2;
+  a.status = L->status;
+  a.has_next = next ? 1 : 0;
+  const int nw_next = next ? next->nwords : 0;
+  if (next) {
+    a.At = next->pred_at; a.Bt = next->pred_bt; a.pc = next->pred_c;
+    a.r = next->r; a.Fn = next->F; a.norm_n = next->norm; a.eps_n = next->eps; a.k_next = k_next;
+    a.z = next->fz_z; a.sumsq = next->fz_z + 2 * next->r; a.range = next->fz_z + 2 * next->r + 4;
+    a.cnt = next->fz_cnt; a.bkey = next->fz_bkey; a.bidx = next->fz_bidx; a.okey = next->fz_okey; a.oidx = next->fz_oidx;
+    a.obin = next->fz_obin; a.range_obs = next->fz_range_obs; a.tmp_idx = next->tmp_idx;
+    a.next_idx = sel_next->idx; a.next_count = sel_next->count; a.next_mask = sel_next->mask; a.next_scores = sel_next->scores;
+    a.next_prio = next->prio; a.next_cap = sel_next->cap;
+    if (sel_next->mask) LS_CUDA(cudaMemsetAsync(sel_next->mask, 0, (size_t)nw_next * 4, st));
+  }
+  a.tr_xtilde = tr.xtilde; a.tr_masks = next ? tr.refine_masks : nullptr; a.tr_counts = next ? tr.refine_counts : nullptr;
+  a.tr_survive = tr.survive_mask;
+  if (a.tr_masks) LS_CUDA(cudaMemsetAsync(a.tr_masks, 0, (size_t)(K + 1) * nw_next * 4, st));
+  if (a.tr_survive) LS_CUDA(cudaMemsetAsync(a.tr_survive, 0, (size_t)L->nwords * 4, st));
+  if (tr.exec_idx) {
+    ls::ls_copy_u32_kernel<<<8, 256, 0, st>>>(reinterpret_cast<const uint32_t*>(sel->idx), reinterpret_cast<uint32_t*>(tr.exec_idx),
+                                              sel->cap);
+    LS_LAUNCHED();
+  }
+  const ls::FusedSmemLayout lay = ls::fused_layout(L->d, L->gated ? 2 : 1, a.r, a.Fn, L->sm_count, a.has_next);
+  const int cpt = ((L->d >> 3) + ls::FZ_STREAM_THREADS - 1) / ls::FZ_STREAM_THREADS;
+  if (L->wd == 0) return launch_fused_cpt<0>(cpt, a, L->sm_count, lay.total, st);
+  return launch_fused_cpt<1>(cpt, a, L->sm_count, lay.total, st);
 }
 
 // ---- speculate / refine: latent -> scores -> top-k (-> union for batch > 1) ------------------------------------------
@@ -345,6 +451,14 @@ size_t ls_last_error(char* buf, size_t n) {
 }
 
 int64_t ls_kernel_launches(void) { return g_launches.load(); }
+
+int32_t ls_set_option(int32_t option, int32_t value) {
+  if (option == LS_OPT_FUSED) {
+    g_opt_fused.store(value ? 1 : 0);
+    return LS_OK;
+  }
+  return fail(LS_ERR_INVALID, "ls_set_option: unknown option %d", option);
+}
 
 int32_t ls_timing_enable(int32_t on) {
   g_timing.store(on ? 1 : 0);
@@ -456,6 +570,8 @@ int32_t ls_sparse_ffn_step(ls_layer* L, ls_layer* next, const float* d_x, float*
   const size_t bd = (size_t)B * d;
   ls_step_trace tr{};
   if (trace) tr = *trace;
+
+  if (fused_eligible(L, next, B, K)) return fused_step(L, next, d_x, d_x_out, sel, K, k_next, sel_next, tr, st);
 
   ls::ls_step_init_kernel<<<std::min(64, (int)((bd + 255) / 256)), 256, 0, st>>>(d_x, L->b_down, L->xin, L->xt, tr.xtilde, B, d,
                                                                                L->survive, L->nwords, nullptr);

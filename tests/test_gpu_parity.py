@@ -14,6 +14,14 @@ pytestmark = pytest.mark.gpu
 DEV = 0
 
 
+@pytest.fixture(autouse=True, params=[1, 0], ids=["fused", "staged"])
+def kernel_path(request):
+    """Every test runs on both implementations of the step: the fused per-layer kernel and the stage-by-stage kernels."""
+    ls.ls_set_option(ls.LS_OPT_FUSED, request.param)
+    yield request.param
+    ls.ls_set_option(ls.LS_OPT_FUSED, 1)
+
+
 def dev_tensor(a):
     return torch.from_numpy(np.ascontiguousarray(a)).cuda(DEV)
 
