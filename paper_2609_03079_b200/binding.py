@@ -63,7 +63,7 @@ def lib() -> C.CDLL:
     """The loaded shared library (built in-tree on first use when nvcc is available)."""
     global _lib
     if _lib is None:
-        path = _build.LIB_PATH
+        path = os.environ.get("LEANSTREAM_LIB") or _build.LIB_PATH  # the override names another build of the same library
         if not os.path.exists(path):
             path = _build.build_library()
         try:

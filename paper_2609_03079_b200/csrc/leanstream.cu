@@ -280,15 +280,32 @@ int32_t create_impl(const ls_layer_desc* D, ls_layer* L) {
 }
 
 // ---- the fused per-layer kernel: eligibility and launch ---------------------------------------------------------------
-bool fused_eligible(const ls_layer* L, const ls_layer* next, int batch, int K) {
+// Shared-memory plan of the fused kernel: as many ring stages as fit beside the predictor operands.
+bool fused_plan(const ls_layer* L, const ls_layer* next, ls::FusedSmemLayout* out) {
+  const size_t budget = 226 * 1024;
+  const int n_in = L->gated ? 2 : 1;
+  const int r = next ? next->r : 0, Fn = next ? next->F : 0, hn = next ? 1 : 0;
+  for (int dn = ls::FZ_MAX_DEPTH / 2; dn >= 2; --dn) {
+    for (int gu = ls::FZ_MAX_DEPTH; gu >= 2; --gu) {
+      if (gu < dn) break;
+      const ls::FusedSmemLayout lay = ls::fused_layout(L->d, n_in, r, Fn, L->sm_count, hn, gu, dn);
+      if (lay.total <= budget) {
+        if (out) *out = lay;
+        return true;
+      }
+    }
+  }
+  return false;
+}
+
+bool fused_eligible(const ls_layer* L, const ls_layer* next, int batch, int K, int sel_cap) {
   if (!g_opt_fused.load(std::memory_order_relaxed)) return false;
   if (batch != 1 || L->cache_rows != 0 || (next && next->cache_rows != 0)) return false;
   if (K > ls::FZ_MAXK) return false;
+  if ((sel_cap + L->sm_count - 1) / L->sm_count > ls::FZ_MAX_MINE) return false;
   if ((L->d >> 3) > ls::FZ_STREAM_THREADS * 4) return false;
-  const ls::FusedSmemLayout lay = ls::fused_layout(L->d, L->gated ? 2 : 1, next ? next->r : 0, next ? next->F : 0, L->sm_count, next ? 1 : 0);
-  if (lay.total > 226 * 1024) return false;
-  if (next && lay.per > 4096) return false;
-  return true;
+  if (next && (next->r > 4 * ls::FZ_PRED_THREADS)) return false;
+  return fused_plan(L, next, nullptr);
 }
 
 template <int WD>
@@ -315,7 +332,7 @@ int32_t fused_step(ls_layer* L, ls_layer* next, const float* d_x, float* d_x_out
   a.x = d_x; a.x_out = d_x_out;
   a.sel_idx = sel->idx; a.sel_count = sel->count; a.sel_cap = sel->cap; a.K = K;
   a.dacc = L->fz_dacc; a.stage_done = L->fz_ctr; a.fin = L->fz_ctr + ls::FZ_MAXK;
-  a.bar_count = L->fz_ctr + ls::FZ_MAXK + 1; a.bar_gen = L->fz_ctr + ls::FZ_MAXK + 2;
+  a.bar_count = reinterpret_cast<unsigned long long*>(L->fz_ctr + ls::FZ_MAXK + 2);  // 8-byte aligned (FZ_MAXK is even)
   a.status = L->status;
   a.has_next = next ? 1 : 0;
   const int nw_next = next ? next->nwords : 0;
@@ -338,7 +355,9 @@ int32_t fused_step(ls_layer* L, ls_layer* next, const float* d_x, float* d_x_out
                                               sel->cap);
     LS_LAUNCHED();
   }
-  const ls::FusedSmemLayout lay = ls::fused_layout(L->d, L->gated ? 2 : 1, a.r, a.Fn, L->sm_count, a.has_next);
+  ls::FusedSmemLayout lay{};
+  if (!fused_plan(L, next, &lay)) return fail(LS_ERR_STATE, "fused step: shared memory plan failed");
+  a.gu_depth = lay.gu_depth; a.dn_depth = lay.dn_depth;
   const int cpt = ((L->d >> 3) + ls::FZ_STREAM_THREADS - 1) / ls::FZ_STREAM_THREADS;
   if (L->wd == 0) return launch_fused_cpt<0>(cpt, a, L->sm_count, lay.total, st);
   return launch_fused_cpt<1>(cpt, a, L->sm_count, lay.total, st);
@@ -451,6 +470,12 @@ size_t ls_last_error(char* buf, size_t n) {
 }
 
 int64_t ls_kernel_launches(void) { return g_launches.load(); }
+
+#ifdef LS_FZ_TIMING
+int32_t ls_debug_read_timing(long long* host, int32_t n) {
+  return cudaMemcpyFromSymbol(host, ls::g_fz_timing, (size_t)n * sizeof(long long)) == cudaSuccess ? LS_OK : LS_ERR_CUDA;
+}
+#endif
 
 int32_t ls_set_option(int32_t option, int32_t value) {
   if (option == LS_OPT_FUSED) {
@@ -571,7 +596,7 @@ int32_t ls_sparse_ffn_step(ls_layer* L, ls_layer* next, const float* d_x, float*
   ls_step_trace tr{};
   if (trace) tr = *trace;
 
-  if (fused_eligible(L, next, B, K)) return fused_step(L, next, d_x, d_x_out, sel, K, k_next, sel_next, tr, st);
+  if (fused_eligible(L, next, B, K, sel->cap)) return fused_step(L, next, d_x, d_x_out, sel, K, k_next, sel_next, tr, st);
 
   ls::ls_step_init_kernel<<<std::min(64, (int)((bd + 255) / 256)), 256, 0, st>>>(d_x, L->b_down, L->xin, L->xt, tr.xtilde, B, d,
                                                                                L->survive, L->nwords, nullptr);
