@@ -175,6 +175,7 @@ def run_ours(args):
     import torch.distributed as dist
 
     from paper_2609_03079_b200 import binding as ls
+    from paper_2609_03079_b200 import replicas
     from paper_2609_03079_b200 import workload as wl
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -209,7 +210,7 @@ def run_ours(args):
     t_build = time.perf_counter() - t_build
 
     n_tok = max(spec.n_tokens, 1)
-    X0_host = torch.from_numpy(wl.make_tokens(spec, n_tok, stream=rank)).pin_memory()
+    X0_host = torch.from_numpy(wl.make_tokens(spec, n_tok, stream=replicas.stream_of_rank(rank))).pin_memory()
     X0 = X0_host.to(dev)
     x_buf = torch.zeros(1, d, dtype=torch.float32, device=dev)
     out_host = torch.zeros(1, d, dtype=torch.float32).pin_memory()
@@ -245,29 +246,25 @@ def run_ours(args):
                 out_host.copy_(x_buf, non_blocking=True)
 
     def timed(n_steps, e2e):
+        """(slowest rank's milliseconds for n_steps, steps of all ranks): barrier + synchronize on both sides."""
         loop(args.warmup, e2e)
         torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
+        replicas.barrier()
         torch.cuda.synchronize()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record()
         loop(n_steps, e2e)
         b.record()
         torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
-        ms = torch.tensor([a.elapsed_time(b)], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-        return float(ms.item())
+        replicas.barrier()
+        return replicas.aggregate(a.elapsed_time(b), n_steps, dev)
 
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    ms_total = timed(args.steps, False)
+    ms_total, steps_total = timed(args.steps, False)
     clocks = sampler.stop() if rank == 0 else None
-    ms_e2e = timed(args.steps, True)
+    ms_e2e, steps_e2e = timed(args.steps, True)
     status = [ls.ls_layer_status(L) for L in layers]
     assert all(s == 0 for s in status), f"device status {status}"
 
@@ -281,6 +278,7 @@ def run_ours(args):
             decode_token()
         torch.cuda.synchronize()
         ls.ls_timing_enable(False)
+        n_fz, ms_fz = ls.ls_timing_read(ls.LS_TIMED_FUSED)
         n_gu, ms_gu = ls.ls_timing_read(ls.LS_TIMED_GATEUP)
         n_dn, ms_dn = ls.ls_timing_read(ls.LS_TIMED_DOWN)
         n_pr, ms_pr = ls.ls_timing_read(ls.LS_TIMED_PREDICT)
@@ -296,18 +294,24 @@ def run_ours(args):
             surv.append(int(np.unpackbits(m.view(np.uint8)).sum()))
         k_surv = float(np.mean(surv))
         row = spec.row_bytes
-        gu_bytes_per_launch = (k / K) * spec.n_in * row
         active_bytes_layer = k * spec.n_in * row + k_surv * row
         ms_step = ms_total / args.steps
         us_layer = ms_step * 1e3 / n_layers
         active_gbs = active_bytes_layer / (us_layer * 1e-6) / 1e9
-        gu_us = ms_gu / max(n_gu, 1) * 1e3
-        gu_gbs = gu_bytes_per_launch / (gu_us * 1e-6) / 1e9 if n_gu else None
-        traffic = None
+        traffic_db = {}
         tp = os.path.join(ROOT, "profiles", "traffic.json")
         if os.path.exists(tp):
             with open(tp) as f:
-                traffic = json.load(f).get("gateup_dram_bytes_per_launch")
+                traffic_db = json.load(f)
+        if n_fz:
+            # the whole layer step is one kernel: its algorithmic bytes are the active-neuron bytes of the layer
+            kname, bytes_launch, us_launch, n_timed = "ls_fused_step_kernel", active_bytes_layer, ms_fz / n_fz * 1e3, n_fz
+            traffic = traffic_db.get("fused_dram_bytes_per_launch")
+        else:
+            kname, bytes_launch, n_timed = "ls_gateup_kernel", (k / K) * spec.n_in * row, n_gu
+            us_launch = ms_gu / max(n_gu, 1) * 1e3
+            traffic = traffic_db.get("gateup_dram_bytes_per_launch")
+        k_gbs = bytes_launch / (us_launch * 1e-6) / 1e9 if n_timed else None
 
         # ---- CPU baseline: the oracle as it stands on a bounded sample
         t0 = time.perf_counter()
@@ -318,7 +322,7 @@ def run_ours(args):
         cpu_val = 1.0 / (float(np.mean(times)) * n_layers)
 
         line = {
-            "metric": METRIC, "value": args.steps * world / (ms_total * 1e-3), "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+            "metric": METRIC, "value": steps_total / (ms_total * 1e-3), "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16 weights, f32 accumulate, f64 predictor scores", "data": "synthetic",
             "config": {"workload": spec.name, "n_layers": n_layers, "d_model": d, "d_ff": spec.d_ff, "pred_rank": spec.rank, "k": k,
@@ -327,13 +331,14 @@ def run_ours(args):
                        "cuda_graph": graph is not None},
             "us_per_layer": us_layer, "active_bytes_per_layer": active_bytes_layer, "k_surviving_mean": k_surv,
             "active_gbs": active_gbs, "active_frac_of_hbm_peak": active_gbs / peaks["hbm_gbs"],
-            "roofline": {"bound": "hbm", "kernel": "ls_gateup_kernel", "achieved": gu_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                         "frac": (gu_gbs / peaks["hbm_gbs"]) if gu_gbs else None, "traffic": traffic, "peak_kind": peak_kind,
-                         "bytes_per_launch": gu_bytes_per_launch, "us_per_launch": gu_us, "launches_timed": n_gu,
-                         "down_us_per_launch": ms_dn / max(n_dn, 1) * 1e3, "predict_us_per_eval": ms_pr / max(n_pr, 1) * 1e3},
+            "roofline": {"bound": "hbm", "kernel": kname, "achieved": k_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": (k_gbs / peaks["hbm_gbs"]) if k_gbs else None, "traffic": traffic, "peak_kind": peak_kind,
+                         "bytes_per_launch": bytes_launch, "us_per_launch": us_launch, "launches_timed": n_timed,
+                         "staged_path": {"gateup_us": ms_gu / max(n_gu, 1) * 1e3, "down_us": ms_dn / max(n_dn, 1) * 1e3,
+                                         "predict_us": ms_pr / max(n_pr, 1) * 1e3} if n_gu else None},
             "cpu_baseline": {"value": cpu_val, "unit": "tokens/s", "cores": blas_threads(), "kind": "oracle",
                              "sample": f"{len(times)} layer-steps on {len(arrays)} distinct layers, scaled to {n_layers} layers; {cpu_wall:.1f} s"},
-            "e2e": {"value": args.steps * world / (ms_e2e * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": d * 4, "d2h_bytes_per_step": d * 4},
+            "e2e": {"value": steps_e2e / (ms_e2e * 1e-3), "unit": "tokens/s", "h2d_bytes_per_step": d * 4, "d2h_bytes_per_step": d * 4},
             "gpu_launches": launches_per_token * args.steps, "launches_per_token": launches_per_token,
             "clocks": clocks, "build_s": t_build,
         }

@@ -123,12 +123,12 @@ struct ls_layer {
 
   // scratch of the fused per-layer kernel (see ls_fused.cuh for the zero-on-entry invariants)
   float* fz_dacc = nullptr;           // [FZ_MAXK][d]
-  unsigned* fz_ctr = nullptr;         // stage_done[FZ_MAXK], fin, bar_count, bar_gen
-  double* fz_z = nullptr;             // [2][r] + sumsq[2] + range[2]
-  unsigned* fz_cnt = nullptr;         // [3][FZ_CNT_STRIDE]
-  unsigned long long* fz_bkey = nullptr;  // [3][FZ_NB * FZ_CAPB]
+  unsigned* fz_ctr = nullptr;         // fin, (pad), barrier counter (64-bit)
+  double* fz_z = nullptr;             // [FZ_MAXE][r] latents, [FZ_MAXE] sums of squares, [2] binning range
+  unsigned* fz_cnt = nullptr;         // [FZ_MAXE][FZ_CNT_STRIDE]
+  unsigned long long* fz_bkey = nullptr;  // [FZ_MAXE][FZ_NB * FZ_CAPB]
   int32_t* fz_bidx = nullptr;
-  unsigned long long* fz_okey = nullptr;  // [3][F]
+  unsigned long long* fz_okey = nullptr;  // [FZ_MAXE][F]
   int32_t* fz_oidx = nullptr;
   int32_t* fz_obin = nullptr;
   unsigned long long* fz_range_obs = nullptr;  // [2]
@@ -241,21 +241,22 @@ int32_t create_impl(const ls_layer_desc* D, ls_layer* L) {
 
   if (L->cache_rows == 0) {
     LS_TRY(dalloc(&L->fz_dacc, (size_t)ls::FZ_MAXK * d));
-    LS_TRY(dalloc(&L->fz_ctr, (size_t)ls::FZ_MAXK + 8));
-    LS_TRY(dalloc(&L->fz_z, (size_t)2 * L->r + 8));
-    LS_TRY(dalloc(&L->fz_cnt, (size_t)3 * ls::FZ_CNT_STRIDE));
-    LS_TRY(dalloc(&L->fz_bkey, (size_t)3 * ls::FZ_NB * ls::FZ_CAPB));
-    LS_TRY(dalloc(&L->fz_bidx, (size_t)3 * ls::FZ_NB * ls::FZ_CAPB));
-    LS_TRY(dalloc(&L->fz_okey, 3 * F));
-    LS_TRY(dalloc(&L->fz_oidx, 3 * F));
-    LS_TRY(dalloc(&L->fz_obin, 3 * F));
+    const size_t NE = ls::FZ_MAXE;
+    LS_TRY(dalloc(&L->fz_ctr, (size_t)8));
+    LS_TRY(dalloc(&L->fz_z, NE * L->r + NE + 8));
+    LS_TRY(dalloc(&L->fz_cnt, NE * ls::FZ_CNT_STRIDE));
+    LS_TRY(dalloc(&L->fz_bkey, NE * ls::FZ_NB * ls::FZ_CAPB));
+    LS_TRY(dalloc(&L->fz_bidx, NE * ls::FZ_NB * ls::FZ_CAPB));
+    LS_TRY(dalloc(&L->fz_okey, NE * F));
+    LS_TRY(dalloc(&L->fz_oidx, NE * F));
+    LS_TRY(dalloc(&L->fz_obin, NE * F));
     LS_TRY(dalloc(&L->fz_range_obs, 2));
     LS_CUDA(cudaMemset(L->fz_dacc, 0, (size_t)ls::FZ_MAXK * d * sizeof(float)));
-    LS_CUDA(cudaMemset(L->fz_ctr, 0, ((size_t)ls::FZ_MAXK + 8) * sizeof(unsigned)));
-    LS_CUDA(cudaMemset(L->fz_cnt, 0, (size_t)3 * ls::FZ_CNT_STRIDE * sizeof(unsigned)));
-    const double zr[8] = {0, 0, 0, 0, -1.0, 1.0, 0, 0};  // sumsq[2] unused slots, range = [-1, 1] until a launch observes one
-    LS_CUDA(cudaMemset(L->fz_z, 0, ((size_t)2 * L->r + 8) * sizeof(double)));
-    LS_CUDA(cudaMemcpy(L->fz_z + 2 * L->r, zr, sizeof zr, cudaMemcpyHostToDevice));
+    LS_CUDA(cudaMemset(L->fz_ctr, 0, 8 * sizeof(unsigned)));
+    LS_CUDA(cudaMemset(L->fz_cnt, 0, NE * ls::FZ_CNT_STRIDE * sizeof(unsigned)));
+    const double zr[2] = {-1.0, 1.0};  // binning range until a launch has observed one
+    LS_CUDA(cudaMemset(L->fz_z, 0, (NE * L->r + NE + 8) * sizeof(double)));
+    LS_CUDA(cudaMemcpy(L->fz_z + NE * L->r + NE, zr, sizeof zr, cudaMemcpyHostToDevice));
     const unsigned long long ro[2] = {0xffffffffffffffffULL, 0ULL};
     LS_CUDA(cudaMemcpy(L->fz_range_obs, ro, sizeof ro, cudaMemcpyHostToDevice));
   }
@@ -304,7 +305,6 @@ bool fused_eligible(const ls_layer* L, const ls_layer* next, int batch, int K, i
   if (K > ls::FZ_MAXK) return false;
   if ((sel_cap + L->sm_count - 1) / L->sm_count > ls::FZ_MAX_MINE) return false;
   if ((L->d >> 3) > ls::FZ_STREAM_THREADS * 4) return false;
-  if (next && (next->r > 4 * ls::FZ_PRED_THREADS)) return false;
   return fused_plan(L, next, nullptr);
 }
 
@@ -331,15 +331,15 @@ int32_t fused_step(ls_layer* L, ls_layer* next, const float* d_x, float* d_x_out
   a.d = L->d; a.F = L->F; a.norm = L->norm; a.eps = L->eps;
   a.x = d_x; a.x_out = d_x_out;
   a.sel_idx = sel->idx; a.sel_count = sel->count; a.sel_cap = sel->cap; a.K = K;
-  a.dacc = L->fz_dacc; a.stage_done = L->fz_ctr; a.fin = L->fz_ctr + ls::FZ_MAXK;
-  a.bar_count = reinterpret_cast<unsigned long long*>(L->fz_ctr + ls::FZ_MAXK + 2);  // 8-byte aligned (FZ_MAXK is even)
+  a.dacc = L->fz_dacc; a.fin = L->fz_ctr;
+  a.bar_count = reinterpret_cast<unsigned long long*>(L->fz_ctr + 2);  // 8-byte aligned
   a.status = L->status;
   a.has_next = next ? 1 : 0;
   const int nw_next = next ? next->nwords : 0;
   if (next) {
     a.At = next->pred_at; a.Bt = next->pred_bt; a.pc = next->pred_c;
     a.r = next->r; a.Fn = next->F; a.norm_n = next->norm; a.eps_n = next->eps; a.k_next = k_next;
-    a.z = next->fz_z; a.sumsq = next->fz_z + 2 * next->r; a.range = next->fz_z + 2 * next->r + 4;
+    a.z = next->fz_z; a.sumsq = next->fz_z + (size_t)ls::FZ_MAXE * next->r; a.range = a.sumsq + ls::FZ_MAXE;
     a.cnt = next->fz_cnt; a.bkey = next->fz_bkey; a.bidx = next->fz_bidx; a.okey = next->fz_okey; a.oidx = next->fz_oidx;
     a.obin = next->fz_obin; a.range_obs = next->fz_range_obs; a.tmp_idx = next->tmp_idx;
     a.next_idx = sel_next->idx; a.next_count = sel_next->count; a.next_mask = sel_next->mask; a.next_scores = sel_next->scores;

@@ -138,6 +138,20 @@ def test_predict_exact_ties_lower_index_first(tiny):
     gt.close()
 
 
+def test_refined_sets_with_exact_ties_in_the_next_layer(tiny):
+    """The next layer has duplicated predictor columns: its refined order must still put the lower index first."""
+    spec, la, OL, gl, toks = tiny
+    pairs = [(5, 700), (123, 124), (1000, 3), (64, 65), (8, 1016)]
+    lt = wl.tied_duplicate_layer(la, pairs)
+    gt = ls.ls_layer_create(lt, DEV)
+    OT = orc.OracleLayer.from_arrays(lt)
+    stats = {}
+    for x in toks[:6]:
+        run_step_and_compare(gl, gt, OL, OT, x, spec.k, 8, 1024, stats)  # k_next = d_ff: the full order is compared
+    assert stats.get("band", 0) == 0
+    gt.close()
+
+
 def test_predict_degenerate_all_equal_scores():
     """Zero predictor and constant bias: every score equal, so the order is the index order."""
     spec, la = custom_arrays(11, 64, 300, 8)
