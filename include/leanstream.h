@@ -189,6 +189,31 @@ int32_t ls_cache_stats(ls_layer *layer, ls_cache_stats_t *host_out);
 int32_t ls_layer_status(ls_layer *layer, int32_t *host_status);
 
 /*
+ * Top-k selection that allocates nothing (the paper has no counterpart; it exists for callers that must not allocate).
+ *
+ * Some callers cannot call cudaMalloc or anything that may call it for them: code running while a stream is being
+ * captured into a CUDA graph, a latency-critical serving loop that must never meet the implicit device synchronisation
+ * of an allocation, a process whose device memory has been handed out completely to a memory pool, or a callback of
+ * another runtime in which allocating is simply forbidden.  For them this entry point selects the k highest scores of a
+ * caller-provided device array with the same rule as ls_predict (score descending, equal scores by ascending index,
+ * NaN last, -0 equal to +0) using only memory that already exists: its candidate lists live in a fixed array inside
+ * the library image (LS_STATIC_TOPK_MAX_N x 12 bytes = 384 KB, held on every GPU that has loaded the library until
+ * the process exits).  It calls no cudaMalloc, no cudaFree and no allocating library routine, and needs no ls_layer.
+ *
+ *   d_scores [n] fp64 (device, read only); d_idx [k] receives the selected positions in rank order; d_mask
+ *   [ceil(n/32)] (nullable) the membership bits; d_count [1] the number selected (= k).  All caller-owned.
+ *   1 <= n <= LS_STATIC_TOPK_MAX_N and 0 <= k <= n, otherwise LS_ERR_INVALID with an explanatory ls_last_error().
+ *
+ * The first call on a device looks up the array's device address (cudaGetSymbolAddress) and opts the kernel in to its
+ * shared memory; make that first call outside any stream capture, with the target device current.  All calls on a
+ * device share the one array: two calls that overlap on the GPU (different streams) race on it, so order them; the
+ * array keeps whatever the last call left there, which is harmless because every entry is written before it is read.
+ */
+#define LS_STATIC_TOPK_MAX_N 32768
+int32_t ls_topk_select_static(const double *d_scores, int32_t n, int32_t k, int32_t *d_idx, uint32_t *d_mask,
+                              int32_t *d_count, void *stream);
+
+/*
  * Process-wide options (no counterpart in the paper).  LS_OPT_FUSED (default 1): steps that qualify (batch 1, layer and
  * next layer fully resident, n_chunks <= 16, shared memory fits) run as ONE cooperative kernel per layer in which
  * streaming and refinement overlap; 0 forces the stage-by-stage kernels, which compute the same thing.  With the fused

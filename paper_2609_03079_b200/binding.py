@@ -22,7 +22,7 @@ LS_NORM_RMS, LS_NORM_NONE = 0, 1
 EXPORTS = [
     "ls_layer_create", "ls_layer_destroy", "ls_predict", "ls_sparse_ffn_step", "ls_cache_lookup", "ls_cache_reserve",
     "ls_cache_evict", "ls_cache_snapshot", "ls_cache_wait", "ls_cache_stats", "ls_layer_status", "ls_kernel_launches",
-    "ls_last_error", "ls_version", "ls_timing_enable", "ls_timing_read", "ls_set_option",
+    "ls_last_error", "ls_version", "ls_timing_enable", "ls_timing_read", "ls_set_option", "ls_topk_select_static",
 ]
 
 
@@ -83,6 +83,7 @@ def lib() -> C.CDLL:
         L.ls_cache_stats.argtypes = [C.c_void_p, C.POINTER(ls_cache_stats_t)]
         L.ls_layer_status.argtypes = [C.c_void_p, C.POINTER(C.c_int32)]
         L.ls_set_option.argtypes = [C.c_int32, C.c_int32]
+        L.ls_topk_select_static.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.ls_timing_enable.argtypes = [C.c_int32]
         L.ls_timing_read.argtypes = [C.c_int32, C.POINTER(C.c_int64), C.POINTER(C.c_double)]
         L.ls_kernel_launches.restype = C.c_int64
@@ -301,3 +302,15 @@ LS_OPT_FUSED = 1
 
 def ls_set_option(option: int, value: int) -> None:
     _check(lib().ls_set_option(option, value))
+
+
+LS_STATIC_TOPK_MAX_N = 32768
+
+
+def ls_topk_select_static(scores: torch.Tensor, k: int, idx: torch.Tensor, mask: Optional[torch.Tensor], count: torch.Tensor,
+                          stream=None) -> None:
+    """Top-k of a caller-provided fp64 device array without any allocation inside the library (for callers that must
+    not allocate: stream capture, allocator-free serving loops).  Outputs go to the caller's tensors."""
+    assert scores.dtype == torch.float64 and scores.is_cuda and scores.is_contiguous()
+    _check(lib().ls_topk_select_static(scores.data_ptr(), scores.numel(), k, idx.data_ptr(), _ptr(mask), count.data_ptr(),
+                                       _stream(stream)))

@@ -455,6 +455,64 @@ int32_t check_layer_call(ls_layer* L, int batch, const char* what) {
 
 }  // namespace
 
+// ---- allocation-free top-k ------------------------------------------------------------------------------------------
+// Scratch of ls_topk_select_static: candidate keys (8 bytes each) followed by candidate indices (4 bytes each) for up to
+// LS_STATIC_TOPK_MAX_N scores.  It lives in the library image, so every GPU that loads the library holds these 384 KB
+// until the process exits.  In host code this name is only a stand-in for the symbol, never a device address: the
+// address is taken per device with cudaGetSymbolAddress (static_topk_setup) and handed to the kernel as an argument.
+static __device__ __align__(256) unsigned char g_static_topk_scratch[(size_t)LS_STATIC_TOPK_MAX_N * 12];
+
+namespace {
+
+// Same selection as ls_topk_kernel, with the candidate lists kept in caller-independent static device memory instead of
+// shared memory / per-layer scratch.  Every position of the lists that is read has been written earlier in the same
+// launch, so nothing in the scratch has to start at zero and the previous call's contents do not matter.
+__global__ void __launch_bounds__(ls::TK_THREADS, 1)
+    ls_topk_static_kernel(const double* __restrict__ keys, int n, int k, int32_t* out_idx, uint32_t* out_mask, int32_t* out_count,
+                          unsigned char* scratch) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  ls::TopkSmem sm = ls::topk_carve(smem_raw);
+  unsigned long long* ckey = reinterpret_cast<unsigned long long*>(scratch);
+  int32_t* cidx = reinterpret_cast<int32_t*>(scratch + (size_t)LS_STATIC_TOPK_MAX_N * 8);
+  sm.key = ckey;  // the candidates go to the static scratch whatever their number
+  sm.idx = cidx;
+  uint32_t* s_mask = reinterpret_cast<uint32_t*>(smem_raw + ls::topk_smem_bytes(n));
+  const int nwords = (n + 31) >> 5;
+  for (int i = threadIdx.x; i < nwords; i += ls::TK_THREADS) s_mask[i] = 0u;
+  const int keff = ls::block_topk(
+      n, k,
+      [&](int v, double& s) {
+        s = keys[v];
+        return true;
+      },
+      [&](int rank, int v) {
+        out_idx[rank] = v;
+        atomicOr(&s_mask[v >> 5], 1u << (v & 31));
+      },
+      sm, ckey, cidx);
+  if (out_mask)
+    for (int w = threadIdx.x; w < nwords; w += ls::TK_THREADS) out_mask[w] = s_mask[w];
+  if (threadIdx.x == 0) *out_count = keff;
+}
+
+std::mutex g_static_mu;
+unsigned char* g_static_ptr[64] = {nullptr};  // device address of the scratch, per device ordinal
+
+// Once per device, with that device current: device address of the static scratch and the kernel's shared-memory opt-in.
+int32_t static_topk_setup(int dev, unsigned char** out) {
+  std::lock_guard<std::mutex> lk(g_static_mu);
+  if (!g_static_ptr[dev]) {
+    void* p = nullptr;
+    LS_CUDA(cudaGetSymbolAddress(&p, g_static_topk_scratch));
+    LS_CUDA(cudaFuncSetAttribute(ls_topk_static_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    g_static_ptr[dev] = static_cast<unsigned char*>(p);
+  }
+  *out = g_static_ptr[dev];
+  return LS_OK;
+}
+
+}  // namespace
+
 // =====================================================================================================================
 extern "C" {
 
@@ -470,6 +528,24 @@ size_t ls_last_error(char* buf, size_t n) {
 }
 
 int64_t ls_kernel_launches(void) { return g_launches.load(); }
+
+int32_t ls_topk_select_static(const double* d_scores, int32_t n, int32_t k, int32_t* d_idx, uint32_t* d_mask, int32_t* d_count,
+                              void* stream) {
+  if (!d_scores || !d_idx || !d_count) return fail(LS_ERR_INVALID, "ls_topk_select_static: scores, idx and count are required");
+  if (n < 1 || n > LS_STATIC_TOPK_MAX_N)
+    return fail(LS_ERR_INVALID, "ls_topk_select_static: n = %d is outside [1, %d] (the static scratch holds at most %d candidates)", n,
+                LS_STATIC_TOPK_MAX_N, LS_STATIC_TOPK_MAX_N);
+  if (k < 0 || k > n) return fail(LS_ERR_INVALID, "ls_topk_select_static: k = %d is outside [0, n = %d]", k, n);
+  int dev = -1;
+  LS_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return fail(LS_ERR_INVALID, "ls_topk_select_static: device ordinal %d not supported", dev);
+  unsigned char* scratch = nullptr;
+  LS_TRY(static_topk_setup(dev, &scratch));
+  ls_topk_static_kernel<<<1, ls::TK_THREADS, ls::topk_kernel_smem(n), (cudaStream_t)stream>>>(d_scores, n, k, d_idx, d_mask, d_count,
+                                                                                               scratch);
+  LS_LAUNCHED();
+  return LS_OK;
+}
 
 #ifdef LS_FZ_TIMING
 int32_t ls_debug_read_timing(long long* host, int32_t n) {
