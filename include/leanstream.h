@@ -38,7 +38,8 @@ extern "C" {
 #define LS_ERR_CUDA (-3)     /* a CUDA runtime call failed; ls_last_error() has the CUDA message */
 #define LS_ERR_STATE (-4)    /* call not valid for this layer (e.g. cache call on a resident layer) */
 #define LS_ERR_CAPACITY (-5) /* wanted + protected neurons exceed the cache capacity, or a list exceeds its cap */
-#define LS_ERR_TIMEOUT (-6)  /* a bounded wait for miss copies gave up */
+#define LS_ERR_TIMEOUT (-6)  /* a bounded wait (miss copies, a barrier inside a kernel) gave up */
+#define LS_ERR_INTERNAL (-7) /* a kernel's self-check failed (reported through ls_layer_status) */
 
 #define LS_ACT_RELU 0
 #define LS_WDTYPE_BF16 0

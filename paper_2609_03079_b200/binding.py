@@ -14,7 +14,7 @@ import torch
 
 from . import build as _build
 
-LS_OK, LS_ERR_INVALID, LS_ERR_NOMEM, LS_ERR_CUDA, LS_ERR_STATE, LS_ERR_CAPACITY, LS_ERR_TIMEOUT = 0, -1, -2, -3, -4, -5, -6
+LS_OK, LS_ERR_INVALID, LS_ERR_NOMEM, LS_ERR_CUDA, LS_ERR_STATE, LS_ERR_CAPACITY, LS_ERR_TIMEOUT, LS_ERR_INTERNAL = 0, -1, -2, -3, -4, -5, -6, -7
 LS_ACT_RELU = 0
 LS_WDTYPE_BF16, LS_WDTYPE_FP16 = 0, 1
 LS_NORM_RMS, LS_NORM_NONE = 0, 1

@@ -121,16 +121,8 @@ struct ls_layer {
   int* status = nullptr;                   // [1]
   int down_splits = 0;
 
-  // scratch of the fused per-layer kernel (see ls_fused.cuh for the zero-on-entry invariants)
-  float* fz_dacc = nullptr;           // [FZ_MAXK][d]
-  unsigned* fz_ctr = nullptr;         // fin, (pad), barrier counter (64-bit)
-  double* fz_z = nullptr;             // [FZ_MAXE][r] latents, [FZ_MAXE] sums of squares, [2] binning range
-  unsigned* fz_cnt = nullptr;         // [FZ_MAXE][FZ_CNT_STRIDE]
-  unsigned long long* fz_bkey = nullptr;  // [FZ_MAXE][FZ_NB * FZ_CAPB]
-  int32_t* fz_bidx = nullptr;
-  unsigned long long* fz_okey = nullptr;  // [FZ_MAXE][F]
-  int32_t* fz_oidx = nullptr;
-  int32_t* fz_obin = nullptr;
+  // per-layer state of the fused kernel; its working scratch is shared per device (DeviceScratch below)
+  double* fz_range = nullptr;                  // [2] binning range of this layer's scores (observed by its last launch)
   unsigned long long* fz_range_obs = nullptr;  // [2]
 
   ls::CacheState cache;  // residency tables, pinned backing store, copy stream
@@ -160,8 +152,7 @@ void free_layer(ls_layer* L) {
   cudaFree(L->bundles); cudaFree(L->b_gate); cudaFree(L->b_down); cudaFree(L->pred_at); cudaFree(L->pred_bt);
   cudaFree(L->pred_c); cudaFree(L->z); cudaFree(L->sumsq); cudaFree(L->scores); cudaFree(L->prio); cudaFree(L->cand_key);
   cudaFree(L->cand_idx); cudaFree(L->umask); cudaFree(L->tmp_idx); cudaFree(L->tmp_count); cudaFree(L->tmp_mask);
-  cudaFree(L->fz_dacc); cudaFree(L->fz_ctr); cudaFree(L->fz_z); cudaFree(L->fz_cnt); cudaFree(L->fz_bkey); cudaFree(L->fz_bidx);
-  cudaFree(L->fz_okey); cudaFree(L->fz_oidx); cudaFree(L->fz_obin); cudaFree(L->fz_range_obs);
+  cudaFree(L->fz_range); cudaFree(L->fz_range_obs);
   cudaFree(L->xin); cudaFree(L->xt); cudaFree(L->actv); cudaFree(L->ypart); cudaFree(L->survive); cudaFree(L->status);
   delete L;
 }
@@ -182,6 +173,48 @@ int32_t upload_transposed16(uint16_t** dst, const void* src, int rows, int cols)
     for (int j = 0; j < cols; ++j) t[(size_t)j * rows + i] = s[(size_t)i * cols + j];
   LS_TRY(dalloc(dst, t.size()));
   LS_CUDA(cudaMemcpy(*dst, t.data(), t.size() * 2, cudaMemcpyHostToDevice));
+  return LS_OK;
+}
+
+// Working scratch of the fused kernel, one per device and shared by all layers on it: a decode loop runs its layers one
+// after the other, and re-using the same few megabytes keeps them in L2 (per-layer copies would come back from HBM at
+// every step).  Consequence: fused steps on one device must not overlap (issue them on one stream, or order the
+// streams).  Sized for the largest shapes the fused path accepts; allocated at the first layer, kept until exit.
+struct DeviceScratch {
+  float* dacc = nullptr;              // [FZ_MAXK][16384] stage accumulators, zero between launches
+  unsigned* ctr = nullptr;            // fin, (pad), barrier counter (64-bit)
+  double* z = nullptr;                // [FZ_MAXE][1024] latents, then [FZ_MAXE] sums of squares
+  unsigned* cnt = nullptr;            // [FZ_MAXE][FZ_CNT_STRIDE], zero between launches
+  uint4* bent = nullptr;              // [FZ_MAXE][FZ_NB * FZ_CAPB] bucket entries
+  uint4* oent = nullptr;              // [FZ_MAXE][32768] overflow entries
+  unsigned* nsel = nullptr;           // [FZ_MAXE] refined-set sizes, zero between launches
+  bool ready = false;
+};
+constexpr int kScratchMaxD = 16384, kScratchMaxR = 1024, kScratchMaxF = 32768;
+std::mutex g_scratch_mu;
+DeviceScratch g_scratch[64];
+
+int32_t device_scratch(int dev, DeviceScratch** out) {
+  if (dev < 0 || dev >= 64) return fail(LS_ERR_INVALID, "device ordinal %d not supported", dev);
+  std::lock_guard<std::mutex> lk(g_scratch_mu);
+  DeviceScratch& S = g_scratch[dev];
+  if (!S.ready) {
+    const size_t NE = ls::FZ_MAXE;
+    LS_TRY(dalloc(&S.dacc, (size_t)ls::FZ_MAXK * kScratchMaxD));
+    LS_TRY(dalloc(&S.ctr, (size_t)8));
+    LS_TRY(dalloc(&S.z, NE * kScratchMaxR + NE));
+    LS_TRY(dalloc(&S.cnt, NE * ls::FZ_CNT_STRIDE));
+    LS_TRY(dalloc(&S.bent, NE * ls::FZ_NB * ls::FZ_CAPB));
+    LS_TRY(dalloc(&S.oent, NE * kScratchMaxF));
+    LS_TRY(dalloc(&S.nsel, NE));
+    LS_CUDA(cudaMemset(S.nsel, 0, NE * sizeof(unsigned)));
+    LS_CUDA(cudaMemset(S.dacc, 0, (size_t)ls::FZ_MAXK * kScratchMaxD * sizeof(float)));
+    LS_CUDA(cudaMemset(S.ctr, 0, 8 * sizeof(unsigned)));
+    LS_CUDA(cudaMemset(S.cnt, 0, NE * ls::FZ_CNT_STRIDE * sizeof(unsigned)));
+    LS_CUDA(cudaMemset(S.z, 0, (NE * kScratchMaxR + NE) * sizeof(double)));
+    S.ready = true;
+  }
+  if (out) *out = &S;
   return LS_OK;
 }
 
@@ -240,23 +273,11 @@ int32_t create_impl(const ls_layer_desc* D, ls_layer* L) {
   LS_CUDA(cudaMemset(L->prio, 0xff, F * sizeof(double)));  // NaN: ranks last until a prediction sets it
 
   if (L->cache_rows == 0) {
-    LS_TRY(dalloc(&L->fz_dacc, (size_t)ls::FZ_MAXK * d));
-    const size_t NE = ls::FZ_MAXE;
-    LS_TRY(dalloc(&L->fz_ctr, (size_t)8));
-    LS_TRY(dalloc(&L->fz_z, NE * L->r + NE + 8));
-    LS_TRY(dalloc(&L->fz_cnt, NE * ls::FZ_CNT_STRIDE));
-    LS_TRY(dalloc(&L->fz_bkey, NE * ls::FZ_NB * ls::FZ_CAPB));
-    LS_TRY(dalloc(&L->fz_bidx, NE * ls::FZ_NB * ls::FZ_CAPB));
-    LS_TRY(dalloc(&L->fz_okey, NE * F));
-    LS_TRY(dalloc(&L->fz_oidx, NE * F));
-    LS_TRY(dalloc(&L->fz_obin, NE * F));
+    LS_TRY(device_scratch(D->device, nullptr));
+    LS_TRY(dalloc(&L->fz_range, 2));
     LS_TRY(dalloc(&L->fz_range_obs, 2));
-    LS_CUDA(cudaMemset(L->fz_dacc, 0, (size_t)ls::FZ_MAXK * d * sizeof(float)));
-    LS_CUDA(cudaMemset(L->fz_ctr, 0, 8 * sizeof(unsigned)));
-    LS_CUDA(cudaMemset(L->fz_cnt, 0, NE * ls::FZ_CNT_STRIDE * sizeof(unsigned)));
     const double zr[2] = {-1.0, 1.0};  // binning range until a launch has observed one
-    LS_CUDA(cudaMemset(L->fz_z, 0, (NE * L->r + NE + 8) * sizeof(double)));
-    LS_CUDA(cudaMemcpy(L->fz_z + NE * L->r + NE, zr, sizeof zr, cudaMemcpyHostToDevice));
+    LS_CUDA(cudaMemcpy(L->fz_range, zr, sizeof zr, cudaMemcpyHostToDevice));
     const unsigned long long ro[2] = {0xffffffffffffffffULL, 0ULL};
     LS_CUDA(cudaMemcpy(L->fz_range_obs, ro, sizeof ro, cudaMemcpyHostToDevice));
   }
@@ -272,9 +293,8 @@ int32_t create_impl(const ls_layer_desc* D, ls_layer* L) {
   LS_ATTR_GU(0, 1); LS_ATTR_GU(0, 4); LS_ATTR_GU(0, 8); LS_ATTR_GU(1, 1); LS_ATTR_GU(1, 4); LS_ATTR_GU(1, 8);
 #undef LS_ATTR_GU
 #define LS_ATTR_FZ(WD, CPT) \
-  LS_CUDA(cudaFuncSetAttribute(ls::ls_fused_step_kernel<WD, CPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024))
-  LS_ATTR_FZ(0, 1); LS_ATTR_FZ(0, 2); LS_ATTR_FZ(0, 3); LS_ATTR_FZ(0, 4);
-  LS_ATTR_FZ(1, 1); LS_ATTR_FZ(1, 2); LS_ATTR_FZ(1, 3); LS_ATTR_FZ(1, 4);
+  LS_CUDA(cudaFuncSetAttribute(ls::ls_fused_step_kernel<WD, CPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 218 * 1024))
+  LS_ATTR_FZ(0, 1); LS_ATTR_FZ(0, 2); LS_ATTR_FZ(1, 1); LS_ATTR_FZ(1, 2);
 #undef LS_ATTR_FZ
   LS_CUDA(cudaDeviceSynchronize());
   return LS_OK;
@@ -283,12 +303,12 @@ int32_t create_impl(const ls_layer_desc* D, ls_layer* L) {
 // ---- the fused per-layer kernel: eligibility and launch ---------------------------------------------------------------
 // Shared-memory plan of the fused kernel: as many ring stages as fit beside the predictor operands.
 bool fused_plan(const ls_layer* L, const ls_layer* next, ls::FusedSmemLayout* out) {
-  const size_t budget = 226 * 1024;
+  const size_t budget = 218 * 1024;  // dynamic part; the kernel also has a few KB of static shared memory
   const int n_in = L->gated ? 2 : 1;
   const int r = next ? next->r : 0, Fn = next ? next->F : 0, hn = next ? 1 : 0;
-  for (int dn = ls::FZ_MAX_DEPTH / 2; dn >= 2; --dn) {
-    for (int gu = ls::FZ_MAX_DEPTH; gu >= 2; --gu) {
-      if (gu < dn) break;
+  // the gate/up ring wants two rounds in flight; the down ring at least one round of survivors
+  for (int gu = ls::FZ_MAX_DEPTH; gu >= ls::FZ_NG + 1; --gu) {
+    for (int dn = 4; dn >= ls::FZ_NG; --dn) {
       const ls::FusedSmemLayout lay = ls::fused_layout(L->d, n_in, r, Fn, L->sm_count, hn, gu, dn);
       if (lay.total <= budget) {
         if (out) *out = lay;
@@ -304,7 +324,7 @@ bool fused_eligible(const ls_layer* L, const ls_layer* next, int batch, int K, i
   if (batch != 1 || L->cache_rows != 0 || (next && next->cache_rows != 0)) return false;
   if (K > ls::FZ_MAXK) return false;
   if ((sel_cap + L->sm_count - 1) / L->sm_count > ls::FZ_MAX_MINE) return false;
-  if ((L->d >> 3) > ls::FZ_STREAM_THREADS * 4) return false;
+  if ((L->d >> 3) > ls::FZ_THREADS * 2) return false;
   return fused_plan(L, next, nullptr);
 }
 
@@ -314,12 +334,10 @@ int32_t launch_fused_cpt(int cpt, const ls::FusedArgs& a, int grid, size_t smem,
   const void* fn = nullptr;
   switch (cpt) {
     case 1: fn = (const void*)ls::ls_fused_step_kernel<WD, 1>; break;
-    case 2: fn = (const void*)ls::ls_fused_step_kernel<WD, 2>; break;
-    case 3: fn = (const void*)ls::ls_fused_step_kernel<WD, 3>; break;
-    default: fn = (const void*)ls::ls_fused_step_kernel<WD, 4>; break;
+    default: fn = (const void*)ls::ls_fused_step_kernel<WD, 2>; break;
   }
   KernelTimer timer(LS_TIMED_FUSED, st);
-  LS_CUDA(cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(ls::FZ_THREADS), params, smem, st));
+  LS_CUDA(cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(ls::FZ_BLOCK), params, smem, st));
   LS_LAUNCHED();
   return LS_OK;
 }
@@ -331,17 +349,19 @@ int32_t fused_step(ls_layer* L, ls_layer* next, const float* d_x, float* d_x_out
   a.d = L->d; a.F = L->F; a.norm = L->norm; a.eps = L->eps;
   a.x = d_x; a.x_out = d_x_out;
   a.sel_idx = sel->idx; a.sel_count = sel->count; a.sel_cap = sel->cap; a.K = K;
-  a.dacc = L->fz_dacc; a.fin = L->fz_ctr;
-  a.bar_count = reinterpret_cast<unsigned long long*>(L->fz_ctr + 2);  // 8-byte aligned
+  DeviceScratch* S = nullptr;
+  LS_TRY(device_scratch(L->device, &S));
+  a.dacc = S->dacc; a.fin = S->ctr;
+  a.bar_count = reinterpret_cast<unsigned long long*>(S->ctr + 2);  // 8-byte aligned
   a.status = L->status;
   a.has_next = next ? 1 : 0;
   const int nw_next = next ? next->nwords : 0;
   if (next) {
     a.At = next->pred_at; a.Bt = next->pred_bt; a.pc = next->pred_c;
     a.r = next->r; a.Fn = next->F; a.norm_n = next->norm; a.eps_n = next->eps; a.k_next = k_next;
-    a.z = next->fz_z; a.sumsq = next->fz_z + (size_t)ls::FZ_MAXE * next->r; a.range = a.sumsq + ls::FZ_MAXE;
-    a.cnt = next->fz_cnt; a.bkey = next->fz_bkey; a.bidx = next->fz_bidx; a.okey = next->fz_okey; a.oidx = next->fz_oidx;
-    a.obin = next->fz_obin; a.range_obs = next->fz_range_obs; a.tmp_idx = next->tmp_idx;
+    a.z = S->z; a.sumsq = S->z + (size_t)ls::FZ_MAXE * next->r; a.range = next->fz_range;
+    a.cnt = S->cnt; a.bent = S->bent; a.oent = S->oent;
+    a.range_obs = next->fz_range_obs; a.nsel = S->nsel;
     a.next_idx = sel_next->idx; a.next_count = sel_next->count; a.next_mask = sel_next->mask; a.next_scores = sel_next->scores;
     a.next_prio = next->prio; a.next_cap = sel_next->cap;
     if (sel_next->mask) LS_CUDA(cudaMemsetAsync(sel_next->mask, 0, (size_t)nw_next * 4, st));
@@ -358,7 +378,7 @@ int32_t fused_step(ls_layer* L, ls_layer* next, const float* d_x, float* d_x_out
   ls::FusedSmemLayout lay{};
   if (!fused_plan(L, next, &lay)) return fail(LS_ERR_STATE, "fused step: shared memory plan failed");
   a.gu_depth = lay.gu_depth; a.dn_depth = lay.dn_depth;
-  const int cpt = ((L->d >> 3) + ls::FZ_STREAM_THREADS - 1) / ls::FZ_STREAM_THREADS;
+  const int cpt = ((L->d >> 3) + ls::FZ_THREADS - 1) / ls::FZ_THREADS;
   if (L->wd == 0) return launch_fused_cpt<0>(cpt, a, L->sm_count, lay.total, st);
   return launch_fused_cpt<1>(cpt, a, L->sm_count, lay.total, st);
 }

@@ -14,6 +14,7 @@ constexpr int ST_OK = 0;
 constexpr int ST_BAD_INDEX = -1;
 constexpr int ST_CAPACITY = -5;
 constexpr int ST_TIMEOUT = -6;
+constexpr int ST_INTERNAL = -7;
 
 __device__ __forceinline__ void set_status(int* status, int code) {
   if (status) atomicCAS(status, 0, code);

@@ -5,11 +5,11 @@
 //
 //   1. stream   The K priority stages of the layer (Eq. 1) run CONCURRENTLY on K disjoint groups of CTAs (the output is
 //               a sum over hidden neurons, so stage order in time is free; only stage membership defines the partial
-//               features).  Inside a CTA the stream warps take two neurons per round: gate+up rows arrive by 1-D TMA
-//               bulk copies into a shared-memory ring, the block reduces the dot products, surviving neurons fetch
-//               their down row into a second ring, and the CTA's whole contribution to its stage is kept in registers
-//               and added once to the stage accumulator (vector reductions).  Meanwhile the loader warps bring this
-//               CTA's share of the next layer's predictor (rows of A^T and of B^T) into shared memory.
+//               features).  A CTA takes three neurons per round: gate+up rows arrive by 1-D TMA bulk copies into a
+//               shared-memory ring, the block reduces the dot products, surviving neurons fetch their down row into a
+//               second ring, and the CTA's whole contribution to its stage is kept in registers and added once to the
+//               stage accumulator (vector reductions).  The CTA's share of the next layer's predictor (rows of A^T and
+//               of B^T) arrives in shared memory by bulk copies issued at the start.
 //      -- barrier --
 //   2. latent   Every partial residual feature x~^(j) = x + sum_{c<j} dm^(c), j = 0..K (Eq. 2), is rebuilt on the fly
 //               from the stage accumulators, and this CTA's rows of all K+1 latents z^(j) = A^T x~^(j) are formed in one
@@ -26,9 +26,9 @@
 
 namespace ls {
 
-constexpr int FZ_STREAM_THREADS = 256;
-constexpr int FZ_THREADS = 512;
-constexpr int FZ_NG = 2;          // neurons the stream warps process per round
+constexpr int FZ_THREADS = 512;        // compute threads (16 warps)
+constexpr int FZ_BLOCK = FZ_THREADS + 32;  // plus the producer warp
+constexpr int FZ_NG = 3;          // neurons processed per round
 constexpr int FZ_NB = 4096;       // fine score bins per evaluation
 constexpr int FZ_NC = 64;         // coarse bins (FZ_NB / FZ_NC fine bins each)
 constexpr int FZ_CNT_STRIDE = FZ_NB + FZ_NC + 4;  // fine counts, coarse counts, overflow count (+ padding to 16 bytes)
@@ -59,14 +59,11 @@ struct FusedArgs {
   double* z;              // [FZ_MAXE][r] un-normalised latents
   double* sumsq;          // [FZ_MAXE]
   unsigned* cnt;          // [FZ_MAXE][FZ_CNT_STRIDE], zero on entry and on exit
-  unsigned long long* bkey;  // [FZ_MAXE][FZ_NB * FZ_CAPB]
-  int32_t* bidx;             // [FZ_MAXE][FZ_NB * FZ_CAPB]
-  unsigned long long* okey;  // [FZ_MAXE][Fn] overflow entries
-  int32_t* oidx;             // [FZ_MAXE][Fn]
-  int32_t* obin;             // [FZ_MAXE][Fn]
+  uint4* bent;            // [FZ_MAXE][FZ_NB * FZ_CAPB] bucket entries {key lo, key hi, neuron, fine bin}, one 16-byte store each
+  uint4* oent;            // [FZ_MAXE][Fn] overflow entries, same format
   double* range;          // [2] lo, hi used for binning (observed by the previous launch on this layer)
   unsigned long long* range_obs;  // [2] ordered keys: min, max observed in the final evaluation
-  int32_t* tmp_idx;       // [max_sel] rank list of the intermediate evaluations (not returned)
+  unsigned* nsel;         // [FZ_MAXE] sizes of the refined sets (all CTAs add theirs), zero on entry and on exit
   // outputs for the next layer
   int32_t* next_idx; int32_t* next_count; uint32_t* next_mask; double* next_scores; double* next_prio; int next_cap;
   // trace (all nullable)
@@ -128,9 +125,10 @@ __device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float 
 
 // Barrier among all CTAs of the (cooperatively launched, co-resident) grid: one monotonically increasing 64-bit counter,
 // never reset.  Arrival is a release, the poll an acquire, so what a CTA wrote before the barrier is visible to all
-// after it.  Every thread of the block calls it.
+// after it.  Every compute thread of the block calls it (block barrier 1 spans the 512 compute threads; the producer
+// warp has left by then).
 __device__ __forceinline__ void grid_barrier(const FusedArgs& A, int G) {
-  __syncthreads();
+  named_bar_sync(1, FZ_THREADS);
   if (threadIdx.x == 0) {
     unsigned long long old;
     asm volatile("atom.add.release.gpu.global.u64 %0, [%1], 1;" : "=l"(old) : "l"(A.bar_count) : "memory");
@@ -144,7 +142,7 @@ __device__ __forceinline__ void grid_barrier(const FusedArgs& A, int G) {
     } while (clock64() - t0 < FZ_SPIN_CYCLES);
     if (!ok) set_status(A.status, ST_TIMEOUT);
   }
-  __syncthreads();
+  named_bar_sync(1, FZ_THREADS);
 }
 
 template <int WD>
@@ -175,8 +173,8 @@ __host__ __device__ inline FusedSmemLayout fused_layout(int d, int n_in, int r, 
   auto take = [&](size_t bytes) { size_t at = o; o += (bytes + 127) & ~(size_t)127; return at; };
   L.gu_off = take((size_t)gu_depth * n_in * d * 2);
   L.dn_off = take((size_t)dn_depth * d * 2);
-  L.bar_off = take(2 * FZ_MAX_DEPTH * 8);
-  L.red_off = take(2 * 8 * 4 * 4);                   // stream dot partials, double-buffered
+  L.bar_off = take((2 * FZ_MAX_DEPTH + 1) * 8);
+  L.red_off = take(2 * 16 * 8 * 4);                  // stream dot partials, double-buffered: [2][warp][8]
   L.redd_off = take((size_t)FZ_MAXE * 3 * 16 * 8);   // fp64 partials of the latent phase: [evaluation][row0,row1,sumsq][warp]
   L.mine_off = take((size_t)FZ_MAX_MINE * 8);        // this CTA's neuron indices and gate biases
   L.per = has_next ? (Fn + G - 1) / G : 0;
@@ -194,7 +192,7 @@ __host__ __device__ inline FusedSmemLayout fused_layout(int d, int n_in, int r, 
 
 // =====================================================================================================================
 template <int WD, int CPT>
-__global__ void __launch_bounds__(FZ_THREADS, 1) ls_fused_step_kernel(const __grid_constant__ FusedArgs A) {
+__global__ void __launch_bounds__(FZ_BLOCK, 1) ls_fused_step_kernel(const __grid_constant__ FusedArgs A) {
   extern __shared__ __align__(128) unsigned char smem[];
   const int G = gridDim.x, cta = blockIdx.x, tid = threadIdx.x;
   const int lane = tid & 31, warp = tid >> 5;
@@ -205,16 +203,28 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) ls_fused_step_kernel(const __gr
   uint16_t* s_gu = reinterpret_cast<uint16_t*>(smem + lay.gu_off);
   uint16_t* s_dn = reinterpret_cast<uint16_t*>(smem + lay.dn_off);
   uint64_t* s_bar = reinterpret_cast<uint64_t*>(smem + lay.bar_off);  // [0..GU) gate/up full, [FZ_MAX_DEPTH..+DN) down full
-  float* s_red = reinterpret_cast<float*>(smem + lay.red_off);        // [2][8 warps][4]
+  float* s_red = reinterpret_cast<float*>(smem + lay.red_off);        // [2][16 warps][8]
   double* s_redd = reinterpret_cast<double*>(smem + lay.redd_off);
   uint16_t* s_A = reinterpret_cast<uint16_t*>(smem + lay.a_off);      // [nA][d]
   uint16_t* s_B = reinterpret_cast<uint16_t*>(smem + lay.b_off);      // [per][r]
   float* s_pc = reinterpret_cast<float*>(smem + lay.pc_off);
   __shared__ int s_last;
+  __shared__ int s_round;      // rounds the compute warps have finished (read by the producer)
+  __shared__ int s_mail[4 * 4];  // per round (ring of four): number of survivors, their neurons
+  __shared__ float s_act[2 * 4]; // activations of the round's neurons, double-buffered
+  __shared__ double s_inv[8];
+  __shared__ int s_cut[FZ_MAXE * 4];             // per evaluation: cut fine bin, its first rank, threshold neuron, fallback flag
+  __shared__ unsigned long long s_cutkey[FZ_MAXE];  // threshold key inside the cut bin
+  __shared__ unsigned s_nsel[FZ_MAXE];              // members found by this CTA, per evaluation
+  __shared__ unsigned long long s_kmm[2 * 16];
+  __shared__ unsigned s_ccnt[FZ_MAXE * FZ_NC];
 
+  if (tid == 0) FZ_STAMP(1, 72);
   if (tid == 0) {
     for (int i = 0; i < GU; ++i) mbar_init(&s_bar[i], 1);
     for (int i = 0; i < DN; ++i) mbar_init(&s_bar[FZ_MAX_DEPTH + i], 1);
+    mbar_init(&s_bar[2 * FZ_MAX_DEPTH], 1);
+    s_round = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -225,8 +235,8 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) ls_fused_step_kernel(const __gr
   const int n_own = max(0, i_hi - i_lo);
   const bool feat_writer = (cta == 0);
 
-  if (tid < FZ_STREAM_THREADS) {
-    // ================================================= stream warps ================================================
+  {
+    // ================================================= stream: all warps ===========================================
     // this CTA serves one stage: the ranks [lo, hi) of the selection, every gsize-th neuron starting at its own offset
     const int count = max(0, min(*A.sel_count, A.sel_cap));
     const int m = count > 0 ? (count + K - 1) / K : 0;
@@ -235,12 +245,22 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) ls_fused_step_kernel(const __gr
     const int lo = min(count, stage * m), hi = min(count, (stage + 1) * m);
     const int first = lo + (cta - g_lo);
     const int n_mine = first < hi ? (hi - first + gsize - 1) / gsize : 0;
+    const uint32_t gu_bytes = (uint32_t)n_in * d * 2, dn_bytes = (uint32_t)d * 2;
+    const size_t bundle_elems = (size_t)A.n_mat * d;
 
+    // this CTA's neurons first (the bulk copies only need the indices), then x and the gate biases
+    int* s_myidx = reinterpret_cast<int*>(smem + lay.mine_off);
+    float* s_mybias = reinterpret_cast<float*>(s_myidx + FZ_MAX_MINE);
+    for (int t = tid; t < n_mine; t += FZ_THREADS) {
+      int i = A.sel_idx[first + t * gsize];
+      if ((unsigned)i >= (unsigned)A.F) { set_status(A.status, ST_BAD_INDEX); i = -1; }
+      s_myidx[t] = i;
+    }
     float xr[CPT][8];
     double sq = 0.0;
 #pragma unroll
     for (int q = 0; q < CPT; ++q) {
-      const int ch = tid + q * FZ_STREAM_THREADS;
+      const int ch = tid + q * FZ_THREADS;
       if (ch < nchunk) {
         const float4 a0 = __ldg(reinterpret_cast<const float4*>(A.x + ch * 8));
         const float4 a1 = __ldg(reinterpret_cast<const float4*>(A.x + ch * 8 + 4));
@@ -253,37 +273,81 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) ls_fused_step_kernel(const __gr
 #pragma unroll
       for (int e = 0; e < 8; ++e) sq = fma((double)xr[q][e], (double)xr[q][e], sq);
     }
-    const uint32_t gu_bytes = (uint32_t)n_in * d * 2, dn_bytes = (uint32_t)d * 2;
-    const size_t bundle_elems = (size_t)A.n_mat * d;
+    __syncthreads();  // indices visible (the producer warp takes part in this barrier, then goes its own way)
 
-    // this CTA's neurons and their gate biases, fetched once (two dependent reads, all entries in parallel)
-    int* s_myidx = reinterpret_cast<int*>(smem + lay.mine_off);
-    float* s_mybias = reinterpret_cast<float*>(s_myidx + FZ_MAX_MINE);
-    for (int t = tid; t < n_mine; t += FZ_STREAM_THREADS) {
-      int i = A.sel_idx[first + t * gsize];
-      if ((unsigned)i >= (unsigned)A.F) { set_status(A.status, ST_BAD_INDEX); i = -1; }
-      s_myidx[t] = i;
+    if (warp == FZ_THREADS / 32) {
+      // ============================================= producer warp (one lane) ======================================
+      // Issues every bulk copy, so that the compute warps never pay for it: the first ring fills, the predictor
+      // operands, and after each round (announced through s_round) the refills and the survivors' down rows.
+      if (lane == 0) {
+        auto issue_gu = [&](int it) {
+          int i = s_myidx[it];
+          if (i < 0) i = 0;  // a rejected index: read row 0, the result is discarded
+          uint64_t* bar = &s_bar[it % GU];
+          mbar_expect_tx(bar, gu_bytes);
+          tma_load_1d(s_gu + (size_t)(it % GU) * n_in * d, A.bundles + (size_t)i * bundle_elems, gu_bytes, bar);
+        };
+        for (int it = 0; it < min(n_mine, GU); ++it) issue_gu(it);
+        if (A.has_next) {
+          // this CTA's share of the next layer's predictor, as stored: rows of A^T, rows of B^T (padded row stride)
+          uint64_t* pbar = &s_bar[2 * FZ_MAX_DEPTH];
+          uint32_t bytes = 0;
+          for (int a = 0; a < lay.nA; ++a)
+            if (cta + a * G < r) bytes += (uint32_t)d * 2;
+          bytes += (uint32_t)n_own * (uint32_t)r * 2;
+          mbar_expect_tx(pbar, bytes);
+          for (int a = 0; a < lay.nA; ++a) {
+            const int j = cta + a * G;
+            if (j < r) tma_load_1d(s_A + (size_t)a * d, A.At + (size_t)j * d, (uint32_t)d * 2, pbar);
+          }
+          for (int li = 0; li < n_own; ++li)
+            tma_load_1d(s_B + (size_t)li * (r + FZ_BPAD), A.Bt + (size_t)(i_lo + li) * r, (uint32_t)r * 2, pbar);
+        }
+        const int n_rounds = (n_mine + FZ_NG - 1) / FZ_NG;
+        int tail = 0;
+        for (int rd = 0; rd < n_rounds; ++rd) {
+          const long long t0 = clock64();
+          bool ok = false;
+          do {
+            int v;
+            asm volatile("ld.acquire.cta.shared.s32 %0, [%1];" : "=r"(v) : "r"(smem_u32(&s_round)) : "memory");
+            if (v > rd) { ok = true; break; }
+          } while (clock64() - t0 < FZ_SPIN_CYCLES);
+          if (!ok) { set_status(A.status, ST_TIMEOUT); break; }
+          const int it0 = rd * FZ_NG, nn = min(FZ_NG, n_mine - it0);
+          for (int e = 0; e < nn; ++e)
+            if (it0 + e + GU < n_mine) issue_gu(it0 + e + GU);
+          const int* mail = s_mail + (rd & 3) * 4;
+          const int ns = mail[0];
+          for (int e = 0; e < ns; ++e) {
+            const int i = mail[1 + e];
+            const int ds = tail % DN;
+            uint64_t* bar = &s_bar[FZ_MAX_DEPTH + ds];
+            mbar_expect_tx(bar, dn_bytes);
+            tma_load_1d(s_dn + (size_t)ds * d, A.bundles + (size_t)i * bundle_elems + (size_t)(A.n_mat - 1) * d, dn_bytes, bar);
+            if (A.tr_survive) atomicOr(&A.tr_survive[i >> 5], 1u << (i & 31));
+            ++tail;
+          }
+        }
+      }
+      return;  // an exited warp counts as arrived at every later block barrier
+    }
+
+    for (int t = tid; t < n_mine; t += FZ_THREADS) {
+      const int i = s_myidx[t];
       s_mybias[t] = (A.b_gate && i >= 0) ? A.b_gate[i] : 0.f;
     }
+    if (A.has_next)
+      for (int li = tid; li < n_own; li += FZ_THREADS) s_pc[li] = A.pc ? A.pc[i_lo + li] : 0.f;
     sq = warp_sum(sq);
     if (lane == 0) s_redd[warp] = sq;
-    named_bar_sync(1, FZ_STREAM_THREADS);
+    named_bar_sync(1, FZ_THREADS);
     double tot = 0.0;
 #pragma unroll
-    for (int w = 0; w < 8; ++w) tot += s_redd[w];
+    for (int w = 0; w < FZ_THREADS / 32; ++w) tot += s_redd[w];
     const float inv_rms = A.norm == 0 ? (float)(1.0 / sqrt(tot / (double)d + (double)A.eps)) : 1.0f;
 
-    auto issue_gu = [&](int it) {  // thread 0 only
-      int i = s_myidx[it];
-      if (i < 0) i = 0;  // a rejected index: read row 0, the result is discarded
-      uint64_t* bar = &s_bar[it % GU];
-      mbar_expect_tx(bar, gu_bytes);
-      tma_load_1d(s_gu + (size_t)(it % GU) * n_in * d, A.bundles + (size_t)i * bundle_elems, gu_bytes, bar);
-    };
-    if (tid == 0)
-      for (int it = 0; it < min(n_mine, GU); ++it) issue_gu(it);
-
-    // pending down rows: FIFO over the down ring; every stream thread tracks the same activations in registers
+    // pending down rows: FIFO over the down ring; every thread tracks the same activations in registers
     float qa[4] = {0.f, 0.f, 0.f, 0.f};
     int dq_head = 0, dq_tail = 0;
     float yacc[CPT][8];
@@ -304,7 +368,7 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) ls_fused_step_kernel(const __gr
       const uint16_t* row = s_dn + (size_t)slot * d;
 #pragma unroll
       for (int q = 0; q < CPT; ++q) {
-        const int ch = tid + q * FZ_STREAM_THREADS;
+        const int ch = tid + q * FZ_THREADS;
         if (ch < nchunk) {
           float w[8];
           unpack8<WD>(*reinterpret_cast<const uint4*>(row + ch * 8), w);
@@ -335,7 +399,7 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) ls_fused_step_kernel(const __gr
           const uint16_t* grow = s_gu + (size_t)slot * n_in * d;
 #pragma unroll
           for (int q = 0; q < CPT; ++q) {
-            const int ch = tid + q * FZ_STREAM_THREADS;
+            const int ch = tid + q * FZ_THREADS;
             if (ch < nchunk) {
               float w[8];
               unpack8<WD>(*reinterpret_cast<const uint4*>(grow + ch * 8), w);
@@ -359,41 +423,54 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) ls_fused_step_kernel(const __gr
           pu[e] += __shfl_xor_sync(0xffffffffu, pu[e], o);
         }
       }
-      float* red = s_red + (rd & 1) * 32;
-      if (lane == 0) *reinterpret_cast<float4*>(red + warp * 4) = make_float4(pg[0], pu[0], pg[1], pu[1]);
-      named_bar_sync(1, FZ_STREAM_THREADS);  // partials visible; every thread is done with the round's ring slots
-      float4 acc4 = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-      for (int w = 0; w < 8; ++w) {
-        const float4 v = *reinterpret_cast<const float4*>(red + w * 4);
-        acc4.x += v.x; acc4.y += v.y; acc4.z += v.z; acc4.w += v.w;
+      float* red = s_red + (rd & 1) * (FZ_THREADS / 32) * 8;  // [warp][8]: g0 u0 g1 u1 g2 u2 - -
+      if (lane == 0) {
+        *reinterpret_cast<float4*>(red + warp * 8) = make_float4(pg[0], pu[0], pg[1], pu[1]);
+        *reinterpret_cast<float2*>(red + warp * 8 + 4) = make_float2(pg[2], pu[2]);
       }
+      named_bar_sync(1, FZ_THREADS);  // partials visible; every thread is done with the round's ring slots
+      // (3) warp 0 finishes the six sums, forms the activations and tells the producer what to fetch
+      if (warp == 0) {
+        float v = 0.f;
+        if (lane < 2 * FZ_NG) {
+#pragma unroll
+          for (int w = 0; w < FZ_THREADS / 32; ++w) v += red[w * 8 + lane];
+        }
+        const float u = __shfl_down_sync(0xffffffffu, v, 1);  // lane 2e holds g_e, lane 2e+1 holds u_e
+        float a = 0.f;
+        int i = -1;
+        const int e = lane >> 1;
+        if (!(lane & 1) && e < nn) {
+          const int it = it0 + e;
+          i = s_myidx[it];
+          const float g = v * inv_rms + s_mybias[it];
+          a = fmaxf(g, 0.f);
+          if (A.gated) a *= u * inv_rms;
+          if (i < 0) a = 0.f;
+          s_act[(rd & 1) * 4 + e] = a;
+        } else if (!(lane & 1) && e < FZ_NG) {
+          s_act[(rd & 1) * 4 + e] = 0.f;
+        }
+        // survivors in neuron order -> mailbox of the round
+        const unsigned surv = __ballot_sync(0xffffffffu, a != 0.f);
+        if (a != 0.f) s_mail[(rd & 3) * 4 + 1 + __popc(surv & ((1u << lane) - 1u))] = i;
+        if (lane == 0) {
+          s_mail[(rd & 3) * 4] = __popc(surv);
+          asm volatile("st.release.cta.shared.s32 [%0], %1;" ::"r"(smem_u32(&s_round)), "r"(rd + 1) : "memory");
+        }
+      }
+      named_bar_sync(1, FZ_THREADS);
       if (tid == 0) FZ_STAMP(0, 3 + rd * 4);
-      // (3) activations; refill the ring slots; survivors queue their down row
-      const float gs[FZ_NG] = {acc4.x, acc4.z}, us[FZ_NG] = {acc4.y, acc4.w};
+      // (4) every thread queues the survivors' activations in the same order as the producer queued their rows
 #pragma unroll
       for (int e = 0; e < FZ_NG; ++e) {
-        if (e < nn) {
-          const int it = it0 + e;
-          const int i = s_myidx[it];
-          const float g = gs[e] * inv_rms + s_mybias[it];
-          float a = fmaxf(g, 0.f);
-          if (A.gated) a *= us[e] * inv_rms;
-          if (i < 0) a = 0.f;
-          if (tid == 0 && it + GU < n_mine) issue_gu(it + GU);
-          if (a != 0.f) {
-            const int ds = dq_tail % DN;
+        const float a = s_act[(rd & 1) * 4 + e];
+        if (e < nn && a != 0.f) {
+          const int ds = dq_tail % DN;
 #pragma unroll
-            for (int t = 0; t < 4; ++t)
-              if (ds == t) qa[t] = a;
-            if (tid == 0) {
-              uint64_t* bar = &s_bar[FZ_MAX_DEPTH + ds];
-              mbar_expect_tx(bar, dn_bytes);
-              tma_load_1d(s_dn + (size_t)ds * d, A.bundles + (size_t)i * bundle_elems + (size_t)(A.n_mat - 1) * d, dn_bytes, bar);
-              if (A.tr_survive) atomicOr(&A.tr_survive[i >> 5], 1u << (i & 31));
-            }
-            ++dq_tail;
-          }
+          for (int t = 0; t < 4; ++t)
+            if (ds == t) qa[t] = a;
+          ++dq_tail;
         }
       }
       if (tid == 0) FZ_STAMP(0, 4 + rd * 4);
@@ -405,7 +482,7 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) ls_fused_step_kernel(const __gr
       float* dst = A.dacc + (size_t)stage * d;
 #pragma unroll
       for (int q = 0; q < CPT; ++q) {
-        const int ch = tid + q * FZ_STREAM_THREADS;
+        const int ch = tid + q * FZ_THREADS;
         if (ch < nchunk) {
           red_add_v4(dst + ch * 8, yacc[q][0], yacc[q][1], yacc[q][2], yacc[q][3]);
           red_add_v4(dst + ch * 8 + 4, yacc[q][4], yacc[q][5], yacc[q][6], yacc[q][7]);
@@ -413,26 +490,7 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) ls_fused_step_kernel(const __gr
       }
     }
     if (tid == 0) FZ_STAMP(0, 501);
-  } else if (A.has_next) {
-    // ================================================= loader warps ================================================
-    // this CTA's rows of A^T and of B^T, and the score biases of its neurons, as stored (128-bit loads)
-    const int ltid = tid - FZ_STREAM_THREADS, LT = FZ_THREADS - FZ_STREAM_THREADS;
-    for (int a = 0; a < lay.nA; ++a) {
-      const int j = cta + a * G;
-      if (j < r) {
-#pragma unroll 4
-        for (int c8 = ltid; c8 < (d >> 3); c8 += LT)
-          *reinterpret_cast<uint4*>(s_A + (size_t)a * d + c8 * 8) = ldg128(A.At + (size_t)j * d + c8 * 8);
-      }
-    }
-    for (int li = ltid; li < n_own; li += LT) s_pc[li] = A.pc ? A.pc[i_lo + li] : 0.f;
-    const int r8 = r >> 3, nB8 = n_own * r8;  // r is a multiple of 8
-    const uint16_t* bsrc = A.Bt + (size_t)i_lo * r;
-#pragma unroll 4
-    for (int t8 = ltid; t8 < nB8; t8 += LT) {
-      const int li = t8 / r8, c8 = t8 - li * r8;
-      *reinterpret_cast<uint4*>(s_B + (size_t)li * (r + FZ_BPAD) + c8 * 8) = ldg128(bsrc + (size_t)t8 * 8);
-    }
+    if (A.has_next) mbar_wait(&s_bar[2 * FZ_MAX_DEPTH], 0u, A.status);  // predictor operands have landed
   }
 
   // ------------------------------------------------------------------------------------------------ barrier 1 of 3
@@ -443,16 +501,15 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) ls_fused_step_kernel(const __gr
   // ============================ phase 2: partial features x~^(j) and this CTA's latent rows ===========================
   // Each thread owns d/512 columns.  For every j = 0..K it rebuilds x~^(j) of its columns (x + the stage accumulators
   // below j) and accumulates the dot products with this CTA's rows of A^T; rows are taken two at a time.
-  constexpr int XC = 4 * CPT;     // columns per thread (d <= 2048 * CPT)
-  float xfin[XC];                 // x~^(K) of this thread's columns (kept by the CTA that writes x_out)
-#pragma unroll
-  for (int q = 0; q < XC; ++q) xfin[q] = 0.f;
+  constexpr int XC = 8 * CPT;     // columns per thread (d <= 4096 * CPT)
+  float* s_xfin = reinterpret_cast<float*>(smem + lay.gu_off);  // x~^(K), kept by the CTA that writes x_out (the ring is idle now)
   if (A.has_next || feat_writer) {
     constexpr int JG = 4;         // evaluations accumulated together
     const int npair = A.has_next ? max(1, (lay.nA + 1) / 2) : 1;
     for (int pr = 0; pr < npair; ++pr) {
       const int a0 = pr * 2;
       const bool one = A.has_next && a0 < lay.nA, two = A.has_next && a0 + 1 < lay.nA;
+      const int sq_eval = (pr == 0 && cta <= K) ? cta : -1;  // CTA j provides the sum of squares of x~^(j)
       float xs[XC];  // x~^(j) of this thread's columns, advanced stage by stage
 #pragma unroll
       for (int q = 0; q < XC; ++q) {
@@ -463,6 +520,7 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) ls_fused_step_kernel(const __gr
         double p0[JG], p1[JG], sq[JG];
 #pragma unroll
         for (int e = 0; e < JG; ++e) { p0[e] = 0.0; p1[e] = 0.0; sq[e] = 0.0; }
+        if (tid == 0) FZ_STAMP(1, 10 + j0);
         // the stage accumulators this group needs, all fetched before anything is stored
         float dv[XC][JG];
 #pragma unroll
@@ -485,10 +543,10 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) ls_fused_step_kernel(const __gr
                 const double xd = (double)xv;
                 p0[e] = fma(w0, xd, p0[e]);
                 p1[e] = fma(w1, xd, p1[e]);
-                sq[e] = fma(xd, xd, sq[e]);
+                if (j == sq_eval) sq[e] = fma(xd, xd, sq[e]);
                 if (feat_writer && pr == 0) {
                   if (A.tr_xtilde) A.tr_xtilde[(size_t)j * d + c] = xv;
-                  if (j == K) xfin[q] = xv;
+                  if (j == K) s_xfin[c] = xv;
                 }
                 xv += dv[q][e];
               }
@@ -515,7 +573,8 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) ls_fused_step_kernel(const __gr
           }
         }
       }
-      __syncthreads();
+      if (tid == 0) FZ_STAMP(1, 30);
+      named_bar_sync(1, FZ_THREADS);
       if (A.has_next) {
         for (int t = tid; t < (K + 1) * 3; t += FZ_THREADS) {
           const int j = t / 3, e = t - j * 3;
@@ -525,12 +584,12 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) ls_fused_step_kernel(const __gr
           if (e < 2) {
             const int row = cta + (a0 + e) * G;
             if (a0 + e < lay.nA && row < r) A.z[(size_t)j * r + row] = v;
-          } else if (cta == 0 && pr == 0) {
+          } else if (j == sq_eval) {
             A.sumsq[j] = v;
           }
         }
       }
-      __syncthreads();
+      named_bar_sync(1, FZ_THREADS);
     }
   }
 
@@ -538,7 +597,7 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) ls_fused_step_kernel(const __gr
 #pragma unroll
     for (int q = 0; q < XC; ++q) {
       const int c = tid + q * FZ_THREADS;
-      if (c < d) A.x_out[c] = xfin[q];
+      if (c < d) A.x_out[c] = s_xfin[c];
     }
   }
   if (A.has_next) {
@@ -550,7 +609,7 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) ls_fused_step_kernel(const __gr
 #pragma unroll
       for (int q = 0; q < XC; ++q) {
         const int c = tid + q * FZ_THREADS;
-        if (c < d) A.x_out[c] = xfin[q];
+        if (c < d) A.x_out[c] = s_xfin[c];
       }
     }
 
@@ -571,17 +630,22 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) ls_fused_step_kernel(const __gr
     const int RSB = r + FZ_BPAD, RSZ = r + FZ_ZPAD;
     const int n_mt = (n_own + 7) >> 3;
     for (int n0 = 0; n0 <= K; n0 += 8) {
-      __syncthreads();  // the previous eight latents are no longer read
-      for (int t = tid; t < 8 * r; t += FZ_THREADS) {
-        const int e = t / r, jj = t - e * r, j = n0 + e;
-        double v = 0.0;
-        if (j <= K) {
-          const double inv = A.norm_n == 0 ? 1.0 / sqrt(__ldcg(&A.sumsq[j]) / (double)d + (double)A.eps_n) : 1.0;
-          v = __ldcg(&A.z[(size_t)j * r + jj]) * inv;
-        }
-        s_zs[e * RSZ + jj] = v;
+      named_bar_sync(1, FZ_THREADS);  // the previous eight latents are no longer read
+      if (tid < 8) {  // 1 / rms of the eight features, once each
+        const int j = n0 + tid;
+        s_inv[tid] = (j <= K && A.norm_n == 0) ? 1.0 / sqrt(__ldcg(&A.sumsq[j]) / (double)d + (double)A.eps_n) : 1.0;
       }
-      __syncthreads();
+      for (int t = tid; t < 8 * r; t += FZ_THREADS) {  // fetched before the scale factors are ready
+        const int e = t / r, jj = t - e * r, j = n0 + e;
+        s_zs[e * RSZ + jj] = j <= K ? __ldcg(&A.z[(size_t)j * r + jj]) : 0.0;
+      }
+      named_bar_sync(1, FZ_THREADS);
+      for (int t = tid; t < 8 * r; t += FZ_THREADS) {
+        const int e = t / r, jj = t - e * r;
+        s_zs[e * RSZ + jj] *= s_inv[e];
+      }
+      named_bar_sync(1, FZ_THREADS);
+      if (tid == 0) FZ_STAMP(1, 40 + n0 / 8 * 2);
       for (int mt = warp; mt < n_mt; mt += FZ_THREADS / 32) {
         const uint16_t* arow = s_B + (size_t)(mt * 8 + (lane >> 2)) * RSB + (lane & 3);
         const double* brow = s_zs + (size_t)(lane >> 2) * RSZ + (lane & 3);
@@ -592,6 +656,7 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) ls_fused_step_kernel(const __gr
           asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};" : "+d"(c0), "+d"(c1) : "d"(a0v), "d"(b0v));
           asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};" : "+d"(e0), "+d"(e1) : "d"(a1v), "d"(b1v));
         }
+        if (tid == 0) FZ_STAMP(1, 41 + n0 / 8 * 2);
         const int li = mt * 8 + (lane >> 2);
         const int j = n0 + (lane & 3) * 2;
         if (li < n_own) {
@@ -600,9 +665,14 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) ls_fused_step_kernel(const __gr
         }
       }
     }
-    __syncthreads();
-    // histogram (fine + coarse) and bucket insert: one thread per (evaluation, neuron), all atomics in flight together
+    named_bar_sync(1, FZ_THREADS);
+    if (tid == 0) FZ_STAMP(1, 50);
+    // histogram (fine + coarse) and bucket insert: one thread per (evaluation, neuron), all atomics in flight together;
+    // the coarse counts of the CTA are summed in shared memory first (they are hot addresses for the whole grid)
     {
+      for (int t = tid; t < (K + 1) * FZ_NC; t += FZ_THREADS) s_ccnt[t] = 0u;
+      if (tid < FZ_MAXE) s_nsel[tid] = 0u;
+      named_bar_sync(1, FZ_THREADS);
       unsigned long long kmin = 0xffffffffffffffffULL, kmax = 0ULL;
       for (int t = tid; t < (K + 1) * n_own; t += FZ_THREADS) {
         const int j = t / n_own, li = t - j * n_own, i = i_lo + li;
@@ -612,16 +682,14 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) ls_fused_step_kernel(const __gr
         bb = max(0, min(FZ_NB - 1, bb));
         unsigned* cnt = A.cnt + (size_t)j * FZ_CNT_STRIDE;
         const unsigned slot = atomicAdd(&cnt[bb], 1u);
-        atomicAdd(&cnt[FZ_NB + bb / (FZ_NB / FZ_NC)], 1u);
+        atomicAdd(&s_ccnt[j * FZ_NC + bb / (FZ_NB / FZ_NC)], 1u);
         const unsigned long long key = ordered_key(sv);
+        const uint4 ent = make_uint4((unsigned)key, (unsigned)(key >> 32), (unsigned)i, (unsigned)bb);
         if (slot < (unsigned)FZ_CAPB) {
-          A.bkey[((size_t)j * FZ_NB + bb) * FZ_CAPB + slot] = key;
-          A.bidx[((size_t)j * FZ_NB + bb) * FZ_CAPB + slot] = i;
+          A.bent[((size_t)j * FZ_NB + bb) * FZ_CAPB + slot] = ent;
         } else {
           const unsigned o = atomicAdd(&cnt[FZ_NB + FZ_NC], 1u);
-          A.okey[(size_t)j * Fn + o] = key;
-          A.oidx[(size_t)j * Fn + o] = i;
-          A.obin[(size_t)j * Fn + o] = bb;
+          A.oent[(size_t)j * Fn + o] = ent;
         }
         s_bin[(size_t)j * per + li] = (uint16_t)bb;
         if (j == K) {
@@ -636,9 +704,18 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) ls_fused_step_kernel(const __gr
         kmin = min(kmin, __shfl_xor_sync(0xffffffffu, kmin, o));
         kmax = max(kmax, __shfl_xor_sync(0xffffffffu, kmax, o));
       }
-      if (lane == 0 && kmin <= kmax) {  // observed score range of the final evaluation: one pair of atomics per warp
-        atomicMin(&A.range_obs[0], kmin);
-        atomicMax(&A.range_obs[1], kmax);
+      if (lane == 0) { s_kmm[warp] = kmin; s_kmm[16 + warp] = kmax; }
+      named_bar_sync(1, FZ_THREADS);
+      for (int t = tid; t < (K + 1) * FZ_NC; t += FZ_THREADS) {
+        const unsigned v = s_ccnt[t];
+        if (v) atomicAdd(&A.cnt[(size_t)(t / FZ_NC) * FZ_CNT_STRIDE + FZ_NB + (t % FZ_NC)], v);
+      }
+      if (tid == 0) {  // observed score range of the final evaluation: one pair of atomics per CTA
+        for (int w = 1; w < 16; ++w) { kmin = min(kmin, s_kmm[w]); kmax = max(kmax, s_kmm[16 + w]); }
+        if (kmin <= kmax) {
+          atomicMin(&A.range_obs[0], kmin);
+          atomicMax(&A.range_obs[1], kmax);
+        }
       }
     }
 
@@ -647,11 +724,15 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) ls_fused_step_kernel(const __gr
     grid_barrier(A, G);
     if (tid == 0) FZ_STAMP(1, 5);
 
-    // ============================ phase 4: exact ranks, every evaluation ============================================
-    // coarse exclusive prefix per evaluation: warp w handles evaluations w, w+16, ... (two coarse bins per lane)
+    // ============================ phase 4: refined sets of every evaluation, exact ranks of the final one ============
+    // Per evaluation (one warp each): coarse prefix -> the coarse bin holding rank keff -> its fine counts -> the CUT
+    // fine bin, the rank b0 where it starts and the threshold entry inside it (the last member).  With that in shared
+    // memory every neuron's membership is decided locally: bins before the cut bin are in, bins after it are out, the
+    // cut bin is split by one comparison.  Exact ranks (bucket comparisons) are needed only for the final selection.
+    constexpr int FPC = FZ_NB / FZ_NC;  // fine bins per coarse bin
     for (int j = warp; j <= K; j += FZ_THREADS / 32) {
-      const unsigned* cc = A.cnt + (size_t)j * FZ_CNT_STRIDE + FZ_NB;
-      const unsigned c0 = __ldcg(&cc[lane * 2]), c1 = __ldcg(&cc[lane * 2 + 1]);
+      const unsigned* cnt = A.cnt + (size_t)j * FZ_CNT_STRIDE;
+      const unsigned c0 = __ldcg(&cnt[FZ_NB + lane * 2]), c1 = __ldcg(&cnt[FZ_NB + lane * 2 + 1]);
       unsigned incl = c0 + c1;
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
@@ -662,70 +743,216 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) ls_fused_step_kernel(const __gr
       s_coarse[j * (FZ_NC + 1) + lane * 2] = ex;
       s_coarse[j * (FZ_NC + 1) + lane * 2 + 1] = ex + c0;
       if (lane == 31) s_coarse[j * (FZ_NC + 1) + FZ_NC] = incl;
+      // coarse bin that holds rank keff-1 (none when keff == 0)
+      int cbsel = -1;
+      if (c0 > 0 && (int)ex < keff && (int)(ex + c0) >= keff) cbsel = lane * 2;
+      if (c1 > 0 && (int)(ex + c0) < keff && (int)incl >= keff) cbsel = lane * 2 + 1;
+      const unsigned vote = __ballot_sync(0xffffffffu, cbsel >= 0);
+      int cut_bin = -1, cut_b0 = 0, cut_need = 0, cut_fallback = 0, t_idx = -1;  // no cut bin: keff == 0, nothing is selected
+      unsigned long long t_key = 0ULL;
+      if (vote) {
+        const int src = __ffs(vote) - 1;
+        const int cb = __shfl_sync(0xffffffffu, cbsel, src);
+        const unsigned cbase = __shfl_sync(0xffffffffu, (cbsel & 1) ? ex + c0 : ex, src);
+        // fine counts of that coarse bin: two per lane
+        const unsigned f0 = __ldcg(&cnt[cb * FPC + lane * 2]), f1 = __ldcg(&cnt[cb * FPC + lane * 2 + 1]);
+        unsigned fin = f0 + f1;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const unsigned t = __shfl_up_sync(0xffffffffu, fin, o);
+          if (lane >= o) fin += t;
+        }
+        const unsigned fex = cbase + fin - (f0 + f1);
+        int fsel = -1;
+        unsigned fb0 = 0, fnb = 0;
+        if (f0 > 0 && (int)fex < keff && (int)(fex + f0) >= keff) { fsel = lane * 2; fb0 = fex; fnb = f0; }
+        if (f1 > 0 && (int)(fex + f0) < keff && (int)(fex + f0 + f1) >= keff) { fsel = lane * 2 + 1; fb0 = fex + f0; fnb = f1; }
+        const unsigned fvote = __ballot_sync(0xffffffffu, fsel >= 0);
+        const int fsrc = __ffs(fvote) - 1;  // exists: the coarse bin holds rank keff-1
+        cut_bin = cb * FPC + __shfl_sync(0xffffffffu, fsel, fsrc);
+        cut_b0 = (int)__shfl_sync(0xffffffffu, fb0, fsrc);
+        const int nbc = (int)__shfl_sync(0xffffffffu, fnb, fsrc);
+        cut_need = keff - cut_b0;  // members inside the cut bin, 1 <= need <= nbc
+        if (nbc > FZ_CAPB) {
+          cut_fallback = 1;        // overflowed bucket: its neurons compare against bucket + overflow list themselves
+        } else {
+          // threshold = the entry with exactly need-1 entries before it
+          uint4 ent = make_uint4(0, 0, 0, 0);
+          if (lane < nbc) ent = __ldcg(&A.bent[((size_t)j * FZ_NB + cut_bin) * FZ_CAPB + lane]);
+          const unsigned long long kmine = ((unsigned long long)ent.y << 32) | ent.x;
+          int before = 0;
+#pragma unroll
+          for (int q = 0; q < FZ_CAPB; ++q) {
+            const unsigned long long kq = ((unsigned long long)__shfl_sync(0xffffffffu, ent.y, q) << 32) | __shfl_sync(0xffffffffu, ent.x, q);
+            const int iq = (int)__shfl_sync(0xffffffffu, ent.z, q);
+            before += (q < nbc) && ((kq > kmine) || (kq == kmine && iq < (int)ent.z));
+          }
+          const unsigned tv = __ballot_sync(0xffffffffu, lane < nbc && before == cut_need - 1);
+          const int ts = __ffs(tv) - 1;
+          t_key = ((unsigned long long)__shfl_sync(0xffffffffu, ent.y, ts) << 32) | __shfl_sync(0xffffffffu, ent.x, ts);
+          t_idx = (int)__shfl_sync(0xffffffffu, ent.z, ts);
+        }
+      }
+      if (lane == 0) {
+        s_cut[j * 4 + 0] = cut_bin;
+        s_cut[j * 4 + 1] = cut_b0;
+        s_cut[j * 4 + 2] = t_idx;
+        s_cut[j * 4 + 3] = cut_fallback;
+        s_cutkey[j] = t_key;
+      }
     }
-    __syncthreads();
-    constexpr int FPC = FZ_NB / FZ_NC;  // fine bins per coarse bin
+    named_bar_sync(1, FZ_THREADS);
+    if (tid == 0) FZ_STAMP(1, 60);
+    if (lane == 0) FZ_STAMP(1, 100 + warp * 4);
     for (int t = tid; t < (K + 1) * n_own; t += FZ_THREADS) {
+      if (lane == 0) FZ_STAMP(1, 101 + warp * 4 + t / FZ_THREADS);
       const int j = t / n_own, li = t - j * n_own, i = i_lo + li;
       const int bb = s_bin[(size_t)j * per + li];
-      const int cb = bb / FPC;
-      const unsigned cbase = s_coarse[j * (FZ_NC + 1) + cb];
-      if ((int)cbase >= keff) continue;  // every neuron of this coarse bin ranks behind the cut
-      const unsigned* cnt = A.cnt + (size_t)j * FZ_CNT_STRIDE;
-      // fine prefix inside the coarse bin: all its counts are fetched with independent 128-bit loads
-      unsigned b0 = cbase, nb = 0;
-#pragma unroll
-      for (int q = 0; q < FPC; q += 4) {
-        const uint4 v = __ldcg(reinterpret_cast<const uint4*>(cnt + cb * FPC + q));
-        const unsigned cv[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const int fb = cb * FPC + q + u;
-          b0 += fb < bb ? cv[u] : 0u;
-          nb = fb == bb ? cv[u] : nb;
-        }
-      }
-      if ((int)b0 >= keff) continue;
-      const unsigned novf = nb > (unsigned)FZ_CAPB ? __ldcg(&cnt[FZ_NB + FZ_NC]) : 0u;
-      nb = min(nb, (unsigned)FZ_CAPB);
+      const int cut_bin = s_cut[j * 4 + 0];
+      if (bb > cut_bin) continue;  // behind the cut
       const unsigned long long kp = ordered_key(s_own[(size_t)j * per + li]);
-      int before = 0;
-      const size_t bo = ((size_t)j * FZ_NB + bb) * FZ_CAPB;
-      {  // the whole bucket is fetched with independent 128-bit loads; entries beyond nb are ignored
-        unsigned long long kq[FZ_CAPB];
-        int iq[FZ_CAPB];
-#pragma unroll
-        for (int q = 0; q < FZ_CAPB; q += 2) {
-          const uint4 v = __ldcg(reinterpret_cast<const uint4*>(A.bkey + bo + q));
-          kq[q] = ((unsigned long long)v.y << 32) | v.x;
-          kq[q + 1] = ((unsigned long long)v.w << 32) | v.z;
-        }
-#pragma unroll
-        for (int q = 0; q < FZ_CAPB; q += 4) {
-          const int4 v = __ldcg(reinterpret_cast<const int4*>(A.bidx + bo + q));
-          iq[q] = v.x; iq[q + 1] = v.y; iq[q + 2] = v.z; iq[q + 3] = v.w;
-        }
-#pragma unroll
-        for (int q = 0; q < FZ_CAPB; ++q)
-          before += ((unsigned)q < nb) && ((kq[q] > kp) || (kq[q] == kp && iq[q] < i));
+      const unsigned* cnt = A.cnt + (size_t)j * FZ_CNT_STRIDE;
+      bool member = true;
+      int rank = -1;
+      if (bb == cut_bin && !s_cut[j * 4 + 3]) {
+        const unsigned long long tk = s_cutkey[j];
+        member = (kp > tk) || (kp == tk && i <= s_cut[j * 4 + 2]);
       }
-      for (unsigned q = 0; q < novf; ++q) {  // only when this neuron's own bin overflowed its bucket
-        if (__ldcg(&A.obin[(size_t)j * Fn + q]) != bb) continue;
-        const unsigned long long kq = __ldcg(&A.okey[(size_t)j * Fn + q]);
-        const int iq = __ldcg(&A.oidx[(size_t)j * Fn + q]);
-        before += (kq > kp) || (kq == kp && iq < i);
-      }
-      const int rank = (int)b0 + before;
-      if (rank < keff) {
-        if (j == K) {
-          if (rank < A.next_cap) A.next_idx[rank] = i;
-          if (A.next_mask) atomicOr(&A.next_mask[i >> 5], 1u << (i & 31));
-        } else {
-          A.tmp_idx[rank] = i;
+      if (j == K) continue;  // the final evaluation is ranked bin by bin below
+      if (bb == cut_bin && s_cut[j * 4 + 3]) {
+        // exact rank: fine prefix inside the coarse bin + comparison inside the neuron's bucket
+        const int cb = bb / FPC;
+        unsigned b0 = s_coarse[j * (FZ_NC + 1) + cb], nb = 0;
+#pragma unroll
+        for (int q = 0; q < FPC; q += 4) {
+          const uint4 v = __ldcg(reinterpret_cast<const uint4*>(cnt + cb * FPC + q));
+          const unsigned cv[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const int fb = cb * FPC + q + u;
+            b0 += fb < bb ? cv[u] : 0u;
+            nb = fb == bb ? cv[u] : nb;
+          }
         }
+        const unsigned novf = nb > (unsigned)FZ_CAPB ? __ldcg(&cnt[FZ_NB + FZ_NC]) : 0u;
+        nb = min(nb, (unsigned)FZ_CAPB);
+        int before = 0;
+        const uint4* bk = A.bent + ((size_t)j * FZ_NB + bb) * FZ_CAPB;
+        uint4 ent[FZ_CAPB];
+#pragma unroll
+        for (int q = 0; q < FZ_CAPB; ++q) ent[q] = __ldcg(bk + q);
+#pragma unroll
+        for (int q = 0; q < FZ_CAPB; ++q) {
+          const unsigned long long kq = ((unsigned long long)ent[q].y << 32) | ent[q].x;
+          before += ((unsigned)q < nb) && ((kq > kp) || (kq == kp && (int)ent[q].z < i));
+        }
+        for (unsigned q = 0; q < novf; ++q) {  // only when this neuron's own bin overflowed its bucket
+          const uint4 e = __ldcg(&A.oent[(size_t)j * Fn + q]);
+          if ((int)e.w != bb) continue;
+          const unsigned long long kq = ((unsigned long long)e.y << 32) | e.x;
+          before += (kq > kp) || (kq == kp && (int)e.z < i);
+        }
+        rank = (int)b0 + before;
+        member = rank < keff;
+      }
+      if (member) {
         if (A.tr_masks) atomicOr(&A.tr_masks[(size_t)j * ((Fn + 31) >> 5) + (i >> 5)], 1u << (i & 31));
+        atomicAdd(&s_nsel[j], 1u);
       }
     }
+    // Final evaluation: exact ranks, bin by bin.  A task is a pair of fine bins; the tasks up to the cut are dealt to
+    // the warps of the whole grid.  A half-warp takes one fine bin: its bucket arrives with one
+    // coalesced load, the order inside the bin comes from 16 shuffles, rank = first rank of the bin + entries before.
+    {
+      const int j = K;
+      const unsigned* cnt = A.cnt + (size_t)j * FZ_CNT_STRIDE;
+      const int cut_bin = s_cut[j * 4 + 0];
+      const int n_task = cut_bin >= 0 ? (cut_bin / 2 + 1) : 0;  // one task = two fine bins (one per half-warp)
+      const unsigned novf = __ldcg(&cnt[FZ_NB + FZ_NC]);
+      const int h = lane >> 4, l16 = lane & 15;
+      // task t goes to CTA t % G, warp (t / G) % 16: spread over the whole grid, at most a few per warp
+      for (int task = cta + warp * G; task < n_task; task += G * (FZ_THREADS / 32)) {
+        const int fbq = task * 2, cb = fbq / FPC;  // first fine bin of the task, its coarse bin
+        // fine counts of the coarse bin (two per lane) and their exclusive prefix
+        const unsigned f0 = __ldcg(&cnt[cb * FPC + lane * 2]), f1 = __ldcg(&cnt[cb * FPC + lane * 2 + 1]);
+        unsigned fin = f0 + f1;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const unsigned t = __shfl_up_sync(0xffffffffu, fin, o);
+          if (lane >= o) fin += t;
+        }
+        const unsigned fex = s_coarse[j * (FZ_NC + 1) + cb] + fin - (f0 + f1);  // first rank of fine bin cb*64 + 2*lane
+        for (int it = 0; it < 1; ++it) {
+          const int bin = fbq + h;
+          const int src = (bin - cb * FPC) >> 1, odd = (bin - cb * FPC) & 1;
+          const unsigned pf0 = __shfl_sync(0xffffffffu, f0, src), pf1 = __shfl_sync(0xffffffffu, f1, src);
+          const unsigned pex = __shfl_sync(0xffffffffu, fex, src);
+          const unsigned b0 = odd ? pex + pf0 : pex, nball = odd ? pf1 : pf0;
+          const int nb = (int)min(nball, (unsigned)FZ_CAPB);
+          uint4 ent = make_uint4(0, 0, 0, 0);
+          if (l16 < nb && (int)b0 < keff) ent = __ldcg(&A.bent[((size_t)j * FZ_NB + bin) * FZ_CAPB + l16]);
+          const unsigned long long kmine = ((unsigned long long)ent.y << 32) | ent.x;
+          int before = 0;
+#pragma unroll
+          for (int q = 0; q < FZ_CAPB; ++q) {
+            const unsigned long long kq = ((unsigned long long)__shfl_sync(0xffffffffu, ent.y, q, 16) << 32) | __shfl_sync(0xffffffffu, ent.x, q, 16);
+            const int iq = (int)__shfl_sync(0xffffffffu, ent.z, q, 16);
+            before += (q < nb) && ((kq > kmine) || (kq == kmine && iq < (int)ent.z));
+          }
+          if ((int)b0 >= keff) continue;  // (uniform per half-warp; the shuffles above were executed by all lanes)
+          if (nball > (unsigned)FZ_CAPB) {
+            // overflowed bin (rare): bucket entries also count the overflow entries before them ...
+            for (unsigned q = 0; q < novf; ++q) {
+              const uint4 e = __ldcg(&A.oent[(size_t)j * Fn + q]);
+              if ((int)e.w != bin) continue;
+              const unsigned long long kq = ((unsigned long long)e.y << 32) | e.x;
+              before += (l16 < nb) && ((kq > kmine) || (kq == kmine && (int)e.z < (int)ent.z));
+            }
+            // ... and one lane ranks the overflow entries of the bin themselves
+            if (l16 == 0) {
+              for (unsigned q = 0; q < novf; ++q) {
+                const uint4 e = __ldcg(&A.oent[(size_t)j * Fn + q]);
+                if ((int)e.w != bin) continue;
+                const unsigned long long ke = ((unsigned long long)e.y << 32) | e.x;
+                int bf = 0;
+                for (int u = 0; u < FZ_CAPB; ++u) {
+                  const uint4 o = __ldcg(&A.bent[((size_t)j * FZ_NB + bin) * FZ_CAPB + u]);
+                  const unsigned long long ko = ((unsigned long long)o.y << 32) | o.x;
+                  bf += (ko > ke) || (ko == ke && (int)o.z < (int)e.z);
+                }
+                for (unsigned u = 0; u < novf; ++u) {
+                  const uint4 o = __ldcg(&A.oent[(size_t)j * Fn + u]);
+                  if ((int)o.w != bin) continue;
+                  const unsigned long long ko = ((unsigned long long)o.y << 32) | o.x;
+                  bf += (ko > ke) || (ko == ke && (int)o.z < (int)e.z);
+                }
+                const int rk = (int)b0 + bf;
+                if (rk < keff) {
+                  const int i = (int)e.z;
+                  if (rk < A.next_cap) A.next_idx[rk] = i;
+                  if (A.next_mask) atomicOr(&A.next_mask[i >> 5], 1u << (i & 31));
+                  if (A.tr_masks) atomicOr(&A.tr_masks[(size_t)j * ((Fn + 31) >> 5) + (i >> 5)], 1u << (i & 31));
+                  atomicAdd(&s_nsel[j], 1u);
+                }
+              }
+            }
+          }
+          const int rank = (int)b0 + before;
+          if (l16 < nb && rank < keff) {
+            const int i = (int)ent.z;
+            if (rank < A.next_cap) A.next_idx[rank] = i;
+            if (A.next_mask) atomicOr(&A.next_mask[i >> 5], 1u << (i & 31));
+            if (A.tr_masks) atomicOr(&A.tr_masks[(size_t)j * ((Fn + 31) >> 5) + (i >> 5)], 1u << (i & 31));
+            atomicAdd(&s_nsel[j], 1u);
+          }
+        }
+      }
+    }
+    if (lane == 0) FZ_STAMP(1, 103 + warp * 4);
+    named_bar_sync(1, FZ_THREADS);
+    // refined-set sizes: every evaluation must have selected exactly keff neurons (checked on the device)
+    for (int j = tid; j <= K; j += FZ_THREADS)
+      if (s_nsel[j]) atomicAdd(&A.nsel[j], s_nsel[j]);
     if (cta == 0 && tid == 0) {
       if (A.tr_counts)
         for (int j = 0; j <= K; ++j) A.tr_counts[j] = keff;
@@ -736,17 +963,22 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) ls_fused_step_kernel(const __gr
   }
 
   // ---- the last CTA to finish restores the zero-on-entry invariants of the per-layer scratch
-  __syncthreads();
+  named_bar_sync(1, FZ_THREADS);
+  if (tid == 0) FZ_STAMP(1, 70);
   if (tid == 0) {
     __threadfence();
     s_last = (atomicAdd(A.fin, 1u) == (unsigned)G - 1u) ? 1 : 0;
   }
-  __syncthreads();
+  named_bar_sync(1, FZ_THREADS);
   if (s_last) {
     __threadfence();
     for (int t = tid; t < K * d; t += FZ_THREADS) A.dacc[t] = 0.f;
     if (A.has_next) {
       for (int t = tid; t < (K + 1) * FZ_CNT_STRIDE; t += FZ_THREADS) A.cnt[t] = 0u;
+      if (tid <= K) {  // self-check: every refined set has exactly min(k_next, d_ff) members
+        if ((int)A.nsel[tid] != min(A.k_next, A.Fn)) set_status(A.status, ST_INTERNAL);
+        A.nsel[tid] = 0u;
+      }
       if (tid == 0) {
         // binning range for the next launch: what the final evaluation observed, widened by 5 % on each side
         const unsigned long long kmin = A.range_obs[0], kmax = A.range_obs[1];
@@ -768,6 +1000,7 @@ __global__ void __launch_bounds__(FZ_THREADS, 1) ls_fused_step_kernel(const __gr
     }
     if (tid == 0) *A.fin = 0u;
   }
+  if (tid == 0) FZ_STAMP(1, 71);
 }
 
 }  // namespace ls
