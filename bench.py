@@ -41,6 +41,7 @@ def parse_args():
     ap.add_argument("--chunks", type=int, default=8, help="K: stages per layer (Section 4.3.1 of the paper uses 8)")
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (debugging only)")
     ap.add_argument("--no-graph", action="store_true", help="launch every call from the host instead of one CUDA graph per token")
+    ap.add_argument("--per-layer", action="store_true", help="one fused kernel per layer (ls_sparse_ffn_step) instead of the whole-token kernel")
     ap.add_argument("--cpu-sample-layers", type=int, default=2)
     return ap.parse_args()
 
@@ -216,11 +217,19 @@ def run_ours(args):
     out_host = torch.zeros(1, d, dtype=torch.float32).pin_memory()
     sels = [ls.Selection(spec.d_ff, k, local) for _ in range(2)]
 
-    def decode_token():
+    stack = None if args.per_layer else ls.ls_stack_create(layers)
+
+    def decode_token_layers():
         ls.ls_predict(layers[0], x_buf, k, sels[0])
         for n in range(n_layers):
             nxt = layers[n + 1] if n + 1 < n_layers else layers[n]
             ls.ls_sparse_ffn_step(layers[n], nxt, x_buf, x_buf, sels[n % 2], K, k, sels[(n + 1) % 2], None)
+
+    def decode_token():
+        if stack is None:
+            return decode_token_layers()
+        ls.ls_predict(layers[0], x_buf, k, sels[0])
+        ls.ls_stack_decode(stack, x_buf, x_buf, sels[0], K, k, sels[1])
 
     # ---- warm-up, launch count per token, optional CUDA graph of one token
     x_buf.copy_(X0[0:1])
@@ -278,6 +287,7 @@ def run_ours(args):
             decode_token()
         torch.cuda.synchronize()
         ls.ls_timing_enable(False)
+        n_st, ms_st = ls.ls_timing_read(ls.LS_TIMED_STACK)
         n_fz, ms_fz = ls.ls_timing_read(ls.LS_TIMED_FUSED)
         n_gu, ms_gu = ls.ls_timing_read(ls.LS_TIMED_GATEUP)
         n_dn, ms_dn = ls.ls_timing_read(ls.LS_TIMED_DOWN)
@@ -303,7 +313,12 @@ def run_ours(args):
         if os.path.exists(tp):
             with open(tp) as f:
                 traffic_db = json.load(f)
-        if n_fz:
+        if n_st:
+            # one launch = one token = n_layers layer steps: algorithmic bytes are the active-neuron bytes of all layers
+            kname, bytes_launch, us_launch, n_timed = "ls_fused_stack_kernel", active_bytes_layer * n_layers, ms_st / n_st * 1e3, n_st
+            per_layer_traffic = traffic_db.get("stack_dram_bytes_per_layer")
+            traffic = per_layer_traffic * n_layers if per_layer_traffic else None
+        elif n_fz:
             # the whole layer step is one kernel: its algorithmic bytes are the active-neuron bytes of the layer
             kname, bytes_launch, us_launch, n_timed = "ls_fused_step_kernel", active_bytes_layer, ms_fz / n_fz * 1e3, n_fz
             traffic = traffic_db.get("fused_dram_bytes_per_launch")
@@ -328,7 +343,7 @@ def run_ours(args):
             "config": {"workload": spec.name, "n_layers": n_layers, "d_model": d, "d_ff": spec.d_ff, "pred_rank": spec.rank, "k": k,
                        "chunks": K, "batch": 1, "parallelism": "replicas only" if world > 1 else "1 gpu",
                        "l2": "inputs larger than L2 (%.2f GB of weight rows touched per token)" % (active_bytes_layer * n_layers / 1e9),
-                       "cuda_graph": graph is not None},
+                       "cuda_graph": graph is not None, "kernel_per": "layer" if stack is None else "token"},
             "us_per_layer": us_layer, "active_bytes_per_layer": active_bytes_layer, "k_surviving_mean": k_surv,
             "active_gbs": active_gbs, "active_frac_of_hbm_peak": active_gbs / peaks["hbm_gbs"],
             "roofline": {"bound": "hbm", "kernel": kname, "achieved": k_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
@@ -343,6 +358,8 @@ def run_ours(args):
             "clocks": clocks, "build_s": t_build,
         }
         print(json.dumps(line))
+    if stack is not None:
+        stack.close()
     for L in layers:
         L.close()
     if world > 1:

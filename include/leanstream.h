@@ -190,6 +190,34 @@ int32_t ls_cache_stats(ls_layer *layer, ls_cache_stats_t *host_out);
 int32_t ls_layer_status(ls_layer *layer, int32_t *host_status);
 
 /*
+ * Whole-token decode of a stack of fully resident layers (Section 2.1 applied layer after layer: x_{n+1} = x~_n^(K), and
+ * the final refined set C^(K) of layer n is the selection of layer n+1).  ls_stack_decode runs every layer's
+ * speculate-and-refine step (exactly what ls_sparse_ffn_step computes at batch 1) inside ONE cooperative kernel, so a
+ * layer boundary costs a grid barrier instead of a kernel launch.  The last layer refines a weight-tied copy of itself.
+ *
+ * ls_stack_create: `layers` (HOST array of n_layers handles) must be resident (cache_rows = 0), on one device, with one
+ *   d_model and one weight type; the handles are borrowed and must outlive the stack.  LS_ERR_STATE if a layer does not
+ *   qualify.  The stack owns small device buffers (per-layer argument table, residual and selection ping-pong).
+ * ls_stack_decode: d_x, d_x_out float [d_model] (may alias); sel_first = selection of layer 0 in rank order (from
+ *   ls_predict); n_chunks in [1, 16]; sel_out receives the final refined set of the last layer (idx, count required;
+ *   mask, scores optional).  `trace` (nullable) exports, for checking: x [n_layers+1][d_model], the residual entering each
+ *   layer and leaving the last (needs d_x != d_x_out); sel_idx [n_layers+1][sel_cap] / sel_count [n_layers+1], the
+ *   selection entering each layer and the final refined one.  Never synchronises or allocates; may be captured in a CUDA
+ *   graph.  Like every fused step, calls on one device must not overlap (they share one scratch).
+ */
+typedef struct ls_stack ls_stack;
+typedef struct {
+  float *x;
+  int32_t *sel_idx;
+  int32_t *sel_count;
+  int32_t sel_cap;
+} ls_stack_trace;
+int32_t ls_stack_create(ls_layer *const *layers, int32_t n_layers, ls_stack **out);
+int32_t ls_stack_destroy(ls_stack *stack);
+int32_t ls_stack_decode(ls_stack *stack, const float *d_x, float *d_x_out, const ls_selection *sel_first, int32_t n_chunks,
+                        int32_t k_next, ls_selection *sel_out, ls_stack_trace *trace, void *stream);
+
+/*
  * Top-k selection that allocates nothing (the paper has no counterpart; it exists for callers that must not allocate).
  *
  * Some callers cannot call cudaMalloc or anything that may call it for them: code running while a stream is being
@@ -220,6 +248,7 @@ int32_t ls_topk_select_static(const double *d_scores, int32_t n, int32_t k, int3
  * streaming and refinement overlap; 0 forces the stage-by-stage kernels, which compute the same thing.  With the fused
  * kernel the partial outputs of different SMs are combined with floating-point atomics, so the low bits of x~^(j) may
  * differ between two runs; the selected sets are always the exact top-k of the features that were actually produced.
+ * Fused steps use one working scratch per device: issue them on one stream, or order the streams that issue them.
  */
 #define LS_OPT_FUSED 1
 int32_t ls_set_option(int32_t option, int32_t value);
@@ -234,6 +263,7 @@ int32_t ls_set_option(int32_t option, int32_t value);
 #define LS_TIMED_DOWN 1    /* sparse down projection of one stage */
 #define LS_TIMED_PREDICT 2 /* latent + scores + top-k of one predictor evaluation */
 #define LS_TIMED_FUSED 3   /* the fused per-layer step kernel */
+#define LS_TIMED_STACK 4   /* the whole-token kernel of ls_stack_decode */
 int32_t ls_timing_enable(int32_t on);
 int32_t ls_timing_read(int32_t kind, int64_t *launches, double *total_ms);
 

@@ -22,7 +22,8 @@ LS_NORM_RMS, LS_NORM_NONE = 0, 1
 EXPORTS = [
     "ls_layer_create", "ls_layer_destroy", "ls_predict", "ls_sparse_ffn_step", "ls_cache_lookup", "ls_cache_reserve",
     "ls_cache_evict", "ls_cache_snapshot", "ls_cache_wait", "ls_cache_stats", "ls_layer_status", "ls_kernel_launches",
-    "ls_last_error", "ls_version", "ls_timing_enable", "ls_timing_read", "ls_set_option", "ls_topk_select_static",
+    "ls_last_error", "ls_version", "ls_timing_enable", "ls_timing_read", "ls_set_option", "ls_topk_select_static", "ls_stack_create",
+    "ls_stack_destroy", "ls_stack_decode",
 ]
 
 
@@ -49,6 +50,10 @@ class ls_selection(C.Structure):
 class ls_step_trace(C.Structure):
     _fields_ = [("xtilde", C.c_void_p), ("refine_masks", C.c_void_p), ("refine_counts", C.c_void_p),
                 ("survive_mask", C.c_void_p), ("exec_idx", C.c_void_p)]
+
+
+class ls_stack_trace(C.Structure):
+    _fields_ = [("x", C.c_void_p), ("sel_idx", C.c_void_p), ("sel_count", C.c_void_p), ("sel_cap", C.c_int32)]
 
 
 class ls_cache_stats_t(C.Structure):
@@ -83,6 +88,10 @@ def lib() -> C.CDLL:
         L.ls_cache_stats.argtypes = [C.c_void_p, C.POINTER(ls_cache_stats_t)]
         L.ls_layer_status.argtypes = [C.c_void_p, C.POINTER(C.c_int32)]
         L.ls_set_option.argtypes = [C.c_int32, C.c_int32]
+        L.ls_stack_create.argtypes = [C.POINTER(C.c_void_p), C.c_int32, C.POINTER(C.c_void_p)]
+        L.ls_stack_destroy.argtypes = [C.c_void_p]
+        L.ls_stack_decode.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(ls_selection), C.c_int32, C.c_int32,
+                                      C.POINTER(ls_selection), C.POINTER(ls_stack_trace), C.c_void_p]
         L.ls_topk_select_static.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.ls_timing_enable.argtypes = [C.c_int32]
         L.ls_timing_read.argtypes = [C.c_int32, C.POINTER(C.c_int64), C.POINTER(C.c_double)]
@@ -283,7 +292,7 @@ def ls_version() -> int:
     return int(lib().ls_version())
 
 
-LS_TIMED_GATEUP, LS_TIMED_DOWN, LS_TIMED_PREDICT, LS_TIMED_FUSED = 0, 1, 2, 3
+LS_TIMED_GATEUP, LS_TIMED_DOWN, LS_TIMED_PREDICT, LS_TIMED_FUSED, LS_TIMED_STACK = 0, 1, 2, 3, 4
 
 
 def ls_timing_enable(on: bool) -> None:
@@ -314,3 +323,53 @@ def ls_topk_select_static(scores: torch.Tensor, k: int, idx: torch.Tensor, mask:
     assert scores.dtype == torch.float64 and scores.is_cuda and scores.is_contiguous()
     _check(lib().ls_topk_select_static(scores.data_ptr(), scores.numel(), k, idx.data_ptr(), _ptr(mask), count.data_ptr(),
                                        _stream(stream)))
+
+
+class Stack:
+    """Owner of one ``ls_stack*`` handle (keeps its layers alive)."""
+
+    def __init__(self, handle: int, layers):
+        self.handle = handle
+        self.layers = list(layers)
+
+    def close(self) -> None:
+        if self.handle:
+            lib().ls_stack_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class StackTrace:
+    """Device buffers of an ``ls_stack_trace``: residuals and selections at every layer boundary."""
+
+    def __init__(self, stack: Stack, sel_cap: int):
+        L0 = stack.layers[0]
+        dev = torch.device("cuda", L0.device)
+        n = len(stack.layers)
+        self.x = torch.zeros(n + 1, L0.d_model, dtype=torch.float32, device=dev)
+        self.sel_idx = torch.full((n + 1, max(sel_cap, 1)), -1, dtype=torch.int32, device=dev)
+        self.sel_count = torch.zeros(n + 1, dtype=torch.int32, device=dev)
+        self.c = ls_stack_trace(_ptr(self.x), _ptr(self.sel_idx), _ptr(self.sel_count), sel_cap)
+
+
+def ls_stack_create(layers) -> Stack:
+    arr = (C.c_void_p * len(layers))(*[L.handle for L in layers])
+    out = C.c_void_p()
+    _check(lib().ls_stack_create(arr, len(layers), C.byref(out)))
+    return Stack(out.value, layers)
+
+
+def ls_stack_destroy(stack: Stack) -> None:
+    stack.close()
+
+
+def ls_stack_decode(stack: Stack, x: torch.Tensor, x_out: torch.Tensor, sel_first: Selection, n_chunks: int, k_next: int,
+                    sel_out: Selection, trace: Optional[StackTrace] = None, stream=None) -> None:
+    assert x.dtype == torch.float32 and x.is_cuda and x.is_contiguous() and x_out.is_contiguous()
+    _check(lib().ls_stack_decode(stack.handle, x.data_ptr(), x_out.data_ptr(), C.byref(sel_first.c), n_chunks, k_next,
+                                 C.byref(sel_out.c), None if trace is None else C.byref(trace.c), _stream(stream)))

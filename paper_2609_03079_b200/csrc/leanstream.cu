@@ -128,6 +128,16 @@ struct ls_layer {
   ls::CacheState cache;  // residency tables, pinned backing store, copy stream
 };
 
+struct ls_stack {
+  int device = 0, n = 0, d = 0, wd = 0, sm_count = 148, max_sel = 0;
+  std::vector<ls_layer*> layers;
+  ls::FusedArgs* d_args = nullptr;  // [n] per-layer arguments (device)
+  float* xbuf = nullptr;            // [2][d] residual ping-pong between layers
+  int32_t* selidx = nullptr;        // [2][max_sel] selection ping-pong
+  int32_t* selcnt = nullptr;        // [2]
+  size_t smem = 0;
+};
+
 namespace {
 
 template <typename T>
@@ -200,17 +210,17 @@ int32_t device_scratch(int dev, DeviceScratch** out) {
   DeviceScratch& S = g_scratch[dev];
   if (!S.ready) {
     const size_t NE = ls::FZ_MAXE;
-    LS_TRY(dalloc(&S.dacc, (size_t)ls::FZ_MAXK * kScratchMaxD));
+    LS_TRY(dalloc(&S.dacc, (size_t)2 * ls::FZ_MAXK * kScratchMaxD));  // two parities (whole-token kernel)
     LS_TRY(dalloc(&S.ctr, (size_t)8));
     LS_TRY(dalloc(&S.z, NE * kScratchMaxR + NE));
-    LS_TRY(dalloc(&S.cnt, NE * ls::FZ_CNT_STRIDE));
+    LS_TRY(dalloc(&S.cnt, 2 * NE * ls::FZ_CNT_STRIDE));
     LS_TRY(dalloc(&S.bent, NE * ls::FZ_NB * ls::FZ_CAPB));
     LS_TRY(dalloc(&S.oent, NE * kScratchMaxF));
-    LS_TRY(dalloc(&S.nsel, NE));
-    LS_CUDA(cudaMemset(S.nsel, 0, NE * sizeof(unsigned)));
-    LS_CUDA(cudaMemset(S.dacc, 0, (size_t)ls::FZ_MAXK * kScratchMaxD * sizeof(float)));
+    LS_TRY(dalloc(&S.nsel, 2 * NE));
+    LS_CUDA(cudaMemset(S.nsel, 0, 2 * NE * sizeof(unsigned)));
+    LS_CUDA(cudaMemset(S.dacc, 0, (size_t)2 * ls::FZ_MAXK * kScratchMaxD * sizeof(float)));
     LS_CUDA(cudaMemset(S.ctr, 0, 8 * sizeof(unsigned)));
-    LS_CUDA(cudaMemset(S.cnt, 0, NE * ls::FZ_CNT_STRIDE * sizeof(unsigned)));
+    LS_CUDA(cudaMemset(S.cnt, 0, 2 * NE * ls::FZ_CNT_STRIDE * sizeof(unsigned)));
     LS_CUDA(cudaMemset(S.z, 0, (NE * kScratchMaxR + NE) * sizeof(double)));
     S.ready = true;
   }
@@ -292,8 +302,9 @@ int32_t create_impl(const ls_layer_desc* D, ls_layer* L) {
   LS_CUDA(cudaFuncSetAttribute(ls::ls_gateup_kernel<WD, BT>, cudaFuncAttributeMaxDynamicSharedMemorySize, big))
   LS_ATTR_GU(0, 1); LS_ATTR_GU(0, 4); LS_ATTR_GU(0, 8); LS_ATTR_GU(1, 1); LS_ATTR_GU(1, 4); LS_ATTR_GU(1, 8);
 #undef LS_ATTR_GU
-#define LS_ATTR_FZ(WD, CPT) \
-  LS_CUDA(cudaFuncSetAttribute(ls::ls_fused_step_kernel<WD, CPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 218 * 1024))
+#define LS_ATTR_FZ(WD, CPT)                                                                                                    \
+  LS_CUDA(cudaFuncSetAttribute(ls::ls_fused_step_kernel<WD, CPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 218 * 1024)); \
+  LS_CUDA(cudaFuncSetAttribute(ls::ls_fused_stack_kernel<WD, CPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 218 * 1024))
   LS_ATTR_FZ(0, 1); LS_ATTR_FZ(0, 2); LS_ATTR_FZ(1, 1); LS_ATTR_FZ(1, 2);
 #undef LS_ATTR_FZ
   LS_CUDA(cudaDeviceSynchronize());
@@ -342,30 +353,47 @@ int32_t launch_fused_cpt(int cpt, const ls::FusedArgs& a, int grid, size_t smem,
   return LS_OK;
 }
 
-int32_t fused_step(ls_layer* L, ls_layer* next, const float* d_x, float* d_x_out, const ls_selection* sel, int K, int k_next,
-                   ls_selection* sel_next, const ls_step_trace& tr, cudaStream_t st) {
+// Arguments of one fused layer step; `parity` picks the half of the alternating scratch.
+int32_t fused_args(ls_layer* L, ls_layer* next, const float* d_x, float* d_x_out, const int32_t* sel_idx, const int32_t* sel_count,
+                   int sel_cap, int K, int k_next, ls_selection* sel_next, int parity, ls::FusedArgs* out, ls::FusedSmemLayout* lay_out) {
   ls::FusedArgs a{};
   a.bundles = L->bundles; a.n_mat = L->n_mat; a.gated = L->gated; a.b_gate = L->b_gate; a.b_down = L->b_down;
   a.d = L->d; a.F = L->F; a.norm = L->norm; a.eps = L->eps;
   a.x = d_x; a.x_out = d_x_out;
-  a.sel_idx = sel->idx; a.sel_count = sel->count; a.sel_cap = sel->cap; a.K = K;
+  a.sel_idx = sel_idx; a.sel_count = sel_count; a.sel_cap = sel_cap; a.K = K;
   DeviceScratch* S = nullptr;
   LS_TRY(device_scratch(L->device, &S));
-  a.dacc = S->dacc; a.fin = S->ctr;
+  a.dacc = S->dacc + (size_t)parity * ls::FZ_MAXK * kScratchMaxD; a.fin = S->ctr;
   a.bar_count = reinterpret_cast<unsigned long long*>(S->ctr + 2);  // 8-byte aligned
   a.status = L->status;
   a.has_next = next ? 1 : 0;
-  const int nw_next = next ? next->nwords : 0;
   if (next) {
     a.At = next->pred_at; a.Bt = next->pred_bt; a.pc = next->pred_c;
     a.r = next->r; a.Fn = next->F; a.norm_n = next->norm; a.eps_n = next->eps; a.k_next = k_next;
     a.z = S->z; a.sumsq = S->z + (size_t)ls::FZ_MAXE * next->r; a.range = next->fz_range;
-    a.cnt = S->cnt; a.bent = S->bent; a.oent = S->oent;
-    a.range_obs = next->fz_range_obs; a.nsel = S->nsel;
-    a.next_idx = sel_next->idx; a.next_count = sel_next->count; a.next_mask = sel_next->mask; a.next_scores = sel_next->scores;
-    a.next_prio = next->prio; a.next_cap = sel_next->cap;
-    if (sel_next->mask) LS_CUDA(cudaMemsetAsync(sel_next->mask, 0, (size_t)nw_next * 4, st));
+    a.cnt = S->cnt + (size_t)parity * ls::FZ_MAXE * ls::FZ_CNT_STRIDE; a.bent = S->bent; a.oent = S->oent;
+    a.range_obs = next->fz_range_obs; a.nsel = S->nsel + (size_t)parity * ls::FZ_MAXE;
+    if (sel_next) {
+      a.next_idx = sel_next->idx; a.next_count = sel_next->count; a.next_mask = sel_next->mask; a.next_scores = sel_next->scores;
+      a.next_cap = sel_next->cap;
+    }
+    a.next_prio = next->prio;
   }
+  ls::FusedSmemLayout lay{};
+  if (!fused_plan(L, next, &lay)) return fail(LS_ERR_STATE, "fused step: shared memory plan failed");
+  a.gu_depth = lay.gu_depth; a.dn_depth = lay.dn_depth;
+  *out = a;
+  if (lay_out) *lay_out = lay;
+  return LS_OK;
+}
+
+int32_t fused_step(ls_layer* L, ls_layer* next, const float* d_x, float* d_x_out, const ls_selection* sel, int K, int k_next,
+                   ls_selection* sel_next, const ls_step_trace& tr, cudaStream_t st) {
+  ls::FusedArgs a{};
+  ls::FusedSmemLayout lay{};
+  LS_TRY(fused_args(L, next, d_x, d_x_out, sel->idx, sel->count, sel->cap, K, k_next, sel_next, 0, &a, &lay));
+  const int nw_next = next ? next->nwords : 0;
+  if (next && sel_next->mask) LS_CUDA(cudaMemsetAsync(sel_next->mask, 0, (size_t)nw_next * 4, st));
   a.tr_xtilde = tr.xtilde; a.tr_masks = next ? tr.refine_masks : nullptr; a.tr_counts = next ? tr.refine_counts : nullptr;
   a.tr_survive = tr.survive_mask;
   if (a.tr_masks) LS_CUDA(cudaMemsetAsync(a.tr_masks, 0, (size_t)(K + 1) * nw_next * 4, st));
@@ -375,9 +403,6 @@ int32_t fused_step(ls_layer* L, ls_layer* next, const float* d_x, float* d_x_out
                                               sel->cap);
     LS_LAUNCHED();
   }
-  ls::FusedSmemLayout lay{};
-  if (!fused_plan(L, next, &lay)) return fail(LS_ERR_STATE, "fused step: shared memory plan failed");
-  a.gu_depth = lay.gu_depth; a.dn_depth = lay.dn_depth;
   const int cpt = ((L->d >> 3) + ls::FZ_THREADS - 1) / ls::FZ_THREADS;
   if (L->wd == 0) return launch_fused_cpt<0>(cpt, a, L->sm_count, lay.total, st);
   return launch_fused_cpt<1>(cpt, a, L->sm_count, lay.total, st);
@@ -548,6 +573,100 @@ size_t ls_last_error(char* buf, size_t n) {
 }
 
 int64_t ls_kernel_launches(void) { return g_launches.load(); }
+
+int32_t ls_stack_create(ls_layer* const* layers, int32_t n_layers, ls_stack** out) {
+  if (out) *out = nullptr;
+  if (!layers || !out || n_layers < 1 || n_layers > 4096) return fail(LS_ERR_INVALID, "ls_stack_create: bad argument");
+  for (int n = 0; n < n_layers; ++n) {
+    const ls_layer* L = layers[n];
+    if (!L) return fail(LS_ERR_INVALID, "ls_stack_create: layer %d is NULL", n);
+    if (L->cache_rows != 0) return fail(LS_ERR_STATE, "ls_stack_create: layer %d has a cache; the whole-token kernel needs resident layers", n);
+    if (L->device != layers[0]->device || L->d != layers[0]->d || L->wd != layers[0]->wd)
+      return fail(LS_ERR_INVALID, "ls_stack_create: layer %d differs in device, d_model or weight type", n);
+  }
+  DeviceGuard guard(layers[0]->device);
+  ls_stack* S = new (std::nothrow) ls_stack();
+  if (!S) return fail(LS_ERR_NOMEM, "host allocation");
+  S->device = layers[0]->device; S->n = n_layers; S->d = layers[0]->d; S->wd = layers[0]->wd; S->sm_count = layers[0]->sm_count;
+  S->layers.assign(layers, layers + n_layers);
+  for (int n = 0; n < n_layers; ++n) S->max_sel = std::max(S->max_sel, layers[n]->max_sel);
+  auto cleanup = [&](int32_t rc) {
+    const std::string keep = g_err;
+    cudaFree(S->d_args); cudaFree(S->xbuf); cudaFree(S->selidx); cudaFree(S->selcnt);
+    delete S;
+    g_err = keep;
+    return rc;
+  };
+  int32_t rc;
+  if ((rc = dalloc(&S->d_args, (size_t)n_layers)) != LS_OK) return cleanup(rc);
+  if ((rc = dalloc(&S->xbuf, (size_t)2 * S->d)) != LS_OK) return cleanup(rc);
+  if ((rc = dalloc(&S->selidx, (size_t)2 * S->max_sel)) != LS_OK) return cleanup(rc);
+  if ((rc = dalloc(&S->selcnt, 2)) != LS_OK) return cleanup(rc);
+  std::vector<ls::FusedArgs> h(n_layers);
+  for (int n = 0; n < n_layers; ++n) {
+    ls_layer* L = layers[n];
+    ls_layer* next = layers[n + 1 < n_layers ? n + 1 : n];  // the last layer refines a weight-tied copy of itself
+    if (!fused_plan(L, next, nullptr) || (L->d >> 3) > ls::FZ_THREADS * 2)
+      return cleanup(fail(LS_ERR_STATE, "ls_stack_create: layer %d does not fit the fused kernel's shared memory", n));
+    ls_selection sn{};
+    sn.idx = S->selidx + (size_t)((n + 1) & 1) * S->max_sel;
+    sn.count = S->selcnt + ((n + 1) & 1);
+    sn.cap = S->max_sel;
+    ls::FusedSmemLayout lay{};
+    rc = fused_args(L, next, S->xbuf + (size_t)(n & 1) * S->d, S->xbuf + (size_t)((n + 1) & 1) * S->d,
+                    S->selidx + (size_t)(n & 1) * S->max_sel, S->selcnt + (n & 1), S->max_sel, 1, 0, &sn, n & 1, &h[n], &lay);
+    if (rc != LS_OK) return cleanup(rc);
+    S->smem = std::max(S->smem, lay.total);
+  }
+  if (cudaMemcpy(S->d_args, h.data(), sizeof(ls::FusedArgs) * n_layers, cudaMemcpyHostToDevice) != cudaSuccess)
+    return cleanup(fail(LS_ERR_CUDA, "ls_stack_create: upload of the layer arguments failed"));
+  *out = S;
+  return LS_OK;
+}
+
+int32_t ls_stack_destroy(ls_stack* S) {
+  if (!S) return LS_OK;
+  DeviceGuard guard(S->device);
+  cudaDeviceSynchronize();
+  cudaFree(S->d_args); cudaFree(S->xbuf); cudaFree(S->selidx); cudaFree(S->selcnt);
+  delete S;
+  return LS_OK;
+}
+
+int32_t ls_stack_decode(ls_stack* S, const float* d_x, float* d_x_out, const ls_selection* sel_first, int32_t K, int32_t k_next,
+                        ls_selection* sel_out, ls_stack_trace* trace, void* stream) {
+  if (!S || !d_x || !d_x_out || !sel_first || !sel_first->idx || !sel_first->count || !sel_out || !sel_out->idx || !sel_out->count)
+    return fail(LS_ERR_INVALID, "ls_stack_decode: x, x_out, sel_first and sel_out (idx, count) are required");
+  if (K < 1 || K > ls::FZ_MAXK) return fail(LS_ERR_INVALID, "ls_stack_decode: n_chunks %d outside [1, %d]", K, ls::FZ_MAXK);
+  if (sel_first->cap < 0 || sel_first->cap > S->layers[0]->max_sel) return fail(LS_ERR_INVALID, "ls_stack_decode: sel_first->cap outside [0, max_sel]");
+  int fmin_ = 1 << 30;
+  for (ls_layer* L : S->layers) fmin_ = std::min(fmin_, std::min(L->F, L->max_sel));
+  if (k_next < 0 || k_next > fmin_) return fail(LS_ERR_INVALID, "ls_stack_decode: k_next %d outside [0, %d] (smallest d_ff / max_sel of the stack)", k_next, fmin_);
+  if ((sel_first->cap + S->sm_count - 1) / S->sm_count > ls::FZ_MAX_MINE || (k_next + S->sm_count - 1) / S->sm_count > ls::FZ_MAX_MINE)
+    return fail(LS_ERR_INVALID, "ls_stack_decode: selection too long for the fused kernel");
+  if (sel_out->cap < k_next) return fail(LS_ERR_INVALID, "ls_stack_decode: sel_out->cap %d < k_next %d", sel_out->cap, k_next);
+  DeviceGuard guard(S->device);
+  cudaStream_t st = (cudaStream_t)stream;
+  ls::StackCall c{};
+  c.x_in = d_x; c.x_out = d_x_out;
+  c.sel_idx = sel_first->idx; c.sel_count = sel_first->count; c.sel_cap = sel_first->cap;
+  c.out_idx = sel_out->idx; c.out_count = sel_out->count; c.out_mask = sel_out->mask; c.out_scores = sel_out->scores; c.out_cap = sel_out->cap;
+  c.K = K; c.k_next = k_next;
+  if (trace) { c.tr_x = trace->x; c.tr_sel = trace->sel_idx; c.tr_cnt = trace->sel_count; c.tr_cap = trace->sel_cap; }
+  if (c.tr_sel && !c.tr_cnt) return fail(LS_ERR_INVALID, "ls_stack_decode: trace->sel_count is required with trace->sel_idx");
+  if (sel_out->mask) LS_CUDA(cudaMemsetAsync(sel_out->mask, 0, (size_t)S->layers.back()->nwords * 4, st));
+  const ls::FusedArgs* args = S->d_args;
+  int n = S->n;
+  void* params[] = {&args, &n, &c};
+  const int cpt = ((S->d >> 3) + ls::FZ_THREADS - 1) / ls::FZ_THREADS;
+  const void* fn = nullptr;
+  if (S->wd == 0) fn = cpt == 1 ? (const void*)ls::ls_fused_stack_kernel<0, 1> : (const void*)ls::ls_fused_stack_kernel<0, 2>;
+  else fn = cpt == 1 ? (const void*)ls::ls_fused_stack_kernel<1, 1> : (const void*)ls::ls_fused_stack_kernel<1, 2>;
+  KernelTimer timer(LS_TIMED_STACK, st);
+  LS_CUDA(cudaLaunchCooperativeKernel(fn, dim3(S->sm_count), dim3(ls::FZ_BLOCK), params, S->smem, st));
+  LS_LAUNCHED();
+  return LS_OK;
+}
 
 int32_t ls_topk_select_static(const double* d_scores, int32_t n, int32_t k, int32_t* d_idx, uint32_t* d_mask, int32_t* d_count,
                               void* stream) {

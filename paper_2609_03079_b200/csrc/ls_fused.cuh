@@ -173,7 +173,7 @@ __host__ __device__ inline FusedSmemLayout fused_layout(int d, int n_in, int r, 
   auto take = [&](size_t bytes) { size_t at = o; o += (bytes + 127) & ~(size_t)127; return at; };
   L.gu_off = take((size_t)gu_depth * n_in * d * 2);
   L.dn_off = take((size_t)dn_depth * d * 2);
-  L.bar_off = take((2 * FZ_MAX_DEPTH + 1) * 8);
+  L.bar_off = take((2 * FZ_MAX_DEPTH + 2) * 8);
   L.red_off = take(2 * 16 * 8 * 4);                  // stream dot partials, double-buffered: [2][warp][8]
   L.redd_off = take((size_t)FZ_MAXE * 3 * 16 * 8);   // fp64 partials of the latent phase: [evaluation][row0,row1,sumsq][warp]
   L.mine_off = take((size_t)FZ_MAX_MINE * 8);        // this CTA's neuron indices and gate biases
@@ -191,9 +191,27 @@ __host__ __device__ inline FusedSmemLayout fused_layout(int d, int n_in, int r, 
 }
 
 // =====================================================================================================================
+// Block-shared state of a layer step (static shared memory of the kernels below).
+struct FusedShared {
+  FusedArgs args;                    // the layer's arguments (whole-token kernel: copied from global memory per layer)
+  FusedArgs prev;                    // whole-token kernel: the layer before, whose scratch is cleaned meanwhile
+  int last;
+  int round;                         // rounds the compute warps have finished (read by the producer)
+  int mail[4 * 4];                   // per round (ring of four): number of survivors, their neurons
+  float act[2 * 4];                  // activations of the round's neurons, double-buffered
+  double inv[8];
+  int cut[FZ_MAXE * 4];              // per evaluation: cut fine bin, its first rank, threshold neuron, fallback flag
+  unsigned long long cutkey[FZ_MAXE];  // threshold key inside the cut bin
+  unsigned nsel[FZ_MAXE];            // members found by this CTA, per evaluation
+  unsigned long long kmm[2 * 16];
+  unsigned ccnt[FZ_MAXE * FZ_NC];
+};
+
+// One layer step, executed by the whole block (16 compute warps + the producer warp).  The producer warp returns as
+// soon as it has issued its last copy; the compute warps return when the layer's refined sets are written.
+// `reinit` says that the mbarriers in shared memory were used by an earlier layer of the same launch.
 template <int WD, int CPT>
-__global__ void __launch_bounds__(FZ_BLOCK, 1) ls_fused_step_kernel(const __grid_constant__ FusedArgs A) {
-  extern __shared__ __align__(128) unsigned char smem[];
+__device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* smem, FusedShared& sh, bool reinit) {
   const int G = gridDim.x, cta = blockIdx.x, tid = threadIdx.x;
   const int lane = tid & 31, warp = tid >> 5;
   const int d = A.d, K = A.K, nchunk = A.d >> 3;
@@ -208,22 +226,22 @@ __global__ void __launch_bounds__(FZ_BLOCK, 1) ls_fused_step_kernel(const __grid
   uint16_t* s_A = reinterpret_cast<uint16_t*>(smem + lay.a_off);      // [nA][d]
   uint16_t* s_B = reinterpret_cast<uint16_t*>(smem + lay.b_off);      // [per][r]
   float* s_pc = reinterpret_cast<float*>(smem + lay.pc_off);
-  __shared__ int s_last;
-  __shared__ int s_round;      // rounds the compute warps have finished (read by the producer)
-  __shared__ int s_mail[4 * 4];  // per round (ring of four): number of survivors, their neurons
-  __shared__ float s_act[2 * 4]; // activations of the round's neurons, double-buffered
-  __shared__ double s_inv[8];
-  __shared__ int s_cut[FZ_MAXE * 4];             // per evaluation: cut fine bin, its first rank, threshold neuron, fallback flag
-  __shared__ unsigned long long s_cutkey[FZ_MAXE];  // threshold key inside the cut bin
-  __shared__ unsigned s_nsel[FZ_MAXE];              // members found by this CTA, per evaluation
-  __shared__ unsigned long long s_kmm[2 * 16];
-  __shared__ unsigned s_ccnt[FZ_MAXE * FZ_NC];
+  int& s_round = sh.round;
+  int* s_mail = sh.mail;
+  float* s_act = sh.act;
+  double* s_inv = sh.inv;
+  int* s_cut = sh.cut;
+  unsigned long long* s_cutkey = sh.cutkey;
+  unsigned* s_nsel = sh.nsel;
+  unsigned long long* s_kmm = sh.kmm;
+  unsigned* s_ccnt = sh.ccnt;
 
-  if (tid == 0) FZ_STAMP(1, 72);
   if (tid == 0) {
-    for (int i = 0; i < GU; ++i) mbar_init(&s_bar[i], 1);
-    for (int i = 0; i < DN; ++i) mbar_init(&s_bar[FZ_MAX_DEPTH + i], 1);
+    if (reinit)  // every copy of the earlier layer has completed; its barriers are retired before the new ones are set up
+      for (int i = 0; i <= 2 * FZ_MAX_DEPTH + 1; ++i) asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(smem_u32(&s_bar[i])) : "memory");
+    for (int i = 0; i < 2 * FZ_MAX_DEPTH; ++i) mbar_init(&s_bar[i], 1);
     mbar_init(&s_bar[2 * FZ_MAX_DEPTH], 1);
+    mbar_init(&s_bar[2 * FZ_MAX_DEPTH + 1], 1);
     s_round = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -238,7 +256,7 @@ __global__ void __launch_bounds__(FZ_BLOCK, 1) ls_fused_step_kernel(const __grid
   {
     // ================================================= stream: all warps ===========================================
     // this CTA serves one stage: the ranks [lo, hi) of the selection, every gsize-th neuron starting at its own offset
-    const int count = max(0, min(*A.sel_count, A.sel_cap));
+    const int count = max(0, min(__ldcg(A.sel_count), A.sel_cap));
     const int m = count > 0 ? (count + K - 1) / K : 0;
     const int stage = fz_stage_of_cta(cta, G, K);
     const int g_lo = fz_group_lo(stage, G, K), gsize = fz_group_lo(stage + 1, G, K) - g_lo;
@@ -252,7 +270,7 @@ __global__ void __launch_bounds__(FZ_BLOCK, 1) ls_fused_step_kernel(const __grid
     int* s_myidx = reinterpret_cast<int*>(smem + lay.mine_off);
     float* s_mybias = reinterpret_cast<float*>(s_myidx + FZ_MAX_MINE);
     for (int t = tid; t < n_mine; t += FZ_THREADS) {
-      int i = A.sel_idx[first + t * gsize];
+      int i = __ldcg(A.sel_idx + first + t * gsize);
       if ((unsigned)i >= (unsigned)A.F) { set_status(A.status, ST_BAD_INDEX); i = -1; }
       s_myidx[t] = i;
     }
@@ -262,8 +280,8 @@ __global__ void __launch_bounds__(FZ_BLOCK, 1) ls_fused_step_kernel(const __grid
     for (int q = 0; q < CPT; ++q) {
       const int ch = tid + q * FZ_THREADS;
       if (ch < nchunk) {
-        const float4 a0 = __ldg(reinterpret_cast<const float4*>(A.x + ch * 8));
-        const float4 a1 = __ldg(reinterpret_cast<const float4*>(A.x + ch * 8 + 4));
+        const float4 a0 = __ldcg(reinterpret_cast<const float4*>(A.x + ch * 8));
+        const float4 a1 = __ldcg(reinterpret_cast<const float4*>(A.x + ch * 8 + 4));
         xr[q][0] = a0.x; xr[q][1] = a0.y; xr[q][2] = a0.z; xr[q][3] = a0.w;
         xr[q][4] = a1.x; xr[q][5] = a1.y; xr[q][6] = a1.z; xr[q][7] = a1.w;
       } else {
@@ -288,21 +306,6 @@ __global__ void __launch_bounds__(FZ_BLOCK, 1) ls_fused_step_kernel(const __grid
           tma_load_1d(s_gu + (size_t)(it % GU) * n_in * d, A.bundles + (size_t)i * bundle_elems, gu_bytes, bar);
         };
         for (int it = 0; it < min(n_mine, GU); ++it) issue_gu(it);
-        if (A.has_next) {
-          // this CTA's share of the next layer's predictor, as stored: rows of A^T, rows of B^T (padded row stride)
-          uint64_t* pbar = &s_bar[2 * FZ_MAX_DEPTH];
-          uint32_t bytes = 0;
-          for (int a = 0; a < lay.nA; ++a)
-            if (cta + a * G < r) bytes += (uint32_t)d * 2;
-          bytes += (uint32_t)n_own * (uint32_t)r * 2;
-          mbar_expect_tx(pbar, bytes);
-          for (int a = 0; a < lay.nA; ++a) {
-            const int j = cta + a * G;
-            if (j < r) tma_load_1d(s_A + (size_t)a * d, A.At + (size_t)j * d, (uint32_t)d * 2, pbar);
-          }
-          for (int li = 0; li < n_own; ++li)
-            tma_load_1d(s_B + (size_t)li * (r + FZ_BPAD), A.Bt + (size_t)(i_lo + li) * r, (uint32_t)r * 2, pbar);
-        }
         const int n_rounds = (n_mine + FZ_NG - 1) / FZ_NG;
         int tail = 0;
         for (int rd = 0; rd < n_rounds; ++rd) {
@@ -328,6 +331,23 @@ __global__ void __launch_bounds__(FZ_BLOCK, 1) ls_fused_step_kernel(const __grid
             if (A.tr_survive) atomicOr(&A.tr_survive[i >> 5], 1u << (i & 31));
             ++tail;
           }
+        }
+        // last, off the streaming's critical path: the predictor operands are needed only after the first grid barrier
+        if (A.has_next) {
+          // this CTA's share of the next layer's predictor, as stored: rows of A^T, rows of B^T (padded row stride)
+          uint64_t* abar = &s_bar[2 * FZ_MAX_DEPTH];      // rows of A^T: awaited before the latent phase
+          uint64_t* bbar = &s_bar[2 * FZ_MAX_DEPTH + 1];  // rows of B^T: awaited before the score phase
+          uint32_t bytes = 0;
+          for (int a = 0; a < lay.nA; ++a)
+            if (cta + a * G < r) bytes += (uint32_t)d * 2;
+          mbar_expect_tx(abar, bytes);
+          for (int a = 0; a < lay.nA; ++a) {
+            const int j = cta + a * G;
+            if (j < r) tma_load_1d(s_A + (size_t)a * d, A.At + (size_t)j * d, (uint32_t)d * 2, abar);
+          }
+          mbar_expect_tx(bbar, (uint32_t)n_own * (uint32_t)r * 2);
+          for (int li = 0; li < n_own; ++li)
+            tma_load_1d(s_B + (size_t)li * (r + FZ_BPAD), A.Bt + (size_t)(i_lo + li) * r, (uint32_t)r * 2, bbar);
         }
       }
       return;  // an exited warp counts as arrived at every later block barrier
@@ -490,7 +510,7 @@ __global__ void __launch_bounds__(FZ_BLOCK, 1) ls_fused_step_kernel(const __grid
       }
     }
     if (tid == 0) FZ_STAMP(0, 501);
-    if (A.has_next) mbar_wait(&s_bar[2 * FZ_MAX_DEPTH], 0u, A.status);  // predictor operands have landed
+    if (A.has_next) mbar_wait(&s_bar[2 * FZ_MAX_DEPTH], 0u, A.status);  // the rows of A^T have landed (B^T is awaited later)
   }
 
   // ------------------------------------------------------------------------------------------------ barrier 1 of 3
@@ -514,7 +534,7 @@ __global__ void __launch_bounds__(FZ_BLOCK, 1) ls_fused_step_kernel(const __grid
 #pragma unroll
       for (int q = 0; q < XC; ++q) {
         const int c = tid + q * FZ_THREADS;
-        xs[q] = c < d ? A.x[c] + (A.b_down ? A.b_down[c] : 0.f) : 0.f;
+        xs[q] = c < d ? __ldcg(A.x + c) + (A.b_down ? A.b_down[c] : 0.f) : 0.f;
       }
       for (int j0 = 0; j0 <= K; j0 += JG) {
         double p0[JG], p1[JG], sq[JG];
@@ -627,6 +647,7 @@ __global__ void __launch_bounds__(FZ_BLOCK, 1) ls_fused_step_kernel(const __grid
     // C[neuron][evaluation] = B^T rows x latents, on the fp64 tensor cores (mma m8n8k4): a warp owns tiles of eight
     // neurons, the evaluations are taken eight at a time.  Every output element is accumulated over the columns in the
     // same order whatever its position in the tile, so equal predictor rows give bit-equal scores.
+    mbar_wait(&s_bar[2 * FZ_MAX_DEPTH + 1], 0u, A.status);  // the rows of B^T have landed
     const int RSB = r + FZ_BPAD, RSZ = r + FZ_ZPAD;
     const int n_mt = (n_own + 7) >> 3;
     for (int n0 = 0; n0 <= K; n0 += 8) {
@@ -962,45 +983,131 @@ __global__ void __launch_bounds__(FZ_BLOCK, 1) ls_fused_step_kernel(const __grid
     if (tid == 0) FZ_STAMP(1, 6);
   }
 
-  // ---- the last CTA to finish restores the zero-on-entry invariants of the per-layer scratch
-  named_bar_sync(1, FZ_THREADS);
-  if (tid == 0) FZ_STAMP(1, 70);
-  if (tid == 0) {
-    __threadfence();
-    s_last = (atomicAdd(A.fin, 1u) == (unsigned)G - 1u) ? 1 : 0;
+}
+
+// Binning range of a layer's scores for its next launch: what the final evaluation observed, widened by 5 % per side.
+__device__ inline void fused_update_range(const FusedArgs& A) {
+  const unsigned long long kmin = A.range_obs[0], kmax = A.range_obs[1];
+  if (kmin <= kmax) {
+    auto unkey = [](unsigned long long k) {
+      const unsigned long long b = (k >> 63) ? (k & 0x7fffffffffffffffULL) : ~k;
+      return __longlong_as_double((long long)b);
+    };
+    double lo = unkey(kmin), hi = unkey(kmax);
+    lo = fmax(lo, -1.0e300);
+    hi = fmin(hi, 1.0e300);
+    const double pad = 0.05 * (hi - lo);
+    A.range[0] = lo - pad;
+    A.range[1] = hi + pad;
   }
-  named_bar_sync(1, FZ_THREADS);
-  if (s_last) {
-    __threadfence();
-    for (int t = tid; t < K * d; t += FZ_THREADS) A.dacc[t] = 0.f;
-    if (A.has_next) {
-      for (int t = tid; t < (K + 1) * FZ_CNT_STRIDE; t += FZ_THREADS) A.cnt[t] = 0u;
-      if (tid <= K) {  // self-check: every refined set has exactly min(k_next, d_ff) members
-        if ((int)A.nsel[tid] != min(A.k_next, A.Fn)) set_status(A.status, ST_INTERNAL);
+  A.range_obs[0] = 0xffffffffffffffffULL;
+  A.range_obs[1] = 0ULL;
+}
+
+// Zeroes the slice [part, parts) of what a layer step dirtied in the scratch (compute threads only); part 0 also runs the
+// self-check of the refined-set sizes and the range update.  The caller guarantees that every CTA is done with the layer.
+__device__ inline void fused_clean(const FusedArgs& A, int part, int parts) {
+  const int tid = threadIdx.x;
+  for (int t = part * FZ_THREADS + tid; t < A.K * A.d; t += parts * FZ_THREADS) A.dacc[t] = 0.f;
+  if (A.has_next) {
+    for (int t = part * FZ_THREADS + tid; t < (A.K + 1) * FZ_CNT_STRIDE; t += parts * FZ_THREADS) A.cnt[t] = 0u;
+    if (part == 0) {
+      if (tid <= A.K) {  // self-check: every refined set has exactly min(k_next, d_ff) members
+        if ((int)__ldcg(&A.nsel[tid]) != min(A.k_next, A.Fn)) set_status(A.status, ST_INTERNAL);
         A.nsel[tid] = 0u;
       }
-      if (tid == 0) {
-        // binning range for the next launch: what the final evaluation observed, widened by 5 % on each side
-        const unsigned long long kmin = A.range_obs[0], kmax = A.range_obs[1];
-        if (kmin <= kmax) {
-          auto unkey = [](unsigned long long k) {
-            const unsigned long long b = (k >> 63) ? (k & 0x7fffffffffffffffULL) : ~k;
-            return __longlong_as_double((long long)b);
-          };
-          double lo = unkey(kmin), hi = unkey(kmax);
-          lo = fmax(lo, -1.0e300);
-          hi = fmin(hi, 1.0e300);
-          const double pad = 0.05 * (hi - lo);
-          A.range[0] = lo - pad;
-          A.range[1] = hi + pad;
-        }
-        A.range_obs[0] = 0xffffffffffffffffULL;
-        A.range_obs[1] = 0ULL;
+      if (tid == 0) fused_update_range(A);
+    }
+  }
+}
+
+// ---- one launch per layer step: the last CTA to finish restores the zero-on-entry invariants of the scratch
+template <int WD, int CPT>
+__global__ void __launch_bounds__(FZ_BLOCK, 1) ls_fused_step_kernel(const __grid_constant__ FusedArgs A) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  __shared__ FusedShared sh;
+  fused_layer<WD, CPT>(A, smem, sh, false);
+  if (threadIdx.x >= FZ_THREADS) return;  // the producer warp is done; an exited warp counts as arrived at block barriers
+  named_bar_sync(1, FZ_THREADS);
+  if (threadIdx.x == 0) {
+    __threadfence();
+    sh.last = (atomicAdd(A.fin, 1u) == gridDim.x - 1u) ? 1 : 0;
+  }
+  named_bar_sync(1, FZ_THREADS);
+  if (sh.last) {
+    __threadfence();
+    fused_clean(A, 0, 1);
+    if (threadIdx.x == 0) *A.fin = 0u;
+  }
+}
+
+// ---- one launch per token: the layers of a resident stack run back to back inside one cooperative kernel ------------
+// Per-call arguments of the whole-token kernel (the per-layer arguments live in a device array built at stack creation).
+struct StackCall {
+  const float* x_in; float* x_out;
+  const int32_t* sel_idx; const int32_t* sel_count; int sel_cap;       // selection of the first layer
+  int32_t* out_idx; int32_t* out_count; uint32_t* out_mask; double* out_scores; int out_cap;  // refined set of the last layer
+  int K, k_next;
+  float* tr_x;       // [n_layers + 1][d]      residual entering every layer and leaving the last (nullable)
+  int32_t* tr_sel;   // [n_layers + 1][tr_cap] selection entering every layer, and the final refined one (nullable)
+  int32_t* tr_cnt;   // [n_layers + 1]
+  int tr_cap;
+};
+
+// Layer n reads x / selection buffers of parity n & 1 and writes those of the other parity; the scratch a layer dirties
+// (stage accumulators, histograms, set sizes) also alternates, and every CTA cleans its slice of the previous layer's
+// scratch while it waits at the end of the current one.  A layer boundary costs one grid barrier instead of a launch.
+template <int WD, int CPT>
+__global__ void __launch_bounds__(FZ_BLOCK, 1)
+    ls_fused_stack_kernel(const FusedArgs* __restrict__ g_args, int n_layers, const __grid_constant__ StackCall C) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  __shared__ FusedShared sh;
+  const int G = gridDim.x, cta = blockIdx.x, tid = threadIdx.x;
+  constexpr int NW = sizeof(FusedArgs) / 4;
+  for (int n = 0; n < n_layers; ++n) {
+    for (int w = tid; w < NW; w += FZ_BLOCK) reinterpret_cast<uint32_t*>(&sh.args)[w] = reinterpret_cast<const uint32_t*>(&g_args[n])[w];
+    __syncthreads();
+    if (tid == 0) {
+      FusedArgs& a = sh.args;
+      a.K = C.K;
+      a.k_next = C.k_next;
+      if (n == 0) { a.x = C.x_in; a.sel_idx = C.sel_idx; a.sel_count = C.sel_count; a.sel_cap = C.sel_cap; }
+      if (n == n_layers - 1) {
+        a.x_out = C.x_out;
+        a.next_idx = C.out_idx; a.next_count = C.out_count; a.next_mask = C.out_mask; a.next_scores = C.out_scores; a.next_cap = C.out_cap;
       }
     }
-    if (tid == 0) *A.fin = 0u;
+    __syncthreads();
+    const FusedArgs& A = sh.args;
+    fused_layer<WD, CPT>(A, smem, sh, n > 0);
+    if (tid < FZ_THREADS) {
+      if (cta == G - 1 && C.tr_x) {  // what entered this layer
+        for (int c = tid; c < A.d; c += FZ_THREADS) C.tr_x[(size_t)n * A.d + c] = __ldcg(A.x + c);
+        if (C.tr_sel) {
+          const int cnt = max(0, min(__ldcg(A.sel_count), min(A.sel_cap, C.tr_cap)));
+          for (int t = tid; t < cnt; t += FZ_THREADS) C.tr_sel[(size_t)n * C.tr_cap + t] = __ldcg(A.sel_idx + t);
+          if (tid == 0) C.tr_cnt[n] = cnt;
+        }
+      }
+      if (n > 0) fused_clean(sh.prev, cta, G);  // nobody touches the previous layer's scratch any more
+      grid_barrier(A, G);                       // layer boundary: x_out and the refined selection are visible to all
+    }
+    __syncthreads();
+    for (int w = tid; w < NW; w += FZ_BLOCK) reinterpret_cast<uint32_t*>(&sh.prev)[w] = reinterpret_cast<const uint32_t*>(&sh.args)[w];
+    __syncthreads();
   }
-  if (tid == 0) FZ_STAMP(1, 71);
+  if (tid < FZ_THREADS && n_layers > 0) {
+    const FusedArgs& A = sh.prev;  // the last layer; every CTA is past its final barrier
+    fused_clean(A, cta, G);
+    if (cta == G - 1 && C.tr_x) {
+      for (int c = tid; c < A.d; c += FZ_THREADS) C.tr_x[(size_t)n_layers * A.d + c] = __ldcg(A.x_out + c);
+      if (C.tr_sel && A.has_next) {
+        const int cnt = max(0, min(__ldcg(A.next_count), min(A.next_cap, C.tr_cap)));
+        for (int t = tid; t < cnt; t += FZ_THREADS) C.tr_sel[(size_t)n_layers * C.tr_cap + t] = __ldcg(A.next_idx + t);
+        if (tid == 0) C.tr_cnt[n_layers] = cnt;
+      }
+    }
+  }
 }
 
 }  // namespace ls

@@ -1,0 +1,115 @@
+"""Whole-token kernel (ls_stack_decode): every layer boundary it exports is replayed through the oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import leanstream_oracle as orc
+from paper_2609_03079_b200 import binding as ls
+from paper_2609_03079_b200 import workload as wl
+from tests.helpers import assert_values_close, check_selection
+
+pytestmark = pytest.mark.gpu
+DEV = 0
+
+
+def decode_and_check(spec, arrays, K, k, n_tokens, stats):
+    OLs = [orc.OracleLayer.from_arrays(a) for a in arrays]
+    GLs = [ls.ls_layer_create(a, DEV) for a in arrays]
+    stack = ls.ls_stack_create(GLs)
+    n = len(GLs)
+    sel0 = ls.Selection(spec.d_ff, k, DEV)
+    sel_out = ls.Selection(spec.d_ff, k, DEV)
+    trace = ls.StackTrace(stack, k)
+    for x0 in wl.make_tokens(spec)[:n_tokens]:
+        x = torch.from_numpy(x0).cuda(DEV)
+        x_out = torch.empty_like(x)
+        ls.ls_predict(GLs[0], x, k, sel0)
+        ls.ls_stack_decode(stack, x, x_out, sel0, K, k, sel_out, trace)
+        torch.cuda.synchronize()
+        assert all(ls.ls_layer_status(g) == 0 for g in GLs)
+        X = trace.x.cpu().numpy()
+        S = trace.sel_idx.cpu().numpy()
+        cnt = trace.sel_count.cpu().numpy()
+        np.testing.assert_array_equal(X[0], x0)
+        np.testing.assert_array_equal(X[n], x_out.cpu().numpy())
+        assert cnt.tolist() == [k] * (n + 1)
+        assert S[0, :k].tolist() == sel0.order().tolist() and S[n, :k].tolist() == sel_out.order().tolist()
+        for layer in range(n):
+            nxt = OLs[min(layer + 1, n - 1)]
+            order = S[layer, :k].astype(np.int64)
+            # the selection entering the layer is the exact top-k of the residual that entered it
+            check_selection(order, orc.predictor_scores(OLs[layer], X[layer]), k, stats)
+            # the layer's output from that residual and that selection
+            res = orc.sparse_ffn_step(OLs[layer], None, X[layer], order, K)
+            assert_values_close(X[layer + 1] - X[layer], res["y"][0], what=f"layer {layer}")
+            # and the refined set handed on is the exact top-k of the residual that left it
+            check_selection(S[layer + 1, :k].astype(np.int64), orc.predictor_scores(nxt, X[layer + 1]), k, stats)
+    stack.close()
+    for g in GLs:
+        g.close()
+
+
+@pytest.mark.parametrize("K", [1, 4, 8])
+def test_tiny4_stack_decode(K):
+    spec = wl.SPECS["tiny4"]
+    stats = {}
+    decode_and_check(spec, wl.make_stack(spec, down_scale=50.0), K, spec.k, 3, stats)
+    assert stats.get("band", 0) == 0
+
+
+def test_stack_decode_matches_layer_by_layer_path():
+    """Same token through ls_stack_decode and through ls_sparse_ffn_step layer by layer: same sets, same values."""
+    spec = wl.SPECS["tiny4"]
+    arrays = wl.make_stack(spec, down_scale=50.0)
+    GLs = [ls.ls_layer_create(a, DEV) for a in arrays]
+    stack = ls.ls_stack_create(GLs)
+    k, K, n = spec.k, 4, len(GLs)
+    x = torch.from_numpy(wl.make_tokens(spec)[5]).cuda(DEV)
+    sel0, sel_out = ls.Selection(spec.d_ff, k, DEV), ls.Selection(spec.d_ff, k, DEV)
+    ls.ls_predict(GLs[0], x, k, sel0)
+    x_stack = torch.empty_like(x)
+    ls.ls_stack_decode(stack, x, x_stack, sel0, K, k, sel_out)
+    sels = [ls.Selection(spec.d_ff, k, DEV) for _ in range(2)]
+    ls.ls_predict(GLs[0], x, k, sels[0])
+    xl = x.clone()
+    for layer in range(n):
+        ls.ls_sparse_ffn_step(GLs[layer], GLs[min(layer + 1, n - 1)], xl, xl, sels[layer % 2], K, k, sels[(layer + 1) % 2])
+    torch.cuda.synchronize()
+    assert sel_out.order().tolist() == sels[n % 2].order().tolist()
+    assert_values_close((x_stack - x).cpu().numpy(), (xl - x).cpu().numpy(), what="stack vs layers")
+    # in place, twice in a row (the scratch is clean again after every launch)
+    for _ in range(2):
+        xi = x.clone()
+        ls.ls_stack_decode(stack, xi, xi, sel0, K, k, sel_out)
+        assert_values_close((xi - x).cpu().numpy(), (xl - x).cpu().numpy(), what="in place")
+    stack.close()
+    for g in GLs:
+        g.close()
+
+
+def test_stack_rejects_cached_layers_and_bad_arguments():
+    spec = wl.SPECS["tiny"]
+    la = wl.make_layer(spec, 0)
+    cached = ls.ls_layer_create(la, DEV, cache_rows=256)
+    with pytest.raises(ls.LeanStreamError) as e:
+        ls.ls_stack_create([cached])
+    assert e.value.code == ls.LS_ERR_STATE
+    plain = ls.ls_layer_create(la, DEV)
+    stack = ls.ls_stack_create([plain])
+    x = torch.zeros(256, device=f"cuda:{DEV}")
+    sel = ls.Selection(1024, 160, DEV)
+    with pytest.raises(ls.LeanStreamError):
+        ls.ls_stack_decode(stack, x, x, sel, 17, 160, sel)  # more stages than the fused kernel supports
+    with pytest.raises(ls.LeanStreamError):
+        ls.ls_stack_decode(stack, x, x, sel, 4, 2000, sel)  # k_next beyond d_ff
+    stack.close()
+    cached.close()
+    plain.close()
+
+
+def test_llama7b_shaped_three_layer_stack():
+    spec = wl.SPECS["llama2-7b"]
+    arrays = [wl.make_layer(spec, l, svd_device="cuda") for l in range(3)]
+    stats = {}
+    decode_and_check(spec, arrays, 8, spec.k, 1, stats)
+    assert stats.get("band", 0) == 0
