@@ -99,6 +99,7 @@ struct ls_layer {
   float* b_gate = nullptr;
   float* b_down = nullptr;
   uint16_t* pred_at = nullptr;  // [r][d]
+  uint16_t* pred_at_sl = nullptr;  // [ceil(d / 32)][r][32] (the fused kernel's column slices)
   uint16_t* pred_bt = nullptr;  // [F][r]
   float* pred_c = nullptr;
 
@@ -159,7 +160,7 @@ int32_t dalloc(T** p, size_t n) {
 void free_layer(ls_layer* L) {
   if (!L) return;
   ls::cache_destroy(L->cache);
-  cudaFree(L->bundles); cudaFree(L->b_gate); cudaFree(L->b_down); cudaFree(L->pred_at); cudaFree(L->pred_bt);
+  cudaFree(L->bundles); cudaFree(L->b_gate); cudaFree(L->b_down); cudaFree(L->pred_at); cudaFree(L->pred_at_sl); cudaFree(L->pred_bt);
   cudaFree(L->pred_c); cudaFree(L->z); cudaFree(L->sumsq); cudaFree(L->scores); cudaFree(L->prio); cudaFree(L->cand_key);
   cudaFree(L->cand_idx); cudaFree(L->umask); cudaFree(L->tmp_idx); cudaFree(L->tmp_count); cudaFree(L->tmp_mask);
   cudaFree(L->fz_range); cudaFree(L->fz_range_obs);
@@ -186,6 +187,20 @@ int32_t upload_transposed16(uint16_t** dst, const void* src, int rows, int cols)
   return LS_OK;
 }
 
+// [d][r] 16-bit host matrix A -> column slices [ceil(d / 32)][r][32] on the device, zero padded: slice s holds the rows
+// 32 s .. 32 s + 31 of A, transposed, so that one contiguous copy brings a slice into shared memory.
+int32_t upload_sliced16(uint16_t** dst, const void* src, int d, int r) {
+  const int nsl = (d + ls::FZ_SL - 1) / ls::FZ_SL;
+  std::vector<uint16_t> t;
+  try { t.assign((size_t)nsl * r * ls::FZ_SL, 0); } catch (const std::bad_alloc&) { return fail(LS_ERR_NOMEM, "host staging buffer"); }
+  const uint16_t* s = static_cast<const uint16_t*>(src);
+  for (int c = 0; c < d; ++c)
+    for (int j = 0; j < r; ++j) t[((size_t)(c / ls::FZ_SL) * r + j) * ls::FZ_SL + (c % ls::FZ_SL)] = s[(size_t)c * r + j];
+  LS_TRY(dalloc(dst, t.size()));
+  LS_CUDA(cudaMemcpy(*dst, t.data(), t.size() * 2, cudaMemcpyHostToDevice));
+  return LS_OK;
+}
+
 // Working scratch of the fused kernel, one per device and shared by all layers on it: a decode loop runs its layers one
 // after the other, and re-using the same few megabytes keeps them in L2 (per-layer copies would come back from HBM at
 // every step).  Consequence: fused steps on one device must not overlap (issue them on one stream, or order the
@@ -194,6 +209,7 @@ struct DeviceScratch {
   float* dacc = nullptr;              // [FZ_MAXK][16384] stage accumulators, zero between launches
   unsigned* ctr = nullptr;            // fin, (pad), barrier counter (64-bit)
   double* z = nullptr;                // [FZ_MAXE][1024] latents, then [FZ_MAXE] sums of squares
+  double* zpart = nullptr;            // [512 slices][FZ_MAXE][1025] per-slice partial latents
   unsigned* cnt = nullptr;            // [FZ_MAXE][FZ_CNT_STRIDE], zero between launches
   uint4* bent = nullptr;              // [FZ_MAXE][FZ_NB * FZ_CAPB] bucket entries
   uint4* oent = nullptr;              // [FZ_MAXE][32768] overflow entries
@@ -213,6 +229,7 @@ int32_t device_scratch(int dev, DeviceScratch** out) {
     LS_TRY(dalloc(&S.dacc, (size_t)2 * ls::FZ_MAXK * kScratchMaxD));  // two parities (whole-token kernel)
     LS_TRY(dalloc(&S.ctr, (size_t)8));
     LS_TRY(dalloc(&S.z, NE * kScratchMaxR + NE));
+    LS_TRY(dalloc(&S.zpart, (size_t)(kScratchMaxD / ls::FZ_SL) * NE * (kScratchMaxR + 1)));
     LS_TRY(dalloc(&S.cnt, 2 * NE * ls::FZ_CNT_STRIDE));
     LS_TRY(dalloc(&S.bent, NE * ls::FZ_NB * ls::FZ_CAPB));
     LS_TRY(dalloc(&S.oent, NE * kScratchMaxF));
@@ -258,6 +275,7 @@ int32_t create_impl(const ls_layer_desc* D, ls_layer* L) {
   LS_TRY(upload_f32(&L->b_gate, D->b_gate, F));
   if (D->b_down) LS_TRY(upload_f32(&L->b_down, D->b_down, d));
   LS_TRY(upload_transposed16(&L->pred_at, D->pred_a, (int)d, L->r));
+  LS_TRY(upload_sliced16(&L->pred_at_sl, D->pred_a, (int)d, L->r));
   LS_TRY(upload_transposed16(&L->pred_bt, D->pred_b, L->r, (int)F));
   LS_TRY(upload_f32(&L->pred_c, D->pred_c, F));
 
@@ -317,13 +335,17 @@ bool fused_plan(const ls_layer* L, const ls_layer* next, ls::FusedSmemLayout* ou
   const size_t budget = 218 * 1024;  // dynamic part; the kernel also has a few KB of static shared memory
   const int n_in = L->gated ? 2 : 1;
   const int r = next ? next->r : 0, Fn = next ? next->F : 0, hn = next ? 1 : 0;
-  // the gate/up ring wants two rounds in flight; the down ring at least one round of survivors
-  for (int gu = ls::FZ_MAX_DEPTH; gu >= ls::FZ_NG + 1; --gu) {
-    for (int dn = 4; dn >= ls::FZ_NG; --dn) {
-      const ls::FusedSmemLayout lay = ls::fused_layout(L->d, n_in, r, Fn, L->sm_count, hn, gu, dn);
-      if (lay.total <= budget) {
-        if (out) *out = lay;
-        return true;
+  // The gate/up ring wants two rounds in flight and the down ring as many rows as memory latency covers; a down row is
+  // half (gated) or all of a gate/up slot, so depth is traded between the two rings at that rate.  The A slices keep a
+  // place of their own (they can then arrive while the rings are still busy) unless that costs the rings their depth.
+  for (int alias = 0; alias <= 1; ++alias) {
+    for (int gu = ls::FZ_MAX_DEPTH; gu >= ls::FZ_NG + 1; --gu) {
+      for (int dn = ls::FZ_MAX_DEPTH; dn >= ls::FZ_NG + 1; --dn) {
+        const ls::FusedSmemLayout lay = ls::fused_layout(L->d, n_in, r, Fn, L->sm_count, hn, gu, dn, alias);
+        if (lay.total <= budget && (alias == 1 || (gu >= 6 && dn >= 6))) {
+          if (out) *out = lay;
+          return true;
+        }
       }
     }
   }
@@ -368,9 +390,9 @@ int32_t fused_args(ls_layer* L, ls_layer* next, const float* d_x, float* d_x_out
   a.status = L->status;
   a.has_next = next ? 1 : 0;
   if (next) {
-    a.At = next->pred_at; a.Bt = next->pred_bt; a.pc = next->pred_c;
+    a.At_sl = next->pred_at_sl; a.Bt = next->pred_bt; a.pc = next->pred_c;
     a.r = next->r; a.Fn = next->F; a.norm_n = next->norm; a.eps_n = next->eps; a.k_next = k_next;
-    a.z = S->z; a.sumsq = S->z + (size_t)ls::FZ_MAXE * next->r; a.range = next->fz_range;
+    a.z = S->z; a.sumsq = S->z + (size_t)ls::FZ_MAXE * next->r; a.zpart = S->zpart; a.range = next->fz_range;
     a.cnt = S->cnt + (size_t)parity * ls::FZ_MAXE * ls::FZ_CNT_STRIDE; a.bent = S->bent; a.oent = S->oent;
     a.range_obs = next->fz_range_obs; a.nsel = S->nsel + (size_t)parity * ls::FZ_MAXE;
     if (sel_next) {
@@ -381,7 +403,7 @@ int32_t fused_args(ls_layer* L, ls_layer* next, const float* d_x, float* d_x_out
   }
   ls::FusedSmemLayout lay{};
   if (!fused_plan(L, next, &lay)) return fail(LS_ERR_STATE, "fused step: shared memory plan failed");
-  a.gu_depth = lay.gu_depth; a.dn_depth = lay.dn_depth;
+  a.gu_depth = lay.gu_depth; a.dn_depth = lay.dn_depth; a.a_alias = lay.a_alias;
   *out = a;
   if (lay_out) *lay_out = lay;
   return LS_OK;
@@ -689,6 +711,12 @@ int32_t ls_topk_select_static(const double* d_scores, int32_t n, int32_t k, int3
 #ifdef LS_FZ_TIMING
 int32_t ls_debug_read_timing(long long* host, int32_t n) {
   return cudaMemcpyFromSymbol(host, ls::g_fz_timing, (size_t)n * sizeof(long long)) == cudaSuccess ? LS_OK : LS_ERR_CUDA;
+}
+int32_t ls_debug_read_fail(int* host) {
+  return cudaMemcpyFromSymbol(host, ls::g_fz_fail, 64 * sizeof(int)) == cudaSuccess ? LS_OK : LS_ERR_CUDA;
+}
+int32_t ls_debug_read_cta(long long* host, int32_t n) {
+  return cudaMemcpyFromSymbol(host, ls::g_fz_cta, (size_t)n * sizeof(long long)) == cudaSuccess ? LS_OK : LS_ERR_CUDA;
 }
 #endif
 

@@ -37,9 +37,17 @@ constexpr int FZ_MAXK = 16;       // stages supported by the fused path
 constexpr int FZ_MAXE = FZ_MAXK + 1;  // evaluations j = 0..K
 constexpr int FZ_BPAD = 8;        // padding (elements) of a predictor row in shared memory: eight rows on distinct banks
 constexpr int FZ_ZPAD = 4;        // padding (doubles) of a latent row in shared memory
-constexpr int FZ_MAX_DEPTH = 8;   // most ring stages; the depths are chosen per launch from the shared memory left
+constexpr int FZ_MAX_DEPTH = 8;   // most gate/up ring stages; the depths are chosen per launch from the shared memory left
+constexpr int FZ_MAX_DN = 16;     // most down ring stages
+constexpr int FZ_SL = 32;         // columns of the feature handled as one slice in the latent phase
+constexpr int FZ_EPAD = 24;       // evaluations rounded up to whole tiles of eight
+constexpr int FZ_KS = 4;          // column splits of a score tile (more independent tasks than warps)
 constexpr int FZ_MAX_MINE = 256;  // neurons one CTA may own in one step
+#ifdef LS_FZ_TIMING
+constexpr long long FZ_SPIN_CYCLES = 40LL * 1000 * 1000;
+#else
 constexpr long long FZ_SPIN_CYCLES = 4000LL * 1000 * 1000;  // every wait gives up after about two seconds of SM clocks
+#endif
 
 struct FusedArgs {
   // layer being executed
@@ -48,16 +56,19 @@ struct FusedArgs {
   const float* x; float* x_out;
   const int32_t* sel_idx; const int32_t* sel_count; int sel_cap; int K;
   int gu_depth, dn_depth; // ring stages (host: as many as fit)
+  int a_alias;            // the A slices share bytes with the rings (see fused_layout)
   float* dacc;            // [FZ_MAXK][d] stage accumulators, zero on entry and on exit
   unsigned* fin;          // [1] CTAs finished, zero on entry and on exit
   unsigned long long* bar_count;  // [1] barrier arrivals since the layer was created (monotonic)
   int* status;
   // next layer's predictor (has_next == 0: no refinement)
   int has_next;
-  const uint16_t* At; const uint16_t* Bt; const float* pc;
+  const uint16_t* At_sl;  // A of the next layer's predictor by column slices: [ceil(d / 32)][r][32], zero padded
+  const uint16_t* Bt; const float* pc;
   int r, Fn, norm_n; float eps_n; int k_next;
   double* z;              // [FZ_MAXE][r] un-normalised latents
   double* sumsq;          // [FZ_MAXE]
+  double* zpart;          // [slices][K + 1][r + 1] per-slice partial latents; entry r of a row: partial sum of squares
   unsigned* cnt;          // [FZ_MAXE][FZ_CNT_STRIDE], zero on entry and on exit
   uint4* bent;            // [FZ_MAXE][FZ_NB * FZ_CAPB] bucket entries {key lo, key hi, neuron, fine bin}, one 16-byte store each
   uint4* oent;            // [FZ_MAXE][Fn] overflow entries, same format
@@ -77,8 +88,29 @@ __device__ long long g_fz_timing[2][512];
   do {                                                                            \
     if (blockIdx.x == 0 && (slot) < 512) g_fz_timing[role][slot] = clock64();     \
   } while (0)
+__device__ long long g_fz_cta[160][16];
+__device__ int g_fz_fail[64];  // first failures: site, cta, tid, extra
+__device__ int g_fz_nfail;
+__device__ __forceinline__ void fz_fail(int site, int extra) {
+  const int k = atomicAdd(&g_fz_nfail, 1);
+  if (k < 16) { g_fz_fail[k * 4] = site; g_fz_fail[k * 4 + 1] = blockIdx.x; g_fz_fail[k * 4 + 2] = threadIdx.x; g_fz_fail[k * 4 + 3] = extra; }
+}
+#define FZ_FAIL(site, extra) fz_fail(site, extra)  // per-CTA wall-clock stamps (ns) and counters
+__device__ __forceinline__ long long fz_now() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return (long long)t; }
+#define FZ_STAMP_DEP(role, slot, fval)                                           \
+  do {                                                                            \
+    long long c_;                                                                 \
+    asm volatile("{ .reg .f32 t_; mov.f32 t_, %1; mov.u64 %0, %%clock64; }" : "=l"(c_) : "f"(fval)); \
+    if (blockIdx.x == 0 && (slot) < 512) g_fz_timing[role][slot] = c_;            \
+  } while (0)
+#define FZ_CSTAMP(slot) do { if (blockIdx.x < 160) g_fz_cta[blockIdx.x][slot] = fz_now(); } while (0)
+#define FZ_CVAL(slot, v) do { if (blockIdx.x < 160) g_fz_cta[blockIdx.x][slot] = (v); } while (0)
 #else
 #define FZ_STAMP(role, slot) do { } while (0)
+#define FZ_STAMP_DEP(role, slot, fval) do { } while (0)
+#define FZ_FAIL(site, extra) do { } while (0)
+#define FZ_CSTAMP(slot) do { } while (0)
+#define FZ_CVAL(slot, v) do { } while (0)
 #endif
 
 // ---- PTX helpers ---------------------------------------------------------------------------------------------------
@@ -140,7 +172,7 @@ __device__ __forceinline__ void grid_barrier(const FusedArgs& A, int G) {
       asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(A.bar_count) : "memory");
       if (v >= target) { ok = true; break; }
     } while (clock64() - t0 < FZ_SPIN_CYCLES);
-    if (!ok) set_status(A.status, ST_TIMEOUT);
+    if (!ok) { set_status(A.status, ST_TIMEOUT); FZ_FAIL(6, (int)target); }
   }
   named_bar_sync(1, FZ_THREADS);
 }
@@ -161,32 +193,54 @@ __host__ __device__ inline int fz_stage_of_cta(int cta, int G, int K) {
 }
 
 struct FusedSmemLayout {
-  size_t gu_off, dn_off, bar_off, red_off, redd_off, mine_off, a_off, b_off, pc_off, zs_off, own_off, bin_off, coarse_off, total;
-  int per, nA, gu_depth, dn_depth;
+  // fixed regions
+  size_t bar_off, red_off, redd_off, mine_off, pc_off, xt_off, qa_off, a_off;
+  // the stream's rings ...
+  size_t gu_off, dn_off;
+  // ... and, in the same bytes once the rings have drained, the operands and results of the refinement
+  size_t b_off, zs_off, part_off, own_off, bin_off, coarse_off;
+  size_t total;
+  int per, ns_cta, a_alias, gu_depth, dn_depth;
 };
 
-__host__ __device__ inline FusedSmemLayout fused_layout(int d, int n_in, int r, int Fn, int G, int has_next, int gu_depth, int dn_depth) {
+// Bar indices: [0, FZ_MAX_DEPTH) gate/up slots, [FZ_MAX_DEPTH, +FZ_MAX_DN) down slots, then the A slices, then B^T rows.
+constexpr int FZ_BAR_DN = FZ_MAX_DEPTH, FZ_BAR_A = FZ_MAX_DEPTH + FZ_MAX_DN, FZ_BAR_B = FZ_BAR_A + 1, FZ_NBAR = FZ_BAR_B + 1;
+
+// `a_alias` != 0 places the A slices inside the ring bytes too (they are then fetched only after the rings have drained).
+__host__ __device__ inline FusedSmemLayout fused_layout(int d, int n_in, int r, int Fn, int G, int has_next, int gu_depth, int dn_depth,
+                                                        int a_alias) {
   FusedSmemLayout L{};
   L.gu_depth = gu_depth;
   L.dn_depth = dn_depth;
+  L.a_alias = a_alias;
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t at = o; o += (bytes + 127) & ~(size_t)127; return at; };
+  const int nsl = (d + FZ_SL - 1) / FZ_SL;
+  L.per = has_next ? (Fn + G - 1) / G : 0;
+  L.ns_cta = (nsl + G - 1) / G;
+  const size_t a_bytes = has_next ? (size_t)L.ns_cta * r * FZ_SL * 2 : 0;
+  L.bar_off = take(FZ_NBAR * 8);
+  L.red_off = take(2 * 16 * 8 * 4);                  // stream dot partials, double-buffered: [2][warp][8]
+  L.redd_off = take(32 * 8);                         // fp64 partials of block reductions
+  L.mine_off = take((size_t)FZ_MAX_MINE * 8);        // this CTA's neuron indices and gate biases
+  L.pc_off = take((size_t)L.per * 4);
+  L.xt_off = take((size_t)FZ_EPAD * (FZ_SL + 4) * 8);  // x~^(j) of one slice, fp64, padded rows
+  L.qa_off = take(FZ_MAX_DN * 4);                    // activations of the queued down rows
+  if (!a_alias) L.a_off = take(a_bytes);
+  const size_t base = o;
   L.gu_off = take((size_t)gu_depth * n_in * d * 2);
   L.dn_off = take((size_t)dn_depth * d * 2);
-  L.bar_off = take((2 * FZ_MAX_DEPTH + 2) * 8);
-  L.red_off = take(2 * 16 * 8 * 4);                  // stream dot partials, double-buffered: [2][warp][8]
-  L.redd_off = take((size_t)FZ_MAXE * 3 * 16 * 8);   // fp64 partials of the latent phase: [evaluation][row0,row1,sumsq][warp]
-  L.mine_off = take((size_t)FZ_MAX_MINE * 8);        // this CTA's neuron indices and gate biases
-  L.per = has_next ? (Fn + G - 1) / G : 0;
-  L.nA = has_next ? (r + G - 1) / G : 0;
-  L.a_off = take((size_t)L.nA * d * 2);
-  L.b_off = take((size_t)((L.per + 7) / 8 * 8) * (r + FZ_BPAD) * 2);
-  L.pc_off = take((size_t)L.per * 4);
-  L.zs_off = take((size_t)(has_next ? 8 * (r + FZ_ZPAD) : 0) * 8);
+  const size_t end_stream = o;
+  o = base;
+  if (a_alias) L.a_off = take(a_bytes);
+  const int per8 = (L.per + 7) / 8 * 8;
+  L.b_off = take((size_t)per8 * (r + FZ_BPAD) * 2);
+  L.zs_off = take(has_next ? (size_t)FZ_EPAD * (r + FZ_ZPAD) * 8 : 0);
+  L.part_off = take(has_next ? (size_t)FZ_KS * FZ_EPAD * per8 * 8 : 0);  // [split][evaluation][neuron]
   L.own_off = take((size_t)FZ_MAXE * L.per * 8);     // this CTA's scores, every evaluation
   L.bin_off = take((size_t)FZ_MAXE * L.per * 2);     // and their fine bins
   L.coarse_off = take(has_next ? (size_t)FZ_MAXE * (FZ_NC + 1) * 4 : 0);
-  L.total = o;
+  L.total = o > end_stream ? o : end_stream;
   return L;
 }
 
@@ -197,9 +251,10 @@ struct FusedShared {
   FusedArgs prev;                    // whole-token kernel: the layer before, whose scratch is cleaned meanwhile
   int last;
   int round;                         // rounds the compute warps have finished (read by the producer)
+  unsigned phase[FZ_NBAR];           // phases every mbarrier has completed in earlier layers of the launch
   int mail[4 * 4];                   // per round (ring of four): number of survivors, their neurons
   float act[2 * 4];                  // activations of the round's neurons, double-buffered
-  double inv[8];
+  double inv[FZ_EPAD];
   int cut[FZ_MAXE * 4];              // per evaluation: cut fine bin, its first rank, threshold neuron, fallback flag
   unsigned long long cutkey[FZ_MAXE];  // threshold key inside the cut bin
   unsigned nsel[FZ_MAXE];            // members found by this CTA, per evaluation
@@ -209,23 +264,25 @@ struct FusedShared {
 
 // One layer step, executed by the whole block (16 compute warps + the producer warp).  The producer warp returns as
 // soon as it has issued its last copy; the compute warps return when the layer's refined sets are written.
-// `reinit` says that the mbarriers in shared memory were used by an earlier layer of the same launch.
+// `first_layer` says that this is the first layer of the launch (the mbarriers in shared memory are set up then).
 template <int WD, int CPT>
-__device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* smem, FusedShared& sh, bool reinit) {
+__device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* smem, FusedShared& sh, bool first_layer) {
   const int G = gridDim.x, cta = blockIdx.x, tid = threadIdx.x;
   const int lane = tid & 31, warp = tid >> 5;
   const int d = A.d, K = A.K, nchunk = A.d >> 3;
   const int n_in = A.gated ? 2 : 1;
-  const FusedSmemLayout lay = fused_layout(d, n_in, A.r, A.Fn, G, A.has_next, A.gu_depth, A.dn_depth);
+  const FusedSmemLayout lay = fused_layout(d, n_in, A.r, A.Fn, G, A.has_next, A.gu_depth, A.dn_depth, A.a_alias);
   const int GU = A.gu_depth, DN = A.dn_depth;
   uint16_t* s_gu = reinterpret_cast<uint16_t*>(smem + lay.gu_off);
   uint16_t* s_dn = reinterpret_cast<uint16_t*>(smem + lay.dn_off);
-  uint64_t* s_bar = reinterpret_cast<uint64_t*>(smem + lay.bar_off);  // [0..GU) gate/up full, [FZ_MAX_DEPTH..+DN) down full
+  uint64_t* s_bar = reinterpret_cast<uint64_t*>(smem + lay.bar_off);  // "full" barriers: gate/up slots, down slots, A, B^T
   float* s_red = reinterpret_cast<float*>(smem + lay.red_off);        // [2][16 warps][8]
   double* s_redd = reinterpret_cast<double*>(smem + lay.redd_off);
-  uint16_t* s_A = reinterpret_cast<uint16_t*>(smem + lay.a_off);      // [nA][d]
-  uint16_t* s_B = reinterpret_cast<uint16_t*>(smem + lay.b_off);      // [per][r]
+  uint16_t* s_A = reinterpret_cast<uint16_t*>(smem + lay.a_off);      // [ns_cta][r][32]
+  uint16_t* s_B = reinterpret_cast<uint16_t*>(smem + lay.b_off);      // [per][r + FZ_BPAD]
   float* s_pc = reinterpret_cast<float*>(smem + lay.pc_off);
+  double* s_xt = reinterpret_cast<double*>(smem + lay.xt_off);        // [K+1][32]
+  float* s_qa = reinterpret_cast<float*>(smem + lay.qa_off);          // [DN]
   int& s_round = sh.round;
   int* s_mail = sh.mail;
   float* s_act = sh.act;
@@ -236,22 +293,27 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
   unsigned long long* s_kmm = sh.kmm;
   unsigned* s_ccnt = sh.ccnt;
 
-  if (tid == 0) {
-    if (reinit)  // every copy of the earlier layer has completed; its barriers are retired before the new ones are set up
-      for (int i = 0; i <= 2 * FZ_MAX_DEPTH + 1; ++i) asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(smem_u32(&s_bar[i])) : "memory");
-    for (int i = 0; i < 2 * FZ_MAX_DEPTH; ++i) mbar_init(&s_bar[i], 1);
-    mbar_init(&s_bar[2 * FZ_MAX_DEPTH], 1);
-    mbar_init(&s_bar[2 * FZ_MAX_DEPTH + 1], 1);
-    s_round = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  if (tid == 0) FZ_CSTAMP(0);
+  // The mbarriers are set up once per launch and keep running from layer to layer: sh.phase[b] counts the phases barrier
+  // b has completed so far, so a wait for the t-th use of a barrier in this layer asks for parity (phase[b] + t) & 1.
+  unsigned* s_phase = sh.phase;
+  if (first_layer) {
+    if (tid == 0) {
+      for (int i = 0; i < FZ_NBAR; ++i) mbar_init(&s_bar[i], 1);
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (tid < FZ_NBAR) s_phase[tid] = 0u;
   }
+  if (tid == 0) s_round = 0;
   __syncthreads();
+  if (tid == 0) FZ_STAMP(1, 20);
 
   const int per = lay.per, r = A.r, Fn = A.Fn;
   const int i_lo = cta * per, i_hi = min(Fn, i_lo + per);
   const int n_own = max(0, i_hi - i_lo);
-  const bool feat_writer = (cta == 0);
+  const int nsl = (d + FZ_SL - 1) / FZ_SL;  // column slices of the feature; this CTA takes slices cta, cta + G, ...
+  int used_gu = 0, used_dn = 0;            // gate/up rows and down rows this CTA fetched in this layer
 
   {
     // ================================================= stream: all warps ===========================================
@@ -292,6 +354,7 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
       for (int e = 0; e < 8; ++e) sq = fma((double)xr[q][e], (double)xr[q][e], sq);
     }
     __syncthreads();  // indices visible (the producer warp takes part in this barrier, then goes its own way)
+    if (tid == 0) FZ_STAMP(1, 21);
 
     if (warp == FZ_THREADS / 32) {
       // ============================================= producer warp (one lane) ======================================
@@ -307,16 +370,34 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
         };
         for (int it = 0; it < min(n_mine, GU); ++it) issue_gu(it);
         const int n_rounds = (n_mine + FZ_NG - 1) / FZ_NG;
-        int tail = 0;
-        for (int rd = 0; rd < n_rounds; ++rd) {
+        auto wait_round = [&](int want) {  // the compute warps have finished `want` rounds (n_rounds + 1: rings drained)
           const long long t0 = clock64();
-          bool ok = false;
           do {
             int v;
             asm volatile("ld.acquire.cta.shared.s32 %0, [%1];" : "=r"(v) : "r"(smem_u32(&s_round)) : "memory");
-            if (v > rd) { ok = true; break; }
+            if (v >= want) return true;
           } while (clock64() - t0 < FZ_SPIN_CYCLES);
-          if (!ok) { set_status(A.status, ST_TIMEOUT); break; }
+          set_status(A.status, ST_TIMEOUT);
+          FZ_FAIL(1, want);
+          return false;
+        };
+        auto issue_a = [&]() {  // this CTA's column slices of the next layer's A
+          uint64_t* abar = &s_bar[FZ_BAR_A];
+          uint32_t bytes = 0;
+          for (int a = 0; a < lay.ns_cta; ++a)
+            if (cta + a * G < nsl) bytes += (uint32_t)r * FZ_SL * 2;
+          mbar_expect_tx(abar, bytes);
+          for (int a = 0; a < lay.ns_cta; ++a) {
+            const int sl = cta + a * G;
+            if (sl < nsl)
+              tma_load_1d(s_A + (size_t)a * r * FZ_SL, A.At_sl + (size_t)sl * r * FZ_SL, (uint32_t)r * FZ_SL * 2, abar);
+          }
+        };
+        int tail = 0;
+        bool ok = true;
+        for (int rd = 0; rd < n_rounds && ok; ++rd) {
+          ok = wait_round(rd + 1);
+          if (!ok) break;
           const int it0 = rd * FZ_NG, nn = min(FZ_NG, n_mine - it0);
           for (int e = 0; e < nn; ++e)
             if (it0 + e + GU < n_mine) issue_gu(it0 + e + GU);
@@ -325,29 +406,24 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
           for (int e = 0; e < ns; ++e) {
             const int i = mail[1 + e];
             const int ds = tail % DN;
-            uint64_t* bar = &s_bar[FZ_MAX_DEPTH + ds];
+            uint64_t* bar = &s_bar[FZ_BAR_DN + ds];
             mbar_expect_tx(bar, dn_bytes);
             tma_load_1d(s_dn + (size_t)ds * d, A.bundles + (size_t)i * bundle_elems + (size_t)(A.n_mat - 1) * d, dn_bytes, bar);
             if (A.tr_survive) atomicOr(&A.tr_survive[i >> 5], 1u << (i & 31));
             ++tail;
           }
         }
-        // last, off the streaming's critical path: the predictor operands are needed only after the first grid barrier
-        if (A.has_next) {
-          // this CTA's share of the next layer's predictor, as stored: rows of A^T, rows of B^T (padded row stride)
-          uint64_t* abar = &s_bar[2 * FZ_MAX_DEPTH];      // rows of A^T: awaited before the latent phase
-          uint64_t* bbar = &s_bar[2 * FZ_MAX_DEPTH + 1];  // rows of B^T: awaited before the score phase
-          uint32_t bytes = 0;
-          for (int a = 0; a < lay.nA; ++a)
-            if (cta + a * G < r) bytes += (uint32_t)d * 2;
-          mbar_expect_tx(abar, bytes);
-          for (int a = 0; a < lay.nA; ++a) {
-            const int j = cta + a * G;
-            if (j < r) tma_load_1d(s_A + (size_t)a * d, A.At + (size_t)j * d, (uint32_t)d * 2, abar);
+        // The next layer's predictor operands, off the streaming's critical path.  A slices that have a place of their
+        // own are fetched now; everything that shares bytes with the rings waits until the compute warps have drained them.
+        if (A.has_next && ok) {
+          if (!lay.a_alias) issue_a();
+          if (wait_round(n_rounds + 1)) {
+            if (lay.a_alias) issue_a();
+            uint64_t* bbar = &s_bar[FZ_BAR_B];  // rows of B^T: awaited before the score phase
+            mbar_expect_tx(bbar, (uint32_t)n_own * (uint32_t)r * 2);
+            for (int li = 0; li < n_own; ++li)
+              tma_load_1d(s_B + (size_t)li * (r + FZ_BPAD), A.Bt + (size_t)(i_lo + li) * r, (uint32_t)r * 2, bbar);
           }
-          mbar_expect_tx(bbar, (uint32_t)n_own * (uint32_t)r * 2);
-          for (int li = 0; li < n_own; ++li)
-            tma_load_1d(s_B + (size_t)li * (r + FZ_BPAD), A.Bt + (size_t)(i_lo + li) * r, (uint32_t)r * 2, bbar);
         }
       }
       return;  // an exited warp counts as arrived at every later block barrier
@@ -361,14 +437,15 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
       for (int li = tid; li < n_own; li += FZ_THREADS) s_pc[li] = A.pc ? A.pc[i_lo + li] : 0.f;
     sq = warp_sum(sq);
     if (lane == 0) s_redd[warp] = sq;
+    if (tid == 0) FZ_STAMP(1, 22);
     named_bar_sync(1, FZ_THREADS);
+    if (tid == 0) FZ_STAMP(1, 23);
     double tot = 0.0;
 #pragma unroll
     for (int w = 0; w < FZ_THREADS / 32; ++w) tot += s_redd[w];
     const float inv_rms = A.norm == 0 ? (float)(1.0 / sqrt(tot / (double)d + (double)A.eps)) : 1.0f;
 
-    // pending down rows: FIFO over the down ring; every thread tracks the same activations in registers
-    float qa[4] = {0.f, 0.f, 0.f, 0.f};
+    // pending down rows: FIFO over the down ring; their activations wait in s_qa, every thread tracks head and tail
     int dq_head = 0, dq_tail = 0;
     float yacc[CPT][8];
 #pragma unroll
@@ -377,14 +454,12 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
       for (int e = 0; e < 8; ++e) yacc[q][e] = 0.f;
     bool dirty = false;
     if (tid == 0) FZ_STAMP(0, 0);
+    if (tid == 0) { FZ_CSTAMP(1); FZ_CVAL(8, n_mine); FZ_CVAL(10, stage); }
 
     auto consume_one = [&]() {  // the oldest pending down row, scaled, joins the CTA's partial output
       const int slot = dq_head % DN;
-      mbar_wait(&s_bar[FZ_MAX_DEPTH + slot], (uint32_t)((dq_head / DN) & 1), A.status);
-      float a = qa[0];
-#pragma unroll
-      for (int e = 1; e < 4; ++e)
-        if (slot == e) a = qa[e];
+      if (!mbar_wait(&s_bar[FZ_BAR_DN + slot], (s_phase[FZ_BAR_DN + slot] + (uint32_t)(dq_head / DN)) & 1u, A.status)) FZ_FAIL(3, dq_head);
+      const float a = s_qa[slot];
       const uint16_t* row = s_dn + (size_t)slot * d;
 #pragma unroll
       for (int q = 0; q < CPT; ++q) {
@@ -415,7 +490,7 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
         pu[e] = 0.f;
         if (e < nn) {
           const int it = it0 + e, slot = it % GU;
-          mbar_wait(&s_bar[slot], (uint32_t)((it / GU) & 1), A.status);
+          if (!mbar_wait(&s_bar[slot], (s_phase[slot] + (uint32_t)(it / GU)) & 1u, A.status)) FZ_FAIL(2, it);
           const uint16_t* grow = s_gu + (size_t)slot * n_in * d;
 #pragma unroll
           for (int q = 0; q < CPT; ++q) {
@@ -471,9 +546,13 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
         } else if (!(lane & 1) && e < FZ_NG) {
           s_act[(rd & 1) * 4 + e] = 0.f;
         }
-        // survivors in neuron order -> mailbox of the round
+        // survivors in neuron order -> mailbox of the round, activations -> the queue slots their rows will use
         const unsigned surv = __ballot_sync(0xffffffffu, a != 0.f);
-        if (a != 0.f) s_mail[(rd & 3) * 4 + 1 + __popc(surv & ((1u << lane) - 1u))] = i;
+        if (a != 0.f) {
+          const int pos = __popc(surv & ((1u << lane) - 1u));
+          s_mail[(rd & 3) * 4 + 1 + pos] = i;
+          s_qa[(dq_tail + pos) % DN] = a;
+        }
         if (lane == 0) {
           s_mail[(rd & 3) * 4] = __popc(surv);
           asm volatile("st.release.cta.shared.s32 [%0], %1;" ::"r"(smem_u32(&s_round)), "r"(rd + 1) : "memory");
@@ -481,22 +560,17 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
       }
       named_bar_sync(1, FZ_THREADS);
       if (tid == 0) FZ_STAMP(0, 3 + rd * 4);
-      // (4) every thread queues the survivors' activations in the same order as the producer queued their rows
-#pragma unroll
-      for (int e = 0; e < FZ_NG; ++e) {
-        const float a = s_act[(rd & 1) * 4 + e];
-        if (e < nn && a != 0.f) {
-          const int ds = dq_tail % DN;
-#pragma unroll
-          for (int t = 0; t < 4; ++t)
-            if (ds == t) qa[t] = a;
-          ++dq_tail;
-        }
-      }
+      // (4) the survivors' rows were queued by the producer in the same order
+      dq_tail += s_mail[(rd & 3) * 4];
       if (tid == 0) FZ_STAMP(0, 4 + rd * 4);
     }
     if (tid == 0) FZ_STAMP(0, 500);
+    if (tid == 0) { FZ_CSTAMP(2); FZ_CVAL(9, dq_tail); }
     while (dq_head < dq_tail) consume_one();
+    used_gu = n_mine;
+    used_dn = dq_tail;
+    named_bar_sync(1, FZ_THREADS);  // nobody reads the rings any more: the producer may overwrite them
+    if (tid == 0) asm volatile("st.release.cta.shared.s32 [%0], %1;" ::"r"(smem_u32(&s_round)), "r"(n_rounds + 1) : "memory");
     // the CTA's whole contribution to its stage, added once (vector reductions; order across CTAs is not fixed)
     if (dirty) {
       float* dst = A.dacc + (size_t)stage * d;
@@ -510,131 +584,139 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
       }
     }
     if (tid == 0) FZ_STAMP(0, 501);
-    if (A.has_next) mbar_wait(&s_bar[2 * FZ_MAX_DEPTH], 0u, A.status);  // the rows of A^T have landed (B^T is awaited later)
+    if (tid == 0) FZ_CSTAMP(3);
   }
 
-  // ------------------------------------------------------------------------------------------------ barrier 1 of 3
+  // ------------------------------------------------------------------------------------------------ barrier 1 of 5
   if (tid == 0) FZ_STAMP(1, 0);
+  if (tid == 0) FZ_CSTAMP(4);
   grid_barrier(A, G);
   if (tid == 0) FZ_STAMP(1, 1);
+  if (tid == 0) FZ_CSTAMP(5);
 
-  // ============================ phase 2: partial features x~^(j) and this CTA's latent rows ===========================
-  // Each thread owns d/512 columns.  For every j = 0..K it rebuilds x~^(j) of its columns (x + the stage accumulators
-  // below j) and accumulates the dot products with this CTA's rows of A^T; rows are taken two at a time.
-  constexpr int XC = 8 * CPT;     // columns per thread (d <= 4096 * CPT)
-  float* s_xfin = reinterpret_cast<float*>(smem + lay.gu_off);  // x~^(K), kept by the CTA that writes x_out (the ring is idle now)
-  if (A.has_next || feat_writer) {
-    constexpr int JG = 4;         // evaluations accumulated together
-    const int npair = A.has_next ? max(1, (lay.nA + 1) / 2) : 1;
-    for (int pr = 0; pr < npair; ++pr) {
-      const int a0 = pr * 2;
-      const bool one = A.has_next && a0 < lay.nA, two = A.has_next && a0 + 1 < lay.nA;
-      const int sq_eval = (pr == 0 && cta <= K) ? cta : -1;  // CTA j provides the sum of squares of x~^(j)
-      float xs[XC];  // x~^(j) of this thread's columns, advanced stage by stage
+  // ============================ phase 2: partial features x~^(j), per-slice partial latents ==========================
+  // The columns of the feature are cut into slices of 32; a CTA owns slices cta, cta + G, ...  For each it rebuilds
+  // x~^(j), j = 0..K, of its columns (x + the stage accumulators below j, Eq. 2), writes x_out = x~^(K), and multiplies
+  // the slice of A (r x 32, in shared memory) with the 32 x (K+1) block of features on the fp64 tensor cores.  The
+  // partial latents (and the partial sums of squares, as row r) go to global memory, one block per slice.
+  const int E = K + 1, NT = (E + 7) >> 3, RS = r + 1;
+  constexpr int XTS = FZ_SL + 4;  // row stride (doubles) of s_xt: the four rows a half-warp reads sit on distinct banks
+  if (A.has_next && cta < nsl)
+    if (!mbar_wait(&s_bar[FZ_BAR_A], s_phase[FZ_BAR_A] & 1u, A.status)) FZ_FAIL(4, 0);  // the A slices have landed
+  if (tid == 0) FZ_STAMP(1, 10);
+  for (int a = 0; cta + a * G < nsl; ++a) {
+    const int sl = cta + a * G;
+    if (a > 0) named_bar_sync(1, FZ_THREADS);  // the previous slice's features are no longer read
+    if (tid < FZ_SL) {
+      const int c = sl * FZ_SL + tid;
+      float* const trx = A.tr_xtilde;  // (the arguments live in shared memory: read them once, not after every store)
+      float* const xo = A.x_out;
+      float dv[FZ_MAXK];
+      float xv = 0.f;
 #pragma unroll
-      for (int q = 0; q < XC; ++q) {
-        const int c = tid + q * FZ_THREADS;
-        xs[q] = c < d ? __ldcg(A.x + c) + (A.b_down ? A.b_down[c] : 0.f) : 0.f;
-      }
-      for (int j0 = 0; j0 <= K; j0 += JG) {
-        double p0[JG], p1[JG], sq[JG];
+      for (int j = 0; j < FZ_MAXK; ++j) dv[j] = (c < d && j < K) ? __ldcg(A.dacc + (size_t)j * d + c) : 0.f;
+      if (c < d) xv = __ldcg(A.x + c) + (A.b_down ? A.b_down[c] : 0.f);
+#ifdef LS_FZ_TIMING
+      if (tid == 0) { FZ_STAMP_DEP(1, 13, xv); float q_ = 0.f; for (int j = 0; j < FZ_MAXK; ++j) q_ += dv[j]; FZ_STAMP_DEP(1, 14, q_); }
+#endif
 #pragma unroll
-        for (int e = 0; e < JG; ++e) { p0[e] = 0.0; p1[e] = 0.0; sq[e] = 0.0; }
-        if (tid == 0) FZ_STAMP(1, 10 + j0);
-        // the stage accumulators this group needs, all fetched before anything is stored
-        float dv[XC][JG];
-#pragma unroll
-        for (int q = 0; q < XC; ++q) {
-          const int c = tid + q * FZ_THREADS;
-#pragma unroll
-          for (int e = 0; e < JG; ++e) dv[q][e] = (c < d && j0 + e < K) ? __ldcg(A.dacc + (size_t)(j0 + e) * d + c) : 0.f;
-        }
-#pragma unroll
-        for (int q = 0; q < XC; ++q) {
-          const int c = tid + q * FZ_THREADS;
-          if (c < d) {
-            const double w0 = one ? w16_to_double<WD>(s_A[(size_t)a0 * d + c]) : 0.0;
-            const double w1 = two ? w16_to_double<WD>(s_A[(size_t)(a0 + 1) * d + c]) : 0.0;
-            float xv = xs[q];
-#pragma unroll
-            for (int e = 0; e < JG; ++e) {
-              const int j = j0 + e;
-              if (j <= K) {
-                const double xd = (double)xv;
-                p0[e] = fma(w0, xd, p0[e]);
-                p1[e] = fma(w1, xd, p1[e]);
-                if (j == sq_eval) sq[e] = fma(xd, xd, sq[e]);
-                if (feat_writer && pr == 0) {
-                  if (A.tr_xtilde) A.tr_xtilde[(size_t)j * d + c] = xv;
-                  if (j == K) s_xfin[c] = xv;
-                }
-                xv += dv[q][e];
-              }
-            }
-            xs[q] = xv;
+      for (int j = 0; j < FZ_EPAD; ++j) {
+        if (j < NT * 8) {
+          s_xt[j * XTS + tid] = j <= K ? (double)xv : 0.0;
+          if (j <= K && c < d) {
+            if (trx) trx[(size_t)j * d + c] = xv;
+            if (j == K) xo[c] = xv;  // may alias x: this thread is the only one that still needs x[c]
           }
+          if (j < FZ_MAXK) xv += dv[j];
         }
+      }
+    }
+    named_bar_sync(1, FZ_THREADS);
+    if (tid == 0) FZ_STAMP(1, 11);
+    if (A.has_next) {
+      double* part = A.zpart + (size_t)sl * E * RS;
+      const uint16_t* As = s_A + (size_t)a * r * FZ_SL;
+      const int n_rt = (r + 7) >> 3;
+      for (int mt = warp; mt < n_rt; mt += FZ_THREADS / 32) {
+        const int row = mt * 8 + (lane >> 2);
+        const uint16_t* arow = As + (size_t)min(row, r - 1) * FZ_SL + (lane & 3);
+        const double* brow = s_xt + (size_t)(lane >> 2) * XTS + (lane & 3);
+        double c[3][2] = {{0.0, 0.0}, {0.0, 0.0}, {0.0, 0.0}};
 #pragma unroll
-        for (int e = 0; e < JG; ++e) {
-          const int j = j0 + e;
-          if (j <= K) {
-            double a = p0[e], b = p1[e], sv = sq[e];
+        for (int ks = 0; ks < FZ_SL / 4; ++ks) {
+          const double av = row < r ? w16_to_double<WD>(arow[ks * 4]) : 0.0;
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-              a += __shfl_xor_sync(0xffffffffu, a, o);
-              b += __shfl_xor_sync(0xffffffffu, b, o);
-              sv += __shfl_xor_sync(0xffffffffu, sv, o);
-            }
-            if (lane == 0) {
-              s_redd[(j * 3 + 0) * 16 + warp] = a;
-              s_redd[(j * 3 + 1) * 16 + warp] = b;
-              s_redd[(j * 3 + 2) * 16 + warp] = sv;
+          for (int nt = 0; nt < 3; ++nt) {
+            if (nt < NT) {
+              const double bv = brow[(size_t)nt * 8 * XTS + ks * 4];
+              asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+                           : "+d"(c[nt][0]), "+d"(c[nt][1]) : "d"(av), "d"(bv));
             }
           }
         }
-      }
-      if (tid == 0) FZ_STAMP(1, 30);
-      named_bar_sync(1, FZ_THREADS);
-      if (A.has_next) {
-        for (int t = tid; t < (K + 1) * 3; t += FZ_THREADS) {
-          const int j = t / 3, e = t - j * 3;
-          double v = 0.0;
+        if (row < r) {
 #pragma unroll
-          for (int w = 0; w < 16; ++w) v += s_redd[t * 16 + w];
-          if (e < 2) {
-            const int row = cta + (a0 + e) * G;
-            if (a0 + e < lay.nA && row < r) A.z[(size_t)j * r + row] = v;
-          } else if (j == sq_eval) {
-            A.sumsq[j] = v;
+          for (int nt = 0; nt < 3; ++nt) {
+            const int j = nt * 8 + (lane & 3) * 2;
+            if (nt < NT && j <= K) part[(size_t)j * RS + row] = c[nt][0];
+            if (nt < NT && j + 1 <= K) part[(size_t)(j + 1) * RS + row] = c[nt][1];
           }
         }
       }
-      named_bar_sync(1, FZ_THREADS);
+      if (tid == 0) FZ_STAMP(1, 12);
+      if (warp == FZ_THREADS / 32 - 1) {  // partial sums of squares of the slice, one evaluation per lane
+        for (int j = lane; j <= K; j += 32) {
+          double sq = 0.0;
+#pragma unroll 8
+          for (int c = 0; c < FZ_SL; ++c) { const double v = s_xt[j * XTS + c]; sq = fma(v, v, sq); }
+          part[(size_t)j * RS + r] = sq;
+        }
+      }
     }
   }
+  if (tid == 0) FZ_STAMP(1, 30);
 
-  if (!A.has_next && feat_writer) {
-#pragma unroll
-    for (int q = 0; q < XC; ++q) {
-      const int c = tid + q * FZ_THREADS;
-      if (c < d) A.x_out[c] = s_xfin[c];
-    }
-  }
   if (A.has_next) {
-    // ---------------------------------------------------------------------------------------------- barrier 2 of 3
+    // ---------------------------------------------------------------------------------------------- barrier 2 of 5
     if (tid == 0) FZ_STAMP(1, 2);
+    if (tid == 0) FZ_CSTAMP(6);
     grid_barrier(A, G);
     if (tid == 0) FZ_STAMP(1, 3);
-    if (feat_writer) {  // x_out may alias x, which every CTA was still reading before this barrier
+
+    // ============================ phase 2b: sum of the slices' partials, one value per warp ===========================
+    // Lane l adds slices l, l + 32, ... in order, the lanes are combined by a butterfly: the result does not depend on
+    // which warp of which CTA computes it.
+    {
+      const int V = E * RS;
+      for (int v = cta * (FZ_THREADS / 32) + warp; v < V; v += G * (FZ_THREADS / 32)) {
+        double acc = 0.0;
+        const double* zp = A.zpart + v;
+        for (int s0 = 0; s0 < nsl; s0 += 128) {  // four loads in flight per lane
+          double q[4];
 #pragma unroll
-      for (int q = 0; q < XC; ++q) {
-        const int c = tid + q * FZ_THREADS;
-        if (c < d) A.x_out[c] = s_xfin[c];
+          for (int u = 0; u < 4; ++u) {
+            const int s2 = s0 + u * 32 + lane;
+            q[u] = s2 < nsl ? __ldcg(zp + (size_t)s2 * V) : 0.0;
+          }
+          acc += (q[0] + q[1]) + (q[2] + q[3]);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        if (lane == 0) {
+          const int j = v / RS, row = v - j * RS;
+          if (row < r) A.z[(size_t)j * r + row] = acc;
+          else A.sumsq[j] = acc;
+        }
       }
     }
+    // ---------------------------------------------------------------------------------------------- barrier 3 of 5
+    if (tid == 0) FZ_STAMP(1, 7);
+    grid_barrier(A, G);
+    if (tid == 0) FZ_STAMP(1, 8);
 
     // ============================ phase 3: scores of this CTA's neurons, every evaluation =============================
-    double* s_zs = reinterpret_cast<double*>(smem + lay.zs_off);            // [8][r + FZ_ZPAD], normalised
+    double* s_zs = reinterpret_cast<double*>(smem + lay.zs_off);            // [NT * 8][r + FZ_ZPAD], un-normalised
+    double* s_part = reinterpret_cast<double*>(smem + lay.part_off);        // [FZ_KS][FZ_EPAD][per8]
     double* s_own = reinterpret_cast<double*>(smem + lay.own_off);          // [K+1][per]
     uint16_t* s_bin = reinterpret_cast<uint16_t*>(smem + lay.bin_off);      // [K+1][per]
     unsigned* s_coarse = reinterpret_cast<unsigned*>(smem + lay.coarse_off);  // [K+1][FZ_NC + 1] exclusive prefix
@@ -643,48 +725,76 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
     const double brange = bin_hi - bin_lo;
     const double bscale = (brange > 0.0 && brange < INF) ? (double)FZ_NB / brange : 0.0;
     const int keff = min(A.k_next, Fn);
-
-    // C[neuron][evaluation] = B^T rows x latents, on the fp64 tensor cores (mma m8n8k4): a warp owns tiles of eight
-    // neurons, the evaluations are taken eight at a time.  Every output element is accumulated over the columns in the
-    // same order whatever its position in the tile, so equal predictor rows give bit-equal scores.
-    mbar_wait(&s_bar[2 * FZ_MAX_DEPTH + 1], 0u, A.status);  // the rows of B^T have landed
     const int RSB = r + FZ_BPAD, RSZ = r + FZ_ZPAD;
+    const int per8 = (per + 7) & ~7;
+
+    // latents of every evaluation (rows past K are zero) and 1 / rms of every feature
+    {
+      const double* zg = A.z;
+      const int nz = NT * 8 * r;
+      for (int t0 = 0; t0 < nz; t0 += 4 * FZ_THREADS) {  // four loads in flight per thread
+        double q[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int t = t0 + u * FZ_THREADS + tid;
+          q[u] = (t < E * r) ? __ldcg(zg + t) : 0.0;  // z is [evaluation][r], contiguous
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int t = t0 + u * FZ_THREADS + tid;
+          if (t < nz) { const int e = t / r; s_zs[e * RSZ + (t - e * r)] = q[u]; }
+        }
+      }
+    }
+    if (tid < FZ_EPAD)
+      s_inv[tid] = (tid <= K && A.norm_n == 0) ? 1.0 / sqrt(__ldcg(&A.sumsq[tid]) / (double)d + (double)A.eps_n) : 1.0;
+    if (!mbar_wait(&s_bar[FZ_BAR_B], s_phase[FZ_BAR_B] & 1u, A.status)) FZ_FAIL(5, 0);  // the rows of B^T have landed
+    named_bar_sync(1, FZ_THREADS);
+    if (tid == 0) FZ_STAMP(1, 40);
+
+    // C[neuron][evaluation] = B^T rows x latents, on the fp64 tensor cores (mma m8n8k4).  A task is a tile of eight
+    // neurons times one of FZ_KS column ranges, for all evaluations at once; the column ranges are added afterwards in
+    // a fixed order.  Every output element is accumulated over the columns in the same order whatever its position in
+    // the tile, so equal predictor rows give bit-equal scores.
     const int n_mt = (n_own + 7) >> 3;
-    for (int n0 = 0; n0 <= K; n0 += 8) {
-      named_bar_sync(1, FZ_THREADS);  // the previous eight latents are no longer read
-      if (tid < 8) {  // 1 / rms of the eight features, once each
-        const int j = n0 + tid;
-        s_inv[tid] = (j <= K && A.norm_n == 0) ? 1.0 / sqrt(__ldcg(&A.sumsq[j]) / (double)d + (double)A.eps_n) : 1.0;
-      }
-      for (int t = tid; t < 8 * r; t += FZ_THREADS) {  // fetched before the scale factors are ready
-        const int e = t / r, jj = t - e * r, j = n0 + e;
-        s_zs[e * RSZ + jj] = j <= K ? __ldcg(&A.z[(size_t)j * r + jj]) : 0.0;
-      }
-      named_bar_sync(1, FZ_THREADS);
-      for (int t = tid; t < 8 * r; t += FZ_THREADS) {
-        const int e = t / r, jj = t - e * r;
-        s_zs[e * RSZ + jj] *= s_inv[e];
-      }
-      named_bar_sync(1, FZ_THREADS);
-      if (tid == 0) FZ_STAMP(1, 40 + n0 / 8 * 2);
-      for (int mt = warp; mt < n_mt; mt += FZ_THREADS / 32) {
-        const uint16_t* arow = s_B + (size_t)(mt * 8 + (lane >> 2)) * RSB + (lane & 3);
-        const double* brow = s_zs + (size_t)(lane >> 2) * RSZ + (lane & 3);
-        double c0 = 0.0, c1 = 0.0, e0 = 0.0, e1 = 0.0;  // two interleaved accumulator pairs (even / odd column steps)
-        for (int k0 = 0; k0 < r; k0 += 8) {
-          const double a0v = w16_to_double<WD>(arow[k0]), b0v = brow[k0];
-          const double a1v = w16_to_double<WD>(arow[k0 + 4]), b1v = brow[k0 + 4];
-          asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};" : "+d"(c0), "+d"(c1) : "d"(a0v), "d"(b0v));
-          asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};" : "+d"(e0), "+d"(e1) : "d"(a1v), "d"(b1v));
-        }
-        if (tid == 0) FZ_STAMP(1, 41 + n0 / 8 * 2);
-        const int li = mt * 8 + (lane >> 2);
-        const int j = n0 + (lane & 3) * 2;
-        if (li < n_own) {
-          if (j <= K) s_own[(size_t)j * per + li] = canonical_score((c0 + e0) + (double)s_pc[li]);
-          if (j + 1 <= K) s_own[(size_t)(j + 1) * per + li] = canonical_score((c1 + e1) + (double)s_pc[li]);
+    const int kchunk = ((r >> 3) + FZ_KS - 1) / FZ_KS * 8;
+    for (int task = warp; task < n_mt * FZ_KS; task += FZ_THREADS / 32) {
+      const int ks = task / n_mt, mt = task - ks * n_mt;
+      const int k_lo = ks * kchunk, k_hi = min(r, k_lo + kchunk);
+      const uint16_t* arow = s_B + (size_t)(mt * 8 + (lane >> 2)) * RSB + (lane & 3);
+      const double* brow = s_zs + (size_t)(lane >> 2) * RSZ + (lane & 3);
+      double c[3][2] = {{0.0, 0.0}, {0.0, 0.0}, {0.0, 0.0}}, e[3][2] = {{0.0, 0.0}, {0.0, 0.0}, {0.0, 0.0}};
+      for (int k0 = k_lo; k0 < k_hi; k0 += 8) {
+        const double a0v = w16_to_double<WD>(arow[k0]), a1v = w16_to_double<WD>(arow[k0 + 4]);
+#pragma unroll
+        for (int nt = 0; nt < 3; ++nt) {
+          if (nt < NT) {
+            const double b0v = brow[(size_t)nt * 8 * RSZ + k0], b1v = brow[(size_t)nt * 8 * RSZ + k0 + 4];
+            asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+                         : "+d"(c[nt][0]), "+d"(c[nt][1]) : "d"(a0v), "d"(b0v));
+            asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+                         : "+d"(e[nt][0]), "+d"(e[nt][1]) : "d"(a1v), "d"(b1v));
+          }
         }
       }
+      const int li = mt * 8 + (lane >> 2);
+#pragma unroll
+      for (int nt = 0; nt < 3; ++nt) {
+        if (nt < NT) {
+          const int j = nt * 8 + (lane & 3) * 2;
+          s_part[((size_t)ks * FZ_EPAD + j) * per8 + li] = c[nt][0] + e[nt][0];
+          s_part[((size_t)ks * FZ_EPAD + j + 1) * per8 + li] = c[nt][1] + e[nt][1];
+        }
+      }
+    }
+    named_bar_sync(1, FZ_THREADS);
+    if (tid == 0) FZ_STAMP(1, 41);
+    for (int t = tid; t < E * n_own; t += FZ_THREADS) {
+      const int j = t / n_own, li = t - j * n_own;
+      double v = 0.0;
+#pragma unroll
+      for (int ks = 0; ks < FZ_KS; ++ks) v += s_part[((size_t)ks * FZ_EPAD + j) * per8 + li];
+      s_own[(size_t)j * per + li] = canonical_score(v * s_inv[j] + (double)s_pc[li]);
     }
     named_bar_sync(1, FZ_THREADS);
     if (tid == 0) FZ_STAMP(1, 50);
@@ -740,8 +850,9 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
       }
     }
 
-    // ---------------------------------------------------------------------------------------------- barrier 3 of 3
+    // ---------------------------------------------------------------------------------------------- barrier 4 of 5
     if (tid == 0) FZ_STAMP(1, 4);
+    if (tid == 0) FZ_CSTAMP(7);
     grid_barrier(A, G);
     if (tid == 0) FZ_STAMP(1, 5);
 
@@ -981,7 +1092,19 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
       if (keff > A.next_cap) set_status(A.status, ST_CAPACITY);
     }
     if (tid == 0) FZ_STAMP(1, 6);
+    if (tid == 0) FZ_CSTAMP(11);
   }
+  // phases completed in this layer (every wait above has returned)
+  named_bar_sync(1, FZ_THREADS);
+  if (tid < FZ_NBAR) {
+    unsigned n = 0;
+    if (tid < FZ_MAX_DEPTH) n = used_gu > tid ? (unsigned)((used_gu - 1 - tid) / GU + 1) : 0u;
+    else if (tid < FZ_BAR_A) { const int sdn = tid - FZ_BAR_DN; n = used_dn > sdn ? (unsigned)((used_dn - 1 - sdn) / DN + 1) : 0u; }
+    else n = A.has_next ? 1u : 0u;
+    s_phase[tid] += n;
+  }
+  // what this layer wrote to shared memory with ordinary stores is ordered before the next layer's bulk copies into it
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 
 }
 
@@ -1026,7 +1149,7 @@ template <int WD, int CPT>
 __global__ void __launch_bounds__(FZ_BLOCK, 1) ls_fused_step_kernel(const __grid_constant__ FusedArgs A) {
   extern __shared__ __align__(128) unsigned char smem[];
   __shared__ FusedShared sh;
-  fused_layer<WD, CPT>(A, smem, sh, false);
+  fused_layer<WD, CPT>(A, smem, sh, true);
   if (threadIdx.x >= FZ_THREADS) return;  // the producer warp is done; an exited warp counts as arrived at block barriers
   named_bar_sync(1, FZ_THREADS);
   if (threadIdx.x == 0) {
@@ -1065,8 +1188,10 @@ __global__ void __launch_bounds__(FZ_BLOCK, 1)
   const int G = gridDim.x, cta = blockIdx.x, tid = threadIdx.x;
   constexpr int NW = sizeof(FusedArgs) / 4;
   for (int n = 0; n < n_layers; ++n) {
+    if (tid == 0) FZ_STAMP(1, 24);
     for (int w = tid; w < NW; w += FZ_BLOCK) reinterpret_cast<uint32_t*>(&sh.args)[w] = reinterpret_cast<const uint32_t*>(&g_args[n])[w];
     __syncthreads();
+    if (tid == 0) FZ_STAMP(1, 25);
     if (tid == 0) {
       FusedArgs& a = sh.args;
       a.K = C.K;
@@ -1079,18 +1204,26 @@ __global__ void __launch_bounds__(FZ_BLOCK, 1)
     }
     __syncthreads();
     const FusedArgs& A = sh.args;
-    fused_layer<WD, CPT>(A, smem, sh, n > 0);
-    if (tid < FZ_THREADS) {
-      if (cta == G - 1 && C.tr_x) {  // what entered this layer
-        for (int c = tid; c < A.d; c += FZ_THREADS) C.tr_x[(size_t)n * A.d + c] = __ldcg(A.x + c);
-        if (C.tr_sel) {
-          const int cnt = max(0, min(__ldcg(A.sel_count), min(A.sel_cap, C.tr_cap)));
-          for (int t = tid; t < cnt; t += FZ_THREADS) C.tr_sel[(size_t)n * C.tr_cap + t] = __ldcg(A.sel_idx + t);
-          if (tid == 0) C.tr_cnt[n] = cnt;
-        }
+    if (cta == G - 1 && C.tr_x && tid < FZ_THREADS) {  // what enters this layer (x_out may overwrite x)
+      for (int c = tid; c < A.d; c += FZ_THREADS) C.tr_x[(size_t)n * A.d + c] = __ldcg(A.x + c);
+      if (C.tr_sel) {
+        const int cnt = max(0, min(__ldcg(A.sel_count), min(A.sel_cap, C.tr_cap)));
+        for (int t = tid; t < cnt; t += FZ_THREADS) C.tr_sel[(size_t)n * C.tr_cap + t] = __ldcg(A.sel_idx + t);
+        if (tid == 0) C.tr_cnt[n] = cnt;
       }
+    }
+    fused_layer<WD, CPT>(A, smem, sh, n == 0);
+    if (tid < FZ_THREADS) {
       if (n > 0) fused_clean(sh.prev, cta, G);  // nobody touches the previous layer's scratch any more
       grid_barrier(A, G);                       // layer boundary: x_out and the refined selection are visible to all
+#ifdef LS_FZ_TIMING
+      if (tid == 0 && cta == 0 && n < 100) {
+        unsigned long long gt;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(gt));
+        g_fz_timing[1][200 + n] = clock64();
+        g_fz_timing[1][300 + n] = (long long)gt;
+      }
+#endif
     }
     __syncthreads();
     for (int w = tid; w < NW; w += FZ_BLOCK) reinterpret_cast<uint32_t*>(&sh.prev)[w] = reinterpret_cast<const uint32_t*>(&sh.args)[w];
