@@ -40,7 +40,7 @@ constexpr int FZ_ZPAD = 4;        // padding (doubles) of a latent row in shared
 constexpr int FZ_MAX_DEPTH = 8;   // most gate/up ring stages; the depths are chosen per launch from the shared memory left
 constexpr int FZ_MAX_DN = 16;     // most down ring stages
 constexpr int FZ_SL = 32;         // columns of the feature handled as one slice in the latent phase
-constexpr int FZ_EPAD = 24;       // evaluations rounded up to whole tiles of eight
+constexpr int FZ_EPAD = 18;       // rows kept per evaluation-indexed buffer: at most two MMA tiles, or FZ_MAXE rows
 constexpr int FZ_KS = 4;          // column splits of a score tile (more independent tasks than warps)
 constexpr int FZ_MAX_MINE = 256;  // neurons one CTA may own in one step
 #ifdef LS_FZ_TIMING
@@ -159,7 +159,7 @@ __device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float 
 // never reset.  Arrival is a release, the poll an acquire, so what a CTA wrote before the barrier is visible to all
 // after it.  Every compute thread of the block calls it (block barrier 1 spans the 512 compute threads; the producer
 // warp has left by then).
-__device__ __forceinline__ void grid_barrier(const FusedArgs& A, int G) {
+__device__ __noinline__ void grid_barrier(const FusedArgs& A, int G) {
   named_bar_sync(1, FZ_THREADS);
   if (threadIdx.x == 0) {
     unsigned long long old;
@@ -194,7 +194,7 @@ __host__ __device__ inline int fz_stage_of_cta(int cta, int G, int K) {
 
 struct FusedSmemLayout {
   // fixed regions
-  size_t bar_off, red_off, redd_off, mine_off, pc_off, xt_off, qa_off, a_off;
+  size_t bar_off, red_off, redd_off, mine_off, pc_off, xt_off, dv_off, qa_off, a_off;
   // the stream's rings ...
   size_t gu_off, dn_off;
   // ... and, in the same bytes once the rings have drained, the operands and results of the refinement
@@ -225,6 +225,7 @@ __host__ __device__ inline FusedSmemLayout fused_layout(int d, int n_in, int r, 
   L.mine_off = take((size_t)FZ_MAX_MINE * 8);        // this CTA's neuron indices and gate biases
   L.pc_off = take((size_t)L.per * 4);
   L.xt_off = take((size_t)FZ_EPAD * (FZ_SL + 4) * 8);  // x~^(j) of one slice, fp64, padded rows
+  L.dv_off = take((size_t)FZ_MAXK * FZ_SL * 4);      // stage accumulators of one slice
   L.qa_off = take(FZ_MAX_DN * 4);                    // activations of the queued down rows
   if (!a_alias) L.a_off = take(a_bytes);
   const size_t base = o;
@@ -261,6 +262,106 @@ struct FusedShared {
   unsigned long long kmm[2 * 16];
   unsigned ccnt[FZ_MAXE * FZ_NC];
 };
+
+// ---- rare paths of the ranking phase, kept out of line so that the common path stays small in the instruction cache ----
+// Rank of the entry (key kp, neuron i) of evaluation j whose fine bin bb overflowed its bucket: the first rank of the bin
+// (coarse prefix + the fine counts before it) plus the entries of the bucket and of the overflow list that precede it.
+__device__ __noinline__ int fz_rank_in_overflowed_bin(const FusedArgs& A, int j, int bb, int i, unsigned long long kp,
+                                                      unsigned coarse_b0) {
+  constexpr int FPC = FZ_NB / FZ_NC;
+  const unsigned* cnt = A.cnt + (size_t)j * FZ_CNT_STRIDE;
+  unsigned b0 = coarse_b0;
+  for (int fb = (bb / FPC) * FPC; fb < bb; ++fb) b0 += __ldcg(&cnt[fb]);
+  int before = 0;
+  const uint4* bk = A.bent + ((size_t)j * FZ_NB + bb) * FZ_CAPB;
+  for (int q = 0; q < FZ_CAPB; ++q) {  // the bucket is full
+    const uint4 e = __ldcg(bk + q);
+    const unsigned long long kq = ((unsigned long long)e.y << 32) | e.x;
+    before += (kq > kp) || (kq == kp && (int)e.z < i);
+  }
+  const unsigned novf = __ldcg(&cnt[FZ_NB + FZ_NC]);
+  for (unsigned q = 0; q < novf; ++q) {
+    const uint4 e = __ldcg(&A.oent[(size_t)j * A.Fn + q]);
+    if ((int)e.w != bb) continue;
+    const unsigned long long kq = ((unsigned long long)e.y << 32) | e.x;
+    before += (kq > kp) || (kq == kp && (int)e.z < i);
+  }
+  return (int)b0 + before;
+}
+
+// Final evaluation, fine bin `bin` with an overflowed bucket, called by the sixteen lanes that hold its bucket entries
+// (entry `ent` in lane l16; the bucket is full).  Returns how many overflow entries precede this lane's entry; lane 0
+// also ranks the overflow entries of the bin themselves and emits those inside the first keff ranks.
+__device__ __noinline__ int fz_final_overflowed_bin(const FusedArgs& A, int j, int bin, unsigned b0, uint4 ent, int l16, int keff,
+                                                    unsigned* s_nsel_j) {
+  const unsigned* cnt = A.cnt + (size_t)j * FZ_CNT_STRIDE;
+  const unsigned novf = __ldcg(&cnt[FZ_NB + FZ_NC]);
+  const unsigned long long kmine = ((unsigned long long)ent.y << 32) | ent.x;
+  int before = 0;
+  for (unsigned q = 0; q < novf; ++q) {
+    const uint4 e = __ldcg(&A.oent[(size_t)j * A.Fn + q]);
+    if ((int)e.w != bin) continue;
+    const unsigned long long kq = ((unsigned long long)e.y << 32) | e.x;
+    before += (kq > kmine) || (kq == kmine && (int)e.z < (int)ent.z);
+  }
+  if (l16 == 0) {
+    for (unsigned q = 0; q < novf; ++q) {
+      const uint4 e = __ldcg(&A.oent[(size_t)j * A.Fn + q]);
+      if ((int)e.w != bin) continue;
+      const unsigned long long ke = ((unsigned long long)e.y << 32) | e.x;
+      int bf = 0;
+      for (int u = 0; u < FZ_CAPB; ++u) {
+        const uint4 o = __ldcg(&A.bent[((size_t)j * FZ_NB + bin) * FZ_CAPB + u]);
+        const unsigned long long ko = ((unsigned long long)o.y << 32) | o.x;
+        bf += (ko > ke) || (ko == ke && (int)o.z < (int)e.z);
+      }
+      for (unsigned u = 0; u < novf; ++u) {
+        const uint4 o = __ldcg(&A.oent[(size_t)j * A.Fn + u]);
+        if ((int)o.w != bin) continue;
+        const unsigned long long ko = ((unsigned long long)o.y << 32) | o.x;
+        bf += (ko > ke) || (ko == ke && (int)o.z < (int)e.z);
+      }
+      const int rk = (int)b0 + bf;
+      if (rk < keff) {
+        const int i = (int)e.z;
+        if (rk < A.next_cap) A.next_idx[rk] = i;
+        if (A.next_mask) atomicOr(&A.next_mask[i >> 5], 1u << (i & 31));
+        if (A.tr_masks) atomicOr(&A.tr_masks[(size_t)j * ((A.Fn + 31) >> 5) + (i >> 5)], 1u << (i & 31));
+        atomicAdd(s_nsel_j, 1u);
+      }
+    }
+  }
+  return before;
+}
+
+// One score task on the fp64 tensor cores: eight predictor rows (16-bit, row stride RSB elements, `arow` already points at
+// this lane's row and column) times NT tiles of eight latents (row stride RSZ doubles, `brow` likewise) over the columns
+// [k_lo, k_hi); partial sums to out[evaluation * ostride] at this lane's neuron.
+template <int WD, int NT>
+__device__ __forceinline__ void score_task_mma(const uint16_t* arow, const double* brow, int RSZ, int k_lo, int k_hi, double* out,
+                                               int ostride, int lane) {
+  double c[NT][2], e[NT][2];
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) { c[nt][0] = c[nt][1] = e[nt][0] = e[nt][1] = 0.0; }
+#pragma unroll 4
+  for (int k0 = k_lo; k0 < k_hi; k0 += 8) {
+    const double a0v = w16_to_double<WD>(arow[k0]), a1v = w16_to_double<WD>(arow[k0 + 4]);
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+      const double b0v = brow[(size_t)nt * 8 * RSZ + k0], b1v = brow[(size_t)nt * 8 * RSZ + k0 + 4];
+      asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+                   : "+d"(c[nt][0]), "+d"(c[nt][1]) : "d"(a0v), "d"(b0v));
+      asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+                   : "+d"(e[nt][0]), "+d"(e[nt][1]) : "d"(a1v), "d"(b1v));
+    }
+  }
+#pragma unroll
+  for (int nt = 0; nt < NT; ++nt) {
+    const int j = nt * 8 + (lane & 3) * 2;
+    out[(size_t)j * ostride] = c[nt][0] + e[nt][0];
+    out[(size_t)(j + 1) * ostride] = c[nt][1] + e[nt][1];
+  }
+}
 
 // One layer step, executed by the whole block (16 compute warps + the producer warp).  The producer warp returns as
 // soon as it has issued its last copy; the compute warps return when the layer's refined sets are written.
@@ -599,7 +700,12 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
   // x~^(j), j = 0..K, of its columns (x + the stage accumulators below j, Eq. 2), writes x_out = x~^(K), and multiplies
   // the slice of A (r x 32, in shared memory) with the 32 x (K+1) block of features on the fp64 tensor cores.  The
   // partial latents (and the partial sums of squares, as row r) go to global memory, one block per slice.
-  const int E = K + 1, NT = (E + 7) >> 3, RS = r + 1;
+  // Evaluations are taken eight at a time on the fp64 tensor cores; a remainder of one or two evaluations is cheaper on
+  // the ordinary fp64 pipe (a padded tile would spend eight evaluations' worth of the same units).
+  const int E = K + 1, RS = r + 1;
+  int NTM = E >> 3, REM = E & 7;
+  if (REM > 2) { ++NTM; REM = 0; }
+  const int EM = NTM * 8;  // evaluations [0, EM) by MMA (rows past K are zero), [EM, E) by scalar code
   constexpr int XTS = FZ_SL + 4;  // row stride (doubles) of s_xt: the four rows a half-warp reads sit on distinct banks
   if (A.has_next && cta < nsl)
     if (!mbar_wait(&s_bar[FZ_BAR_A], s_phase[FZ_BAR_A] & 1u, A.status)) FZ_FAIL(4, 0);  // the A slices have landed
@@ -607,28 +713,30 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
   for (int a = 0; cta + a * G < nsl; ++a) {
     const int sl = cta + a * G;
     if (a > 0) named_bar_sync(1, FZ_THREADS);  // the previous slice's features are no longer read
+    float* s_dv = reinterpret_cast<float*>(smem + lay.dv_off);  // [K][32]
+    float xv = 0.f;
+    if (tid < K * FZ_SL) {  // one stage accumulator per thread, all loads in flight together
+      const int c = sl * FZ_SL + (tid & (FZ_SL - 1));
+      s_dv[tid] = c < d ? __ldcg(A.dacc + (size_t)(tid / FZ_SL) * d + c) : 0.f;
+    }
+    if (tid < FZ_SL) {
+      const int c = sl * FZ_SL + tid;
+      if (c < d) xv = __ldcg(A.x + c) + (A.b_down ? A.b_down[c] : 0.f);
+    }
+    named_bar_sync(1, FZ_THREADS);
     if (tid < FZ_SL) {
       const int c = sl * FZ_SL + tid;
       float* const trx = A.tr_xtilde;  // (the arguments live in shared memory: read them once, not after every store)
       float* const xo = A.x_out;
-      float dv[FZ_MAXK];
-      float xv = 0.f;
-#pragma unroll
-      for (int j = 0; j < FZ_MAXK; ++j) dv[j] = (c < d && j < K) ? __ldcg(A.dacc + (size_t)j * d + c) : 0.f;
-      if (c < d) xv = __ldcg(A.x + c) + (A.b_down ? A.b_down[c] : 0.f);
-#ifdef LS_FZ_TIMING
-      if (tid == 0) { FZ_STAMP_DEP(1, 13, xv); float q_ = 0.f; for (int j = 0; j < FZ_MAXK; ++j) q_ += dv[j]; FZ_STAMP_DEP(1, 14, q_); }
-#endif
-#pragma unroll
-      for (int j = 0; j < FZ_EPAD; ++j) {
-        if (j < NT * 8) {
-          s_xt[j * XTS + tid] = j <= K ? (double)xv : 0.0;
-          if (j <= K && c < d) {
-            if (trx) trx[(size_t)j * d + c] = xv;
-            if (j == K) xo[c] = xv;  // may alias x: this thread is the only one that still needs x[c]
-          }
-          if (j < FZ_MAXK) xv += dv[j];
+      const int rows = max(EM, E);
+#pragma unroll 1
+      for (int j = 0; j < rows; ++j) {
+        s_xt[j * XTS + tid] = j <= K ? (double)xv : 0.0;
+        if (j <= K && c < d) {
+          if (trx) trx[(size_t)j * d + c] = xv;
+          if (j == K) xo[c] = xv;  // may alias x: this thread is the only one that still needs x[c]
         }
+        if (j < K) xv += s_dv[j * FZ_SL + tid];
       }
     }
     named_bar_sync(1, FZ_THREADS);
@@ -641,13 +749,13 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
         const int row = mt * 8 + (lane >> 2);
         const uint16_t* arow = As + (size_t)min(row, r - 1) * FZ_SL + (lane & 3);
         const double* brow = s_xt + (size_t)(lane >> 2) * XTS + (lane & 3);
-        double c[3][2] = {{0.0, 0.0}, {0.0, 0.0}, {0.0, 0.0}};
+        double c[2][2] = {{0.0, 0.0}, {0.0, 0.0}};
 #pragma unroll
         for (int ks = 0; ks < FZ_SL / 4; ++ks) {
           const double av = row < r ? w16_to_double<WD>(arow[ks * 4]) : 0.0;
 #pragma unroll
-          for (int nt = 0; nt < 3; ++nt) {
-            if (nt < NT) {
+          for (int nt = 0; nt < 2; ++nt) {
+            if (nt < NTM) {
               const double bv = brow[(size_t)nt * 8 * XTS + ks * 4];
               asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
                            : "+d"(c[nt][0]), "+d"(c[nt][1]) : "d"(av), "d"(bv));
@@ -656,12 +764,30 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
         }
         if (row < r) {
 #pragma unroll
-          for (int nt = 0; nt < 3; ++nt) {
+          for (int nt = 0; nt < 2; ++nt) {
             const int j = nt * 8 + (lane & 3) * 2;
-            if (nt < NT && j <= K) part[(size_t)j * RS + row] = c[nt][0];
-            if (nt < NT && j + 1 <= K) part[(size_t)(j + 1) * RS + row] = c[nt][1];
+            if (nt < NTM && j <= K) part[(size_t)j * RS + row] = c[nt][0];
+            if (nt < NTM && j + 1 <= K) part[(size_t)(j + 1) * RS + row] = c[nt][1];
           }
         }
+      }
+      for (int t = tid; t < REM * r; t += FZ_THREADS) {  // remainder evaluations: one thread per (evaluation, row of A)
+        const int jr = t / r, row = t - jr * r, j = EM + jr;
+        const uint16_t* arow = As + (size_t)row * FZ_SL;
+        const double* xr2 = s_xt + (size_t)j * XTS;
+        double acc = 0.0;
+#pragma unroll
+        for (int c0 = 0; c0 < FZ_SL; c0 += 8) {
+          const uint4 w = *reinterpret_cast<const uint4*>(arow + c0);
+          const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const double2 xx = *reinterpret_cast<const double2*>(xr2 + c0 + 2 * q);
+            acc = fma(w16_to_double<WD>((uint16_t)(ww[q] & 0xffffu)), xx.x, acc);
+            acc = fma(w16_to_double<WD>((uint16_t)(ww[q] >> 16)), xx.y, acc);
+          }
+        }
+        part[(size_t)j * RS + row] = acc;
       }
       if (tid == 0) FZ_STAMP(1, 12);
       if (warp == FZ_THREADS / 32 - 1) {  // partial sums of squares of the slice, one evaluation per lane
@@ -715,7 +841,7 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
     if (tid == 0) FZ_STAMP(1, 8);
 
     // ============================ phase 3: scores of this CTA's neurons, every evaluation =============================
-    double* s_zs = reinterpret_cast<double*>(smem + lay.zs_off);            // [NT * 8][r + FZ_ZPAD], un-normalised
+    double* s_zs = reinterpret_cast<double*>(smem + lay.zs_off);            // [max(EM, E)][r + FZ_ZPAD], un-normalised
     double* s_part = reinterpret_cast<double*>(smem + lay.part_off);        // [FZ_KS][FZ_EPAD][per8]
     double* s_own = reinterpret_cast<double*>(smem + lay.own_off);          // [K+1][per]
     uint16_t* s_bin = reinterpret_cast<uint16_t*>(smem + lay.bin_off);      // [K+1][per]
@@ -728,10 +854,10 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
     const int RSB = r + FZ_BPAD, RSZ = r + FZ_ZPAD;
     const int per8 = (per + 7) & ~7;
 
-    // latents of every evaluation (rows past K are zero) and 1 / rms of every feature
+    // latents of every evaluation and 1 / rms of every feature
     {
       const double* zg = A.z;
-      const int nz = NT * 8 * r;
+      const int nz = max(EM, E) * r;
       for (int t0 = 0; t0 < nz; t0 += 4 * FZ_THREADS) {  // four loads in flight per thread
         double q[4];
 #pragma unroll
@@ -752,82 +878,107 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
     named_bar_sync(1, FZ_THREADS);
     if (tid == 0) FZ_STAMP(1, 40);
 
-    // C[neuron][evaluation] = B^T rows x latents, on the fp64 tensor cores (mma m8n8k4).  A task is a tile of eight
-    // neurons times one of FZ_KS column ranges, for all evaluations at once; the column ranges are added afterwards in
-    // a fixed order.  Every output element is accumulated over the columns in the same order whatever its position in
-    // the tile, so equal predictor rows give bit-equal scores.
+    // C[neuron][evaluation] = B^T rows x latents.  A task is a group of neurons times one of FZ_KS column ranges; the
+    // column ranges are added afterwards in a fixed order.  Within one evaluation every neuron's score is accumulated
+    // over the columns in the same order whatever its position in a tile, so equal predictor rows give bit-equal scores.
     const int n_mt = (n_own + 7) >> 3;
     const int kchunk = ((r >> 3) + FZ_KS - 1) / FZ_KS * 8;
-    for (int task = warp; task < n_mt * FZ_KS; task += FZ_THREADS / 32) {
-      const int ks = task / n_mt, mt = task - ks * n_mt;
-      const int k_lo = ks * kchunk, k_hi = min(r, k_lo + kchunk);
-      const uint16_t* arow = s_B + (size_t)(mt * 8 + (lane >> 2)) * RSB + (lane & 3);
-      const double* brow = s_zs + (size_t)(lane >> 2) * RSZ + (lane & 3);
-      double c[3][2] = {{0.0, 0.0}, {0.0, 0.0}, {0.0, 0.0}}, e[3][2] = {{0.0, 0.0}, {0.0, 0.0}, {0.0, 0.0}};
-      for (int k0 = k_lo; k0 < k_hi; k0 += 8) {
-        const double a0v = w16_to_double<WD>(arow[k0]), a1v = w16_to_double<WD>(arow[k0 + 4]);
+    const int n_mma = NTM > 0 ? n_mt * FZ_KS : 0;
+    const int n_blk = (n_own + 31) >> 5;
+    const int n_task = n_mma + n_blk * REM * FZ_KS;
+    if (lane == 0) FZ_STAMP(1, 400 + warp * 4);
+    for (int task = warp; task < n_task; task += FZ_THREADS / 32) {
+      if (lane == 0 && task == warp + 16) FZ_STAMP(1, 401 + warp * 4);
+      if (task < n_mma) {  // eight neurons x the MMA evaluations
+        const int ks = task / n_mt, mt = task - ks * n_mt;
+        const int k_lo = ks * kchunk, k_hi = min(r, k_lo + kchunk);
+        const uint16_t* arow = s_B + (size_t)(mt * 8 + (lane >> 2)) * RSB + (lane & 3);
+        const double* brow = s_zs + (size_t)(lane >> 2) * RSZ + (lane & 3);
+        double* outp = s_part + (size_t)ks * FZ_EPAD * per8 + mt * 8 + (lane >> 2);
+        if (NTM == 1) score_task_mma<WD, 1>(arow, brow, RSZ, k_lo, k_hi, outp, per8, lane);  // (K + 1 <= 17: at most two tiles)
+        else score_task_mma<WD, 2>(arow, brow, RSZ, k_lo, k_hi, outp, per8, lane);
+      } else {  // thirty-two neurons (one per lane) x one remainder evaluation
+        const int t2 = task - n_mma;
+        const int ks = t2 % FZ_KS, bj = t2 / FZ_KS, blk = bj % n_blk, j = EM + bj / n_blk;
+        const int k_lo = ks * kchunk, k_hi = min(r, k_lo + kchunk);
+        const int li = min(blk * 32 + lane, per8 - 1);  // lanes past the last neuron repeat a valid row; not stored
+        const uint16_t* brw = s_B + (size_t)li * RSB;
+        const double* zr = s_zs + (size_t)j * RSZ;
+        double acc = 0.0;
+#pragma unroll 2
+        for (int k0 = k_lo; k0 < k_hi; k0 += 8) {
+          const uint4 w = *reinterpret_cast<const uint4*>(brw + k0);
+          const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
-        for (int nt = 0; nt < 3; ++nt) {
-          if (nt < NT) {
-            const double b0v = brow[(size_t)nt * 8 * RSZ + k0], b1v = brow[(size_t)nt * 8 * RSZ + k0 + 4];
-            asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
-                         : "+d"(c[nt][0]), "+d"(c[nt][1]) : "d"(a0v), "d"(b0v));
-            asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
-                         : "+d"(e[nt][0]), "+d"(e[nt][1]) : "d"(a1v), "d"(b1v));
+          for (int q = 0; q < 4; ++q) {
+            const double2 zz = *reinterpret_cast<const double2*>(zr + k0 + 2 * q);
+            acc = fma(w16_to_double<WD>((uint16_t)(ww[q] & 0xffffu)), zz.x, acc);
+            acc = fma(w16_to_double<WD>((uint16_t)(ww[q] >> 16)), zz.y, acc);
           }
         }
-      }
-      const int li = mt * 8 + (lane >> 2);
-#pragma unroll
-      for (int nt = 0; nt < 3; ++nt) {
-        if (nt < NT) {
-          const int j = nt * 8 + (lane & 3) * 2;
-          s_part[((size_t)ks * FZ_EPAD + j) * per8 + li] = c[nt][0] + e[nt][0];
-          s_part[((size_t)ks * FZ_EPAD + j + 1) * per8 + li] = c[nt][1] + e[nt][1];
-        }
+        if (blk * 32 + lane < n_own) s_part[((size_t)ks * FZ_EPAD + j) * per8 + blk * 32 + lane] = acc;
       }
     }
+    if (lane == 0) FZ_STAMP(1, 402 + warp * 4);
     named_bar_sync(1, FZ_THREADS);
     if (tid == 0) FZ_STAMP(1, 41);
-    for (int t = tid; t < E * n_own; t += FZ_THREADS) {
-      const int j = t / n_own, li = t - j * n_own;
-      double v = 0.0;
-#pragma unroll
-      for (int ks = 0; ks < FZ_KS; ++ks) v += s_part[((size_t)ks * FZ_EPAD + j) * per8 + li];
-      s_own[(size_t)j * per + li] = canonical_score(v * s_inv[j] + (double)s_pc[li]);
-    }
-    named_bar_sync(1, FZ_THREADS);
-    if (tid == 0) FZ_STAMP(1, 50);
-    // histogram (fine + coarse) and bucket insert: one thread per (evaluation, neuron), all atomics in flight together;
-    // the coarse counts of the CTA are summed in shared memory first (they are hot addresses for the whole grid)
+    // final scores, histogram (fine + coarse) and bucket insert: one thread per (evaluation, neuron), two entries at a
+    // time so that their atomics are in flight together; the coarse counts of the CTA are summed in shared memory first
+    // (they are hot addresses for the whole grid)
     {
       for (int t = tid; t < (K + 1) * FZ_NC; t += FZ_THREADS) s_ccnt[t] = 0u;
       if (tid < FZ_MAXE) s_nsel[tid] = 0u;
       named_bar_sync(1, FZ_THREADS);
       unsigned long long kmin = 0xffffffffffffffffULL, kmax = 0ULL;
-      for (int t = tid; t < (K + 1) * n_own; t += FZ_THREADS) {
-        const int j = t / n_own, li = t - j * n_own, i = i_lo + li;
-        const double sv = s_own[(size_t)j * per + li];
-        const double sc = fmin(fmax(sv, -1.7976931348623157e308), 1.7976931348623157e308);
-        int bb = (int)((bin_hi - sc) * bscale);
-        bb = max(0, min(FZ_NB - 1, bb));
-        unsigned* cnt = A.cnt + (size_t)j * FZ_CNT_STRIDE;
-        const unsigned slot = atomicAdd(&cnt[bb], 1u);
-        atomicAdd(&s_ccnt[j * FZ_NC + bb / (FZ_NB / FZ_NC)], 1u);
-        const unsigned long long key = ordered_key(sv);
-        const uint4 ent = make_uint4((unsigned)key, (unsigned)(key >> 32), (unsigned)i, (unsigned)bb);
-        if (slot < (unsigned)FZ_CAPB) {
-          A.bent[((size_t)j * FZ_NB + bb) * FZ_CAPB + slot] = ent;
-        } else {
-          const unsigned o = atomicAdd(&cnt[FZ_NB + FZ_NC], 1u);
-          A.oent[(size_t)j * Fn + o] = ent;
+      const int n_ent = E * n_own;
+      double* const nprio = A.next_prio;
+      double* const nscores = A.next_scores;
+      unsigned* const cnt_all = A.cnt;
+      uint4* const bent = A.bent;
+      uint4* const oent = A.oent;
+      for (int t0 = 0; t0 < n_ent; t0 += 2 * FZ_THREADS) {
+        int jj[2], ll[2], bb[2];
+        unsigned slot[2];
+        unsigned long long key[2];
+        double sv[2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          const int t = t0 + u * FZ_THREADS + tid;
+          jj[u] = -1;
+          if (t < n_ent) {
+            const int j = t / n_own, li = t - j * n_own;
+            double v = 0.0;
+#pragma unroll
+            for (int ks = 0; ks < FZ_KS; ++ks) v += s_part[((size_t)ks * FZ_EPAD + j) * per8 + li];
+            v = canonical_score(v * s_inv[j] + (double)s_pc[li]);
+            const double sc = fmin(fmax(v, -1.7976931348623157e308), 1.7976931348623157e308);
+            int b = (int)((bin_hi - sc) * bscale);
+            b = max(0, min(FZ_NB - 1, b));
+            jj[u] = j; ll[u] = li; bb[u] = b; sv[u] = v; key[u] = ordered_key(v);
+            slot[u] = atomicAdd(&cnt_all[(size_t)j * FZ_CNT_STRIDE + b], 1u);
+          }
         }
-        s_bin[(size_t)j * per + li] = (uint16_t)bb;
-        if (j == K) {
-          if (A.next_prio) A.next_prio[i] = sv;
-          if (A.next_scores) A.next_scores[i] = sv;
-          kmin = min(kmin, key);
-          kmax = max(kmax, key);
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+          if (jj[u] >= 0) {
+            const int j = jj[u], li = ll[u], i = i_lo + li, b = bb[u];
+            s_own[(size_t)j * per + li] = sv[u];
+            s_bin[(size_t)j * per + li] = (uint16_t)b;
+            atomicAdd(&s_ccnt[j * FZ_NC + b / (FZ_NB / FZ_NC)], 1u);
+            const uint4 ent = make_uint4((unsigned)key[u], (unsigned)(key[u] >> 32), (unsigned)i, (unsigned)b);
+            if (slot[u] < (unsigned)FZ_CAPB) {
+              bent[((size_t)j * FZ_NB + b) * FZ_CAPB + slot[u]] = ent;
+            } else {
+              const unsigned o = atomicAdd(&cnt_all[(size_t)j * FZ_CNT_STRIDE + FZ_NB + FZ_NC], 1u);
+              oent[(size_t)j * Fn + o] = ent;
+            }
+            if (j == K) {
+              if (nprio) nprio[i] = sv[u];
+              if (nscores) nscores[i] = sv[u];
+              kmin = min(kmin, key[u]);
+              kmax = max(kmax, key[u]);
+            }
+          }
         }
       }
 #pragma unroll
@@ -880,7 +1031,7 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
       if (c0 > 0 && (int)ex < keff && (int)(ex + c0) >= keff) cbsel = lane * 2;
       if (c1 > 0 && (int)(ex + c0) < keff && (int)incl >= keff) cbsel = lane * 2 + 1;
       const unsigned vote = __ballot_sync(0xffffffffu, cbsel >= 0);
-      int cut_bin = -1, cut_b0 = 0, cut_need = 0, cut_fallback = 0, t_idx = -1;  // no cut bin: keff == 0, nothing is selected
+      int cut_bin = -1, cut_b0 = 0, cut_fallback = 0, t_idx = -1;  // no cut bin: keff == 0, nothing is selected
       unsigned long long t_key = 0ULL;
       if (vote) {
         const int src = __ffs(vote) - 1;
@@ -904,7 +1055,7 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
         cut_bin = cb * FPC + __shfl_sync(0xffffffffu, fsel, fsrc);
         cut_b0 = (int)__shfl_sync(0xffffffffu, fb0, fsrc);
         const int nbc = (int)__shfl_sync(0xffffffffu, fnb, fsrc);
-        cut_need = keff - cut_b0;  // members inside the cut bin, 1 <= need <= nbc
+        const int cut_need = keff - cut_b0;  // members inside the cut bin, 1 <= need <= nbc
         if (nbc > FZ_CAPB) {
           cut_fallback = 1;        // overflowed bucket: its neurons compare against bucket + overflow list themselves
         } else {
@@ -913,7 +1064,7 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
           if (lane < nbc) ent = __ldcg(&A.bent[((size_t)j * FZ_NB + cut_bin) * FZ_CAPB + lane]);
           const unsigned long long kmine = ((unsigned long long)ent.y << 32) | ent.x;
           int before = 0;
-#pragma unroll
+#pragma unroll 2
           for (int q = 0; q < FZ_CAPB; ++q) {
             const unsigned long long kq = ((unsigned long long)__shfl_sync(0xffffffffu, ent.y, q) << 32) | __shfl_sync(0xffffffffu, ent.x, q);
             const int iq = (int)__shfl_sync(0xffffffffu, ent.z, q);
@@ -935,61 +1086,29 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
     }
     named_bar_sync(1, FZ_THREADS);
     if (tid == 0) FZ_STAMP(1, 60);
-    if (lane == 0) FZ_STAMP(1, 100 + warp * 4);
-    for (int t = tid; t < (K + 1) * n_own; t += FZ_THREADS) {
-      if (lane == 0) FZ_STAMP(1, 101 + warp * 4 + t / FZ_THREADS);
-      const int j = t / n_own, li = t - j * n_own, i = i_lo + li;
-      const int bb = s_bin[(size_t)j * per + li];
-      const int cut_bin = s_cut[j * 4 + 0];
-      if (bb > cut_bin) continue;  // behind the cut
-      const unsigned long long kp = ordered_key(s_own[(size_t)j * per + li]);
-      const unsigned* cnt = A.cnt + (size_t)j * FZ_CNT_STRIDE;
-      bool member = true;
-      int rank = -1;
-      if (bb == cut_bin && !s_cut[j * 4 + 3]) {
-        const unsigned long long tk = s_cutkey[j];
-        member = (kp > tk) || (kp == tk && i <= s_cut[j * 4 + 2]);
-      }
-      if (j == K) continue;  // the final evaluation is ranked bin by bin below
-      if (bb == cut_bin && s_cut[j * 4 + 3]) {
-        // exact rank: fine prefix inside the coarse bin + comparison inside the neuron's bucket
-        const int cb = bb / FPC;
-        unsigned b0 = s_coarse[j * (FZ_NC + 1) + cb], nb = 0;
-#pragma unroll
-        for (int q = 0; q < FPC; q += 4) {
-          const uint4 v = __ldcg(reinterpret_cast<const uint4*>(cnt + cb * FPC + q));
-          const unsigned cv[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            const int fb = cb * FPC + q + u;
-            b0 += fb < bb ? cv[u] : 0u;
-            nb = fb == bb ? cv[u] : nb;
+    {
+      // intermediate evaluations: membership only (bins before the cut bin are in, the cut bin is split by the threshold)
+      uint32_t* const trm = A.tr_masks;
+      const int nwn = (Fn + 31) >> 5;
+      for (int t = tid; t < K * n_own; t += FZ_THREADS) {
+        const int j = t / n_own, li = t - j * n_own, i = i_lo + li;
+        const int bb = s_bin[(size_t)j * per + li];
+        const int cut_bin = s_cut[j * 4 + 0];
+        if (bb > cut_bin) continue;  // behind the cut
+        bool member = true;
+        if (bb == cut_bin) {
+          const unsigned long long kp = ordered_key(s_own[(size_t)j * per + li]);
+          if (!s_cut[j * 4 + 3]) {
+            const unsigned long long tk = s_cutkey[j];
+            member = (kp > tk) || (kp == tk && i <= s_cut[j * 4 + 2]);
+          } else {
+            member = fz_rank_in_overflowed_bin(A, j, bb, i, kp, s_coarse[j * (FZ_NC + 1) + bb / FPC]) < keff;
           }
         }
-        const unsigned novf = nb > (unsigned)FZ_CAPB ? __ldcg(&cnt[FZ_NB + FZ_NC]) : 0u;
-        nb = min(nb, (unsigned)FZ_CAPB);
-        int before = 0;
-        const uint4* bk = A.bent + ((size_t)j * FZ_NB + bb) * FZ_CAPB;
-        uint4 ent[FZ_CAPB];
-#pragma unroll
-        for (int q = 0; q < FZ_CAPB; ++q) ent[q] = __ldcg(bk + q);
-#pragma unroll
-        for (int q = 0; q < FZ_CAPB; ++q) {
-          const unsigned long long kq = ((unsigned long long)ent[q].y << 32) | ent[q].x;
-          before += ((unsigned)q < nb) && ((kq > kp) || (kq == kp && (int)ent[q].z < i));
+        if (member) {
+          if (trm) atomicOr(&trm[(size_t)j * nwn + (i >> 5)], 1u << (i & 31));
+          atomicAdd(&s_nsel[j], 1u);
         }
-        for (unsigned q = 0; q < novf; ++q) {  // only when this neuron's own bin overflowed its bucket
-          const uint4 e = __ldcg(&A.oent[(size_t)j * Fn + q]);
-          if ((int)e.w != bb) continue;
-          const unsigned long long kq = ((unsigned long long)e.y << 32) | e.x;
-          before += (kq > kp) || (kq == kp && (int)e.z < i);
-        }
-        rank = (int)b0 + before;
-        member = rank < keff;
-      }
-      if (member) {
-        if (A.tr_masks) atomicOr(&A.tr_masks[(size_t)j * ((Fn + 31) >> 5) + (i >> 5)], 1u << (i & 31));
-        atomicAdd(&s_nsel[j], 1u);
       }
     }
     // Final evaluation: exact ranks, bin by bin.  A task is a pair of fine bins; the tasks up to the cut are dealt to
@@ -1000,13 +1119,21 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
       const unsigned* cnt = A.cnt + (size_t)j * FZ_CNT_STRIDE;
       const int cut_bin = s_cut[j * 4 + 0];
       const int n_task = cut_bin >= 0 ? (cut_bin / 2 + 1) : 0;  // one task = two fine bins (one per half-warp)
-      const unsigned novf = __ldcg(&cnt[FZ_NB + FZ_NC]);
       const int h = lane >> 4, l16 = lane & 15;
+      int32_t* const nidx = A.next_idx;
+      uint32_t* const nmask = A.next_mask;
+      uint32_t* const trm = A.tr_masks;
+      const int ncap = A.next_cap, nwn = (Fn + 31) >> 5;
+      const uint4* const bent = A.bent + (size_t)j * FZ_NB * FZ_CAPB;
+      unsigned found = 0;
       // task t goes to CTA t % G, warp (t / G) % 16: spread over the whole grid, at most a few per warp
       for (int task = cta + warp * G; task < n_task; task += G * (FZ_THREADS / 32)) {
         const int fbq = task * 2, cb = fbq / FPC;  // first fine bin of the task, its coarse bin
         // fine counts of the coarse bin (two per lane) and their exclusive prefix
         const unsigned f0 = __ldcg(&cnt[cb * FPC + lane * 2]), f1 = __ldcg(&cnt[cb * FPC + lane * 2 + 1]);
+        // this half-warp's bucket, fetched before its first rank is known (the counts arrive at the same time)
+        const int bin = fbq + h;
+        uint4 ent = __ldcg(&bent[(size_t)bin * FZ_CAPB + l16]);
         unsigned fin = f0 + f1;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -1014,71 +1141,34 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
           if (lane >= o) fin += t;
         }
         const unsigned fex = s_coarse[j * (FZ_NC + 1) + cb] + fin - (f0 + f1);  // first rank of fine bin cb*64 + 2*lane
-        for (int it = 0; it < 1; ++it) {
-          const int bin = fbq + h;
-          const int src = (bin - cb * FPC) >> 1, odd = (bin - cb * FPC) & 1;
-          const unsigned pf0 = __shfl_sync(0xffffffffu, f0, src), pf1 = __shfl_sync(0xffffffffu, f1, src);
-          const unsigned pex = __shfl_sync(0xffffffffu, fex, src);
-          const unsigned b0 = odd ? pex + pf0 : pex, nball = odd ? pf1 : pf0;
-          const int nb = (int)min(nball, (unsigned)FZ_CAPB);
-          uint4 ent = make_uint4(0, 0, 0, 0);
-          if (l16 < nb && (int)b0 < keff) ent = __ldcg(&A.bent[((size_t)j * FZ_NB + bin) * FZ_CAPB + l16]);
-          const unsigned long long kmine = ((unsigned long long)ent.y << 32) | ent.x;
-          int before = 0;
-#pragma unroll
-          for (int q = 0; q < FZ_CAPB; ++q) {
-            const unsigned long long kq = ((unsigned long long)__shfl_sync(0xffffffffu, ent.y, q, 16) << 32) | __shfl_sync(0xffffffffu, ent.x, q, 16);
-            const int iq = (int)__shfl_sync(0xffffffffu, ent.z, q, 16);
-            before += (q < nb) && ((kq > kmine) || (kq == kmine && iq < (int)ent.z));
-          }
-          if ((int)b0 >= keff) continue;  // (uniform per half-warp; the shuffles above were executed by all lanes)
-          if (nball > (unsigned)FZ_CAPB) {
-            // overflowed bin (rare): bucket entries also count the overflow entries before them ...
-            for (unsigned q = 0; q < novf; ++q) {
-              const uint4 e = __ldcg(&A.oent[(size_t)j * Fn + q]);
-              if ((int)e.w != bin) continue;
-              const unsigned long long kq = ((unsigned long long)e.y << 32) | e.x;
-              before += (l16 < nb) && ((kq > kmine) || (kq == kmine && (int)e.z < (int)ent.z));
-            }
-            // ... and one lane ranks the overflow entries of the bin themselves
-            if (l16 == 0) {
-              for (unsigned q = 0; q < novf; ++q) {
-                const uint4 e = __ldcg(&A.oent[(size_t)j * Fn + q]);
-                if ((int)e.w != bin) continue;
-                const unsigned long long ke = ((unsigned long long)e.y << 32) | e.x;
-                int bf = 0;
-                for (int u = 0; u < FZ_CAPB; ++u) {
-                  const uint4 o = __ldcg(&A.bent[((size_t)j * FZ_NB + bin) * FZ_CAPB + u]);
-                  const unsigned long long ko = ((unsigned long long)o.y << 32) | o.x;
-                  bf += (ko > ke) || (ko == ke && (int)o.z < (int)e.z);
-                }
-                for (unsigned u = 0; u < novf; ++u) {
-                  const uint4 o = __ldcg(&A.oent[(size_t)j * Fn + u]);
-                  if ((int)o.w != bin) continue;
-                  const unsigned long long ko = ((unsigned long long)o.y << 32) | o.x;
-                  bf += (ko > ke) || (ko == ke && (int)o.z < (int)e.z);
-                }
-                const int rk = (int)b0 + bf;
-                if (rk < keff) {
-                  const int i = (int)e.z;
-                  if (rk < A.next_cap) A.next_idx[rk] = i;
-                  if (A.next_mask) atomicOr(&A.next_mask[i >> 5], 1u << (i & 31));
-                  if (A.tr_masks) atomicOr(&A.tr_masks[(size_t)j * ((Fn + 31) >> 5) + (i >> 5)], 1u << (i & 31));
-                  atomicAdd(&s_nsel[j], 1u);
-                }
-              }
-            }
-          }
-          const int rank = (int)b0 + before;
-          if (l16 < nb && rank < keff) {
-            const int i = (int)ent.z;
-            if (rank < A.next_cap) A.next_idx[rank] = i;
-            if (A.next_mask) atomicOr(&A.next_mask[i >> 5], 1u << (i & 31));
-            if (A.tr_masks) atomicOr(&A.tr_masks[(size_t)j * ((Fn + 31) >> 5) + (i >> 5)], 1u << (i & 31));
-            atomicAdd(&s_nsel[j], 1u);
-          }
+        const int src = (bin - cb * FPC) >> 1, odd = (bin - cb * FPC) & 1;
+        const unsigned pf0 = __shfl_sync(0xffffffffu, f0, src), pf1 = __shfl_sync(0xffffffffu, f1, src);
+        const unsigned pex = __shfl_sync(0xffffffffu, fex, src);
+        const unsigned b0 = odd ? pex + pf0 : pex, nball = odd ? pf1 : pf0;
+        const int nb = (int)min(nball, (unsigned)FZ_CAPB);
+        if (l16 >= nb) ent = make_uint4(0, 0, 0, 0);  // stale bucket slots are ignored
+        const unsigned long long kmine = ((unsigned long long)ent.y << 32) | ent.x;
+        int before = 0;
+#pragma unroll 2
+        for (int q = 0; q < FZ_CAPB; ++q) {
+          const unsigned long long kq = ((unsigned long long)__shfl_sync(0xffffffffu, ent.y, q, 16) << 32) | __shfl_sync(0xffffffffu, ent.x, q, 16);
+          const int iq = (int)__shfl_sync(0xffffffffu, ent.z, q, 16);
+          before += (q < nb) && ((kq > kmine) || (kq == kmine && iq < (int)ent.z));
+        }
+        if ((int)b0 >= keff) continue;  // (uniform per half-warp; the shuffles above were executed by all lanes)
+        if (nball > (unsigned)FZ_CAPB) before += fz_final_overflowed_bin(A, j, bin, b0, ent, l16, keff, &s_nsel[j]);
+        const int rank = (int)b0 + before;
+        if (l16 < nb && rank < keff) {
+          const int i = (int)ent.z;
+          if (rank < ncap) nidx[rank] = i;
+          if (nmask) atomicOr(&nmask[i >> 5], 1u << (i & 31));
+          if (trm) atomicOr(&trm[(size_t)j * nwn + (i >> 5)], 1u << (i & 31));
+          ++found;
         }
       }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) found += __shfl_xor_sync(0xffffffffu, found, o);
+      if (lane == 0 && found) atomicAdd(&s_nsel[j], found);
     }
     if (lane == 0) FZ_STAMP(1, 103 + warp * 4);
     named_bar_sync(1, FZ_THREADS);
