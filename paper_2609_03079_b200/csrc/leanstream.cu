@@ -380,7 +380,7 @@ int32_t fused_args(ls_layer* L, ls_layer* next, const float* d_x, float* d_x_out
                    int sel_cap, int K, int k_next, ls_selection* sel_next, int parity, ls::FusedArgs* out, ls::FusedSmemLayout* lay_out) {
   ls::FusedArgs a{};
   a.bundles = L->bundles; a.n_mat = L->n_mat; a.gated = L->gated; a.b_gate = L->b_gate; a.b_down = L->b_down;
-  a.d = L->d; a.F = L->F; a.norm = L->norm; a.eps = L->eps;
+  a.d = L->d; a.F = L->F; a.norm = L->norm; a.eps = L->eps; a.inv_d = 1.0 / (double)L->d;
   a.x = d_x; a.x_out = d_x_out;
   a.sel_idx = sel_idx; a.sel_count = sel_count; a.sel_cap = sel_cap; a.K = K;
   DeviceScratch* S = nullptr;
@@ -403,7 +403,7 @@ int32_t fused_args(ls_layer* L, ls_layer* next, const float* d_x, float* d_x_out
   }
   ls::FusedSmemLayout lay{};
   if (!fused_plan(L, next, &lay)) return fail(LS_ERR_STATE, "fused step: shared memory plan failed");
-  a.gu_depth = lay.gu_depth; a.dn_depth = lay.dn_depth; a.a_alias = lay.a_alias;
+  a.lay = lay;
   *out = a;
   if (lay_out) *lay_out = lay;
   return LS_OK;
@@ -638,7 +638,15 @@ int32_t ls_stack_create(ls_layer* const* layers, int32_t n_layers, ls_stack** ou
     rc = fused_args(L, next, S->xbuf + (size_t)(n & 1) * S->d, S->xbuf + (size_t)((n + 1) & 1) * S->d,
                     S->selidx + (size_t)(n & 1) * S->max_sel, S->selcnt + (n & 1), S->max_sel, 1, 0, &sn, n & 1, &h[n], &lay);
     if (rc != LS_OK) return cleanup(rc);
-    S->smem = std::max(S->smem, lay.total);
+    S->smem = std::max(S->smem, (size_t)lay.total);
+  }
+  for (int n = 0; n + 1 < n_layers; ++n) {  // what layer n + 1 reads first: its arguments, gate biases, down bias, predictor offsets
+    const ls_layer* L1 = layers[n + 1];
+    const ls_layer* L2 = layers[n + 2 < n_layers ? n + 2 : n + 1];
+    h[n].pf_ptr[0] = S->d_args + (n + 1); h[n].pf_bytes[0] = (unsigned)sizeof(ls::FusedArgs);
+    h[n].pf_ptr[1] = L1->b_gate;          h[n].pf_bytes[1] = L1->b_gate ? (unsigned)(L1->F * sizeof(float)) : 0u;
+    h[n].pf_ptr[2] = L1->b_down;          h[n].pf_bytes[2] = L1->b_down ? (unsigned)(L1->d * sizeof(float)) : 0u;
+    h[n].pf_ptr[3] = L2->pred_c;          h[n].pf_bytes[3] = L2->pred_c ? (unsigned)(L2->F * sizeof(float)) : 0u;
   }
   if (cudaMemcpy(S->d_args, h.data(), sizeof(ls::FusedArgs) * n_layers, cudaMemcpyHostToDevice) != cudaSuccess)
     return cleanup(fail(LS_ERR_CUDA, "ls_stack_create: upload of the layer arguments failed"));

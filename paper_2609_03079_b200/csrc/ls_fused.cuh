@@ -35,8 +35,6 @@ constexpr int FZ_CNT_STRIDE = FZ_NB + FZ_NC + 4;  // fine counts, coarse counts,
 constexpr int FZ_CAPB = 16;       // bucket capacity per fine bin; the rest goes to the overflow list
 constexpr int FZ_MAXK = 16;       // stages supported by the fused path
 constexpr int FZ_MAXE = FZ_MAXK + 1;  // evaluations j = 0..K
-constexpr int FZ_BPAD = 8;        // padding (elements) of a predictor row in shared memory: eight rows on distinct banks
-constexpr int FZ_ZPAD = 4;        // padding (doubles) of a latent row in shared memory
 constexpr int FZ_MAX_DEPTH = 8;   // most gate/up ring stages; the depths are chosen per launch from the shared memory left
 constexpr int FZ_MAX_DN = 16;     // most down ring stages
 constexpr int FZ_SL = 32;         // columns of the feature handled as one slice in the latent phase
@@ -49,14 +47,26 @@ constexpr long long FZ_SPIN_CYCLES = 40LL * 1000 * 1000;
 constexpr long long FZ_SPIN_CYCLES = 4000LL * 1000 * 1000;  // every wait gives up after about two seconds of SM clocks
 #endif
 
+// Shared-memory plan of a layer step (computed on the host, carried in the arguments).
+struct FusedSmemLayout {
+  // fixed regions
+  unsigned bar_off, red_off, redd_off, mine_off, pc_off, xt_off, dv_off, qa_off, a_off;
+  // the stream's rings ...
+  unsigned gu_off, dn_off;
+  // ... and, in the same bytes once the rings have drained, the operands and results of the refinement
+  unsigned b_off, zs_off, part_off, own_off, bin_off, coarse_off;
+  unsigned total;
+  int per, ns_cta, a_alias, gu_depth, dn_depth;
+};
+
 struct FusedArgs {
   // layer being executed
   const uint16_t* bundles; int n_mat; int gated; const float* b_gate; const float* b_down;
   int d, F, norm; float eps;
+  double inv_d;           // 1 / d
   const float* x; float* x_out;
   const int32_t* sel_idx; const int32_t* sel_count; int sel_cap; int K;
-  int gu_depth, dn_depth; // ring stages (host: as many as fit)
-  int a_alias;            // the A slices share bytes with the rings (see fused_layout)
+  FusedSmemLayout lay;    // where everything sits in dynamic shared memory
   float* dacc;            // [FZ_MAXK][d] stage accumulators, zero on entry and on exit
   unsigned* fin;          // [1] CTAs finished, zero on entry and on exit
   unsigned long long* bar_count;  // [1] barrier arrivals since the layer was created (monotonic)
@@ -77,6 +87,8 @@ struct FusedArgs {
   unsigned* nsel;         // [FZ_MAXE] sizes of the refined sets (all CTAs add theirs), zero on entry and on exit
   // outputs for the next layer
   int32_t* next_idx; int32_t* next_count; uint32_t* next_mask; double* next_scores; double* next_prio; int next_cap;
+  // what the layer after this one will read first (whole-token kernel): brought into L2 while this layer refines
+  const void* pf_ptr[4]; unsigned pf_bytes[4];
   // trace (all nullable)
   float* tr_xtilde; uint32_t* tr_masks; int32_t* tr_counts; uint32_t* tr_survive;
 };
@@ -133,14 +145,43 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait: gives up after a fixed number of SM clocks and records a timeout instead of hanging.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* status) {
-  if (mbar_try_wait(bar, parity)) return true;
+// Bounded wait: gives up after a fixed number of SM clocks and records a timeout instead of hanging.  The first probe is
+// inline; the spinning part is a call, so that a wait costs a handful of instructions where it stands.
+__device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, int* status) {
   const long long t0 = clock64();
   while (clock64() - t0 < FZ_SPIN_CYCLES)
     if (mbar_try_wait(bar, parity)) return true;
   set_status(status, ST_TIMEOUT);
   return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, status);
+}
+// The producer's wait for the compute warps: s_round >= want (bounded like every other wait).
+__device__ __noinline__ bool fz_wait_round(int* s_round, int want, int* status) {
+  const long long t0 = clock64();
+  do {
+    int v;
+    asm volatile("ld.acquire.cta.shared.s32 %0, [%1];" : "=r"(v) : "r"((uint32_t)__cvta_generic_to_shared(s_round)) : "memory");
+    if (v >= want) return true;
+  } while (clock64() - t0 < FZ_SPIN_CYCLES);
+  set_status(status, ST_TIMEOUT);
+  return false;
+}
+// 1 / sqrt(a) in double precision from the hardware approximation and two Newton steps (relative error of a few ulp; a
+// full-precision divide and square root would be over a hundred instructions where they stand).
+__device__ __forceinline__ double fz_rsqrt(double a) {
+  double y;
+  asm("rsqrt.approx.ftz.f64 %0, %1;" : "=d"(y) : "d"(a));
+  if (a > 0.0 && a < 1.0e300) {  // (zero, infinity and NaN keep what the approximation returns)
+#pragma unroll
+    for (int it = 0; it < 2; ++it) {
+      const double h = 0.5 * a * y;
+      y = fma(y, fma(-h, y, 0.5), y);
+    }
+  }
+  return y;
 }
 // 1-D bulk copy global -> shared, completion counted in bytes on an mbarrier (no multicast).
 __device__ __forceinline__ void tma_load_1d(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
@@ -183,38 +224,69 @@ __device__ __forceinline__ double w16_to_double(uint16_t b) {
   return (double)__half2float(__ushort_as_half(b));
 }
 
-// Stage c of K runs on the CTAs [c*G/K, (c+1)*G/K).
-__host__ __device__ inline int fz_group_lo(int c, int G, int K) { return (int)(((long long)c * G) / K); }
-__host__ __device__ inline int fz_stage_of_cta(int cta, int G, int K) {
-  int c = (int)(((long long)cta * K) / G);
-  while (c + 1 < K && fz_group_lo(c + 1, G, K) <= cta) ++c;
-  while (c > 0 && fz_group_lo(c, G, K) > cta) --c;
-  return c;
+// ---- fp64 tensor-core blocks ------------------------------------------------------------------------------------------
+// Both predictor products (A^T x~ and B^T z) are cut into blocks of 32 columns, and the order of the columns INSIDE a
+// block is permuted (the sum over a block does not depend on it): lane (g, t) of a warp, g = lane / 4, t = lane % 4,
+// takes the eight consecutive columns 8t .. 8t+7, so that its eight weights are ONE 16-byte load, and the k-th MMA of the
+// block pairs column 8t + k of the weights with the same column of the features.  Features are stored for that access:
+// column c of a block sits at (c / 8) * 10 + c % 8 doubles (eight doubles, two of padding), which makes the 16-byte
+// feature loads of a quarter-warp fall on distinct banks when the row stride is 16 words modulo 32.
+constexpr int FZ_XBLK = 40;  // doubles a 32-column block of features occupies in shared memory
+__host__ __device__ inline int fz_feat_pos(int c) { return (c >> 5) * FZ_XBLK + ((c >> 3) & 3) * 10 + (c & 7); }
+// Row stride (doubles) of a feature array with `cols` columns: whole blocks, 16 words modulo 32.
+__host__ __device__ inline int fz_feat_stride(int cols) {
+  const int nb = (cols + 31) >> 5;
+  return nb * FZ_XBLK + ((nb & 1) ? 0 : 8);
+}
+// Row stride (16-bit elements) of the B^T rows in shared memory: whole blocks, 64 bytes modulo 128.
+__host__ __device__ inline int fz_brow_stride(int r) {
+  const int c = ((r + 31) >> 5) << 5;
+  return c + ((c & 63) == 32 ? 0 : 32);
 }
 
-struct FusedSmemLayout {
-  // fixed regions
-  size_t bar_off, red_off, redd_off, mine_off, pc_off, xt_off, dv_off, qa_off, a_off;
-  // the stream's rings ...
-  size_t gu_off, dn_off;
-  // ... and, in the same bytes once the rings have drained, the operands and results of the refinement
-  size_t b_off, zs_off, part_off, own_off, bin_off, coarse_off;
-  size_t total;
-  int per, ns_cta, a_alias, gu_depth, dn_depth;
-};
+template <int WD>
+__device__ __forceinline__ void cvt8_to_double(const uint4 w, double a[8]) {
+  const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    a[2 * q] = w16_to_double<WD>((uint16_t)(ww[q] & 0xffffu));
+    a[2 * q + 1] = w16_to_double<WD>((uint16_t)(ww[q] >> 16));
+  }
+}
+__device__ __forceinline__ void load8d(const double* p, double v[8]) {  // 16-byte aligned
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const double2 t = *reinterpret_cast<const double2*>(p + 2 * q);
+    v[2 * q] = t.x;
+    v[2 * q + 1] = t.y;
+  }
+}
+// c (8 rows x 8 features, this lane's two elements) += one block: weights a[8] of this lane's row, features b[8]
+__device__ __forceinline__ void mma_block(double (&c)[2], const double a[8], const double b[8]) {
+#pragma unroll
+  for (int k = 0; k < 8; ++k)
+    asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
+                 : "+d"(c[0]), "+d"(c[1]) : "d"(a[k]), "d"(b[k]));
+}
+// sum over the four lanes of a row (fixed order)
+__device__ __forceinline__ double quad_sum(double v) {
+  v += __shfl_xor_sync(0xffffffffu, v, 1);
+  v += __shfl_xor_sync(0xffffffffu, v, 2);
+  return v;
+}
 
 // Bar indices: [0, FZ_MAX_DEPTH) gate/up slots, [FZ_MAX_DEPTH, +FZ_MAX_DN) down slots, then the A slices, then B^T rows.
 constexpr int FZ_BAR_DN = FZ_MAX_DEPTH, FZ_BAR_A = FZ_MAX_DEPTH + FZ_MAX_DN, FZ_BAR_B = FZ_BAR_A + 1, FZ_NBAR = FZ_BAR_B + 1;
 
 // `a_alias` != 0 places the A slices inside the ring bytes too (they are then fetched only after the rings have drained).
-__host__ __device__ inline FusedSmemLayout fused_layout(int d, int n_in, int r, int Fn, int G, int has_next, int gu_depth, int dn_depth,
+inline FusedSmemLayout fused_layout(int d, int n_in, int r, int Fn, int G, int has_next, int gu_depth, int dn_depth,
                                                         int a_alias) {
   FusedSmemLayout L{};
   L.gu_depth = gu_depth;
   L.dn_depth = dn_depth;
   L.a_alias = a_alias;
   size_t o = 0;
-  auto take = [&](size_t bytes) { size_t at = o; o += (bytes + 127) & ~(size_t)127; return at; };
+  auto take = [&](size_t bytes) { size_t at = o; o += (bytes + 127) & ~(size_t)127; return (unsigned)at; };
   const int nsl = (d + FZ_SL - 1) / FZ_SL;
   L.per = has_next ? (Fn + G - 1) / G : 0;
   L.ns_cta = (nsl + G - 1) / G;
@@ -224,7 +296,7 @@ __host__ __device__ inline FusedSmemLayout fused_layout(int d, int n_in, int r, 
   L.redd_off = take(32 * 8);                         // fp64 partials of block reductions
   L.mine_off = take((size_t)FZ_MAX_MINE * 8);        // this CTA's neuron indices and gate biases
   L.pc_off = take((size_t)L.per * 4);
-  L.xt_off = take((size_t)FZ_EPAD * (FZ_SL + 4) * 8);  // x~^(j) of one slice, fp64, padded rows
+  L.xt_off = take((size_t)FZ_EPAD * FZ_XBLK * 8);  // x~^(j) of one slice, fp64, one padded block per row
   L.dv_off = take((size_t)FZ_MAXK * FZ_SL * 4);      // stage accumulators of one slice
   L.qa_off = take(FZ_MAX_DN * 4);                    // activations of the queued down rows
   if (!a_alias) L.a_off = take(a_bytes);
@@ -235,13 +307,13 @@ __host__ __device__ inline FusedSmemLayout fused_layout(int d, int n_in, int r, 
   o = base;
   if (a_alias) L.a_off = take(a_bytes);
   const int per8 = (L.per + 7) / 8 * 8;
-  L.b_off = take((size_t)per8 * (r + FZ_BPAD) * 2);
-  L.zs_off = take(has_next ? (size_t)FZ_EPAD * (r + FZ_ZPAD) * 8 : 0);
+  L.b_off = take((size_t)per8 * fz_brow_stride(r) * 2);
+  L.zs_off = take(has_next ? (size_t)FZ_EPAD * fz_feat_stride(r) * 8 : 0);
   L.part_off = take(has_next ? (size_t)FZ_KS * FZ_EPAD * per8 * 8 : 0);  // [split][evaluation][neuron]
   L.own_off = take((size_t)FZ_MAXE * L.per * 8);     // this CTA's scores, every evaluation
   L.bin_off = take((size_t)FZ_MAXE * L.per * 2);     // and their fine bins
   L.coarse_off = take(has_next ? (size_t)FZ_MAXE * (FZ_NC + 1) * 4 : 0);
-  L.total = o > end_stream ? o : end_stream;
+  L.total = (unsigned)(o > end_stream ? o : end_stream);
   return L;
 }
 
@@ -252,6 +324,7 @@ struct FusedShared {
   FusedArgs prev;                    // whole-token kernel: the layer before, whose scratch is cleaned meanwhile
   int last;
   int round;                         // rounds the compute warps have finished (read by the producer)
+  int stage, g_lo, gsize;            // this CTA's stage, the first CTA of the stage's group and the group's size
   unsigned phase[FZ_NBAR];           // phases every mbarrier has completed in earlier layers of the launch
   int mail[4 * 4];                   // per round (ring of four): number of survivors, their neurons
   float act[2 * 4];                  // activations of the round's neurons, double-buffered
@@ -271,15 +344,18 @@ __device__ __noinline__ int fz_rank_in_overflowed_bin(const FusedArgs& A, int j,
   constexpr int FPC = FZ_NB / FZ_NC;
   const unsigned* cnt = A.cnt + (size_t)j * FZ_CNT_STRIDE;
   unsigned b0 = coarse_b0;
+#pragma unroll 1
   for (int fb = (bb / FPC) * FPC; fb < bb; ++fb) b0 += __ldcg(&cnt[fb]);
   int before = 0;
   const uint4* bk = A.bent + ((size_t)j * FZ_NB + bb) * FZ_CAPB;
+#pragma unroll 1
   for (int q = 0; q < FZ_CAPB; ++q) {  // the bucket is full
     const uint4 e = __ldcg(bk + q);
     const unsigned long long kq = ((unsigned long long)e.y << 32) | e.x;
     before += (kq > kp) || (kq == kp && (int)e.z < i);
   }
   const unsigned novf = __ldcg(&cnt[FZ_NB + FZ_NC]);
+#pragma unroll 1
   for (unsigned q = 0; q < novf; ++q) {
     const uint4 e = __ldcg(&A.oent[(size_t)j * A.Fn + q]);
     if ((int)e.w != bb) continue;
@@ -298,6 +374,7 @@ __device__ __noinline__ int fz_final_overflowed_bin(const FusedArgs& A, int j, i
   const unsigned novf = __ldcg(&cnt[FZ_NB + FZ_NC]);
   const unsigned long long kmine = ((unsigned long long)ent.y << 32) | ent.x;
   int before = 0;
+#pragma unroll 1
   for (unsigned q = 0; q < novf; ++q) {
     const uint4 e = __ldcg(&A.oent[(size_t)j * A.Fn + q]);
     if ((int)e.w != bin) continue;
@@ -305,16 +382,19 @@ __device__ __noinline__ int fz_final_overflowed_bin(const FusedArgs& A, int j, i
     before += (kq > kmine) || (kq == kmine && (int)e.z < (int)ent.z);
   }
   if (l16 == 0) {
+#pragma unroll 1
     for (unsigned q = 0; q < novf; ++q) {
       const uint4 e = __ldcg(&A.oent[(size_t)j * A.Fn + q]);
       if ((int)e.w != bin) continue;
       const unsigned long long ke = ((unsigned long long)e.y << 32) | e.x;
       int bf = 0;
+#pragma unroll 1
       for (int u = 0; u < FZ_CAPB; ++u) {
         const uint4 o = __ldcg(&A.bent[((size_t)j * FZ_NB + bin) * FZ_CAPB + u]);
         const unsigned long long ko = ((unsigned long long)o.y << 32) | o.x;
         bf += (ko > ke) || (ko == ke && (int)o.z < (int)e.z);
       }
+#pragma unroll 1
       for (unsigned u = 0; u < novf; ++u) {
         const uint4 o = __ldcg(&A.oent[(size_t)j * A.Fn + u]);
         if ((int)o.w != bin) continue;
@@ -334,59 +414,31 @@ __device__ __noinline__ int fz_final_overflowed_bin(const FusedArgs& A, int j, i
   return before;
 }
 
-// One score task on the fp64 tensor cores: eight predictor rows (16-bit, row stride RSB elements, `arow` already points at
-// this lane's row and column) times NT tiles of eight latents (row stride RSZ doubles, `brow` likewise) over the columns
-// [k_lo, k_hi); partial sums to out[evaluation * ostride] at this lane's neuron.
-template <int WD, int NT>
-__device__ __forceinline__ void score_task_mma(const uint16_t* arow, const double* brow, int RSZ, int k_lo, int k_hi, double* out,
-                                               int ostride, int lane) {
-  double c[NT][2], e[NT][2];
-#pragma unroll
-  for (int nt = 0; nt < NT; ++nt) { c[nt][0] = c[nt][1] = e[nt][0] = e[nt][1] = 0.0; }
-#pragma unroll 4
-  for (int k0 = k_lo; k0 < k_hi; k0 += 8) {
-    const double a0v = w16_to_double<WD>(arow[k0]), a1v = w16_to_double<WD>(arow[k0 + 4]);
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt) {
-      const double b0v = brow[(size_t)nt * 8 * RSZ + k0], b1v = brow[(size_t)nt * 8 * RSZ + k0 + 4];
-      asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
-                   : "+d"(c[nt][0]), "+d"(c[nt][1]) : "d"(a0v), "d"(b0v));
-      asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
-                   : "+d"(e[nt][0]), "+d"(e[nt][1]) : "d"(a1v), "d"(b1v));
-    }
-  }
-#pragma unroll
-  for (int nt = 0; nt < NT; ++nt) {
-    const int j = nt * 8 + (lane & 3) * 2;
-    out[(size_t)j * ostride] = c[nt][0] + e[nt][0];
-    out[(size_t)(j + 1) * ostride] = c[nt][1] + e[nt][1];
-  }
-}
-
 // One layer step, executed by the whole block (16 compute warps + the producer warp).  The producer warp returns as
 // soon as it has issued its last copy; the compute warps return when the layer's refined sets are written.
-// `first_layer` says that this is the first layer of the launch (the mbarriers in shared memory are set up then).
+// `first_layer` says that this is the first layer of the launch (the mbarriers in shared memory are set up then);
+// `known_count` >= 0 is the size of the selection when the caller knows it without reading it.
 template <int WD, int CPT>
-__device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* smem, FusedShared& sh, bool first_layer) {
+__device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* smem, FusedShared& sh, bool first_layer,
+                                            int known_count) {
   const int G = gridDim.x, cta = blockIdx.x, tid = threadIdx.x;
   const int lane = tid & 31, warp = tid >> 5;
   const int d = A.d, K = A.K, nchunk = A.d >> 3;
   const int n_in = A.gated ? 2 : 1;
-  const FusedSmemLayout lay = fused_layout(d, n_in, A.r, A.Fn, G, A.has_next, A.gu_depth, A.dn_depth, A.a_alias);
-  const int GU = A.gu_depth, DN = A.dn_depth;
+  const FusedSmemLayout& lay = A.lay;
+  const int GU = lay.gu_depth, DN = lay.dn_depth;
   uint16_t* s_gu = reinterpret_cast<uint16_t*>(smem + lay.gu_off);
   uint16_t* s_dn = reinterpret_cast<uint16_t*>(smem + lay.dn_off);
   uint64_t* s_bar = reinterpret_cast<uint64_t*>(smem + lay.bar_off);  // "full" barriers: gate/up slots, down slots, A, B^T
   float* s_red = reinterpret_cast<float*>(smem + lay.red_off);        // [2][16 warps][8]
   double* s_redd = reinterpret_cast<double*>(smem + lay.redd_off);
   uint16_t* s_A = reinterpret_cast<uint16_t*>(smem + lay.a_off);      // [ns_cta][r][32]
-  uint16_t* s_B = reinterpret_cast<uint16_t*>(smem + lay.b_off);      // [per][r + FZ_BPAD]
+  uint16_t* s_B = reinterpret_cast<uint16_t*>(smem + lay.b_off);      // [per8][fz_brow_stride(r)]
   float* s_pc = reinterpret_cast<float*>(smem + lay.pc_off);
   double* s_xt = reinterpret_cast<double*>(smem + lay.xt_off);        // [K+1][32]
   float* s_qa = reinterpret_cast<float*>(smem + lay.qa_off);          // [DN]
   int& s_round = sh.round;
   int* s_mail = sh.mail;
-  float* s_act = sh.act;
   double* s_inv = sh.inv;
   int* s_cut = sh.cut;
   unsigned long long* s_cutkey = sh.cutkey;
@@ -400,11 +452,18 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
   unsigned* s_phase = sh.phase;
   if (first_layer) {
     if (tid == 0) {
+#pragma unroll 1
       for (int i = 0; i < FZ_NBAR; ++i) mbar_init(&s_bar[i], 1);
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     if (tid < FZ_NBAR) s_phase[tid] = 0u;
+    if (tid == 32) {  // stage c of K runs on the CTAs [c G / K, (c + 1) G / K)
+      const int c = ((cta + 1) * K - 1) / G;
+      sh.stage = c;
+      sh.g_lo = c * G / K;
+      sh.gsize = (c + 1) * G / K - sh.g_lo;
+    }
   }
   if (tid == 0) s_round = 0;
   __syncthreads();
@@ -419,170 +478,168 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
   {
     // ================================================= stream: all warps ===========================================
     // this CTA serves one stage: the ranks [lo, hi) of the selection, every gsize-th neuron starting at its own offset
-    const int count = max(0, min(__ldcg(A.sel_count), A.sel_cap));
+    const int count = max(0, min(known_count >= 0 ? known_count : __ldcg(A.sel_count), A.sel_cap));
     const int m = count > 0 ? (count + K - 1) / K : 0;
-    const int stage = fz_stage_of_cta(cta, G, K);
-    const int g_lo = fz_group_lo(stage, G, K), gsize = fz_group_lo(stage + 1, G, K) - g_lo;
+    const int stage = sh.stage, g_lo = sh.g_lo, gsize = sh.gsize;
     const int lo = min(count, stage * m), hi = min(count, (stage + 1) * m);
     const int first = lo + (cta - g_lo);
     const int n_mine = first < hi ? (hi - first + gsize - 1) / gsize : 0;
+    const int n_rounds = (n_mine + FZ_NG - 1) / FZ_NG;
     const uint32_t gu_bytes = (uint32_t)n_in * d * 2, dn_bytes = (uint32_t)d * 2;
     const size_t bundle_elems = (size_t)A.n_mat * d;
 
-    // this CTA's neurons first (the bulk copies only need the indices), then x and the gate biases
+    // this CTA's neurons first (the bulk copies only need the indices), then x
     int* s_myidx = reinterpret_cast<int*>(smem + lay.mine_off);
     float* s_mybias = reinterpret_cast<float*>(s_myidx + FZ_MAX_MINE);
+#pragma unroll 1
     for (int t = tid; t < n_mine; t += FZ_THREADS) {
       int i = __ldcg(A.sel_idx + first + t * gsize);
       if ((unsigned)i >= (unsigned)A.F) { set_status(A.status, ST_BAD_INDEX); i = -1; }
       s_myidx[t] = i;
     }
     float xr[CPT][8];
-    double sq = 0.0;
+    {
+      double sq = 0.0;
 #pragma unroll
-    for (int q = 0; q < CPT; ++q) {
-      const int ch = tid + q * FZ_THREADS;
-      if (ch < nchunk) {
-        const float4 a0 = __ldcg(reinterpret_cast<const float4*>(A.x + ch * 8));
-        const float4 a1 = __ldcg(reinterpret_cast<const float4*>(A.x + ch * 8 + 4));
-        xr[q][0] = a0.x; xr[q][1] = a0.y; xr[q][2] = a0.z; xr[q][3] = a0.w;
-        xr[q][4] = a1.x; xr[q][5] = a1.y; xr[q][6] = a1.z; xr[q][7] = a1.w;
-      } else {
+      for (int q = 0; q < CPT; ++q) {
+        const int ch = tid + q * FZ_THREADS;
+        if (ch < nchunk) {
+          const float4 a0 = __ldcg(reinterpret_cast<const float4*>(A.x + ch * 8));
+          const float4 a1 = __ldcg(reinterpret_cast<const float4*>(A.x + ch * 8 + 4));
+          xr[q][0] = a0.x; xr[q][1] = a0.y; xr[q][2] = a0.z; xr[q][3] = a0.w;
+          xr[q][4] = a1.x; xr[q][5] = a1.y; xr[q][6] = a1.z; xr[q][7] = a1.w;
+        } else {
 #pragma unroll
-        for (int e = 0; e < 8; ++e) xr[q][e] = 0.f;
+          for (int e = 0; e < 8; ++e) xr[q][e] = 0.f;
+        }
+#pragma unroll
+        for (int e = 0; e < 8; ++e) sq = fma((double)xr[q][e], (double)xr[q][e], sq);
       }
-#pragma unroll
-      for (int e = 0; e < 8; ++e) sq = fma((double)xr[q][e], (double)xr[q][e], sq);
+      sq = warp_sum(sq);
+      if (lane == 0 && warp < FZ_THREADS / 32) s_redd[warp] = sq;
     }
-    __syncthreads();  // indices visible (the producer warp takes part in this barrier, then goes its own way)
+    __syncthreads();  // indices and the sums of squares visible (the producer warp goes its own way from here)
     if (tid == 0) FZ_STAMP(1, 21);
 
     if (warp == FZ_THREADS / 32) {
       // ============================================= producer warp (one lane) ======================================
-      // Issues every bulk copy, so that the compute warps never pay for it: the first ring fills, the predictor
-      // operands, and after each round (announced through s_round) the refills and the survivors' down rows.
+      // Issues every bulk copy, so that the compute warps never pay for it.  Step rd waits until the compute warps have
+      // finished rd rounds (announced through s_round), tops the gate/up ring up to the rows that may then be in
+      // flight, and fetches the down rows of round rd-1's survivors.
       if (lane == 0) {
-        auto issue_gu = [&](int it) {
-          int i = s_myidx[it];
-          if (i < 0) i = 0;  // a rejected index: read row 0, the result is discarded
-          uint64_t* bar = &s_bar[it % GU];
-          mbar_expect_tx(bar, gu_bytes);
-          tma_load_1d(s_gu + (size_t)(it % GU) * n_in * d, A.bundles + (size_t)i * bundle_elems, gu_bytes, bar);
-        };
-        for (int it = 0; it < min(n_mine, GU); ++it) issue_gu(it);
-        const int n_rounds = (n_mine + FZ_NG - 1) / FZ_NG;
-        auto wait_round = [&](int want) {  // the compute warps have finished `want` rounds (n_rounds + 1: rings drained)
-          const long long t0 = clock64();
-          do {
-            int v;
-            asm volatile("ld.acquire.cta.shared.s32 %0, [%1];" : "=r"(v) : "r"(smem_u32(&s_round)) : "memory");
-            if (v >= want) return true;
-          } while (clock64() - t0 < FZ_SPIN_CYCLES);
-          set_status(A.status, ST_TIMEOUT);
-          FZ_FAIL(1, want);
-          return false;
-        };
-        auto issue_a = [&]() {  // this CTA's column slices of the next layer's A
-          uint64_t* abar = &s_bar[FZ_BAR_A];
-          uint32_t bytes = 0;
-          for (int a = 0; a < lay.ns_cta; ++a)
-            if (cta + a * G < nsl) bytes += (uint32_t)r * FZ_SL * 2;
-          mbar_expect_tx(abar, bytes);
-          for (int a = 0; a < lay.ns_cta; ++a) {
-            const int sl = cta + a * G;
-            if (sl < nsl)
-              tma_load_1d(s_A + (size_t)a * r * FZ_SL, A.At_sl + (size_t)sl * r * FZ_SL, (uint32_t)r * FZ_SL * 2, abar);
-          }
-        };
-        int tail = 0;
+        int issued = 0, gslot = 0, dslot = 0;
         bool ok = true;
-        for (int rd = 0; rd < n_rounds && ok; ++rd) {
-          ok = wait_round(rd + 1);
-          if (!ok) break;
-          const int it0 = rd * FZ_NG, nn = min(FZ_NG, n_mine - it0);
-          for (int e = 0; e < nn; ++e)
-            if (it0 + e + GU < n_mine) issue_gu(it0 + e + GU);
-          const int* mail = s_mail + (rd & 3) * 4;
-          const int ns = mail[0];
-          for (int e = 0; e < ns; ++e) {
-            const int i = mail[1 + e];
-            const int ds = tail % DN;
-            uint64_t* bar = &s_bar[FZ_BAR_DN + ds];
-            mbar_expect_tx(bar, dn_bytes);
-            tma_load_1d(s_dn + (size_t)ds * d, A.bundles + (size_t)i * bundle_elems + (size_t)(A.n_mat - 1) * d, dn_bytes, bar);
-            if (A.tr_survive) atomicOr(&A.tr_survive[i >> 5], 1u << (i & 31));
-            ++tail;
+#pragma unroll 1
+        for (int rd = 0; rd <= n_rounds; ++rd) {
+          if (rd > 0 && !(ok = fz_wait_round(&s_round, rd, A.status))) break;
+          const int want = min(n_mine, rd * FZ_NG + GU);
+#pragma unroll 1
+          for (; issued < want; ++issued) {
+            int i = s_myidx[issued];
+            if (i < 0) i = 0;  // a rejected index: read row 0, the result is discarded
+            uint64_t* bar = &s_bar[gslot];
+            mbar_expect_tx(bar, gu_bytes);
+            tma_load_1d(s_gu + (size_t)gslot * n_in * d, A.bundles + (size_t)i * bundle_elems, gu_bytes, bar);
+            if (++gslot == GU) gslot = 0;
+          }
+          if (rd > 0) {
+            const int* mail = s_mail + ((rd - 1) & 3) * 4;
+            const int ns = mail[0];
+#pragma unroll 1
+            for (int e = 0; e < ns; ++e) {
+              const int i = mail[1 + e];
+              uint64_t* bar = &s_bar[FZ_BAR_DN + dslot];
+              mbar_expect_tx(bar, dn_bytes);
+              tma_load_1d(s_dn + (size_t)dslot * d, A.bundles + (size_t)i * bundle_elems + (size_t)(A.n_mat - 1) * d, dn_bytes, bar);
+              if (A.tr_survive) atomicOr(&A.tr_survive[i >> 5], 1u << (i & 31));
+              if (++dslot == DN) dslot = 0;
+            }
           }
         }
         // The next layer's predictor operands, off the streaming's critical path.  A slices that have a place of their
         // own are fetched now; everything that shares bytes with the rings waits until the compute warps have drained them.
         if (A.has_next && ok) {
-          if (!lay.a_alias) issue_a();
-          if (wait_round(n_rounds + 1)) {
-            if (lay.a_alias) issue_a();
-            uint64_t* bbar = &s_bar[FZ_BAR_B];  // rows of B^T: awaited before the score phase
+          bool drained = false;
+          if (lay.a_alias) drained = ok = fz_wait_round(&s_round, n_rounds + 1, A.status);
+          if (ok) {  // this CTA's column slices of the next layer's A
+            uint64_t* abar = &s_bar[FZ_BAR_A];
+            const uint32_t sl_bytes = (uint32_t)r * FZ_SL * 2;
+            int nmy = 0;
+#pragma unroll 1
+            for (int sl = cta; sl < nsl; sl += G) ++nmy;
+            mbar_expect_tx(abar, (uint32_t)nmy * sl_bytes);
+            int a = 0;
+#pragma unroll 1
+            for (int sl = cta; sl < nsl; sl += G, ++a)
+              tma_load_1d(s_A + (size_t)a * r * FZ_SL, A.At_sl + (size_t)sl * r * FZ_SL, sl_bytes, abar);
+          }
+          if (!drained) ok = ok && fz_wait_round(&s_round, n_rounds + 1, A.status);
+          if (ok) {  // rows of B^T: awaited before the score phase
+            uint64_t* bbar = &s_bar[FZ_BAR_B];
             mbar_expect_tx(bbar, (uint32_t)n_own * (uint32_t)r * 2);
+#pragma unroll 1
             for (int li = 0; li < n_own; ++li)
-              tma_load_1d(s_B + (size_t)li * (r + FZ_BPAD), A.Bt + (size_t)(i_lo + li) * r, (uint32_t)r * 2, bbar);
+              tma_load_1d(s_B + (size_t)li * fz_brow_stride(r), A.Bt + (size_t)(i_lo + li) * r, (uint32_t)r * 2, bbar);
           }
         }
       }
       return;  // an exited warp counts as arrived at every later block barrier
     }
 
+#pragma unroll 1
     for (int t = tid; t < n_mine; t += FZ_THREADS) {
       const int i = s_myidx[t];
       s_mybias[t] = (A.b_gate && i >= 0) ? A.b_gate[i] : 0.f;
     }
     if (A.has_next)
+#pragma unroll 1
       for (int li = tid; li < n_own; li += FZ_THREADS) s_pc[li] = A.pc ? A.pc[i_lo + li] : 0.f;
-    sq = warp_sum(sq);
-    if (lane == 0) s_redd[warp] = sq;
-    if (tid == 0) FZ_STAMP(1, 22);
-    named_bar_sync(1, FZ_THREADS);
-    if (tid == 0) FZ_STAMP(1, 23);
-    double tot = 0.0;
-#pragma unroll
-    for (int w = 0; w < FZ_THREADS / 32; ++w) tot += s_redd[w];
-    const float inv_rms = A.norm == 0 ? (float)(1.0 / sqrt(tot / (double)d + (double)A.eps)) : 1.0f;
+    float inv_rms = 1.0f;
+    if (A.norm == 0) {
+      double tot = 0.0;
+#pragma unroll 4
+      for (int w = 0; w < FZ_THREADS / 32; ++w) tot += s_redd[w];
+      inv_rms = (float)fz_rsqrt(fma(tot, A.inv_d, (double)A.eps));
+    }
 
-    // pending down rows: FIFO over the down ring; their activations wait in s_qa, every thread tracks head and tail
-    int dq_head = 0, dq_tail = 0;
+    // pending down rows: FIFO over the down ring (head slot hslot, its use count hwrap; tail slot tslot); their
+    // activations wait in s_qa; every thread tracks the same head and tail
+    int dq_head = 0, dq_tail = 0, hslot = 0, tslot = 0, gslot = 0;
+    unsigned hwrap = 0, gwrap = 0;
     float yacc[CPT][8];
 #pragma unroll
     for (int q = 0; q < CPT; ++q)
 #pragma unroll
       for (int e = 0; e < 8; ++e) yacc[q][e] = 0.f;
-    bool dirty = false;
     if (tid == 0) FZ_STAMP(0, 0);
     if (tid == 0) { FZ_CSTAMP(1); FZ_CVAL(8, n_mine); FZ_CVAL(10, stage); }
 
-    auto consume_one = [&]() {  // the oldest pending down row, scaled, joins the CTA's partial output
-      const int slot = dq_head % DN;
-      if (!mbar_wait(&s_bar[FZ_BAR_DN + slot], (s_phase[FZ_BAR_DN + slot] + (uint32_t)(dq_head / DN)) & 1u, A.status)) FZ_FAIL(3, dq_head);
-      const float a = s_qa[slot];
-      const uint16_t* row = s_dn + (size_t)slot * d;
-#pragma unroll
-      for (int q = 0; q < CPT; ++q) {
-        const int ch = tid + q * FZ_THREADS;
-        if (ch < nchunk) {
-          float w[8];
-          unpack8<WD>(*reinterpret_cast<const uint4*>(row + ch * 8), w);
-#pragma unroll
-          for (int e = 0; e < 8; ++e) yacc[q][e] = fmaf(a, w[e], yacc[q][e]);
-        }
-      }
-      dirty = true;
-      ++dq_head;
-    };
-
-    const int n_rounds = (n_mine + FZ_NG - 1) / FZ_NG;
-    for (int rd = 0; rd < n_rounds; ++rd) {
+#pragma unroll 1
+    for (int rd = 0; rd <= n_rounds; ++rd) {  // the last pass only drains the down ring
       const int it0 = rd * FZ_NG;
       const int nn = min(FZ_NG, n_mine - it0);
       if (tid == 0) FZ_STAMP(0, 1 + rd * 4);
-      // (1) make room in the down ring for this round's survivors (reads of a slot end before the round barrier)
-      while (dq_tail - dq_head > DN - FZ_NG) consume_one();
+      // (1) make room in the down ring for this round's survivors (reads of a slot end before the round barrier);
+      //     each pending row, scaled by its activation, joins the CTA's partial output
+#pragma unroll 1
+      while (rd == n_rounds ? dq_head < dq_tail : dq_tail - dq_head > DN - FZ_NG) {
+        mbar_wait(&s_bar[FZ_BAR_DN + hslot], (s_phase[FZ_BAR_DN + hslot] + hwrap) & 1u, A.status);
+        const float a = s_qa[hslot];
+        const uint16_t* row = s_dn + (size_t)hslot * d;
+#pragma unroll
+        for (int q = 0; q < CPT; ++q) {
+          const int ch = tid + q * FZ_THREADS;
+          if (ch < nchunk) {
+            float w[8];
+            unpack8<WD>(*reinterpret_cast<const uint4*>(row + ch * 8), w);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) yacc[q][e] = fmaf(a, w[e], yacc[q][e]);
+          }
+        }
+        ++dq_head;
+        if (++hslot == DN) { hslot = 0; ++hwrap; }
+      }
+      if (rd == n_rounds) break;
       // (2) partial dot products of the round's neurons
       float pg[FZ_NG], pu[FZ_NG];
 #pragma unroll
@@ -590,9 +647,8 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
         pg[e] = 0.f;
         pu[e] = 0.f;
         if (e < nn) {
-          const int it = it0 + e, slot = it % GU;
-          if (!mbar_wait(&s_bar[slot], (s_phase[slot] + (uint32_t)(it / GU)) & 1u, A.status)) FZ_FAIL(2, it);
-          const uint16_t* grow = s_gu + (size_t)slot * n_in * d;
+          mbar_wait(&s_bar[gslot], (s_phase[gslot] + gwrap) & 1u, A.status);
+          const uint16_t* grow = s_gu + (size_t)gslot * n_in * d;
 #pragma unroll
           for (int q = 0; q < CPT; ++q) {
             const int ch = tid + q * FZ_THREADS;
@@ -608,6 +664,7 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
               }
             }
           }
+          if (++gslot == GU) { gslot = 0; ++gwrap; }
         }
       }
       if (tid == 0) FZ_STAMP(0, 2 + rd * 4);
@@ -629,7 +686,7 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
       if (warp == 0) {
         float v = 0.f;
         if (lane < 2 * FZ_NG) {
-#pragma unroll
+#pragma unroll 4
           for (int w = 0; w < FZ_THREADS / 32; ++w) v += red[w * 8 + lane];
         }
         const float u = __shfl_down_sync(0xffffffffu, v, 1);  // lane 2e holds g_e, lane 2e+1 holds u_e
@@ -643,16 +700,15 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
           a = fmaxf(g, 0.f);
           if (A.gated) a *= u * inv_rms;
           if (i < 0) a = 0.f;
-          s_act[(rd & 1) * 4 + e] = a;
-        } else if (!(lane & 1) && e < FZ_NG) {
-          s_act[(rd & 1) * 4 + e] = 0.f;
         }
         // survivors in neuron order -> mailbox of the round, activations -> the queue slots their rows will use
         const unsigned surv = __ballot_sync(0xffffffffu, a != 0.f);
         if (a != 0.f) {
           const int pos = __popc(surv & ((1u << lane) - 1u));
           s_mail[(rd & 3) * 4 + 1 + pos] = i;
-          s_qa[(dq_tail + pos) % DN] = a;
+          int qs = tslot + pos;
+          if (qs >= DN) qs -= DN;
+          s_qa[qs] = a;
         }
         if (lane == 0) {
           s_mail[(rd & 3) * 4] = __popc(surv);
@@ -662,18 +718,21 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
       named_bar_sync(1, FZ_THREADS);
       if (tid == 0) FZ_STAMP(0, 3 + rd * 4);
       // (4) the survivors' rows were queued by the producer in the same order
-      dq_tail += s_mail[(rd & 3) * 4];
-      if (tid == 0) FZ_STAMP(0, 4 + rd * 4);
+      {
+        const int ns = s_mail[(rd & 3) * 4];
+        dq_tail += ns;
+        tslot += ns;
+        if (tslot >= DN) tslot -= DN;
+      }
     }
     if (tid == 0) FZ_STAMP(0, 500);
     if (tid == 0) { FZ_CSTAMP(2); FZ_CVAL(9, dq_tail); }
-    while (dq_head < dq_tail) consume_one();
     used_gu = n_mine;
     used_dn = dq_tail;
     named_bar_sync(1, FZ_THREADS);  // nobody reads the rings any more: the producer may overwrite them
     if (tid == 0) asm volatile("st.release.cta.shared.s32 [%0], %1;" ::"r"(smem_u32(&s_round)), "r"(n_rounds + 1) : "memory");
     // the CTA's whole contribution to its stage, added once (vector reductions; order across CTAs is not fixed)
-    if (dirty) {
+    if (dq_tail > 0) {
       float* dst = A.dacc + (size_t)stage * d;
 #pragma unroll
       for (int q = 0; q < CPT; ++q) {
@@ -694,6 +753,16 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
   grid_barrier(A, G);
   if (tid == 0) FZ_STAMP(1, 1);
   if (tid == 0) FZ_CSTAMP(5);
+  if (tid >= 32 && tid < 36) {  // HBM is idle now: this CTA's share of what the next layer reads first goes to L2
+    const int i = tid - 32;
+    const unsigned bytes = A.pf_bytes[i] & ~15u;
+    const char* p = static_cast<const char*>(A.pf_ptr[i]);
+    if (p && bytes) {
+      const unsigned chunk = ((bytes + G - 1) / G + 127u) & ~127u, off = (unsigned)cta * chunk;
+      if (off < bytes)
+        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p + off), "r"(min(chunk, bytes - off)) : "memory");
+    }
+  }
 
   // ============================ phase 2: partial features x~^(j), per-slice partial latents ==========================
   // The columns of the feature are cut into slices of 32; a CTA owns slices cta, cta + G, ...  For each it rebuilds
@@ -706,10 +775,11 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
   int NTM = E >> 3, REM = E & 7;
   if (REM > 2) { ++NTM; REM = 0; }
   const int EM = NTM * 8;  // evaluations [0, EM) by MMA (rows past K are zero), [EM, E) by scalar code
-  constexpr int XTS = FZ_SL + 4;  // row stride (doubles) of s_xt: the four rows a half-warp reads sit on distinct banks
+  constexpr int XTS = FZ_XBLK;    // row stride (doubles) of s_xt: one block of features per row
   if (A.has_next && cta < nsl)
-    if (!mbar_wait(&s_bar[FZ_BAR_A], s_phase[FZ_BAR_A] & 1u, A.status)) FZ_FAIL(4, 0);  // the A slices have landed
+    mbar_wait(&s_bar[FZ_BAR_A], s_phase[FZ_BAR_A] & 1u, A.status);  // the A slices have landed
   if (tid == 0) FZ_STAMP(1, 10);
+#pragma unroll 1
   for (int a = 0; cta + a * G < nsl; ++a) {
     const int sl = cta + a * G;
     if (a > 0) named_bar_sync(1, FZ_THREADS);  // the previous slice's features are no longer read
@@ -731,7 +801,7 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
       const int rows = max(EM, E);
 #pragma unroll 1
       for (int j = 0; j < rows; ++j) {
-        s_xt[j * XTS + tid] = j <= K ? (double)xv : 0.0;
+        s_xt[j * XTS + fz_feat_pos(tid)] = j <= K ? (double)xv : 0.0;
         if (j <= K && c < d) {
           if (trx) trx[(size_t)j * d + c] = xv;
           if (j == K) xo[c] = xv;  // may alias x: this thread is the only one that still needs x[c]
@@ -742,59 +812,51 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
     named_bar_sync(1, FZ_THREADS);
     if (tid == 0) FZ_STAMP(1, 11);
     if (A.has_next) {
+      // 32 x (K+1) block of features times the slice of A: evaluations [0, EM) on the tensor cores, eight at a time,
+      // evaluations [EM, E) (at most two) with ordinary FMAs on the same weights
       double* part = A.zpart + (size_t)sl * E * RS;
       const uint16_t* As = s_A + (size_t)a * r * FZ_SL;
       const int n_rt = (r + 7) >> 3;
+      const int g = lane >> 2, t4 = lane & 3;
+#pragma unroll 1
       for (int mt = warp; mt < n_rt; mt += FZ_THREADS / 32) {
-        const int row = mt * 8 + (lane >> 2);
-        const uint16_t* arow = As + (size_t)min(row, r - 1) * FZ_SL + (lane & 3);
-        const double* brow = s_xt + (size_t)(lane >> 2) * XTS + (lane & 3);
-        double c[2][2] = {{0.0, 0.0}, {0.0, 0.0}};
+        const int row = mt * 8 + g;
+        double av[8];
+        cvt8_to_double<WD>(*reinterpret_cast<const uint4*>(As + (size_t)min(row, r - 1) * FZ_SL + t4 * 8), av);
+        double c[2][2] = {{0.0, 0.0}, {0.0, 0.0}}, rs[2] = {0.0, 0.0}, bv[8];
 #pragma unroll
-        for (int ks = 0; ks < FZ_SL / 4; ++ks) {
-          const double av = row < r ? w16_to_double<WD>(arow[ks * 4]) : 0.0;
+        for (int nt = 0; nt < 2; ++nt) {
+          if (nt < NTM) {
+            load8d(s_xt + (size_t)(nt * 8 + g) * XTS + t4 * 10, bv);
+            mma_block(c[nt], av, bv);
+          }
+        }
 #pragma unroll
-          for (int nt = 0; nt < 2; ++nt) {
-            if (nt < NTM) {
-              const double bv = brow[(size_t)nt * 8 * XTS + ks * 4];
-              asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};"
-                           : "+d"(c[nt][0]), "+d"(c[nt][1]) : "d"(av), "d"(bv));
-            }
+        for (int rm = 0; rm < 2; ++rm) {
+          if (rm < REM) {
+            load8d(s_xt + (size_t)(EM + rm) * XTS + t4 * 10, bv);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) rs[rm] = fma(av[k], bv[k], rs[rm]);
+            rs[rm] = quad_sum(rs[rm]);
           }
         }
         if (row < r) {
 #pragma unroll
           for (int nt = 0; nt < 2; ++nt) {
-            const int j = nt * 8 + (lane & 3) * 2;
+            const int j = nt * 8 + t4 * 2;
             if (nt < NTM && j <= K) part[(size_t)j * RS + row] = c[nt][0];
             if (nt < NTM && j + 1 <= K) part[(size_t)(j + 1) * RS + row] = c[nt][1];
           }
+          if (t4 < REM) part[(size_t)(EM + t4) * RS + row] = t4 == 0 ? rs[0] : rs[1];
         }
-      }
-      for (int t = tid; t < REM * r; t += FZ_THREADS) {  // remainder evaluations: one thread per (evaluation, row of A)
-        const int jr = t / r, row = t - jr * r, j = EM + jr;
-        const uint16_t* arow = As + (size_t)row * FZ_SL;
-        const double* xr2 = s_xt + (size_t)j * XTS;
-        double acc = 0.0;
-#pragma unroll
-        for (int c0 = 0; c0 < FZ_SL; c0 += 8) {
-          const uint4 w = *reinterpret_cast<const uint4*>(arow + c0);
-          const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            const double2 xx = *reinterpret_cast<const double2*>(xr2 + c0 + 2 * q);
-            acc = fma(w16_to_double<WD>((uint16_t)(ww[q] & 0xffffu)), xx.x, acc);
-            acc = fma(w16_to_double<WD>((uint16_t)(ww[q] >> 16)), xx.y, acc);
-          }
-        }
-        part[(size_t)j * RS + row] = acc;
       }
       if (tid == 0) FZ_STAMP(1, 12);
       if (warp == FZ_THREADS / 32 - 1) {  // partial sums of squares of the slice, one evaluation per lane
+#pragma unroll 1
         for (int j = lane; j <= K; j += 32) {
           double sq = 0.0;
 #pragma unroll 8
-          for (int c = 0; c < FZ_SL; ++c) { const double v = s_xt[j * XTS + c]; sq = fma(v, v, sq); }
+          for (int c = 0; c < FZ_SL; ++c) { const double v = s_xt[j * XTS + fz_feat_pos(c)]; sq = fma(v, v, sq); }
           part[(size_t)j * RS + r] = sq;
         }
       }
@@ -809,26 +871,33 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
     grid_barrier(A, G);
     if (tid == 0) FZ_STAMP(1, 3);
 
-    // ============================ phase 2b: sum of the slices' partials, one value per warp ===========================
-    // Lane l adds slices l, l + 32, ... in order, the lanes are combined by a butterfly: the result does not depend on
-    // which warp of which CTA computes it.
+    // ============================ phase 2b: sum of the slices' partials, four values per warp =========================
+    // A warp takes four consecutive values (one 32-byte sector per slice); lane (q, v), q = lane / 4, adds the slices
+    // q, q + 8, ... of value v in order, the eight partial sums are combined by a butterfly: the result does not depend on
+    // which warp of which CTA computes it, and every sector fetched is used whole.
     {
       const int V = E * RS;
-      for (int v = cta * (FZ_THREADS / 32) + warp; v < V; v += G * (FZ_THREADS / 32)) {
+      const int q8 = lane >> 2, v4 = lane & 3;
+#pragma unroll 1
+      for (int v0 = (warp * G + cta) * 4; v0 < V; v0 += G * (FZ_THREADS / 32) * 4) {  // tasks dealt round-robin over the CTAs
+        const int v = v0 + v4;
+        const double* zp = A.zpart + min(v, V - 1);
         double acc = 0.0;
-        const double* zp = A.zpart + v;
-        for (int s0 = 0; s0 < nsl; s0 += 128) {  // four loads in flight per lane
-          double q[4];
+#pragma unroll 1
+        for (int s0 = 0; s0 < nsl; s0 += 64) {  // eight loads in flight per lane
+          double q[8];
 #pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            const int s2 = s0 + u * 32 + lane;
+          for (int u = 0; u < 8; ++u) {
+            const int s2 = s0 + u * 8 + q8;
             q[u] = s2 < nsl ? __ldcg(zp + (size_t)s2 * V) : 0.0;
           }
-          acc += (q[0] + q[1]) + (q[2] + q[3]);
-        }
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-        if (lane == 0) {
+          for (int u = 0; u < 8; ++u) acc += q[u];
+        }
+        acc += __shfl_xor_sync(0xffffffffu, acc, 4);
+        acc += __shfl_xor_sync(0xffffffffu, acc, 8);
+        acc += __shfl_xor_sync(0xffffffffu, acc, 16);
+        if (q8 == 0 && v < V) {
           const int j = v / RS, row = v - j * RS;
           if (row < r) A.z[(size_t)j * r + row] = acc;
           else A.sumsq[j] = acc;
@@ -841,7 +910,7 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
     if (tid == 0) FZ_STAMP(1, 8);
 
     // ============================ phase 3: scores of this CTA's neurons, every evaluation =============================
-    double* s_zs = reinterpret_cast<double*>(smem + lay.zs_off);            // [max(EM, E)][r + FZ_ZPAD], un-normalised
+    double* s_zs = reinterpret_cast<double*>(smem + lay.zs_off);            // [max(EM, E)][fz_feat_stride(r)], un-normalised, blocked
     double* s_part = reinterpret_cast<double*>(smem + lay.part_off);        // [FZ_KS][FZ_EPAD][per8]
     double* s_own = reinterpret_cast<double*>(smem + lay.own_off);          // [K+1][per]
     uint16_t* s_bin = reinterpret_cast<uint16_t*>(smem + lay.bin_off);      // [K+1][per]
@@ -851,72 +920,107 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
     const double brange = bin_hi - bin_lo;
     const double bscale = (brange > 0.0 && brange < INF) ? (double)FZ_NB / brange : 0.0;
     const int keff = min(A.k_next, Fn);
-    const int RSB = r + FZ_BPAD, RSZ = r + FZ_ZPAD;
+    const int RSB = fz_brow_stride(r), RSZ = fz_feat_stride(r);
+    const int nblk = (r + 31) >> 5, cpad_b = nblk * 32;
     const int per8 = (per + 7) & ~7;
 
-    // latents of every evaluation and 1 / rms of every feature
+    // latents of every evaluation (un-normalised, in the blocked order the tensor-core loads want) and 1 / rms of every
+    // feature; eight loads in flight per thread
     {
       const double* zg = A.z;
-      const int nz = max(EM, E) * r;
-      for (int t0 = 0; t0 < nz; t0 += 4 * FZ_THREADS) {  // four loads in flight per thread
-        double q[4];
+      const int nz = E * r;
+      const unsigned rmagic = 0xffffffffu / (unsigned)r + 1u;  // t / r == umulhi(t, rmagic) for t < 2^16
+#pragma unroll 1
+      for (int t0 = 0; t0 < nz; t0 += 8 * FZ_THREADS) {
+        double q[8];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < 8; ++u) {
           const int t = t0 + u * FZ_THREADS + tid;
-          q[u] = (t < E * r) ? __ldcg(zg + t) : 0.0;  // z is [evaluation][r], contiguous
+          q[u] = (t < nz) ? __ldcg(zg + t) : 0.0;  // z is [evaluation][r], contiguous
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < 8; ++u) {
           const int t = t0 + u * FZ_THREADS + tid;
-          if (t < nz) { const int e = t / r; s_zs[e * RSZ + (t - e * r)] = q[u]; }
+          if (t < nz) {
+            const int e = (int)__umulhi((unsigned)t, rmagic);
+            s_zs[e * RSZ + fz_feat_pos(t - e * r)] = q[u];
+          }
         }
+      }
+      // rows of a padded tile past K, and the columns past r of a last partial block, must read as zero
+      const int rows = max(EM, E), cpad = nblk * 32;
+#pragma unroll 1
+      for (int t = tid; t < (rows - E) * cpad; t += FZ_THREADS) s_zs[(E + t / cpad) * RSZ + fz_feat_pos(t % cpad)] = 0.0;
+      if (cpad > r) {
+#pragma unroll 1
+        for (int t = tid; t < E * (cpad - r); t += FZ_THREADS)
+          s_zs[(t / (cpad - r)) * RSZ + fz_feat_pos(r + t % (cpad - r))] = 0.0;
       }
     }
     if (tid < FZ_EPAD)
-      s_inv[tid] = (tid <= K && A.norm_n == 0) ? 1.0 / sqrt(__ldcg(&A.sumsq[tid]) / (double)d + (double)A.eps_n) : 1.0;
-    if (!mbar_wait(&s_bar[FZ_BAR_B], s_phase[FZ_BAR_B] & 1u, A.status)) FZ_FAIL(5, 0);  // the rows of B^T have landed
+      s_inv[tid] = (tid <= K && A.norm_n == 0) ? fz_rsqrt(fma(__ldcg(&A.sumsq[tid]), A.inv_d, (double)A.eps_n)) : 1.0;
+    mbar_wait(&s_bar[FZ_BAR_B], s_phase[FZ_BAR_B] & 1u, A.status);  // the rows of B^T have landed
+    if (cpad_b > r) {  // (only when r is not a multiple of 32) the tail of the last block of every row reads as zero
+#pragma unroll 1
+      for (int t = tid; t < per8 * (cpad_b - r); t += FZ_THREADS)
+        s_B[(size_t)(t / (cpad_b - r)) * RSB + r + t % (cpad_b - r)] = 0;
+    }
     named_bar_sync(1, FZ_THREADS);
     if (tid == 0) FZ_STAMP(1, 40);
 
-    // C[neuron][evaluation] = B^T rows x latents.  A task is a group of neurons times one of FZ_KS column ranges; the
-    // column ranges are added afterwards in a fixed order.  Within one evaluation every neuron's score is accumulated
-    // over the columns in the same order whatever its position in a tile, so equal predictor rows give bit-equal scores.
+    // C[neuron][evaluation] = B^T rows x latents.  A task is a tile of eight neurons times one of FZ_KS ranges of
+    // 32-column blocks; the ranges are added afterwards in a fixed order.  Evaluations [0, EM) go through the tensor
+    // cores, evaluations [EM, E) (at most two) through ordinary FMAs on the same converted weights.  Within one evaluation
+    // every neuron's score is accumulated in the same order whatever its position in a tile, so equal predictor rows give
+    // bit-equal scores.
     const int n_mt = (n_own + 7) >> 3;
-    const int kchunk = ((r >> 3) + FZ_KS - 1) / FZ_KS * 8;
-    const int n_mma = NTM > 0 ? n_mt * FZ_KS : 0;
-    const int n_blk = (n_own + 31) >> 5;
-    const int n_task = n_mma + n_blk * REM * FZ_KS;
+    const int bchunk = (nblk + FZ_KS - 1) / FZ_KS;  // blocks per range
     if (lane == 0) FZ_STAMP(1, 400 + warp * 4);
-    for (int task = warp; task < n_task; task += FZ_THREADS / 32) {
+#pragma unroll 1
+    for (int task = warp; task < n_mt * FZ_KS; task += FZ_THREADS / 32) {
       if (lane == 0 && task == warp + 16) FZ_STAMP(1, 401 + warp * 4);
-      if (task < n_mma) {  // eight neurons x the MMA evaluations
-        const int ks = task / n_mt, mt = task - ks * n_mt;
-        const int k_lo = ks * kchunk, k_hi = min(r, k_lo + kchunk);
-        const uint16_t* arow = s_B + (size_t)(mt * 8 + (lane >> 2)) * RSB + (lane & 3);
-        const double* brow = s_zs + (size_t)(lane >> 2) * RSZ + (lane & 3);
-        double* outp = s_part + (size_t)ks * FZ_EPAD * per8 + mt * 8 + (lane >> 2);
-        if (NTM == 1) score_task_mma<WD, 1>(arow, brow, RSZ, k_lo, k_hi, outp, per8, lane);  // (K + 1 <= 17: at most two tiles)
-        else score_task_mma<WD, 2>(arow, brow, RSZ, k_lo, k_hi, outp, per8, lane);
-      } else {  // thirty-two neurons (one per lane) x one remainder evaluation
-        const int t2 = task - n_mma;
-        const int ks = t2 % FZ_KS, bj = t2 / FZ_KS, blk = bj % n_blk, j = EM + bj / n_blk;
-        const int k_lo = ks * kchunk, k_hi = min(r, k_lo + kchunk);
-        const int li = min(blk * 32 + lane, per8 - 1);  // lanes past the last neuron repeat a valid row; not stored
-        const uint16_t* brw = s_B + (size_t)li * RSB;
-        const double* zr = s_zs + (size_t)j * RSZ;
-        double acc = 0.0;
-#pragma unroll 2
-        for (int k0 = k_lo; k0 < k_hi; k0 += 8) {
-          const uint4 w = *reinterpret_cast<const uint4*>(brw + k0);
-          const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+      const int ks = task / n_mt, mt = task - ks * n_mt;
+      const int b_lo = ks * bchunk, b_hi = min(nblk, b_lo + bchunk);
+      const int g = lane >> 2, t4 = lane & 3;
+      const uint16_t* arow = s_B + (size_t)(mt * 8 + g) * RSB + t4 * 8;
+      const double* zrow = s_zs + (size_t)g * RSZ + t4 * 10;      // MMA tiles: evaluation nt * 8 + g
+      const double* zrem = s_zs + (size_t)EM * RSZ + t4 * 10;     // remainder evaluations EM, EM + 1
+      double c[2][2] = {{0.0, 0.0}, {0.0, 0.0}}, rs[2] = {0.0, 0.0};
+#pragma unroll 1
+      for (int b = b_lo; b < b_hi; ++b) {
+        double av[8], bv[8];
+        cvt8_to_double<WD>(*reinterpret_cast<const uint4*>(arow + b * 32), av);
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            const double2 zz = *reinterpret_cast<const double2*>(zr + k0 + 2 * q);
-            acc = fma(w16_to_double<WD>((uint16_t)(ww[q] & 0xffffu)), zz.x, acc);
-            acc = fma(w16_to_double<WD>((uint16_t)(ww[q] >> 16)), zz.y, acc);
+        for (int nt = 0; nt < 2; ++nt) {
+          if (nt < NTM) {
+            load8d(zrow + (size_t)nt * 8 * RSZ + b * FZ_XBLK, bv);
+            mma_block(c[nt], av, bv);
           }
         }
-        if (blk * 32 + lane < n_own) s_part[((size_t)ks * FZ_EPAD + j) * per8 + blk * 32 + lane] = acc;
+#pragma unroll
+        for (int rm = 0; rm < 2; ++rm) {
+          if (rm < REM) {
+            load8d(zrem + (size_t)rm * RSZ + b * FZ_XBLK, bv);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) rs[rm] = fma(av[k], bv[k], rs[rm]);
+          }
+        }
+      }
+      double* outp = s_part + (size_t)ks * FZ_EPAD * per8 + mt * 8 + g;
+#pragma unroll
+      for (int nt = 0; nt < 2; ++nt) {
+        if (nt < NTM) {
+          const int j = nt * 8 + t4 * 2;
+          outp[(size_t)j * per8] = c[nt][0];
+          outp[(size_t)(j + 1) * per8] = c[nt][1];
+        }
+      }
+#pragma unroll
+      for (int rm = 0; rm < 2; ++rm) {
+        if (rm < REM) {
+          const double v = quad_sum(rs[rm]);
+          if (t4 == 0) outp[(size_t)(EM + rm) * per8] = v;
+        }
       }
     }
     if (lane == 0) FZ_STAMP(1, 402 + warp * 4);
@@ -926,6 +1030,7 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
     // time so that their atomics are in flight together; the coarse counts of the CTA are summed in shared memory first
     // (they are hot addresses for the whole grid)
     {
+#pragma unroll 1
       for (int t = tid; t < (K + 1) * FZ_NC; t += FZ_THREADS) s_ccnt[t] = 0u;
       if (tid < FZ_MAXE) s_nsel[tid] = 0u;
       named_bar_sync(1, FZ_THREADS);
@@ -936,6 +1041,7 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
       unsigned* const cnt_all = A.cnt;
       uint4* const bent = A.bent;
       uint4* const oent = A.oent;
+#pragma unroll 1
       for (int t0 = 0; t0 < n_ent; t0 += 2 * FZ_THREADS) {
         int jj[2], ll[2], bb[2];
         unsigned slot[2];
@@ -988,11 +1094,13 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
       }
       if (lane == 0) { s_kmm[warp] = kmin; s_kmm[16 + warp] = kmax; }
       named_bar_sync(1, FZ_THREADS);
+#pragma unroll 1
       for (int t = tid; t < (K + 1) * FZ_NC; t += FZ_THREADS) {
         const unsigned v = s_ccnt[t];
         if (v) atomicAdd(&A.cnt[(size_t)(t / FZ_NC) * FZ_CNT_STRIDE + FZ_NB + (t % FZ_NC)], v);
       }
       if (tid == 0) {  // observed score range of the final evaluation: one pair of atomics per CTA
+#pragma unroll 1
         for (int w = 1; w < 16; ++w) { kmin = min(kmin, s_kmm[w]); kmax = max(kmax, s_kmm[16 + w]); }
         if (kmin <= kmax) {
           atomicMin(&A.range_obs[0], kmin);
@@ -1013,6 +1121,7 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
     // memory every neuron's membership is decided locally: bins before the cut bin are in, bins after it are out, the
     // cut bin is split by one comparison.  Exact ranks (bucket comparisons) are needed only for the final selection.
     constexpr int FPC = FZ_NB / FZ_NC;  // fine bins per coarse bin
+#pragma unroll 1
     for (int j = warp; j <= K; j += FZ_THREADS / 32) {
       const unsigned* cnt = A.cnt + (size_t)j * FZ_CNT_STRIDE;
       const unsigned c0 = __ldcg(&cnt[FZ_NB + lane * 2]), c1 = __ldcg(&cnt[FZ_NB + lane * 2 + 1]);
@@ -1090,6 +1199,7 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
       // intermediate evaluations: membership only (bins before the cut bin are in, the cut bin is split by the threshold)
       uint32_t* const trm = A.tr_masks;
       const int nwn = (Fn + 31) >> 5;
+#pragma unroll 1
       for (int t = tid; t < K * n_own; t += FZ_THREADS) {
         const int j = t / n_own, li = t - j * n_own, i = i_lo + li;
         const int bb = s_bin[(size_t)j * per + li];
@@ -1127,6 +1237,7 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
       const uint4* const bent = A.bent + (size_t)j * FZ_NB * FZ_CAPB;
       unsigned found = 0;
       // task t goes to CTA t % G, warp (t / G) % 16: spread over the whole grid, at most a few per warp
+#pragma unroll 1
       for (int task = cta + warp * G; task < n_task; task += G * (FZ_THREADS / 32)) {
         const int fbq = task * 2, cb = fbq / FPC;  // first fine bin of the task, its coarse bin
         // fine counts of the coarse bin (two per lane) and their exclusive prefix
@@ -1173,10 +1284,12 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
     if (lane == 0) FZ_STAMP(1, 103 + warp * 4);
     named_bar_sync(1, FZ_THREADS);
     // refined-set sizes: every evaluation must have selected exactly keff neurons (checked on the device)
+#pragma unroll 1
     for (int j = tid; j <= K; j += FZ_THREADS)
       if (s_nsel[j]) atomicAdd(&A.nsel[j], s_nsel[j]);
     if (cta == 0 && tid == 0) {
       if (A.tr_counts)
+#pragma unroll 1
         for (int j = 0; j <= K; ++j) A.tr_counts[j] = keff;
       *A.next_count = min(keff, A.next_cap);
       if (keff > A.next_cap) set_status(A.status, ST_CAPACITY);
@@ -1221,8 +1334,10 @@ __device__ inline void fused_update_range(const FusedArgs& A) {
 // self-check of the refined-set sizes and the range update.  The caller guarantees that every CTA is done with the layer.
 __device__ inline void fused_clean(const FusedArgs& A, int part, int parts) {
   const int tid = threadIdx.x;
+#pragma unroll 1
   for (int t = part * FZ_THREADS + tid; t < A.K * A.d; t += parts * FZ_THREADS) A.dacc[t] = 0.f;
   if (A.has_next) {
+#pragma unroll 1
     for (int t = part * FZ_THREADS + tid; t < (A.K + 1) * FZ_CNT_STRIDE; t += parts * FZ_THREADS) A.cnt[t] = 0u;
     if (part == 0) {
       if (tid <= A.K) {  // self-check: every refined set has exactly min(k_next, d_ff) members
@@ -1239,7 +1354,7 @@ template <int WD, int CPT>
 __global__ void __launch_bounds__(FZ_BLOCK, 1) ls_fused_step_kernel(const __grid_constant__ FusedArgs A) {
   extern __shared__ __align__(128) unsigned char smem[];
   __shared__ FusedShared sh;
-  fused_layer<WD, CPT>(A, smem, sh, true);
+  fused_layer<WD, CPT>(A, smem, sh, true, -1);
   if (threadIdx.x >= FZ_THREADS) return;  // the producer warp is done; an exited warp counts as arrived at block barriers
   named_bar_sync(1, FZ_THREADS);
   if (threadIdx.x == 0) {
@@ -1277,8 +1392,11 @@ __global__ void __launch_bounds__(FZ_BLOCK, 1)
   __shared__ FusedShared sh;
   const int G = gridDim.x, cta = blockIdx.x, tid = threadIdx.x;
   constexpr int NW = sizeof(FusedArgs) / 4;
+  int known_count = -1;
+#pragma unroll 1
   for (int n = 0; n < n_layers; ++n) {
     if (tid == 0) FZ_STAMP(1, 24);
+#pragma unroll 1
     for (int w = tid; w < NW; w += FZ_BLOCK) reinterpret_cast<uint32_t*>(&sh.args)[w] = reinterpret_cast<const uint32_t*>(&g_args[n])[w];
     __syncthreads();
     if (tid == 0) FZ_STAMP(1, 25);
@@ -1295,14 +1413,17 @@ __global__ void __launch_bounds__(FZ_BLOCK, 1)
     __syncthreads();
     const FusedArgs& A = sh.args;
     if (cta == G - 1 && C.tr_x && tid < FZ_THREADS) {  // what enters this layer (x_out may overwrite x)
+#pragma unroll 1
       for (int c = tid; c < A.d; c += FZ_THREADS) C.tr_x[(size_t)n * A.d + c] = __ldcg(A.x + c);
       if (C.tr_sel) {
         const int cnt = max(0, min(__ldcg(A.sel_count), min(A.sel_cap, C.tr_cap)));
+#pragma unroll 1
         for (int t = tid; t < cnt; t += FZ_THREADS) C.tr_sel[(size_t)n * C.tr_cap + t] = __ldcg(A.sel_idx + t);
         if (tid == 0) C.tr_cnt[n] = cnt;
       }
     }
-    fused_layer<WD, CPT>(A, smem, sh, n == 0);
+    fused_layer<WD, CPT>(A, smem, sh, n == 0, known_count);
+    known_count = A.has_next ? min(min(A.k_next, A.Fn), A.next_cap) : -1;  // what this layer wrote to *next_count
     if (tid < FZ_THREADS) {
       if (n > 0) fused_clean(sh.prev, cta, G);  // nobody touches the previous layer's scratch any more
       grid_barrier(A, G);                       // layer boundary: x_out and the refined selection are visible to all
@@ -1316,6 +1437,7 @@ __global__ void __launch_bounds__(FZ_BLOCK, 1)
 #endif
     }
     __syncthreads();
+#pragma unroll 1
     for (int w = tid; w < NW; w += FZ_BLOCK) reinterpret_cast<uint32_t*>(&sh.prev)[w] = reinterpret_cast<const uint32_t*>(&sh.args)[w];
     __syncthreads();
   }
@@ -1323,9 +1445,11 @@ __global__ void __launch_bounds__(FZ_BLOCK, 1)
     const FusedArgs& A = sh.prev;  // the last layer; every CTA is past its final barrier
     fused_clean(A, cta, G);
     if (cta == G - 1 && C.tr_x) {
+#pragma unroll 1
       for (int c = tid; c < A.d; c += FZ_THREADS) C.tr_x[(size_t)n_layers * A.d + c] = __ldcg(A.x_out + c);
       if (C.tr_sel && A.has_next) {
         const int cnt = max(0, min(__ldcg(A.next_count), min(A.next_cap, C.tr_cap)));
+#pragma unroll 1
         for (int t = tid; t < cnt; t += FZ_THREADS) C.tr_sel[(size_t)n_layers * C.tr_cap + t] = __ldcg(A.next_idx + t);
         if (tid == 0) C.tr_cnt[n_layers] = cnt;
       }
