@@ -165,6 +165,7 @@ __device__ __noinline__ bool fz_wait_round(int* s_round, int want, int* status) 
     int v;
     asm volatile("ld.acquire.cta.shared.s32 %0, [%1];" : "=r"(v) : "r"((uint32_t)__cvta_generic_to_shared(s_round)) : "memory");
     if (v >= want) return true;
+    __nanosleep(128);  // the poll shares an instruction scheduler with four compute warps: leave them the issue slots
   } while (clock64() - t0 < FZ_SPIN_CYCLES);
   set_status(status, ST_TIMEOUT);
   return false;
@@ -496,6 +497,8 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
       int i = __ldcg(A.sel_idx + first + t * gsize);
       if ((unsigned)i >= (unsigned)A.F) { set_status(A.status, ST_BAD_INDEX); i = -1; }
       s_myidx[t] = i;
+      // the gate bias follows at once: a small load issued after the ring's bulk copies would queue behind all of them
+      s_mybias[t] = (A.b_gate && i >= 0) ? A.b_gate[i] : 0.f;
     }
     float xr[CPT][8];
     {
@@ -586,14 +589,6 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
       return;  // an exited warp counts as arrived at every later block barrier
     }
 
-#pragma unroll 1
-    for (int t = tid; t < n_mine; t += FZ_THREADS) {
-      const int i = s_myidx[t];
-      s_mybias[t] = (A.b_gate && i >= 0) ? A.b_gate[i] : 0.f;
-    }
-    if (A.has_next)
-#pragma unroll 1
-      for (int li = tid; li < n_own; li += FZ_THREADS) s_pc[li] = A.pc ? A.pc[i_lo + li] : 0.f;
     float inv_rms = 1.0f;
     if (A.norm == 0) {
       double tot = 0.0;
@@ -753,6 +748,10 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
   grid_barrier(A, G);
   if (tid == 0) FZ_STAMP(1, 1);
   if (tid == 0) FZ_CSTAMP(5);
+  if (A.has_next) {  // offsets of this CTA's share of the next layer's predictor (needed in the score phase)
+#pragma unroll 1
+    for (int li = tid; li < n_own; li += FZ_THREADS) s_pc[li] = A.pc ? A.pc[i_lo + li] : 0.f;
+  }
   if (tid >= 32 && tid < 36) {  // HBM is idle now: this CTA's share of what the next layer reads first goes to L2
     const int i = tid - 32;
     const unsigned bytes = A.pf_bytes[i] & ~15u;
@@ -911,7 +910,7 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
 
     // ============================ phase 3: scores of this CTA's neurons, every evaluation =============================
     double* s_zs = reinterpret_cast<double*>(smem + lay.zs_off);            // [max(EM, E)][fz_feat_stride(r)], un-normalised, blocked
-    double* s_part = reinterpret_cast<double*>(smem + lay.part_off);        // [FZ_KS][FZ_EPAD][per8]
+    double* s_part = reinterpret_cast<double*>(smem + lay.part_off);        // [KSd][prow][per8], KSd * prow <= FZ_KS * FZ_EPAD
     double* s_own = reinterpret_cast<double*>(smem + lay.own_off);          // [K+1][per]
     uint16_t* s_bin = reinterpret_cast<uint16_t*>(smem + lay.bin_off);      // [K+1][per]
     unsigned* s_coarse = reinterpret_cast<unsigned*>(smem + lay.coarse_off);  // [K+1][FZ_NC + 1] exclusive prefix
@@ -974,10 +973,12 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
     // every neuron's score is accumulated in the same order whatever its position in a tile, so equal predictor rows give
     // bit-equal scores.
     const int n_mt = (n_own + 7) >> 3;
-    const int bchunk = (nblk + FZ_KS - 1) / FZ_KS;  // blocks per range
+    const int prow = max(EM, E);                                   // rows of a range's partial sums
+    const int KSd = min(FZ_KS, (FZ_KS * FZ_EPAD) / prow);         // ranges (fewer if the partial sums lack room)
+    const int bchunk = (nblk + KSd - 1) / KSd;                     // blocks per range
     if (lane == 0) FZ_STAMP(1, 400 + warp * 4);
 #pragma unroll 1
-    for (int task = warp; task < n_mt * FZ_KS; task += FZ_THREADS / 32) {
+    for (int task = warp; task < n_mt * KSd; task += FZ_THREADS / 32) {
       if (lane == 0 && task == warp + 16) FZ_STAMP(1, 401 + warp * 4);
       const int ks = task / n_mt, mt = task - ks * n_mt;
       const int b_lo = ks * bchunk, b_hi = min(nblk, b_lo + bchunk);
@@ -1006,7 +1007,7 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
           }
         }
       }
-      double* outp = s_part + (size_t)ks * FZ_EPAD * per8 + mt * 8 + g;
+      double* outp = s_part + (size_t)ks * prow * per8 + mt * 8 + g;
 #pragma unroll
       for (int nt = 0; nt < 2; ++nt) {
         if (nt < NTM) {
@@ -1054,8 +1055,8 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
           if (t < n_ent) {
             const int j = t / n_own, li = t - j * n_own;
             double v = 0.0;
-#pragma unroll
-            for (int ks = 0; ks < FZ_KS; ++ks) v += s_part[((size_t)ks * FZ_EPAD + j) * per8 + li];
+#pragma unroll 4
+            for (int ks = 0; ks < KSd; ++ks) v += s_part[((size_t)ks * prow + j) * per8 + li];
             v = canonical_score(v * s_inv[j] + (double)s_pc[li]);
             const double sc = fmin(fmax(v, -1.7976931348623157e308), 1.7976931348623157e308);
             int b = (int)((bin_hi - sc) * bscale);
