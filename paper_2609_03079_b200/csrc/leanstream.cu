@@ -210,10 +210,10 @@ struct DeviceScratch {
   unsigned* ctr = nullptr;            // fin, (pad), barrier counter (64-bit)
   double* z = nullptr;                // [FZ_MAXE][1024] latents, then [FZ_MAXE] sums of squares
   double* zpart = nullptr;            // [512 slices][FZ_MAXE][1025] per-slice partial latents
-  unsigned* cnt = nullptr;            // [FZ_MAXE][FZ_CNT_STRIDE], zero between launches
-  uint4* bent = nullptr;              // [FZ_MAXE][FZ_NB * FZ_CAPB] bucket entries
-  uint4* oent = nullptr;              // [FZ_MAXE][32768] overflow entries
-  unsigned* nsel = nullptr;           // [FZ_MAXE] refined-set sizes, zero between launches
+  double* sc = nullptr;               // [FZ_MAXE][32768] final scores of every evaluation
+  uint16_t* sb = nullptr;             // [FZ_MAXE][32768] their fine bins
+  uint4* bent = nullptr;              // [32768] members of the final evaluation, grouped by bin
+  unsigned long long* kmm = nullptr;  // [2 x 1024] per-CTA smallest / largest key of the final evaluation
   bool ready = false;
 };
 constexpr int kScratchMaxD = 16384, kScratchMaxR = 1024, kScratchMaxF = 32768;
@@ -230,14 +230,12 @@ int32_t device_scratch(int dev, DeviceScratch** out) {
     LS_TRY(dalloc(&S.ctr, (size_t)8));
     LS_TRY(dalloc(&S.z, NE * kScratchMaxR + NE));
     LS_TRY(dalloc(&S.zpart, (size_t)(kScratchMaxD / ls::FZ_SL) * NE * (kScratchMaxR + 1)));
-    LS_TRY(dalloc(&S.cnt, 2 * NE * ls::FZ_CNT_STRIDE));
-    LS_TRY(dalloc(&S.bent, NE * ls::FZ_NB * ls::FZ_CAPB));
-    LS_TRY(dalloc(&S.oent, NE * kScratchMaxF));
-    LS_TRY(dalloc(&S.nsel, 2 * NE));
-    LS_CUDA(cudaMemset(S.nsel, 0, 2 * NE * sizeof(unsigned)));
+    LS_TRY(dalloc(&S.sc, NE * kScratchMaxF));
+    LS_TRY(dalloc(&S.sb, NE * kScratchMaxF));
+    LS_TRY(dalloc(&S.bent, (size_t)kScratchMaxF));
+    LS_TRY(dalloc(&S.kmm, (size_t)2048));
     LS_CUDA(cudaMemset(S.dacc, 0, (size_t)2 * ls::FZ_MAXK * kScratchMaxD * sizeof(float)));
     LS_CUDA(cudaMemset(S.ctr, 0, 8 * sizeof(unsigned)));
-    LS_CUDA(cudaMemset(S.cnt, 0, 2 * NE * ls::FZ_CNT_STRIDE * sizeof(unsigned)));
     LS_CUDA(cudaMemset(S.z, 0, (NE * kScratchMaxR + NE) * sizeof(double)));
     S.ready = true;
   }
@@ -333,19 +331,19 @@ int32_t create_impl(const ls_layer_desc* D, ls_layer* L) {
 // Shared-memory plan of the fused kernel: as many ring stages as fit beside the predictor operands.
 bool fused_plan(const ls_layer* L, const ls_layer* next, ls::FusedSmemLayout* out) {
   const size_t budget = 218 * 1024;  // dynamic part; the kernel also has a few KB of static shared memory
-  const int n_in = L->gated ? 2 : 1;
   const int r = next ? next->r : 0, Fn = next ? next->F : 0, hn = next ? 1 : 0;
-  // The gate/up ring wants two rounds in flight and the down ring as many rows as memory latency covers; a down row is
-  // half (gated) or all of a gate/up slot, so depth is traded between the two rings at that rate.  The A slices keep a
-  // place of their own (they can then arrive while the rings are still busy) unless that costs the rings their depth.
+  // First ring (first row of every bundle): as deep as fits, ideally all of a CTA's neurons at once.  Second ring (the
+  // rest of a survivor's bundle): a few slots; the producer refills them as survivors are consumed.  The A slices keep a
+  // place of their own (they can then arrive while the rings are still busy) unless that costs the first ring its depth.
+  const int g2s[3] = {5, 6, 4};
   for (int alias = 0; alias <= 1; ++alias) {
-    for (int gu = ls::FZ_MAX_DEPTH; gu >= ls::FZ_NG + 1; --gu) {
-      for (int dn = ls::FZ_MAX_DEPTH; dn >= ls::FZ_NG + 1; --dn) {
-        const ls::FusedSmemLayout lay = ls::fused_layout(L->d, n_in, r, Fn, L->sm_count, hn, gu, dn, alias);
-        if (lay.total <= budget && (alias == 1 || (gu >= 6 && dn >= 6))) {
-          if (out) *out = lay;
-          return true;
-        }
+    for (int c = 0; c < 3; ++c) {
+      for (int g1 = ls::FZ_MAX_G1; g1 >= ls::FZ_NG + 1; --g1) {
+        const ls::FusedSmemLayout lay = ls::fused_layout(L->d, L->n_mat, r, Fn, L->sm_count, hn, g1, g2s[c], alias);
+        if (lay.total > budget) continue;
+        if (alias == 0 && g1 < 8) break;  // too shallow with the A slices apart: try the next arrangement
+        if (out) *out = lay;
+        return true;
       }
     }
   }
@@ -393,13 +391,16 @@ int32_t fused_args(ls_layer* L, ls_layer* next, const float* d_x, float* d_x_out
     a.At_sl = next->pred_at_sl; a.Bt = next->pred_bt; a.pc = next->pred_c;
     a.r = next->r; a.Fn = next->F; a.norm_n = next->norm; a.eps_n = next->eps; a.k_next = k_next;
     a.z = S->z; a.sumsq = S->z + (size_t)ls::FZ_MAXE * next->r; a.zpart = S->zpart; a.range = next->fz_range;
-    a.cnt = S->cnt + (size_t)parity * ls::FZ_MAXE * ls::FZ_CNT_STRIDE; a.bent = S->bent; a.oent = S->oent;
-    a.range_obs = next->fz_range_obs; a.nsel = S->nsel + (size_t)parity * ls::FZ_MAXE;
+    a.sc = S->sc; a.sb = S->sb; a.bent = S->bent; a.kmm = S->kmm;
     if (sel_next) {
       a.next_idx = sel_next->idx; a.next_count = sel_next->count; a.next_mask = sel_next->mask; a.next_scores = sel_next->scores;
       a.next_cap = sel_next->cap;
     }
     a.next_prio = next->prio;
+    if (next->cache_rows == 0 && (next->d * 2) % 16 == 0) {  // first rows of the next layer's bundles: speculative L2 prefetch
+      a.spec_ptr = reinterpret_cast<const char*>(next->bundles);
+      a.spec_stride = (unsigned long long)next->n_mat * next->d * 2ull; a.spec_bytes = (unsigned)next->d * 2u;
+    }
   }
   ls::FusedSmemLayout lay{};
   if (!fused_plan(L, next, &lay)) return fail(LS_ERR_STATE, "fused step: shared memory plan failed");
@@ -647,6 +648,9 @@ int32_t ls_stack_create(ls_layer* const* layers, int32_t n_layers, ls_stack** ou
     h[n].pf_ptr[1] = L1->b_gate;          h[n].pf_bytes[1] = L1->b_gate ? (unsigned)(L1->F * sizeof(float)) : 0u;
     h[n].pf_ptr[2] = L1->b_down;          h[n].pf_bytes[2] = L1->b_down ? (unsigned)(L1->d * sizeof(float)) : 0u;
     h[n].pf_ptr[3] = L2->pred_c;          h[n].pf_bytes[3] = L2->pred_c ? (unsigned)(L2->F * sizeof(float)) : 0u;
+    h[n].pg_ptr[0] = L1->bundles; h[n].pg_bytes[0] = (unsigned long long)L1->nslots * L1->n_mat * L1->d * 2ull;
+    h[n].pg_ptr[1] = L2->pred_at_sl; h[n].pg_bytes[1] = (unsigned long long)((L2->d + ls::FZ_SL - 1) / ls::FZ_SL) * L2->r * ls::FZ_SL * 2ull;
+    h[n].pg_ptr[2] = L2->pred_bt; h[n].pg_bytes[2] = (unsigned long long)L2->F * L2->r * 2ull;
   }
   if (cudaMemcpy(S->d_args, h.data(), sizeof(ls::FusedArgs) * n_layers, cudaMemcpyHostToDevice) != cudaSuccess)
     return cleanup(fail(LS_ERR_CUDA, "ls_stack_create: upload of the layer arguments failed"));

@@ -30,13 +30,13 @@ constexpr int FZ_THREADS = 512;        // compute threads (16 warps)
 constexpr int FZ_BLOCK = FZ_THREADS + 32;  // plus the producer warp
 constexpr int FZ_NG = 3;          // neurons processed per round
 constexpr int FZ_NB = 4096;       // fine score bins per evaluation
-constexpr int FZ_NC = 64;         // coarse bins (FZ_NB / FZ_NC fine bins each)
-constexpr int FZ_CNT_STRIDE = FZ_NB + FZ_NC + 4;  // fine counts, coarse counts, overflow count (+ padding to 16 bytes)
-constexpr int FZ_CAPB = 16;       // bucket capacity per fine bin; the rest goes to the overflow list
+constexpr int FZ_FIN_PARTS = 8;   // CTAs that share the ranking of the final evaluation
+constexpr int FZ_CUTLIST = 1024;  // entries of the cut bin ranked in shared memory (a fuller bin falls back to global loops)
+constexpr int FZ_CCAP = 4096;     // members grouped in shared memory (more: in the global scratch)
 constexpr int FZ_MAXK = 16;       // stages supported by the fused path
 constexpr int FZ_MAXE = FZ_MAXK + 1;  // evaluations j = 0..K
-constexpr int FZ_MAX_DEPTH = 8;   // most gate/up ring stages; the depths are chosen per launch from the shared memory left
-constexpr int FZ_MAX_DN = 16;     // most down ring stages
+constexpr int FZ_MAX_G1 = 16;     // most slots of the first ring (first row of a bundle); depths are chosen per launch
+constexpr int FZ_MAX_G2 = 8;      // most slots of the second ring (the rest of a survivor's bundle)
 constexpr int FZ_SL = 32;         // columns of the feature handled as one slice in the latent phase
 constexpr int FZ_EPAD = 18;       // rows kept per evaluation-indexed buffer: at most two MMA tiles, or FZ_MAXE rows
 constexpr int FZ_KS = 4;          // column splits of a score tile (more independent tasks than warps)
@@ -50,16 +50,16 @@ constexpr long long FZ_SPIN_CYCLES = 4000LL * 1000 * 1000;  // every wait gives 
 // Shared-memory plan of a layer step (computed on the host, carried in the arguments).
 struct FusedSmemLayout {
   // fixed regions
-  unsigned bar_off, red_off, redd_off, mine_off, pc_off, xt_off, dv_off, qa_off, a_off;
+  unsigned bar_off, red_off, redd_off, mine_off, pc_off, xt_off, dv_off, a_off;
   // the stream's rings ...
-  unsigned gu_off, dn_off;
+  unsigned r1_off, r2_off;
   // ... and, in the same bytes once the rings have drained, the operands and results of the refinement
-  unsigned b_off, zs_off, part_off, own_off, bin_off, coarse_off;
+  unsigned b_off, zs_off, part_off, own_off, sel_off;
   unsigned total;
-  int per, ns_cta, a_alias, gu_depth, dn_depth;
+  int per, ns_cta, a_alias, g1, g2;
 };
 
-struct FusedArgs {
+struct alignas(16) FusedArgs {  // (an array of these is prefetched with 16-byte granularity)
   // layer being executed
   const uint16_t* bundles; int n_mat; int gated; const float* b_gate; const float* b_down;
   int d, F, norm; float eps;
@@ -79,16 +79,19 @@ struct FusedArgs {
   double* z;              // [FZ_MAXE][r] un-normalised latents
   double* sumsq;          // [FZ_MAXE]
   double* zpart;          // [slices][K + 1][r + 1] per-slice partial latents; entry r of a row: partial sum of squares
-  unsigned* cnt;          // [FZ_MAXE][FZ_CNT_STRIDE], zero on entry and on exit
-  uint4* bent;            // [FZ_MAXE][FZ_NB * FZ_CAPB] bucket entries {key lo, key hi, neuron, fine bin}, one 16-byte store each
-  uint4* oent;            // [FZ_MAXE][Fn] overflow entries, same format
+  double* sc;             // [K + 1][Fn] final scores of every evaluation (written by all CTAs, read by the selecting ones)
+  uint16_t* sb;           // [K + 1][Fn] their fine bins
+  uint4* bent;            // [Fn] members of the final evaluation grouped by bin: {key lo, key hi, neuron, fine bin}
+  unsigned long long* kmm;  // [2 G] per CTA: smallest and largest ordered key it saw in the final evaluation
   double* range;          // [2] lo, hi used for binning (observed by the previous launch on this layer)
-  unsigned long long* range_obs;  // [2] ordered keys: min, max observed in the final evaluation
-  unsigned* nsel;         // [FZ_MAXE] sizes of the refined sets (all CTAs add theirs), zero on entry and on exit
   // outputs for the next layer
   int32_t* next_idx; int32_t* next_count; uint32_t* next_mask; double* next_scores; double* next_prio; int next_cap;
   // what the layer after this one will read first (whole-token kernel): brought into L2 while this layer refines
   const void* pf_ptr[4]; unsigned pf_bytes[4];
+  // big arrays the next layer gathers from: one line per 2 MB page is touched, so that its address translations are warm
+  const void* pg_ptr[3]; unsigned long long pg_bytes[3];
+  // speculation into L2: the next layer's bundles (first row of a neuron at spec_ptr + i * spec_stride, spec_bytes long)
+  const char* spec_ptr; unsigned long long spec_stride; unsigned spec_bytes;
   // trace (all nullable)
   float* tr_xtilde; uint32_t* tr_masks; int32_t* tr_counts; uint32_t* tr_survive;
 };
@@ -115,12 +118,14 @@ __device__ __forceinline__ long long fz_now() { unsigned long long t; asm volati
     asm volatile("{ .reg .f32 t_; mov.f32 t_, %1; mov.u64 %0, %%clock64; }" : "=l"(c_) : "f"(fval)); \
     if (blockIdx.x == 0 && (slot) < 512) g_fz_timing[role][slot] = c_;            \
   } while (0)
+#define FZ_STAMPB(slot) do { if (blockIdx.x == 131 && threadIdx.x == 0) g_fz_timing[0][(slot)] = clock64(); } while (0)
 #define FZ_CSTAMP(slot) do { if (blockIdx.x < 160) g_fz_cta[blockIdx.x][slot] = fz_now(); } while (0)
 #define FZ_CVAL(slot, v) do { if (blockIdx.x < 160) g_fz_cta[blockIdx.x][slot] = (v); } while (0)
 #else
 #define FZ_STAMP(role, slot) do { } while (0)
 #define FZ_STAMP_DEP(role, slot, fval) do { } while (0)
 #define FZ_FAIL(site, extra) do { } while (0)
+#define FZ_STAMPB(slot) do { } while (0)
 #define FZ_CSTAMP(slot) do { } while (0)
 #define FZ_CVAL(slot, v) do { } while (0)
 #endif
@@ -201,9 +206,8 @@ __device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float 
 // never reset.  Arrival is a release, the poll an acquire, so what a CTA wrote before the barrier is visible to all
 // after it.  Every compute thread of the block calls it (block barrier 1 spans the 512 compute threads; the producer
 // warp has left by then).
-__device__ __noinline__ void grid_barrier(const FusedArgs& A, int G) {
-  named_bar_sync(1, FZ_THREADS);
-  if (threadIdx.x == 0) {
+__device__ __noinline__ void grid_barrier_thread0(const FusedArgs& A, int G) {
+  {
     unsigned long long old;
     asm volatile("atom.add.release.gpu.global.u64 %0, [%1], 1;" : "=l"(old) : "l"(A.bar_count) : "memory");
     const unsigned long long target = (old / (unsigned long long)G + 1ULL) * (unsigned long long)G;
@@ -216,6 +220,10 @@ __device__ __noinline__ void grid_barrier(const FusedArgs& A, int G) {
     } while (clock64() - t0 < FZ_SPIN_CYCLES);
     if (!ok) { set_status(A.status, ST_TIMEOUT); FZ_FAIL(6, (int)target); }
   }
+}
+__device__ __forceinline__ void grid_barrier(const FusedArgs& A, int G) {
+  named_bar_sync(1, FZ_THREADS);
+  if (threadIdx.x == 0) grid_barrier_thread0(A, G);
   named_bar_sync(1, FZ_THREADS);
 }
 
@@ -276,15 +284,20 @@ __device__ __forceinline__ double quad_sum(double v) {
   return v;
 }
 
-// Bar indices: [0, FZ_MAX_DEPTH) gate/up slots, [FZ_MAX_DEPTH, +FZ_MAX_DN) down slots, then the A slices, then B^T rows.
-constexpr int FZ_BAR_DN = FZ_MAX_DEPTH, FZ_BAR_A = FZ_MAX_DEPTH + FZ_MAX_DN, FZ_BAR_B = FZ_BAR_A + 1, FZ_NBAR = FZ_BAR_B + 1;
+// Shared-memory work area of the selection (see fz_select).
+__host__ __device__ inline size_t fz_select_bytes(int Fn) {
+  return (size_t)2 * FZ_NB * 4 + 128 + (size_t)((Fn + 7) & ~7) * 2 + (size_t)FZ_CUTLIST * 12 + (size_t)FZ_CCAP * 16;
+}
+
+// Bar indices: [0, FZ_MAX_G1) first-ring slots, [FZ_MAX_G1, +FZ_MAX_G2) second-ring slots, then the A slices, then B^T rows.
+constexpr int FZ_BAR_R2 = FZ_MAX_G1, FZ_BAR_A = FZ_MAX_G1 + FZ_MAX_G2, FZ_BAR_B = FZ_BAR_A + 1, FZ_NBAR = FZ_BAR_B + 1;
 
 // `a_alias` != 0 places the A slices inside the ring bytes too (they are then fetched only after the rings have drained).
-inline FusedSmemLayout fused_layout(int d, int n_in, int r, int Fn, int G, int has_next, int gu_depth, int dn_depth,
+inline FusedSmemLayout fused_layout(int d, int n_mat, int r, int Fn, int G, int has_next, int g1, int g2,
                                                         int a_alias) {
   FusedSmemLayout L{};
-  L.gu_depth = gu_depth;
-  L.dn_depth = dn_depth;
+  L.g1 = g1;
+  L.g2 = g2;
   L.a_alias = a_alias;
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t at = o; o += (bytes + 127) & ~(size_t)127; return (unsigned)at; };
@@ -295,15 +308,14 @@ inline FusedSmemLayout fused_layout(int d, int n_in, int r, int Fn, int G, int h
   L.bar_off = take(FZ_NBAR * 8);
   L.red_off = take(2 * 16 * 8 * 4);                  // stream dot partials, double-buffered: [2][warp][8]
   L.redd_off = take(32 * 8);                         // fp64 partials of block reductions
-  L.mine_off = take((size_t)FZ_MAX_MINE * 8);        // this CTA's neuron indices and gate biases
+  L.mine_off = take((size_t)FZ_MAX_MINE * 16);       // this CTA's neurons, their gate biases; the survivors, their activations
   L.pc_off = take((size_t)L.per * 4);
   L.xt_off = take((size_t)FZ_EPAD * FZ_XBLK * 8);  // x~^(j) of one slice, fp64, one padded block per row
   L.dv_off = take((size_t)FZ_MAXK * FZ_SL * 4);      // stage accumulators of one slice
-  L.qa_off = take(FZ_MAX_DN * 4);                    // activations of the queued down rows
   if (!a_alias) L.a_off = take(a_bytes);
   const size_t base = o;
-  L.gu_off = take((size_t)gu_depth * n_in * d * 2);
-  L.dn_off = take((size_t)dn_depth * d * 2);
+  L.r1_off = take((size_t)g1 * d * 2);
+  L.r2_off = take((size_t)g2 * (n_mat - 1) * d * 2);
   const size_t end_stream = o;
   o = base;
   if (a_alias) L.a_off = take(a_bytes);
@@ -311,9 +323,12 @@ inline FusedSmemLayout fused_layout(int d, int n_in, int r, int Fn, int G, int h
   L.b_off = take((size_t)per8 * fz_brow_stride(r) * 2);
   L.zs_off = take(has_next ? (size_t)FZ_EPAD * fz_feat_stride(r) * 8 : 0);
   L.part_off = take(has_next ? (size_t)FZ_KS * FZ_EPAD * per8 * 8 : 0);  // [split][evaluation][neuron]
-  L.own_off = take((size_t)FZ_MAXE * L.per * 8);     // this CTA's scores, every evaluation
-  L.bin_off = take((size_t)FZ_MAXE * L.per * 2);     // and their fine bins
-  L.coarse_off = take(has_next ? (size_t)FZ_MAXE * (FZ_NC + 1) * 4 : 0);
+  L.own_off = take((size_t)L.per * 8);               // this CTA's scores of the final evaluation
+  const size_t end_refine = o;
+  o = base;  // the selection works when the score operands are dead: it shares their bytes
+  L.sel_off = take(has_next ? fz_select_bytes(Fn) : 0);
+  const size_t end_select = o;
+  o = end_refine > end_select ? end_refine : end_select;
   L.total = (unsigned)(o > end_stream ? o : end_stream);
   return L;
 }
@@ -327,92 +342,314 @@ struct FusedShared {
   int round;                         // rounds the compute warps have finished (read by the producer)
   int stage, g_lo, gsize;            // this CTA's stage, the first CTA of the stage's group and the group's size
   unsigned phase[FZ_NBAR];           // phases every mbarrier has completed in earlier layers of the launch
-  int mail[4 * 4];                   // per round (ring of four): number of survivors, their neurons
-  float act[2 * 4];                  // activations of the round's neurons, double-buffered
+  int nsurv, done;                   // survivors found so far / consumed so far (read by the producer)
   double inv[FZ_EPAD];
-  int cut[FZ_MAXE * 4];              // per evaluation: cut fine bin, its first rank, threshold neuron, fallback flag
-  unsigned long long cutkey[FZ_MAXE];  // threshold key inside the cut bin
-  unsigned nsel[FZ_MAXE];            // members found by this CTA, per evaluation
   unsigned long long kmm[2 * 16];
-  unsigned ccnt[FZ_MAXE * FZ_NC];
 };
 
-// ---- rare paths of the ranking phase, kept out of line so that the common path stays small in the instruction cache ----
-// Rank of the entry (key kp, neuron i) of evaluation j whose fine bin bb overflowed its bucket: the first rank of the bin
-// (coarse prefix + the fine counts before it) plus the entries of the bucket and of the overflow list that precede it.
-__device__ __noinline__ int fz_rank_in_overflowed_bin(const FusedArgs& A, int j, int bb, int i, unsigned long long kp,
-                                                      unsigned coarse_b0) {
-  constexpr int FPC = FZ_NB / FZ_NC;
-  const unsigned* cnt = A.cnt + (size_t)j * FZ_CNT_STRIDE;
-  unsigned b0 = coarse_b0;
-#pragma unroll 1
-  for (int fb = (bb / FPC) * FPC; fb < bb; ++fb) b0 += __ldcg(&cnt[fb]);
-  int before = 0;
-  const uint4* bk = A.bent + ((size_t)j * FZ_NB + bb) * FZ_CAPB;
-#pragma unroll 1
-  for (int q = 0; q < FZ_CAPB; ++q) {  // the bucket is full
-    const uint4 e = __ldcg(bk + q);
-    const unsigned long long kq = ((unsigned long long)e.y << 32) | e.x;
-    before += (kq > kp) || (kq == kp && (int)e.z < i);
-  }
-  const unsigned novf = __ldcg(&cnt[FZ_NB + FZ_NC]);
-#pragma unroll 1
-  for (unsigned q = 0; q < novf; ++q) {
-    const uint4 e = __ldcg(&A.oent[(size_t)j * A.Fn + q]);
-    if ((int)e.w != bb) continue;
-    const unsigned long long kq = ((unsigned long long)e.y << 32) | e.x;
-    before += (kq > kp) || (kq == kp && (int)e.z < i);
-  }
-  return (int)b0 + before;
+// Inverse of ordered_key.
+__device__ __forceinline__ double fz_unkey(unsigned long long k) {
+  const unsigned long long b = (k >> 63) ? (k & 0x7fffffffffffffffULL) : ~k;
+  return __longlong_as_double((long long)b);
 }
 
-// Final evaluation, fine bin `bin` with an overflowed bucket, called by the sixteen lanes that hold its bucket entries
-// (entry `ent` in lane l16; the bucket is full).  Returns how many overflow entries precede this lane's entry; lane 0
-// also ranks the overflow entries of the bin themselves and emits those inside the first keff ranks.
-__device__ __noinline__ int fz_final_overflowed_bin(const FusedArgs& A, int j, int bin, unsigned b0, uint4 ent, int l16, int keff,
-                                                    unsigned* s_nsel_j) {
-  const unsigned* cnt = A.cnt + (size_t)j * FZ_CNT_STRIDE;
-  const unsigned novf = __ldcg(&cnt[FZ_NB + FZ_NC]);
-  const unsigned long long kmine = ((unsigned long long)ent.y << 32) | ent.x;
-  int before = 0;
+// ---- exact top-k of one evaluation by one CTA ------------------------------------------------------------------------
+// Inputs (global, written by all CTAs before the preceding grid barrier): sc[j][Fn] scores, sb[j][Fn] their fine bins
+// (FZ_NB bins, descending score).  Shared-memory work area `wk` (see fz_select_bytes): the bins of all neurons, FZ_NB
+// counters (then their exclusive prefix), FZ_NB fill counters, the entries of the cut bin, and the members grouped by
+// bin.  Output: membership (trace mask) for j < K; for j == K the ranked index list, mask, count, and the observed score
+// range for the layer's next launch.  Every evaluation checks that its set has exactly keff members.
+// The final evaluation is shared by `nparts` CTAs: each builds the whole histogram (cheap), then ranks only the members
+// of the bins whose first rank falls in its share of the ranks; nothing is exchanged between them.
+template <int WD>
+__device__ __noinline__ void fz_select(const FusedArgs& A, int j, int K, int keff, unsigned wk_off, int part, int nparts) {
+  // (the work area is addressed through the kernel's dynamic shared array, so that the compiler emits shared-memory
+  // loads, stores and atomics: through a plain pointer argument they would be generic ones, several times slower)
+  extern __shared__ __align__(128) unsigned char fz_dyn_smem[];
+  unsigned char* const wk = fz_dyn_smem + wk_off;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int Fn = A.Fn, G = gridDim.x;
+  uint4* s_cand = reinterpret_cast<uint4*>(wk);                               // [FZ_CCAP] {key lo, key hi, neuron, bin}
+  unsigned long long* s_lkey = reinterpret_cast<unsigned long long*>(s_cand + FZ_CCAP);  // [FZ_CUTLIST]
+  unsigned* s_cnt = reinterpret_cast<unsigned*>(s_lkey + FZ_CUTLIST);        // [FZ_NB] counts, then exclusive prefix
+  unsigned* s_fill = s_cnt + FZ_NB;                                           // [FZ_NB]
+  unsigned* s_wsum = s_fill + FZ_NB;                                          // [32] warp totals of the scan; [16..19] the cut; [20..] key ranges
+  int* s_cutv = reinterpret_cast<int*>(s_wsum + 16);                          // cut fine bin, its first rank, its size; members counted
+  int* s_list = reinterpret_cast<int*>(s_wsum + 32);                          // [FZ_CUTLIST] neurons of the cut bin
+  uint16_t* s_ball = reinterpret_cast<uint16_t*>(s_list + FZ_CUTLIST);        // [Fn8] the bin of every neuron
+  const double* sc = A.sc + (size_t)j * Fn;
+  const uint16_t* sb = A.sb + (size_t)j * Fn;
+  const bool fin = (j == K);
 #pragma unroll 1
-  for (unsigned q = 0; q < novf; ++q) {
-    const uint4 e = __ldcg(&A.oent[(size_t)j * A.Fn + q]);
-    if ((int)e.w != bin) continue;
-    const unsigned long long kq = ((unsigned long long)e.y << 32) | e.x;
-    before += (kq > kmine) || (kq == kmine && (int)e.z < (int)ent.z);
+  for (int t = tid; t < 2 * FZ_NB / 4; t += FZ_THREADS) reinterpret_cast<uint4*>(s_cnt)[t] = make_uint4(0u, 0u, 0u, 0u);
+  // (final evaluation) the per-CTA score ranges are fetched now and folded at the end
+  unsigned long long kmin = 0xffffffffffffffffULL, kmax = 0ULL;
+  if (fin) {
+#pragma unroll 1
+    for (int c = tid; c < G; c += FZ_THREADS) { kmin = min(kmin, __ldcg(&A.kmm[2 * c])); kmax = max(kmax, __ldcg(&A.kmm[2 * c + 1])); }
   }
-  if (l16 == 0) {
+  if (tid == 0) { s_cutv[0] = -1; s_cutv[1] = 0; s_cutv[2] = 0; s_cutv[3] = 0; }
+  named_bar_sync(1, FZ_THREADS);
+  if (tid == 0) FZ_STAMP(1, 61);
+  if (tid == 0) FZ_CSTAMP(12);
+  FZ_STAMPB(300);
+  // pass 1: the bins come to shared memory (eight neurons per 16-byte load when the row is aligned) and are counted
+  if ((((size_t)j * Fn) & 7) == 0) {
+    const uint4* sb8 = reinterpret_cast<const uint4*>(sb);
+    const int n8 = Fn >> 3;
 #pragma unroll 1
-    for (unsigned q = 0; q < novf; ++q) {
-      const uint4 e = __ldcg(&A.oent[(size_t)j * A.Fn + q]);
-      if ((int)e.w != bin) continue;
-      const unsigned long long ke = ((unsigned long long)e.y << 32) | e.x;
-      int bf = 0;
-#pragma unroll 1
-      for (int u = 0; u < FZ_CAPB; ++u) {
-        const uint4 o = __ldcg(&A.bent[((size_t)j * FZ_NB + bin) * FZ_CAPB + u]);
-        const unsigned long long ko = ((unsigned long long)o.y << 32) | o.x;
-        bf += (ko > ke) || (ko == ke && (int)o.z < (int)e.z);
+    for (int t0 = 0; t0 < n8; t0 += 4 * FZ_THREADS) {
+      uint4 q[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int t = t0 + u * FZ_THREADS + tid;
+        q[u] = t < n8 ? __ldcg(sb8 + t) : make_uint4(0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu);
       }
-#pragma unroll 1
-      for (unsigned u = 0; u < novf; ++u) {
-        const uint4 o = __ldcg(&A.oent[(size_t)j * A.Fn + u]);
-        if ((int)o.w != bin) continue;
-        const unsigned long long ko = ((unsigned long long)o.y << 32) | o.x;
-        bf += (ko > ke) || (ko == ke && (int)o.z < (int)e.z);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int t = t0 + u * FZ_THREADS + tid;
+        if (t < n8) {
+          reinterpret_cast<uint4*>(s_ball)[t] = q[u];
+          const uint32_t w[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            atomicAdd(&s_cnt[w[e] & 0xffffu], 1u);
+            atomicAdd(&s_cnt[w[e] >> 16], 1u);
+          }
+        }
       }
-      const int rk = (int)b0 + bf;
-      if (rk < keff) {
-        const int i = (int)e.z;
-        if (rk < A.next_cap) A.next_idx[rk] = i;
-        if (A.next_mask) atomicOr(&A.next_mask[i >> 5], 1u << (i & 31));
-        if (A.tr_masks) atomicOr(&A.tr_masks[(size_t)j * ((A.Fn + 31) >> 5) + (i >> 5)], 1u << (i & 31));
-        atomicAdd(s_nsel_j, 1u);
+    }
+#pragma unroll 1
+    for (int t = (n8 << 3) + tid; t < Fn; t += FZ_THREADS) { const unsigned b = __ldcg(sb + t); s_ball[t] = (uint16_t)b; atomicAdd(&s_cnt[b], 1u); }
+  } else {
+#pragma unroll 1
+    for (int t = tid; t < Fn; t += FZ_THREADS) { const unsigned b = __ldcg(sb + t); s_ball[t] = (uint16_t)b; atomicAdd(&s_cnt[b], 1u); }
+  }
+  named_bar_sync(1, FZ_THREADS);
+  if (tid == 0) FZ_STAMP(1, 62);
+  FZ_STAMPB(301);
+  // exclusive scan of the FZ_NB counts (eight per thread), and the cut bin
+  {
+    constexpr int PT = FZ_NB / FZ_THREADS;
+    unsigned c[PT], tot = 0;
+#pragma unroll
+    for (int q = 0; q < PT; ++q) { c[q] = s_cnt[tid * PT + q]; tot += c[q]; }
+    unsigned incl = tot;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned v = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += v;
+    }
+    if (lane == 31) s_wsum[warp] = incl;
+    named_bar_sync(1, FZ_THREADS);
+    unsigned base = 0;
+#pragma unroll 4
+    for (int w = 0; w < FZ_THREADS / 32; ++w) base += w < warp ? s_wsum[w] : 0u;
+    unsigned ex = base + incl - tot;
+#pragma unroll
+    for (int q = 0; q < PT; ++q) {
+      s_cnt[tid * PT + q] = ex;
+      if (c[q] > 0 && (int)ex < keff && (int)(ex + c[q]) >= keff) { s_cutv[0] = tid * PT + q; s_cutv[1] = (int)ex; s_cutv[2] = (int)c[q]; }
+      ex += c[q];
+    }
+  }
+  named_bar_sync(1, FZ_THREADS);
+  if (tid == 0) FZ_STAMP(1, 63);
+  if (tid == 0) FZ_CSTAMP(13);
+  FZ_STAMPB(302);
+  const int cut_bin = s_cutv[0], cut_b0 = s_cutv[1], cut_nb = s_cutv[2];  // no cut bin (-1): keff == 0, nothing is selected
+  const int need = keff - cut_b0;                                         // members inside the cut bin
+  uint32_t* const trm = A.tr_masks ? A.tr_masks + (size_t)j * ((Fn + 31) >> 5) : nullptr;
+  if (!fin) {
+    // Intermediate evaluation: its refined set is now fixed by the cut (bins before the cut bin are in, the cut bin is
+    // split by exact comparison: entry e is a member iff fewer than `need` entries of the bin precede it).  Nothing
+    // consumes the set itself when every bundle is resident, so it is written out only when a trace asks for it.
+    if (cut_bin >= 0 && trm) {
+#pragma unroll 1
+      for (int t = tid; t < Fn; t += FZ_THREADS) {
+        const int b = s_ball[t];
+        if (b < cut_bin) {
+          if (trm) atomicOr(&trm[t >> 5], 1u << (t & 31));
+        } else if (b == cut_bin) {
+          const unsigned p = atomicAdd(&s_fill[b], 1u);
+          if (p < (unsigned)FZ_CUTLIST) s_list[p] = t;
+        }
+      }
+      named_bar_sync(1, FZ_THREADS);
+      if (tid == 0) FZ_STAMP(1, 64);
+      if (cut_nb <= FZ_CUTLIST) {
+#pragma unroll 1
+        for (int e = tid; e < cut_nb; e += FZ_THREADS) s_lkey[e] = ordered_key(__ldcg(sc + s_list[e]));
+        named_bar_sync(1, FZ_THREADS);
+#pragma unroll 1
+        for (int e = tid; e < cut_nb; e += FZ_THREADS) {
+          const int i = s_list[e];
+          const unsigned long long kp = s_lkey[e];
+          int before = 0;
+#pragma unroll 1
+          for (int q = 0; q < cut_nb; ++q) before += (s_lkey[q] > kp) || (s_lkey[q] == kp && s_list[q] < i);
+          if (before < need) {
+            atomicAdd(&s_cutv[3], 1);
+            if (trm) atomicOr(&trm[i >> 5], 1u << (i & 31));
+          }
+        }
+      } else {  // an overfull cut bin (degenerate score distributions): every neuron of the bin scans the whole row
+#pragma unroll 1
+        for (int i = tid; i < Fn; i += FZ_THREADS) {
+          if ((int)s_ball[i] != cut_bin) continue;
+          const unsigned long long kp = ordered_key(__ldcg(sc + i));
+          int before = 0;
+#pragma unroll 1
+          for (int iq = 0; iq < Fn; ++iq) {
+            if ((int)s_ball[iq] != cut_bin) continue;
+            const unsigned long long kq = ordered_key(__ldcg(sc + iq));
+            before += (kq > kp) || (kq == kp && iq < i);
+          }
+          if (before < need) {
+            atomicAdd(&s_cutv[3], 1);
+            if (trm) atomicOr(&trm[i >> 5], 1u << (i & 31));
+          }
+        }
+      }
+      named_bar_sync(1, FZ_THREADS);
+      if (tid == 0 && cut_b0 + s_cutv[3] != keff) set_status(A.status, ST_INTERNAL);  // self-check of the set's size
+    }
+    return;
+  }
+  // final evaluation: the members of this CTA's share of the bins are scattered into `cand`, grouped by bin (position =
+  // first rank of the bin + arrival order); a member's exact rank = first rank of its bin + entries of the bin before it
+  const int ncand = cut_bin >= 0 ? cut_b0 + cut_nb : 0;
+  const unsigned lo_r = (unsigned)(((long long)part * ncand) / nparts), hi_r = (unsigned)(((long long)(part + 1) * ncand) / nparts);
+  uint4* const cand = ncand <= FZ_CCAP ? s_cand : A.bent;
+  if (tid == 0) { s_cutv[4] = 0x7fffffff; s_cutv[5] = 0; }
+  named_bar_sync(1, FZ_THREADS);
+  if (cut_bin >= 0) {
+    // (a) neuron and bin of every member, shared memory only
+    unsigned pmin = 0x7fffffffu, pmax = 0u;
+#pragma unroll 1
+    for (int t0 = tid; t0 < Fn; t0 += 8 * FZ_THREADS) {
+      int bb[8];
+      unsigned pre[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {  // all the loads first: behind a store or an atomic they could not be moved up
+        const int t = t0 + u * FZ_THREADS;
+        bb[u] = t < Fn ? (int)s_ball[t] : FZ_NB;
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) pre[u] = bb[u] <= cut_bin ? s_cnt[bb[u]] : 0xffffffffu;
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        if (pre[u] >= lo_r && pre[u] < hi_r) {
+          const unsigned pos = pre[u] + atomicAdd(&s_fill[bb[u]], 1u);
+          cand[pos] = make_uint4(0u, 0u, (unsigned)(t0 + u * FZ_THREADS), (unsigned)bb[u]);
+          pmin = min(pmin, pos);
+          pmax = max(pmax, pos + 1u);
+        }
+      }
+    }
+    pmin = __reduce_min_sync(0xffffffffu, pmin);
+    pmax = __reduce_max_sync(0xffffffffu, pmax);
+    if (lane == 0 && pmax > 0u) { atomicMin(&s_cutv[4], (int)pmin); atomicMax(&s_cutv[5], (int)pmax); }
+  }
+  named_bar_sync(1, FZ_THREADS);
+  if (tid == 0) FZ_CSTAMP(14);
+  FZ_STAMPB(303);
+  const int pstart = min(s_cutv[4], s_cutv[5]), pend = s_cutv[5];  // this CTA's positions [pstart, pend)
+  // (b) their keys: four score loads in flight per thread
+#pragma unroll 1
+  for (int p0 = pstart; p0 < pend; p0 += 4 * FZ_THREADS) {
+    double v[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int p = p0 + u * FZ_THREADS + tid;
+      v[u] = p < pend ? __ldcg(sc + cand[p].z) : 0.0;
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int p = p0 + u * FZ_THREADS + tid;
+      if (p < pend) {
+        const unsigned long long key = ordered_key(v[u]);
+        cand[p].x = (unsigned)key;
+        cand[p].y = (unsigned)(key >> 32);
       }
     }
   }
-  return before;
+  named_bar_sync(1, FZ_THREADS);  // (also makes this CTA's writes to the global scratch visible to all its threads)
+  if (tid == 0) FZ_CSTAMP(15);
+  FZ_STAMPB(304);
+  {
+    int32_t* const nidx = A.next_idx;
+    uint32_t* const nmask = A.next_mask;
+    const int ncap = A.next_cap;
+    int found = 0;
+#pragma unroll 1
+    for (int p = pstart + tid; p < pend; p += FZ_THREADS) {
+      const uint4 me = cand[p];
+      const int b = (int)me.w, i = (int)me.z;
+      const unsigned long long kp = ((unsigned long long)me.y << 32) | me.x;
+      const int b0 = (int)s_cnt[b], nb = (int)s_fill[b];
+      int before = 0;
+#pragma unroll 1
+      for (int q = b0; nb > 1 && q < b0 + nb; ++q) {  // (a member alone in its bin has the bin's first rank)
+        const uint4 o = cand[q];
+        const unsigned long long kq = ((unsigned long long)o.y << 32) | o.x;
+        before += (kq > kp) || (kq == kp && (int)o.z < i);
+      }
+      const int rank = b0 + before;
+      if (rank < keff) {
+        ++found;
+        if (rank < ncap) nidx[rank] = i;
+        if (nmask) atomicOr(&nmask[i >> 5], 1u << (i & 31));
+        if (trm) atomicOr(&trm[i >> 5], 1u << (i & 31));
+      }
+    }
+    FZ_STAMPB(305);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) found += __shfl_xor_sync(0xffffffffu, found, o);
+    if (lane == 0 && found) atomicAdd(&s_cutv[3], found);
+    FZ_STAMPB(306);
+  }
+  named_bar_sync(1, FZ_THREADS);
+  if (tid == 0 && s_cutv[3] != max(0, min(keff, pend) - pstart)) set_status(A.status, ST_INTERNAL);  // self-check: one member per rank
+  if (part != 0) return;
+  // the layer's binning range for its next launch: what all CTAs observed in this evaluation, widened by 5 % per side
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    kmin = min(kmin, __shfl_xor_sync(0xffffffffu, kmin, o));
+    kmax = max(kmax, __shfl_xor_sync(0xffffffffu, kmax, o));
+  }
+  unsigned long long* s_kmm2 = reinterpret_cast<unsigned long long*>(s_lkey);  // (the cut list is dead by now)
+  if (lane == 0) { s_kmm2[warp] = kmin; s_kmm2[16 + warp] = kmax; }
+  named_bar_sync(1, FZ_THREADS);
+  if (tid == 0) {
+#pragma unroll 1
+    for (int w = 1; w < 16; ++w) { kmin = min(kmin, s_kmm2[w]); kmax = max(kmax, s_kmm2[16 + w]); }
+    if (kmin <= kmax) {
+      double lo = fmax(fz_unkey(kmin), -1.0e300), hi = fmin(fz_unkey(kmax), 1.0e300);
+      const double pad = 0.05 * (hi - lo);
+      A.range[0] = lo - pad;
+      A.range[1] = hi + pad;
+    }
+    FZ_STAMPB(307);
+    if (A.tr_counts)
+#pragma unroll 1
+      for (int jj = 0; jj <= K; ++jj) A.tr_counts[jj] = keff;
+    *A.next_count = min(keff, A.next_cap);
+    if (keff > A.next_cap) set_status(A.status, ST_CAPACITY);
+  }
+}
+
+// The producer's copy of this CTA's column slices of the next layer's A (one mbarrier for all of them).
+__device__ __noinline__ void fz_issue_a(const FusedArgs& A, uint16_t* s_A, uint64_t* abar, int cta, int G, int nsl) {
+  const uint32_t sl_bytes = (uint32_t)A.r * FZ_SL * 2;
+  int nmy = 0;
+#pragma unroll 1
+  for (int sl = cta; sl < nsl; sl += G) ++nmy;
+  mbar_expect_tx(abar, (uint32_t)nmy * sl_bytes);
+  int a = 0;
+#pragma unroll 1
+  for (int sl = cta; sl < nsl; sl += G, ++a)
+    tma_load_1d(s_A + (size_t)a * A.r * FZ_SL, A.At_sl + (size_t)sl * A.r * FZ_SL, sl_bytes, abar);
 }
 
 // One layer step, executed by the whole block (16 compute warps + the producer warp).  The producer warp returns as
@@ -425,11 +662,10 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
   const int G = gridDim.x, cta = blockIdx.x, tid = threadIdx.x;
   const int lane = tid & 31, warp = tid >> 5;
   const int d = A.d, K = A.K, nchunk = A.d >> 3;
-  const int n_in = A.gated ? 2 : 1;
   const FusedSmemLayout& lay = A.lay;
-  const int GU = lay.gu_depth, DN = lay.dn_depth;
-  uint16_t* s_gu = reinterpret_cast<uint16_t*>(smem + lay.gu_off);
-  uint16_t* s_dn = reinterpret_cast<uint16_t*>(smem + lay.dn_off);
+  const int G1 = lay.g1, G2 = lay.g2;
+  uint16_t* s_r1 = reinterpret_cast<uint16_t*>(smem + lay.r1_off);  // [G1][d]
+  uint16_t* s_r2 = reinterpret_cast<uint16_t*>(smem + lay.r2_off);  // [G2][(n_mat - 1) d]
   uint64_t* s_bar = reinterpret_cast<uint64_t*>(smem + lay.bar_off);  // "full" barriers: gate/up slots, down slots, A, B^T
   float* s_red = reinterpret_cast<float*>(smem + lay.red_off);        // [2][16 warps][8]
   double* s_redd = reinterpret_cast<double*>(smem + lay.redd_off);
@@ -437,15 +673,9 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
   uint16_t* s_B = reinterpret_cast<uint16_t*>(smem + lay.b_off);      // [per8][fz_brow_stride(r)]
   float* s_pc = reinterpret_cast<float*>(smem + lay.pc_off);
   double* s_xt = reinterpret_cast<double*>(smem + lay.xt_off);        // [K+1][32]
-  float* s_qa = reinterpret_cast<float*>(smem + lay.qa_off);          // [DN]
   int& s_round = sh.round;
-  int* s_mail = sh.mail;
   double* s_inv = sh.inv;
-  int* s_cut = sh.cut;
-  unsigned long long* s_cutkey = sh.cutkey;
-  unsigned* s_nsel = sh.nsel;
   unsigned long long* s_kmm = sh.kmm;
-  unsigned* s_ccnt = sh.ccnt;
 
   if (tid == 0) FZ_CSTAMP(0);
   // The mbarriers are set up once per launch and keep running from layer to layer: sh.phase[b] counts the phases barrier
@@ -466,7 +696,7 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
       sh.gsize = (c + 1) * G / K - sh.g_lo;
     }
   }
-  if (tid == 0) s_round = 0;
+  if (tid == 0) { s_round = 0; sh.nsurv = 0; sh.done = 0; }
   __syncthreads();
   if (tid == 0) FZ_STAMP(1, 20);
 
@@ -474,7 +704,7 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
   const int i_lo = cta * per, i_hi = min(Fn, i_lo + per);
   const int n_own = max(0, i_hi - i_lo);
   const int nsl = (d + FZ_SL - 1) / FZ_SL;  // column slices of the feature; this CTA takes slices cta, cta + G, ...
-  int used_gu = 0, used_dn = 0;            // gate/up rows and down rows this CTA fetched in this layer
+  int used_r1 = 0, used_r2 = 0;            // first-ring and second-ring copies this CTA waited for in this layer
 
   {
     // ================================================= stream: all warps ===========================================
@@ -486,12 +716,15 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
     const int first = lo + (cta - g_lo);
     const int n_mine = first < hi ? (hi - first + gsize - 1) / gsize : 0;
     const int n_rounds = (n_mine + FZ_NG - 1) / FZ_NG;
-    const uint32_t gu_bytes = (uint32_t)n_in * d * 2, dn_bytes = (uint32_t)d * 2;
+    const uint32_t r1_bytes = (uint32_t)d * 2, r2_bytes = (uint32_t)(A.n_mat - 1) * d * 2;
     const size_t bundle_elems = (size_t)A.n_mat * d;
+    const int up_off = A.gated ? 0 : -1, dn_off = A.gated ? d : 0;  // where the rows sit inside a second-ring slot
 
     // this CTA's neurons first (the bulk copies only need the indices), then x
     int* s_myidx = reinterpret_cast<int*>(smem + lay.mine_off);
     float* s_mybias = reinterpret_cast<float*>(s_myidx + FZ_MAX_MINE);
+    int* s_surv = s_myidx + 2 * FZ_MAX_MINE;                       // surviving neurons, in the order they were found
+    float* s_qa = reinterpret_cast<float*>(s_myidx + 3 * FZ_MAX_MINE);  // their activations
 #pragma unroll 1
     for (int t = tid; t < n_mine; t += FZ_THREADS) {
       int i = __ldcg(A.sel_idx + first + t * gsize);
@@ -526,64 +759,68 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
 
     if (warp == FZ_THREADS / 32) {
       // ============================================= producer warp (one lane) ======================================
-      // Issues every bulk copy, so that the compute warps never pay for it.  Step rd waits until the compute warps have
-      // finished rd rounds (announced through s_round), tops the gate/up ring up to the rows that may then be in
-      // flight, and fetches the down rows of round rd-1's survivors.
+      // Issues every bulk copy, so that the compute warps never pay for it.  First ring: the first row of each of this
+      // CTA's neurons (gate, or the only input matrix), as many as fit at once, topped up as rounds finish.  Second
+      // ring: the rest of a neuron's bundle (up and down rows), fetched only for the neurons whose activation
+      // survived, as slots come free.  The compute warps publish rounds finished, survivors found and survivors
+      // consumed in sh.round / sh.nsurv / sh.done.
       if (lane == 0) {
-        int issued = 0, gslot = 0, dslot = 0;
-        bool ok = true;
+        int issued1 = 0, slot1 = 0, issued2 = 0, slot2 = 0, rounds = 0, nsurv = 0;
+        bool a_sent = false, ok = true;
+        const long long t0 = clock64();
+        while (true) {
+          // top the first ring up to the rows that may be in flight
+          const int want = min(n_mine, rounds * FZ_NG + G1);
 #pragma unroll 1
-        for (int rd = 0; rd <= n_rounds; ++rd) {
-          if (rd > 0 && !(ok = fz_wait_round(&s_round, rd, A.status))) break;
-          const int want = min(n_mine, rd * FZ_NG + GU);
-#pragma unroll 1
-          for (; issued < want; ++issued) {
-            int i = s_myidx[issued];
+          for (; issued1 < want; ++issued1) {
+            int i = s_myidx[issued1];
             if (i < 0) i = 0;  // a rejected index: read row 0, the result is discarded
-            uint64_t* bar = &s_bar[gslot];
-            mbar_expect_tx(bar, gu_bytes);
-            tma_load_1d(s_gu + (size_t)gslot * n_in * d, A.bundles + (size_t)i * bundle_elems, gu_bytes, bar);
-            if (++gslot == GU) gslot = 0;
+            uint64_t* bar = &s_bar[slot1];
+            mbar_expect_tx(bar, r1_bytes);
+            tma_load_1d(s_r1 + (size_t)slot1 * d, A.bundles + (size_t)i * bundle_elems, r1_bytes, bar);
+            if (++slot1 == G1) slot1 = 0;
           }
-          if (rd > 0) {
-            const int* mail = s_mail + ((rd - 1) & 3) * 4;
-            const int ns = mail[0];
+          if (!a_sent && A.has_next && !lay.a_alias) {  // A slices with a place of their own: right behind the first burst
+            a_sent = true;
+            fz_issue_a(A, s_A, &s_bar[FZ_BAR_A], cta, G, nsl);
+          }
+          // survivors whose slot is free
+          int done;
+          asm volatile("ld.acquire.cta.shared.s32 %0, [%1];" : "=r"(done) : "r"(smem_u32(&sh.done)) : "memory");
 #pragma unroll 1
-            for (int e = 0; e < ns; ++e) {
-              const int i = mail[1 + e];
-              uint64_t* bar = &s_bar[FZ_BAR_DN + dslot];
-              mbar_expect_tx(bar, dn_bytes);
-              tma_load_1d(s_dn + (size_t)dslot * d, A.bundles + (size_t)i * bundle_elems + (size_t)(A.n_mat - 1) * d, dn_bytes, bar);
-              if (A.tr_survive) atomicOr(&A.tr_survive[i >> 5], 1u << (i & 31));
-              if (++dslot == DN) dslot = 0;
-            }
+          for (; issued2 < nsurv && issued2 - done < G2; ++issued2) {
+            const int i = s_surv[issued2];
+            uint64_t* bar = &s_bar[FZ_BAR_R2 + slot2];
+            mbar_expect_tx(bar, r2_bytes);
+            tma_load_1d(s_r2 + (size_t)slot2 * (A.n_mat - 1) * d, A.bundles + (size_t)i * bundle_elems + d, r2_bytes, bar);
+            if (A.tr_survive) atomicOr(&A.tr_survive[i >> 5], 1u << (i & 31));
+            if (++slot2 == G2) slot2 = 0;
+          }
+          if (rounds == n_rounds && issued2 == nsurv) break;  // every row of this layer has been requested
+          // wait for news: a round finished (more survivors, room in the first ring) or survivors consumed
+          int rnow, dnow;
+          while (true) {
+            asm volatile("ld.acquire.cta.shared.s32 %0, [%1];" : "=r"(rnow) : "r"(smem_u32(&s_round)) : "memory");
+            asm volatile("ld.acquire.cta.shared.s32 %0, [%1];" : "=r"(dnow) : "r"(smem_u32(&sh.done)) : "memory");
+            if (rnow > rounds || (dnow > done && issued2 < nsurv)) break;
+            if (clock64() - t0 > FZ_SPIN_CYCLES) { ok = false; break; }
+            __nanosleep(64);  // the poll shares an instruction scheduler with four compute warps
+          }
+          if (!ok) { set_status(A.status, ST_TIMEOUT); break; }
+          if (rnow > rounds) {
+            rounds = min(rnow, n_rounds);
+            asm volatile("ld.acquire.cta.shared.s32 %0, [%1];" : "=r"(nsurv) : "r"(smem_u32(&sh.nsurv)) : "memory");
           }
         }
-        // The next layer's predictor operands, off the streaming's critical path.  A slices that have a place of their
-        // own are fetched now; everything that shares bytes with the rings waits until the compute warps have drained them.
-        if (A.has_next && ok) {
-          bool drained = false;
-          if (lay.a_alias) drained = ok = fz_wait_round(&s_round, n_rounds + 1, A.status);
-          if (ok) {  // this CTA's column slices of the next layer's A
-            uint64_t* abar = &s_bar[FZ_BAR_A];
-            const uint32_t sl_bytes = (uint32_t)r * FZ_SL * 2;
-            int nmy = 0;
+        // The next layer's predictor operands that share bytes with the rings wait until the compute warps have drained them.
+        if (A.has_next && ok && fz_wait_round(&s_round, n_rounds + 1, A.status)) {
+          if (lay.a_alias) fz_issue_a(A, s_A, &s_bar[FZ_BAR_A], cta, G, nsl);
+          uint64_t* bbar = &s_bar[FZ_BAR_B];  // rows of B^T: awaited before the score phase
+          mbar_expect_tx(bbar, (uint32_t)n_own * (uint32_t)r * 2);
+          const int rsb = fz_brow_stride(r);
 #pragma unroll 1
-            for (int sl = cta; sl < nsl; sl += G) ++nmy;
-            mbar_expect_tx(abar, (uint32_t)nmy * sl_bytes);
-            int a = 0;
-#pragma unroll 1
-            for (int sl = cta; sl < nsl; sl += G, ++a)
-              tma_load_1d(s_A + (size_t)a * r * FZ_SL, A.At_sl + (size_t)sl * r * FZ_SL, sl_bytes, abar);
-          }
-          if (!drained) ok = ok && fz_wait_round(&s_round, n_rounds + 1, A.status);
-          if (ok) {  // rows of B^T: awaited before the score phase
-            uint64_t* bbar = &s_bar[FZ_BAR_B];
-            mbar_expect_tx(bbar, (uint32_t)n_own * (uint32_t)r * 2);
-#pragma unroll 1
-            for (int li = 0; li < n_own; ++li)
-              tma_load_1d(s_B + (size_t)li * fz_brow_stride(r), A.Bt + (size_t)(i_lo + li) * r, (uint32_t)r * 2, bbar);
-          }
+          for (int li = 0; li < n_own; ++li)
+            tma_load_1d(s_B + (size_t)li * rsb, A.Bt + (size_t)(i_lo + li) * r, (uint32_t)r * 2, bbar);
         }
       }
       return;  // an exited warp counts as arrived at every later block barrier
@@ -596,54 +833,24 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
       for (int w = 0; w < FZ_THREADS / 32; ++w) tot += s_redd[w];
       inv_rms = (float)fz_rsqrt(fma(tot, A.inv_d, (double)A.eps));
     }
-
-    // pending down rows: FIFO over the down ring (head slot hslot, its use count hwrap; tail slot tslot); their
-    // activations wait in s_qa; every thread tracks the same head and tail
-    int dq_head = 0, dq_tail = 0, hslot = 0, tslot = 0, gslot = 0;
-    unsigned hwrap = 0, gwrap = 0;
-    float yacc[CPT][8];
-#pragma unroll
-    for (int q = 0; q < CPT; ++q)
-#pragma unroll
-      for (int e = 0; e < 8; ++e) yacc[q][e] = 0.f;
     if (tid == 0) FZ_STAMP(0, 0);
     if (tid == 0) { FZ_CSTAMP(1); FZ_CVAL(8, n_mine); FZ_CVAL(10, stage); }
 
+    // ---- first ring: the pre-activation of every neuron, three neurons per round; survivors go to the producer -------
+    int nsurv = 0, slot1 = 0;
+    unsigned wrap1 = 0;
 #pragma unroll 1
-    for (int rd = 0; rd <= n_rounds; ++rd) {  // the last pass only drains the down ring
+    for (int rd = 0; rd < n_rounds; ++rd) {
       const int it0 = rd * FZ_NG;
       const int nn = min(FZ_NG, n_mine - it0);
       if (tid == 0) FZ_STAMP(0, 1 + rd * 4);
-      // (1) make room in the down ring for this round's survivors (reads of a slot end before the round barrier);
-      //     each pending row, scaled by its activation, joins the CTA's partial output
-#pragma unroll 1
-      while (rd == n_rounds ? dq_head < dq_tail : dq_tail - dq_head > DN - FZ_NG) {
-        mbar_wait(&s_bar[FZ_BAR_DN + hslot], (s_phase[FZ_BAR_DN + hslot] + hwrap) & 1u, A.status);
-        const float a = s_qa[hslot];
-        const uint16_t* row = s_dn + (size_t)hslot * d;
-#pragma unroll
-        for (int q = 0; q < CPT; ++q) {
-          const int ch = tid + q * FZ_THREADS;
-          if (ch < nchunk) {
-            float w[8];
-            unpack8<WD>(*reinterpret_cast<const uint4*>(row + ch * 8), w);
-#pragma unroll
-            for (int e = 0; e < 8; ++e) yacc[q][e] = fmaf(a, w[e], yacc[q][e]);
-          }
-        }
-        ++dq_head;
-        if (++hslot == DN) { hslot = 0; ++hwrap; }
-      }
-      if (rd == n_rounds) break;
-      // (2) partial dot products of the round's neurons
-      float pg[FZ_NG], pu[FZ_NG];
+      float pg[FZ_NG];
 #pragma unroll
       for (int e = 0; e < FZ_NG; ++e) {
         pg[e] = 0.f;
-        pu[e] = 0.f;
         if (e < nn) {
-          mbar_wait(&s_bar[gslot], (s_phase[gslot] + gwrap) & 1u, A.status);
-          const uint16_t* grow = s_gu + (size_t)gslot * n_in * d;
+          mbar_wait(&s_bar[slot1], (s_phase[slot1] + wrap1) & 1u, A.status);
+          const uint16_t* grow = s_r1 + (size_t)slot1 * d;
 #pragma unroll
           for (int q = 0; q < CPT; ++q) {
             const int ch = tid + q * FZ_THREADS;
@@ -652,82 +859,128 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
               unpack8<WD>(*reinterpret_cast<const uint4*>(grow + ch * 8), w);
 #pragma unroll
               for (int t = 0; t < 8; ++t) pg[e] = fmaf(w[t], xr[q][t], pg[e]);
-              if (A.gated) {
-                unpack8<WD>(*reinterpret_cast<const uint4*>(grow + d + ch * 8), w);
-#pragma unroll
-                for (int t = 0; t < 8; ++t) pu[e] = fmaf(w[t], xr[q][t], pu[e]);
-              }
             }
           }
-          if (++gslot == GU) { gslot = 0; ++gwrap; }
+          if (++slot1 == G1) { slot1 = 0; ++wrap1; }
         }
       }
       if (tid == 0) FZ_STAMP(0, 2 + rd * 4);
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) {
 #pragma unroll
-        for (int e = 0; e < FZ_NG; ++e) {
-          pg[e] += __shfl_xor_sync(0xffffffffu, pg[e], o);
-          pu[e] += __shfl_xor_sync(0xffffffffu, pu[e], o);
-        }
+        for (int e = 0; e < FZ_NG; ++e) pg[e] += __shfl_xor_sync(0xffffffffu, pg[e], o);
       }
-      float* red = s_red + (rd & 1) * (FZ_THREADS / 32) * 8;  // [warp][8]: g0 u0 g1 u1 g2 u2 - -
-      if (lane == 0) {
-        *reinterpret_cast<float4*>(red + warp * 8) = make_float4(pg[0], pu[0], pg[1], pu[1]);
-        *reinterpret_cast<float2*>(red + warp * 8 + 4) = make_float2(pg[2], pu[2]);
-      }
+      float* red = s_red + (rd & 1) * (FZ_THREADS / 32) * 4;  // [warp][4]
+      if (lane == 0) *reinterpret_cast<float4*>(red + warp * 4) = make_float4(pg[0], pg[1], pg[2], 0.f);
       named_bar_sync(1, FZ_THREADS);  // partials visible; every thread is done with the round's ring slots
-      // (3) warp 0 finishes the six sums, forms the activations and tells the producer what to fetch
-      if (warp == 0) {
-        float v = 0.f;
-        if (lane < 2 * FZ_NG) {
-#pragma unroll 4
-          for (int w = 0; w < FZ_THREADS / 32; ++w) v += red[w * 8 + lane];
-        }
-        const float u = __shfl_down_sync(0xffffffffu, v, 1);  // lane 2e holds g_e, lane 2e+1 holds u_e
+      if (warp == 0) {  // pre-activations; the neurons that survive the ReLU join the list the producer fetches from
         float a = 0.f;
         int i = -1;
-        const int e = lane >> 1;
-        if (!(lane & 1) && e < nn) {
-          const int it = it0 + e;
-          i = s_myidx[it];
-          const float g = v * inv_rms + s_mybias[it];
-          a = fmaxf(g, 0.f);
-          if (A.gated) a *= u * inv_rms;
+        if (lane < nn) {
+          float v = 0.f;
+#pragma unroll 4
+          for (int w = 0; w < FZ_THREADS / 32; ++w) v += red[w * 4 + lane];
+          i = s_myidx[it0 + lane];
+          a = fmaxf(v * inv_rms + s_mybias[it0 + lane], 0.f);
           if (i < 0) a = 0.f;
         }
-        // survivors in neuron order -> mailbox of the round, activations -> the queue slots their rows will use
         const unsigned surv = __ballot_sync(0xffffffffu, a != 0.f);
         if (a != 0.f) {
-          const int pos = __popc(surv & ((1u << lane) - 1u));
-          s_mail[(rd & 3) * 4 + 1 + pos] = i;
-          int qs = tslot + pos;
-          if (qs >= DN) qs -= DN;
-          s_qa[qs] = a;
+          const int pos = nsurv + __popc(surv & ((1u << lane) - 1u));
+          s_surv[pos] = i;
+          s_qa[pos] = a;
         }
         if (lane == 0) {
-          s_mail[(rd & 3) * 4] = __popc(surv);
+          asm volatile("st.release.cta.shared.s32 [%0], %1;" ::"r"(smem_u32(&sh.nsurv)), "r"(nsurv + __popc(surv)) : "memory");
           asm volatile("st.release.cta.shared.s32 [%0], %1;" ::"r"(smem_u32(&s_round)), "r"(rd + 1) : "memory");
         }
       }
       named_bar_sync(1, FZ_THREADS);
+      nsurv = sh.nsurv;
       if (tid == 0) FZ_STAMP(0, 3 + rd * 4);
-      // (4) the survivors' rows were queued by the producer in the same order
-      {
-        const int ns = s_mail[(rd & 3) * 4];
-        dq_tail += ns;
-        tslot += ns;
-        if (tslot >= DN) tslot -= DN;
-      }
     }
     if (tid == 0) FZ_STAMP(0, 500);
-    if (tid == 0) { FZ_CSTAMP(2); FZ_CVAL(9, dq_tail); }
-    used_gu = n_mine;
-    used_dn = dq_tail;
+    if (tid == 0) { FZ_CSTAMP(2); FZ_CVAL(9, nsurv); }
+
+    // ---- second ring: the survivors, three at a time: (gated) their up rows complete the activations, then their down
+    //      rows, scaled, join the CTA's partial output (kept in registers) ------------------------------------------------
+    float yacc[CPT][8];
+#pragma unroll
+    for (int q = 0; q < CPT; ++q)
+#pragma unroll
+      for (int e = 0; e < 8; ++e) yacc[q][e] = 0.f;
+    int slot2 = 0;
+    unsigned wrap2 = 0;
+#pragma unroll 1
+    for (int q0 = 0; q0 < nsurv; q0 += FZ_NG) {
+      const int nb = min(FZ_NG, nsurv - q0);
+      int sl[FZ_NG];
+      float pu[FZ_NG];
+#pragma unroll
+      for (int e = 0; e < FZ_NG; ++e) {
+        pu[e] = 0.f;
+        sl[e] = slot2;
+        if (e < nb) {
+          mbar_wait(&s_bar[FZ_BAR_R2 + slot2], (s_phase[FZ_BAR_R2 + slot2] + wrap2) & 1u, A.status);
+          if (up_off >= 0) {
+            const uint16_t* urow = s_r2 + (size_t)slot2 * (A.n_mat - 1) * d;
+#pragma unroll
+            for (int q = 0; q < CPT; ++q) {
+              const int ch = tid + q * FZ_THREADS;
+              if (ch < nchunk) {
+                float w[8];
+                unpack8<WD>(*reinterpret_cast<const uint4*>(urow + ch * 8), w);
+#pragma unroll
+                for (int t = 0; t < 8; ++t) pu[e] = fmaf(w[t], xr[q][t], pu[e]);
+              }
+            }
+          }
+          if (++slot2 == G2) { slot2 = 0; ++wrap2; }
+        }
+      }
+      if (up_off >= 0) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+          for (int e = 0; e < FZ_NG; ++e) pu[e] += __shfl_xor_sync(0xffffffffu, pu[e], o);
+        }
+        float* red = s_red + ((q0 / FZ_NG) & 1) * (FZ_THREADS / 32) * 4;
+        if (lane == 0) *reinterpret_cast<float4*>(red + warp * 4) = make_float4(pu[0], pu[1], pu[2], 0.f);
+        named_bar_sync(1, FZ_THREADS);
+        if (warp == 0 && lane < nb) {
+          float v = 0.f;
+#pragma unroll 4
+          for (int w = 0; w < FZ_THREADS / 32; ++w) v += red[w * 4 + lane];
+          s_qa[q0 + lane] *= v * inv_rms;
+        }
+        named_bar_sync(1, FZ_THREADS);
+      }
+#pragma unroll
+      for (int e = 0; e < FZ_NG; ++e) {
+        if (e < nb) {
+          const float a = s_qa[q0 + e];
+          const uint16_t* row = s_r2 + (size_t)sl[e] * (A.n_mat - 1) * d + dn_off;
+#pragma unroll
+          for (int q = 0; q < CPT; ++q) {
+            const int ch = tid + q * FZ_THREADS;
+            if (ch < nchunk) {
+              float w[8];
+              unpack8<WD>(*reinterpret_cast<const uint4*>(row + ch * 8), w);
+#pragma unroll
+              for (int t = 0; t < 8; ++t) yacc[q][t] = fmaf(a, w[t], yacc[q][t]);
+            }
+          }
+        }
+      }
+      named_bar_sync(1, FZ_THREADS);  // every thread is done with the batch's slots: the producer may refill them
+      if (tid == 0) asm volatile("st.release.cta.shared.s32 [%0], %1;" ::"r"(smem_u32(&sh.done)), "r"(q0 + nb) : "memory");
+    }
+    used_r1 = n_mine;
+    used_r2 = nsurv;
     named_bar_sync(1, FZ_THREADS);  // nobody reads the rings any more: the producer may overwrite them
     if (tid == 0) asm volatile("st.release.cta.shared.s32 [%0], %1;" ::"r"(smem_u32(&s_round)), "r"(n_rounds + 1) : "memory");
     // the CTA's whole contribution to its stage, added once (vector reductions; order across CTAs is not fixed)
-    if (dq_tail > 0) {
+    if (nsurv > 0) {
       float* dst = A.dacc + (size_t)stage * d;
 #pragma unroll
       for (int q = 0; q < CPT; ++q) {
@@ -752,11 +1005,20 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
 #pragma unroll 1
     for (int li = tid; li < n_own; li += FZ_THREADS) s_pc[li] = A.pc ? A.pc[i_lo + li] : 0.f;
   }
+  if (tid >= 64 && tid < 67) {  // one line of every 2 MB page of the next layer's weights and predictor (this CTA's share)
+    const int i = tid - 64;
+    const char* p = static_cast<const char*>(A.pg_ptr[i]);
+    if (p) {
+#pragma unroll 1
+      for (unsigned long long off = (unsigned long long)cta << 21; off < A.pg_bytes[i]; off += (unsigned long long)G << 21)
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(p + off));
+    }
+  }
   if (tid >= 32 && tid < 36) {  // HBM is idle now: this CTA's share of what the next layer reads first goes to L2
     const int i = tid - 32;
     const unsigned bytes = A.pf_bytes[i] & ~15u;
     const char* p = static_cast<const char*>(A.pf_ptr[i]);
-    if (p && bytes) {
+    if (p && bytes && (reinterpret_cast<uintptr_t>(p) & 15) == 0) {
       const unsigned chunk = ((bytes + G - 1) / G + 127u) & ~127u, off = (unsigned)cta * chunk;
       if (off < bytes)
         asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p + off), "r"(min(chunk, bytes - off)) : "memory");
@@ -911,9 +1173,7 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
     // ============================ phase 3: scores of this CTA's neurons, every evaluation =============================
     double* s_zs = reinterpret_cast<double*>(smem + lay.zs_off);            // [max(EM, E)][fz_feat_stride(r)], un-normalised, blocked
     double* s_part = reinterpret_cast<double*>(smem + lay.part_off);        // [KSd][prow][per8], KSd * prow <= FZ_KS * FZ_EPAD
-    double* s_own = reinterpret_cast<double*>(smem + lay.own_off);          // [K+1][per]
-    uint16_t* s_bin = reinterpret_cast<uint16_t*>(smem + lay.bin_off);      // [K+1][per]
-    unsigned* s_coarse = reinterpret_cast<unsigned*>(smem + lay.coarse_off);  // [K+1][FZ_NC + 1] exclusive prefix
+    double* s_own = reinterpret_cast<double*>(smem + lay.own_off);          // [per] scores of the final evaluation
     const double bin_lo = __ldcg(&A.range[0]), bin_hi = __ldcg(&A.range[1]);
     const double INF = __longlong_as_double(0x7ff0000000000000LL);
     const double brange = bin_hi - bin_lo;
@@ -1027,65 +1287,34 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
     if (lane == 0) FZ_STAMP(1, 402 + warp * 4);
     named_bar_sync(1, FZ_THREADS);
     if (tid == 0) FZ_STAMP(1, 41);
-    // final scores, histogram (fine + coarse) and bucket insert: one thread per (evaluation, neuron), two entries at a
-    // time so that their atomics are in flight together; the coarse counts of the CTA are summed in shared memory first
-    // (they are hot addresses for the whole grid)
+    // final scores of this CTA's neurons, every evaluation: to global memory with their fine bin (one thread per
+    // (evaluation, neuron), no atomics); the exact selection is made per evaluation by ONE CTA after the next barrier
     {
-#pragma unroll 1
-      for (int t = tid; t < (K + 1) * FZ_NC; t += FZ_THREADS) s_ccnt[t] = 0u;
-      if (tid < FZ_MAXE) s_nsel[tid] = 0u;
-      named_bar_sync(1, FZ_THREADS);
       unsigned long long kmin = 0xffffffffffffffffULL, kmax = 0ULL;
       const int n_ent = E * n_own;
       double* const nprio = A.next_prio;
       double* const nscores = A.next_scores;
-      unsigned* const cnt_all = A.cnt;
-      uint4* const bent = A.bent;
-      uint4* const oent = A.oent;
+      double* const sc = A.sc;
+      uint16_t* const sb = A.sb;
 #pragma unroll 1
-      for (int t0 = 0; t0 < n_ent; t0 += 2 * FZ_THREADS) {
-        int jj[2], ll[2], bb[2];
-        unsigned slot[2];
-        unsigned long long key[2];
-        double sv[2];
-#pragma unroll
-        for (int u = 0; u < 2; ++u) {
-          const int t = t0 + u * FZ_THREADS + tid;
-          jj[u] = -1;
-          if (t < n_ent) {
-            const int j = t / n_own, li = t - j * n_own;
-            double v = 0.0;
+      for (int t = tid; t < n_ent; t += FZ_THREADS) {
+        const int j = t / n_own, li = t - j * n_own, i = i_lo + li;
+        double v = 0.0;
 #pragma unroll 4
-            for (int ks = 0; ks < KSd; ++ks) v += s_part[((size_t)ks * prow + j) * per8 + li];
-            v = canonical_score(v * s_inv[j] + (double)s_pc[li]);
-            const double sc = fmin(fmax(v, -1.7976931348623157e308), 1.7976931348623157e308);
-            int b = (int)((bin_hi - sc) * bscale);
-            b = max(0, min(FZ_NB - 1, b));
-            jj[u] = j; ll[u] = li; bb[u] = b; sv[u] = v; key[u] = ordered_key(v);
-            slot[u] = atomicAdd(&cnt_all[(size_t)j * FZ_CNT_STRIDE + b], 1u);
-          }
-        }
-#pragma unroll
-        for (int u = 0; u < 2; ++u) {
-          if (jj[u] >= 0) {
-            const int j = jj[u], li = ll[u], i = i_lo + li, b = bb[u];
-            s_own[(size_t)j * per + li] = sv[u];
-            s_bin[(size_t)j * per + li] = (uint16_t)b;
-            atomicAdd(&s_ccnt[j * FZ_NC + b / (FZ_NB / FZ_NC)], 1u);
-            const uint4 ent = make_uint4((unsigned)key[u], (unsigned)(key[u] >> 32), (unsigned)i, (unsigned)b);
-            if (slot[u] < (unsigned)FZ_CAPB) {
-              bent[((size_t)j * FZ_NB + b) * FZ_CAPB + slot[u]] = ent;
-            } else {
-              const unsigned o = atomicAdd(&cnt_all[(size_t)j * FZ_CNT_STRIDE + FZ_NB + FZ_NC], 1u);
-              oent[(size_t)j * Fn + o] = ent;
-            }
-            if (j == K) {
-              if (nprio) nprio[i] = sv[u];
-              if (nscores) nscores[i] = sv[u];
-              kmin = min(kmin, key[u]);
-              kmax = max(kmax, key[u]);
-            }
-          }
+        for (int ks = 0; ks < KSd; ++ks) v += s_part[((size_t)ks * prow + j) * per8 + li];
+        v = canonical_score(v * s_inv[j] + (double)s_pc[li]);
+        const double scl = fmin(fmax(v, -1.7976931348623157e308), 1.7976931348623157e308);
+        int b = (int)((bin_hi - scl) * bscale);
+        b = max(0, min(FZ_NB - 1, b));
+        sc[(size_t)j * Fn + i] = v;
+        sb[(size_t)j * Fn + i] = (uint16_t)b;
+        if (j == K) {
+          s_own[li] = v;  // kept for the speculation below
+          if (nprio) nprio[i] = v;
+          if (nscores) nscores[i] = v;
+          const unsigned long long key = ordered_key(v);
+          kmin = min(kmin, key);
+          kmax = max(kmax, key);
         }
       }
 #pragma unroll
@@ -1095,206 +1324,53 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
       }
       if (lane == 0) { s_kmm[warp] = kmin; s_kmm[16 + warp] = kmax; }
       named_bar_sync(1, FZ_THREADS);
-#pragma unroll 1
-      for (int t = tid; t < (K + 1) * FZ_NC; t += FZ_THREADS) {
-        const unsigned v = s_ccnt[t];
-        if (v) atomicAdd(&A.cnt[(size_t)(t / FZ_NC) * FZ_CNT_STRIDE + FZ_NB + (t % FZ_NC)], v);
-      }
-      if (tid == 0) {  // observed score range of the final evaluation: one pair of atomics per CTA
+      if (tid == 0) {  // observed score range of the final evaluation, this CTA's part (no atomics: the selecting CTA folds them)
 #pragma unroll 1
         for (int w = 1; w < 16; ++w) { kmin = min(kmin, s_kmm[w]); kmax = max(kmax, s_kmm[16 + w]); }
-        if (kmin <= kmax) {
-          atomicMin(&A.range_obs[0], kmin);
-          atomicMax(&A.range_obs[1], kmax);
-        }
+        A.kmm[2 * cta] = kmin;
+        A.kmm[2 * cta + 1] = kmax;
       }
     }
 
     // ---------------------------------------------------------------------------------------------- barrier 4 of 5
     if (tid == 0) FZ_STAMP(1, 4);
     if (tid == 0) FZ_CSTAMP(7);
-    grid_barrier(A, G);
+    // the exact selection is made per evaluation after the barrier: the final one by the first FZ_FIN_PARTS CTAs
+    // together (each ranks its share of the members), every earlier one by one CTA of its own
+    const int fparts = max(1, min(FZ_FIN_PARTS, G - K));
+    const bool selects = cta < fparts + K;
+    const int jme = cta < fparts ? K : cta - fparts;
+    named_bar_sync(1, FZ_THREADS);
+    if (tid == 0) {
+      grid_barrier_thread0(A, G);
+    } else if (tid >= 32 && A.spec_ptr && !selects) {
+      // While thread 0 waits for the grid: speculate.  The neurons this CTA scored highest in the final evaluation will
+      // most likely be in the refined set, which takes another grid barrier to establish; the first row of their bundles
+      // in the next layer is asked into L2 now, so that the next layer's ring fill finds it there.  A wrong guess costs
+      // bandwidth that is idle at this point, never correctness.
+      const int li = tid - 32;
+      if (li < n_own) {
+        const double v = s_own[li];
+        const int m_spec = (int)(((long long)keff * n_own * 9 / 8 + Fn - 1) / Fn) + 1;
+        int above = 0;
+#pragma unroll 1
+        for (int l2 = 0; l2 < n_own; ++l2) {
+          const double o = s_own[l2];
+          above += (o > v) || (o == v && l2 < li);
+        }
+        if (above < m_spec)
+          asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(A.spec_ptr + (size_t)(i_lo + li) * A.spec_stride), "r"(A.spec_bytes) : "memory");
+      }
+    }
+    named_bar_sync(1, FZ_THREADS);
     if (tid == 0) FZ_STAMP(1, 5);
 
-    // ============================ phase 4: refined sets of every evaluation, exact ranks of the final one ============
-    // Per evaluation (one warp each): coarse prefix -> the coarse bin holding rank keff -> its fine counts -> the CUT
-    // fine bin, the rank b0 where it starts and the threshold entry inside it (the last member).  With that in shared
-    // memory every neuron's membership is decided locally: bins before the cut bin are in, bins after it are out, the
-    // cut bin is split by one comparison.  Exact ranks (bucket comparisons) are needed only for the final selection.
-    constexpr int FPC = FZ_NB / FZ_NC;  // fine bins per coarse bin
-#pragma unroll 1
-    for (int j = warp; j <= K; j += FZ_THREADS / 32) {
-      const unsigned* cnt = A.cnt + (size_t)j * FZ_CNT_STRIDE;
-      const unsigned c0 = __ldcg(&cnt[FZ_NB + lane * 2]), c1 = __ldcg(&cnt[FZ_NB + lane * 2 + 1]);
-      unsigned incl = c0 + c1;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const unsigned t = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += t;
-      }
-      const unsigned ex = incl - (c0 + c1);
-      s_coarse[j * (FZ_NC + 1) + lane * 2] = ex;
-      s_coarse[j * (FZ_NC + 1) + lane * 2 + 1] = ex + c0;
-      if (lane == 31) s_coarse[j * (FZ_NC + 1) + FZ_NC] = incl;
-      // coarse bin that holds rank keff-1 (none when keff == 0)
-      int cbsel = -1;
-      if (c0 > 0 && (int)ex < keff && (int)(ex + c0) >= keff) cbsel = lane * 2;
-      if (c1 > 0 && (int)(ex + c0) < keff && (int)incl >= keff) cbsel = lane * 2 + 1;
-      const unsigned vote = __ballot_sync(0xffffffffu, cbsel >= 0);
-      int cut_bin = -1, cut_b0 = 0, cut_fallback = 0, t_idx = -1;  // no cut bin: keff == 0, nothing is selected
-      unsigned long long t_key = 0ULL;
-      if (vote) {
-        const int src = __ffs(vote) - 1;
-        const int cb = __shfl_sync(0xffffffffu, cbsel, src);
-        const unsigned cbase = __shfl_sync(0xffffffffu, (cbsel & 1) ? ex + c0 : ex, src);
-        // fine counts of that coarse bin: two per lane
-        const unsigned f0 = __ldcg(&cnt[cb * FPC + lane * 2]), f1 = __ldcg(&cnt[cb * FPC + lane * 2 + 1]);
-        unsigned fin = f0 + f1;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          const unsigned t = __shfl_up_sync(0xffffffffu, fin, o);
-          if (lane >= o) fin += t;
-        }
-        const unsigned fex = cbase + fin - (f0 + f1);
-        int fsel = -1;
-        unsigned fb0 = 0, fnb = 0;
-        if (f0 > 0 && (int)fex < keff && (int)(fex + f0) >= keff) { fsel = lane * 2; fb0 = fex; fnb = f0; }
-        if (f1 > 0 && (int)(fex + f0) < keff && (int)(fex + f0 + f1) >= keff) { fsel = lane * 2 + 1; fb0 = fex + f0; fnb = f1; }
-        const unsigned fvote = __ballot_sync(0xffffffffu, fsel >= 0);
-        const int fsrc = __ffs(fvote) - 1;  // exists: the coarse bin holds rank keff-1
-        cut_bin = cb * FPC + __shfl_sync(0xffffffffu, fsel, fsrc);
-        cut_b0 = (int)__shfl_sync(0xffffffffu, fb0, fsrc);
-        const int nbc = (int)__shfl_sync(0xffffffffu, fnb, fsrc);
-        const int cut_need = keff - cut_b0;  // members inside the cut bin, 1 <= need <= nbc
-        if (nbc > FZ_CAPB) {
-          cut_fallback = 1;        // overflowed bucket: its neurons compare against bucket + overflow list themselves
-        } else {
-          // threshold = the entry with exactly need-1 entries before it
-          uint4 ent = make_uint4(0, 0, 0, 0);
-          if (lane < nbc) ent = __ldcg(&A.bent[((size_t)j * FZ_NB + cut_bin) * FZ_CAPB + lane]);
-          const unsigned long long kmine = ((unsigned long long)ent.y << 32) | ent.x;
-          int before = 0;
-#pragma unroll 2
-          for (int q = 0; q < FZ_CAPB; ++q) {
-            const unsigned long long kq = ((unsigned long long)__shfl_sync(0xffffffffu, ent.y, q) << 32) | __shfl_sync(0xffffffffu, ent.x, q);
-            const int iq = (int)__shfl_sync(0xffffffffu, ent.z, q);
-            before += (q < nbc) && ((kq > kmine) || (kq == kmine && iq < (int)ent.z));
-          }
-          const unsigned tv = __ballot_sync(0xffffffffu, lane < nbc && before == cut_need - 1);
-          const int ts = __ffs(tv) - 1;
-          t_key = ((unsigned long long)__shfl_sync(0xffffffffu, ent.y, ts) << 32) | __shfl_sync(0xffffffffu, ent.x, ts);
-          t_idx = (int)__shfl_sync(0xffffffffu, ent.z, ts);
-        }
-      }
-      if (lane == 0) {
-        s_cut[j * 4 + 0] = cut_bin;
-        s_cut[j * 4 + 1] = cut_b0;
-        s_cut[j * 4 + 2] = t_idx;
-        s_cut[j * 4 + 3] = cut_fallback;
-        s_cutkey[j] = t_key;
-      }
-    }
-    named_bar_sync(1, FZ_THREADS);
-    if (tid == 0) FZ_STAMP(1, 60);
-    {
-      // intermediate evaluations: membership only (bins before the cut bin are in, the cut bin is split by the threshold)
-      uint32_t* const trm = A.tr_masks;
-      const int nwn = (Fn + 31) >> 5;
-#pragma unroll 1
-      for (int t = tid; t < K * n_own; t += FZ_THREADS) {
-        const int j = t / n_own, li = t - j * n_own, i = i_lo + li;
-        const int bb = s_bin[(size_t)j * per + li];
-        const int cut_bin = s_cut[j * 4 + 0];
-        if (bb > cut_bin) continue;  // behind the cut
-        bool member = true;
-        if (bb == cut_bin) {
-          const unsigned long long kp = ordered_key(s_own[(size_t)j * per + li]);
-          if (!s_cut[j * 4 + 3]) {
-            const unsigned long long tk = s_cutkey[j];
-            member = (kp > tk) || (kp == tk && i <= s_cut[j * 4 + 2]);
-          } else {
-            member = fz_rank_in_overflowed_bin(A, j, bb, i, kp, s_coarse[j * (FZ_NC + 1) + bb / FPC]) < keff;
-          }
-        }
-        if (member) {
-          if (trm) atomicOr(&trm[(size_t)j * nwn + (i >> 5)], 1u << (i & 31));
-          atomicAdd(&s_nsel[j], 1u);
-        }
-      }
-    }
-    // Final evaluation: exact ranks, bin by bin.  A task is a pair of fine bins; the tasks up to the cut are dealt to
-    // the warps of the whole grid.  A half-warp takes one fine bin: its bucket arrives with one
-    // coalesced load, the order inside the bin comes from 16 shuffles, rank = first rank of the bin + entries before.
-    {
-      const int j = K;
-      const unsigned* cnt = A.cnt + (size_t)j * FZ_CNT_STRIDE;
-      const int cut_bin = s_cut[j * 4 + 0];
-      const int n_task = cut_bin >= 0 ? (cut_bin / 2 + 1) : 0;  // one task = two fine bins (one per half-warp)
-      const int h = lane >> 4, l16 = lane & 15;
-      int32_t* const nidx = A.next_idx;
-      uint32_t* const nmask = A.next_mask;
-      uint32_t* const trm = A.tr_masks;
-      const int ncap = A.next_cap, nwn = (Fn + 31) >> 5;
-      const uint4* const bent = A.bent + (size_t)j * FZ_NB * FZ_CAPB;
-      unsigned found = 0;
-      // task t goes to CTA t % G, warp (t / G) % 16: spread over the whole grid, at most a few per warp
-#pragma unroll 1
-      for (int task = cta + warp * G; task < n_task; task += G * (FZ_THREADS / 32)) {
-        const int fbq = task * 2, cb = fbq / FPC;  // first fine bin of the task, its coarse bin
-        // fine counts of the coarse bin (two per lane) and their exclusive prefix
-        const unsigned f0 = __ldcg(&cnt[cb * FPC + lane * 2]), f1 = __ldcg(&cnt[cb * FPC + lane * 2 + 1]);
-        // this half-warp's bucket, fetched before its first rank is known (the counts arrive at the same time)
-        const int bin = fbq + h;
-        uint4 ent = __ldcg(&bent[(size_t)bin * FZ_CAPB + l16]);
-        unsigned fin = f0 + f1;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          const unsigned t = __shfl_up_sync(0xffffffffu, fin, o);
-          if (lane >= o) fin += t;
-        }
-        const unsigned fex = s_coarse[j * (FZ_NC + 1) + cb] + fin - (f0 + f1);  // first rank of fine bin cb*64 + 2*lane
-        const int src = (bin - cb * FPC) >> 1, odd = (bin - cb * FPC) & 1;
-        const unsigned pf0 = __shfl_sync(0xffffffffu, f0, src), pf1 = __shfl_sync(0xffffffffu, f1, src);
-        const unsigned pex = __shfl_sync(0xffffffffu, fex, src);
-        const unsigned b0 = odd ? pex + pf0 : pex, nball = odd ? pf1 : pf0;
-        const int nb = (int)min(nball, (unsigned)FZ_CAPB);
-        if (l16 >= nb) ent = make_uint4(0, 0, 0, 0);  // stale bucket slots are ignored
-        const unsigned long long kmine = ((unsigned long long)ent.y << 32) | ent.x;
-        int before = 0;
-#pragma unroll 2
-        for (int q = 0; q < FZ_CAPB; ++q) {
-          const unsigned long long kq = ((unsigned long long)__shfl_sync(0xffffffffu, ent.y, q, 16) << 32) | __shfl_sync(0xffffffffu, ent.x, q, 16);
-          const int iq = (int)__shfl_sync(0xffffffffu, ent.z, q, 16);
-          before += (q < nb) && ((kq > kmine) || (kq == kmine && iq < (int)ent.z));
-        }
-        if ((int)b0 >= keff) continue;  // (uniform per half-warp; the shuffles above were executed by all lanes)
-        if (nball > (unsigned)FZ_CAPB) before += fz_final_overflowed_bin(A, j, bin, b0, ent, l16, keff, &s_nsel[j]);
-        const int rank = (int)b0 + before;
-        if (l16 < nb && rank < keff) {
-          const int i = (int)ent.z;
-          if (rank < ncap) nidx[rank] = i;
-          if (nmask) atomicOr(&nmask[i >> 5], 1u << (i & 31));
-          if (trm) atomicOr(&trm[(size_t)j * nwn + (i >> 5)], 1u << (i & 31));
-          ++found;
-        }
-      }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) found += __shfl_xor_sync(0xffffffffu, found, o);
-      if (lane == 0 && found) atomicAdd(&s_nsel[j], found);
-    }
-    if (lane == 0) FZ_STAMP(1, 103 + warp * 4);
-    named_bar_sync(1, FZ_THREADS);
-    // refined-set sizes: every evaluation must have selected exactly keff neurons (checked on the device)
-#pragma unroll 1
-    for (int j = tid; j <= K; j += FZ_THREADS)
-      if (s_nsel[j]) atomicAdd(&A.nsel[j], s_nsel[j]);
-    if (cta == 0 && tid == 0) {
-      if (A.tr_counts)
-#pragma unroll 1
-        for (int j = 0; j <= K; ++j) A.tr_counts[j] = keff;
-      *A.next_count = min(keff, A.next_cap);
-      if (keff > A.next_cap) set_status(A.status, ST_CAPACITY);
-    }
+    // ============================ phase 4: the refined set of evaluation j, selected by one CTA =======================
+    // Evaluation j belongs to CTA j * G / E.  The CTA histograms the fine bins of all Fn scores (shared-memory atomics),
+    // scans them, finds the CUT bin (the one holding rank keff - 1): bins before it are in, bins after it are out, the
+    // cut bin is split by exact comparison of its few entries.  The final evaluation also needs every member's exact
+    // rank: members are scattered bin by bin into a scratch array and ranked against the other entries of their bin.
+    if (selects) fz_select<WD>(A, jme, K, keff, lay.sel_off, cta < fparts ? cta : 0, cta < fparts ? fparts : 1);
     if (tid == 0) FZ_STAMP(1, 6);
     if (tid == 0) FZ_CSTAMP(11);
   }
@@ -1302,8 +1378,8 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
   named_bar_sync(1, FZ_THREADS);
   if (tid < FZ_NBAR) {
     unsigned n = 0;
-    if (tid < FZ_MAX_DEPTH) n = used_gu > tid ? (unsigned)((used_gu - 1 - tid) / GU + 1) : 0u;
-    else if (tid < FZ_BAR_A) { const int sdn = tid - FZ_BAR_DN; n = used_dn > sdn ? (unsigned)((used_dn - 1 - sdn) / DN + 1) : 0u; }
+    if (tid < FZ_MAX_G1) n = used_r1 > tid ? (unsigned)((used_r1 - 1 - tid) / G1 + 1) : 0u;
+    else if (tid < FZ_BAR_A) { const int s2 = tid - FZ_BAR_R2; n = used_r2 > s2 ? (unsigned)((used_r2 - 1 - s2) / G2 + 1) : 0u; }
     else n = A.has_next ? 1u : 0u;
     s_phase[tid] += n;
   }
@@ -1312,42 +1388,12 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
 
 }
 
-// Binning range of a layer's scores for its next launch: what the final evaluation observed, widened by 5 % per side.
-__device__ inline void fused_update_range(const FusedArgs& A) {
-  const unsigned long long kmin = A.range_obs[0], kmax = A.range_obs[1];
-  if (kmin <= kmax) {
-    auto unkey = [](unsigned long long k) {
-      const unsigned long long b = (k >> 63) ? (k & 0x7fffffffffffffffULL) : ~k;
-      return __longlong_as_double((long long)b);
-    };
-    double lo = unkey(kmin), hi = unkey(kmax);
-    lo = fmax(lo, -1.0e300);
-    hi = fmin(hi, 1.0e300);
-    const double pad = 0.05 * (hi - lo);
-    A.range[0] = lo - pad;
-    A.range[1] = hi + pad;
-  }
-  A.range_obs[0] = 0xffffffffffffffffULL;
-  A.range_obs[1] = 0ULL;
-}
-
-// Zeroes the slice [part, parts) of what a layer step dirtied in the scratch (compute threads only); part 0 also runs the
-// self-check of the refined-set sizes and the range update.  The caller guarantees that every CTA is done with the layer.
+// Zeroes the slice [part, parts) of the stage accumulators a layer step dirtied (compute threads only).  The caller
+// guarantees that every CTA is done with the layer.
 __device__ inline void fused_clean(const FusedArgs& A, int part, int parts) {
   const int tid = threadIdx.x;
 #pragma unroll 1
   for (int t = part * FZ_THREADS + tid; t < A.K * A.d; t += parts * FZ_THREADS) A.dacc[t] = 0.f;
-  if (A.has_next) {
-#pragma unroll 1
-    for (int t = part * FZ_THREADS + tid; t < (A.K + 1) * FZ_CNT_STRIDE; t += parts * FZ_THREADS) A.cnt[t] = 0u;
-    if (part == 0) {
-      if (tid <= A.K) {  // self-check: every refined set has exactly min(k_next, d_ff) members
-        if ((int)__ldcg(&A.nsel[tid]) != min(A.k_next, A.Fn)) set_status(A.status, ST_INTERNAL);
-        A.nsel[tid] = 0u;
-      }
-      if (tid == 0) fused_update_range(A);
-    }
-  }
 }
 
 // ---- one launch per layer step: the last CTA to finish restores the zero-on-entry invariants of the scratch
