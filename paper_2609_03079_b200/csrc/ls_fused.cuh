@@ -28,7 +28,8 @@ namespace ls {
 
 constexpr int FZ_THREADS = 512;        // compute threads (16 warps)
 constexpr int FZ_BLOCK = FZ_THREADS + 32;  // plus the producer warp
-constexpr int FZ_NG = 3;          // neurons processed per round
+constexpr int FZ_NG = 3;          // survivors processed per batch of the second ring
+constexpr int FZ_NG1 = 16;        // most neurons per round of the first ring
 constexpr int FZ_NB = 4096;       // fine score bins per evaluation
 constexpr int FZ_FIN_PARTS = 8;   // CTAs that share the ranking of the final evaluation
 constexpr int FZ_CUTLIST = 1024;  // entries of the cut bin ranked in shared memory (a fuller bin falls back to global loops)
@@ -36,7 +37,7 @@ constexpr int FZ_CCAP = 4096;     // members grouped in shared memory (more: in 
 constexpr int FZ_MAXK = 16;       // stages supported by the fused path
 constexpr int FZ_MAXE = FZ_MAXK + 1;  // evaluations j = 0..K
 constexpr int FZ_MAX_G1 = 16;     // most slots of the first ring (first row of a bundle); depths are chosen per launch
-constexpr int FZ_MAX_G2 = 8;      // most slots of the second ring (the rest of a survivor's bundle)
+constexpr int FZ_MAX_G2 = 16;     // most slots of the second ring (the rest of a survivor's bundle), carved slots included
 constexpr int FZ_SL = 32;         // columns of the feature handled as one slice in the latent phase
 constexpr int FZ_EPAD = 18;       // rows kept per evaluation-indexed buffer: at most two MMA tiles, or FZ_MAXE rows
 constexpr int FZ_KS = 4;          // column splits of a score tile (more independent tasks than warps)
@@ -56,7 +57,7 @@ struct FusedSmemLayout {
   // ... and, in the same bytes once the rings have drained, the operands and results of the refinement
   unsigned b_off, zs_off, part_off, own_off, sel_off;
   unsigned total;
-  int per, ns_cta, a_alias, g1, g2;
+  int per, ns_cta, a_alias, g1, g2, g2x;  // g2x: extra second-ring slots carved from the first ring once it is idle
 };
 
 struct alignas(16) FusedArgs {  // (an array of these is prefetched with 16-byte granularity)
@@ -298,6 +299,10 @@ inline FusedSmemLayout fused_layout(int d, int n_mat, int r, int Fn, int G, int 
   FusedSmemLayout L{};
   L.g1 = g1;
   L.g2 = g2;
+  {
+    const long long extra = ((long long)g1 * d * 2) / ((long long)(n_mat - 1) * d * 2);
+    L.g2x = (int)(extra < FZ_MAX_G2 - g2 ? extra : FZ_MAX_G2 - g2);
+  }
   L.a_alias = a_alias;
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t at = o; o += (bytes + 127) & ~(size_t)127; return (unsigned)at; };
@@ -306,7 +311,7 @@ inline FusedSmemLayout fused_layout(int d, int n_mat, int r, int Fn, int G, int 
   L.ns_cta = (nsl + G - 1) / G;
   const size_t a_bytes = has_next ? (size_t)L.ns_cta * r * FZ_SL * 2 : 0;
   L.bar_off = take(FZ_NBAR * 8);
-  L.red_off = take(2 * 16 * 8 * 4);                  // stream dot partials, double-buffered: [2][warp][8]
+  L.red_off = take(2 * 16 * FZ_NG1 * 4);             // stream dot partials, double-buffered: [2][warp][FZ_NG1]
   L.redd_off = take(32 * 8);                         // fp64 partials of block reductions
   L.mine_off = take((size_t)FZ_MAX_MINE * 16);       // this CTA's neurons, their gate biases; the survivors, their activations
   L.pc_off = take((size_t)L.per * 4);
@@ -663,7 +668,7 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
   const int lane = tid & 31, warp = tid >> 5;
   const int d = A.d, K = A.K, nchunk = A.d >> 3;
   const FusedSmemLayout& lay = A.lay;
-  const int G1 = lay.g1, G2 = lay.g2;
+  const int G1 = lay.g1, G2 = lay.g2, G2T = lay.g2 + lay.g2x, NG1 = min(FZ_NG1, lay.g1);
   uint16_t* s_r1 = reinterpret_cast<uint16_t*>(smem + lay.r1_off);  // [G1][d]
   uint16_t* s_r2 = reinterpret_cast<uint16_t*>(smem + lay.r2_off);  // [G2][(n_mat - 1) d]
   uint64_t* s_bar = reinterpret_cast<uint64_t*>(smem + lay.bar_off);  // "full" barriers: gate/up slots, down slots, A, B^T
@@ -715,7 +720,7 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
     const int lo = min(count, stage * m), hi = min(count, (stage + 1) * m);
     const int first = lo + (cta - g_lo);
     const int n_mine = first < hi ? (hi - first + gsize - 1) / gsize : 0;
-    const int n_rounds = (n_mine + FZ_NG - 1) / FZ_NG;
+    const int n_rounds = (n_mine + NG1 - 1) / NG1;
     const uint32_t r1_bytes = (uint32_t)d * 2, r2_bytes = (uint32_t)(A.n_mat - 1) * d * 2;
     const size_t bundle_elems = (size_t)A.n_mat * d;
     const int up_off = A.gated ? 0 : -1, dn_off = A.gated ? d : 0;  // where the rows sit inside a second-ring slot
@@ -770,7 +775,7 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
         const long long t0 = clock64();
         while (true) {
           // top the first ring up to the rows that may be in flight
-          const int want = min(n_mine, rounds * FZ_NG + G1);
+          const int want = min(n_mine, rounds * NG1 + G1);
 #pragma unroll 1
           for (; issued1 < want; ++issued1) {
             int i = s_myidx[issued1];
@@ -788,13 +793,15 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
           int done;
           asm volatile("ld.acquire.cta.shared.s32 %0, [%1];" : "=r"(done) : "r"(smem_u32(&sh.done)) : "memory");
 #pragma unroll 1
-          for (; issued2 < nsurv && issued2 - done < G2; ++issued2) {
+          for (; issued2 < nsurv && issued2 - done < G2T; ++issued2) {
+            if (slot2 >= G2 && rounds < n_rounds) break;  // slots carved from the first ring: only once it is idle
             const int i = s_surv[issued2];
             uint64_t* bar = &s_bar[FZ_BAR_R2 + slot2];
+            uint16_t* dst = slot2 < G2 ? s_r2 + (size_t)slot2 * (A.n_mat - 1) * d : s_r1 + (size_t)(slot2 - G2) * (A.n_mat - 1) * d;
             mbar_expect_tx(bar, r2_bytes);
-            tma_load_1d(s_r2 + (size_t)slot2 * (A.n_mat - 1) * d, A.bundles + (size_t)i * bundle_elems + d, r2_bytes, bar);
+            tma_load_1d(dst, A.bundles + (size_t)i * bundle_elems + d, r2_bytes, bar);
             if (A.tr_survive) atomicOr(&A.tr_survive[i >> 5], 1u << (i & 31));
-            if (++slot2 == G2) slot2 = 0;
+            if (++slot2 == G2T) slot2 = 0;
           }
           if (rounds == n_rounds && issued2 == nsurv) break;  // every row of this layer has been requested
           // wait for news: a round finished (more survivors, room in the first ring) or survivors consumed
@@ -836,42 +843,36 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
     if (tid == 0) FZ_STAMP(0, 0);
     if (tid == 0) { FZ_CSTAMP(1); FZ_CVAL(8, n_mine); FZ_CVAL(10, stage); }
 
-    // ---- first ring: the pre-activation of every neuron, three neurons per round; survivors go to the producer -------
+    // ---- first ring: the pre-activation of every neuron, a ring-full of neurons per round; survivors go to the producer -
     int nsurv = 0, slot1 = 0;
     unsigned wrap1 = 0;
 #pragma unroll 1
     for (int rd = 0; rd < n_rounds; ++rd) {
-      const int it0 = rd * FZ_NG;
-      const int nn = min(FZ_NG, n_mine - it0);
+      const int it0 = rd * NG1;
+      const int nn = min(NG1, n_mine - it0);
       if (tid == 0) FZ_STAMP(0, 1 + rd * 4);
-      float pg[FZ_NG];
+      float* red = s_red + (rd & 1) * (FZ_THREADS / 32) * FZ_NG1;  // [warp][FZ_NG1]
+#pragma unroll 1
+      for (int e = 0; e < nn; ++e) {  // (a rolled loop: each neuron's dot product is a few dozen instructions, fetched once)
+        mbar_wait(&s_bar[slot1], (s_phase[slot1] + wrap1) & 1u, A.status);
+        const uint16_t* grow = s_r1 + (size_t)slot1 * d;
+        float pg = 0.f;
 #pragma unroll
-      for (int e = 0; e < FZ_NG; ++e) {
-        pg[e] = 0.f;
-        if (e < nn) {
-          mbar_wait(&s_bar[slot1], (s_phase[slot1] + wrap1) & 1u, A.status);
-          const uint16_t* grow = s_r1 + (size_t)slot1 * d;
+        for (int q = 0; q < CPT; ++q) {
+          const int ch = tid + q * FZ_THREADS;
+          if (ch < nchunk) {
+            float w[8];
+            unpack8<WD>(*reinterpret_cast<const uint4*>(grow + ch * 8), w);
 #pragma unroll
-          for (int q = 0; q < CPT; ++q) {
-            const int ch = tid + q * FZ_THREADS;
-            if (ch < nchunk) {
-              float w[8];
-              unpack8<WD>(*reinterpret_cast<const uint4*>(grow + ch * 8), w);
-#pragma unroll
-              for (int t = 0; t < 8; ++t) pg[e] = fmaf(w[t], xr[q][t], pg[e]);
-            }
+            for (int t = 0; t < 8; ++t) pg = fmaf(w[t], xr[q][t], pg);
           }
-          if (++slot1 == G1) { slot1 = 0; ++wrap1; }
         }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) pg += __shfl_xor_sync(0xffffffffu, pg, o);
+        if (lane == 0) red[warp * FZ_NG1 + e] = pg;
+        if (++slot1 == G1) { slot1 = 0; ++wrap1; }
       }
       if (tid == 0) FZ_STAMP(0, 2 + rd * 4);
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-#pragma unroll
-        for (int e = 0; e < FZ_NG; ++e) pg[e] += __shfl_xor_sync(0xffffffffu, pg[e], o);
-      }
-      float* red = s_red + (rd & 1) * (FZ_THREADS / 32) * 4;  // [warp][4]
-      if (lane == 0) *reinterpret_cast<float4*>(red + warp * 4) = make_float4(pg[0], pg[1], pg[2], 0.f);
       named_bar_sync(1, FZ_THREADS);  // partials visible; every thread is done with the round's ring slots
       if (warp == 0) {  // pre-activations; the neurons that survive the ReLU join the list the producer fetches from
         float a = 0.f;
@@ -879,7 +880,7 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
         if (lane < nn) {
           float v = 0.f;
 #pragma unroll 4
-          for (int w = 0; w < FZ_THREADS / 32; ++w) v += red[w * 4 + lane];
+          for (int w = 0; w < FZ_THREADS / 32; ++w) v += red[w * FZ_NG1 + lane];
           i = s_myidx[it0 + lane];
           a = fmaxf(v * inv_rms + s_mybias[it0 + lane], 0.f);
           if (i < 0) a = 0.f;
@@ -890,15 +891,18 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
           s_surv[pos] = i;
           s_qa[pos] = a;
         }
+        nsurv += __popc(surv);
         if (lane == 0) {
-          asm volatile("st.release.cta.shared.s32 [%0], %1;" ::"r"(smem_u32(&sh.nsurv)), "r"(nsurv + __popc(surv)) : "memory");
+          asm volatile("st.release.cta.shared.s32 [%0], %1;" ::"r"(smem_u32(&sh.nsurv)), "r"(nsurv) : "memory");
           asm volatile("st.release.cta.shared.s32 [%0], %1;" ::"r"(smem_u32(&s_round)), "r"(rd + 1) : "memory");
         }
+        if (tid == 0) FZ_STAMP(0, 3 + rd * 4);
       }
-      named_bar_sync(1, FZ_THREADS);
-      nsurv = sh.nsurv;
-      if (tid == 0) FZ_STAMP(0, 3 + rd * 4);
+      // (no second barrier: the partials are double-buffered, and warp 0 joins the next round's barrier only after it has
+      // read this round's)
     }
+    named_bar_sync(1, FZ_THREADS);
+    nsurv = sh.nsurv;
     if (tid == 0) FZ_STAMP(0, 500);
     if (tid == 0) { FZ_CSTAMP(2); FZ_CVAL(9, nsurv); }
 
@@ -923,7 +927,7 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
         if (e < nb) {
           mbar_wait(&s_bar[FZ_BAR_R2 + slot2], (s_phase[FZ_BAR_R2 + slot2] + wrap2) & 1u, A.status);
           if (up_off >= 0) {
-            const uint16_t* urow = s_r2 + (size_t)slot2 * (A.n_mat - 1) * d;
+            const uint16_t* urow = (slot2 < G2 ? s_r2 + (size_t)slot2 * (A.n_mat - 1) * d : s_r1 + (size_t)(slot2 - G2) * (A.n_mat - 1) * d);
 #pragma unroll
             for (int q = 0; q < CPT; ++q) {
               const int ch = tid + q * FZ_THREADS;
@@ -935,7 +939,7 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
               }
             }
           }
-          if (++slot2 == G2) { slot2 = 0; ++wrap2; }
+          if (++slot2 == G2T) { slot2 = 0; ++wrap2; }
         }
       }
       if (up_off >= 0) {
@@ -959,7 +963,7 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
       for (int e = 0; e < FZ_NG; ++e) {
         if (e < nb) {
           const float a = s_qa[q0 + e];
-          const uint16_t* row = s_r2 + (size_t)sl[e] * (A.n_mat - 1) * d + dn_off;
+          const uint16_t* row = (sl[e] < G2 ? s_r2 + (size_t)sl[e] * (A.n_mat - 1) * d : s_r1 + (size_t)(sl[e] - G2) * (A.n_mat - 1) * d) + dn_off;
 #pragma unroll
           for (int q = 0; q < CPT; ++q) {
             const int ch = tid + q * FZ_THREADS;
@@ -1379,7 +1383,7 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
   if (tid < FZ_NBAR) {
     unsigned n = 0;
     if (tid < FZ_MAX_G1) n = used_r1 > tid ? (unsigned)((used_r1 - 1 - tid) / G1 + 1) : 0u;
-    else if (tid < FZ_BAR_A) { const int s2 = tid - FZ_BAR_R2; n = used_r2 > s2 ? (unsigned)((used_r2 - 1 - s2) / G2 + 1) : 0u; }
+    else if (tid < FZ_BAR_A) { const int s2 = tid - FZ_BAR_R2; n = used_r2 > s2 ? (unsigned)((used_r2 - 1 - s2) / G2T + 1) : 0u; }
     else n = A.has_next ? 1u : 0u;
     s_phase[tid] += n;
   }
