@@ -853,24 +853,38 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
       if (tid == 0) FZ_STAMP(0, 1 + rd * 4);
       float* red = s_red + (rd & 1) * (FZ_THREADS / 32) * FZ_NG1;  // [warp][FZ_NG1]
 #pragma unroll 1
-      for (int e = 0; e < nn; ++e) {  // (a rolled loop: each neuron's dot product is a few dozen instructions, fetched once)
-        mbar_wait(&s_bar[slot1], (s_phase[slot1] + wrap1) & 1u, A.status);
-        const uint16_t* grow = s_r1 + (size_t)slot1 * d;
-        float pg = 0.f;
+      for (int e0 = 0; e0 < nn; e0 += 4) {  // four neurons at a time: four independent chains of loads, FMAs and shuffles
+        const uint16_t* grow[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          grow[u] = s_r1 + (size_t)slot1 * d;
+          if (e0 + u < nn) {
+            mbar_wait(&s_bar[slot1], (s_phase[slot1] + wrap1) & 1u, A.status);
+            if (++slot1 == G1) { slot1 = 0; ++wrap1; }
+          }
+        }
+        float pg[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int q = 0; q < CPT; ++q) {
           const int ch = tid + q * FZ_THREADS;
           if (ch < nchunk) {
-            float w[8];
-            unpack8<WD>(*reinterpret_cast<const uint4*>(grow + ch * 8), w);
 #pragma unroll
-            for (int t = 0; t < 8; ++t) pg = fmaf(w[t], xr[q][t], pg);
+            for (int u = 0; u < 4; ++u) {
+              if (e0 + u < nn) {
+                float w[8];
+                unpack8<WD>(*reinterpret_cast<const uint4*>(grow[u] + ch * 8), w);
+#pragma unroll
+                for (int t = 0; t < 8; ++t) pg[u] = fmaf(w[t], xr[q][t], pg[u]);
+              }
+            }
           }
         }
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) pg += __shfl_xor_sync(0xffffffffu, pg, o);
-        if (lane == 0) red[warp * FZ_NG1 + e] = pg;
-        if (++slot1 == G1) { slot1 = 0; ++wrap1; }
+        for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+          for (int u = 0; u < 4; ++u) pg[u] += __shfl_xor_sync(0xffffffffu, pg[u], o);
+        }
+        if (lane == 0) *reinterpret_cast<float4*>(red + warp * FZ_NG1 + e0) = make_float4(pg[0], pg[1], pg[2], pg[3]);
       }
       if (tid == 0) FZ_STAMP(0, 2 + rd * 4);
       named_bar_sync(1, FZ_THREADS);  // partials visible; every thread is done with the round's ring slots
@@ -1355,15 +1369,18 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
       const int li = tid - 32;
       if (li < n_own) {
         const double v = s_own[li];
-        const int m_spec = (int)(((long long)keff * n_own * 9 / 8 + Fn - 1) / Fn) + 1;
+        const int m_spec = (int)(((long long)keff * n_own * 3 / 2 + Fn - 1) / Fn) + 1;  // half again this CTA's fair share: a round waits for its slowest row
         int above = 0;
 #pragma unroll 1
         for (int l2 = 0; l2 < n_own; ++l2) {
           const double o = s_own[l2];
           above += (o > v) || (o == v && l2 < li);
         }
+        // The score estimates the gate pre-activation (B is W_gate A, c the gate bias): a likely member with a positive
+        // score will probably survive the ReLU too, so the rest of its bundle (up and down rows) is asked for as well.
         if (above < m_spec)
-          asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(A.spec_ptr + (size_t)(i_lo + li) * A.spec_stride), "r"(A.spec_bytes) : "memory");
+          asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(A.spec_ptr + (size_t)(i_lo + li) * A.spec_stride),
+                       "r"(v > 0.0 ? (unsigned)A.spec_stride : A.spec_bytes) : "memory");
       }
     }
     named_bar_sync(1, FZ_THREADS);
