@@ -124,7 +124,6 @@ struct ls_layer {
 
   // per-layer state of the fused kernel; its working scratch is shared per device (DeviceScratch below)
   double* fz_range = nullptr;                  // [2] binning range of this layer's scores (observed by its last launch)
-  unsigned long long* fz_range_obs = nullptr;  // [2]
 
   ls::CacheState cache;  // residency tables, pinned backing store, copy stream
 };
@@ -163,7 +162,7 @@ void free_layer(ls_layer* L) {
   cudaFree(L->bundles); cudaFree(L->b_gate); cudaFree(L->b_down); cudaFree(L->pred_at); cudaFree(L->pred_at_sl); cudaFree(L->pred_bt);
   cudaFree(L->pred_c); cudaFree(L->z); cudaFree(L->sumsq); cudaFree(L->scores); cudaFree(L->prio); cudaFree(L->cand_key);
   cudaFree(L->cand_idx); cudaFree(L->umask); cudaFree(L->tmp_idx); cudaFree(L->tmp_count); cudaFree(L->tmp_mask);
-  cudaFree(L->fz_range); cudaFree(L->fz_range_obs);
+  cudaFree(L->fz_range);
   cudaFree(L->xin); cudaFree(L->xt); cudaFree(L->actv); cudaFree(L->ypart); cudaFree(L->survive); cudaFree(L->status);
   delete L;
 }
@@ -301,11 +300,8 @@ int32_t create_impl(const ls_layer_desc* D, ls_layer* L) {
   if (L->cache_rows == 0) {
     LS_TRY(device_scratch(D->device, nullptr));
     LS_TRY(dalloc(&L->fz_range, 2));
-    LS_TRY(dalloc(&L->fz_range_obs, 2));
     const double zr[2] = {-1.0, 1.0};  // binning range until a launch has observed one
     LS_CUDA(cudaMemcpy(L->fz_range, zr, sizeof zr, cudaMemcpyHostToDevice));
-    const unsigned long long ro[2] = {0xffffffffffffffffULL, 0ULL};
-    LS_CUDA(cudaMemcpy(L->fz_range_obs, ro, sizeof ro, cudaMemcpyHostToDevice));
   }
   // opt in to the large dynamic shared memory the kernels may ask for
   const int big = 200 * 1024;

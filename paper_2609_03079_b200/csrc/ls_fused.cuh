@@ -1,26 +1,35 @@
-// One kernel per layer step for the all-resident, batch-1 case (the decode hot path).
+// One kernel per layer step (or per token: all layers of a resident stack) for the all-resident, batch-1 case: the
+// decode hot path.  16 compute warps and one producer warp per CTA, one CTA per SM, cooperatively launched.
 //
-// Grid barriers cost far more on this machine than any of the small predictor phases, so the step is organised to need
-// only three of them, whatever the number of stages K:
+// A layer step has five phases separated by grid barriers (a barrier costs about 2,700 SM clocks here, more than most of
+// the phases' arithmetic, so the phases are organised around needing as few as possible):
 //
 //   1. stream   The K priority stages of the layer (Eq. 1) run CONCURRENTLY on K disjoint groups of CTAs (the output is
 //               a sum over hidden neurons, so stage order in time is free; only stage membership defines the partial
-//               features).  A CTA takes three neurons per round: gate+up rows arrive by 1-D TMA bulk copies into a
-//               shared-memory ring, the block reduces the dot products, surviving neurons fetch their down row into a
-//               second ring, and the CTA's whole contribution to its stage is kept in registers and added once to the
-//               stage accumulator (vector reductions).  The CTA's share of the next layer's predictor (rows of A^T and
-//               of B^T) arrives in shared memory by bulk copies issued at the start.
+//               features).  Every bundle is [gate | up | down] rows of one neuron.  The producer warp brings the GATE
+//               rows of the CTA's neurons into a first shared-memory ring by 1-D bulk copies (TMA), all at once when they
+//               fit; the compute warps form the pre-activations; only the neurons that survive the ReLU have the rest of
+//               their bundle (up and down rows) fetched into a second ring, their activation completed and their down
+//               row, scaled, added to the CTA's partial output, which is kept in registers and added once to the stage
+//               accumulator (vector reductions).
 //      -- barrier --
-//   2. latent   Every partial residual feature x~^(j) = x + sum_{c<j} dm^(c), j = 0..K (Eq. 2), is rebuilt on the fly
-//               from the stage accumulators, and this CTA's rows of all K+1 latents z^(j) = A^T x~^(j) are formed in one
-//               pass (fp64), each weight converted once and used K+1 times.
+//   2. latent   The feature is cut into slices of 32 columns, one per CTA.  The owner rebuilds the K+1 partial residual
+//               features x~^(j) = x + sum_{c<j} dm^(c) (Eq. 2) of its columns from the stage accumulators, writes
+//               x_out = x~^(K), and multiplies them with its slice of the next layer's predictor matrix A on the fp64
+//               tensor cores: per-slice partial latents.
 //      -- barrier --
-//   3. scores   All K+1 score vectors of this CTA's neurons (fp64), histogram + bucket insert per evaluation.
+//   2b. sum     The slices' partials are added (fixed order) into the K+1 latents z^(j) and sums of squares.
 //      -- barrier --
-//   4. ranks    Exact rank of every neuron that can be inside the first k ranks, for every evaluation: coarse prefix,
-//               fine prefix inside one coarse bin, comparison inside the neuron's bucket.
+//   3. scores   Every CTA scores its share of the next layer's neurons for all K+1 evaluations (fp64 tensor cores; a
+//               remainder of one or two evaluations on the ordinary fp64 pipe) and stores scores and their fine bins.
+//      -- barrier --
+//   4. select   One CTA per evaluation makes the exact top-k from the stored bins (histogram, scan, cut bin, exact
+//               comparison inside the cut bin); the final evaluation, which also needs every member's exact rank, is
+//               shared by eight CTAs.  Meanwhile the other CTAs ask the next layer's likely rows into L2.
 //
-// Everything a launch dirties in the per-layer scratch is zero again when it ends (the last CTA to finish cleans).
+// Instruction fetch matters as much as arithmetic in phases that run once per layer: code that is not resident in the
+// 16 KB per-scheduler instruction cache streams at 5 to 9 clocks per instruction, so loops are kept rolled unless the
+// unrolling buys memory-level parallelism, and rare paths are out of line.
 #pragma once
 #include "ls_common.cuh"
 
