@@ -38,7 +38,7 @@ namespace ls {
 constexpr int FZ_THREADS = 512;        // compute threads (16 warps)
 constexpr int FZ_BLOCK = FZ_THREADS + 32;  // plus the producer warp
 constexpr int FZ_NG = 3;          // survivors processed per batch of the second ring
-constexpr int FZ_NG1 = 16;        // most neurons per round of the first ring
+constexpr int FZ_NG1 = 4;         // most neurons per round of the first ring
 constexpr int FZ_NB = 4096;       // fine score bins per evaluation
 constexpr int FZ_FIN_PARTS = 8;   // CTAs that share the ranking of the final evaluation
 constexpr int FZ_CUTLIST = 1024;  // entries of the cut bin ranked in shared memory (a fuller bin falls back to global loops)
@@ -1367,33 +1367,45 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
     const int fparts = max(1, min(FZ_FIN_PARTS, G - K));
     const bool selects = cta < fparts + K;
     const int jme = cta < fparts ? K : cta - fparts;
+    // Speculation into L2 (thread li of a group that holds, in s_own, the final scores of the n neurons from i_base on):
+    // the neurons scored highest will most likely be in the refined set, whose exact ranks take another grid barrier to
+    // establish; the first row of their bundles in the next layer is asked into L2 now, so that the next layer's ring
+    // fill finds it there.  The score estimates the gate pre-activation (B is W_gate A, c the gate bias): a likely member
+    // with a positive score will probably survive the ReLU too, so the rest of its bundle is asked for as well.  A wrong
+    // guess costs bandwidth that is idle at this point, never correctness.
+    auto speculate = [&](int li, int i_base, int n) {
+      if (li >= n) return;
+      const double v = s_own[li];
+      const int m_spec = (int)(((long long)keff * n * 3 / 2 + Fn - 1) / Fn) + 1;  // half again the fair share: a round waits for its slowest row
+      int above = 0;
+#pragma unroll 1
+      for (int l2 = 0; l2 < n; ++l2) {
+        const double o = s_own[l2];
+        above += (o > v) || (o == v && l2 < li);
+      }
+      if (above < m_spec)
+        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(A.spec_ptr + (size_t)(i_base + li) * A.spec_stride),
+                     "r"(v > 0.0 ? (unsigned)A.spec_stride : A.spec_bytes) : "memory");
+    };
     named_bar_sync(1, FZ_THREADS);
     if (tid == 0) {
       grid_barrier_thread0(A, G);
     } else if (tid >= 32 && A.spec_ptr && !selects) {
-      // While thread 0 waits for the grid: speculate.  The neurons this CTA scored highest in the final evaluation will
-      // most likely be in the refined set, which takes another grid barrier to establish; the first row of their bundles
-      // in the next layer is asked into L2 now, so that the next layer's ring fill finds it there.  A wrong guess costs
-      // bandwidth that is idle at this point, never correctness.
-      const int li = tid - 32;
-      if (li < n_own) {
-        const double v = s_own[li];
-        const int m_spec = (int)(((long long)keff * n_own * 3 / 2 + Fn - 1) / Fn) + 1;  // half again this CTA's fair share: a round waits for its slowest row
-        int above = 0;
-#pragma unroll 1
-        for (int l2 = 0; l2 < n_own; ++l2) {
-          const double o = s_own[l2];
-          above += (o > v) || (o == v && l2 < li);
-        }
-        // The score estimates the gate pre-activation (B is W_gate A, c the gate bias): a likely member with a positive
-        // score will probably survive the ReLU too, so the rest of its bundle (up and down rows) is asked for as well.
-        if (above < m_spec)
-          asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(A.spec_ptr + (size_t)(i_lo + li) * A.spec_stride),
-                       "r"(v > 0.0 ? (unsigned)A.spec_stride : A.spec_bytes) : "memory");
-      }
+      speculate(tid - 32, i_lo, n_own);
     }
     named_bar_sync(1, FZ_THREADS);
     if (tid == 0) FZ_STAMP(1, 5);
+    {
+      // the selecting CTAs have no time to speculate: the next CTAs do it for them, from the scores now in global memory
+      const int nsel = fparts + K, c2 = cta - nsel;
+      if (A.spec_ptr && c2 >= 0 && c2 < nsel) {
+        const int i2 = c2 * per, n2 = max(0, min(Fn, i2 + per) - i2);
+#pragma unroll 1
+        for (int li = tid; li < n2; li += FZ_THREADS) s_own[li] = __ldcg(A.sc + (size_t)K * Fn + i2 + li);
+        named_bar_sync(1, FZ_THREADS);
+        speculate(tid, i2, n2);
+      }
+    }
 
     // ============================ phase 4: the refined set of evaluation j, selected by one CTA =======================
     // Evaluation j belongs to CTA j * G / E.  The CTA histograms the fine bins of all Fn scores (shared-memory atomics),
