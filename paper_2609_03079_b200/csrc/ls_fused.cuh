@@ -747,13 +747,14 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
       // the gate bias follows at once: a small load issued after the ring's bulk copies would queue behind all of them
       s_mybias[t] = (A.b_gate && i >= 0) ? A.b_gate[i] : 0.f;
     }
+    int issued1 = 0;  // (producer warp) rows of the first ring requested so far
     float xr[CPT][8];
     {
       double sq = 0.0;
 #pragma unroll
       for (int q = 0; q < CPT; ++q) {
         const int ch = tid + q * FZ_THREADS;
-        if (ch < nchunk) {
+        if (ch < nchunk && warp < FZ_THREADS / 32) {
           const float4 a0 = __ldcg(reinterpret_cast<const float4*>(A.x + ch * 8));
           const float4 a1 = __ldcg(reinterpret_cast<const float4*>(A.x + ch * 8 + 4));
           xr[q][0] = a0.x; xr[q][1] = a0.y; xr[q][2] = a0.z; xr[q][3] = a0.w;
@@ -772,45 +773,51 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
     if (tid == 0) FZ_STAMP(1, 21);
 
     if (warp == FZ_THREADS / 32) {
-      // ============================================= producer warp (one lane) ======================================
-      // Issues every bulk copy, so that the compute warps never pay for it.  First ring: the first row of each of this
-      // CTA's neurons (gate, or the only input matrix), as many as fit at once, topped up as rounds finish.  Second
-      // ring: the rest of a neuron's bundle (up and down rows), fetched only for the neurons whose activation
-      // survived, as slots come free.  The compute warps publish rounds finished, survivors found and survivors
-      // consumed in sh.round / sh.nsurv / sh.done.
-      if (lane == 0) {
-        int issued1 = 0, slot1 = 0, issued2 = 0, slot2 = 0, rounds = 0, nsurv = 0;
+      // ============================================= producer warp ================================================
+      // Issues every bulk copy, so that the compute warps never pay for it; the whole warp runs the loop and lane l
+      // issues the l-th copy of a batch.  First ring: the first row of each of this CTA's neurons (gate, or the only
+      // input matrix), as many as fit at once, topped up as rounds finish.  Second ring: the rest of a neuron's bundle
+      // (up and down rows), fetched only for the neurons whose activation survived, as slots come free.  The compute
+      // warps publish rounds finished, survivors found and survivors consumed in sh.round / sh.nsurv / sh.done.
+      {
+        int issued2 = 0, slot2 = 0, rounds = 0, nsurv = 0;
         bool a_sent = false, ok = true;
         const long long t0 = clock64();
         while (true) {
           // top the first ring up to the rows that may be in flight
           const int want = min(n_mine, rounds * NG1 + G1);
-#pragma unroll 1
-          for (; issued1 < want; ++issued1) {
-            int i = s_myidx[issued1];
+          if (issued1 + lane < want) {
+            const int it = issued1 + lane, sl1 = it % G1;
+            int i = s_myidx[it];
             if (i < 0) i = 0;  // a rejected index: read row 0, the result is discarded
-            uint64_t* bar = &s_bar[slot1];
+            uint64_t* bar = &s_bar[sl1];
             mbar_expect_tx(bar, r1_bytes);
-            tma_load_1d(s_r1 + (size_t)slot1 * d, A.bundles + (size_t)i * bundle_elems, r1_bytes, bar);
-            if (++slot1 == G1) slot1 = 0;
+            tma_load_1d(s_r1 + (size_t)sl1 * d, A.bundles + (size_t)i * bundle_elems, r1_bytes, bar);
           }
+          issued1 = max(issued1, want);
           if (!a_sent && A.has_next && !lay.a_alias) {  // A slices with a place of their own: right behind the first burst
             a_sent = true;
-            fz_issue_a(A, s_A, &s_bar[FZ_BAR_A], cta, G, nsl);
+            if (lane == 0) fz_issue_a(A, s_A, &s_bar[FZ_BAR_A], cta, G, nsl);
           }
-          // survivors whose slot is free
+          // survivors whose slot is free (slots carved from the first ring only once that ring is idle)
           int done;
           asm volatile("ld.acquire.cta.shared.s32 %0, [%1];" : "=r"(done) : "r"(smem_u32(&sh.done)) : "memory");
-#pragma unroll 1
-          for (; issued2 < nsurv && issued2 - done < G2T; ++issued2) {
-            if (slot2 >= G2 && rounds < n_rounds) break;  // slots carved from the first ring: only once it is idle
-            const int i = s_surv[issued2];
-            uint64_t* bar = &s_bar[FZ_BAR_R2 + slot2];
-            uint16_t* dst = slot2 < G2 ? s_r2 + (size_t)slot2 * (A.n_mat - 1) * d : s_r1 + (size_t)(slot2 - G2) * (A.n_mat - 1) * d;
+          int n_can = min(nsurv - issued2, G2T - (issued2 - done));
+          if (rounds < n_rounds) n_can = min(n_can, slot2 < G2 ? G2 - slot2 : 0);
+          if (lane < n_can) {
+            int sl2 = slot2 + lane;
+            if (sl2 >= G2T) sl2 -= G2T;
+            const int i = s_surv[issued2 + lane];
+            uint64_t* bar = &s_bar[FZ_BAR_R2 + sl2];
+            uint16_t* dst = sl2 < G2 ? s_r2 + (size_t)sl2 * (A.n_mat - 1) * d : s_r1 + (size_t)(sl2 - G2) * (A.n_mat - 1) * d;
             mbar_expect_tx(bar, r2_bytes);
             tma_load_1d(dst, A.bundles + (size_t)i * bundle_elems + d, r2_bytes, bar);
             if (A.tr_survive) atomicOr(&A.tr_survive[i >> 5], 1u << (i & 31));
-            if (++slot2 == G2T) slot2 = 0;
+          }
+          if (n_can > 0) {
+            issued2 += n_can;
+            slot2 += n_can;
+            if (slot2 >= G2T) slot2 -= G2T;
           }
           if (rounds == n_rounds && issued2 == nsurv) break;  // every row of this layer has been requested
           // wait for news: a round finished (more survivors, room in the first ring) or survivors consumed
@@ -818,25 +825,36 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
           while (true) {
             asm volatile("ld.acquire.cta.shared.s32 %0, [%1];" : "=r"(rnow) : "r"(smem_u32(&s_round)) : "memory");
             asm volatile("ld.acquire.cta.shared.s32 %0, [%1];" : "=r"(dnow) : "r"(smem_u32(&sh.done)) : "memory");
+            rnow = __shfl_sync(0xffffffffu, rnow, 0);  // (one view for the whole warp)
+            dnow = __shfl_sync(0xffffffffu, dnow, 0);
             if (rnow > rounds || (dnow > done && issued2 < nsurv)) break;
-            if (clock64() - t0 > FZ_SPIN_CYCLES) { ok = false; break; }
+            if (__shfl_sync(0xffffffffu, (int)(clock64() - t0 > FZ_SPIN_CYCLES), 0)) { ok = false; break; }
             __nanosleep(64);  // the poll shares an instruction scheduler with four compute warps
           }
-          if (!ok) { set_status(A.status, ST_TIMEOUT); break; }
+          if (!ok) { if (lane == 0) set_status(A.status, ST_TIMEOUT); break; }
           if (rnow > rounds) {
             rounds = min(rnow, n_rounds);
             asm volatile("ld.acquire.cta.shared.s32 %0, [%1];" : "=r"(nsurv) : "r"(smem_u32(&sh.nsurv)) : "memory");
+            nsurv = __shfl_sync(0xffffffffu, nsurv, 0);
           }
         }
         // The next layer's predictor operands that share bytes with the rings wait until the compute warps have drained them.
-        if (A.has_next && ok && fz_wait_round(&s_round, n_rounds + 1, A.status)) {
-          if (lay.a_alias) fz_issue_a(A, s_A, &s_bar[FZ_BAR_A], cta, G, nsl);
-          uint64_t* bbar = &s_bar[FZ_BAR_B];  // rows of B^T: awaited before the score phase
-          mbar_expect_tx(bbar, (uint32_t)n_own * (uint32_t)r * 2);
-          const int rsb = fz_brow_stride(r);
+        if (A.has_next && ok) {
+          int drained = 0;
+          if (lane == 0) drained = fz_wait_round(&s_round, n_rounds + 1, A.status) ? 1 : 0;
+          drained = __shfl_sync(0xffffffffu, drained, 0);
+          if (drained) {
+            uint64_t* bbar = &s_bar[FZ_BAR_B];  // rows of B^T: awaited before the score phase
+            if (lane == 0) {
+              if (lay.a_alias) fz_issue_a(A, s_A, &s_bar[FZ_BAR_A], cta, G, nsl);
+              mbar_expect_tx(bbar, (uint32_t)n_own * (uint32_t)r * 2);
+            }
+            __syncwarp();
+            const int rsb = fz_brow_stride(r);
 #pragma unroll 1
-          for (int li = 0; li < n_own; ++li)
-            tma_load_1d(s_B + (size_t)li * rsb, A.Bt + (size_t)(i_lo + li) * r, (uint32_t)r * 2, bbar);
+            for (int li = lane; li < n_own; li += 32)
+              tma_load_1d(s_B + (size_t)li * rsb, A.Bt + (size_t)(i_lo + li) * r, (uint32_t)r * 2, bbar);
+          }
         }
       }
       return;  // an exited warp counts as arrived at every later block barrier
