@@ -291,3 +291,19 @@ def test_llama7b_shaped_layer_full_size():
     assert stats.get("band", 0) == 0
     ga.close()
     gb.close()
+
+
+def test_llama7b_shaped_layer_wide_selection():
+    """Benchmark-shaped layer pair with k = 6016 (more members than the selection keeps in shared memory: the grouped
+    members go through the global scratch) and with the intermediate refined sets traced."""
+    spec = wl.SPECS["llama2-7b"]
+    la = wl.make_layer(spec, 0, svd_device="cuda")
+    lb = wl.make_layer(spec, 1, svd_device="cuda")
+    ga, gb = ls.ls_layer_create(la, DEV), ls.ls_layer_create(lb, DEV)
+    OA, OB = orc.OracleLayer.from_arrays(la), orc.OracleLayer.from_arrays(lb)
+    stats = {}
+    x = wl.make_tokens(spec, 1)[0]
+    run_step_and_compare(ga, gb, OA, OB, x, 6016, 3, 6016, stats)
+    assert stats.get("band", 0) == 0
+    ga.close()
+    gb.close()
