@@ -337,7 +337,7 @@ def run_ours(args):
         # ---- CPU baseline: the oracle as it stands on a bounded sample
         t0 = time.perf_counter()
         arrays = [keep_host[l] for l in sorted(keep_host)]
-        n_cpu = 16 * len(arrays)  # about ten seconds of CPU work at the Llama-2-7B shape
+        n_cpu = 48 * len(arrays)  # fifteen to twenty seconds of CPU work at the Llama-2-7B shape
         times = oracle_layer_step_seconds(arrays, spec, K, n_cpu, warmup=0)
         cpu_wall = time.perf_counter() - t0
         cpu_val = 1.0 / (float(np.mean(times)) * n_layers)
