@@ -205,7 +205,7 @@ int32_t upload_sliced16(uint16_t** dst, const void* src, int d, int r) {
 // every step).  Consequence: fused steps on one device must not overlap (issue them on one stream, or order the
 // streams).  Sized for the largest shapes the fused path accepts; allocated at the first layer, kept until exit.
 struct DeviceScratch {
-  float* dacc = nullptr;              // [FZ_MAXK][16384] stage accumulators, zero between launches
+  float* ypart = nullptr;             // [256 CTAs][16384] every CTA's partial output of its stage
   unsigned* ctr = nullptr;            // fin, (pad), barrier counter (64-bit)
   double* z = nullptr;                // [FZ_MAXE][1024] latents, then [FZ_MAXE] sums of squares
   double* zpart = nullptr;            // [512 slices][FZ_MAXE][1025] per-slice partial latents
@@ -215,7 +215,7 @@ struct DeviceScratch {
   unsigned long long* kmm = nullptr;  // [2 x 1024] per-CTA smallest / largest key of the final evaluation
   bool ready = false;
 };
-constexpr int kScratchMaxD = 16384, kScratchMaxR = 1024, kScratchMaxF = 32768;
+constexpr int kScratchMaxD = 16384, kScratchMaxR = 1024, kScratchMaxF = 32768, kScratchMaxCtas = 256;
 std::mutex g_scratch_mu;
 DeviceScratch g_scratch[64];
 
@@ -225,7 +225,7 @@ int32_t device_scratch(int dev, DeviceScratch** out) {
   DeviceScratch& S = g_scratch[dev];
   if (!S.ready) {
     const size_t NE = ls::FZ_MAXE;
-    LS_TRY(dalloc(&S.dacc, (size_t)2 * ls::FZ_MAXK * kScratchMaxD));  // two parities (whole-token kernel)
+    LS_TRY(dalloc(&S.ypart, (size_t)kScratchMaxCtas * kScratchMaxD));
     LS_TRY(dalloc(&S.ctr, (size_t)8));
     LS_TRY(dalloc(&S.z, NE * kScratchMaxR + NE));
     LS_TRY(dalloc(&S.zpart, (size_t)(kScratchMaxD / ls::FZ_SL) * NE * (kScratchMaxR + 1)));
@@ -233,7 +233,6 @@ int32_t device_scratch(int dev, DeviceScratch** out) {
     LS_TRY(dalloc(&S.sb, NE * kScratchMaxF));
     LS_TRY(dalloc(&S.bent, (size_t)kScratchMaxF));
     LS_TRY(dalloc(&S.kmm, (size_t)2048));
-    LS_CUDA(cudaMemset(S.dacc, 0, (size_t)2 * ls::FZ_MAXK * kScratchMaxD * sizeof(float)));
     LS_CUDA(cudaMemset(S.ctr, 0, 8 * sizeof(unsigned)));
     LS_CUDA(cudaMemset(S.z, 0, (NE * kScratchMaxR + NE) * sizeof(double)));
     S.ready = true;
@@ -350,7 +349,7 @@ bool fused_eligible(const ls_layer* L, const ls_layer* next, int batch, int K, i
   if (!g_opt_fused.load(std::memory_order_relaxed)) return false;
   if (batch != 1 || L->cache_rows != 0 || (next && next->cache_rows != 0)) return false;
   if (K > ls::FZ_MAXK) return false;
-  if ((sel_cap + L->sm_count - 1) / L->sm_count > ls::FZ_MAX_MINE) return false;
+  if ((sel_cap + L->sm_count - 1) / L->sm_count > ls::FZ_MAX_MINE || L->sm_count > kScratchMaxCtas) return false;
   if ((L->d >> 3) > ls::FZ_THREADS * 2) return false;
   return fused_plan(L, next, nullptr);
 }
@@ -379,7 +378,8 @@ int32_t fused_args(ls_layer* L, ls_layer* next, const float* d_x, float* d_x_out
   a.sel_idx = sel_idx; a.sel_count = sel_count; a.sel_cap = sel_cap; a.K = K;
   DeviceScratch* S = nullptr;
   LS_TRY(device_scratch(L->device, &S));
-  a.dacc = S->dacc + (size_t)parity * ls::FZ_MAXK * kScratchMaxD; a.fin = S->ctr;
+  a.ypart = S->ypart;
+  (void)parity;
   a.bar_count = reinterpret_cast<unsigned long long*>(S->ctr + 2);  // 8-byte aligned
   a.status = L->status;
   a.has_next = next ? 1 : 0;

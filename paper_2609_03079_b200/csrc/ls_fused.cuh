@@ -10,11 +10,12 @@
 //               rows of the CTA's neurons into a first shared-memory ring by 1-D bulk copies (TMA), all at once when they
 //               fit; the compute warps form the pre-activations; only the neurons that survive the ReLU have the rest of
 //               their bundle (up and down rows) fetched into a second ring, their activation completed and their down
-//               row, scaled, added to the CTA's partial output, which is kept in registers and added once to the stage
-//               accumulator (vector reductions).
+//               row, scaled, added to the CTA's partial output, which is kept in registers and written once to the
+//               CTA's own row of a partial-output array (no floating-point atomics: every sum has a fixed order, the
+//               kernel is bitwise repeatable).
 //      -- barrier --
 //   2. latent   The feature is cut into slices of 32 columns, one per CTA.  The owner rebuilds the K+1 partial residual
-//               features x~^(j) = x + sum_{c<j} dm^(c) (Eq. 2) of its columns from the stage accumulators, writes
+//               features x~^(j) = x + sum_{c<j} dm^(c) (Eq. 2) of its columns from the CTAs' partial outputs, writes
 //               x_out = x~^(K), and multiplies them with its slice of the next layer's predictor matrix A on the fp64
 //               tensor cores: per-slice partial latents.
 //      -- barrier --
@@ -77,8 +78,7 @@ struct alignas(16) FusedArgs {  // (an array of these is prefetched with 16-byte
   const float* x; float* x_out;
   const int32_t* sel_idx; const int32_t* sel_count; int sel_cap; int K;
   FusedSmemLayout lay;    // where everything sits in dynamic shared memory
-  float* dacc;            // [FZ_MAXK][d] stage accumulators, zero on entry and on exit
-  unsigned* fin;          // [1] CTAs finished, zero on entry and on exit
+  float* ypart;           // [G][d] every CTA's partial output of its stage (no atomics: summed in a fixed order later)
   unsigned long long* bar_count;  // [1] barrier arrivals since the layer was created (monotonic)
   int* status;
   // next layer's predictor (has_next == 0: no refinement)
@@ -325,7 +325,7 @@ inline FusedSmemLayout fused_layout(int d, int n_mat, int r, int Fn, int G, int 
   L.mine_off = take((size_t)FZ_MAX_MINE * 16);       // this CTA's neurons, their gate biases; the survivors, their activations
   L.pc_off = take((size_t)L.per * 4);
   L.xt_off = take((size_t)FZ_EPAD * FZ_XBLK * 8);  // x~^(j) of one slice, fp64, one padded block per row
-  L.dv_off = take((size_t)FZ_MAXK * FZ_SL * 4);      // stage accumulators of one slice
+  L.dv_off = take((size_t)(FZ_MAXK + FZ_THREADS / 32) * FZ_SL * 4);  // stage sums of one slice, and their partial sums
   if (!a_alias) L.a_off = take(a_bytes);
   const size_t base = o;
   L.r1_off = take((size_t)g1 * d * 2);
@@ -351,8 +351,6 @@ inline FusedSmemLayout fused_layout(int d, int n_mat, int r, int Fn, int G, int 
 // Block-shared state of a layer step (static shared memory of the kernels below).
 struct FusedShared {
   FusedArgs args;                    // the layer's arguments (whole-token kernel: copied from global memory per layer)
-  FusedArgs prev;                    // whole-token kernel: the layer before, whose scratch is cleaned meanwhile
-  int last;
   int round;                         // rounds the compute warps have finished (read by the producer)
   int stage, g_lo, gsize;            // this CTA's stage, the first CTA of the stage's group and the group's size
   unsigned phase[FZ_NBAR];           // phases every mbarrier has completed in earlier layers of the launch
@@ -1024,15 +1022,16 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
     used_r2 = nsurv;
     named_bar_sync(1, FZ_THREADS);  // nobody reads the rings any more: the producer may overwrite them
     if (tid == 0) asm volatile("st.release.cta.shared.s32 [%0], %1;" ::"r"(smem_u32(&s_round)), "r"(n_rounds + 1) : "memory");
-    // the CTA's whole contribution to its stage, added once (vector reductions; order across CTAs is not fixed)
-    if (nsurv > 0) {
-      float* dst = A.dacc + (size_t)stage * d;
+    // the CTA's whole contribution to its stage (zeros when nothing survived) goes to its own row of ypart: the stage
+    // sums are formed later in a fixed order, so the features do not depend on the order in which CTAs finish
+    {
+      float* dst = A.ypart + (size_t)cta * d;
 #pragma unroll
       for (int q = 0; q < CPT; ++q) {
         const int ch = tid + q * FZ_THREADS;
         if (ch < nchunk) {
-          red_add_v4(dst + ch * 8, yacc[q][0], yacc[q][1], yacc[q][2], yacc[q][3]);
-          red_add_v4(dst + ch * 8 + 4, yacc[q][4], yacc[q][5], yacc[q][6], yacc[q][7]);
+          *reinterpret_cast<float4*>(dst + ch * 8) = make_float4(yacc[q][0], yacc[q][1], yacc[q][2], yacc[q][3]);
+          *reinterpret_cast<float4*>(dst + ch * 8 + 4) = make_float4(yacc[q][4], yacc[q][5], yacc[q][6], yacc[q][7]);
         }
       }
     }
@@ -1089,15 +1088,41 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
   for (int a = 0; cta + a * G < nsl; ++a) {
     const int sl = cta + a * G;
     if (a > 0) named_bar_sync(1, FZ_THREADS);  // the previous slice's features are no longer read
-    float* s_dv = reinterpret_cast<float*>(smem + lay.dv_off);  // [K][32]
+    float* s_dv = reinterpret_cast<float*>(smem + lay.dv_off);  // [K][32] stage sums dm^(c) of the slice's columns
+    float* s_dvp = s_dv + FZ_MAXK * FZ_SL;                        // [16][32] partial sums of thread groups
     float xv = 0.f;
-    if (tid < K * FZ_SL) {  // one stage accumulator per thread, all loads in flight together
-      const int c = sl * FZ_SL + (tid & (FZ_SL - 1));
-      s_dv[tid] = c < d ? __ldcg(A.dacc + (size_t)(tid / FZ_SL) * d + c) : 0.f;
+    {
+      // Stage c is the sum of the partial outputs of the CTAs [c G / K, (c + 1) G / K).  The 16 groups of 32 threads
+      // (one thread per column) share the stages: nh groups per stage, group h adds every nh-th CTA of the stage in
+      // order, twelve loads in flight; the nh partial sums are then added in order: a fixed summation tree.
+      const int col = tid & (FZ_SL - 1), u = tid >> 5, c = sl * FZ_SL + col;
+      const int nh = max(1, (FZ_THREADS / 32) / K), cs = u / nh, h = u - cs * nh;
+      float acc = 0.f;
+      if (cs < K && c < d) {
+        const int p_hi = (cs + 1) * G / K;
+        const float* yp = A.ypart + c;
+#pragma unroll 1
+        for (int p = cs * G / K + h; p < p_hi; p += 12 * nh) {  // (148 CTAs: at most ten per thread, one batch)
+          float q[12];
+#pragma unroll
+          for (int v = 0; v < 12; ++v) q[v] = p + v * nh < p_hi ? __ldcg(yp + (size_t)(p + v * nh) * d) : 0.f;
+#pragma unroll
+          for (int v = 0; v < 12; ++v) acc += q[v];
+        }
+      }
+      s_dvp[tid] = acc;
     }
     if (tid < FZ_SL) {
       const int c = sl * FZ_SL + tid;
       if (c < d) xv = __ldcg(A.x + c) + (A.b_down ? A.b_down[c] : 0.f);
+    }
+    named_bar_sync(1, FZ_THREADS);
+    if (tid < K * FZ_SL) {
+      const int nh = max(1, (FZ_THREADS / 32) / K), cs = tid >> 5, col = tid & (FZ_SL - 1);
+      float v = 0.f;
+#pragma unroll 1
+      for (int h = 0; h < nh; ++h) v += s_dvp[(cs * nh + h) * FZ_SL + col];
+      s_dv[tid] = v;
     }
     named_bar_sync(1, FZ_THREADS);
     if (tid < FZ_SL) {
@@ -1448,32 +1473,12 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
 
 }
 
-// Zeroes the slice [part, parts) of the stage accumulators a layer step dirtied (compute threads only).  The caller
-// guarantees that every CTA is done with the layer.
-__device__ inline void fused_clean(const FusedArgs& A, int part, int parts) {
-  const int tid = threadIdx.x;
-#pragma unroll 1
-  for (int t = part * FZ_THREADS + tid; t < A.K * A.d; t += parts * FZ_THREADS) A.dacc[t] = 0.f;
-}
-
-// ---- one launch per layer step: the last CTA to finish restores the zero-on-entry invariants of the scratch
+// ---- one launch per layer step ------------------------------------------------------------------------------------------
 template <int WD, int CPT>
 __global__ void __launch_bounds__(FZ_BLOCK, 1) ls_fused_step_kernel(const __grid_constant__ FusedArgs A) {
   extern __shared__ __align__(128) unsigned char smem[];
   __shared__ FusedShared sh;
   fused_layer<WD, CPT>(A, smem, sh, true, -1);
-  if (threadIdx.x >= FZ_THREADS) return;  // the producer warp is done; an exited warp counts as arrived at block barriers
-  named_bar_sync(1, FZ_THREADS);
-  if (threadIdx.x == 0) {
-    __threadfence();
-    sh.last = (atomicAdd(A.fin, 1u) == gridDim.x - 1u) ? 1 : 0;
-  }
-  named_bar_sync(1, FZ_THREADS);
-  if (sh.last) {
-    __threadfence();
-    fused_clean(A, 0, 1);
-    if (threadIdx.x == 0) *A.fin = 0u;
-  }
 }
 
 // ---- one launch per token: the layers of a resident stack run back to back inside one cooperative kernel ------------
@@ -1489,9 +1494,9 @@ struct StackCall {
   int tr_cap;
 };
 
-// Layer n reads x / selection buffers of parity n & 1 and writes those of the other parity; the scratch a layer dirties
-// (stage accumulators, histograms, set sizes) also alternates, and every CTA cleans its slice of the previous layer's
-// scratch while it waits at the end of the current one.  A layer boundary costs one grid barrier instead of a launch.
+// Layer n reads x / selection buffers of parity n & 1 and writes those of the other parity; the device-wide scratch is
+// overwritten by every layer, never accumulated into, so nothing has to be cleaned between layers.  A layer boundary
+// costs one grid barrier instead of a launch.
 template <int WD, int CPT>
 __global__ void __launch_bounds__(FZ_BLOCK, 1)
     ls_fused_stack_kernel(const FusedArgs* __restrict__ g_args, int n_layers, const __grid_constant__ StackCall C) {
@@ -1532,7 +1537,6 @@ __global__ void __launch_bounds__(FZ_BLOCK, 1)
     fused_layer<WD, CPT>(A, smem, sh, n == 0, known_count);
     known_count = A.has_next ? min(min(A.k_next, A.Fn), A.next_cap) : -1;  // what this layer wrote to *next_count
     if (tid < FZ_THREADS) {
-      if (n > 0) fused_clean(sh.prev, cta, G);  // nobody touches the previous layer's scratch any more
       grid_barrier(A, G);                       // layer boundary: x_out and the refined selection are visible to all
 #ifdef LS_FZ_TIMING
       if (tid == 0 && cta == 0 && n < 100) {
@@ -1544,13 +1548,9 @@ __global__ void __launch_bounds__(FZ_BLOCK, 1)
 #endif
     }
     __syncthreads();
-#pragma unroll 1
-    for (int w = tid; w < NW; w += FZ_BLOCK) reinterpret_cast<uint32_t*>(&sh.prev)[w] = reinterpret_cast<const uint32_t*>(&sh.args)[w];
-    __syncthreads();
   }
   if (tid < FZ_THREADS && n_layers > 0) {
-    const FusedArgs& A = sh.prev;  // the last layer; every CTA is past its final barrier
-    fused_clean(A, cta, G);
+    const FusedArgs& A = sh.args;  // the last layer; every CTA is past its final barrier
     if (cta == G - 1 && C.tr_x) {
 #pragma unroll 1
       for (int c = tid; c < A.d; c += FZ_THREADS) C.tr_x[(size_t)n_layers * A.d + c] = __ldcg(A.x_out + c);

@@ -113,3 +113,28 @@ def test_llama7b_shaped_three_layer_stack():
     stats = {}
     decode_and_check(spec, arrays, 8, spec.k, 1, stats)
     assert stats.get("band", 0) == 0
+
+
+def test_whole_token_kernel_is_bitwise_repeatable():
+    """Partial outputs are summed in a fixed order (no floating-point atomics), so the same token gives the same bits."""
+    spec = wl.SPECS["tiny4"]
+    GLs = [ls.ls_layer_create(a, DEV) for a in wl.make_stack(spec, down_scale=50.0)]
+    stack = ls.ls_stack_create(GLs)
+    k = spec.k
+    sel0 = ls.Selection(spec.d_ff, k, DEV)
+    x = torch.from_numpy(wl.make_tokens(spec)[1]).cuda(DEV)
+    outs = []
+    for _ in range(4):
+        x_out = torch.empty_like(x)
+        sel_out = ls.Selection(spec.d_ff, k, DEV)
+        ls.ls_predict(GLs[0], x, k, sel0)
+        ls.ls_stack_decode(stack, x, x_out, sel0, 8, k, sel_out)
+        torch.cuda.synchronize()
+        outs.append((x_out.cpu().numpy().view(np.uint32).copy(), sel_out.order().copy()))
+    for xo, idx in outs[1:]:
+        assert np.array_equal(xo, outs[0][0])
+        assert np.array_equal(idx, outs[0][1])
+    assert all(ls.ls_layer_status(g) == 0 for g in GLs)
+    stack.close()
+    for g in GLs:
+        g.close()
