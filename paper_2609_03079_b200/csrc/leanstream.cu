@@ -335,6 +335,7 @@ bool fused_plan(const ls_layer* L, const ls_layer* next, ls::FusedSmemLayout* ou
     for (int c = 0; c < 3; ++c) {
       for (int g1 = ls::FZ_MAX_G1; g1 >= ls::FZ_NG + 1; --g1) {
         const ls::FusedSmemLayout lay = ls::fused_layout(L->d, L->n_mat, r, Fn, L->sm_count, hn, g1, g2s[c], alias);
+        if (lay.per > 512) return false;  // the kernel keeps one slot count per tile of eight neurons, 64 at most
         if (lay.total > budget) continue;
         if (alias == 0 && g1 < 8) break;  // too shallow with the A slices apart: try the next arrangement
         if (out) *out = lay;

@@ -50,7 +50,6 @@ constexpr int FZ_MAX_G1 = 16;     // most slots of the first ring (first row of 
 constexpr int FZ_MAX_G2 = 16;     // most slots of the second ring (the rest of a survivor's bundle), carved slots included
 constexpr int FZ_SL = 32;         // columns of the feature handled as one slice in the latent phase
 constexpr int FZ_EPAD = 18;       // rows kept per evaluation-indexed buffer: at most two MMA tiles, or FZ_MAXE rows
-constexpr int FZ_KS = 4;          // column splits of a score tile (more independent tasks than warps)
 constexpr int FZ_MAX_MINE = 256;  // neurons one CTA may own in one step
 #ifdef LS_FZ_TIMING
 constexpr long long FZ_SPIN_CYCLES = 40LL * 1000 * 1000;
@@ -333,7 +332,13 @@ inline FusedSmemLayout fused_layout(int d, int n_mat, int r, int Fn, int G, int 
   const int per8 = (L.per + 7) / 8 * 8;
   L.b_off = take((size_t)per8 * fz_brow_stride(r) * 2);
   L.zs_off = take(has_next ? (size_t)FZ_EPAD * fz_feat_stride(r) * 8 : 0);
-  L.part_off = take(has_next ? (size_t)FZ_KS * FZ_EPAD * per8 * 8 : 0);  // [split][evaluation][neuron]
+  {
+    // partial sums of the score tiles: [slot][evaluation][neuron]; a tile's blocks are spread over at most `slots` warps
+    const int n_mt = per8 / 8, nblk = (r + 31) / 32, nun = n_mt * nblk;
+    const int U = nun > 0 ? (nun + 15) / 16 : 1;
+    const int slots = (nblk + U - 1) / U + 1;
+    L.part_off = take(has_next ? (size_t)slots * FZ_EPAD * per8 * 8 : 0);
+  }
   L.own_off = take((size_t)L.per * 8);               // this CTA's scores of the final evaluation
   const size_t end_refine = o;
   o = base;  // the selection works when the score operands are dead: it shares their bytes
@@ -352,7 +357,7 @@ struct FusedShared {
   int stage, g_lo, gsize;            // this CTA's stage, the first CTA of the stage's group and the group's size
   unsigned phase[FZ_NBAR];           // phases every mbarrier has completed in earlier layers of the launch
   int nsurv, done;                   // survivors found so far / consumed so far (read by the producer)
-  double inv[FZ_EPAD];
+  double inv[FZ_EPAD + 32];          // 1 / rms per evaluation; behind them: partial-sum slots per score tile (ints)
   unsigned long long kmm[2 * 16];
 };
 
@@ -1239,7 +1244,7 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
 
     // ============================ phase 3: scores of this CTA's neurons, every evaluation =============================
     double* s_zs = reinterpret_cast<double*>(smem + lay.zs_off);            // [max(EM, E)][fz_feat_stride(r)], un-normalised, blocked
-    double* s_part = reinterpret_cast<double*>(smem + lay.part_off);        // [KSd][prow][per8], KSd * prow <= FZ_KS * FZ_EPAD
+    double* s_part = reinterpret_cast<double*>(smem + lay.part_off);        // [slot][prow][per8]
     double* s_own = reinterpret_cast<double*>(smem + lay.own_off);          // [per] scores of the final evaluation
     const double bin_lo = __ldcg(&A.range[0]), bin_hi = __ldcg(&A.range[1]);
     const double INF = __longlong_as_double(0x7ff0000000000000LL);
@@ -1294,30 +1299,31 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
     named_bar_sync(1, FZ_THREADS);
     if (tid == 0) FZ_STAMP(1, 40);
 
-    // C[neuron][evaluation] = B^T rows x latents.  A task is a tile of eight neurons times one of FZ_KS ranges of
-    // 32-column blocks; the ranges are added afterwards in a fixed order.  Evaluations [0, EM) go through the tensor
-    // cores, evaluations [EM, E) (at most two) through ordinary FMAs on the same converted weights.  Within one evaluation
-    // every neuron's score is accumulated in the same order whatever its position in a tile, so equal predictor rows give
-    // bit-equal scores.
+    // C[neuron][evaluation] = B^T rows x latents.  Evaluations [0, EM) go through the tensor cores, evaluations [EM, E)
+    // (at most two) through ordinary FMAs on the same converted weights.  Within one evaluation every neuron's score is
+    // accumulated in the same order whatever its position in a tile, so equal predictor rows give bit-equal scores.
+    // Work units are (tile of eight neurons, 32-column block), in tile-major order, dealt evenly: warp w takes the units
+    // [w U, (w + 1) U).  A warp's share of a tile goes to the partial-sum slot `w - first warp of the tile`; the slots
+    // of a tile are added afterwards in order.
     const int n_mt = (n_own + 7) >> 3;
-    const int prow = max(EM, E);                                   // rows of a range's partial sums
-    const int KSd = min(FZ_KS, (FZ_KS * FZ_EPAD) / prow);         // ranges (fewer if the partial sums lack room)
-    const int bchunk = (nblk + KSd - 1) / KSd;                     // blocks per range
-    if (lane == 0) FZ_STAMP(1, 400 + warp * 4);
+    const int prow = max(EM, E);                                   // rows of a slot of partial sums
+    const int n_units = n_mt * nblk, U = max(1, (n_units + FZ_THREADS / 32 - 1) / (FZ_THREADS / 32));
+    int* s_nslot = reinterpret_cast<int*>(s_inv + FZ_EPAD);  // [n_mt] slots per tile (n_mt <= 64: behind the scale factors)
 #pragma unroll 1
-    for (int task = warp; task < n_mt * KSd; task += FZ_THREADS / 32) {
-      if (lane == 0 && task == warp + 16) FZ_STAMP(1, 401 + warp * 4);
-      const int ks = task / n_mt, mt = task - ks * n_mt;
-      const int b_lo = ks * bchunk, b_hi = min(nblk, b_lo + bchunk);
+    for (int m2 = tid; m2 < n_mt; m2 += FZ_THREADS) s_nslot[m2] = (m2 * nblk + nblk - 1) / U - (m2 * nblk) / U + 1;
+    if (lane == 0) FZ_STAMP(1, 400 + warp * 4);
+    {
+      const int u_lo = warp * U, u_hi = min(n_units, u_lo + U);
       const int g = lane >> 2, t4 = lane & 3;
-      const uint16_t* arow = s_B + (size_t)(mt * 8 + g) * RSB + t4 * 8;
       const double* zrow = s_zs + (size_t)g * RSZ + t4 * 10;      // MMA tiles: evaluation nt * 8 + g
       const double* zrem = s_zs + (size_t)EM * RSZ + t4 * 10;     // remainder evaluations EM, EM + 1
       double c[2][2] = {{0.0, 0.0}, {0.0, 0.0}}, rs[2] = {0.0, 0.0};
+      int mt = u_lo < u_hi ? u_lo / nblk : -1;
 #pragma unroll 1
-      for (int b = b_lo; b < b_hi; ++b) {
+      for (int u = u_lo; u < u_hi; ++u) {
+        const int b = u - mt * nblk;
         double av[8], bv[8];
-        cvt8_to_double<WD>(*reinterpret_cast<const uint4*>(arow + b * 32), av);
+        cvt8_to_double<WD>(*reinterpret_cast<const uint4*>(s_B + (size_t)(mt * 8 + g) * RSB + t4 * 8 + b * 32), av);
 #pragma unroll
         for (int nt = 0; nt < 2; ++nt) {
           if (nt < NTM) {
@@ -1333,21 +1339,27 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
             for (int k = 0; k < 8; ++k) rs[rm] = fma(av[k], bv[k], rs[rm]);
           }
         }
-      }
-      double* outp = s_part + (size_t)ks * prow * per8 + mt * 8 + g;
+        if (b == nblk - 1 || u == u_hi - 1) {  // the warp's share of this tile is complete: to its slot
+          const int slot = warp - (mt * nblk) / U;
+          double* outp = s_part + (size_t)slot * prow * per8 + mt * 8 + g;
 #pragma unroll
-      for (int nt = 0; nt < 2; ++nt) {
-        if (nt < NTM) {
-          const int j = nt * 8 + t4 * 2;
-          outp[(size_t)j * per8] = c[nt][0];
-          outp[(size_t)(j + 1) * per8] = c[nt][1];
-        }
-      }
+          for (int nt = 0; nt < 2; ++nt) {
+            if (nt < NTM) {
+              const int j = nt * 8 + t4 * 2;
+              outp[(size_t)j * per8] = c[nt][0];
+              outp[(size_t)(j + 1) * per8] = c[nt][1];
+              c[nt][0] = c[nt][1] = 0.0;
+            }
+          }
 #pragma unroll
-      for (int rm = 0; rm < 2; ++rm) {
-        if (rm < REM) {
-          const double v = quad_sum(rs[rm]);
-          if (t4 == 0) outp[(size_t)(EM + rm) * per8] = v;
+          for (int rm = 0; rm < 2; ++rm) {
+            if (rm < REM) {
+              const double v = quad_sum(rs[rm]);
+              if (t4 == 0) outp[(size_t)(EM + rm) * per8] = v;
+              rs[rm] = 0.0;
+            }
+          }
+          ++mt;
         }
       }
     }
@@ -1367,8 +1379,11 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
       for (int t = tid; t < n_ent; t += FZ_THREADS) {
         const int j = t / n_own, li = t - j * n_own, i = i_lo + li;
         double v = 0.0;
-#pragma unroll 4
-        for (int ks = 0; ks < KSd; ++ks) v += s_part[((size_t)ks * prow + j) * per8 + li];
+        {
+          const int nsl2 = s_nslot[li >> 3];  // slots of this neuron's tile
+#pragma unroll 1
+          for (int sl2 = 0; sl2 < nsl2; ++sl2) v += s_part[((size_t)sl2 * prow + j) * per8 + li];
+        }
         v = canonical_score(v * s_inv[j] + (double)s_pc[li]);
         const double scl = fmin(fmax(v, -1.7976931348623157e308), 1.7976931348623157e308);
         int b = (int)((bin_hi - scl) * bscale);
