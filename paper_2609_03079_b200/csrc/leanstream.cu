@@ -322,10 +322,13 @@ int32_t create_impl(const ls_layer_desc* D, ls_layer* L) {
   return LS_OK;
 }
 
+// Dynamic shared memory the fused kernels may ask for; they also have a few KB of static shared memory.
+constexpr size_t kFusedSmemBudget = 218 * 1024;
+
 // ---- the fused per-layer kernel: eligibility and launch ---------------------------------------------------------------
 // Shared-memory plan of the fused kernel: as many ring stages as fit beside the predictor operands.
 bool fused_plan(const ls_layer* L, const ls_layer* next, ls::FusedSmemLayout* out) {
-  const size_t budget = 218 * 1024;  // dynamic part; the kernel also has a few KB of static shared memory
+  const size_t budget = kFusedSmemBudget;
   const int r = next ? next->r : 0, Fn = next ? next->F : 0, hn = next ? 1 : 0;
   // First ring (first row of every bundle): as deep as fits, ideally all of a CTA's neurons at once.  Second ring (the
   // rest of a survivor's bundle): a few slots; the producer refills them as survivors are consumed.  The A slices keep a
@@ -402,6 +405,7 @@ int32_t fused_args(ls_layer* L, ls_layer* next, const float* d_x, float* d_x_out
   ls::FusedSmemLayout lay{};
   if (!fused_plan(L, next, &lay)) return fail(LS_ERR_STATE, "fused step: shared memory plan failed");
   a.lay = lay;
+  a.xs_put = -1; a.xs_get = -1;
   *out = a;
   if (lay_out) *lay_out = lay;
   return LS_OK;
@@ -637,6 +641,18 @@ int32_t ls_stack_create(ls_layer* const* layers, int32_t n_layers, ls_stack** ou
                     S->selidx + (size_t)(n & 1) * S->max_sel, S->selcnt + (n & 1), S->max_sel, 1, 0, &sn, n & 1, &h[n], &lay);
     if (rc != LS_OK) return cleanup(rc);
     S->smem = std::max(S->smem, (size_t)lay.total);
+  }
+  {
+    // x travels from layer to layer through shared memory where some bytes are free from the end of a layer's stream
+    // phase to the first survivors' rows of the next one: above everything the refinement phases use, inside (or
+    // above) the second ring.
+    size_t lo = 0;
+    for (int n = 0; n < n_layers; ++n) lo = std::max(lo, (size_t)std::max(h[n].lay.free_lo, h[n].lay.r2_off));
+    lo = (lo + 127) & ~(size_t)127;
+    if (lo + (size_t)S->d * 4 <= kFusedSmemBudget && S->d % 8 == 0 && !getenv("LS_DBG_NOSTASH")) {
+      S->smem = std::max(S->smem, lo + (size_t)S->d * 4);
+      for (int n = 0; n + 1 < n_layers; ++n) { h[n].xs_put = (int)lo; h[n + 1].xs_get = (int)lo; }
+    }
   }
   for (int n = 0; n + 1 < n_layers; ++n) {  // what layer n + 1 reads first: its arguments, gate biases, down bias, predictor offsets
     const ls_layer* L1 = layers[n + 1];

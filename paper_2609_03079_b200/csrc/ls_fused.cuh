@@ -65,7 +65,7 @@ struct FusedSmemLayout {
   unsigned r1_off, r2_off;
   // ... and, in the same bytes once the rings have drained, the operands and results of the refinement
   unsigned b_off, zs_off, part_off, own_off, sel_off;
-  unsigned total;
+  unsigned total, free_lo;
   int per, ns_cta, a_alias, g1, g2, g2x;  // g2x: extra second-ring slots carved from the first ring once it is idle
 };
 
@@ -101,6 +101,9 @@ struct alignas(16) FusedArgs {  // (an array of these is prefetched with 16-byte
   const void* pg_ptr[3]; unsigned long long pg_bytes[3];
   // speculation into L2: the next layer's bundles (first row of a neuron at spec_ptr + i * spec_stride, spec_bytes long)
   const char* spec_ptr; unsigned long long spec_stride; unsigned spec_bytes;
+  // (whole-token kernel) the residual feature handed from layer to layer through shared memory: where this layer leaves
+  // x_out for the next one, and where it finds its own x (byte offsets into the dynamic shared memory; -1: global memory)
+  int xs_put, xs_get;
   // trace (all nullable)
   float* tr_xtilde; uint32_t* tr_masks; int32_t* tr_counts; uint32_t* tr_survive;
 };
@@ -345,6 +348,7 @@ inline FusedSmemLayout fused_layout(int d, int n_mat, int r, int Fn, int G, int 
   L.sel_off = take(has_next ? fz_select_bytes(Fn) : 0);
   const size_t end_select = o;
   o = end_refine > end_select ? end_refine : end_select;
+  L.free_lo = (unsigned)o;  // no phase after the stream uses shared memory from here on
   L.total = (unsigned)(o > end_stream ? o : end_stream);
   return L;
 }
@@ -352,7 +356,7 @@ inline FusedSmemLayout fused_layout(int d, int n_mat, int r, int Fn, int G, int 
 // =====================================================================================================================
 // Block-shared state of a layer step (static shared memory of the kernels below).
 struct FusedShared {
-  FusedArgs args;                    // the layer's arguments (whole-token kernel: copied from global memory per layer)
+  FusedArgs args[2];                 // (whole-token kernel) this layer's arguments and, fetched meanwhile, the next layer's
   int round;                         // rounds the compute warps have finished (read by the producer)
   int stage, g_lo, gsize;            // this CTA's stage, the first CTA of the stage's group and the group's size
   unsigned phase[FZ_NBAR];           // phases every mbarrier has completed in earlier layers of the launch
@@ -708,10 +712,10 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
       sh.stage = c;
       sh.g_lo = c * G / K;
       sh.gsize = (c + 1) * G / K - sh.g_lo;
+      s_round = 0; sh.nsurv = 0; sh.done = 0;  // (the whole-token kernel clears them again at every layer boundary)
     }
+    __syncthreads();
   }
-  if (tid == 0) { s_round = 0; sh.nsurv = 0; sh.done = 0; }
-  __syncthreads();
   if (tid == 0) FZ_STAMP(1, 20);
 
   const int per = lay.per, r = A.r, Fn = A.Fn;
@@ -734,20 +738,12 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
     const size_t bundle_elems = (size_t)A.n_mat * d;
     const int up_off = A.gated ? 0 : -1, dn_off = A.gated ? d : 0;  // where the rows sit inside a second-ring slot
 
-    // this CTA's neurons first (the bulk copies only need the indices), then x
     int* s_myidx = reinterpret_cast<int*>(smem + lay.mine_off);
     float* s_mybias = reinterpret_cast<float*>(s_myidx + FZ_MAX_MINE);
     int* s_surv = s_myidx + 2 * FZ_MAX_MINE;                       // surviving neurons, in the order they were found
     float* s_qa = reinterpret_cast<float*>(s_myidx + 3 * FZ_MAX_MINE);  // their activations
-#pragma unroll 1
-    for (int t = tid; t < n_mine; t += FZ_THREADS) {
-      int i = __ldcg(A.sel_idx + first + t * gsize);
-      if ((unsigned)i >= (unsigned)A.F) { set_status(A.status, ST_BAD_INDEX); i = -1; }
-      s_myidx[t] = i;
-      // the gate bias follows at once: a small load issued after the ring's bulk copies would queue behind all of them
-      s_mybias[t] = (A.b_gate && i >= 0) ? A.b_gate[i] : 0.f;
-    }
-    int issued1 = 0;  // (producer warp) rows of the first ring requested so far
+    const int n_first = min(n_mine, G1);  // rows of the first ring requested in the prologue, by the compute warps
+    int issued1 = n_first;                // (producer warp) rows of the first ring requested so far
     float xr[CPT][8];
     {
       double sq = 0.0;
@@ -755,18 +751,61 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
       for (int q = 0; q < CPT; ++q) {
         const int ch = tid + q * FZ_THREADS;
         if (ch < nchunk && warp < FZ_THREADS / 32) {
-          const float4 a0 = __ldcg(reinterpret_cast<const float4*>(A.x + ch * 8));
-          const float4 a1 = __ldcg(reinterpret_cast<const float4*>(A.x + ch * 8 + 4));
+          // (x left in shared memory by the layer before: every CTA reading the same 16 KB of global memory at the same
+          // moment, right after a grid barrier, holds up everything issued behind it)
+          const float4* xsrc = A.xs_get >= 0 ? reinterpret_cast<const float4*>(smem + A.xs_get) + ch * 2 : nullptr;
+          const float4 a0 = xsrc ? xsrc[0] : __ldcg(reinterpret_cast<const float4*>(A.x + ch * 8));
+          const float4 a1 = xsrc ? xsrc[1] : __ldcg(reinterpret_cast<const float4*>(A.x + ch * 8 + 4));
           xr[q][0] = a0.x; xr[q][1] = a0.y; xr[q][2] = a0.z; xr[q][3] = a0.w;
           xr[q][4] = a1.x; xr[q][5] = a1.y; xr[q][6] = a1.z; xr[q][7] = a1.w;
         } else {
 #pragma unroll
           for (int e = 0; e < 8; ++e) xr[q][e] = 0.f;
         }
+      }
+      // This CTA's neurons: warp w takes the neurons w, w + 16, ... of the CTA's list.  One lane fetches the index and,
+      // at once, the gate bias (a small load issued after bulk copies would queue behind all of them); the row of the
+      // first ring follows in four pieces from four lanes (several smaller copies from many warps land sooner than one
+      // copy per row issued by one warp: a warp's bulk-copy instructions go out one lane after the other).
+      if (warp < FZ_THREADS / 32) {
+#ifdef LS_DBG_NP1
+        const int np = 1;
+#else
+        const int np = (r1_bytes & 63u) == 0 ? 4 : 1;
+#endif
+        const uint32_t piece = r1_bytes / (uint32_t)np;
+#pragma unroll 1
+        for (int t = warp; t < n_mine; t += FZ_THREADS / 32) {
+          int i = 0;
+          float b = 0.f;
+          if (lane == 0) {
+            i = __ldcg(A.sel_idx + first + t * gsize);
+            if ((unsigned)i >= (unsigned)A.F) { set_status(A.status, ST_BAD_INDEX); i = -1; }
+            if (A.b_gate && i >= 0) b = A.b_gate[i];
+            if (t < n_first) mbar_expect_tx(&s_bar[t], r1_bytes);
+          }
+          i = __shfl_sync(0xffffffffu, i, 0);
+          if (tid == 0) FZ_STAMP_DEP(1, 27, __int_as_float(i));
+          if (t < n_first && lane < np)  // (a rejected index reads row 0; the result is discarded)
+            tma_load_1d(s_r1 + (size_t)t * d + lane * (piece / 2), A.bundles + (size_t)max(i, 0) * bundle_elems + lane * (piece / 2), piece, &s_bar[t]);
+          if (tid == 0) FZ_STAMP(1, 28);
+#ifdef LS_DBG_ARRIVE
+          if (lane == 0 && t < n_first) {
+            FZ_STAMP(1, 440 + 2 * t);
+            while (!mbar_try_wait(&s_bar[t], s_phase[t] & 1u)) {}
+            FZ_STAMP(1, 441 + 2 * t);
+          }
+#endif
+          if (lane == 0) { s_myidx[t] = i; s_mybias[t] = b; }
+          if (tid == 0) FZ_STAMP_DEP(1, 29, b);
+        }
+      }
+#pragma unroll
+      for (int q = 0; q < CPT; ++q)
 #pragma unroll
         for (int e = 0; e < 8; ++e) sq = fma((double)xr[q][e], (double)xr[q][e], sq);
-      }
       sq = warp_sum(sq);
+      if (tid == 0) FZ_STAMP_DEP(1, 31, (float)sq);
       if (lane == 0 && warp < FZ_THREADS / 32) s_redd[warp] = sq;
     }
     __syncthreads();  // indices and the sums of squares visible (the producer warp goes its own way from here)
@@ -890,6 +929,8 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
             if (++slot1 == G1) { slot1 = 0; ++wrap1; }
           }
         }
+        if (tid == 0) FZ_STAMP(0, 4 + rd * 4);
+        if (tid == 480) FZ_STAMP(0, 140 + rd * 4);
         float pg[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int q = 0; q < CPT; ++q) {
@@ -906,11 +947,14 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
             }
           }
         }
+        if (tid == 0) FZ_STAMP_DEP(0, 100 + rd * 4, pg[0] + pg[1] + pg[2] + pg[3]);
+        if (tid == 480) FZ_STAMP_DEP(0, 141 + rd * 4, pg[0] + pg[1] + pg[2] + pg[3]);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
 #pragma unroll
           for (int u = 0; u < 4; ++u) pg[u] += __shfl_xor_sync(0xffffffffu, pg[u], o);
         }
+        if (tid == 480) FZ_STAMP_DEP(0, 142 + rd * 4, pg[0] + pg[1] + pg[2] + pg[3]);
         if (lane == 0) *reinterpret_cast<float4*>(red + warp * FZ_NG1 + e0) = make_float4(pg[0], pg[1], pg[2], pg[3]);
       }
       if (tid == 0) FZ_STAMP(0, 2 + rd * 4);
@@ -1445,8 +1489,13 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
     named_bar_sync(1, FZ_THREADS);
     if (tid == 0) {
       grid_barrier_thread0(A, G);
-    } else if (tid >= 32 && A.spec_ptr && !selects) {
-      speculate(tid - 32, i_lo, n_own);
+    } else {
+      if (tid >= 32 && A.spec_ptr && !selects) speculate(tid - 32, i_lo, n_own);
+      if (A.xs_put >= 0) {  // the next layer's x (complete since the second barrier) waits in shared memory for its start
+        float4* xs = reinterpret_cast<float4*>(smem + A.xs_put);
+#pragma unroll 1
+        for (int c4 = tid - 1; c4 < (d >> 2); c4 += FZ_THREADS - 1) xs[c4] = __ldcg(reinterpret_cast<const float4*>(A.x_out) + c4);
+      }
     }
     named_bar_sync(1, FZ_THREADS);
     if (tid == 0) FZ_STAMP(1, 5);
@@ -1517,25 +1566,40 @@ __global__ void __launch_bounds__(FZ_BLOCK, 1)
   const int G = gridDim.x, cta = blockIdx.x, tid = threadIdx.x;
   constexpr int NW = sizeof(FusedArgs) / 4;
   int known_count = -1;
+  // The arguments of layer m go to sh.args[m & 1]: layer 0's here, every later layer's by the producer warp while the
+  // layer before it runs (that warp leaves the layer early), so a layer starts without a round trip to global memory.
+  auto fetch_args = [&](int m, int t0, int nt) {
+    FusedArgs& a = sh.args[m > 0];
 #pragma unroll 1
-  for (int n = 0; n < n_layers; ++n) {
+    for (int w = t0; w < NW; w += nt) reinterpret_cast<uint32_t*>(&a)[w] = __ldcg(reinterpret_cast<const uint32_t*>(&g_args[m]) + w);
+  };
+  auto patch_args = [&](int m) {  // (one thread, after the copy is visible to it)
+    FusedArgs& a = sh.args[m > 0];
+    a.K = C.K;
+    a.k_next = C.k_next;
+    if (m == 0) { a.x = C.x_in; a.sel_idx = C.sel_idx; a.sel_count = C.sel_count; a.sel_cap = C.sel_cap; }
+    if (m == n_layers - 1) {
+      a.x_out = C.x_out;
+      a.next_idx = C.out_idx; a.next_count = C.out_count; a.next_mask = C.out_mask; a.next_scores = C.out_scores; a.next_cap = C.out_cap;
+    }
+  };
+  if (n_layers > 0) {
     if (tid == 0) FZ_STAMP(1, 24);
-#pragma unroll 1
-    for (int w = tid; w < NW; w += FZ_BLOCK) reinterpret_cast<uint32_t*>(&sh.args)[w] = reinterpret_cast<const uint32_t*>(&g_args[n])[w];
+    fetch_args(0, tid, FZ_BLOCK);
+    __syncthreads();
+    if (tid == 0) patch_args(0);
     __syncthreads();
     if (tid == 0) FZ_STAMP(1, 25);
-    if (tid == 0) {
-      FusedArgs& a = sh.args;
-      a.K = C.K;
-      a.k_next = C.k_next;
-      if (n == 0) { a.x = C.x_in; a.sel_idx = C.sel_idx; a.sel_count = C.sel_count; a.sel_cap = C.sel_cap; }
-      if (n == n_layers - 1) {
-        a.x_out = C.x_out;
-        a.next_idx = C.out_idx; a.next_count = C.out_count; a.next_mask = C.out_mask; a.next_scores = C.out_scores; a.next_cap = C.out_cap;
-      }
+  }
+#pragma unroll 1
+  for (int n = 0; n < n_layers; ++n) {
+    const FusedArgs& A = sh.args[0];
+    if (n > 0) {  // fetched while the layer before ran
+#pragma unroll 1
+      for (int w = tid; w < NW; w += FZ_BLOCK) reinterpret_cast<uint32_t*>(&sh.args[0])[w] = reinterpret_cast<const uint32_t*>(&sh.args[1])[w];
+      __syncthreads();
     }
-    __syncthreads();
-    const FusedArgs& A = sh.args;
+    if (tid == 0) FZ_STAMP(1, 26);
     if (cta == G - 1 && C.tr_x && tid < FZ_THREADS) {  // what enters this layer (x_out may overwrite x)
 #pragma unroll 1
       for (int c = tid; c < A.d; c += FZ_THREADS) C.tr_x[(size_t)n * A.d + c] = __ldcg(A.x + c);
@@ -1548,6 +1612,11 @@ __global__ void __launch_bounds__(FZ_BLOCK, 1)
     }
     fused_layer<WD, CPT>(A, smem, sh, n == 0, known_count);
     known_count = A.has_next ? min(min(A.k_next, A.Fn), A.next_cap) : -1;  // what this layer wrote to *next_count
+    if (tid >= FZ_THREADS && n + 1 < n_layers) {  // the producer warp is back early: the next layer's arguments
+      fetch_args(n + 1, tid - FZ_THREADS, FZ_BLOCK - FZ_THREADS);
+      __syncwarp();
+      if (tid == FZ_THREADS) patch_args(n + 1);
+    }
     if (tid < FZ_THREADS) {
       grid_barrier(A, G);                       // layer boundary: x_out and the refined selection are visible to all
 #ifdef LS_FZ_TIMING
@@ -1558,11 +1627,12 @@ __global__ void __launch_bounds__(FZ_BLOCK, 1)
         g_fz_timing[1][300 + n] = (long long)gt;
       }
 #endif
+      if (tid == 0) { sh.round = 0; sh.nsurv = 0; sh.done = 0; }  // the stream phase's counters start every layer at zero
     }
     __syncthreads();
   }
   if (tid < FZ_THREADS && n_layers > 0) {
-    const FusedArgs& A = sh.args;  // the last layer; every CTA is past its final barrier
+    const FusedArgs& A = sh.args[0];  // the last layer; every CTA is past its final barrier
     if (cta == G - 1 && C.tr_x) {
 #pragma unroll 1
       for (int c = tid; c < A.d; c += FZ_THREADS) C.tr_x[(size_t)n_layers * A.d + c] = __ldcg(A.x_out + c);
