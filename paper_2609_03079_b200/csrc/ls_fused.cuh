@@ -40,6 +40,7 @@ constexpr int FZ_THREADS = 512;        // compute threads (16 warps)
 constexpr int FZ_BLOCK = FZ_THREADS + 32;  // plus the producer warp
 constexpr int FZ_NG = 3;          // survivors processed per batch of the second ring
 constexpr int FZ_NG1 = 4;         // most neurons per round of the first ring
+constexpr int FZ_NB2 = 8;         // most survivors per batch of the second ring
 constexpr int FZ_NB = 4096;       // fine score bins per evaluation
 constexpr int FZ_FIN_PARTS = 32;  // CTAs that share the ranking of the final evaluation
 constexpr int FZ_CUTLIST = 1024;  // entries of the cut bin ranked in shared memory (a fuller bin falls back to global loops)
@@ -319,7 +320,7 @@ inline FusedSmemLayout fused_layout(int d, int n_mat, int r, int Fn, int G, int 
   L.ns_cta = (nsl + G - 1) / G;
   const size_t a_bytes = has_next ? (size_t)L.ns_cta * r * FZ_SL * 2 : 0;
   L.bar_off = take(FZ_NBAR * 8);
-  L.red_off = take(2 * 16 * FZ_NG1 * 4);             // stream dot partials, double-buffered: [2][warp][FZ_NG1]
+  L.red_off = take(2 * 16 * FZ_NG1 * 4 + 16 * FZ_NB2 * 4);  // stream dot partials: first ring [2][warp][FZ_NG1] (double-buffered), second ring [warp][FZ_NB2]
   L.redd_off = take(32 * 8);                         // fp64 partials of block reductions
   L.mine_off = take((size_t)FZ_MAX_MINE * 16);       // this CTA's neurons, their gate biases; the survivors, their activations
   L.pc_off = take((size_t)L.per * 4);
@@ -361,6 +362,7 @@ struct FusedShared {
   int stage, g_lo, gsize;            // this CTA's stage, the first CTA of the stage's group and the group's size
   unsigned phase[FZ_NBAR];           // phases every mbarrier has completed in earlier layers of the launch
   int nsurv, done;                   // survivors found so far / consumed so far (read by the producer)
+  int b_hi, b_last;                  // the second ring's current batch ends before survivor b_hi; it is the last one
   double inv[FZ_EPAD + 32];          // 1 / rms per evaluation; behind them: partial-sum slots per score tile (ints)
   unsigned long long kmm[2 * 16];
 };
@@ -742,8 +744,10 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
     float* s_mybias = reinterpret_cast<float*>(s_myidx + FZ_MAX_MINE);
     int* s_surv = s_myidx + 2 * FZ_MAX_MINE;                       // surviving neurons, in the order they were found
     float* s_qa = reinterpret_cast<float*>(s_myidx + 3 * FZ_MAX_MINE);  // their activations
-    const int n_first = min(n_mine, G1);  // rows of the first ring requested in the prologue, by the compute warps
-    int issued1 = n_first;                // (producer warp) rows of the first ring requested so far
+    // The first ring is used in rounds of NG1 neurons: G1R rounds fit; the rows of a round complete one barrier together
+    // (a wait costs a warp some two hundred clocks even when the data is there: one per round, not one per row).
+    const int G1R = G1 / NG1;
+    const int n_first = min(n_mine, G1R * NG1);  // rows requested in the prologue, by the compute warps
     float xr[CPT][8];
     {
       double sq = 0.0;
@@ -782,20 +786,13 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
             i = __ldcg(A.sel_idx + first + t * gsize);
             if ((unsigned)i >= (unsigned)A.F) { set_status(A.status, ST_BAD_INDEX); i = -1; }
             if (A.b_gate && i >= 0) b = A.b_gate[i];
-            if (t < n_first) mbar_expect_tx(&s_bar[t], r1_bytes);
+            if (t < n_first && t % NG1 == 0) mbar_expect_tx(&s_bar[t / NG1], (uint32_t)min(NG1, n_mine - t) * r1_bytes);
           }
           i = __shfl_sync(0xffffffffu, i, 0);
           if (tid == 0) FZ_STAMP_DEP(1, 27, __int_as_float(i));
           if (t < n_first && lane < np)  // (a rejected index reads row 0; the result is discarded)
-            tma_load_1d(s_r1 + (size_t)t * d + lane * (piece / 2), A.bundles + (size_t)max(i, 0) * bundle_elems + lane * (piece / 2), piece, &s_bar[t]);
+            tma_load_1d(s_r1 + (size_t)t * d + lane * (piece / 2), A.bundles + (size_t)max(i, 0) * bundle_elems + lane * (piece / 2), piece, &s_bar[t / NG1]);
           if (tid == 0) FZ_STAMP(1, 28);
-#ifdef LS_DBG_ARRIVE
-          if (lane == 0 && t < n_first) {
-            FZ_STAMP(1, 440 + 2 * t);
-            while (!mbar_try_wait(&s_bar[t], s_phase[t] & 1u)) {}
-            FZ_STAMP(1, 441 + 2 * t);
-          }
-#endif
           if (lane == 0) { s_myidx[t] = i; s_mybias[t] = b; }
           if (tid == 0) FZ_STAMP_DEP(1, 29, b);
         }
@@ -813,36 +810,26 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
 
     if (warp == FZ_THREADS / 32) {
       // ============================================= producer warp ================================================
-      // Issues every bulk copy, so that the compute warps never pay for it; the whole warp runs the loop and lane l
-      // issues the l-th copy of a batch.  First ring: the first row of each of this CTA's neurons (gate, or the only
-      // input matrix), as many as fit at once, topped up as rounds finish.  Second ring: the rest of a neuron's bundle
-      // (up and down rows), fetched only for the neurons whose activation survived, as slots come free.  The compute
-      // warps publish rounds finished, survivors found and survivors consumed in sh.round / sh.nsurv / sh.done.
+      // After every round of the first ring it turns the compute warps' partial dot products into activations, keeps
+      // the list of survivors, and issues every further bulk copy (lane l the l-th copy of a batch): the next rounds
+      // of the first ring when more neurons than fit were assigned, and, for the survivors only, the rest of the bundle
+      // (up and down rows) into the second ring as slots come free.  The compute warps never wait for any of this:
+      // they signal a finished round on a named barrier without blocking and go on to the next round's rows.
       {
-        int issued2 = 0, slot2 = 0, rounds = 0, nsurv = 0;
-        bool a_sent = false, ok = true;
+        float inv_rms_p = 1.0f;
+        if (A.norm == 0) {
+          double tot = 0.0;
+#pragma unroll 4
+          for (int w = 0; w < FZ_THREADS / 32; ++w) tot += s_redd[w];
+          inv_rms_p = (float)fz_rsqrt(fma(tot, A.inv_d, (double)A.eps));
+        }
+        int issued2 = 0, nsurv = 0;
+        bool ok = true;
         const long long t0 = clock64();
-        while (true) {
-          // top the first ring up to the rows that may be in flight
-          const int want = min(n_mine, rounds * NG1 + G1);
-          if (issued1 + lane < want) {
-            const int it = issued1 + lane, sl1 = it % G1;
-            int i = s_myidx[it];
-            if (i < 0) i = 0;  // a rejected index: read row 0, the result is discarded
-            uint64_t* bar = &s_bar[sl1];
-            mbar_expect_tx(bar, r1_bytes);
-            tma_load_1d(s_r1 + (size_t)sl1 * d, A.bundles + (size_t)i * bundle_elems, r1_bytes, bar);
-          }
-          issued1 = max(issued1, want);
-          if (!a_sent && A.has_next && !lay.a_alias) {  // A slices with a place of their own: right behind the first burst
-            a_sent = true;
-            if (lane == 0) fz_issue_a(A, s_A, &s_bar[FZ_BAR_A], cta, G, nsl);
-          }
-          // survivors whose slot is free (slots carved from the first ring only once that ring is idle)
-          int done;
-          asm volatile("ld.acquire.cta.shared.s32 %0, [%1];" : "=r"(done) : "r"(smem_u32(&sh.done)) : "memory");
-          int n_can = min(nsurv - issued2, G2T - (issued2 - done));
-          if (rounds < n_rounds) n_can = min(n_can, slot2 < G2 ? G2 - slot2 : 0);
+        // (after the rounds) survivors whose slot is free
+        auto issue_survivors = [&](int done) {
+          const int slot2 = issued2 % G2T;  // (survivor q goes to slot q % G2T)
+          const int n_can = min(nsurv - issued2, G2T - (issued2 - done));
           if (lane < n_can) {
             int sl2 = slot2 + lane;
             if (sl2 >= G2T) sl2 -= G2T;
@@ -853,29 +840,85 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
             tma_load_1d(dst, A.bundles + (size_t)i * bundle_elems + d, r2_bytes, bar);
             if (A.tr_survive) atomicOr(&A.tr_survive[i >> 5], 1u << (i & 31));
           }
-          if (n_can > 0) {
-            issued2 += n_can;
-            slot2 += n_can;
-            if (slot2 >= G2T) slot2 -= G2T;
+          if (n_can > 0) issued2 += n_can;
+        };
+        if (!lay.a_alias && A.has_next && lane == 0) fz_issue_a(A, s_A, &s_bar[FZ_BAR_A], cta, G, nsl);  // A slices with a place of their own
+#pragma unroll 1
+        for (int rd = 0; rd < n_rounds; ++rd) {
+          named_bar_sync(2 + (rd & 1), FZ_BLOCK);  // every compute warp has left its partial sums of round rd
+          const int it0 = rd * NG1, nn = min(NG1, n_mine - it0);
+          const float* red = s_red + (rd & 1) * (FZ_THREADS / 32) * FZ_NG1;  // [warp][FZ_NG1]
+          float a = 0.f;
+          int i = -1;
+          {
+            // lane l adds the partial sums of neuron l & 3 left by the warps 2 (l >> 2) and 2 (l >> 2) + 1; three
+            // exchanges complete the sums (always in the same order)
+            float v = red[(2 * (lane >> 2)) * FZ_NG1 + (lane & 3)] + red[(2 * (lane >> 2) + 1) * FZ_NG1 + (lane & 3)];
+            v += __shfl_xor_sync(0xffffffffu, v, 4);
+            v += __shfl_xor_sync(0xffffffffu, v, 8);
+            v += __shfl_xor_sync(0xffffffffu, v, 16);
+            if (lane < nn) {
+              i = s_myidx[it0 + lane];
+              a = fmaxf(v * inv_rms_p + s_mybias[it0 + lane], 0.f);
+              if (i < 0) a = 0.f;
+            }
           }
-          if (rounds == n_rounds && issued2 == nsurv) break;  // every row of this layer has been requested
-          // wait for news: a round finished (more survivors, room in the first ring) or survivors consumed
-          int rnow, dnow;
+          const unsigned surv = __ballot_sync(0xffffffffu, a != 0.f);
+          {
+            // a survivor's lane requests the rest of its bundle at once when a slot is certainly free (nothing consumed yet)
+            const int limit = rd + 1 == n_rounds ? G2T : G2;
+            const bool direct = issued2 == nsurv;
+            if (a != 0.f) {
+              const int pos = nsurv + __popc(surv & ((1u << lane) - 1u));
+              if (direct && pos < limit) {
+                uint64_t* bar = &s_bar[FZ_BAR_R2 + pos];
+                uint16_t* dst = pos < G2 ? s_r2 + (size_t)pos * (A.n_mat - 1) * d : s_r1 + (size_t)(pos - G2) * (A.n_mat - 1) * d;
+                mbar_expect_tx(bar, r2_bytes);
+                tma_load_1d(dst, A.bundles + (size_t)i * bundle_elems + d, r2_bytes, bar);
+                if (A.tr_survive) atomicOr(&A.tr_survive[i >> 5], 1u << (i & 31));
+              }
+              s_surv[pos] = i;
+              s_qa[pos] = a;
+            }
+            const int nnew = nsurv + __popc(surv);
+            if (direct) issued2 = max(issued2, min(nnew, limit));
+            nsurv = nnew;
+          }
+          __syncwarp();
+          if (lane == 0) {
+            sh.nsurv = nsurv;
+            asm volatile("st.release.cta.shared.s32 [%0], %1;" ::"r"(smem_u32(&s_round)), "r"(rd + 1) : "memory");
+          }
+          // the round's slot is free: the round G1R ahead moves in
+          const int rn = rd + G1R;
+          if (rn < n_rounds) {
+            const int t1 = rn * NG1, n1 = min(NG1, n_mine - t1), rs = rn % G1R;
+            if (lane == 0) mbar_expect_tx(&s_bar[rs], (uint32_t)n1 * r1_bytes);
+            __syncwarp();
+            if (lane < n1) {
+              int i1 = s_myidx[t1 + lane];
+              if (i1 < 0) i1 = 0;  // a rejected index: read row 0, the result is discarded
+              tma_load_1d(s_r1 + (size_t)(rs * NG1 + lane) * d, A.bundles + (size_t)i1 * bundle_elems, r1_bytes, &s_bar[rs]);
+            }
+          }
+          if (tid == FZ_THREADS) FZ_STAMP(0, 3 + rd * 4);
+        }
+        // the remaining survivors (the first ring is idle now: every slot may be used), as the compute warps consume the second ring
+        int done = 0;
+#pragma unroll 1
+        while (issued2 < nsurv) {
+          issue_survivors(done);
+          if (issued2 == nsurv) break;
+          int dnow;
           while (true) {
-            asm volatile("ld.acquire.cta.shared.s32 %0, [%1];" : "=r"(rnow) : "r"(smem_u32(&s_round)) : "memory");
             asm volatile("ld.acquire.cta.shared.s32 %0, [%1];" : "=r"(dnow) : "r"(smem_u32(&sh.done)) : "memory");
-            rnow = __shfl_sync(0xffffffffu, rnow, 0);  // (one view for the whole warp)
-            dnow = __shfl_sync(0xffffffffu, dnow, 0);
-            if (rnow > rounds || (dnow > done && issued2 < nsurv)) break;
+            dnow = __shfl_sync(0xffffffffu, dnow, 0);  // (one view for the whole warp)
+            if (dnow > done) break;
             if (__shfl_sync(0xffffffffu, (int)(clock64() - t0 > FZ_SPIN_CYCLES), 0)) { ok = false; break; }
             __nanosleep(64);  // the poll shares an instruction scheduler with four compute warps
           }
           if (!ok) { if (lane == 0) set_status(A.status, ST_TIMEOUT); break; }
-          if (rnow > rounds) {
-            rounds = min(rnow, n_rounds);
-            asm volatile("ld.acquire.cta.shared.s32 %0, [%1];" : "=r"(nsurv) : "r"(smem_u32(&sh.nsurv)) : "memory");
-            nsurv = __shfl_sync(0xffffffffu, nsurv, 0);
-          }
+          done = dnow;
         }
         // The next layer's predictor operands that share bytes with the rings wait until the compute warps have drained them.
         if (A.has_next && ok) {
@@ -909,28 +952,35 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
     if (tid == 0) FZ_STAMP(0, 0);
     if (tid == 0) { FZ_CSTAMP(1); FZ_CVAL(8, n_mine); FZ_CVAL(10, stage); }
 
-    // ---- first ring: the pre-activation of every neuron, a ring-full of neurons per round; survivors go to the producer -
-    int nsurv = 0, slot1 = 0;
-    unsigned wrap1 = 0;
+    // ---- first ring: the dot products of every neuron's first row with x, a round of NG1 neurons at a time; each warp
+    //      leaves its partial sums for the producer warp and moves on ---------------------------------------------------
+    int rslot = 0;
+    unsigned wrapr = 0;
+#ifdef LS_FZ_TIMING
+    unsigned tw[6] = {0, 0, 0, 0, 0, 0};
+#endif
 #pragma unroll 1
     for (int rd = 0; rd < n_rounds; ++rd) {
       const int it0 = rd * NG1;
       const int nn = min(NG1, n_mine - it0);
       if (tid == 0) FZ_STAMP(0, 1 + rd * 4);
+#ifdef LS_FZ_TIMING
+      if (rd == 1) tw[0] = clock();
+      if (rd == 2) tw[5] = clock();
+#endif
+      // the partial sums and the named barrier of round rd - 2 are used again: the producer must be through with them
+      if (rd >= 2) {
+        if (lane == 0) fz_wait_round(&s_round, rd - 1, A.status);
+        __syncwarp();
+      }
       float* red = s_red + (rd & 1) * (FZ_THREADS / 32) * FZ_NG1;  // [warp][FZ_NG1]
-#pragma unroll 1
-      for (int e0 = 0; e0 < nn; e0 += 4) {  // four neurons at a time: four independent chains of loads, FMAs and shuffles
-        const uint16_t* grow[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          grow[u] = s_r1 + (size_t)slot1 * d;
-          if (e0 + u < nn) {
-            mbar_wait(&s_bar[slot1], (s_phase[slot1] + wrap1) & 1u, A.status);
-            if (++slot1 == G1) { slot1 = 0; ++wrap1; }
-          }
-        }
-        if (tid == 0) FZ_STAMP(0, 4 + rd * 4);
-        if (tid == 480) FZ_STAMP(0, 140 + rd * 4);
+      mbar_wait(&s_bar[rslot], (s_phase[rslot] + wrapr) & 1u, A.status);
+      const uint16_t* g0 = s_r1 + (size_t)rslot * NG1 * d;
+      if (++rslot == G1R) { rslot = 0; ++wrapr; }
+#ifdef LS_FZ_TIMING
+      if (rd == 1) tw[1] = clock();
+#endif
+      {  // up to four neurons: four independent chains of loads, FMAs and shuffles
         float pg[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int q = 0; q < CPT; ++q) {
@@ -938,117 +988,144 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
           if (ch < nchunk) {
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
-              if (e0 + u < nn) {
+              if (u < nn) {
                 float w[8];
-                unpack8<WD>(*reinterpret_cast<const uint4*>(grow[u] + ch * 8), w);
+                unpack8<WD>(*reinterpret_cast<const uint4*>(g0 + (size_t)u * d + ch * 8), w);
 #pragma unroll
                 for (int t = 0; t < 8; ++t) pg[u] = fmaf(w[t], xr[q][t], pg[u]);
               }
             }
           }
         }
-        if (tid == 0) FZ_STAMP_DEP(0, 100 + rd * 4, pg[0] + pg[1] + pg[2] + pg[3]);
-        if (tid == 480) FZ_STAMP_DEP(0, 141 + rd * 4, pg[0] + pg[1] + pg[2] + pg[3]);
+#ifdef LS_FZ_TIMING
+        if (rd == 1) asm volatile("{ .reg .f32 t_; add.f32 t_, %1, %2; mov.u32 %0, %%clock; }" : "=r"(tw[2]) : "f"(pg[0] + pg[1]), "f"(pg[2] + pg[3]));
+#endif
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
 #pragma unroll
           for (int u = 0; u < 4; ++u) pg[u] += __shfl_xor_sync(0xffffffffu, pg[u], o);
         }
-        if (tid == 480) FZ_STAMP_DEP(0, 142 + rd * 4, pg[0] + pg[1] + pg[2] + pg[3]);
-        if (lane == 0) *reinterpret_cast<float4*>(red + warp * FZ_NG1 + e0) = make_float4(pg[0], pg[1], pg[2], pg[3]);
+#ifdef LS_FZ_TIMING
+        if (rd == 1) asm volatile("{ .reg .f32 t_; add.f32 t_, %1, %2; mov.u32 %0, %%clock; }" : "=r"(tw[3]) : "f"(pg[0] + pg[1]), "f"(pg[2] + pg[3]));
+#endif
+        if (lane == 0) *reinterpret_cast<float4*>(red + warp * FZ_NG1) = make_float4(pg[0], pg[1], pg[2], pg[3]);
       }
       if (tid == 0) FZ_STAMP(0, 2 + rd * 4);
-      named_bar_sync(1, FZ_THREADS);  // partials visible; every thread is done with the round's ring slots
-      if (warp == 0) {  // pre-activations; the neurons that survive the ReLU join the list the producer fetches from
-        float a = 0.f;
-        int i = -1;
-        if (lane < nn) {
-          float v = 0.f;
-#pragma unroll 4
-          for (int w = 0; w < FZ_THREADS / 32; ++w) v += red[w * FZ_NG1 + lane];
-          i = s_myidx[it0 + lane];
-          a = fmaxf(v * inv_rms + s_mybias[it0 + lane], 0.f);
-          if (i < 0) a = 0.f;
-        }
-        const unsigned surv = __ballot_sync(0xffffffffu, a != 0.f);
-        if (a != 0.f) {
-          const int pos = nsurv + __popc(surv & ((1u << lane) - 1u));
-          s_surv[pos] = i;
-          s_qa[pos] = a;
-        }
-        nsurv += __popc(surv);
-        if (lane == 0) {
-          asm volatile("st.release.cta.shared.s32 [%0], %1;" ::"r"(smem_u32(&sh.nsurv)), "r"(nsurv) : "memory");
-          asm volatile("st.release.cta.shared.s32 [%0], %1;" ::"r"(smem_u32(&s_round)), "r"(rd + 1) : "memory");
-        }
-        if (tid == 0) FZ_STAMP(0, 3 + rd * 4);
-      }
-      // (no second barrier: the partials are double-buffered, and warp 0 joins the next round's barrier only after it has
-      // read this round's)
+      __syncwarp();
+      asm volatile("bar.arrive %0, %1;" ::"r"(2 + (rd & 1)), "r"(FZ_BLOCK) : "memory");  // (does not block)
+#ifdef LS_FZ_TIMING
+      if (rd == 1) tw[4] = clock();
+#endif
     }
-    named_bar_sync(1, FZ_THREADS);
-    nsurv = sh.nsurv;
     if (tid == 0) FZ_STAMP(0, 500);
-    if (tid == 0) { FZ_CSTAMP(2); FZ_CVAL(9, nsurv); }
+#ifdef LS_FZ_TIMING
+    if (lane == 0 && blockIdx.x == 0)
+      for (int i_ = 0; i_ < 6; ++i_) g_fz_timing[0][160 + warp * 6 + i_] = tw[i_];
+#endif
 
-    // ---- second ring: the survivors, three at a time: (gated) their up rows complete the activations, then their down
-    //      rows, scaled, join the CTA's partial output (kept in registers) ------------------------------------------------
+    // ---- second ring: the survivors, in batches of up to FZ_NB2, as the producer finds them (a batch starts with whatever
+    //      is known, so the survivors of the early rounds are worked on while the last round's rows are still in flight):
+    //      (gated) their up rows complete the activations, then their down rows, scaled, join the CTA's partial output
+    //      (kept in registers).  Survivor q sits in slot q % G2T and is the (q / G2T)-th use of that slot in this layer.
     float yacc[CPT][8];
 #pragma unroll
     for (int q = 0; q < CPT; ++q)
 #pragma unroll
       for (int e = 0; e < 8; ++e) yacc[q][e] = 0.f;
-    int slot2 = 0;
-    unsigned wrap2 = 0;
+    float* red2 = s_red + 2 * (FZ_THREADS / 32) * FZ_NG1;  // [warp][FZ_NB2]
+    const size_t r2_elems = (size_t)(A.n_mat - 1) * d;
+    int q0 = 0, slot0 = 0;  // the batch starts at survivor q0, which sits in slot slot0 = q0 % G2T
+    unsigned wrap0 = 0;     // q0 / G2T
 #pragma unroll 1
-    for (int q0 = 0; q0 < nsurv; q0 += FZ_NG) {
-      const int nb = min(FZ_NG, nsurv - q0);
-      int sl[FZ_NG];
-      float pu[FZ_NG];
+    while (true) {
+      if (warp == 0) {
+        // what is known: survivors [q0, known) are listed; after round n_rounds the list is final
+        int known = 0, fin = 0;
+        if (lane == 0) {
+          const long long t0 = clock64();
+          while (true) {
+            int rnow;
+            asm volatile("ld.acquire.cta.shared.s32 %0, [%1];" : "=r"(rnow) : "r"(smem_u32(&s_round)) : "memory");
+            known = *reinterpret_cast<volatile int*>(&sh.nsurv);
+            fin = rnow >= n_rounds;
+            if (known > q0 || fin) break;
+            if (clock64() - t0 > FZ_SPIN_CYCLES) { set_status(A.status, ST_TIMEOUT); fin = 1; break; }
+          }
+        }
+        known = __shfl_sync(0xffffffffu, known, 0);
+        fin = __shfl_sync(0xffffffffu, fin, 0);
+        const int hi = min(known, q0 + min(FZ_NB2, G2T));  // (a batch never needs more slots than there are)
+        if (q0 + lane < hi) {  // the batch's rows: each lane waits for one
+          int sl = slot0 + lane;
+          unsigned wr = wrap0;
+          if (sl >= G2T) { sl -= G2T; ++wr; }
+          mbar_wait(&s_bar[FZ_BAR_R2 + sl], (s_phase[FZ_BAR_R2 + sl] + wr) & 1u, A.status);
+        }
+        __syncwarp();
+        if (lane == 0) { sh.b_hi = hi; sh.b_last = (fin && hi == known) ? 1 : 0; }
+      }
+      named_bar_sync(1, FZ_THREADS);  // the batch is known to all, its rows have landed
+      const int hi = *reinterpret_cast<volatile int*>(&sh.b_hi), last = *reinterpret_cast<volatile int*>(&sh.b_last);
+      const int nb = hi - q0;
+      if (nb > 0) {
+        if (up_off >= 0) {
+#pragma unroll 1
+          for (int e0 = 0; e0 < nb; e0 += 4) {  // four up rows at a time: four independent chains of loads, FMAs and shuffles
+            float pu[4] = {0.f, 0.f, 0.f, 0.f};
+            const uint16_t* urow[4];
 #pragma unroll
-      for (int e = 0; e < FZ_NG; ++e) {
-        pu[e] = 0.f;
-        sl[e] = slot2;
-        if (e < nb) {
-          mbar_wait(&s_bar[FZ_BAR_R2 + slot2], (s_phase[FZ_BAR_R2 + slot2] + wrap2) & 1u, A.status);
-          if (up_off >= 0) {
-            const uint16_t* urow = (slot2 < G2 ? s_r2 + (size_t)slot2 * (A.n_mat - 1) * d : s_r1 + (size_t)(slot2 - G2) * (A.n_mat - 1) * d);
+            for (int u = 0; u < 4; ++u) {
+              int sl = slot0 + e0 + u;
+              if (sl >= G2T) sl -= G2T;
+              urow[u] = sl < G2 ? s_r2 + (size_t)sl * r2_elems : s_r1 + (size_t)(sl - G2) * r2_elems;
+            }
 #pragma unroll
             for (int q = 0; q < CPT; ++q) {
               const int ch = tid + q * FZ_THREADS;
               if (ch < nchunk) {
-                float w[8];
-                unpack8<WD>(*reinterpret_cast<const uint4*>(urow + ch * 8), w);
 #pragma unroll
-                for (int t = 0; t < 8; ++t) pu[e] = fmaf(w[t], xr[q][t], pu[e]);
+                for (int u = 0; u < 4; ++u) {
+                  if (e0 + u < nb) {
+                    float w[8];
+                    unpack8<WD>(*reinterpret_cast<const uint4*>(urow[u] + ch * 8), w);
+#pragma unroll
+                    for (int t = 0; t < 8; ++t) pu[u] = fmaf(w[t], xr[q][t], pu[u]);
+                  }
+                }
               }
             }
+            // four sums over the warp in six shuffles: at every step a lane hands over the half it does not keep
+            const bool h16 = (lane & 16) != 0, h8 = (lane & 8) != 0;
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+              const float give = h16 ? pu[u] : pu[u + 2], keep = h16 ? pu[u + 2] : pu[u];
+              pu[u] = keep + __shfl_xor_sync(0xffffffffu, give, 16);
+            }
+            {
+              const float give = h8 ? pu[0] : pu[1], keep = h8 ? pu[1] : pu[0];
+              pu[0] = keep + __shfl_xor_sync(0xffffffffu, give, 8);
+            }
+            pu[0] += __shfl_xor_sync(0xffffffffu, pu[0], 4);
+            pu[0] += __shfl_xor_sync(0xffffffffu, pu[0], 2);
+            pu[0] += __shfl_xor_sync(0xffffffffu, pu[0], 1);
+            if ((lane & 7) == 0) red2[warp * FZ_NB2 + e0 + (lane >> 3)] = pu[0];  // lane 8 u holds the sum of row e0 + u
           }
-          if (++slot2 == G2T) { slot2 = 0; ++wrap2; }
+          named_bar_sync(1, FZ_THREADS);
+          if (warp == 0) {  // lane l adds the partial sums of survivor l & 7 left by the warps 4 (l >> 3) .. 4 (l >> 3) + 3
+            const int w4 = 4 * (lane >> 3), e = lane & 7;
+            float v = (red2[w4 * FZ_NB2 + e] + red2[(w4 + 1) * FZ_NB2 + e]) + (red2[(w4 + 2) * FZ_NB2 + e] + red2[(w4 + 3) * FZ_NB2 + e]);
+            v += __shfl_xor_sync(0xffffffffu, v, 8);
+            v += __shfl_xor_sync(0xffffffffu, v, 16);
+            if (lane < nb) s_qa[q0 + lane] *= v * inv_rms;
+          }
+          named_bar_sync(1, FZ_THREADS);
         }
-      }
-      if (up_off >= 0) {
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-#pragma unroll
-          for (int e = 0; e < FZ_NG; ++e) pu[e] += __shfl_xor_sync(0xffffffffu, pu[e], o);
-        }
-        float* red = s_red + ((q0 / FZ_NG) & 1) * (FZ_THREADS / 32) * 4;
-        if (lane == 0) *reinterpret_cast<float4*>(red + warp * 4) = make_float4(pu[0], pu[1], pu[2], 0.f);
-        named_bar_sync(1, FZ_THREADS);
-        if (warp == 0 && lane < nb) {
-          float v = 0.f;
-#pragma unroll 4
-          for (int w = 0; w < FZ_THREADS / 32; ++w) v += red[w * 4 + lane];
-          s_qa[q0 + lane] *= v * inv_rms;
-        }
-        named_bar_sync(1, FZ_THREADS);
-      }
-#pragma unroll
-      for (int e = 0; e < FZ_NG; ++e) {
-        if (e < nb) {
+#pragma unroll 1
+        for (int e = 0; e < nb; ++e) {
           const float a = s_qa[q0 + e];
-          const uint16_t* row = (sl[e] < G2 ? s_r2 + (size_t)sl[e] * (A.n_mat - 1) * d : s_r1 + (size_t)(sl[e] - G2) * (A.n_mat - 1) * d) + dn_off;
+          int sl = slot0 + e;
+          if (sl >= G2T) sl -= G2T;
+          const uint16_t* row = (sl < G2 ? s_r2 + (size_t)sl * r2_elems : s_r1 + (size_t)(sl - G2) * r2_elems) + dn_off;
 #pragma unroll
           for (int q = 0; q < CPT; ++q) {
             const int ch = tid + q * FZ_THREADS;
@@ -1060,11 +1137,19 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
             }
           }
         }
+        q0 = hi;
+        slot0 += nb;
+        if (slot0 >= G2T) { slot0 -= G2T; ++wrap0; }
+        if (!last) {
+          named_bar_sync(1, FZ_THREADS);  // every thread is done with the batch's slots: the producer may refill them
+          if (tid == 0) asm volatile("st.release.cta.shared.s32 [%0], %1;" ::"r"(smem_u32(&sh.done)), "r"(q0) : "memory");
+        }
       }
-      named_bar_sync(1, FZ_THREADS);  // every thread is done with the batch's slots: the producer may refill them
-      if (tid == 0) asm volatile("st.release.cta.shared.s32 [%0], %1;" ::"r"(smem_u32(&sh.done)), "r"(q0 + nb) : "memory");
+      if (last) break;
     }
-    used_r1 = n_mine;
+    const int nsurv = q0;
+    if (tid == 0) { FZ_CSTAMP(2); FZ_CVAL(9, nsurv); }
+    used_r1 = n_rounds;
     used_r2 = nsurv;
     named_bar_sync(1, FZ_THREADS);  // nobody reads the rings any more: the producer may overwrite them
     if (tid == 0) asm volatile("st.release.cta.shared.s32 [%0], %1;" ::"r"(smem_u32(&s_round)), "r"(n_rounds + 1) : "memory");
@@ -1524,7 +1609,7 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
   named_bar_sync(1, FZ_THREADS);
   if (tid < FZ_NBAR) {
     unsigned n = 0;
-    if (tid < FZ_MAX_G1) n = used_r1 > tid ? (unsigned)((used_r1 - 1 - tid) / G1 + 1) : 0u;
+    if (tid < FZ_MAX_G1) n = used_r1 > tid ? (unsigned)((used_r1 - 1 - tid) / (G1 / NG1) + 1) : 0u;  // (rounds, one barrier per round-slot)
     else if (tid < FZ_BAR_A) { const int s2 = tid - FZ_BAR_R2; n = used_r2 > s2 ? (unsigned)((used_r2 - 1 - s2) / G2T + 1) : 0u; }
     else n = A.has_next ? 1u : 0u;
     s_phase[tid] += n;
