@@ -1000,15 +1000,23 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
 #ifdef LS_FZ_TIMING
         if (rd == 1) asm volatile("{ .reg .f32 t_; add.f32 t_, %1, %2; mov.u32 %0, %%clock; }" : "=r"(tw[2]) : "f"(pg[0] + pg[1]), "f"(pg[2] + pg[3]));
 #endif
+        {  // four sums over the warp in six shuffles: at every step a lane hands over the half it does not keep
+          const bool h16 = (lane & 16) != 0, h8 = (lane & 8) != 0;
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-#pragma unroll
-          for (int u = 0; u < 4; ++u) pg[u] += __shfl_xor_sync(0xffffffffu, pg[u], o);
+          for (int u = 0; u < 2; ++u) {
+            const float give = h16 ? pg[u] : pg[u + 2], keep = h16 ? pg[u + 2] : pg[u];
+            pg[u] = keep + __shfl_xor_sync(0xffffffffu, give, 16);
+          }
+          const float give = h8 ? pg[0] : pg[1], keep = h8 ? pg[1] : pg[0];
+          pg[0] = keep + __shfl_xor_sync(0xffffffffu, give, 8);
+          pg[0] += __shfl_xor_sync(0xffffffffu, pg[0], 4);
+          pg[0] += __shfl_xor_sync(0xffffffffu, pg[0], 2);
+          pg[0] += __shfl_xor_sync(0xffffffffu, pg[0], 1);
         }
 #ifdef LS_FZ_TIMING
-        if (rd == 1) asm volatile("{ .reg .f32 t_; add.f32 t_, %1, %2; mov.u32 %0, %%clock; }" : "=r"(tw[3]) : "f"(pg[0] + pg[1]), "f"(pg[2] + pg[3]));
+        if (rd == 1) asm volatile("{ .reg .f32 t_; add.f32 t_, %1, %2; mov.u32 %0, %%clock; }" : "=r"(tw[3]) : "f"(pg[0]), "f"(pg[0]));
 #endif
-        if (lane == 0) *reinterpret_cast<float4*>(red + warp * FZ_NG1) = make_float4(pg[0], pg[1], pg[2], pg[3]);
+        if ((lane & 7) == 0) red[warp * FZ_NG1 + (lane >> 3)] = pg[0];  // lane 8 u holds the sum of neuron u
       }
       if (tid == 0) FZ_STAMP(0, 2 + rd * 4);
       __syncwarp();
