@@ -451,9 +451,14 @@ __device__ __noinline__ void fz_select(const FusedArgs& A, int j, int K, int kef
   // exclusive scan of the FZ_NB counts (eight per thread), and the cut bin
   {
     constexpr int PT = FZ_NB / FZ_THREADS;
+    static_assert(PT == 8, "a thread owns eight consecutive counters: two 16-byte accesses");
     unsigned c[PT], tot = 0;
+    {  // (16-byte accesses: word accesses at a stride of eight would be eight-way bank conflicts)
+      const uint4 c0 = reinterpret_cast<const uint4*>(s_cnt)[tid * 2], c1 = reinterpret_cast<const uint4*>(s_cnt)[tid * 2 + 1];
+      c[0] = c0.x; c[1] = c0.y; c[2] = c0.z; c[3] = c0.w; c[4] = c1.x; c[5] = c1.y; c[6] = c1.z; c[7] = c1.w;
 #pragma unroll
-    for (int q = 0; q < PT; ++q) { c[q] = s_cnt[tid * PT + q]; tot += c[q]; }
+      for (int q = 0; q < PT; ++q) tot += c[q];
+    }
     unsigned incl = tot;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -465,13 +470,15 @@ __device__ __noinline__ void fz_select(const FusedArgs& A, int j, int K, int kef
     unsigned base = 0;
 #pragma unroll 4
     for (int w = 0; w < FZ_THREADS / 32; ++w) base += w < warp ? s_wsum[w] : 0u;
-    unsigned ex = base + incl - tot;
+    unsigned ex = base + incl - tot, pre[PT];
 #pragma unroll
     for (int q = 0; q < PT; ++q) {
-      s_cnt[tid * PT + q] = ex;
+      pre[q] = ex;
       if (c[q] > 0 && (int)ex < keff && (int)(ex + c[q]) >= keff) { s_cutv[0] = tid * PT + q; s_cutv[1] = (int)ex; s_cutv[2] = (int)c[q]; }
       ex += c[q];
     }
+    reinterpret_cast<uint4*>(s_cnt)[tid * 2] = make_uint4(pre[0], pre[1], pre[2], pre[3]);
+    reinterpret_cast<uint4*>(s_cnt)[tid * 2 + 1] = make_uint4(pre[4], pre[5], pre[6], pre[7]);
   }
   named_bar_sync(1, FZ_THREADS);
   if (tid == 0) FZ_STAMP(1, 63);
