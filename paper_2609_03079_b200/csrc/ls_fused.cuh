@@ -131,7 +131,7 @@ __device__ __forceinline__ long long fz_now() { unsigned long long t; asm volati
     asm volatile("{ .reg .f32 t_; mov.f32 t_, %1; mov.u64 %0, %%clock64; }" : "=l"(c_) : "f"(fval)); \
     if (blockIdx.x == 0 && (slot) < 512) g_fz_timing[role][slot] = c_;            \
   } while (0)
-#define FZ_STAMPB(slot) do { if (blockIdx.x == 131 && threadIdx.x == 0) g_fz_timing[0][(slot)] = clock64(); } while (0)
+#define FZ_STAMPB(slot) do { if (blockIdx.x == 1 && threadIdx.x == 0) g_fz_timing[0][(slot)] = clock64(); } while (0)
 #define FZ_CSTAMP(slot) do { if (blockIdx.x < 160) g_fz_cta[blockIdx.x][slot] = fz_now(); } while (0)
 #define FZ_CVAL(slot, v) do { if (blockIdx.x < 160) g_fz_cta[blockIdx.x][slot] = (v); } while (0)
 #else
@@ -382,7 +382,7 @@ __device__ __forceinline__ double fz_unkey(unsigned long long k) {
 // The final evaluation is shared by `nparts` CTAs: each builds the whole histogram (cheap), then ranks only the members
 // of the bins whose first rank falls in its share of the ranks; nothing is exchanged between them.
 template <int WD>
-__device__ __noinline__ void fz_select(const FusedArgs& A, int j, int K, int keff, unsigned wk_off, int part, int nparts) {
+__device__ __noinline__ void fz_select(const FusedArgs& A, int j, int K, int keff, unsigned wk_off, int part, int nparts, bool fold) {
   // (the work area is addressed through the kernel's dynamic shared array, so that the compiler emits shared-memory
   // loads, stores and atomics: through a plain pointer argument they would be generic ones, several times slower)
   extern __shared__ __align__(128) unsigned char fz_dyn_smem[];
@@ -402,9 +402,10 @@ __device__ __noinline__ void fz_select(const FusedArgs& A, int j, int K, int kef
   const bool fin = (j == K);
 #pragma unroll 1
   for (int t = tid; t < 2 * FZ_NB / 4; t += FZ_THREADS) reinterpret_cast<uint4*>(s_cnt)[t] = make_uint4(0u, 0u, 0u, 0u);
-  // (final evaluation) the per-CTA score ranges are fetched now and folded at the end
+  // (the CTA that folds the per-CTA score ranges: an early finisher, not one of the final evaluation's) they are fetched
+  // now and folded at the end
   unsigned long long kmin = 0xffffffffffffffffULL, kmax = 0ULL;
-  if (fin) {
+  if (fold) {
 #pragma unroll 1
     for (int c = tid; c < G; c += FZ_THREADS) { kmin = min(kmin, __ldcg(&A.kmm[2 * c])); kmax = max(kmax, __ldcg(&A.kmm[2 * c + 1])); }
   }
@@ -541,8 +542,8 @@ __device__ __noinline__ void fz_select(const FusedArgs& A, int j, int K, int kef
       named_bar_sync(1, FZ_THREADS);
       if (tid == 0 && cut_b0 + s_cutv[3] != keff) set_status(A.status, ST_INTERNAL);  // self-check of the set's size
     }
-    return;
-  }
+    if (!fold) return;
+  } else {
   // final evaluation: the members of this CTA's share of the bins are scattered into `cand`, grouped by bin (position =
   // first rank of the bin + arrival order); a member's exact rank = first rank of its bin + entries of the bin before it
   const int ncand = cut_bin >= 0 ? cut_b0 + cut_nb : 0;
@@ -638,7 +639,9 @@ __device__ __noinline__ void fz_select(const FusedArgs& A, int j, int K, int kef
   }
   named_bar_sync(1, FZ_THREADS);
   if (tid == 0 && s_cutv[3] != max(0, min(keff, pend) - pstart)) set_status(A.status, ST_INTERNAL);  // self-check: one member per rank
-  if (part != 0) return;
+  if (!fold) return;
+  }
+  named_bar_sync(1, FZ_THREADS);  // (the cut list's bytes are reused below)
   // the layer's binning range for its next launch: what all CTAs observed in this evaluation, widened by 5 % per side
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
@@ -1513,7 +1516,9 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
     // final scores of this CTA's neurons, every evaluation: to global memory with their fine bin (one thread per
     // (evaluation, neuron), no atomics); the exact selection is made per evaluation by ONE CTA after the next barrier
     {
-      unsigned long long kmin = 0xffffffffffffffffULL, kmax = 0ULL;
+      // (the observed range only steers the next launch's binning: the upper halves of the ordered keys, rounded outwards,
+      // are enough, and 32-bit minima and maxima cross a warp in one instruction)
+      unsigned kmin = 0xffffffffu, kmax = 0u;
       const int n_ent = E * n_own;
       double* const nprio = A.next_prio;
       double* const nscores = A.next_scores;
@@ -1538,23 +1543,23 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
           s_own[li] = v;  // kept for the speculation below
           if (nprio) nprio[i] = v;
           if (nscores) nscores[i] = v;
-          const unsigned long long key = ordered_key(v);
-          kmin = min(kmin, key);
-          kmax = max(kmax, key);
+          const unsigned kh = (unsigned)(ordered_key(v) >> 32);
+          kmin = min(kmin, kh);
+          kmax = max(kmax, kh);
         }
       }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        kmin = min(kmin, __shfl_xor_sync(0xffffffffu, kmin, o));
-        kmax = max(kmax, __shfl_xor_sync(0xffffffffu, kmax, o));
-      }
-      if (lane == 0) { s_kmm[warp] = kmin; s_kmm[16 + warp] = kmax; }
+      kmin = __reduce_min_sync(0xffffffffu, kmin);
+      kmax = __reduce_max_sync(0xffffffffu, kmax);
+      unsigned* s_kmm32 = reinterpret_cast<unsigned*>(s_kmm);
+      if (lane == 0) { s_kmm32[warp] = kmin; s_kmm32[16 + warp] = kmax; }
       named_bar_sync(1, FZ_THREADS);
-      if (tid == 0) {  // observed score range of the final evaluation, this CTA's part (no atomics: the selecting CTA folds them)
-#pragma unroll 1
-        for (int w = 1; w < 16; ++w) { kmin = min(kmin, s_kmm[w]); kmax = max(kmax, s_kmm[16 + w]); }
-        A.kmm[2 * cta] = kmin;
-        A.kmm[2 * cta + 1] = kmax;
+      if (warp == 0) {  // observed score range of the final evaluation, this CTA's part (no atomics: a selecting CTA folds them)
+        kmin = __reduce_min_sync(0xffffffffu, lane < 16 ? s_kmm32[lane] : 0xffffffffu);
+        kmax = __reduce_max_sync(0xffffffffu, lane < 16 ? s_kmm32[16 + lane] : 0u);
+        if (lane == 0) {
+          A.kmm[2 * cta] = (unsigned long long)kmin << 32;
+          A.kmm[2 * cta + 1] = ((unsigned long long)kmax << 32) | 0xffffffffULL;
+        }
       }
     }
 
@@ -1616,7 +1621,9 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
     // scans them, finds the CUT bin (the one holding rank keff - 1): bins before it are in, bins after it are out, the
     // cut bin is split by exact comparison of its few entries.  The final evaluation also needs every member's exact
     // rank: members are scattered bin by bin into a scratch array and ranked against the other entries of their bin.
-    if (selects) fz_select<WD>(A, jme, K, keff, lay.sel_off, cta < fparts ? cta : 0, cta < fparts ? fparts : 1);
+    // (what is written once per layer - the score range for the next launch, the counts - is left to the CTA of
+    // evaluation 0, which finishes early; to the final evaluation's first CTA when there is no such CTA)
+    if (selects) fz_select<WD>(A, jme, K, keff, lay.sel_off, cta < fparts ? cta : 0, cta < fparts ? fparts : 1, cta == (fparts < G ? fparts : 0));
     if (tid == 0) FZ_STAMP(1, 6);
     if (tid == 0) FZ_CSTAMP(11);
   }
