@@ -138,3 +138,31 @@ def test_whole_token_kernel_is_bitwise_repeatable():
     stack.close()
     for g in GLs:
         g.close()
+
+
+def test_llama7b_shaped_stack_with_a_wide_selection_matches_the_layer_path():
+    """k = 4096 of 11008 in three stages: a CTA owns ~28 neurons (seven rounds of the first ring, refilled as rounds
+    finish) and keeps ~10 survivors (two batches of the second ring, slots used twice).  The whole-token kernel and the
+    per-layer kernel run the same phases: same sets, same values."""
+    spec = wl.SPECS["llama2-7b"]
+    arrays = [wl.make_layer(spec, l, svd_device="cuda") for l in range(2)]
+    GLs = [ls.ls_layer_create(a, DEV) for a in arrays]
+    stack = ls.ls_stack_create(GLs)
+    k, K, n = 4096, 3, len(GLs)
+    x = torch.from_numpy(wl.make_tokens(spec, 2)[1]).cuda(DEV)
+    sel0, sel_out = ls.Selection(spec.d_ff, k, DEV), ls.Selection(spec.d_ff, k, DEV)
+    ls.ls_predict(GLs[0], x, k, sel0)
+    x_stack = torch.empty_like(x)
+    ls.ls_stack_decode(stack, x, x_stack, sel0, K, k, sel_out)
+    sels = [ls.Selection(spec.d_ff, k, DEV) for _ in range(2)]
+    ls.ls_predict(GLs[0], x, k, sels[0])
+    xl = x.clone()
+    for layer in range(n):
+        ls.ls_sparse_ffn_step(GLs[layer], GLs[min(layer + 1, n - 1)], xl, xl, sels[layer % 2], K, k, sels[(layer + 1) % 2])
+    torch.cuda.synchronize()
+    assert all(ls.ls_layer_status(g) == 0 for g in GLs)
+    assert sel_out.order().tolist() == sels[n % 2].order().tolist()
+    assert_values_close((x_stack - x).cpu().numpy(), (xl - x).cpu().numpy(), what="stack vs layers, wide selection")
+    stack.close()
+    for g in GLs:
+        g.close()
