@@ -336,7 +336,7 @@ bool fused_plan(const ls_layer* L, const ls_layer* next, ls::FusedSmemLayout* ou
   const int g2s[3] = {5, 6, 4};
   for (int alias = 0; alias <= 1; ++alias) {
     for (int c = 0; c < 3; ++c) {
-      for (int g1 = ls::FZ_MAX_G1; g1 >= ls::FZ_NG + 1; --g1) {
+      for (int g1 = ls::FZ_MAX_G1; g1 >= ls::FZ_NG1; --g1) {
         const ls::FusedSmemLayout lay = ls::fused_layout(L->d, L->n_mat, r, Fn, L->sm_count, hn, g1, g2s[c], alias);
         if (lay.per > 512) return false;  // the kernel keeps one slot count per tile of eight neurons, 64 at most
         if (lay.total > budget) continue;
@@ -649,7 +649,7 @@ int32_t ls_stack_create(ls_layer* const* layers, int32_t n_layers, ls_stack** ou
     size_t lo = 0;
     for (int n = 0; n < n_layers; ++n) lo = std::max(lo, (size_t)std::max(h[n].lay.free_lo, h[n].lay.r2_off));
     lo = (lo + 127) & ~(size_t)127;
-    if (lo + (size_t)S->d * 4 <= kFusedSmemBudget && S->d % 8 == 0 && !getenv("LS_DBG_NOSTASH")) {
+    if (lo + (size_t)S->d * 4 <= kFusedSmemBudget && S->d % 8 == 0) {
       S->smem = std::max(S->smem, lo + (size_t)S->d * 4);
       for (int n = 0; n + 1 < n_layers; ++n) { h[n].xs_put = (int)lo; h[n + 1].xs_get = (int)lo; }
     }

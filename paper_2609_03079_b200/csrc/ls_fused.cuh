@@ -38,7 +38,6 @@ namespace ls {
 
 constexpr int FZ_THREADS = 512;        // compute threads (16 warps)
 constexpr int FZ_BLOCK = FZ_THREADS + 32;  // plus the producer warp
-constexpr int FZ_NG = 3;          // survivors processed per batch of the second ring
 constexpr int FZ_NG1 = 4;         // most neurons per round of the first ring
 constexpr int FZ_NB2 = 8;         // most survivors per batch of the second ring
 constexpr int FZ_NB = 4096;       // fine score bins per evaluation
