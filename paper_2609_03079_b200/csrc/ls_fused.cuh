@@ -1576,25 +1576,34 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
     // fill finds it there.  The score estimates the gate pre-activation (B is W_gate A, c the gate bias): a likely member
     // with a positive score will probably survive the ReLU too, so the rest of its bundle is asked for as well.  A wrong
     // guess costs bandwidth that is idle at this point, never correctness.
-    auto speculate = [&](int li, int i_base, int n) {
-      if (li >= n) return;
-      const double v = s_own[li];
+    // Called by whole warps: thread t of nthr; four threads share a neuron's comparisons.
+    auto speculate = [&](int t, int nthr, int i_base, int n) {
       const int m_spec = (int)(((long long)keff * n * 3 / 2 + Fn - 1) / Fn) + 1;  // half again the fair share: a round waits for its slowest row
-      int above = 0;
 #pragma unroll 1
-      for (int l2 = 0; l2 < n; ++l2) {
-        const double o = s_own[l2];
-        above += (o > v) || (o == v && l2 < li);
+      for (int base = 0; base < n; base += nthr >> 2) {
+        const int li = base + (t >> 2), p = t & 3;
+        const bool mine = li < n;
+        const double v = mine ? s_own[li] : 0.0;
+        int above = 0;
+        if (mine) {
+#pragma unroll 4
+          for (int l2 = p; l2 < n; l2 += 4) {
+            const double o = s_own[l2];
+            above += (o > v) || (o == v && l2 < li);
+          }
+        }
+        above += __shfl_xor_sync(0xffffffffu, above, 1);
+        above += __shfl_xor_sync(0xffffffffu, above, 2);
+        if (mine && p == 0 && above < m_spec)
+          asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(A.spec_ptr + (size_t)(i_base + li) * A.spec_stride),
+                       "r"(v > 0.0 ? (unsigned)A.spec_stride : A.spec_bytes) : "memory");
       }
-      if (above < m_spec)
-        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(A.spec_ptr + (size_t)(i_base + li) * A.spec_stride),
-                     "r"(v > 0.0 ? (unsigned)A.spec_stride : A.spec_bytes) : "memory");
     };
     named_bar_sync(1, FZ_THREADS);
     if (tid == 0) {
       grid_barrier_thread0(A, G);
     } else {
-      if (tid >= 32 && A.spec_ptr && !selects) speculate(tid - 32, i_lo, n_own);
+      if (tid >= 32 && A.spec_ptr && !selects) speculate(tid - 32, FZ_THREADS - 32, i_lo, n_own);
       if (A.xs_put >= 0) {  // the next layer's x (complete since the second barrier) waits in shared memory for its start
         float4* xs = reinterpret_cast<float4*>(smem + A.xs_put);
 #pragma unroll 1
@@ -1611,7 +1620,7 @@ __device__ __forceinline__ void fused_layer(const FusedArgs& A, unsigned char* s
 #pragma unroll 1
         for (int li = tid; li < n2; li += FZ_THREADS) s_own[li] = __ldcg(A.sc + (size_t)K * Fn + i2 + li);
         named_bar_sync(1, FZ_THREADS);
-        speculate(tid, i2, n2);
+        speculate(tid, FZ_THREADS, i2, n2);
       }
     }
 
