@@ -26,7 +26,7 @@
 //      -- barrier --
 //   4. select   One CTA per evaluation makes the exact top-k from the stored bins (histogram, scan, cut bin, exact
 //               comparison inside the cut bin); the final evaluation, which also needs every member's exact rank, is
-//               shared by 32 CTAs.  Meanwhile the other CTAs ask the next layer's likely rows into L2.
+//               shared by 64 CTAs.  Meanwhile the other CTAs ask the next layer's likely rows into L2.
 //
 // Instruction fetch matters as much as arithmetic in phases that run once per layer: code that is not resident in the
 // 16 KB per-scheduler instruction cache streams at 5 to 9 clocks per instruction, so loops are kept rolled unless the
@@ -41,7 +41,7 @@ constexpr int FZ_BLOCK = FZ_THREADS + 32;  // plus the producer warp
 constexpr int FZ_NG1 = 4;         // most neurons per round of the first ring
 constexpr int FZ_NB2 = 8;         // most survivors per batch of the second ring
 constexpr int FZ_NB = 4096;       // fine score bins per evaluation
-constexpr int FZ_FIN_PARTS = 32;  // CTAs that share the ranking of the final evaluation
+constexpr int FZ_FIN_PARTS = 64;  // CTAs that share the ranking of the final evaluation
 constexpr int FZ_CUTLIST = 1024;  // entries of the cut bin ranked in shared memory (a fuller bin falls back to global loops)
 constexpr int FZ_CCAP = 4096;     // members grouped in shared memory (more: in the global scratch)
 constexpr int FZ_MAXK = 16;       // stages supported by the fused path
