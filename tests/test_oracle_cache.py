@@ -155,13 +155,44 @@ def test_tiny4_stack_refinement_moves_and_fetch_lists():
     layers = [orc.OracleLayer.from_arrays(a) for a in arrays]
     caches = [orc.LogicalCache(spec.d_ff, 400) for _ in layers]
     x = wl.make_tokens(spec)[0]
-    _, results = orc.decode_token(layers, x, spec.k, 4, caches)
+    K, k, C = 4, spec.k, 400
+    _, results = orc.decode_token(layers, x, k, K, caches)
     moved = 0
-    for n, res in enumerate(results[:-1]):
-        first, last = set(res["refine_orders"][0].tolist()), set(res["refine_orders"][4].tolist())
+    # Independent replay of the residency of every layer's cache (Section 3.3.3: priority-ordered loading, eviction by
+    # priority): the set rule is restated here with plain set operations and a sort, not through LogicalCache.
+    shadow = [set() for _ in layers]
+
+    def replay_reserve(res_set, wanted, rho):
+        universe = res_set | set(wanted)
+        keep = sorted(universe, key=lambda i: (0 if i in wanted else 1, -rho[i], i))[:C]
+        return set(keep)
+
+    order0 = orc.topk_order(orc.predictor_scores(layers[0], x), k)
+    prio_of = [None] * len(layers)
+    prio_of[0] = orc._canonical(orc.predictor_scores(layers[0], x))
+    sel = [None] * len(layers)
+    sel[0] = order0
+    for n, res in enumerate(results):
+        # the step first reserves its own selection (residents first, then misses)
+        shadow[n] = replay_reserve(shadow[n], set(sel[n].tolist()), prio_of[n])
+        if n + 1 == len(layers):
+            break
+        first, last = set(res["refine_orders"][0].tolist()), set(res["refine_orders"][K].tolist())
         moved += len(first ^ last)
-        assert len(res["fetch"]) == 4
-        # each fetch list is the admitted prefix minus what was resident at that moment
-        assert all(len(f) <= orc.fetch_prefix(spec.k, j, 4) for j, f in enumerate(res["fetch"]))
-        assert set(res["refine_orders"][4].tolist()) <= caches[n + 1].resident  # reserved by the next step
+        assert len(res["fetch"]) == K
+        for j in range(K):
+            Cj = res["refine_orders"][j]
+            # stage j admits exactly the first ceil(k (j+1)/(K+1)) ranks of C^(j) ...
+            n_adm = -(-(len(Cj) * (j + 1)) // (K + 1))
+            admitted = Cj[:n_adm].tolist()
+            # ... and fetches those of them that hold no slot at that moment, under the priorities of evaluation j
+            expect = sorted(set(admitted) - shadow[n + 1])
+            assert res["fetch"][j] == expect, (n, j)
+            rho = orc._canonical(res["refine_prio"][j])
+            shadow[n + 1] = replay_reserve(shadow[n + 1], set(admitted), rho)
+        prio_of[n + 1] = orc._canonical(res["refine_prio"][K])
+        sel[n + 1] = res["refine_orders"][K]
+        assert set(res["refine_orders"][K].tolist()) <= caches[n + 1].resident  # reserved by the next step
+    for n in range(len(layers)):
+        assert shadow[n] == caches[n].resident, n
     assert moved > 0  # with a 50x down projection the partial features do change the ranking

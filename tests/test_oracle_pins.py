@@ -26,6 +26,37 @@ def rand_layer(rng, d=16, F=24, r=6, gated=True, bias=-0.3, eps=1e-5):
     )
 
 
+# ------------------------------------------------------------------ stored 16-bit operands of Eq. 1
+def test_decode16_literal_bit_patterns():
+    """Bit patterns written out by hand from the two formats' definitions (sign, exponent bias 127 / 15, 7 / 10
+    fraction bits), not produced by any conversion routine."""
+    bf = np.array([0x3F80, 0xC040, 0x0000, 0x8000, 0x3F00, 0x4049, 0x0001, 0x7F7F], dtype=np.uint16)
+    want_bf = [1.0, -3.0, 0.0, -0.0, 0.5, 3.140625, 2.0 ** -133, (2.0 - 2.0 ** -7) * 2.0 ** 127]
+    got = orc.decode16(bf, "bf16")
+    assert got.dtype == np.float64 and got.tolist() == want_bf
+    assert math.copysign(1.0, got[3]) == -1.0
+    fp = np.array([0x3C00, 0xC200, 0x0000, 0x3800, 0x0001, 0x03FF, 0x7BFF, 0x3555], dtype=np.uint16)
+    want_fp = [1.0, -3.0, 0.0, 0.5, 2.0 ** -24, 1023 * 2.0 ** -24, 65504.0, (1 + 0x155 / 1024) * 0.25]
+    assert orc.decode16(fp, "fp16").tolist() == want_fp
+    with pytest.raises(ValueError):
+        orc.decode16(bf, "fp8")
+
+
+def test_silu_branch_of_the_activation():
+    """Eq. 1 prints SiLU: g * sigmoid(g).  Closed-form values: SiLU(0) = 0, SiLU(ln 3) = 0.75 ln 3,
+    SiLU(-ln 3) = -0.25 ln 3, SiLU(g) - SiLU(-g) = g, and SiLU -> ReLU for large |g|."""
+    L = hand_layer()
+    L.act = orc.SILU
+    ln3 = math.log(3.0)
+    g = np.array([0.0, ln3, -ln3, 40.0, -40.0])
+    a = orc.activation(L, g)
+    np.testing.assert_allclose(a, [0.0, 0.75 * ln3, -0.25 * ln3, 40.0, 0.0], atol=1e-15)
+    gg = np.linspace(-5, 5, 41)
+    np.testing.assert_allclose(orc.activation(L, gg) - orc.activation(L, -gg), gg, atol=1e-14)
+    L.act = orc.RELU
+    assert orc.activation(L, g).tolist() == [0.0, ln3, 0.0, 40.0, 0.0]
+
+
 # ------------------------------------------------------------------ hand-worked layer (Eq. 1)
 def hand_layer():
     return orc.OracleLayer(
