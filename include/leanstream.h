@@ -200,17 +200,33 @@ int32_t ls_layer_status(ls_layer *layer, int32_t *host_status);
  *   qualify.  The stack owns small device buffers (per-layer argument table, residual and selection ping-pong).
  * ls_stack_decode: d_x, d_x_out float [d_model] (may alias); sel_first = selection of layer 0 in rank order (from
  *   ls_predict); n_chunks in [1, 16]; sel_out receives the final refined set of the last layer (idx, count required;
- *   mask, scores optional).  `trace` (nullable) exports, for checking: x [n_layers+1][d_model], the residual entering each
- *   layer and leaving the last (needs d_x != d_x_out); sel_idx [n_layers+1][sel_cap] / sel_count [n_layers+1], the
- *   selection entering each layer and the final refined one.  Never synchronises or allocates; may be captured in a CUDA
- *   graph.  Like every fused step, calls on one device must not overlap (they share one scratch).
+ *   mask, scores optional).  Never synchronises or allocates; may be captured in a CUDA graph.  Calls on one device
+ *   must not overlap (they share one scratch).  The kernel is bitwise repeatable (every sum has a fixed order).
+ *
+ * `trace` (nullable; every member nullable) exports what a layer boundary and every refinement produced, for checking
+ * and profiling:
+ *   x            [n_layers+1][d_model]  the residual entering each layer and leaving the last
+ *   sel_idx      [n_layers+1][sel_cap], sel_count [n_layers+1]: the selection entering each layer (rank order) and
+ *                the final refined one
+ *   xtilde       [n_layers][n_chunks+1][d_model]  the partial residual features x~^(j) of every layer (Eq. 2)
+ *   refine_masks [n_layers][n_chunks+1][mask_words]  the refined sets C^(j) of every layer (Section 2.1), j = 0..K;
+ *                mask_words >= ceil(d_ff/32) of every layer
+ *   phase_ns     [n_layers][SMs][LS_STACK_NSTAMP] nanosecond time stamps (GPU global timer) of every CTA at the ends
+ *                of the kernel's phases: 0 layer start, 1 partial output written, 2 barrier 1 passed, 3 features and
+ *                partial latents written, 4 barrier 2 passed, 5 latents summed, 6 barrier 3 passed, 7 scores written,
+ *                8 barrier 4 passed, 9 own slice of the next selection known, 10 layer end
  */
+#define LS_STACK_NSTAMP 12
 typedef struct ls_stack ls_stack;
 typedef struct {
   float *x;
   int32_t *sel_idx;
   int32_t *sel_count;
   int32_t sel_cap;
+  float *xtilde;
+  uint32_t *refine_masks;
+  int32_t mask_words;
+  long long *phase_ns;
 } ls_stack_trace;
 int32_t ls_stack_create(ls_layer *const *layers, int32_t n_layers, ls_stack **out);
 int32_t ls_stack_destroy(ls_stack *stack);

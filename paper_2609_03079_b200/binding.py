@@ -53,7 +53,11 @@ class ls_step_trace(C.Structure):
 
 
 class ls_stack_trace(C.Structure):
-    _fields_ = [("x", C.c_void_p), ("sel_idx", C.c_void_p), ("sel_count", C.c_void_p), ("sel_cap", C.c_int32)]
+    _fields_ = [("x", C.c_void_p), ("sel_idx", C.c_void_p), ("sel_count", C.c_void_p), ("sel_cap", C.c_int32),
+                ("xtilde", C.c_void_p), ("refine_masks", C.c_void_p), ("mask_words", C.c_int32), ("phase_ns", C.c_void_p)]
+
+
+LS_STACK_NSTAMP = 12
 
 
 class ls_cache_stats_t(C.Structure):
@@ -68,7 +72,7 @@ def lib() -> C.CDLL:
     """The loaded shared library (built in-tree on first use when nvcc is available)."""
     global _lib
     if _lib is None:
-        path = os.environ.get("LEANSTREAM_LIB") or _build.LIB_PATH  # the override names another build of the same library
+        path = _build.LIB_PATH
         if not os.path.exists(path):
             path = _build.build_library()
         try:
@@ -345,16 +349,26 @@ class Stack:
 
 
 class StackTrace:
-    """Device buffers of an ``ls_stack_trace``: residuals and selections at every layer boundary."""
+    """Device buffers of an ``ls_stack_trace``: residuals and selections at every layer boundary and, when ``n_chunks``
+    is given, every partial residual feature and refined set; ``phases=True`` adds the per-CTA phase time stamps."""
 
-    def __init__(self, stack: Stack, sel_cap: int):
+    def __init__(self, stack: Stack, sel_cap: int, n_chunks: int = 0, phases: bool = False):
         L0 = stack.layers[0]
         dev = torch.device("cuda", L0.device)
         n = len(stack.layers)
         self.x = torch.zeros(n + 1, L0.d_model, dtype=torch.float32, device=dev)
         self.sel_idx = torch.full((n + 1, max(sel_cap, 1)), -1, dtype=torch.int32, device=dev)
         self.sel_count = torch.zeros(n + 1, dtype=torch.int32, device=dev)
-        self.c = ls_stack_trace(_ptr(self.x), _ptr(self.sel_idx), _ptr(self.sel_count), sel_cap)
+        self.xtilde = self.refine_masks = self.phase_ns = None
+        self.mask_words = max(L.nwords for L in stack.layers)
+        if n_chunks > 0:
+            self.xtilde = torch.zeros(n, n_chunks + 1, L0.d_model, dtype=torch.float32, device=dev)
+            self.refine_masks = torch.zeros(n, n_chunks + 1, self.mask_words, dtype=torch.int32, device=dev)
+        if phases:
+            sms = torch.cuda.get_device_properties(dev).multi_processor_count
+            self.phase_ns = torch.zeros(n, sms, LS_STACK_NSTAMP, dtype=torch.int64, device=dev)
+        self.c = ls_stack_trace(_ptr(self.x), _ptr(self.sel_idx), _ptr(self.sel_count), sel_cap, _ptr(self.xtilde),
+                                _ptr(self.refine_masks), self.mask_words, _ptr(self.phase_ns))
 
 
 def ls_stack_create(layers) -> Stack:

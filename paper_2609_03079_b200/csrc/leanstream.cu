@@ -13,6 +13,7 @@
 #include "ls_cache.cuh"
 #include "ls_fused.cuh"
 #include "ls_kernels.cuh"
+#include "ls_token.cuh"
 
 namespace {
 
@@ -130,12 +131,13 @@ struct ls_layer {
 
 struct ls_stack {
   int device = 0, n = 0, d = 0, wd = 0, sm_count = 148, max_sel = 0;
+  int r_max = 0, f_max = 0, ns_cta = 0, cpt = 1;
   std::vector<ls_layer*> layers;
-  ls::FusedArgs* d_args = nullptr;  // [n] per-layer arguments (device)
-  float* xbuf = nullptr;            // [2][d] residual ping-pong between layers
-  int32_t* selidx = nullptr;        // [2][max_sel] selection ping-pong
-  int32_t* selcnt = nullptr;        // [2]
-  size_t smem = 0;
+  ls::WtLayer* d_layers = nullptr;       // [n] per-layer arguments (device)
+  float* xbuf = nullptr;                 // [2][d] residual ping-pong between layers
+  double* ranges = nullptr;              // [n][2] score-bin range of every layer's refinement, carried from launch to launch
+  unsigned long long* cuts = nullptr;    // [n][WT_MAXE] key of the last member of every refined set
+  int32_t* sellist = nullptr;            // [max_sel] ranked list of a selection that took the slow route
 };
 
 namespace {
@@ -226,15 +228,15 @@ int32_t device_scratch(int dev, DeviceScratch** out) {
   if (!S.ready) {
     const size_t NE = ls::FZ_MAXE;
     LS_TRY(dalloc(&S.ypart, (size_t)kScratchMaxCtas * kScratchMaxD));
-    LS_TRY(dalloc(&S.ctr, (size_t)8));
-    LS_TRY(dalloc(&S.z, NE * kScratchMaxR + NE));
-    LS_TRY(dalloc(&S.zpart, (size_t)(kScratchMaxD / ls::FZ_SL) * NE * (kScratchMaxR + 1)));
+    LS_TRY(dalloc(&S.ctr, (size_t)64));
+    LS_TRY(dalloc(&S.z, NE * (kScratchMaxR + 4) + NE));
+    LS_TRY(dalloc(&S.zpart, (size_t)(kScratchMaxD / ls::FZ_SL) * NE * (kScratchMaxR + 4)));
     LS_TRY(dalloc(&S.sc, NE * kScratchMaxF));
     LS_TRY(dalloc(&S.sb, NE * kScratchMaxF));
     LS_TRY(dalloc(&S.bent, (size_t)kScratchMaxF));
     LS_TRY(dalloc(&S.kmm, (size_t)2048));
-    LS_CUDA(cudaMemset(S.ctr, 0, 8 * sizeof(unsigned)));
-    LS_CUDA(cudaMemset(S.z, 0, (NE * kScratchMaxR + NE) * sizeof(double)));
+    LS_CUDA(cudaMemset(S.ctr, 0, 64 * sizeof(unsigned)));
+    LS_CUDA(cudaMemset(S.z, 0, (NE * (kScratchMaxR + 4) + NE) * sizeof(double)));
     S.ready = true;
   }
   if (out) *out = &S;
@@ -313,9 +315,8 @@ int32_t create_impl(const ls_layer_desc* D, ls_layer* L) {
   LS_CUDA(cudaFuncSetAttribute(ls::ls_gateup_kernel<WD, BT>, cudaFuncAttributeMaxDynamicSharedMemorySize, big))
   LS_ATTR_GU(0, 1); LS_ATTR_GU(0, 4); LS_ATTR_GU(0, 8); LS_ATTR_GU(1, 1); LS_ATTR_GU(1, 4); LS_ATTR_GU(1, 8);
 #undef LS_ATTR_GU
-#define LS_ATTR_FZ(WD, CPT)                                                                                                    \
-  LS_CUDA(cudaFuncSetAttribute(ls::ls_fused_step_kernel<WD, CPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 218 * 1024)); \
-  LS_CUDA(cudaFuncSetAttribute(ls::ls_fused_stack_kernel<WD, CPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 218 * 1024))
+#define LS_ATTR_FZ(WD, CPT) \
+  LS_CUDA(cudaFuncSetAttribute(ls::ls_fused_step_kernel<WD, CPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 218 * 1024))
   LS_ATTR_FZ(0, 1); LS_ATTR_FZ(0, 2); LS_ATTR_FZ(1, 1); LS_ATTR_FZ(1, 2);
 #undef LS_ATTR_FZ
   LS_CUDA(cudaDeviceSynchronize());
@@ -356,6 +357,37 @@ bool fused_eligible(const ls_layer* L, const ls_layer* next, int batch, int K, i
   if ((sel_cap + L->sm_count - 1) / L->sm_count > ls::FZ_MAX_MINE || L->sm_count > kScratchMaxCtas) return false;
   if ((L->d >> 3) > ls::FZ_THREADS * 2) return false;
   return fused_plan(L, next, nullptr);
+}
+
+// Dynamic shared memory of the whole-token kernel for K stages (see ls_token.cuh): fixed regions, then one region whose
+// users have disjoint lifetimes (the A slices, the latents of all evaluations, the selection's work area, the general
+// top-k's work area).
+constexpr size_t kTokenSmemBudget = 222 * 1024;
+bool token_layout(const ls_stack* S, int K, ls::WtSmem* out) {
+  const int E = K + 1;
+  ls::WtSmem L{};
+  size_t o = 0;
+  auto take = [&](size_t bytes) { const size_t at = o; o += (bytes + 127) & ~(size_t)127; return (unsigned)at; };
+  L.x_off = take((size_t)S->d * 4);
+  L.xt_off = take((size_t)ls::wt_rows(E) * ls::WT_XBLK * 8);
+  L.dm_off = take((size_t)ls::WT_MAXK * 32 * 4);
+  L.mine_off = take((size_t)ls::WT_MAXMINE * (4 + 16 + 4 + 4) + 2 * 32 * 4);
+  L.bits_off = take((size_t)((S->f_max + 31) / 32) * 4);
+  L.u_off = take(0);
+  const size_t a_bytes = (size_t)S->ns_cta * S->r_max * 32 * 2;
+  const size_t z_bytes = (size_t)ls::wt_rows(E) * ls::wt_feat_stride(S->r_max) * 8;
+  size_t q = 0;
+  auto sub = [&](size_t bytes) { const size_t at = q; q += (bytes + 127) & ~(size_t)127; return (unsigned)at; };
+  L.bin_off = sub((size_t)S->f_max * 2);
+  L.hist_off = sub((size_t)ls::WT_NB * 4);
+  L.pref_off = sub((size_t)(ls::WT_NB + 1) * 4);
+  L.ckey_off = sub((size_t)ls::WT_CANDCAP * 8);
+  L.cidx_off = sub((size_t)ls::WT_CANDCAP * 4);
+  const size_t u_bytes = std::max(std::max(a_bytes, z_bytes), std::max(q, ls::topk_smem_bytes(S->f_max)));
+  L.total = (unsigned)(o + ((u_bytes + 127) & ~(size_t)127));
+  if (L.total > kTokenSmemBudget) return false;
+  if (out) *out = L;
+  return true;
 }
 
 template <int WD>
@@ -608,65 +640,64 @@ int32_t ls_stack_create(ls_layer* const* layers, int32_t n_layers, ls_stack** ou
     if (L->device != layers[0]->device || L->d != layers[0]->d || L->wd != layers[0]->wd)
       return fail(LS_ERR_INVALID, "ls_stack_create: layer %d differs in device, d_model or weight type", n);
   }
+  if (layers[0]->d > 8 * ls::WT_THREADS * 2) return fail(LS_ERR_STATE, "ls_stack_create: d_model %d is beyond the whole-token kernel (8192)", layers[0]->d);
+  if (layers[0]->sm_count > kScratchMaxCtas) return fail(LS_ERR_STATE, "ls_stack_create: more SMs than the scratch is sized for");
   DeviceGuard guard(layers[0]->device);
   ls_stack* S = new (std::nothrow) ls_stack();
   if (!S) return fail(LS_ERR_NOMEM, "host allocation");
   S->device = layers[0]->device; S->n = n_layers; S->d = layers[0]->d; S->wd = layers[0]->wd; S->sm_count = layers[0]->sm_count;
+  S->cpt = ((S->d >> 3) + ls::WT_THREADS - 1) / ls::WT_THREADS;
+  S->ns_cta = (((S->d + 31) >> 5) + S->sm_count - 1) / S->sm_count;
   S->layers.assign(layers, layers + n_layers);
-  for (int n = 0; n < n_layers; ++n) S->max_sel = std::max(S->max_sel, layers[n]->max_sel);
+  for (int n = 0; n < n_layers; ++n) {
+    S->max_sel = std::max(S->max_sel, layers[n]->max_sel);
+    S->r_max = std::max(S->r_max, layers[n]->r);
+    S->f_max = std::max(S->f_max, layers[n]->F);
+  }
   auto cleanup = [&](int32_t rc) {
     const std::string keep = g_err;
-    cudaFree(S->d_args); cudaFree(S->xbuf); cudaFree(S->selidx); cudaFree(S->selcnt);
+    cudaFree(S->d_layers); cudaFree(S->xbuf); cudaFree(S->ranges); cudaFree(S->cuts); cudaFree(S->sellist);
     delete S;
     g_err = keep;
     return rc;
   };
   int32_t rc;
-  if ((rc = dalloc(&S->d_args, (size_t)n_layers)) != LS_OK) return cleanup(rc);
+  if ((rc = device_scratch(S->device, nullptr)) != LS_OK) return cleanup(rc);
+  if ((rc = dalloc(&S->d_layers, (size_t)n_layers)) != LS_OK) return cleanup(rc);
   if ((rc = dalloc(&S->xbuf, (size_t)2 * S->d)) != LS_OK) return cleanup(rc);
-  if ((rc = dalloc(&S->selidx, (size_t)2 * S->max_sel)) != LS_OK) return cleanup(rc);
-  if ((rc = dalloc(&S->selcnt, 2)) != LS_OK) return cleanup(rc);
-  std::vector<ls::FusedArgs> h(n_layers);
+  if ((rc = dalloc(&S->ranges, (size_t)2 * n_layers)) != LS_OK) return cleanup(rc);
+  if ((rc = dalloc(&S->cuts, (size_t)n_layers * ls::WT_MAXE)) != LS_OK) return cleanup(rc);
+  if ((rc = dalloc(&S->sellist, (size_t)std::max(1, S->max_sel))) != LS_OK) return cleanup(rc);
+  std::vector<ls::WtLayer> h(n_layers);
+  std::vector<double> hr((size_t)2 * n_layers);
   for (int n = 0; n < n_layers; ++n) {
     ls_layer* L = layers[n];
     ls_layer* next = layers[n + 1 < n_layers ? n + 1 : n];  // the last layer refines a weight-tied copy of itself
-    if (!fused_plan(L, next, nullptr) || (L->d >> 3) > ls::FZ_THREADS * 2)
-      return cleanup(fail(LS_ERR_STATE, "ls_stack_create: layer %d does not fit the fused kernel's shared memory", n));
-    ls_selection sn{};
-    sn.idx = S->selidx + (size_t)((n + 1) & 1) * S->max_sel;
-    sn.count = S->selcnt + ((n + 1) & 1);
-    sn.cap = S->max_sel;
-    ls::FusedSmemLayout lay{};
-    rc = fused_args(L, next, S->xbuf + (size_t)(n & 1) * S->d, S->xbuf + (size_t)((n + 1) & 1) * S->d,
-                    S->selidx + (size_t)(n & 1) * S->max_sel, S->selcnt + (n & 1), S->max_sel, 1, 0, &sn, n & 1, &h[n], &lay);
-    if (rc != LS_OK) return cleanup(rc);
-    S->smem = std::max(S->smem, (size_t)lay.total);
+    ls::WtLayer& a = h[n];
+    a.bundles = L->bundles; a.b_gate = L->b_gate; a.b_down = L->b_down;
+    a.n_mat = L->n_mat; a.F = L->F; a.norm = L->norm; a.eps = L->eps;
+    a.At_sl = next->pred_at_sl; a.Bt = next->pred_bt; a.pc = next->pred_c;
+    a.r = next->r; a.Fn = next->F; a.norm_n = next->norm; a.eps_n = next->eps;
+    a.range = S->ranges + 2 * n;
+    a.status = L->status;
+    hr[2 * n] = 1.0;                          // scores binned over [-1, 1] until a launch has observed their range
+    hr[2 * n + 1] = (double)ls::WT_NB / 2.0;
   }
-  {
-    // x travels from layer to layer through shared memory where some bytes are free from the end of a layer's stream
-    // phase to the first survivors' rows of the next one: above everything the refinement phases use, inside (or
-    // above) the second ring.
-    size_t lo = 0;
-    for (int n = 0; n < n_layers; ++n) lo = std::max(lo, (size_t)std::max(h[n].lay.free_lo, h[n].lay.r2_off));
-    lo = (lo + 127) & ~(size_t)127;
-    if (lo + (size_t)S->d * 4 <= kFusedSmemBudget && S->d % 8 == 0) {
-      S->smem = std::max(S->smem, lo + (size_t)S->d * 4);
-      for (int n = 0; n + 1 < n_layers; ++n) { h[n].xs_put = (int)lo; h[n + 1].xs_get = (int)lo; }
-    }
-  }
-  for (int n = 0; n + 1 < n_layers; ++n) {  // what layer n + 1 reads first: its arguments, gate biases, down bias, predictor offsets
-    const ls_layer* L1 = layers[n + 1];
-    const ls_layer* L2 = layers[n + 2 < n_layers ? n + 2 : n + 1];
-    h[n].pf_ptr[0] = S->d_args + (n + 1); h[n].pf_bytes[0] = (unsigned)sizeof(ls::FusedArgs);
-    h[n].pf_ptr[1] = L1->b_gate;          h[n].pf_bytes[1] = L1->b_gate ? (unsigned)(L1->F * sizeof(float)) : 0u;
-    h[n].pf_ptr[2] = L1->b_down;          h[n].pf_bytes[2] = L1->b_down ? (unsigned)(L1->d * sizeof(float)) : 0u;
-    h[n].pf_ptr[3] = L2->pred_c;          h[n].pf_bytes[3] = L2->pred_c ? (unsigned)(L2->F * sizeof(float)) : 0u;
-    h[n].pg_ptr[0] = L1->bundles; h[n].pg_bytes[0] = (unsigned long long)L1->nslots * L1->n_mat * L1->d * 2ull;
-    h[n].pg_ptr[1] = L2->pred_at_sl; h[n].pg_bytes[1] = (unsigned long long)((L2->d + ls::FZ_SL - 1) / ls::FZ_SL) * L2->r * ls::FZ_SL * 2ull;
-    h[n].pg_ptr[2] = L2->pred_bt; h[n].pg_bytes[2] = (unsigned long long)L2->F * L2->r * 2ull;
-  }
-  if (cudaMemcpy(S->d_args, h.data(), sizeof(ls::FusedArgs) * n_layers, cudaMemcpyHostToDevice) != cudaSuccess)
+  if (cudaMemcpy(S->d_layers, h.data(), sizeof(ls::WtLayer) * n_layers, cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(S->ranges, hr.data(), sizeof(double) * hr.size(), cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemset(S->cuts, 0, sizeof(unsigned long long) * n_layers * ls::WT_MAXE) != cudaSuccess)
     return cleanup(fail(LS_ERR_CUDA, "ls_stack_create: upload of the layer arguments failed"));
+#define LS_ATTR_WT(WD, CPT)                                                                                                       \
+  if (cudaFuncSetAttribute(ls::ls_token_kernel<WD, CPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTokenSmemBudget) != \
+      cudaSuccess)                                                                                                                \
+    return cleanup(fail(LS_ERR_CUDA, "ls_stack_create: shared-memory opt-in failed"))
+  LS_ATTR_WT(0, 1); LS_ATTR_WT(0, 2); LS_ATTR_WT(1, 1); LS_ATTR_WT(1, 2);
+#undef LS_ATTR_WT
+  {
+    ls::WtSmem lay{};
+    if (!token_layout(S, ls::WT_MAXK, &lay) && !token_layout(S, 1, &lay))
+      return cleanup(fail(LS_ERR_STATE, "ls_stack_create: the stack does not fit the whole-token kernel's shared memory"));
+  }
   *out = S;
   return LS_OK;
 }
@@ -675,7 +706,7 @@ int32_t ls_stack_destroy(ls_stack* S) {
   if (!S) return LS_OK;
   DeviceGuard guard(S->device);
   cudaDeviceSynchronize();
-  cudaFree(S->d_args); cudaFree(S->xbuf); cudaFree(S->selidx); cudaFree(S->selcnt);
+  cudaFree(S->d_layers); cudaFree(S->xbuf); cudaFree(S->ranges); cudaFree(S->cuts); cudaFree(S->sellist);
   delete S;
   return LS_OK;
 }
@@ -684,33 +715,50 @@ int32_t ls_stack_decode(ls_stack* S, const float* d_x, float* d_x_out, const ls_
                         ls_selection* sel_out, ls_stack_trace* trace, void* stream) {
   if (!S || !d_x || !d_x_out || !sel_first || !sel_first->idx || !sel_first->count || !sel_out || !sel_out->idx || !sel_out->count)
     return fail(LS_ERR_INVALID, "ls_stack_decode: x, x_out, sel_first and sel_out (idx, count) are required");
-  if (K < 1 || K > ls::FZ_MAXK) return fail(LS_ERR_INVALID, "ls_stack_decode: n_chunks %d outside [1, %d]", K, ls::FZ_MAXK);
+  if (K < 1 || K > ls::WT_MAXK) return fail(LS_ERR_INVALID, "ls_stack_decode: n_chunks %d outside [1, %d]", K, ls::WT_MAXK);
   if (sel_first->cap < 0 || sel_first->cap > S->layers[0]->max_sel) return fail(LS_ERR_INVALID, "ls_stack_decode: sel_first->cap outside [0, max_sel]");
   int fmin_ = 1 << 30;
   for (ls_layer* L : S->layers) fmin_ = std::min(fmin_, std::min(L->F, L->max_sel));
   if (k_next < 0 || k_next > fmin_) return fail(LS_ERR_INVALID, "ls_stack_decode: k_next %d outside [0, %d] (smallest d_ff / max_sel of the stack)", k_next, fmin_);
-  if ((sel_first->cap + S->sm_count - 1) / S->sm_count > ls::FZ_MAX_MINE || (k_next + S->sm_count - 1) / S->sm_count > ls::FZ_MAX_MINE)
-    return fail(LS_ERR_INVALID, "ls_stack_decode: selection too long for the fused kernel");
+  const int G = S->sm_count, gs = std::max(1, G / K);
+  auto per_cta = [&](int count) { const int m = (count + K - 1) / K; return (m + gs - 1) / gs; };
+  if (per_cta(sel_first->cap) > ls::WT_MAXMINE || per_cta(k_next) > ls::WT_MAXMINE)
+    return fail(LS_ERR_INVALID, "ls_stack_decode: selection too long for the whole-token kernel");
   if (sel_out->cap < k_next) return fail(LS_ERR_INVALID, "ls_stack_decode: sel_out->cap %d < k_next %d", sel_out->cap, k_next);
   DeviceGuard guard(S->device);
   cudaStream_t st = (cudaStream_t)stream;
-  ls::StackCall c{};
+  DeviceScratch* D = nullptr;
+  LS_TRY(device_scratch(S->device, &D));
+  ls::WtCall c{};
+  if (!token_layout(S, K, &c.lay)) return fail(LS_ERR_STATE, "ls_stack_decode: %d stages do not fit the whole-token kernel's shared memory", K);
+  c.n_layers = S->n; c.d = S->d; c.K = K; c.k_next = k_next; c.gs = gs;
+  c.piece_len = ((S->d + 3) / 4 + 255) / 256 * 256;
   c.x_in = d_x; c.x_out = d_x_out;
   c.sel_idx = sel_first->idx; c.sel_count = sel_first->count; c.sel_cap = sel_first->cap;
   c.out_idx = sel_out->idx; c.out_count = sel_out->count; c.out_mask = sel_out->mask; c.out_scores = sel_out->scores; c.out_cap = sel_out->cap;
-  c.K = K; c.k_next = k_next;
-  if (trace) { c.tr_x = trace->x; c.tr_sel = trace->sel_idx; c.tr_cnt = trace->sel_count; c.tr_cap = trace->sel_cap; }
-  if (c.tr_sel && !c.tr_cnt) return fail(LS_ERR_INVALID, "ls_stack_decode: trace->sel_count is required with trace->sel_idx");
+  c.xbuf = S->xbuf; c.ypart = D->ypart; c.zpart = D->zpart; c.z = D->z; c.sc = D->sc; c.sb = D->sb; c.kmm = D->kmm;
+  c.cuts = S->cuts; c.sellist = S->sellist;
+  c.tk_key = reinterpret_cast<unsigned long long*>(D->bent);
+  c.tk_idx = reinterpret_cast<int32_t*>(reinterpret_cast<unsigned char*>(D->bent) + (size_t)kScratchMaxF * 8);
+  c.bar = D->ctr + 32;
+  const int nwords_max = (S->f_max + 31) / 32;
+  if (trace) {
+    c.tr_x = trace->x; c.tr_sel = trace->sel_idx; c.tr_cnt = trace->sel_count; c.tr_cap = trace->sel_cap;
+    c.tr_xtilde = trace->xtilde; c.tr_masks = trace->refine_masks; c.tr_words = trace->mask_words; c.tr_ns = trace->phase_ns;
+    if (c.tr_sel && !c.tr_cnt) return fail(LS_ERR_INVALID, "ls_stack_decode: trace->sel_count is required with trace->sel_idx");
+    if (c.tr_masks && c.tr_words < nwords_max)
+      return fail(LS_ERR_INVALID, "ls_stack_decode: trace->mask_words %d < %d", c.tr_words, nwords_max);
+    if (c.tr_masks) LS_CUDA(cudaMemsetAsync(c.tr_masks, 0, (size_t)S->n * (K + 1) * c.tr_words * 4, st));
+  }
   if (sel_out->mask) LS_CUDA(cudaMemsetAsync(sel_out->mask, 0, (size_t)S->layers.back()->nwords * 4, st));
-  const ls::FusedArgs* args = S->d_args;
-  int n = S->n;
-  void* params[] = {&args, &n, &c};
-  const int cpt = ((S->d >> 3) + ls::FZ_THREADS - 1) / ls::FZ_THREADS;
+  LS_CUDA(cudaMemsetAsync(c.bar, 0, sizeof(unsigned), st));
+  const ls::WtLayer* args = S->d_layers;
+  void* params[] = {&args, &c};
   const void* fn = nullptr;
-  if (S->wd == 0) fn = cpt == 1 ? (const void*)ls::ls_fused_stack_kernel<0, 1> : (const void*)ls::ls_fused_stack_kernel<0, 2>;
-  else fn = cpt == 1 ? (const void*)ls::ls_fused_stack_kernel<1, 1> : (const void*)ls::ls_fused_stack_kernel<1, 2>;
+  if (S->wd == 0) fn = S->cpt == 1 ? (const void*)ls::ls_token_kernel<0, 1> : (const void*)ls::ls_token_kernel<0, 2>;
+  else fn = S->cpt == 1 ? (const void*)ls::ls_token_kernel<1, 1> : (const void*)ls::ls_token_kernel<1, 2>;
   KernelTimer timer(LS_TIMED_STACK, st);
-  LS_CUDA(cudaLaunchCooperativeKernel(fn, dim3(S->sm_count), dim3(ls::FZ_BLOCK), params, S->smem, st));
+  LS_CUDA(cudaLaunchCooperativeKernel(fn, dim3(G), dim3(ls::WT_THREADS), params, c.lay.total, st));
   LS_LAUNCHED();
   return LS_OK;
 }

@@ -41,10 +41,12 @@ __device__ inline TopkSmem topk_carve(unsigned char* raw) {
 
 // keyfn(v, s): returns whether element v takes part and, if so, its score in s.
 // emit(rank, v): called by exactly one thread for every element with rank < min(k, participants).
-// Every thread of the 1024-thread block must call this; returns min(k, participants) to all of them.
+// Every thread of the NT-thread block must call this (NT = 1024 or 512); returns min(k, participants) to all of them.
 // g_key / g_idx: global fallback arrays of F entries, used when the candidates do not fit in shared memory.
-template <class KeyFn, class EmitFn>
-__device__ int block_topk(int F, int k, KeyFn keyfn, EmitFn emit, const TopkSmem& sm, unsigned long long* g_key, int32_t* g_idx) {
+template <int NT, class KeyFn, class EmitFn>
+__device__ int block_topk_nt(int F, int k, KeyFn keyfn, EmitFn emit, const TopkSmem& sm, unsigned long long* g_key, int32_t* g_idx) {
+  constexpr int BPT = TK_NB / NT;  // bins per thread in the prefix sum
+  constexpr int TK_THREADS = NT;   // (shadows the namespace constant inside this function)
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   __syncthreads();
   for (int i = tid; i < TK_NB; i += TK_THREADS) { sm.base[i] = 0u; sm.cur[i] = 0u; }
@@ -70,7 +72,8 @@ __device__ int block_topk(int F, int k, KeyFn keyfn, EmitFn emit, const TopkSmem
   if (lane == 0) { sm.redd[warp] = lo; sm.redd[32 + warp] = hi; sm.redi[warp] = npart; }
   __syncthreads();
   if (warp == 0) {
-    lo = sm.redd[lane]; hi = sm.redd[32 + lane]; npart = sm.redi[lane];
+    const bool have = lane < NT / 32;
+    lo = have ? sm.redd[lane] : INF; hi = have ? sm.redd[32 + lane] : -INF; npart = have ? sm.redi[lane] : 0;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
       lo = fmin(lo, __shfl_xor_sync(0xffffffffu, lo, o));
@@ -98,10 +101,10 @@ __device__ int block_topk(int F, int k, KeyFn keyfn, EmitFn emit, const TopkSmem
   }
   __syncthreads();
 
-  // exclusive prefix sum over the bins, 4 bins per thread
-  uint32_t cnt[4], run = 0;
+  // exclusive prefix sum over the bins, BPT consecutive bins per thread
+  uint32_t cnt[BPT], run = 0;
 #pragma unroll
-  for (int e = 0; e < 4; ++e) { cnt[e] = sm.base[tid * 4 + e]; run += cnt[e]; }
+  for (int e = 0; e < BPT; ++e) { cnt[e] = sm.base[tid * BPT + e]; run += cnt[e]; }
   uint32_t incl = run;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -111,7 +114,7 @@ __device__ int block_topk(int F, int k, KeyFn keyfn, EmitFn emit, const TopkSmem
   if (lane == 31) sm.redi[32 + warp] = (int)incl;
   __syncthreads();
   if (warp == 0) {
-    const uint32_t w = (uint32_t)sm.redi[32 + lane];
+    const uint32_t w = lane < NT / 32 ? (uint32_t)sm.redi[32 + lane] : 0u;
     uint32_t wi = w;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -124,8 +127,8 @@ __device__ int block_topk(int F, int k, KeyFn keyfn, EmitFn emit, const TopkSmem
   __syncthreads();
   uint32_t base = (uint32_t)sm.redi[32 + warp] + incl - run;
 #pragma unroll
-  for (int e = 0; e < 4; ++e) {
-    sm.base[tid * 4 + e] = base;
+  for (int e = 0; e < BPT; ++e) {
+    sm.base[tid * BPT + e] = base;
     if (cnt[e] > 0 && (int)base < keff && (int)(base + cnt[e]) >= keff) sm.redi[1] = (int)(base + cnt[e]);
     base += cnt[e];
   }
@@ -162,6 +165,11 @@ __device__ int block_topk(int F, int k, KeyFn keyfn, EmitFn emit, const TopkSmem
   }
   __syncthreads();
   return keff;
+}
+
+template <class KeyFn, class EmitFn>
+__device__ int block_topk(int F, int k, KeyFn keyfn, EmitFn emit, const TopkSmem& sm, unsigned long long* g_key, int32_t* g_idx) {
+  return block_topk_nt<1024>(F, k, keyfn, emit, sm, g_key, g_idx);
 }
 
 // Block-wide exclusive scan of one int per thread (1024 threads); returns the exclusive prefix, total in `total`.

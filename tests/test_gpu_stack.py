@@ -6,21 +6,25 @@ import torch
 from oracle import leanstream_oracle as orc
 from paper_2609_03079_b200 import binding as ls
 from paper_2609_03079_b200 import workload as wl
-from tests.helpers import assert_values_close, check_selection
+from tests.helpers import assert_set_in_tie_band, assert_values_close, check_selection, mask_to_set
 
 pytestmark = pytest.mark.gpu
 DEV = 0
 
 
-def decode_and_check(spec, arrays, K, k, n_tokens, stats):
+def decode_and_check(spec, arrays, K, k, n_tokens, stats, tokens=None):
+    """Every token through ls_stack_decode; every layer boundary AND every refinement it exports is replayed through
+    the oracle: selections bit-exact from the residual bits the GPU produced, values within the output tolerance, every
+    partial residual feature x~^(j) (Eq. 2), and every refined set C^(j), j = 0..K, bit-exact from the GPU's own x~^(j)."""
     OLs = [orc.OracleLayer.from_arrays(a) for a in arrays]
     GLs = [ls.ls_layer_create(a, DEV) for a in arrays]
     stack = ls.ls_stack_create(GLs)
     n = len(GLs)
     sel0 = ls.Selection(spec.d_ff, k, DEV)
     sel_out = ls.Selection(spec.d_ff, k, DEV)
-    trace = ls.StackTrace(stack, k)
-    for x0 in wl.make_tokens(spec)[:n_tokens]:
+    trace = ls.StackTrace(stack, k, n_chunks=K)
+    toks = wl.make_tokens(spec)[:n_tokens] if tokens is None else tokens
+    for x0 in toks:
         x = torch.from_numpy(x0).cuda(DEV)
         x_out = torch.empty_like(x)
         ls.ls_predict(GLs[0], x, k, sel0)
@@ -30,20 +34,35 @@ def decode_and_check(spec, arrays, K, k, n_tokens, stats):
         X = trace.x.cpu().numpy()
         S = trace.sel_idx.cpu().numpy()
         cnt = trace.sel_count.cpu().numpy()
+        XT = trace.xtilde.cpu().numpy()
+        M = trace.refine_masks.cpu().numpy().view(np.uint32)
         np.testing.assert_array_equal(X[0], x0)
         np.testing.assert_array_equal(X[n], x_out.cpu().numpy())
         assert cnt.tolist() == [k] * (n + 1)
         assert S[0, :k].tolist() == sel0.order().tolist() and S[n, :k].tolist() == sel_out.order().tolist()
+        assert mask_to_set(sel_out.mask_np(), spec.d_ff) == set(sel_out.order().tolist())
         for layer in range(n):
             nxt = OLs[min(layer + 1, n - 1)]
             order = S[layer, :k].astype(np.int64)
             # the selection entering the layer is the exact top-k of the residual that entered it
             check_selection(order, orc.predictor_scores(OLs[layer], X[layer]), k, stats)
-            # the layer's output from that residual and that selection
+            # the layer's output and every partial residual feature from that residual and that selection
             res = orc.sparse_ffn_step(OLs[layer], None, X[layer], order, K)
             assert_values_close(X[layer + 1] - X[layer], res["y"][0], what=f"layer {layer}")
-            # and the refined set handed on is the exact top-k of the residual that left it
+            np.testing.assert_array_equal(XT[layer, K], X[layer + 1])  # x_out is x~^(K)
+            np.testing.assert_array_equal(XT[layer, 0], X[layer])      # x~^(0) = x (no down bias in these stacks)
+            for j in range(1, K + 1):
+                assert_values_close(XT[layer, j] - XT[layer, j - 1], res["xtilde"][j][0] - res["xtilde"][j - 1][0],
+                                    scale_ref=res["y"][0], what=f"layer {layer} stage {j}")
+            # every refined set is the exact top-k of the partial feature the GPU produced
+            for j in range(K + 1):
+                want = orc.topk_order(orc.predictor_scores(nxt, XT[layer, j]), k)
+                got = mask_to_set(M[layer, j], spec.d_ff)
+                if got != set(want.tolist()):
+                    assert_set_in_tie_band(got, orc.predictor_scores(nxt, XT[layer, j]), k, stats)
+            # and the refined set handed on is the final one, in rank order
             check_selection(S[layer + 1, :k].astype(np.int64), orc.predictor_scores(nxt, X[layer + 1]), k, stats)
+            assert mask_to_set(M[layer, K], spec.d_ff) == set(S[layer + 1, :k].tolist())
     stack.close()
     for g in GLs:
         g.close()
@@ -58,7 +77,7 @@ def test_tiny4_stack_decode(K):
 
 
 def test_stack_decode_matches_layer_by_layer_path():
-    """Same token through ls_stack_decode and through ls_sparse_ffn_step layer by layer: same sets, same values."""
+    """Same token through ls_stack_decode and through ls_sparse_ffn_step layer by layer: same values."""
     spec = wl.SPECS["tiny4"]
     arrays = wl.make_stack(spec, down_scale=50.0)
     GLs = [ls.ls_layer_create(a, DEV) for a in arrays]
@@ -75,7 +94,10 @@ def test_stack_decode_matches_layer_by_layer_path():
     for layer in range(n):
         ls.ls_sparse_ffn_step(GLs[layer], GLs[min(layer + 1, n - 1)], xl, xl, sels[layer % 2], K, k, sels[(layer + 1) % 2])
     torch.cuda.synchronize()
-    assert sel_out.order().tolist() == sels[n % 2].order().tolist()
+    # the two paths add the partial outputs in different orders, so their features differ in the last fp32 bits and a
+    # near-tie at the cut may fall differently: values agree within the output tolerance, the sets almost entirely
+    # (each path's sets are checked exactly against the oracle elsewhere)
+    assert len(set(sel_out.order().tolist()) & set(sels[n % 2].order().tolist())) >= k - 2
     assert_values_close((x_stack - x).cpu().numpy(), (xl - x).cpu().numpy(), what="stack vs layers")
     # in place, twice in a row (the scratch is clean again after every launch)
     for _ in range(2):
@@ -140,29 +162,11 @@ def test_whole_token_kernel_is_bitwise_repeatable():
         g.close()
 
 
-def test_llama7b_shaped_stack_with_a_wide_selection_matches_the_layer_path():
-    """k = 4096 of 11008 in three stages: a CTA owns ~28 neurons (seven rounds of the first ring, refilled as rounds
-    finish) and keeps ~10 survivors (two batches of the second ring, slots used twice).  The whole-token kernel and the
-    per-layer kernel run the same phases: same sets, same values."""
+def test_llama7b_shaped_stack_with_a_wide_selection():
+    """k = 4096 of 11008 in three stages: a CTA owns ~28 neurons (three rounds of gate rows) and keeps ~10 survivors
+    (two batches of up/down rows); replayed through the oracle like every other stack."""
     spec = wl.SPECS["llama2-7b"]
     arrays = [wl.make_layer(spec, l, svd_device="cuda") for l in range(2)]
-    GLs = [ls.ls_layer_create(a, DEV) for a in arrays]
-    stack = ls.ls_stack_create(GLs)
-    k, K, n = 4096, 3, len(GLs)
-    x = torch.from_numpy(wl.make_tokens(spec, 2)[1]).cuda(DEV)
-    sel0, sel_out = ls.Selection(spec.d_ff, k, DEV), ls.Selection(spec.d_ff, k, DEV)
-    ls.ls_predict(GLs[0], x, k, sel0)
-    x_stack = torch.empty_like(x)
-    ls.ls_stack_decode(stack, x, x_stack, sel0, K, k, sel_out)
-    sels = [ls.Selection(spec.d_ff, k, DEV) for _ in range(2)]
-    ls.ls_predict(GLs[0], x, k, sels[0])
-    xl = x.clone()
-    for layer in range(n):
-        ls.ls_sparse_ffn_step(GLs[layer], GLs[min(layer + 1, n - 1)], xl, xl, sels[layer % 2], K, k, sels[(layer + 1) % 2])
-    torch.cuda.synchronize()
-    assert all(ls.ls_layer_status(g) == 0 for g in GLs)
-    assert sel_out.order().tolist() == sels[n % 2].order().tolist()
-    assert_values_close((x_stack - x).cpu().numpy(), (xl - x).cpu().numpy(), what="stack vs layers, wide selection")
-    stack.close()
-    for g in GLs:
-        g.close()
+    stats = {}
+    decode_and_check(spec, arrays, 3, 4096, 1, stats, tokens=wl.make_tokens(spec, 2)[1:2])
+    assert stats.get("band", 0) == 0
