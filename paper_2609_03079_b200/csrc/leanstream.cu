@@ -102,6 +102,7 @@ struct ls_layer {
   uint16_t* pred_at = nullptr;  // [r][d]
   uint16_t* pred_at_sl = nullptr;  // [ceil(d / 32)][r][32] (the fused kernel's column slices)
   uint16_t* pred_bt = nullptr;  // [F][r]
+  uint16_t* pred_bt_pad = nullptr;  // resident layers: [F + 264][wt_brow_bytes(r) / 2], zero padded (whole-token kernel)
   float* pred_c = nullptr;
 
   // scratch (device)
@@ -161,7 +162,7 @@ int32_t dalloc(T** p, size_t n) {
 void free_layer(ls_layer* L) {
   if (!L) return;
   ls::cache_destroy(L->cache);
-  cudaFree(L->bundles); cudaFree(L->b_gate); cudaFree(L->b_down); cudaFree(L->pred_at); cudaFree(L->pred_at_sl); cudaFree(L->pred_bt);
+  cudaFree(L->bundles); cudaFree(L->b_gate); cudaFree(L->b_down); cudaFree(L->pred_at); cudaFree(L->pred_at_sl); cudaFree(L->pred_bt); cudaFree(L->pred_bt_pad);
   cudaFree(L->pred_c); cudaFree(L->z); cudaFree(L->sumsq); cudaFree(L->scores); cudaFree(L->prio); cudaFree(L->cand_key);
   cudaFree(L->cand_idx); cudaFree(L->umask); cudaFree(L->tmp_idx); cudaFree(L->tmp_count); cudaFree(L->tmp_mask);
   cudaFree(L->fz_range);
@@ -275,6 +276,13 @@ int32_t create_impl(const ls_layer_desc* D, ls_layer* L) {
   LS_TRY(upload_transposed16(&L->pred_at, D->pred_a, (int)d, L->r));
   LS_TRY(upload_sliced16(&L->pred_at_sl, D->pred_a, (int)d, L->r));
   LS_TRY(upload_transposed16(&L->pred_bt, D->pred_b, L->r, (int)F));
+  if (L->cache_rows == 0) {
+    // the same rows at the padded stride the whole-token kernel copies to shared memory, with zero rows behind the last
+    const size_t rs = (size_t)ls::wt_brow_bytes(L->r) / 2, nrows = F + 264;
+    LS_TRY(dalloc(&L->pred_bt_pad, nrows * rs));
+    LS_CUDA(cudaMemset(L->pred_bt_pad, 0, nrows * rs * 2));
+    LS_CUDA(cudaMemcpy2D(L->pred_bt_pad, rs * 2, L->pred_bt, (size_t)L->r * 2, (size_t)L->r * 2, F, cudaMemcpyDeviceToDevice));
+  }
   LS_TRY(upload_f32(&L->pred_c, D->pred_c, F));
 
   const size_t MB = L->max_batch;
@@ -364,26 +372,35 @@ bool fused_eligible(const ls_layer* L, const ls_layer* next, int batch, int K, i
 // top-k's work area).
 constexpr size_t kTokenSmemBudget = 222 * 1024;
 bool token_layout(const ls_stack* S, int K, ls::WtSmem* out) {
-  const int E = K + 1;
+  const int E = K + 1, G = S->sm_count;
   ls::WtSmem L{};
   size_t o = 0;
   auto take = [&](size_t bytes) { const size_t at = o; o += (bytes + 127) & ~(size_t)127; return (unsigned)at; };
   L.x_off = take((size_t)S->d * 4);
-  L.xt_off = take((size_t)ls::wt_rows(E) * ls::WT_XBLK * 8);
+  L.xt_off = take((size_t)(ls::WT_MAXE + 1) * ls::WT_XBLK * 8);
   L.dm_off = take((size_t)ls::WT_MAXK * 32 * 4);
-  L.mine_off = take((size_t)ls::WT_MAXMINE * (4 + 16 + 4 + 4) + 2 * 32 * 4);
+  L.mine_off = take((size_t)ls::WT_MAXMINE * (4 + 16 + 4 + 4) + 32 * 4);
   L.bits_off = take((size_t)((S->f_max + 31) / 32) * 4);
+  L.pc_off = take((size_t)((S->f_max + G - 1) / G) * 4);
+  L.hist_off = take((size_t)ls::WT_NB * 4);
   L.u_off = take(0);
-  const size_t a_bytes = (size_t)S->ns_cta * S->r_max * 32 * 2;
-  const size_t z_bytes = (size_t)ls::wt_rows(E) * ls::wt_feat_stride(S->r_max) * 8;
+  // while a layer runs: A slices | B^T rows | max(partial outputs of a slice, latents) | raw scores
   size_t q = 0;
   auto sub = [&](size_t bytes) { const size_t at = q; q += (bytes + 127) & ~(size_t)127; return (unsigned)at; };
-  L.bin_off = sub((size_t)S->f_max * 2);
-  L.hist_off = sub((size_t)ls::WT_NB * 4);
+  const int per8 = (((S->f_max + G - 1) / G) + 7) / 8 * 8;
+  sub((size_t)S->ns_cta * S->r_max * 32 * 2);
+  L.b_off = sub((size_t)per8 * ls::wt_brow_bytes(S->r_max));
+  L.yz_off = sub(std::max((size_t)ls::WT_WARPS * 32 * 4, (size_t)ls::wt_rows(E) * ls::wt_feat_stride(S->r_max) * 8));
+  L.dot_off = sub((size_t)E * per8 * 8);
+  const size_t run_bytes = q;
+  // during the selection
+  q = 0;
+  L.bin_off = sub((size_t)((S->f_max + 7) / 8 * 8) * 2);
   L.pref_off = sub((size_t)(ls::WT_NB + 1) * 4);
   L.ckey_off = sub((size_t)ls::WT_CANDCAP * 8);
   L.cidx_off = sub((size_t)ls::WT_CANDCAP * 4);
-  const size_t u_bytes = std::max(std::max(a_bytes, z_bytes), std::max(q, ls::topk_smem_bytes(S->f_max)));
+  L.cbin_off = sub((size_t)ls::WT_CANDCAP * 2);
+  const size_t u_bytes = std::max(std::max(run_bytes, q), ls::topk_smem_bytes(S->f_max));
   L.total = (unsigned)(o + ((u_bytes + 127) & ~(size_t)127));
   if (L.total > kTokenSmemBudget) return false;
   if (out) *out = L;
@@ -676,7 +693,7 @@ int32_t ls_stack_create(ls_layer* const* layers, int32_t n_layers, ls_stack** ou
     ls::WtLayer& a = h[n];
     a.bundles = L->bundles; a.b_gate = L->b_gate; a.b_down = L->b_down;
     a.n_mat = L->n_mat; a.F = L->F; a.norm = L->norm; a.eps = L->eps;
-    a.At_sl = next->pred_at_sl; a.Bt = next->pred_bt; a.pc = next->pred_c;
+    a.At_sl = next->pred_at_sl; a.Bt_pad = next->pred_bt_pad; a.pc = next->pred_c;
     a.r = next->r; a.Fn = next->F; a.norm_n = next->norm; a.eps_n = next->eps;
     a.range = S->ranges + 2 * n;
     a.status = L->status;
