@@ -378,31 +378,31 @@ bool token_layout(const ls_stack* S, int K, ls::WtSmem* out) {
   auto take = [&](size_t bytes) { const size_t at = o; o += (bytes + 127) & ~(size_t)127; return (unsigned)at; };
   L.x_off = take((size_t)S->d * 4);
   L.xt_off = take((size_t)(ls::WT_MAXE + 1) * ls::WT_XBLK * 8);
-  L.dm_off = take((size_t)ls::WT_MAXK * 32 * 4);
+  L.dm_off = take((size_t)ls::WT_WARPS * 32 * 4);
   L.mine_off = take((size_t)ls::WT_MAXMINE * (4 + 16 + 4 + 4) + 32 * 4);
   L.bits_off = take((size_t)((S->f_max + 31) / 32) * 4);
   L.pc_off = take((size_t)((S->f_max + G - 1) / G) * 4);
-  L.hist_off = take((size_t)ls::WT_NB * 4);
+  L.hist_off = take((size_t)(ls::WT_NB + 8) * 4);
   L.u_off = take(0);
-  // while a layer runs: A slices | B^T rows | max(partial outputs of a slice, latents) | raw scores
+  // A slices | B^T rows | max(a slice of the partial outputs, latents) | raw scores | work area (ring / selection lists)
   size_t q = 0;
   auto sub = [&](size_t bytes) { const size_t at = q; q += (bytes + 127) & ~(size_t)127; return (unsigned)at; };
   const int per8 = (((S->f_max + G - 1) / G) + 7) / 8 * 8;
+  const int ne = E;  // evaluations scored at once
   sub((size_t)S->ns_cta * S->r_max * 32 * 2);
   L.b_off = sub((size_t)per8 * ls::wt_brow_bytes(S->r_max));
-  L.yz_off = sub(std::max((size_t)ls::WT_WARPS * 32 * 4, (size_t)ls::wt_rows(E) * ls::wt_feat_stride(S->r_max) * 8));
-  L.dot_off = sub((size_t)E * per8 * 8);
-  const size_t run_bytes = q;
-  // during the selection
-  q = 0;
+  L.yz_off = sub(std::max((size_t)G * 32 * 4, (size_t)ls::wt_rows(ne) * ls::wt_feat_stride(S->r_max) * 8));
+  L.dot_off = sub((size_t)ls::wt_rows(ne) * per8 * 8);
+  L.w_off = sub(0);
   L.bin_off = sub((size_t)((S->f_max + 7) / 8 * 8) * 2);
   L.pref_off = sub((size_t)(ls::WT_NB + 1) * 4);
   L.ckey_off = sub((size_t)ls::WT_CANDCAP * 8);
   L.cidx_off = sub((size_t)ls::WT_CANDCAP * 4);
   L.cbin_off = sub((size_t)ls::WT_CANDCAP * 2);
-  const size_t u_bytes = std::max(std::max(run_bytes, q), ls::topk_smem_bytes(S->f_max));
-  L.total = (unsigned)(o + ((u_bytes + 127) & ~(size_t)127));
-  if (L.total > kTokenSmemBudget) return false;
+  const size_t bundle_rest = (size_t)2 * S->d * 2;  // up and down rows of one survivor
+  const size_t u_need = std::max(std::max(q, bundle_rest), ls::topk_smem_bytes(S->f_max));
+  if (o + u_need > kTokenSmemBudget) return false;
+  L.total = (unsigned)kTokenSmemBudget;  // the rest of the budget lets more rows travel at once
   if (out) *out = L;
   return true;
 }
@@ -704,11 +704,11 @@ int32_t ls_stack_create(ls_layer* const* layers, int32_t n_layers, ls_stack** ou
       cudaMemcpy(S->ranges, hr.data(), sizeof(double) * hr.size(), cudaMemcpyHostToDevice) != cudaSuccess ||
       cudaMemset(S->cuts, 0, sizeof(unsigned long long) * n_layers * ls::WT_MAXE) != cudaSuccess)
     return cleanup(fail(LS_ERR_CUDA, "ls_stack_create: upload of the layer arguments failed"));
-#define LS_ATTR_WT(WD, CPT)                                                                                                       \
-  if (cudaFuncSetAttribute(ls::ls_token_kernel<WD, CPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTokenSmemBudget) != \
-      cudaSuccess)                                                                                                                \
+#define LS_ATTR_WT(WD)                                                                                                       \
+  if (cudaFuncSetAttribute(ls::ls_token_kernel<WD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTokenSmemBudget) != \
+      cudaSuccess)                                                                                                           \
     return cleanup(fail(LS_ERR_CUDA, "ls_stack_create: shared-memory opt-in failed"))
-  LS_ATTR_WT(0, 1); LS_ATTR_WT(0, 2); LS_ATTR_WT(1, 1); LS_ATTR_WT(1, 2);
+  LS_ATTR_WT(0); LS_ATTR_WT(1);
 #undef LS_ATTR_WT
   {
     ls::WtSmem lay{};
@@ -750,6 +750,8 @@ int32_t ls_stack_decode(ls_stack* S, const float* d_x, float* d_x_out, const ls_
   if (!token_layout(S, K, &c.lay)) return fail(LS_ERR_STATE, "ls_stack_decode: %d stages do not fit the whole-token kernel's shared memory", K);
   c.n_layers = S->n; c.d = S->d; c.K = K; c.k_next = k_next; c.gs = gs;
   c.piece_len = ((S->d + 3) / 4 + 255) / 256 * 256;
+  c.ring_bytes = (int)(c.lay.total - c.lay.u_off);
+  c.inv_d = 1.0 / (double)S->d;
   c.x_in = d_x; c.x_out = d_x_out;
   c.sel_idx = sel_first->idx; c.sel_count = sel_first->count; c.sel_cap = sel_first->cap;
   c.out_idx = sel_out->idx; c.out_count = sel_out->count; c.out_mask = sel_out->mask; c.out_scores = sel_out->scores; c.out_cap = sel_out->cap;
@@ -772,8 +774,7 @@ int32_t ls_stack_decode(ls_stack* S, const float* d_x, float* d_x_out, const ls_
   const ls::WtLayer* args = S->d_layers;
   void* params[] = {&args, &c};
   const void* fn = nullptr;
-  if (S->wd == 0) fn = S->cpt == 1 ? (const void*)ls::ls_token_kernel<0, 1> : (const void*)ls::ls_token_kernel<0, 2>;
-  else fn = S->cpt == 1 ? (const void*)ls::ls_token_kernel<1, 1> : (const void*)ls::ls_token_kernel<1, 2>;
+  fn = S->wd == 0 ? (const void*)ls::ls_token_kernel<0> : (const void*)ls::ls_token_kernel<1>;
   KernelTimer timer(LS_TIMED_STACK, st);
   LS_CUDA(cudaLaunchCooperativeKernel(fn, dim3(G), dim3(ls::WT_THREADS), params, c.lay.total, st));
   LS_LAUNCHED();

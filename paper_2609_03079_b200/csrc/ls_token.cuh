@@ -27,8 +27,8 @@
 //                memory and finds by itself the neurons whose rank falls in ITS slice of the next layer's ranks: the bins
 //                that cover the slice, their members, exact comparison of the members' keys.  Nothing is exchanged, so
 //                the next layer's stream phase starts without a further barrier.  The refined sets of the evaluations
-//                j < K (Section 2.1: they steer fetching and retention, nothing on a resident stack waits for them) are
-//                established by the same routine (the slice being the set's last rank) on CTAs with little to stream.
+//                j < K are established by the same routine (the slice being the set's last rank) during the next layer's
+//                P1, on CTAs that own no slice of the feature.
 //
 // A selection whose bins are too full for this (ties, a score range that moved) takes a slower, equally exact route
 // through one CTA and an extra barrier; the decision is taken from the same histogram by every CTA alike.
@@ -86,15 +86,17 @@ struct WtLayer {  // one per layer of the stack (device array)
 
 struct WtSmem {  // byte offsets into dynamic shared memory (computed on the host)
   unsigned x_off, xt_off, dm_off, mine_off, bits_off, pc_off, hist_off, u_off;
-  // region u.  While a layer runs: A slices | B^T rows | partial outputs of a slice (P1), then latents and raw scores (P3).
-  unsigned b_off, yz_off, dot_off;
-  // region u during the selection (everything above is dead by then), or the general top-k's work area instead
-  unsigned bin_off, pref_off, ckey_off, cidx_off, cbin_off;
+  // region u: A slices | B^T rows | a slice of the partial outputs (P1) or latents (P3) | raw scores | selection lists.
+  // While the layer streams the whole region is the ring of the rows in flight (the predictor operands are requested
+  // when the stream is over); the general top-k also takes it from its start.
+  unsigned b_off, yz_off, dot_off, w_off;
+  unsigned bin_off, pref_off, ckey_off, cidx_off, cbin_off;  // (from the start of region u)
   unsigned total;
 };
 
 struct WtCall {
-  int n_layers, d, K, k_next, piece_len, gs;  // gs: CTAs per stage
+  double inv_d;  // 1 / d
+  int n_layers, d, K, k_next, piece_len, gs, ring_bytes;  // gs: CTAs per stage; ring_bytes: room for rows in shared memory
   const float* x_in; float* x_out;
   const int32_t* sel_idx; const int32_t* sel_count; int sel_cap;
   int32_t* out_idx; int32_t* out_count; uint32_t* out_mask; double* out_scores; int out_cap;
@@ -125,6 +127,11 @@ struct WtShared {
   float inv_x;            // 1 / rms of the layer's input
   float act8[8];          // activations of a batch of survivors
   unsigned long long kmin, kmax;  // key range of this CTA's final scores
+  double bin_hi, bin_scale;       // the score bins of the refinement in progress (all its evaluations use the same)
+  double pf_thr;                  // final scores from here on: the neuron's gate row is asked into L2 (speculation)
+  const unsigned char* pf_base;   // first gate row of the next layer (nullptr: no speculation)
+  unsigned pf_stride, pf_bytes;
+  int b_valid;                    // the B^T rows in shared memory are intact (the general top-k borrows their place)
   double inv[WT_MAXE + 7];
   double redd[WT_WARPS];
   unsigned long long redk[2 * WT_WARPS];
@@ -225,43 +232,44 @@ __device__ __forceinline__ void wt_share(int count, int K, int gs, int cta, int&
 }
 
 // ---- S: gate rows, survivors, up and down rows -----------------------------------------------------------------------
-// Dot products of up to three rows with x over one piece of the columns: r0..r2 and xs already point at this lane's first
-// eight elements of the piece, `rem` is the length of the piece from there on (may be <= 0); four 16-byte loads per row,
-// all issued before the first is used; the three sums are returned to every lane.
-struct WtF3 { float a, b, c; };
-template <int WD>
-__device__ __noinline__ WtF3 wt_rows_dot(const uint16_t* r0, const uint16_t* r1, const uint16_t* r2, const float* xs, int rem, int nrows) {
-  float acc[3] = {0.f, 0.f, 0.f};
-  const uint16_t* rows[3] = {r0, r1, r2};
+// Rows travel global -> shared memory by cp.async (requested by tiny loops, all in flight at once, no registers held),
+// and every computation is a small rolled loop over shared memory: the phase's code stays a few hundred instructions.
+
+// `nrow` rows of `bytes` bytes each, row i from src_of(i), to consecutive places in the ring (a warp per row).
+template <class SrcFn>
+__device__ __forceinline__ void wt_request_rows(unsigned char* ring, int nrow, int bytes, SrcFn src_of) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll 1
-  for (int base = 0; base < rem; base += 1024) {
-    uint4 w[3][4];
-#pragma unroll
-    for (int q = 0; q < 3; ++q)
-#pragma unroll
-      for (int it = 0; it < 4; ++it)
-        w[q][it] = (q < nrows && base + it * 256 < rem) ? ld_stream128(rows[q] + base + it * 256) : make_uint4(0u, 0u, 0u, 0u);
-#pragma unroll
-    for (int it = 0; it < 4; ++it) {
-      if (base + it * 256 < rem) {
-        const float4 x0 = *reinterpret_cast<const float4*>(xs + base + it * 256);
-        const float4 x1 = *reinterpret_cast<const float4*>(xs + base + it * 256 + 4);
-        const float xv[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
-#pragma unroll
-        for (int q = 0; q < 3; ++q) {
-          float f[8];
-          unpack8<WD>(w[q][it], f);
-#pragma unroll
-          for (int e = 0; e < 8; ++e) acc[q] = fmaf(f[e], xv[e], acc[q]);
-        }
-      }
-    }
+  for (int i = warp; i < nrow; i += WT_WARPS) {
+    const unsigned char* src = src_of(i);
+    if (src == nullptr) continue;
+    unsigned char* dst = ring + (size_t)i * bytes;
+#pragma unroll 1
+    for (int o = lane * 16; o < bytes; o += 512) wt_cp_async16(dst + o, src + o);
   }
-  WtF3 o;
-  o.a = warp_sum(acc[0]);
-  o.b = warp_sum(acc[1]);
-  o.c = warp_sum(acc[2]);
-  return o;
+}
+
+// Dot products of `nrow` rows in the ring (row i at ring + i * stride) with x, a quarter of a row per warp and turn:
+// out[4 i + q] = partial sum of quarter q of row i.
+template <int WD>
+__device__ __forceinline__ void wt_ring_dots(const unsigned char* ring, int stride, int nrow, const float* s_x, int d, int piece_len, float* out) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll 1
+  for (int u = warp; u < 4 * nrow; u += WT_WARPS) {
+    const int c_lo = min(d, (u & 3) * piece_len), c_hi = min(d, c_lo + piece_len);
+    const uint16_t* w = reinterpret_cast<const uint16_t*>(ring + (size_t)(u >> 2) * stride);
+    float acc = 0.f;
+#pragma unroll 1
+    for (int c = c_lo + lane * 8; c < c_hi; c += 256) {
+      float f[8];
+      unpack8<WD>(*reinterpret_cast<const uint4*>(w + c), f);
+      const float4 x0 = *reinterpret_cast<const float4*>(s_x + c), x1 = *reinterpret_cast<const float4*>(s_x + c + 4);
+      acc = fmaf(f[0], x0.x, acc); acc = fmaf(f[1], x0.y, acc); acc = fmaf(f[2], x0.z, acc); acc = fmaf(f[3], x0.w, acc);
+      acc = fmaf(f[4], x1.x, acc); acc = fmaf(f[5], x1.y, acc); acc = fmaf(f[6], x1.z, acc); acc = fmaf(f[7], x1.w, acc);
+    }
+    acc = warp_sum(acc);
+    if (lane == 0) out[u] = acc;
+  }
 }
 
 // This CTA's slices of the next layer's predictor matrix A, its rows of B^T (stored padded, so both are plain linear
@@ -285,27 +293,31 @@ __device__ __forceinline__ void wt_fetch_predictor(const WtCall& C, const WtLaye
   for (int i = tid; i < npieces; i += WT_THREADS) wt_cp_async16(s_b + i * 16, src + (size_t)i * 16);
   float* s_pc = reinterpret_cast<float*>(smem + C.lay.pc_off);
 #pragma unroll 1
-  for (int i = tid; i < n1 - n0; i += WT_THREADS) s_pc[i] = L.pc ? __ldg(L.pc + n0 + i) : 0.f;
+  for (int i = tid; i < n1 - n0; i += WT_THREADS) {
+    if (L.pc) asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(s_pc + i)), "l"(L.pc + n0 + i) : "memory");
+    else s_pc[i] = 0.f;
+  }
 }
 
-template <int WD, int CPT>
+template <int WD>
+__device__ __noinline__ void wt_score_evals(const WtCall& C, WtShared& sh, const WtLayer& L, int e0, int ne, bool last);
+
+template <int WD>
 __device__ __forceinline__ void wt_stream(const WtCall& C, WtShared& sh, const WtLayer& L, unsigned char* smem, bool active) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int d = C.d;
   const float* s_x = reinterpret_cast<const float*>(smem + C.lay.x_off);
   int* s_mine = reinterpret_cast<int*>(smem + C.lay.mine_off);           // [256] neurons of this CTA, rank order
-  float* s_gsum = reinterpret_cast<float*>(s_mine + WT_MAXMINE);         // [256][4] partial gate dot products
+  float* s_gsum = reinterpret_cast<float*>(s_mine + WT_MAXMINE);         // [256][4] partial dot products
   int* s_sidx = reinterpret_cast<int*>(s_gsum + 4 * WT_MAXMINE);         // [256] survivors
-  float* s_sact = reinterpret_cast<float*>(s_sidx + WT_MAXMINE);         // [256] their relu(g)
-  float* s_up = s_sact + WT_MAXMINE;                                     // [8][4] partial up dot products of a batch
+  float* s_sact = reinterpret_cast<float*>(s_sidx + WT_MAXMINE);         // [256] their relu(g), then their activation
+  unsigned char* ring = smem + C.lay.u_off;  // (nothing else in region u is alive while the layer streams)
   const int nmine = sh.nmine;
   const float inv = sh.inv_x;
-  const unsigned bstride = (unsigned)L.n_mat * d;
-  const int p = warp & 3, wq = warp >> 2;
-  const int c_lo = min(d, p * C.piece_len);
-  const int rem = min(d, c_lo + C.piece_len) - c_lo - lane * 8;
-  const float* xs = s_x + c_lo + lane * 8;
-  const uint16_t* wbase = L.bundles + c_lo + lane * 8;
+  const int row_b = d * 2;
+  const size_t bundle_b = (size_t)L.n_mat * row_b;
+  const unsigned char* wbase = reinterpret_cast<const unsigned char*>(L.bundles);
+  const bool gated = L.n_mat == 3;
 
   // gate bias of "my" neuron (used after the dot products; the load is in flight meanwhile)
   int my_idx = -1;
@@ -314,21 +326,20 @@ __device__ __forceinline__ void wt_stream(const WtCall& C, WtShared& sh, const W
     my_idx = s_mine[tid];
     if (my_idx >= 0 && L.b_gate) my_b = __ldg(L.b_gate + my_idx);
   }
+  // gate rows: as many at a time as the ring holds (all of them in the usual case)
+  const int cap_g = C.ring_bytes / row_b;
 #pragma unroll 1
-  for (int i0 = wq; i0 < nmine; i0 += 12) {
-    const int nrows = min(3, (nmine - i0 + 3) >> 2);
-    const uint16_t* r0 = wbase + (size_t)max(s_mine[i0], 0) * bstride;
-    const uint16_t* r1 = nrows > 1 ? wbase + (size_t)max(s_mine[i0 + 4], 0) * bstride : r0;
-    const uint16_t* r2 = nrows > 2 ? wbase + (size_t)max(s_mine[i0 + 8], 0) * bstride : r0;
-    const WtF3 v = wt_rows_dot<WD>(r0, r1, r2, xs, rem, nrows);
-    if (lane == 0) {
-      s_gsum[i0 * 4 + p] = v.a;
-      if (nrows > 1) s_gsum[(i0 + 4) * 4 + p] = v.b;
-      if (nrows > 2) s_gsum[(i0 + 8) * 4 + p] = v.c;
-    }
+  for (int g0 = 0; g0 < nmine; g0 += cap_g) {
+    const int ng = min(cap_g, nmine - g0);
+    wt_request_rows(ring, ng, row_b, [&](int i) -> const unsigned char* {
+      const int v = s_mine[g0 + i];
+      return v >= 0 ? wbase + (size_t)v * bundle_b : nullptr;
+    });
+    wt_cp_async_wait();
+    __syncthreads();
+    wt_ring_dots<WD>(ring, row_b, ng, s_x, d, C.piece_len, s_gsum + 4 * g0);
+    __syncthreads();
   }
-  wt_fetch_predictor(C, L, smem);
-  __syncthreads();
   // activation of the gate branch and the ordered list of survivors (a_i = relu(g_i) u_i: g_i <= 0 needs no other row)
   {
     float g = 0.f;
@@ -352,67 +363,65 @@ __device__ __forceinline__ void wt_stream(const WtCall& C, WtShared& sh, const W
   }
   __syncthreads();
   const int nsurv = sh.nsurv;
-  const bool gated = L.n_mat == 3;
-  constexpr int NB = CPT == 1 ? 8 : 4;  // survivors per batch
-  float acc8[CPT][8];
-#pragma unroll
-  for (int cp = 0; cp < CPT; ++cp)
-#pragma unroll
-    for (int e = 0; e < 8; ++e) acc8[cp][e] = 0.f;
-  const uint16_t* dbase = L.bundles + (size_t)(L.n_mat - 1) * d + tid * 8;
+  // survivors: the rest of their bundles (up and down rows are adjacent: one linear copy), as many as the ring holds
+  const int rest_b = (L.n_mat - 1) * row_b;
+  const int cap_s = C.ring_bytes / rest_b;
+  float acc8[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};  // (d <= 4096: one column group per thread; beyond: see below)
+  float* yp = C.ypart + (size_t)blockIdx.x * d;
+  const bool wide = d > WT_THREADS * 8;
+  if (wide && active) {
 #pragma unroll 1
-  for (int b0 = 0; b0 < nsurv; b0 += NB) {
-    const int nb = min(NB, nsurv - b0);
-    uint4 dw[NB][CPT];
-#pragma unroll
-    for (int s = 0; s < NB; ++s)
-#pragma unroll
-      for (int cp = 0; cp < CPT; ++cp)
-        dw[s][cp] = (s < nb && (tid + cp * WT_THREADS) * 8 < d) ? ld_stream128(dbase + (size_t)s_sidx[b0 + s] * bstride + cp * WT_THREADS * 8)
-                                                                : make_uint4(0u, 0u, 0u, 0u);
+    for (int c = tid * 4; c < d; c += WT_THREADS * 4) __stcg(reinterpret_cast<float4*>(yp + c), make_float4(0.f, 0.f, 0.f, 0.f));
+  }
+#pragma unroll 1
+  for (int b0 = 0; b0 < nsurv; b0 += cap_s) {
+    const int nb = min(cap_s, nsurv - b0);
+    wt_request_rows(ring, nb, rest_b, [&](int i) -> const unsigned char* { return wbase + (size_t)s_sidx[b0 + i] * bundle_b + row_b; });
+    wt_cp_async_wait();
+    __syncthreads();
     if (gated) {
-      // up rows of the batch: warp (p, wq) takes piece p of the survivors wq and wq + 4
-      if (wq < nb) {
-        const int nrows = wq + 4 < nb ? 2 : 1;
-        const uint16_t* r0 = wbase + d + (size_t)s_sidx[b0 + wq] * bstride;
-        const uint16_t* r1 = nrows > 1 ? wbase + d + (size_t)s_sidx[b0 + wq + 4] * bstride : r0;
-        const WtF3 v = wt_rows_dot<WD>(r0, r1, r0, xs, rem, nrows);
-        if (lane == 0) {
-          s_up[wq * 4 + p] = v.a;
-          if (nrows > 1) s_up[(wq + 4) * 4 + p] = v.b;
-        }
-      }
+      wt_ring_dots<WD>(ring, rest_b, nb, s_x, d, C.piece_len, s_gsum);
       __syncthreads();
       if (tid < nb) {
-        const float4 u4 = *reinterpret_cast<const float4*>(s_up + tid * 4);
-        sh.act8[tid] = s_sact[b0 + tid] * (((u4.x + u4.y) + (u4.z + u4.w)) * inv);
+        const float4 u4 = *reinterpret_cast<const float4*>(s_gsum + tid * 4);
+        s_sact[b0 + tid] *= ((u4.x + u4.y) + (u4.z + u4.w)) * inv;
       }
-    } else if (tid < nb) {
-      sh.act8[tid] = s_sact[b0 + tid];
+      __syncthreads();
     }
-    __syncthreads();
+    // down rows scaled into the partial output: every thread owns eight columns
+    const unsigned char* dn = ring + (rest_b - row_b);
+#pragma unroll 1
+    for (int col = tid * 8; col < d; col += WT_THREADS * 8) {
+      float a8[8];
 #pragma unroll
-    for (int s = 0; s < NB; ++s) {
-      const float a = s < nb ? sh.act8[s] : 0.f;
-#pragma unroll
-      for (int cp = 0; cp < CPT; ++cp) {
+      for (int e = 0; e < 8; ++e) a8[e] = wide ? 0.f : acc8[e];
+#pragma unroll 1
+      for (int s0 = 0; s0 < nb; ++s0) {
+        const float a = s_sact[b0 + s0];
         float f[8];
-        unpack8<WD>(dw[s][cp], f);
+        unpack8<WD>(*reinterpret_cast<const uint4*>(dn + (size_t)s0 * rest_b + col * 2), f);
 #pragma unroll
-        for (int e = 0; e < 8; ++e) acc8[cp][e] = fmaf(a, f[e], acc8[cp][e]);
+        for (int e = 0; e < 8; ++e) a8[e] = fmaf(a, f[e], a8[e]);
+      }
+      if (wide) {  // (more than 4096 columns: the partial output is accumulated in its global row, which this CTA alone touches)
+        if (active) {
+          float4* o = reinterpret_cast<float4*>(yp + col);
+          const float4 p0 = __ldcg(o), p1 = __ldcg(o + 1);
+          __stcg(o, make_float4(p0.x + a8[0], p0.y + a8[1], p0.z + a8[2], p0.w + a8[3]));
+          __stcg(o + 1, make_float4(p1.x + a8[4], p1.y + a8[5], p1.z + a8[6], p1.w + a8[7]));
+        }
+      } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc8[e] = a8[e];
       }
     }
     __syncthreads();
   }
-  if (active) {
-    float* yp = C.ypart + (size_t)blockIdx.x * d + tid * 8;
-#pragma unroll
-    for (int cp = 0; cp < CPT; ++cp)
-      if ((tid + cp * WT_THREADS) * 8 < d) {
-        __stcg(reinterpret_cast<float4*>(yp + cp * WT_THREADS * 8), make_float4(acc8[cp][0], acc8[cp][1], acc8[cp][2], acc8[cp][3]));
-        __stcg(reinterpret_cast<float4*>(yp + cp * WT_THREADS * 8 + 4), make_float4(acc8[cp][4], acc8[cp][5], acc8[cp][6], acc8[cp][7]));
-      }
+  if (active && !wide && tid * 8 < d) {
+    __stcg(reinterpret_cast<float4*>(yp + tid * 8), make_float4(acc8[0], acc8[1], acc8[2], acc8[3]));
+    __stcg(reinterpret_cast<float4*>(yp + tid * 8 + 4), make_float4(acc8[4], acc8[5], acc8[6], acc8[7]));
   }
+  wt_fetch_predictor(C, L, smem);
 }
 
 // ---- P1: stage sums, partial residual features, x_out, partial latents of this CTA's slices ----------------------------
@@ -426,34 +435,34 @@ __device__ __forceinline__ void wt_feature(const WtCall& C, WtShared& sh, const 
   const int d = C.d, K = C.K, G = gridDim.x, r = L.r;
   const float* s_x = reinterpret_cast<const float*>(smem + C.lay.x_off);
   double* s_xt = reinterpret_cast<double*>(smem + C.lay.xt_off);  // [rows][WT_XBLK]
-  float* s_dm = reinterpret_cast<float*>(smem + C.lay.dm_off);    // [K][32] stage sums
-  float* s_part = reinterpret_cast<float*>(smem + C.lay.u_off + C.lay.yz_off);  // [16 warps][32] partial stage sums
+  float* s_dm = reinterpret_cast<float*>(smem + C.lay.dm_off);    // [16 warps][32] partial stage sums
+  float* s_y = reinterpret_cast<float*>(smem + C.lay.u_off + C.lay.yz_off);  // [active CTAs][32] this slice of every partial output
   const uint16_t* s_a = reinterpret_cast<const uint16_t*>(smem + C.lay.u_off);
-  const int nsl = (d + 31) >> 5;
+  const int nsl = (d + 31) >> 5, n_act = C.gs * K;
   const int ntile = wt_tiles(E), nplain = wt_plain(E), rows = wt_rows(E);
   const int pos = (lane >> 3) * 10 + (lane & 7);
-  // warps per stage and the rows (CTAs) of a stage one warp adds: all loads of a warp are in flight together
+  // warps per stage and the rows (CTAs) of a stage one warp adds
   const int wps = max(1, WT_WARPS / K), rpw = (C.gs + wps - 1) / wps;
-  wt_cp_async_wait();
 #pragma unroll 1
   for (int s = blockIdx.x, si = 0; s < nsl; s += G, ++si) {
     const int col = 32 * s + lane;
+    // this slice of every CTA's partial output: 128 bytes per CTA, eight lanes each
+    if (lane < 8) {
+      const float* yp = C.ypart + 32 * s + lane * 4;
+#pragma unroll 1
+      for (int row = warp; row < n_act; row += WT_WARPS) wt_cp_async16(s_y + row * 32 + lane * 4, yp + (size_t)row * d);
+    }
+    wt_cp_async_wait();
+    __syncthreads();
     {
       const int c = warp / wps, h = warp - c * wps;
       float a = 0.f;
-      if (c < K && col < d) {
-        const int g0 = h * rpw, g1 = min(C.gs, g0 + rpw);
-        const float* yp = C.ypart + (size_t)(c * C.gs + g0) * d + col;
+      if (c < K) {
+        const int g1 = min(C.gs, (h + 1) * rpw);
 #pragma unroll 1
-        for (int q0 = g0; q0 < g1; q0 += 10, yp += (size_t)10 * d) {
-          float v[10];
-#pragma unroll
-          for (int i = 0; i < 10; ++i) v[i] = q0 + i < g1 ? __ldcg(yp + (size_t)i * d) : 0.f;
-#pragma unroll
-          for (int i = 0; i < 10; ++i) a += v[i];
-        }
+        for (int q = h * rpw; q < g1; ++q) a += s_y[(c * C.gs + q) * 32 + lane];
       }
-      s_part[warp * 32 + lane] = a;
+      s_dm[warp * 32 + lane] = a;
     }
     __syncthreads();
     if (warp == 0) {
@@ -465,7 +474,7 @@ __device__ __forceinline__ void wt_feature(const WtCall& C, WtShared& sh, const 
       for (int c = 0; c < K; ++c) {
         float dm = 0.f;
 #pragma unroll 1
-        for (int h = 0; h < wps; ++h) dm += s_part[(c * wps + h) * 32 + lane];
+        for (int h = 0; h < wps; ++h) dm += s_dm[(c * wps + h) * 32 + lane];
         xt += dm;
         s_xt[(c + 1) * WT_XBLK + pos] = (double)xt;
       }
@@ -530,13 +539,19 @@ __device__ __forceinline__ void wt_latent_sums(const WtCall& C, int r, int E, in
   const int nsl = (C.d + 31) >> 5, ngrp = rz >> 2, units = E * ngrp, G = gridDim.x;
   const int step = E * rz;
 #pragma unroll 1
-  for (int u = blockIdx.x * WT_WARPS + warp; u < units; u += G * WT_WARPS) {
+  for (int u = warp * G + blockIdx.x; u < units; u += G * WT_WARPS) {  // (the units are dealt over all CTAs)
     const int e = u / ngrp, l = 4 * (u - e * ngrp) + v;
     double a = 0.0;
     if (l <= r) {
       const double* zp = C.zpart + e * rz + l + (size_t)sg * step;
-#pragma unroll 4
-      for (int s = sg; s < nsl; s += 8, zp += 8 * step) a += __ldcg(zp);
+#pragma unroll 1
+      for (int s0 = sg; s0 < nsl; s0 += 128, zp += (size_t)128 * step) {  // sixteen partials in flight, added in order
+        double v[16];
+#pragma unroll
+        for (int q = 0; q < 16; ++q) v[q] = s0 + 8 * q < nsl ? __ldcg(zp + (size_t)(8 * q) * step) : 0.0;
+#pragma unroll
+        for (int q = 0; q < 16; ++q) a += v[q];
+      }
     }
     a += __shfl_xor_sync(0xffffffffu, a, 4);
     a += __shfl_xor_sync(0xffffffffu, a, 8);
@@ -550,63 +565,84 @@ __device__ __forceinline__ int wt_bin_of(double s, double hi, double scale) {
   return (int)fmin(fmax((hi - s) * scale, 0.0), (double)(WT_NB - 1));
 }
 
+// Evaluations e0 .. e0 + ne - 1 of the refinement described by L: scores, bins (and, for the final evaluation, the key
+// range this CTA saw).
 template <int WD>
-__device__ __forceinline__ void wt_scores(const WtCall& C, WtShared& sh, const WtLayer& L, unsigned char* smem, int E, int rz, bool last) {
+__device__ __noinline__ void wt_score_evals(const WtCall& C, WtShared& sh, const WtLayer& L, int e0, int ne, bool last) {
+  extern __shared__ __align__(128) unsigned char wt_smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
   const int r = L.r, Fn = L.Fn, G = gridDim.x, K = C.K;
-  double* s_z = reinterpret_cast<double*>(smem + C.lay.u_off + C.lay.yz_off);
-  double* s_dot = reinterpret_cast<double*>(smem + C.lay.u_off + C.lay.dot_off);  // [E][per8] raw dot products
-  const float* s_pc = reinterpret_cast<const float*>(smem + C.lay.pc_off);
-  const unsigned char* s_b = smem + C.lay.u_off + C.lay.b_off;
+  const int rz = (r + 4) & ~3;
+  double* s_z = reinterpret_cast<double*>(wt_smem + C.lay.u_off + C.lay.yz_off);
+  double* s_dot = reinterpret_cast<double*>(wt_smem + C.lay.u_off + C.lay.dot_off);  // [ne][per8] raw dot products
+  const float* s_pc = reinterpret_cast<const float*>(wt_smem + C.lay.pc_off);
+  const unsigned char* s_b = wt_smem + C.lay.u_off + C.lay.b_off;
   const int RS = wt_feat_stride(r), RB = wt_brow_bytes(r);
-  const int ntile = wt_tiles(E), nplain = wt_plain(E), rows = wt_rows(E);
+  const int ntile = wt_tiles(ne), nplain = wt_plain(ne), rows = wt_rows(ne);
   const int nblk = (r + 31) >> 5;
   const int per = (Fn + G - 1) / G, n0 = min(Fn, (int)blockIdx.x * per), n1 = min(Fn, n0 + per);
   const int n_mt = (n1 - n0 + 7) >> 3, per8 = n_mt * 8;
-  // latents to shared memory in the block layout: thread (e, c) pairs, six loads in flight each; 1 / rms of every evaluation
+  if (ne <= 0) return;
   {
-    const int ncol = nblk * 32, total = rows * ncol;
-#pragma unroll 1
-    for (int i0 = tid; i0 < total; i0 += 6 * WT_THREADS) {
-      double v[6];
-      int o[6];
-#pragma unroll
-      for (int q = 0; q < 6; ++q) {
-        const int i = i0 + q * WT_THREADS;
-        const int e = i / ncol, c = i - e * ncol;
-        o[q] = i < total ? e * RS + (c >> 5) * WT_XBLK + ((c >> 3) & 3) * 10 + (c & 7) : -1;
-        v[q] = (i < total && e < E && c < r) ? __ldcg(C.z + e * rz + c) : 0.0;
-      }
-#pragma unroll
-      for (int q = 0; q < 6; ++q)
-        if (o[q] >= 0) s_z[o[q]] = v[q];
+    const int bv = sh.b_valid;
+    __syncthreads();
+    if (!bv) {  // (a general top-k borrowed the place of the B^T rows: fetch them again)
+      wt_fetch_predictor(C, L, wt_smem);
+      wt_cp_async_wait();
+      if (tid == 0) sh.b_valid = 1;
+      __syncthreads();
     }
-    if (tid < E) {
-      const double ss = __ldcg(C.z + tid * rz + r);
-      sh.inv[tid] = L.norm_n == 0 ? wt_rsqrt(ss / (double)C.d + (double)L.eps_n) : 1.0;
-    }
-    if (tid == 0) { sh.kmin = 0xffffffffffffffffULL; sh.kmax = 0ULL; }
   }
+  // latents to shared memory in the block layout, two at a time (pairs stay adjacent in it); 1 / rms of every evaluation
+  if ((r & 31) || rows > ne) {  // (a rank that does not fill its last block, evaluations that do not fill their tile: zeros there)
+#pragma unroll 1
+    for (int i = tid; i < rows * RS; i += WT_THREADS) s_z[i] = 0.0;
+    __syncthreads();
+  }
+#pragma unroll 1
+  for (int e = warp; e < ne; e += WT_WARPS) {  // (plain loads: an asynchronous copy would also wait for the rows in flight)
+    const double* zr = C.z + (e0 + e) * rz;
+    double* zd = s_z + e * RS;
+#pragma unroll 1
+    for (int c0 = 2 * lane; c0 < r; c0 += 256) {
+      double2 v[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) v[q] = c0 + 64 * q < r ? __ldcg(reinterpret_cast<const double2*>(zr + c0 + 64 * q)) : make_double2(0.0, 0.0);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int c = c0 + 64 * q;
+        if (c < r) *reinterpret_cast<double2*>(zd + (c >> 5) * WT_XBLK + ((c >> 3) & 3) * 10 + (c & 7)) = v[q];
+      }
+    }
+  }
+  if (tid < ne) {
+    const double ss = __ldcg(C.z + (e0 + tid) * rz + r);
+    sh.inv[e0 + tid] = L.norm_n == 0 ? wt_rsqrt(ss * C.inv_d + (double)L.eps_n) : 1.0;
+  }
+  if (tid == 0) { sh.kmin = 0xffffffffffffffffULL; sh.kmax = 0ULL; }
   __syncthreads();
-  // raw dot products: a warp per m-tile of eight neurons, all blocks of the rank; two accumulator sets alternate between
-  // the blocks so that consecutive MMAs do not wait for one another
+  // raw dot products: a warp per m-tile of eight neurons, all blocks of the rank
 #pragma unroll 1
   for (int mt = warp; mt < n_mt; mt += WT_WARPS) {
     const unsigned char* wrow = s_b + (8 * mt + g) * RB + 16 * t;
     const double* zb = s_z + t * 10;
-    double c0[2][2] = {{0.0, 0.0}, {0.0, 0.0}}, c1[2][2] = {{0.0, 0.0}, {0.0, 0.0}}, pl[2] = {0.0, 0.0};
-#pragma unroll 2
+    double c0[2] = {0.0, 0.0}, c1[2] = {0.0, 0.0}, pl[2] = {0.0, 0.0};
+#pragma unroll 1
     for (int b = 0; b < nblk; ++b, wrow += 64, zb += WT_XBLK) {
       double a[8], f[8];
       wt_cvt8<WD>(*reinterpret_cast<const uint4*>(wrow), a);
-      if (ntile > 0) { wt_load8d(zb + g * RS, f); wt_mma_block(c0[b & 1], a, f); }
-      if (ntile > 1) { wt_load8d(zb + (8 + g) * RS, f); wt_mma_block(c1[b & 1], a, f); }
-      if (nplain > 0) { wt_load8d(zb + (8 * ntile) * RS, f); pl[0] = wt_dot8(a, f, pl[0]); }
-      if (nplain > 1) { wt_load8d(zb + (8 * ntile + 1) * RS, f); pl[1] = wt_dot8(a, f, pl[1]); }
+      if (ntile > 0) { wt_load8d(zb + g * RS, f); wt_mma_block(c0, a, f); }
+      if (ntile > 1) { wt_load8d(zb + (8 + g) * RS, f); wt_mma_block(c1, a, f); }
+#pragma unroll 1
+      for (int q = 0; q < nplain; ++q) {
+        wt_load8d(zb + (8 * ntile + q) * RS, f);
+        const double v = (a[0] * f[0] + a[1] * f[1]) + (a[2] * f[2] + a[3] * f[3]) + ((a[4] * f[4] + a[5] * f[5]) + (a[6] * f[6] + a[7] * f[7]));
+        if (q == 0) pl[0] += v; else pl[1] += v;
+      }
     }
     double* dp = s_dot + 8 * mt + g;
-    if (ntile > 0) { dp[(2 * t) * per8] = c0[0][0] + c0[1][0]; dp[(2 * t + 1) * per8] = c0[0][1] + c0[1][1]; }
-    if (ntile > 1) { dp[(8 + 2 * t) * per8] = c1[0][0] + c1[1][0]; dp[(8 + 2 * t + 1) * per8] = c1[0][1] + c1[1][1]; }
+    if (ntile > 0) { dp[(2 * t) * per8] = c0[0]; dp[(2 * t + 1) * per8] = c0[1]; }
+    if (ntile > 1) { dp[(8 + 2 * t) * per8] = c1[0]; dp[(8 + 2 * t + 1) * per8] = c1[1]; }
 #pragma unroll
     for (int q = 0; q < 2; ++q)
       if (q < nplain) {
@@ -617,29 +653,41 @@ __device__ __forceinline__ void wt_scores(const WtCall& C, WtShared& sh, const W
       }
   }
   __syncthreads();
-  // scores, bins, key range of the final evaluation: thread (e, i) pairs
-  const double hi = L.range[0], scale = L.range[1];
+  // scores, bins, key range of the final evaluation: (evaluation, neuron) pairs dealt over the threads
+  const double hi = sh.bin_hi, scale = sh.bin_scale;
   const int nown = n1 - n0;
   const int Fs = (Fn + 7) & ~7;
   unsigned long long kmin = 0xffffffffffffffffULL, kmax = 0ULL;
 #pragma unroll 1
-  for (int q = tid; q < E * nown; q += WT_THREADS) {
-    const int e = q / nown, i = q - e * nown, row = n0 + i;
-    const double s = canonical_score(s_dot[e * per8 + i] * sh.inv[e] + (double)s_pc[i]);
-    __stcg(C.sc + (size_t)e * Fn + row, s);
-    C.sb[(size_t)e * Fs + row] = (uint16_t)wt_bin_of(s, hi, scale);
+  for (int q = tid; q < ne * nown; q += WT_THREADS) {
+    const int el = ne == 1 ? 0 : q / nown, i = q - el * nown, row = n0 + i, e = e0 + el;
+    const double sv = canonical_score(s_dot[el * per8 + i] * sh.inv[e] + (double)s_pc[i]);
+    __stcg(C.sc + (size_t)e * Fn + row, sv);
+    C.sb[(size_t)e * Fs + row] = (uint16_t)wt_bin_of(sv, hi, scale);
     if (e == K) {
-      if (last && C.out_scores) C.out_scores[row] = s;
-      if (fabs(s) <= 1.7976931348623157e308) {
-        const unsigned long long key = ordered_key(s);
+      if (last && C.out_scores) C.out_scores[row] = sv;
+      // Speculation (beyond the paper's): the exact selection is two phases away, but a final score at or above the cut
+      // the layer's previous token ended with (less a margin) almost certainly belongs to it, so its gate row is asked
+      // into L2 now and travels while the selection is made.  A wrong guess costs idle bandwidth, never a result.
+      if (sh.pf_base && sv >= sh.pf_thr)
+        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(sh.pf_base + (size_t)row * sh.pf_stride), "r"(sh.pf_bytes) : "memory");
+      if (fabs(sv) <= 1.7976931348623157e308) {
+        const unsigned long long key = ordered_key(sv);
         kmin = min(kmin, key);
         kmax = max(kmax, key);
       }
     }
   }
-  if (kmax >= kmin) { atomicMin(&sh.kmin, kmin); atomicMax(&sh.kmax, kmax); }
+  if (n1 == Fn && nown > 0 && tid < ne * 8) {  // (entries that pad a row of bins to a multiple of eight: a bin of their own)
+    const int e = e0 + (tid >> 3), i = Fn + (tid & 7);
+    if (i < Fs) C.sb[(size_t)e * Fs + i] = (uint16_t)WT_NB;
+  }
+  if (e0 + ne > K) {
+    if (kmax >= kmin) { atomicMin(&sh.kmin, kmin); atomicMax(&sh.kmax, kmax); }
+    __syncthreads();
+    if (tid == 0) { __stcg(C.kmm + 2 * blockIdx.x, sh.kmin); __stcg(C.kmm + 2 * blockIdx.x + 1, sh.kmax); }
+  }
   __syncthreads();
-  if (tid == 0) { __stcg(C.kmm + 2 * blockIdx.x, sh.kmin); __stcg(C.kmm + 2 * blockIdx.x + 1, sh.kmax); }
 }
 
 // ---- P4: selection ---------------------------------------------------------------------------------------------------
@@ -654,7 +702,7 @@ __device__ __noinline__ bool wt_select(const WtCall& C, WtShared& sh, int j, int
   extern __shared__ __align__(128) unsigned char wt_smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   unsigned char* u = wt_smem + C.lay.u_off;
-  uint4* s_bin8 = reinterpret_cast<uint4*>(u + C.lay.bin_off);
+  unsigned* s_bin2 = reinterpret_cast<unsigned*>(u + C.lay.bin_off);  // two bins per word
   unsigned* s_hist = reinterpret_cast<unsigned*>(wt_smem + C.lay.hist_off);
   unsigned* s_pref = reinterpret_cast<unsigned*>(u + C.lay.pref_off);
   unsigned long long* s_ckey = reinterpret_cast<unsigned long long*>(u + C.lay.ckey_off);
@@ -662,33 +710,22 @@ __device__ __noinline__ bool wt_select(const WtCall& C, WtShared& sh, int j, int
   uint16_t* s_cbin = reinterpret_cast<uint16_t*>(u + C.lay.cbin_off);
   unsigned* s_bits = reinterpret_cast<unsigned*>(wt_smem + C.lay.bits_off);
   int* out = reinterpret_cast<int*>(wt_smem + out_off);
-  const int Fs = (Fn + 7) & ~7, n8 = Fs >> 3;
-  const uint4* sb8 = reinterpret_cast<const uint4*>(C.sb + (size_t)j * Fs);
+  const int Fs = (Fn + 7) & ~7, n2 = Fs >> 1;
+  const unsigned char* sb = reinterpret_cast<const unsigned char*>(C.sb + (size_t)j * Fs);
   const double* sc = C.sc + (size_t)j * Fn;
   // the bins are requested first; the histogram is cleared while they are on their way
-  uint4 v[3];
-#pragma unroll
-  for (int q = 0; q < 3; ++q) v[q] = tid + q * WT_THREADS < n8 ? __ldcg(sb8 + tid + q * WT_THREADS) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll 1
+  for (int o = tid * 16; o < Fs * 2; o += WT_THREADS * 16) wt_cp_async16(reinterpret_cast<unsigned char*>(s_bin2) + o, sb + o);
   reinterpret_cast<uint4*>(s_hist)[tid] = make_uint4(0u, 0u, 0u, 0u);
   reinterpret_cast<uint4*>(s_hist)[tid + WT_THREADS] = make_uint4(0u, 0u, 0u, 0u);
   if (tid == 0) { sh.blo = WT_NB; sh.bhi = -1; sh.ncand = 0; sh.slow = 0; sh.found = 0; }
+  wt_cp_async_wait();
   __syncthreads();
 #pragma unroll 1
-  for (int i0 = 0; i0 < n8; i0 += 3 * WT_THREADS) {
-#pragma unroll
-    for (int q = 0; q < 3; ++q) {
-      const int i = i0 + tid + q * WT_THREADS;
-      if (i < n8) {
-        const uint4 w = i0 == 0 ? v[q] : __ldcg(sb8 + i);
-        s_bin8[i] = w;
-        const unsigned ww[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          if (8 * i + 2 * e < Fn) atomicAdd(&s_hist[ww[e] & 0xffffu], 1u);
-          if (8 * i + 2 * e + 1 < Fn) atomicAdd(&s_hist[ww[e] >> 16], 1u);
-        }
-      }
-    }
+  for (int i = tid; i < n2; i += WT_THREADS) {  // (the entries that pad the row fall into a bin of their own)
+    const unsigned w = s_bin2[i];
+    atomicAdd(&s_hist[w & 0xffffu], 1u);
+    atomicAdd(&s_hist[w >> 16], 1u);
   }
   __syncthreads();
   {
@@ -701,16 +738,16 @@ __device__ __noinline__ bool wt_select(const WtCall& C, WtShared& sh, int j, int
     unsigned incl = run;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-      const unsigned t = __shfl_up_sync(0xffffffffu, incl, o);
-      if (lane >= o) incl += t;
+      const unsigned v = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += v;
     }
     if (lane == 31) sh.redu[warp] = incl;
     __syncthreads();
     unsigned wtot = lane < WT_WARPS ? sh.redu[lane] : 0u, wincl = wtot;
 #pragma unroll
     for (int o = 1; o < WT_WARPS; o <<= 1) {
-      const unsigned t = __shfl_up_sync(0xffffffffu, wincl, o);
-      if (lane >= o) wincl += t;
+      const unsigned v = __shfl_up_sync(0xffffffffu, wincl, o);
+      if (lane >= o) wincl += v;
     }
     int base = (int)(__shfl_sync(0xffffffffu, wincl - wtot, warp) + incl - run);
     int blo = WT_NB, bhi = -1, slow = 0;
@@ -732,23 +769,20 @@ __device__ __noinline__ bool wt_select(const WtCall& C, WtShared& sh, int j, int
   }
   __syncthreads();
   if (sh.slow) return false;
-  const int blo = sh.blo, bhi = sh.bhi;
+  const int blo = sh.blo, span = sh.bhi - blo;  // (span < 0: no bin covers the ranks)
   if (hi > lo || want_mask) {
-    // the members of the covering bins (the bins are read back from shared memory, eight at a time)
+    // the members of the covering bins
 #pragma unroll 1
-    for (int i = tid; i < n8; i += WT_THREADS) {
-      const uint4 w = s_bin8[i];
-      const unsigned ww[4] = {w.x, w.y, w.z, w.w};
+    for (int i = tid; i < n2; i += WT_THREADS) {
+      const unsigned w = s_bin2[i];
 #pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        const int b = (int)((e & 1) ? ww[e >> 1] >> 16 : ww[e >> 1] & 0xffffu), idx = 8 * i + e;
-        if (idx < Fn) {
-          if (b >= blo && b <= bhi) {
-            const int pos = atomicAdd(&sh.ncand, 1);
-            if (pos < WT_CANDCAP) { s_cidx[pos] = idx; s_cbin[pos] = (uint16_t)b; }
-          } else if (want_mask && b < blo) {
-            atomicOr(&s_bits[idx >> 5], 1u << (idx & 31));
-          }
+      for (int e = 0; e < 2; ++e) {
+        const int b = (int)(e ? w >> 16 : w & 0xffffu), idx = 2 * i + e;
+        if ((unsigned)(b - blo) <= (unsigned)span && span >= 0) {
+          const int pos = atomicAdd(&sh.ncand, 1);
+          if (pos < WT_CANDCAP) { s_cidx[pos] = idx; s_cbin[pos] = (uint16_t)b; }
+        } else if (want_mask && b < blo) {
+          atomicOr(&s_bits[idx >> 5], 1u << (idx & 31));
         }
       }
     }
@@ -788,12 +822,13 @@ __device__ __noinline__ bool wt_select(const WtCall& C, WtShared& sh, int j, int
 
 // General route: exact top-k of evaluation j by ONE CTA for any input (all scores equal, a range that does not fit),
 // only slower.  Writes the ranked list (when given), the shared bitmap (when asked) and the key of the last member.
-__device__ __noinline__ void wt_select_general(const WtCall& C, unsigned char* smem, int j, int Fn, int keff, int32_t* ranked, bool want_mask,
-                                               unsigned long long* cut_out) {
+__device__ __noinline__ void wt_select_general(const WtCall& C, WtShared& sh, unsigned char* smem, int j, int Fn, int keff, int32_t* ranked,
+                                               bool want_mask, unsigned long long* cut_out) {
   unsigned* s_bits = reinterpret_cast<unsigned*>(smem + C.lay.bits_off);
   const double* sc = C.sc + (size_t)j * Fn;
   __syncthreads();
   if (keff <= 0) return;
+  if (threadIdx.x == 0) sh.b_valid = 0;  // (the work area below covers this CTA's rows of B^T)
   TopkSmem sm = topk_carve(smem + C.lay.u_off);
   block_topk_nt<WT_THREADS>(
       Fn, keff,
@@ -825,7 +860,7 @@ __device__ __noinline__ void wt_refined_set(const WtCall& C, WtShared& sh, unsig
       __syncthreads();
       for (int w = tid; w < nwords; w += WT_THREADS) s_bits[w] = 0u;
     }
-    wt_select_general(C, smem, j, Fn, keff, nullptr, mask_out != nullptr, cut_out);
+    wt_select_general(C, sh, smem, j, Fn, keff, nullptr, mask_out != nullptr, cut_out);
   }
   if (mask_out) {
     __syncthreads();
@@ -880,7 +915,7 @@ __device__ __noinline__ void wt_update_range(const WtCall& C, const WtLayer& L) 
 }
 
 // =====================================================================================================================
-template <int WD, int CPT>
+template <int WD>
 __global__ void __launch_bounds__(WT_THREADS, 1) ls_token_kernel(const WtLayer* __restrict__ g_layers, const __grid_constant__ WtCall C) {
   extern __shared__ __align__(128) unsigned char smem[];
   __shared__ WtShared sh;
@@ -896,7 +931,7 @@ __global__ void __launch_bounds__(WT_THREADS, 1) ls_token_kernel(const WtLayer* 
 
   // ---- prologue: arguments of layer 0, x, 1 / rms, this CTA's slice of the first selection
   if (tid < NW) reinterpret_cast<uint32_t*>(&sh.L[0])[tid] = reinterpret_cast<const uint32_t*>(&g_layers[0])[tid];
-  if (tid == 0) sh.dead = 0;
+  if (tid == 0) { sh.dead = 0; sh.b_valid = 1; }
   {
     double sq = 0.0;
     for (int c = tid * 4; c < d; c += WT_THREADS * 4) {
@@ -931,6 +966,19 @@ __global__ void __launch_bounds__(WT_THREADS, 1) ls_token_kernel(const WtLayer* 
   }
   __syncthreads();
 
+  // The refined sets of layer m's evaluations j < K: one CTA each, CTAs that own no slice of the feature when there are
+  // enough of them (they have nothing else to do in P1).
+  auto refined_sets = [&](int m, const WtLayer& Lm) {
+    const int nsl = (d + 31) >> 5, keff_m = min(C.k_next, Lm.Fn);
+    unsigned long long* cuts = C.cuts + (size_t)m * E;
+#pragma unroll 1
+    for (int j = 0; j < K; ++j) {
+      const int owner = nsl + K <= G ? nsl + j : G - 1 - (j % G);
+      if (cta == owner)
+        wt_refined_set(C, sh, smem, j, Lm.Fn, keff_m, C.tr_masks ? C.tr_masks + ((size_t)m * E + j) * C.tr_words : nullptr, cuts + j);
+    }
+  };
+
 #pragma unroll 1
   for (int n = 0; n < C.n_layers; ++n) {
     const WtLayer& L = sh.L[n & 1];
@@ -938,20 +986,20 @@ __global__ void __launch_bounds__(WT_THREADS, 1) ls_token_kernel(const WtLayer* 
     const int rz = (L.r + 4) & ~3;
     const int keff = min(C.k_next, L.Fn);
     if (stamps) wt_stamp(C, n, 0);
-    // next layer's arguments
-    if (!last && tid >= WT_THREADS - NW)
-      reinterpret_cast<uint32_t*>(&sh.L[(n + 1) & 1])[tid - (WT_THREADS - NW)] =
-          reinterpret_cast<const uint32_t*>(&g_layers[n + 1])[tid - (WT_THREADS - NW)];
     // ---- S
-    wt_stream<WD, CPT>(C, sh, L, smem, active);
+    wt_stream<WD>(C, sh, L, smem, active);
     if (stamps) wt_stamp(C, n, 1);
     wt_grid_sync(C, sh, ++epoch * G);
     if (sh.dead) return;
     if (stamps) wt_stamp(C, n, 2);
-    // ---- P1
+    // ---- P1 (and the refined sets of the layer before, whose scores are complete now)
     float* x_out = last ? C.x_out : C.xbuf + (size_t)((n + 1) & 1) * d;
     wt_feature<WD>(C, sh, L, smem, n, x_out, E, rz);
+    if (n > 0) refined_sets(n - 1, sh.L[(n - 1) & 1]);
     if (stamps) wt_stamp(C, n, 3);
+    // next layer's arguments (the layer before's are not needed any more)
+    __syncthreads();
+    if (!last && tid < NW) reinterpret_cast<uint32_t*>(&sh.L[(n + 1) & 1])[tid] = reinterpret_cast<const uint32_t*>(&g_layers[n + 1])[tid];
     wt_grid_sync(C, sh, ++epoch * G);
     if (sh.dead) return;
     if (stamps) wt_stamp(C, n, 4);
@@ -961,12 +1009,26 @@ __global__ void __launch_bounds__(WT_THREADS, 1) ls_token_kernel(const WtLayer* 
 #pragma unroll 1
       for (int c = tid * 4; c < d; c += WT_THREADS * 4) *reinterpret_cast<float4*>(s_x + c) = __ldcg(reinterpret_cast<const float4*>(x_out + c));
     }
+    if (tid == 32) {
+      const double bh = L.range[0], bs = L.range[1];
+      sh.bin_hi = bh; sh.bin_scale = bs;
+      const unsigned long long ck = C.cuts[(size_t)n * E + K];  // (what the previous launch left: the previous token's cut)
+      const WtLayer& Ln = sh.L[(n + 1) & 1];
+      const bool spec = !last && ck != 0ULL && bs > 0.0 && ((d * 2) & 15) == 0;
+      sh.pf_base = spec ? reinterpret_cast<const unsigned char*>(Ln.bundles) : nullptr;
+      sh.pf_stride = (unsigned)Ln.n_mat * d * 2u;
+      sh.pf_bytes = (unsigned)d * 2u;
+      const unsigned long long cb = (ck >> 63) ? (ck & 0x7fffffffffffffffULL) : ~ck;
+      sh.pf_thr = __longlong_as_double((long long)cb) - 48.0 / bs;  // (a margin of 48 of the 4096 bins)
+    }
     if (stamps) wt_stamp(C, n, 5);
     wt_grid_sync(C, sh, ++epoch * G);
     if (sh.dead) return;
     if (stamps) wt_stamp(C, n, 6);
     // ---- P3
-    wt_scores<WD>(C, sh, L, smem, E, rz, last);
+    wt_cp_async_wait();  // (this CTA's rows of B^T, requested at the end of S)
+    __syncthreads();
+    wt_score_evals<WD>(C, sh, L, 0, E, last);
     if (stamps) wt_stamp(C, n, 7);
     wt_grid_sync(C, sh, ++epoch * G);
     if (sh.dead) return;
@@ -977,7 +1039,7 @@ __global__ void __launch_bounds__(WT_THREADS, 1) ls_token_kernel(const WtLayer* 
     if (tid == 0) sh.inv_x = (float)sh.inv[K];
     unsigned long long* cuts = C.cuts + (size_t)n * E;  // the keys of the last members of this layer's refined sets
     if (!wt_select(C, sh, K, L.Fn, keff, lo, hi, C.lay.mine_off, false, cuts + K)) {
-      if (cta == 0) wt_select_general(C, smem, K, L.Fn, keff, C.sellist, false, cuts + K);
+      if (cta == 0) wt_select_general(C, sh, smem, K, L.Fn, keff, C.sellist, false, cuts + K);
       wt_grid_sync(C, sh, ++epoch * G);
       if (sh.dead) return;
       if (tid < hi - lo) s_mine[tid] = __ldcg(C.sellist + lo + tid);
@@ -987,19 +1049,11 @@ __global__ void __launch_bounds__(WT_THREADS, 1) ls_token_kernel(const WtLayer* 
     if (tid == 0) sh.nmine = hi - lo;
     if (last || C.tr_sel || C.tr_masks) wt_export_selection(C, s_mine, n, lo, hi - lo, keff, last);
     if (cta == 0 && tid < 32) wt_update_range(C, L);
-    // refined sets of the evaluations j < K, on the CTAs with no rows to stream (when there are some)
-    {
-      const int n_idle = G - n_act;
-#pragma unroll 1
-      for (int j = 0; j < K; ++j) {
-        const int owner = n_idle > 0 ? n_act + (j % n_idle) : G - 1 - (j % G);
-        if (cta == owner)
-          wt_refined_set(C, sh, smem, j, L.Fn, keff, C.tr_masks ? C.tr_masks + ((size_t)n * E + j) * C.tr_words : nullptr, cuts + j);
-      }
-    }
     __syncthreads();
     if (stamps) wt_stamp(C, n, 10);
   }
+  // ---- the last layer's refined sets
+  refined_sets(C.n_layers - 1, sh.L[(C.n_layers - 1) & 1]);
 }
 
 }  // namespace ls
