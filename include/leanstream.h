@@ -260,11 +260,12 @@ int32_t ls_topk_select_static(const double *d_scores, int32_t n, int32_t k, int3
 
 /*
  * Process-wide options (no counterpart in the paper).  LS_OPT_FUSED (default 1): steps that qualify (batch 1, layer and
- * next layer fully resident, n_chunks <= 16, shared memory fits) run as ONE cooperative kernel per layer in which
- * streaming and refinement overlap; 0 forces the stage-by-stage kernels, which compute the same thing.  With the fused
- * kernel the partial outputs of different SMs are combined with floating-point atomics, so the low bits of x~^(j) may
- * differ between two runs; the selected sets are always the exact top-k of the features that were actually produced.
- * Fused steps use one working scratch per device: issue them on one stream, or order the streams that issue them.
+ * next layer fully resident, a next layer given, n_chunks <= 16, d_model <= 8192, shared memory fits) run as ONE
+ * cooperative kernel, the same one ls_stack_decode runs over a whole stack; 0 forces the stage-by-stage kernels, which
+ * compute the same thing.  Both paths add partial outputs in a fixed order (no floating-point atomics) and are bitwise
+ * repeatable; the two orders differ, so their features may differ in the last fp32 bits.  The selected sets are always
+ * the exact top-k of the features that were actually produced.  Fused steps and ls_stack_decode share one working
+ * scratch per device: issue them on one stream, or order the streams that issue them.
  */
 #define LS_OPT_FUSED 1
 int32_t ls_set_option(int32_t option, int32_t value);

@@ -11,7 +11,6 @@
 #include <vector>
 
 #include "ls_cache.cuh"
-#include "ls_fused.cuh"
 #include "ls_kernels.cuh"
 #include "ls_token.cuh"
 
@@ -69,6 +68,9 @@ struct KernelTimer {
   }
 };
 
+// Dynamic shared memory the whole-token kernel is launched with (it also has about 1 KB of static shared memory).
+constexpr size_t kTokenSmemBudget = 222 * 1024;
+
 struct DeviceGuard {
   int prev = -1;
   explicit DeviceGuard(int dev) {
@@ -125,7 +127,7 @@ struct ls_layer {
   int down_splits = 0;
 
   // per-layer state of the fused kernel; its working scratch is shared per device (DeviceScratch below)
-  double* fz_range = nullptr;                  // [2] binning range of this layer's scores (observed by its last launch)
+  double* wt_range = nullptr;  // [2] {hi, scale} of the score bins used when a fused step refines THIS layer (carried from call to call)
 
   ls::CacheState cache;  // residency tables, pinned backing store, copy stream
 };
@@ -165,7 +167,7 @@ void free_layer(ls_layer* L) {
   cudaFree(L->bundles); cudaFree(L->b_gate); cudaFree(L->b_down); cudaFree(L->pred_at); cudaFree(L->pred_at_sl); cudaFree(L->pred_bt); cudaFree(L->pred_bt_pad);
   cudaFree(L->pred_c); cudaFree(L->z); cudaFree(L->sumsq); cudaFree(L->scores); cudaFree(L->prio); cudaFree(L->cand_key);
   cudaFree(L->cand_idx); cudaFree(L->umask); cudaFree(L->tmp_idx); cudaFree(L->tmp_count); cudaFree(L->tmp_mask);
-  cudaFree(L->fz_range);
+  cudaFree(L->wt_range);
   cudaFree(L->xin); cudaFree(L->xt); cudaFree(L->actv); cudaFree(L->ypart); cudaFree(L->survive); cudaFree(L->status);
   delete L;
 }
@@ -192,12 +194,12 @@ int32_t upload_transposed16(uint16_t** dst, const void* src, int rows, int cols)
 // [d][r] 16-bit host matrix A -> column slices [ceil(d / 32)][r][32] on the device, zero padded: slice s holds the rows
 // 32 s .. 32 s + 31 of A, transposed, so that one contiguous copy brings a slice into shared memory.
 int32_t upload_sliced16(uint16_t** dst, const void* src, int d, int r) {
-  const int nsl = (d + ls::FZ_SL - 1) / ls::FZ_SL;
+  const int nsl = (d + ls::WT_SL - 1) / ls::WT_SL;
   std::vector<uint16_t> t;
-  try { t.assign((size_t)nsl * r * ls::FZ_SL, 0); } catch (const std::bad_alloc&) { return fail(LS_ERR_NOMEM, "host staging buffer"); }
+  try { t.assign((size_t)nsl * r * ls::WT_SL, 0); } catch (const std::bad_alloc&) { return fail(LS_ERR_NOMEM, "host staging buffer"); }
   const uint16_t* s = static_cast<const uint16_t*>(src);
   for (int c = 0; c < d; ++c)
-    for (int j = 0; j < r; ++j) t[((size_t)(c / ls::FZ_SL) * r + j) * ls::FZ_SL + (c % ls::FZ_SL)] = s[(size_t)c * r + j];
+    for (int j = 0; j < r; ++j) t[((size_t)(c / ls::WT_SL) * r + j) * ls::WT_SL + (c % ls::WT_SL)] = s[(size_t)c * r + j];
   LS_TRY(dalloc(dst, t.size()));
   LS_CUDA(cudaMemcpy(*dst, t.data(), t.size() * 2, cudaMemcpyHostToDevice));
   return LS_OK;
@@ -209,7 +211,8 @@ int32_t upload_sliced16(uint16_t** dst, const void* src, int d, int r) {
 // streams).  Sized for the largest shapes the fused path accepts; allocated at the first layer, kept until exit.
 struct DeviceScratch {
   float* ypart = nullptr;             // [256 CTAs][16384] every CTA's partial output of its stage
-  unsigned* ctr = nullptr;            // fin, (pad), barrier counter (64-bit)
+  unsigned* ctr = nullptr;            // [64] word 32: the grid-barrier counter (zeroed before every launch)
+  unsigned long long* cuts1 = nullptr;  // [WT_MAXE] cut keys of a single fused step
   double* z = nullptr;                // [FZ_MAXE][1024] latents, then [FZ_MAXE] sums of squares
   double* zpart = nullptr;            // [512 slices][FZ_MAXE][1025] per-slice partial latents
   double* sc = nullptr;               // [FZ_MAXE][32768] final scores of every evaluation
@@ -227,15 +230,17 @@ int32_t device_scratch(int dev, DeviceScratch** out) {
   std::lock_guard<std::mutex> lk(g_scratch_mu);
   DeviceScratch& S = g_scratch[dev];
   if (!S.ready) {
-    const size_t NE = ls::FZ_MAXE;
+    const size_t NE = ls::WT_MAXE;
     LS_TRY(dalloc(&S.ypart, (size_t)kScratchMaxCtas * kScratchMaxD));
     LS_TRY(dalloc(&S.ctr, (size_t)64));
     LS_TRY(dalloc(&S.z, NE * (kScratchMaxR + 4) + NE));
-    LS_TRY(dalloc(&S.zpart, (size_t)(kScratchMaxD / ls::FZ_SL) * NE * (kScratchMaxR + 4)));
+    LS_TRY(dalloc(&S.zpart, (size_t)(kScratchMaxD / ls::WT_SL) * NE * (kScratchMaxR + 4)));
     LS_TRY(dalloc(&S.sc, NE * kScratchMaxF));
     LS_TRY(dalloc(&S.sb, NE * kScratchMaxF));
     LS_TRY(dalloc(&S.bent, (size_t)kScratchMaxF));
     LS_TRY(dalloc(&S.kmm, (size_t)2048));
+    LS_TRY(dalloc(&S.cuts1, (size_t)ls::WT_MAXE));
+    LS_CUDA(cudaMemset(S.cuts1, 0, ls::WT_MAXE * sizeof(unsigned long long)));
     LS_CUDA(cudaMemset(S.ctr, 0, 64 * sizeof(unsigned)));
     LS_CUDA(cudaMemset(S.z, 0, (NE * (kScratchMaxR + 4) + NE) * sizeof(double)));
     S.ready = true;
@@ -308,9 +313,9 @@ int32_t create_impl(const ls_layer_desc* D, ls_layer* L) {
 
   if (L->cache_rows == 0) {
     LS_TRY(device_scratch(D->device, nullptr));
-    LS_TRY(dalloc(&L->fz_range, 2));
-    const double zr[2] = {-1.0, 1.0};  // binning range until a launch has observed one
-    LS_CUDA(cudaMemcpy(L->fz_range, zr, sizeof zr, cudaMemcpyHostToDevice));
+    LS_TRY(dalloc(&L->wt_range, 2));
+    const double zr[2] = {1.0, (double)ls::WT_NB / 2.0};  // scores binned over [-1, 1] until a launch has observed their range
+    LS_CUDA(cudaMemcpy(L->wt_range, zr, sizeof zr, cudaMemcpyHostToDevice));
   }
   // opt in to the large dynamic shared memory the kernels may ask for
   const int big = 200 * 1024;
@@ -323,55 +328,17 @@ int32_t create_impl(const ls_layer_desc* D, ls_layer* L) {
   LS_CUDA(cudaFuncSetAttribute(ls::ls_gateup_kernel<WD, BT>, cudaFuncAttributeMaxDynamicSharedMemorySize, big))
   LS_ATTR_GU(0, 1); LS_ATTR_GU(0, 4); LS_ATTR_GU(0, 8); LS_ATTR_GU(1, 1); LS_ATTR_GU(1, 4); LS_ATTR_GU(1, 8);
 #undef LS_ATTR_GU
-#define LS_ATTR_FZ(WD, CPT) \
-  LS_CUDA(cudaFuncSetAttribute(ls::ls_fused_step_kernel<WD, CPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 218 * 1024))
-  LS_ATTR_FZ(0, 1); LS_ATTR_FZ(0, 2); LS_ATTR_FZ(1, 1); LS_ATTR_FZ(1, 2);
-#undef LS_ATTR_FZ
+  LS_CUDA(cudaFuncSetAttribute(ls::ls_token_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTokenSmemBudget));
+  LS_CUDA(cudaFuncSetAttribute(ls::ls_token_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTokenSmemBudget));
   LS_CUDA(cudaDeviceSynchronize());
   return LS_OK;
-}
-
-// Dynamic shared memory the fused kernels may ask for; they also have a few KB of static shared memory.
-constexpr size_t kFusedSmemBudget = 218 * 1024;
-
-// ---- the fused per-layer kernel: eligibility and launch ---------------------------------------------------------------
-// Shared-memory plan of the fused kernel: as many ring stages as fit beside the predictor operands.
-bool fused_plan(const ls_layer* L, const ls_layer* next, ls::FusedSmemLayout* out) {
-  const size_t budget = kFusedSmemBudget;
-  const int r = next ? next->r : 0, Fn = next ? next->F : 0, hn = next ? 1 : 0;
-  // First ring (first row of every bundle): as deep as fits, ideally all of a CTA's neurons at once.  Second ring (the
-  // rest of a survivor's bundle): a few slots; the producer refills them as survivors are consumed.  The A slices keep a
-  // place of their own (they can then arrive while the rings are still busy) unless that costs the first ring its depth.
-  const int g2s[3] = {5, 6, 4};
-  for (int alias = 0; alias <= 1; ++alias) {
-    for (int c = 0; c < 3; ++c) {
-      for (int g1 = ls::FZ_MAX_G1; g1 >= ls::FZ_NG1; --g1) {
-        const ls::FusedSmemLayout lay = ls::fused_layout(L->d, L->n_mat, r, Fn, L->sm_count, hn, g1, g2s[c], alias);
-        if (lay.per > 512) return false;  // the kernel keeps one slot count per tile of eight neurons, 64 at most
-        if (lay.total > budget) continue;
-        if (alias == 0 && g1 < 8) break;  // too shallow with the A slices apart: try the next arrangement
-        if (out) *out = lay;
-        return true;
-      }
-    }
-  }
-  return false;
-}
-
-bool fused_eligible(const ls_layer* L, const ls_layer* next, int batch, int K, int sel_cap) {
-  if (!g_opt_fused.load(std::memory_order_relaxed)) return false;
-  if (batch != 1 || L->cache_rows != 0 || (next && next->cache_rows != 0)) return false;
-  if (K > ls::FZ_MAXK) return false;
-  if ((sel_cap + L->sm_count - 1) / L->sm_count > ls::FZ_MAX_MINE || L->sm_count > kScratchMaxCtas) return false;
-  if ((L->d >> 3) > ls::FZ_THREADS * 2) return false;
-  return fused_plan(L, next, nullptr);
 }
 
 // Dynamic shared memory of the whole-token kernel for K stages (see ls_token.cuh): fixed regions, then one region whose
 // users have disjoint lifetimes (the A slices, the latents of all evaluations, the selection's work area, the general
 // top-k's work area).
-constexpr size_t kTokenSmemBudget = 222 * 1024;
-bool token_layout(const ls_stack* S, int K, ls::WtSmem* out) {
+struct TokenShape { int d, sm_count, r_max, f_max, ns_cta; };
+bool token_layout(const TokenShape* S, int K, ls::WtSmem* out) {
   const int E = K + 1, G = S->sm_count;
   ls::WtSmem L{};
   size_t o = 0;
@@ -407,78 +374,82 @@ bool token_layout(const ls_stack* S, int K, ls::WtSmem* out) {
   return true;
 }
 
-template <int WD>
-int32_t launch_fused_cpt(int cpt, const ls::FusedArgs& a, int grid, size_t smem, cudaStream_t st) {
-  void* params[] = {const_cast<ls::FusedArgs*>(&a)};
-  const void* fn = nullptr;
-  switch (cpt) {
-    case 1: fn = (const void*)ls::ls_fused_step_kernel<WD, 1>; break;
-    default: fn = (const void*)ls::ls_fused_step_kernel<WD, 2>; break;
-  }
-  KernelTimer timer(LS_TIMED_FUSED, st);
-  LS_CUDA(cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(ls::FZ_BLOCK), params, smem, st));
+// Launch of the whole-token kernel (a table of layers, or the single layer in c.one): the part common to ls_stack_decode
+// and to a fused ls_sparse_ffn_step.  The caller has filled the trace pointers, cuts, sellist, xbuf (and c.one).
+int32_t launch_token(const TokenShape* shp, int device, int wd, const ls::WtLayer* d_layers, int n_layers, ls::WtCall& c, const float* d_x,
+                     float* d_x_out, const ls_selection* sel_first, int K, int k_next, ls_selection* sel_out, int out_words, cudaStream_t st,
+                     const char* who) {
+  const int G = shp->sm_count, gs = std::max(1, G / K);
+  auto per_cta = [&](int count) { const int m = (count + K - 1) / K; return (m + gs - 1) / gs; };
+  if (per_cta(sel_first->cap) > ls::WT_MAXMINE || per_cta(k_next) > ls::WT_MAXMINE)
+    return fail(LS_ERR_INVALID, "%s: selection too long for the whole-token kernel", who);
+  DeviceScratch* D = nullptr;
+  LS_TRY(device_scratch(device, &D));
+  if (!token_layout(shp, K, &c.lay)) return fail(LS_ERR_STATE, "%s: %d stages do not fit the whole-token kernel's shared memory", who, K);
+  c.n_layers = n_layers; c.d = shp->d; c.K = K; c.k_next = k_next; c.gs = gs;
+  c.piece_len = ((shp->d + 3) / 4 + 255) / 256 * 256;
+  c.ring_bytes = (int)(c.lay.total - c.lay.u_off);
+  c.inv_d = 1.0 / (double)shp->d;
+  c.x_in = d_x; c.x_out = d_x_out;
+  c.sel_idx = sel_first->idx; c.sel_count = sel_first->count; c.sel_cap = sel_first->cap;
+  c.out_idx = sel_out->idx; c.out_count = sel_out->count; c.out_mask = sel_out->mask; c.out_scores = sel_out->scores; c.out_cap = sel_out->cap;
+  c.ypart = D->ypart; c.zpart = D->zpart; c.z = D->z; c.sc = D->sc; c.sb = D->sb; c.kmm = D->kmm;
+  c.tk_key = reinterpret_cast<unsigned long long*>(D->bent);
+  c.tk_idx = reinterpret_cast<int32_t*>(reinterpret_cast<unsigned char*>(D->bent) + (size_t)kScratchMaxF * 8);
+  c.bar = D->ctr + 32;
+  if (c.tr_masks) LS_CUDA(cudaMemsetAsync(c.tr_masks, 0, (size_t)n_layers * (K + 1) * c.tr_words * 4, st));
+  if (sel_out->mask) LS_CUDA(cudaMemsetAsync(sel_out->mask, 0, (size_t)out_words * 4, st));
+  LS_CUDA(cudaMemsetAsync(c.bar, 0, sizeof(unsigned), st));
+  void* params[] = {&d_layers, &c};
+  const void* fn = wd == 0 ? (const void*)ls::ls_token_kernel<0> : (const void*)ls::ls_token_kernel<1>;
+  LS_CUDA(cudaLaunchCooperativeKernel(fn, dim3(G), dim3(ls::WT_THREADS), params, c.lay.total, st));
   LS_LAUNCHED();
   return LS_OK;
 }
 
-// Arguments of one fused layer step; `parity` picks the half of the alternating scratch.
-int32_t fused_args(ls_layer* L, ls_layer* next, const float* d_x, float* d_x_out, const int32_t* sel_idx, const int32_t* sel_count,
-                   int sel_cap, int K, int k_next, ls_selection* sel_next, int parity, ls::FusedArgs* out, ls::FusedSmemLayout* lay_out) {
-  ls::FusedArgs a{};
-  a.bundles = L->bundles; a.n_mat = L->n_mat; a.gated = L->gated; a.b_gate = L->b_gate; a.b_down = L->b_down;
-  a.d = L->d; a.F = L->F; a.norm = L->norm; a.eps = L->eps; a.inv_d = 1.0 / (double)L->d;
-  a.x = d_x; a.x_out = d_x_out;
-  a.sel_idx = sel_idx; a.sel_count = sel_count; a.sel_cap = sel_cap; a.K = K;
-  DeviceScratch* S = nullptr;
-  LS_TRY(device_scratch(L->device, &S));
-  a.ypart = S->ypart;
-  (void)parity;
-  a.bar_count = reinterpret_cast<unsigned long long*>(S->ctr + 2);  // 8-byte aligned
-  a.status = L->status;
-  a.has_next = next ? 1 : 0;
-  if (next) {
-    a.At_sl = next->pred_at_sl; a.Bt = next->pred_bt; a.pc = next->pred_c;
-    a.r = next->r; a.Fn = next->F; a.norm_n = next->norm; a.eps_n = next->eps; a.k_next = k_next;
-    a.z = S->z; a.sumsq = S->z + (size_t)ls::FZ_MAXE * next->r; a.zpart = S->zpart; a.range = next->fz_range;
-    a.sc = S->sc; a.sb = S->sb; a.bent = S->bent; a.kmm = S->kmm;
-    if (sel_next) {
-      a.next_idx = sel_next->idx; a.next_count = sel_next->count; a.next_mask = sel_next->mask; a.next_scores = sel_next->scores;
-      a.next_cap = sel_next->cap;
-    }
-    a.next_prio = next->prio;
-    if (next->cache_rows == 0 && (next->d * 2) % 16 == 0) {  // first rows of the next layer's bundles: speculative L2 prefetch
-      a.spec_ptr = reinterpret_cast<const char*>(next->bundles);
-      a.spec_stride = (unsigned long long)next->n_mat * next->d * 2ull; a.spec_bytes = (unsigned)next->d * 2u;
-    }
-  }
-  ls::FusedSmemLayout lay{};
-  if (!fused_plan(L, next, &lay)) return fail(LS_ERR_STATE, "fused step: shared memory plan failed");
-  a.lay = lay;
-  a.xs_put = -1; a.xs_get = -1;
-  *out = a;
-  if (lay_out) *lay_out = lay;
-  return LS_OK;
+// ---- the fused per-layer step: the whole-token kernel on a single layer --------------------------------------------------
+bool fused_shape(const ls_layer* L, const ls_layer* next, TokenShape* shp) {
+  shp->d = L->d; shp->sm_count = L->sm_count; shp->r_max = next->r; shp->f_max = std::max(L->F, next->F);
+  shp->ns_cta = (((L->d + 31) >> 5) + L->sm_count - 1) / L->sm_count;
+  return true;
+}
+bool fused_eligible(const ls_layer* L, const ls_layer* next, int batch, int K, int sel_cap, int k_next) {
+  if (!g_opt_fused.load(std::memory_order_relaxed)) return false;
+  if (batch != 1 || !next || L->cache_rows != 0 || next->cache_rows != 0) return false;
+  if (K > ls::WT_MAXK || L->d > 8 * ls::WT_THREADS * 2 || L->sm_count > kScratchMaxCtas || L->wd != next->wd) return false;
+  const int G = L->sm_count, gs = std::max(1, G / K);
+  auto per_cta = [&](int count) { const int m = (count + K - 1) / K; return (m + gs - 1) / gs; };
+  if (per_cta(sel_cap) > ls::WT_MAXMINE || per_cta(k_next) > ls::WT_MAXMINE) return false;
+  TokenShape shp{};
+  fused_shape(L, next, &shp);
+  return token_layout(&shp, K, nullptr);
 }
 
 int32_t fused_step(ls_layer* L, ls_layer* next, const float* d_x, float* d_x_out, const ls_selection* sel, int K, int k_next,
                    ls_selection* sel_next, const ls_step_trace& tr, cudaStream_t st) {
-  ls::FusedArgs a{};
-  ls::FusedSmemLayout lay{};
-  LS_TRY(fused_args(L, next, d_x, d_x_out, sel->idx, sel->count, sel->cap, K, k_next, sel_next, 0, &a, &lay));
-  const int nw_next = next ? next->nwords : 0;
-  if (next && sel_next->mask) LS_CUDA(cudaMemsetAsync(sel_next->mask, 0, (size_t)nw_next * 4, st));
-  a.tr_xtilde = tr.xtilde; a.tr_masks = next ? tr.refine_masks : nullptr; a.tr_counts = next ? tr.refine_counts : nullptr;
-  a.tr_survive = tr.survive_mask;
-  if (a.tr_masks) LS_CUDA(cudaMemsetAsync(a.tr_masks, 0, (size_t)(K + 1) * nw_next * 4, st));
-  if (a.tr_survive) LS_CUDA(cudaMemsetAsync(a.tr_survive, 0, (size_t)L->nwords * 4, st));
+  ls::WtCall c{};
+  TokenShape shp{};
+  fused_shape(L, next, &shp);
+  DeviceScratch* D = nullptr;
+  LS_TRY(device_scratch(L->device, &D));
+  ls::WtLayer& a = c.one;
+  a.bundles = L->bundles; a.b_gate = L->b_gate; a.b_down = L->b_down;
+  a.n_mat = L->n_mat; a.F = L->F; a.norm = L->norm; a.eps = L->eps;
+  a.At_sl = next->pred_at_sl; a.Bt_pad = next->pred_bt_pad; a.pc = next->pred_c;
+  a.r = next->r; a.Fn = next->F; a.norm_n = next->norm; a.eps_n = next->eps;
+  a.range = next->wt_range;
+  a.status = L->status;
+  c.cuts = D->cuts1; c.sellist = next->tmp_idx; c.xbuf = nullptr;
+  c.tr_xtilde = tr.xtilde; c.tr_masks = tr.refine_masks; c.tr_words = next->nwords; c.tr_counts = tr.refine_counts;
+  c.tr_survive = tr.survive_mask;
+  if (c.tr_survive) LS_CUDA(cudaMemsetAsync(c.tr_survive, 0, (size_t)L->nwords * 4, st));
   if (tr.exec_idx) {
     ls::ls_copy_u32_kernel<<<8, 256, 0, st>>>(reinterpret_cast<const uint32_t*>(sel->idx), reinterpret_cast<uint32_t*>(tr.exec_idx),
                                               sel->cap);
     LS_LAUNCHED();
   }
-  const int cpt = ((L->d >> 3) + ls::FZ_THREADS - 1) / ls::FZ_THREADS;
-  if (L->wd == 0) return launch_fused_cpt<0>(cpt, a, L->sm_count, lay.total, st);
-  return launch_fused_cpt<1>(cpt, a, L->sm_count, lay.total, st);
+  KernelTimer timer(LS_TIMED_FUSED, st);
+  return launch_token(&shp, L->device, L->wd, nullptr, 1, c, d_x, d_x_out, sel, K, k_next, sel_next, next->nwords, st, "ls_sparse_ffn_step");
 }
 
 // ---- speculate / refine: latent -> scores -> top-k (-> union for batch > 1) ------------------------------------------
@@ -712,7 +683,8 @@ int32_t ls_stack_create(ls_layer* const* layers, int32_t n_layers, ls_stack** ou
 #undef LS_ATTR_WT
   {
     ls::WtSmem lay{};
-    if (!token_layout(S, ls::WT_MAXK, &lay) && !token_layout(S, 1, &lay))
+    const TokenShape shp{S->d, S->sm_count, S->r_max, S->f_max, S->ns_cta};
+    if (!token_layout(&shp, ls::WT_MAXK, &lay) && !token_layout(&shp, 1, &lay))
       return cleanup(fail(LS_ERR_STATE, "ls_stack_create: the stack does not fit the whole-token kernel's shared memory"));
   }
   *out = S;
@@ -737,29 +709,10 @@ int32_t ls_stack_decode(ls_stack* S, const float* d_x, float* d_x_out, const ls_
   int fmin_ = 1 << 30;
   for (ls_layer* L : S->layers) fmin_ = std::min(fmin_, std::min(L->F, L->max_sel));
   if (k_next < 0 || k_next > fmin_) return fail(LS_ERR_INVALID, "ls_stack_decode: k_next %d outside [0, %d] (smallest d_ff / max_sel of the stack)", k_next, fmin_);
-  const int G = S->sm_count, gs = std::max(1, G / K);
-  auto per_cta = [&](int count) { const int m = (count + K - 1) / K; return (m + gs - 1) / gs; };
-  if (per_cta(sel_first->cap) > ls::WT_MAXMINE || per_cta(k_next) > ls::WT_MAXMINE)
-    return fail(LS_ERR_INVALID, "ls_stack_decode: selection too long for the whole-token kernel");
   if (sel_out->cap < k_next) return fail(LS_ERR_INVALID, "ls_stack_decode: sel_out->cap %d < k_next %d", sel_out->cap, k_next);
   DeviceGuard guard(S->device);
   cudaStream_t st = (cudaStream_t)stream;
-  DeviceScratch* D = nullptr;
-  LS_TRY(device_scratch(S->device, &D));
   ls::WtCall c{};
-  if (!token_layout(S, K, &c.lay)) return fail(LS_ERR_STATE, "ls_stack_decode: %d stages do not fit the whole-token kernel's shared memory", K);
-  c.n_layers = S->n; c.d = S->d; c.K = K; c.k_next = k_next; c.gs = gs;
-  c.piece_len = ((S->d + 3) / 4 + 255) / 256 * 256;
-  c.ring_bytes = (int)(c.lay.total - c.lay.u_off);
-  c.inv_d = 1.0 / (double)S->d;
-  c.x_in = d_x; c.x_out = d_x_out;
-  c.sel_idx = sel_first->idx; c.sel_count = sel_first->count; c.sel_cap = sel_first->cap;
-  c.out_idx = sel_out->idx; c.out_count = sel_out->count; c.out_mask = sel_out->mask; c.out_scores = sel_out->scores; c.out_cap = sel_out->cap;
-  c.xbuf = S->xbuf; c.ypart = D->ypart; c.zpart = D->zpart; c.z = D->z; c.sc = D->sc; c.sb = D->sb; c.kmm = D->kmm;
-  c.cuts = S->cuts; c.sellist = S->sellist;
-  c.tk_key = reinterpret_cast<unsigned long long*>(D->bent);
-  c.tk_idx = reinterpret_cast<int32_t*>(reinterpret_cast<unsigned char*>(D->bent) + (size_t)kScratchMaxF * 8);
-  c.bar = D->ctr + 32;
   const int nwords_max = (S->f_max + 31) / 32;
   if (trace) {
     c.tr_x = trace->x; c.tr_sel = trace->sel_idx; c.tr_cnt = trace->sel_count; c.tr_cap = trace->sel_cap;
@@ -767,18 +720,12 @@ int32_t ls_stack_decode(ls_stack* S, const float* d_x, float* d_x_out, const ls_
     if (c.tr_sel && !c.tr_cnt) return fail(LS_ERR_INVALID, "ls_stack_decode: trace->sel_count is required with trace->sel_idx");
     if (c.tr_masks && c.tr_words < nwords_max)
       return fail(LS_ERR_INVALID, "ls_stack_decode: trace->mask_words %d < %d", c.tr_words, nwords_max);
-    if (c.tr_masks) LS_CUDA(cudaMemsetAsync(c.tr_masks, 0, (size_t)S->n * (K + 1) * c.tr_words * 4, st));
   }
-  if (sel_out->mask) LS_CUDA(cudaMemsetAsync(sel_out->mask, 0, (size_t)S->layers.back()->nwords * 4, st));
-  LS_CUDA(cudaMemsetAsync(c.bar, 0, sizeof(unsigned), st));
-  const ls::WtLayer* args = S->d_layers;
-  void* params[] = {&args, &c};
-  const void* fn = nullptr;
-  fn = S->wd == 0 ? (const void*)ls::ls_token_kernel<0> : (const void*)ls::ls_token_kernel<1>;
+  c.cuts = S->cuts; c.sellist = S->sellist; c.xbuf = S->xbuf;
+  const TokenShape shp{S->d, S->sm_count, S->r_max, S->f_max, S->ns_cta};
   KernelTimer timer(LS_TIMED_STACK, st);
-  LS_CUDA(cudaLaunchCooperativeKernel(fn, dim3(G), dim3(ls::WT_THREADS), params, c.lay.total, st));
-  LS_LAUNCHED();
-  return LS_OK;
+  return launch_token(&shp, S->device, S->wd, S->d_layers, S->n, c, d_x, d_x_out, sel_first, K, k_next, sel_out, S->layers.back()->nwords, st,
+                      "ls_stack_decode");
 }
 
 int32_t ls_topk_select_static(const double* d_scores, int32_t n, int32_t k, int32_t* d_idx, uint32_t* d_mask, int32_t* d_count,
@@ -799,17 +746,6 @@ int32_t ls_topk_select_static(const double* d_scores, int32_t n, int32_t k, int3
   return LS_OK;
 }
 
-#ifdef LS_FZ_TIMING
-int32_t ls_debug_read_timing(long long* host, int32_t n) {
-  return cudaMemcpyFromSymbol(host, ls::g_fz_timing, (size_t)n * sizeof(long long)) == cudaSuccess ? LS_OK : LS_ERR_CUDA;
-}
-int32_t ls_debug_read_fail(int* host) {
-  return cudaMemcpyFromSymbol(host, ls::g_fz_fail, 64 * sizeof(int)) == cudaSuccess ? LS_OK : LS_ERR_CUDA;
-}
-int32_t ls_debug_read_cta(long long* host, int32_t n) {
-  return cudaMemcpyFromSymbol(host, ls::g_fz_cta, (size_t)n * sizeof(long long)) == cudaSuccess ? LS_OK : LS_ERR_CUDA;
-}
-#endif
 
 int32_t ls_set_option(int32_t option, int32_t value) {
   if (option == LS_OPT_FUSED) {
@@ -930,7 +866,7 @@ int32_t ls_sparse_ffn_step(ls_layer* L, ls_layer* next, const float* d_x, float*
   ls_step_trace tr{};
   if (trace) tr = *trace;
 
-  if (fused_eligible(L, next, B, K, sel->cap)) return fused_step(L, next, d_x, d_x_out, sel, K, k_next, sel_next, tr, st);
+  if (fused_eligible(L, next, B, K, sel->cap, k_next)) return fused_step(L, next, d_x, d_x_out, sel, K, k_next, sel_next, tr, st);
 
   ls::ls_step_init_kernel<<<std::min(64, (int)((bd + 255) / 256)), 256, 0, st>>>(d_x, L->b_down, L->xin, L->xt, tr.xtilde, B, d,
                                                                                L->survive, L->nwords, nullptr);

@@ -50,6 +50,7 @@ constexpr int WT_MAXE = WT_MAXK + 1;
 constexpr int WT_MAXMINE = 256;    // neurons one CTA may own in a layer
 constexpr int WT_BINCAP = 64;      // fast selection: no bin reaching into the first k ranks may hold more than this
 constexpr int WT_CANDCAP = 1024;   // candidates a CTA compares exactly
+constexpr int WT_SL = 32;          // columns of the feature one CTA owns in P1 (one slice)
 constexpr int WT_XBLK = 40;        // doubles a 32-column block of features occupies in shared memory (see wt_feat_pos)
 constexpr int WT_NSTAMP = 12;      // time stamps per CTA and layer (profiling export)
 constexpr long long WT_SPIN_CLOCKS = 4000LL * 1000 * 1000;  // about two seconds
@@ -115,7 +116,9 @@ struct WtCall {
   // trace (all nullable)
   float* tr_x; int32_t* tr_sel; int32_t* tr_cnt; int tr_cap;
   float* tr_xtilde; uint32_t* tr_masks; int tr_words; long long* tr_ns;
+  uint32_t* tr_survive; int32_t* tr_counts;  // (single step) selected neurons with a nonzero activation; sizes of the refined sets
   WtSmem lay;
+  WtLayer one;  // the layer of a single step (used when no table of layers is given)
 };
 
 struct WtShared {
@@ -388,6 +391,7 @@ __device__ __forceinline__ void wt_stream(const WtCall& C, WtShared& sh, const W
       }
       __syncthreads();
     }
+    if (C.tr_survive && tid < nb && s_sact[b0 + tid] != 0.f) atomicOr(C.tr_survive + (s_sidx[b0 + tid] >> 5), 1u << (s_sidx[b0 + tid] & 31));
     // down rows scaled into the partial output: every thread owns eight columns
     const unsigned char* dn = ring + (rest_b - row_b);
 #pragma unroll 1
@@ -885,6 +889,7 @@ __device__ __noinline__ void wt_export_selection(const WtCall& C, const int* s_m
     if (C.tr_cnt) C.tr_cnt[n + 1] = keff;
     if (last) *C.out_count = min(keff, C.out_cap);
   }
+  if (blockIdx.x == 0 && C.tr_counts && tid < E) C.tr_counts[tid] = keff;
 }
 
 // New bin range of the layer's scores from what this launch observed (one warp; used by the next launch).
@@ -930,7 +935,8 @@ __global__ void __launch_bounds__(WT_THREADS, 1) ls_token_kernel(const WtLayer* 
   unsigned epoch = 0;
 
   // ---- prologue: arguments of layer 0, x, 1 / rms, this CTA's slice of the first selection
-  if (tid < NW) reinterpret_cast<uint32_t*>(&sh.L[0])[tid] = reinterpret_cast<const uint32_t*>(&g_layers[0])[tid];
+  if (tid < NW)
+    reinterpret_cast<uint32_t*>(&sh.L[0])[tid] = g_layers ? reinterpret_cast<const uint32_t*>(&g_layers[0])[tid] : reinterpret_cast<const uint32_t*>(&C.one)[tid];
   if (tid == 0) { sh.dead = 0; sh.b_valid = 1; }
   {
     double sq = 0.0;
@@ -1047,7 +1053,7 @@ __global__ void __launch_bounds__(WT_THREADS, 1) ls_token_kernel(const WtLayer* 
     }
     if (stamps) wt_stamp(C, n, 9);
     if (tid == 0) sh.nmine = hi - lo;
-    if (last || C.tr_sel || C.tr_masks) wt_export_selection(C, s_mine, n, lo, hi - lo, keff, last);
+    if (last || C.tr_sel || C.tr_masks || C.tr_counts) wt_export_selection(C, s_mine, n, lo, hi - lo, keff, last);
     if (cta == 0 && tid < 32) wt_update_range(C, L);
     __syncthreads();
     if (stamps) wt_stamp(C, n, 10);

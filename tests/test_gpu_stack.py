@@ -170,3 +170,94 @@ def test_llama7b_shaped_stack_with_a_wide_selection():
     stats = {}
     decode_and_check(spec, arrays, 3, 4096, 1, stats, tokens=wl.make_tokens(spec, 2)[1:2])
     assert stats.get("band", 0) == 0
+
+
+def test_degenerate_selection_through_the_whole_token_kernel():
+    """Layer 1's predictor is zero with a constant offset: every score of every evaluation is equal, one bin holds all
+    neurons, so the selection takes the kernel's general route (one CTA, an extra barrier).  Expected: index order, and
+    every refined set equal to the first k indices; the outputs still follow from those selections."""
+    spec = wl.SPECS["tiny4"]
+    arrays = wl.make_stack(spec, n_layers=3, down_scale=50.0)
+    arrays[1].pred_b = np.zeros_like(arrays[1].pred_b)
+    arrays[1].pred_c = np.full_like(arrays[1].pred_c, 0.25)
+    OLs = [orc.OracleLayer.from_arrays(a) for a in arrays]
+    GLs = [ls.ls_layer_create(a, DEV) for a in arrays]
+    stack = ls.ls_stack_create(GLs)
+    k, K, n = spec.k, 4, 3
+    sel0, sel_out = ls.Selection(spec.d_ff, k, DEV), ls.Selection(spec.d_ff, k, DEV)
+    trace = ls.StackTrace(stack, k, n_chunks=K)
+    for x0 in wl.make_tokens(spec)[:2]:  # (twice: the second launch starts from the bin range the first one left)
+        x = torch.from_numpy(x0).cuda(DEV)
+        x_out = torch.empty_like(x)
+        ls.ls_predict(GLs[0], x, k, sel0)
+        ls.ls_stack_decode(stack, x, x_out, sel0, K, k, sel_out, trace)
+        torch.cuda.synchronize()
+        assert all(ls.ls_layer_status(g) == 0 for g in GLs)
+        S = trace.sel_idx.cpu().numpy()
+        M = trace.refine_masks.cpu().numpy().view(np.uint32)
+        X = trace.x.cpu().numpy()
+        assert S[1, :k].tolist() == list(range(k))                       # layer 0 refined layer 1: all scores equal
+        for j in range(K + 1):
+            assert mask_to_set(M[0, j], spec.d_ff) == set(range(k))
+        stats = {}
+        for layer in range(n):
+            nxt = OLs[min(layer + 1, n - 1)]
+            res = orc.sparse_ffn_step(OLs[layer], None, X[layer], S[layer, :k].astype(np.int64), K)
+            assert_values_close(X[layer + 1] - X[layer], res["y"][0], what=f"layer {layer}")
+            check_selection(S[layer + 1, :k].astype(np.int64), orc.predictor_scores(nxt, X[layer + 1]), k, stats)
+        assert stats.get("band", 0) == 0
+    stack.close()
+    for g in GLs:
+        g.close()
+
+
+def test_llama7b_full_stack_two_consecutive_tokens():
+    """The benchmark configuration itself: all 32 layers of the Llama-2-7B-shaped stack, K = 8, k = 1728, two tokens in a
+    row through the same stack (the second launch starts from the first one's bin ranges, cut keys and scratch).  Every
+    layer boundary, every partial residual feature and every refined set of both tokens is replayed through the oracle.
+    Host arrays are regenerated layer by layer (the generator is seeded), so that only two layers are held at a time."""
+    spec = wl.SPECS["llama2-7b"]
+    n, K, k = spec.n_layers, 8, spec.k
+    GLs = []
+    for l in range(n):
+        GLs.append(ls.ls_layer_create(wl.make_layer(spec, l, svd_device="cuda"), DEV))
+    stack = ls.ls_stack_create(GLs)
+    sel0, sel_out = ls.Selection(spec.d_ff, k, DEV), ls.Selection(spec.d_ff, k, DEV)
+    toks = wl.make_tokens(spec, 2)
+    rec = []
+    for x0 in toks:
+        trace = ls.StackTrace(stack, k, n_chunks=K)
+        x = torch.from_numpy(x0).cuda(DEV)
+        x_out = torch.empty_like(x)
+        ls.ls_predict(GLs[0], x, k, sel0)
+        ls.ls_stack_decode(stack, x, x_out, sel0, K, k, sel_out, trace)
+        torch.cuda.synchronize()
+        assert all(ls.ls_layer_status(g) == 0 for g in GLs)
+        rec.append((trace.x.cpu().numpy(), trace.sel_idx.cpu().numpy(), trace.xtilde.cpu().numpy(),
+                    trace.refine_masks.cpu().numpy().view(np.uint32), x_out.cpu().numpy(), sel_out.order().copy()))
+    stack.close()
+    for g in GLs:
+        g.close()
+    stats = {}
+    cur = orc.OracleLayer.from_arrays(wl.make_layer(spec, 0, svd_device="cuda"))
+    for layer in range(n):
+        nxt = cur if layer + 1 == n else orc.OracleLayer.from_arrays(wl.make_layer(spec, layer + 1, svd_device="cuda"))
+        for t, (X, S, XT, M, x_out, order_out) in enumerate(rec):
+            order = S[layer, :k].astype(np.int64)
+            if layer == 0:
+                np.testing.assert_array_equal(X[0], toks[t])
+                check_selection(order, orc.predictor_scores(cur, X[0]), k, stats)
+            res = orc.sparse_ffn_step(cur, None, X[layer], order, K)
+            assert_values_close(X[layer + 1] - X[layer], res["y"][0], what=f"token {t} layer {layer}")
+            np.testing.assert_array_equal(XT[layer, K], X[layer + 1])
+            for j in range(1, K + 1):
+                assert_values_close(XT[layer, j] - XT[layer, j - 1], res["xtilde"][j][0] - res["xtilde"][j - 1][0],
+                                    scale_ref=res["y"][0], what=f"token {t} layer {layer} stage {j}")
+            for j in range(K + 1):
+                assert_set_in_tie_band(mask_to_set(M[layer, j], spec.d_ff), orc.predictor_scores(nxt, XT[layer, j]), k, stats)
+            check_selection(S[layer + 1, :k].astype(np.int64), orc.predictor_scores(nxt, X[layer + 1]), k, stats)
+            if layer + 1 == n:
+                np.testing.assert_array_equal(X[n], x_out)
+                assert S[n, :k].tolist() == order_out.tolist()
+        cur = nxt
+    assert stats.get("band", 0) == 0

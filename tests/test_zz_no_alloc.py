@@ -10,6 +10,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import leanstream_oracle as orc
 from paper_2609_03079_b200 import binding as ls
 from paper_2609_03079_b200 import workload as wl
 
@@ -53,3 +54,27 @@ def test_static_topk_rejects_sizes_beyond_its_scratch():
     assert e.value.code == ls.LS_ERR_INVALID and str(ls.LS_STATIC_TOPK_MAX_N) in str(e.value)
     with pytest.raises(ls.LeanStreamError):
         ls.ls_topk_select_static(big[:16], 17, idx, None, count)
+
+
+@pytest.mark.parametrize("n,k,kind", [(1024, 160, "normal"), (32768, 20000, "normal"), (32768, 5000, "coarse"), (4096, 1000, "equal")])
+def test_static_topk_against_the_oracle(n, k, kind):
+    """The allocation-free entry point against the oracle's total order itself, at its largest size (where the
+    candidates no longer fit in shared memory and live in the static array), with heavy ties and with all scores equal."""
+    dev = torch.device("cuda", 0)
+    rng = np.random.default_rng(n + k)
+    if kind == "normal":
+        s = rng.standard_normal(n)
+    elif kind == "coarse":
+        s = np.round(rng.standard_normal(n) * 4.0) / 4.0  # about thirty distinct values: long runs of exact ties
+    else:
+        s = np.full(n, -1.5)
+    idx = torch.full((n,), -1, dtype=torch.int32, device=dev)
+    mask = torch.zeros((n + 31) // 32, dtype=torch.int32, device=dev)
+    count = torch.zeros(1, dtype=torch.int32, device=dev)
+    want = orc.topk_order(s, k)
+    for _ in range(2):
+        ls.ls_topk_select_static(torch.from_numpy(s).to(dev), k, idx, mask, count)
+        torch.cuda.synchronize()
+        assert int(count.item()) == k
+        assert idx[:k].cpu().numpy().astype(np.int64).tolist() == want.tolist()
+        assert np.array_equal(mask.cpu().numpy().view(np.uint32), orc.mask_of(want, n))
