@@ -15,9 +15,9 @@
  *    caller; the library neither frees nor keeps them after the call has been enqueued.  Pointers inside
  *    ls_layer_desc are HOST pointers read only during ls_layer_create().
  *  - `stream` arguments carry a cudaStream_t (0 = the legacy default stream).  Work is enqueued asynchronously;
- *    argument validation is synchronous.  Calls on layers with a cache (cache_rows > 0) synchronise with the host
- *    to issue the miss copies and must not be made during stream capture; calls on fully resident layers never
- *    synchronise or allocate and may be captured in a CUDA graph.
+ *    argument validation is synchronous.  Calls on fully resident layers never synchronise or allocate and may be
+ *    captured in a CUDA graph; calls on layers with a cache (cache_rows > 0) do not synchronise either (except where a
+ *    result is returned to the host) but use a second stream and events and are not meant for capture.
  *  - A layer handle is not thread safe: one call at a time per layer; per-layer scratch is reused by every call.
  *  - Neuron i of a layer owns gate row i, up row i and down-projection row i (column i of the paper's W_gate /
  *    W_up, row i of W_down).  Index lists are int32, masks hold neuron i at bit (i & 31) of word (i >> 5).
@@ -138,9 +138,10 @@ typedef struct {
  * formed; C^(K) is returned in sel_next (required when next != NULL) and next's retention priorities are updated
  * at each stage.  When `next` has a cache, the first ceil(count_j (j+1)/(K+1)) ranks of C^(j), j < K, are reserved
  * in it (miss copies start on next's copy stream).  When `layer` has a cache, the whole selection is reserved
- * first, residents run before misses, and the stages that need copied rows wait for them on `stream`.
+ * first, residents run before misses, and the stages that need copied rows wait for them on the device.
  * d_x, d_x_out: float [batch][d_model]; d_x_out may alias d_x.  next may equal layer.
- * Errors: LS_ERR_INVALID, LS_ERR_CAPACITY (cached layer: selection larger than the cache), LS_ERR_CUDA.
+ * Errors: LS_ERR_INVALID, LS_ERR_CAPACITY (cached layer: sel->cap larger than the cache; a list whose actual count
+ * overflows is reported through ls_layer_status), LS_ERR_CUDA.
  */
 int32_t ls_sparse_ffn_step(ls_layer *layer, ls_layer *next, const float *d_x, float *d_x_out, int32_t batch,
                            const ls_selection *sel, int32_t n_chunks, int32_t k_next, ls_selection *sel_next,
@@ -148,21 +149,24 @@ int32_t ls_sparse_ffn_step(ls_layer *layer, ls_layer *next, const float *d_x, fl
 
 /*
  * HBM neuron cache (Section 3.3.3 cache-eviction task; Section 4.3 cache miss ratio).  Residency is logical: a
- * neuron is resident once a slot is assigned to it; its bytes arrive on the layer's copy stream and consumers
- * wait for the copy event.  All three calls return LS_ERR_STATE on a layer created with cache_rows = 0.
+ * neuron is resident once a slot is assigned to it; its bytes arrive on the layer's copy stream (LS_OPT_MISS_PATH) and
+ * the kernels that read them wait on the device until they have landed.  All calls return LS_ERR_STATE on a layer
+ * created with cache_rows = 0.
  *
  * ls_cache_lookup: d_slot[j] = slot of neuron d_idx[j] or -1 (miss); *d_nhit = number of residents.  n <= max_sel.
  *
  * ls_cache_reserve: makes the first `admit_ranks` entries (< 0: all) of want->idx resident.  The new resident set
  *   is the cache_rows best of (residents + wanted) under the key (wanted or protected first, then retention
  *   priority descending, then index ascending); the rest are evicted and their slots given to the misses, whose
- *   bundles are copied from pinned host memory with cudaMemcpyAsync on the layer's copy stream.  When
- *   want->scores is given it first replaces the layer's retention priorities.  d_protect_mask (nullable) marks
- *   neurons that must not be evicted.  *h_nmiss (nullable, HOST) receives the number of misses.  Synchronises
- *   `stream` with the host.  LS_ERR_CAPACITY if wanted + protected exceed cache_rows (nothing changes).
+ *   bundles are brought from pinned host memory on the layer's copy stream.  When want->scores is given it first
+ *   replaces the layer's retention priorities.  d_protect_mask (nullable) marks neurons that must not be evicted.
+ *   *h_nmiss (nullable, HOST) receives the number of misses: for it the call waits on the calling thread for the decision
+ *   (not for the copies), at most LS_OPT_HOST_WAIT_MS (LS_ERR_TIMEOUT otherwise; the request stays enqueued).
+ *   LS_ERR_CAPACITY if wanted + protected exceed cache_rows (nothing changes).
+ *   (ls_sparse_ffn_step reserves through the same machinery without waiting on the host at all.)
  *
  * ls_cache_evict: evicts lowest-priority unprotected residents until at least min_free slots are free (fewer when
- *   only protected ones remain); d_evicted (nullable, [cache_rows]) and d_nevicted (nullable) receive them.
+ *   only protected ones remain); d_evicted (nullable, [cache_rows]) and d_nevicted (nullable) receive them.  Asynchronous.
  */
 int32_t ls_cache_lookup(ls_layer *layer, const int32_t *d_idx, int32_t n, int32_t *d_slot, int32_t *d_nhit,
                         void *stream);
@@ -172,16 +176,16 @@ int32_t ls_cache_evict(ls_layer *layer, int32_t min_free, const uint32_t *d_prot
                        int32_t *d_nevicted, void *stream);
 /* d_resident_mask [ceil(d_ff/32)] <- current logical resident set (for parity checks). */
 int32_t ls_cache_snapshot(ls_layer *layer, uint32_t *d_resident_mask, void *stream);
-/* Makes `stream` wait until every miss copy issued so far for this layer has landed. */
+/* Makes `stream` wait (on the device, bounded) until the rows of every request made so far for this layer have landed. */
 int32_t ls_cache_wait(ls_layer *layer, void *stream);
 
 typedef struct {
   int64_t hits, misses, evictions; /* counted over reserve calls (wanted entries found / not found resident) */
-  int64_t h2d_bytes;               /* bytes copied from pinned host memory into cache slots */
-  int64_t h2d_copies;              /* number of cudaMemcpyAsync calls issued for them */
+  int64_t h2d_bytes;               /* bytes brought from pinned host memory into cache slots */
+  int64_t h2d_copies;              /* copy operations issued for them: cudaMemcpyAsync calls (I/O lane) or gather launches */
   int64_t resident;                /* current number of resident neurons */
 } ls_cache_stats_t;
-/* Host-side counters (no synchronisation needed; they are updated when a reserve call returns). */
+/* Counters kept on the device by the decision kernels; the call synchronises the device. */
 int32_t ls_cache_stats(ls_layer *layer, ls_cache_stats_t *host_out);
 
 /* Reads and clears the layer's device-side status word (0 = no problem seen by any kernel since the last read;
@@ -268,6 +272,22 @@ int32_t ls_topk_select_static(const double *d_scores, int32_t n, int32_t k, int3
  * scratch per device: issue them on one stream, or order the streams that issue them.
  */
 #define LS_OPT_FUSED 1
+/*
+ * LS_OPT_MISS_PATH: how the misses of a cached layer travel from pinned host memory to their cache slots.  Either way the
+ * calling thread only enqueues work and the stages that need copied rows wait on the device (bounded) for a word the copy
+ * stream raises; set the option before the first call on a cached layer and do not change it while requests are in flight.
+ *   LS_MISS_PATH_LANE:   Section 3.2.1 / Algorithm 1 of the paper re-targeted: the decision kernel writes its miss list
+ *     and a sequence flag to mapped pinned memory; a host thread of the library (the paper's I/O lane) polls the flag and
+ *     issues one cudaMemcpyAsync per run of adjacent neurons and slots on the layer's copy stream.
+ *   LS_MISS_PATH_GATHER (default): the list stays on the device and one kernel on the copy stream reads the missing
+ *     bundles straight from the mapped pinned store over the host link; no host thread takes part.
+ * LS_OPT_HOST_WAIT_MS (default 30000): how long ls_cache_reserve waits on the calling thread for the number of misses
+ * before it returns LS_ERR_TIMEOUT.  A request that timed out stays enqueued and takes effect when its stream reaches it.
+ */
+#define LS_OPT_MISS_PATH 2
+#define LS_MISS_PATH_LANE 0
+#define LS_MISS_PATH_GATHER 1
+#define LS_OPT_HOST_WAIT_MS 3
 int32_t ls_set_option(int32_t option, int32_t value);
 
 /*

@@ -310,7 +310,8 @@ def ls_timing_read(kind: int):
     return n.value, ms.value
 
 
-LS_OPT_FUSED = 1
+LS_OPT_FUSED, LS_OPT_MISS_PATH, LS_OPT_HOST_WAIT_MS = 1, 2, 3
+LS_MISS_PATH_LANE, LS_MISS_PATH_GATHER = 0, 1
 
 
 def ls_set_option(option: int, value: int) -> None:

@@ -19,6 +19,8 @@ namespace {
 thread_local std::string g_err;
 std::atomic<int64_t> g_launches{0};
 std::atomic<int> g_opt_fused{1};
+std::atomic<int> g_opt_miss_path{1};     // ls::MISS_PATH_GATHER
+std::atomic<int> g_opt_host_wait_ms{30000};
 
 int32_t fail(int32_t code, const char* fmt, ...) {
   char buf[512];
@@ -269,7 +271,7 @@ int32_t create_impl(const ls_layer_desc* D, ls_layer* L) {
       LS_CUDA(cudaMemcpy2D(reinterpret_cast<char*>(L->bundles) + m * row_bytes, bundle_bytes, mats[m], row_bytes, row_bytes, F,
                            cudaMemcpyHostToDevice));
   } else {
-    LS_TRY(ls::cache_create(L->cache, (int)F, (int)L->cache_rows, bundle_bytes, L->max_sel, g_err));
+    LS_TRY(ls::cache_create(L->cache, D->device, (int)F, (int)L->cache_rows, bundle_bytes, L->max_sel, L->bundles, g_err));
     char* hb = static_cast<char*>(L->cache.h_bundles);
     for (int m = 0; m < L->n_mat; ++m) {
       const char* src = static_cast<const char*>(mats[m]);
@@ -496,7 +498,7 @@ int32_t predict_impl(ls_layer* L, const float* d_feature, int B, int k, double* 
 
 template <int WD, int BT>
 int32_t launch_stage(ls_layer* L, int B, const int32_t* exec_idx, const int32_t* count_ptr, int sel_cap, int K, int c,
-                     cudaStream_t st) {
+                     cudaStream_t st, unsigned need_seq) {
   const int d = L->d;
   const int32_t* slot_of = L->cache_rows > 0 ? L->cache.d_slot_of : nullptr;
   const int per_stage = (sel_cap + K - 1) / K;
@@ -506,7 +508,8 @@ int32_t launch_stage(ls_layer* L, int B, const int32_t* exec_idx, const int32_t*
     const size_t sm = (size_t)B * d * sizeof(float);
     ls::ls_gateup_kernel<WD, BT><<<grid, 256, sm, st>>>(L->bundles, L->n_mat, L->gated, slot_of, L->b_gate, L->xin, B, d, L->norm,
                                                         L->eps, exec_idx, count_ptr, K, c, L->F, L->actv, L->max_sel, L->survive,
-                                                        L->status);
+                                                        L->status, need_seq ? L->cache.d_landed : nullptr, need_seq,
+                                                        need_seq ? ls::cache_list_header(L->cache, need_seq) : nullptr);
     LS_LAUNCHED();
   }
   {
@@ -522,8 +525,8 @@ int32_t launch_stage(ls_layer* L, int B, const int32_t* exec_idx, const int32_t*
 }
 
 int32_t launch_stage_dispatch(ls_layer* L, int B, const int32_t* exec_idx, const int32_t* count_ptr, int sel_cap, int K, int c,
-                              cudaStream_t st) {
-#define LS_STAGE(WD, BT) return launch_stage<WD, BT>(L, B, exec_idx, count_ptr, sel_cap, K, c, st)
+                              cudaStream_t st, unsigned need_seq) {
+#define LS_STAGE(WD, BT) return launch_stage<WD, BT>(L, B, exec_idx, count_ptr, sel_cap, K, c, st, need_seq)
   if (L->wd == 0) {
     if (B == 1) LS_STAGE(0, 1);
     if (B <= 4) LS_STAGE(0, 4);
@@ -535,6 +538,8 @@ int32_t launch_stage_dispatch(ls_layer* L, int B, const int32_t* exec_idx, const
   }
 #undef LS_STAGE
 }
+
+inline int32_t cache_rc(int32_t rc) { return rc; }  // (the cache layer returns the public codes and has set the error text)
 
 int32_t check_layer_call(ls_layer* L, int batch, const char* what) {
   if (!L) return fail(LS_ERR_INVALID, "%s: layer is NULL", what);
@@ -752,6 +757,16 @@ int32_t ls_set_option(int32_t option, int32_t value) {
     g_opt_fused.store(value ? 1 : 0);
     return LS_OK;
   }
+  if (option == LS_OPT_MISS_PATH) {
+    if (value != LS_MISS_PATH_LANE && value != LS_MISS_PATH_GATHER) return fail(LS_ERR_INVALID, "ls_set_option: unknown miss path %d", value);
+    g_opt_miss_path.store(value);
+    return LS_OK;
+  }
+  if (option == LS_OPT_HOST_WAIT_MS) {
+    if (value < 0) return fail(LS_ERR_INVALID, "ls_set_option: negative wait limit");
+    g_opt_host_wait_ms.store(value);
+    return LS_OK;
+  }
   return fail(LS_ERR_INVALID, "ls_set_option: unknown option %d", option);
 }
 
@@ -873,17 +888,15 @@ int32_t ls_sparse_ffn_step(ls_layer* L, ls_layer* next, const float* d_x, float*
   LS_LAUNCHED();
 
   const int32_t* exec_idx = sel->idx;
-  int first_miss_stage = K;
+  unsigned own_seq = 0;
+  const int miss_path = g_opt_miss_path.load(std::memory_order_relaxed);
   if (L->cache_rows > 0) {
-    // reserve the whole selection; residents run first, misses after (in the order their copies were issued)
-    int32_t nmiss = 0;
-    LS_TRY(ls::cache_reserve(L->cache, L->prio, L->F, sel->idx, sel->count, -1, 0, 0, sel->cap, nullptr, L->bundles, L->status, st,
-                             &nmiss, g_err, g_launches));
+    // reserve the whole selection; residents run first, misses after (in the order their copies are issued).  Nothing
+    // waits here: the stages that reach into the misses wait on the device for the request's rows.
+    if (sel->cap > L->cache_rows) return fail(LS_ERR_CAPACITY, "ls_sparse_ffn_step: selection capacity %d exceeds the cache (%lld rows)", sel->cap, (long long)L->cache_rows);
+    LS_TRY(cache_rc(ls::cache_reserve_async(L->cache, miss_path, L->prio, L->F, sel->idx, sel->count, -1, 0, 0, sel->cap, nullptr, L->status, st,
+                                            &own_seq, g_err, g_launches)));
     exec_idx = L->cache.d_exec_idx;
-    // stages made of residents only may start before the copies have landed
-    const int count = L->cache.last_nhit + L->cache.last_nmiss;
-    const int m = count > 0 ? (count + K - 1) / K : 1;
-    first_miss_stage = nmiss > 0 ? L->cache.last_nhit / m : K;
   }
   if (tr.exec_idx) {
     ls::ls_copy_u32_kernel<<<8, 256, 0, st>>>(reinterpret_cast<const uint32_t*>(exec_idx), reinterpret_cast<uint32_t*>(tr.exec_idx),
@@ -910,17 +923,15 @@ int32_t ls_sparse_ffn_step(ls_layer* L, ls_layer* next, const float* d_x, float*
     }
     if (!last && next->cache_rows > 0 && next != L) {
       // fetch rule: the first ceil(count (j+1)/(K+1)) ranks of C^(j) are admitted
-      int32_t nmiss = 0;
-      LS_TRY(ls::cache_reserve(next->cache, next->prio, next->F, idx_out, cnt_out, 0, j + 1, K + 1, next->max_sel, nullptr,
-                               next->bundles, next->status, st, &nmiss, g_err, g_launches));
+      LS_TRY(cache_rc(ls::cache_reserve_async(next->cache, miss_path, next->prio, next->F, idx_out, cnt_out, 0, j + 1, K + 1, next->max_sel,
+                                              nullptr, next->status, st, nullptr, g_err, g_launches)));
     }
     return LS_OK;
   };
 
   LS_TRY(refine(0));
   for (int c = 0; c < K; ++c) {
-    if (c == first_miss_stage) LS_TRY(ls::cache_wait(L->cache, st, g_err));
-    const int32_t splits = launch_stage_dispatch(L, B, exec_idx, sel->count, sel->cap, K, c, st);
+    const int32_t splits = launch_stage_dispatch(L, B, exec_idx, sel->count, sel->cap, K, c, st, own_seq);
     if (splits < 0) return splits;
     const bool last = (c + 1 == K);
     ls::ls_stage_finalize_kernel<<<std::min(64, (int)((bd + 255) / 256)), 256, 0, st>>>(
@@ -952,8 +963,12 @@ int32_t ls_cache_reserve(ls_layer* L, const ls_selection* want, int32_t admit_ra
   DeviceGuard guard(L->device);
   cudaStream_t st = (cudaStream_t)stream;
   if (want->scores) LS_CUDA(cudaMemcpyAsync(L->prio, want->scores, (size_t)L->F * sizeof(double), cudaMemcpyDeviceToDevice, st));
-  return ls::cache_reserve(L->cache, L->prio, L->F, want->idx, want->count, admit_ranks < 0 ? -1 : admit_ranks, 0, 0, want->cap,
-                           d_protect_mask, L->bundles, L->status, st, h_nmiss, g_err, g_launches);
+  unsigned seq = 0;
+  LS_TRY(cache_rc(ls::cache_reserve_async(L->cache, g_opt_miss_path.load(std::memory_order_relaxed), L->prio, L->F, want->idx, want->count,
+                                          admit_ranks < 0 ? -1 : admit_ranks, 0, 0, want->cap, d_protect_mask, L->status, st, &seq, g_err,
+                                          g_launches)));
+  // this call reports the number of misses: it waits (bounded) for the decision, not for the copies
+  return cache_rc(ls::cache_request_result(L->cache, seq, st, g_opt_host_wait_ms.load(std::memory_order_relaxed) * 1e-3, h_nmiss, g_err));
 }
 
 int32_t ls_cache_evict(ls_layer* L, int32_t min_free, const uint32_t* d_protect_mask, int32_t* d_evicted, int32_t* d_nevicted,
@@ -977,14 +992,16 @@ int32_t ls_cache_wait(ls_layer* L, void* stream) {
   if (!L) return fail(LS_ERR_INVALID, "ls_cache_wait: NULL layer");
   if (L->cache_rows == 0) return fail(LS_ERR_STATE, "ls_cache_wait: layer has no cache");
   DeviceGuard guard(L->device);
-  return ls::cache_wait(L->cache, (cudaStream_t)stream, g_err);
+  return cache_rc(ls::cache_wait(L->cache, L->status, (cudaStream_t)stream, g_err, g_launches));
 }
 
 int32_t ls_cache_stats(ls_layer* L, ls_cache_stats_t* out) {
   if (!L || !out) return fail(LS_ERR_INVALID, "ls_cache_stats: NULL argument");
   if (L->cache_rows == 0) return fail(LS_ERR_STATE, "ls_cache_stats: layer has no cache");
-  out->hits = L->cache.hits; out->misses = L->cache.misses; out->evictions = L->cache.evictions;
-  out->h2d_bytes = L->cache.h2d_bytes; out->h2d_copies = L->cache.h2d_copies; out->resident = L->cache.resident;
+  DeviceGuard guard(L->device);
+  long long v[8];
+  LS_TRY(cache_rc(ls::cache_stats(L->cache, v, g_err)));
+  out->hits = v[0]; out->misses = v[1]; out->evictions = v[2]; out->resident = v[3]; out->h2d_bytes = v[4]; out->h2d_copies = v[5];
   return LS_OK;
 }
 

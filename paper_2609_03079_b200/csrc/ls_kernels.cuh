@@ -118,7 +118,8 @@ __global__ void __launch_bounds__(256)
     ls_gateup_kernel(const uint16_t* __restrict__ bundles, int n_mat, int gated, const int32_t* __restrict__ slot_of,
                      const float* __restrict__ b_gate, const float* __restrict__ xin, int B, int d, int norm, float eps,
                      const int32_t* __restrict__ exec_idx, const int32_t* __restrict__ count_ptr, int K, int c, int F,
-                     float* __restrict__ act, int act_stride, uint32_t* survive, int* status) {
+                     float* __restrict__ act, int act_stride, uint32_t* survive, int* status, const unsigned* landed, unsigned need_seq,
+                     const int32_t* list_hdr) {
   extern __shared__ __align__(16) float xs[];  // [B][d]
   __shared__ float s_inv[8];
   __shared__ double s_red[8][8];
@@ -126,6 +127,15 @@ __global__ void __launch_bounds__(256)
   int lo, hi;
   stage_bounds(*count_ptr, K, c, lo, hi);
   if (lo + (int)blockIdx.x * 8 >= hi) return;
+  // Cached layer: the residents come first in the execution order; a stage that reaches into the misses waits (bounded)
+  // until the rows of the layer's request have landed in their slots.
+  if (landed && threadIdx.x == 0 && hi > list_hdr[1]) {
+    const long long t0 = clock64();
+    while (*reinterpret_cast<const volatile unsigned*>(landed) < need_seq) {
+      if (clock64() - t0 > 4000LL * 1000 * 1000) { set_status(status, ST_TIMEOUT); break; }
+    }
+    __threadfence();
+  }
 
   for (int b = 0; b < B; ++b) {
     double sq = 0.0;

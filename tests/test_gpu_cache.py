@@ -10,6 +10,17 @@ from paper_2609_03079_b200 import workload as wl
 from tests.helpers import assert_values_close, mask_to_set
 
 pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(autouse=True, params=[ls.LS_MISS_PATH_GATHER, ls.LS_MISS_PATH_LANE], ids=["gather", "lane"])
+def miss_path(request):
+    """Every test runs on both transports of the misses: the gather kernel that reads pinned host memory itself, and the
+    host I/O lane (a thread of the library polling the flags the decision kernels raise, copies by cudaMemcpyAsync)."""
+    torch.cuda.synchronize()
+    ls.ls_set_option(ls.LS_OPT_MISS_PATH, request.param)
+    yield request.param
+    torch.cuda.synchronize()
+    ls.ls_set_option(ls.LS_OPT_MISS_PATH, ls.LS_MISS_PATH_GATHER)
 DEV = 0
 
 
@@ -154,3 +165,43 @@ def test_cached_stack_decode_matches_oracle(K):
         assert ls.ls_layer_status(GLs[n]) == 0
     for g in GLs + plain:
         g.close()
+
+
+def test_reserve_times_out_on_the_host_and_the_layer_stays_usable():
+    """Failure path of the one wait the calling thread has: with the compute stream still busy with ordinary earlier work
+    and a wait limit of zero, ls_cache_reserve gives up with LS_ERR_TIMEOUT and a useful message.  Nothing is lost: the
+    request stays enqueued and takes effect when the stream reaches it (it COUNTS: the oracle's cache makes the same
+    reserve), the next call works, and the resident set equals the oracle's."""
+    spec = ar1_spec(seed=35)
+    la = wl.make_layer(spec, 0)
+    C_ROWS, k = 300, 160
+    gl = ls.ls_layer_create(la, DEV, cache_rows=C_ROWS)
+    cache = orc.LogicalCache(1024, C_ROWS)
+    sel = ls.Selection(gl.d_ff, k, DEV)
+    toks = wl.make_tokens(spec)
+    try:
+        ls.ls_predict(gl, dev_tensor(toks[0]), k, sel)
+        cache.set_priorities(sel.scores.cpu().numpy())
+        order = sel.order()
+        torch.cuda.synchronize()
+        ls.ls_set_option(ls.LS_OPT_HOST_WAIT_MS, 0)
+        # ordinary work that keeps the stream busy for a moment (a few large matrix products), then the reserve behind it
+        a = torch.randn(8192, 8192, device=f"cuda:{DEV}")
+        for _ in range(20):
+            a = (a @ a).clamp_(-1, 1)
+        with pytest.raises(ls.LeanStreamError) as e:
+            ls.ls_cache_reserve(gl, sel)
+        assert e.value.code == ls.LS_ERR_TIMEOUT and "timed out" in str(e.value)
+    finally:
+        ls.ls_set_option(ls.LS_OPT_HOST_WAIT_MS, 30000)
+    torch.cuda.synchronize()
+    misses, _ = cache.reserve(order)  # the request that timed out on the host did run
+    assert snapshot(gl) == cache.resident
+    st = ls.ls_cache_stats(gl)
+    assert st["misses"] == len(misses) == cache.misses
+    ls.ls_predict(gl, dev_tensor(toks[1]), k, sel)
+    cache.set_priorities(sel.scores.cpu().numpy())
+    m2, _ = cache.reserve(sel.order())
+    assert ls.ls_cache_reserve(gl, sel) == len(m2)
+    assert snapshot(gl) == cache.resident and ls.ls_layer_status(gl) == 0
+    gl.close()
