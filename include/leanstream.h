@@ -278,7 +278,9 @@ int32_t ls_topk_select_static(const double *d_scores, int32_t n, int32_t k, int3
  * stream raises; set the option before the first call on a cached layer and do not change it while requests are in flight.
  *   LS_MISS_PATH_LANE:   Section 3.2.1 / Algorithm 1 of the paper re-targeted: the decision kernel writes its miss list
  *     and a sequence flag to mapped pinned memory; a host thread of the library (the paper's I/O lane) polls the flag and
- *     issues one cudaMemcpyAsync per run of adjacent neurons and slots on the layer's copy stream.
+ *     issues one cudaMemcpyAsync per run of adjacent neurons and slots on the layer's copy stream.  The calling thread
+ *     lets at most two requests of a layer be in flight and enqueues the stages of a step once the lane has issued the
+ *     copies of the step's own request (bounded host waits on the lane's acknowledgement word, never on the stream).
  *   LS_MISS_PATH_GATHER (default): the list stays on the device and one kernel on the copy stream reads the missing
  *     bundles straight from the mapped pinned store over the host link; no host thread takes part.
  * LS_OPT_HOST_WAIT_MS (default 30000): how long ls_cache_reserve waits on the calling thread for the number of misses

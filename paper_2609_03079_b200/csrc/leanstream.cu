@@ -894,8 +894,11 @@ int32_t ls_sparse_ffn_step(ls_layer* L, ls_layer* next, const float* d_x, float*
     // reserve the whole selection; residents run first, misses after (in the order their copies are issued).  Nothing
     // waits here: the stages that reach into the misses wait on the device for the request's rows.
     if (sel->cap > L->cache_rows) return fail(LS_ERR_CAPACITY, "ls_sparse_ffn_step: selection capacity %d exceeds the cache (%lld rows)", sel->cap, (long long)L->cache_rows);
+    const double limit_s = g_opt_host_wait_ms.load(std::memory_order_relaxed) * 1e-3;
     LS_TRY(cache_rc(ls::cache_reserve_async(L->cache, miss_path, L->prio, L->F, sel->idx, sel->count, -1, 0, 0, sel->cap, nullptr, L->status, st,
-                                            &own_seq, g_err, g_launches)));
+                                            &own_seq, limit_s, g_err, g_launches)));
+    // (I/O lane: the stages are enqueued once the copies of this request have been issued; see cache_lane_wait)
+    if (miss_path == ls::MISS_PATH_LANE) LS_TRY(cache_rc(ls::cache_lane_wait(L->cache, own_seq, limit_s, g_err)));
     exec_idx = L->cache.d_exec_idx;
   }
   if (tr.exec_idx) {
@@ -924,7 +927,8 @@ int32_t ls_sparse_ffn_step(ls_layer* L, ls_layer* next, const float* d_x, float*
     if (!last && next->cache_rows > 0 && next != L) {
       // fetch rule: the first ceil(count (j+1)/(K+1)) ranks of C^(j) are admitted
       LS_TRY(cache_rc(ls::cache_reserve_async(next->cache, miss_path, next->prio, next->F, idx_out, cnt_out, 0, j + 1, K + 1, next->max_sel,
-                                              nullptr, next->status, st, nullptr, g_err, g_launches)));
+                                              nullptr, next->status, st, nullptr, g_opt_host_wait_ms.load(std::memory_order_relaxed) * 1e-3,
+                                              g_err, g_launches)));
     }
     return LS_OK;
   };
@@ -965,8 +969,8 @@ int32_t ls_cache_reserve(ls_layer* L, const ls_selection* want, int32_t admit_ra
   if (want->scores) LS_CUDA(cudaMemcpyAsync(L->prio, want->scores, (size_t)L->F * sizeof(double), cudaMemcpyDeviceToDevice, st));
   unsigned seq = 0;
   LS_TRY(cache_rc(ls::cache_reserve_async(L->cache, g_opt_miss_path.load(std::memory_order_relaxed), L->prio, L->F, want->idx, want->count,
-                                          admit_ranks < 0 ? -1 : admit_ranks, 0, 0, want->cap, d_protect_mask, L->status, st, &seq, g_err,
-                                          g_launches)));
+                                          admit_ranks < 0 ? -1 : admit_ranks, 0, 0, want->cap, d_protect_mask, L->status, st, &seq,
+                                          g_opt_host_wait_ms.load(std::memory_order_relaxed) * 1e-3, g_err, g_launches)));
   // this call reports the number of misses: it waits (bounded) for the decision, not for the copies
   return cache_rc(ls::cache_request_result(L->cache, seq, st, g_opt_host_wait_ms.load(std::memory_order_relaxed) * 1e-3, h_nmiss, g_err));
 }

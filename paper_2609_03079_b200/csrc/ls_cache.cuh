@@ -480,11 +480,31 @@ inline int32_t wait_event_bounded(cudaEvent_t ev, double limit_s, std::string& e
 
 // Enqueues a reserve: the decision kernel on `st`, then the hand-over of its miss list (see the top of this file).
 // Nothing here waits; the request's sequence number is returned for the kernels that will need its rows.
+// Host-side wait of the I/O-lane path (bounded): until the lane has taken over request `seq`.  A kernel must never spin on
+// the device for something only the host can provide while that host work is not yet secured (the launching thread may be
+// held up behind the spinning kernel), so in lane mode the calling thread (a) lets at most two requests of a layer be in
+// flight and (b) enqueues the stages of a step only once the copies of the step's own request have been issued.
+inline int32_t cache_lane_wait(CacheState& c, unsigned seq, double limit_s, std::string& err) {
+  const auto t0 = std::chrono::steady_clock::now();
+  for (long it = 0; *reinterpret_cast<const volatile unsigned*>(c.h_ack) < seq; ++it) {
+    if (std::chrono::duration<double>(std::chrono::steady_clock::now() - t0).count() > limit_s) {
+      err = "timed out waiting for the I/O lane to take over a cache request";
+      return -6;
+    }
+    if (it > 4000) std::this_thread::sleep_for(std::chrono::microseconds(20));
+  }
+  return 0;
+}
+
 inline int32_t cache_reserve_async(CacheState& c, int miss_path, const double* prio, int F, const int32_t* want, const int32_t* count_ptr,
                                    int admit_ranks, int admit_num, int admit_den, int cap, const uint32_t* protect, int* status,
-                                   cudaStream_t st, unsigned* seq_out, std::string& err, std::atomic<int64_t>& launches) {
-  const unsigned seq = ++c.seq_issued;
+                                   cudaStream_t st, unsigned* seq_out, double limit_s, std::string& err, std::atomic<int64_t>& launches) {
   const bool lane = miss_path == MISS_PATH_LANE;
+  if (lane && c.seq_issued >= 2) {
+    const int32_t rc = cache_lane_wait(c, c.seq_issued - 1, limit_s, err);
+    if (rc != 0) return rc;
+  }
+  const unsigned seq = ++c.seq_issued;
   const size_t list_ints = CACHE_HDR + 2 * (size_t)c.max_sel;
   int32_t* h_list = lane ? c.h_list_dev + (size_t)(seq & 1u) * list_ints : nullptr;
   int32_t* d_list = c.d_list + (size_t)(seq & 1u) * list_ints;
