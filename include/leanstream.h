@@ -306,6 +306,24 @@ int32_t ls_set_option(int32_t option, int32_t value);
 int32_t ls_timing_enable(int32_t on);
 int32_t ls_timing_read(int32_t kind, int64_t *launches, double *total_ms);
 
+/*
+ * Streaming controller (Section 3.2.3: state q_n = Q(R_n), coordination plan phi_n, finite-horizon stochastic dynamic
+ * programme solved offline, LUT[n, q] looked up at every layer boundary).  Host-side: every pointer is HOST memory.
+ * In this library a plan is an index into a caller-defined list of candidates (for instance stage counts n_chunks).
+ *
+ * ls_controller_quantize: q = Q(R): the remaining-load volume cut into n_states equal bins over [0, vmax] (0 = nothing
+ *   left; the last state collects everything from vmax on).  Returns the state, or LS_ERR_INVALID.
+ * ls_controller_build: Bellman backward recursion V_n^h(q) = min_a [ t_bar[n][q][a] + mean_s V_{n+1}^{h-1}(next_state[n][q][a][s]) ],
+ *   V^0 = 0 and V = 0 beyond the last layer.  t_bar [n_layers][n_states][n_plans]: profiled time of layer n from state q
+ *   under plan a (infinite or negative: plan not allowed in that state).  next_state [n_layers][n_states][n_plans][n_samples]:
+ *   the profiled samples of the next layer's state (negative entries are unused).  lut [n_layers][n_states] receives the
+ *   minimising plan at h = horizon (lowest index among equals, -1 when none is allowed); value (nullable, same shape)
+ *   receives V_n^horizon(q).  LS_ERR_INVALID on bad sizes or a sample outside [0, n_states).
+ */
+int32_t ls_controller_quantize(double remaining, double vmax, int32_t n_states);
+int32_t ls_controller_build(int32_t n_layers, int32_t n_states, int32_t n_plans, int32_t n_samples, int32_t horizon, const double *t_bar,
+                            const int32_t *next_state, int32_t *lut, double *value);
+
 /* Number of kernels launched by this library in the calling process since load (for launch accounting). */
 int64_t ls_kernel_launches(void);
 /* Copies the calling thread's last error text (NUL terminated, truncated to n) and returns its length. */

@@ -422,3 +422,55 @@ def lru_miss_ratio(trace: Sequence[Sequence[int]], capacity: int) -> float:
                 if len(lru) > capacity:
                     lru.popitem(last=False)
     return miss / max(1, tot)
+
+
+# ----------------------------------------------------------------------------------------------
+# Streaming controller (Section 3.2.3): finite-horizon stochastic dynamic programme -> LUT[n, q]
+# ----------------------------------------------------------------------------------------------
+def quantize_state(remaining: float, vmax: float, n_states: int) -> int:
+    """``q = Q(R)``: the remaining-load volume cut into ``n_states`` equal bins over ``[0, vmax]`` (state 0 = nothing
+    left to load, the last state collects everything from ``vmax`` on).  The paper says only that Q maps the volume to a
+    finite set of controller states (Section 3.2.3, item 1); equal bins are the reading taken."""
+    if n_states < 1 or not vmax > 0:
+        raise ValueError("n_states >= 1 and vmax > 0")
+    if not remaining > 0:
+        return 0
+    return min(n_states - 1, int(math.floor(remaining / vmax * n_states)))
+
+
+def controller_lut(t_bar: np.ndarray, next_state: np.ndarray, horizon: int):
+    """Bellman backward recursion of Section 3.2.3 (item 3).
+
+    ``t_bar[n, q, a]``: profiled execution time of layer ``n`` from state ``q`` under plan ``a`` (``T^I + T^II``);
+    ``inf`` or a negative value marks a plan that is not in ``Phi_n(q)``.  ``next_state[n, q, a, s]``: the profiled
+    samples of the next layer's state (the empirical transition distribution; a negative entry is an unused sample).
+    ``V_n^0 = 0``; ``V_n^h(q) = min_a [ t_bar[n,q,a] + mean_s V_{n+1}^{h-1}(next_state[n,q,a,s]) ]`` with ``V = 0`` beyond
+    the last layer; ``LUT[n, q]`` is the minimising plan at ``h = horizon`` (the lowest plan index among equals, -1 when no
+    plan is feasible).  Returns ``(lut, value)`` with ``value[n, q] = V_n^horizon(q)``.
+    """
+    t_bar = np.asarray(t_bar, dtype=np.float64)
+    nxt = np.asarray(next_state, dtype=np.int64)
+    N, Q, A = t_bar.shape
+    if horizon < 1:
+        raise ValueError("horizon >= 1")
+    V_prev = np.zeros((N + 1, Q))  # V^{h-1}; row N: beyond the last layer
+    lut = np.full((N, Q), -1, dtype=np.int64)
+    for h in range(1, horizon + 1):
+        V = np.zeros((N + 1, Q))
+        for n in range(N):
+            for q in range(Q):
+                best, best_a = math.inf, -1
+                for a in range(A):
+                    t = t_bar[n, q, a]
+                    if not (t >= 0.0) or math.isinf(t):
+                        continue
+                    samples = [int(v) for v in nxt[n, q, a] if v >= 0]
+                    future = 0.0 if (n + 1 >= N or not samples) else sum(V_prev[n + 1, v] for v in samples) / len(samples)
+                    cost = t + future
+                    if cost < best:
+                        best, best_a = cost, a
+                V[n, q] = best if best_a >= 0 else math.inf
+                if h == horizon:
+                    lut[n, q] = best_a
+        V_prev = V
+    return lut, V_prev[:N]

@@ -23,7 +23,7 @@ EXPORTS = [
     "ls_layer_create", "ls_layer_destroy", "ls_predict", "ls_sparse_ffn_step", "ls_cache_lookup", "ls_cache_reserve",
     "ls_cache_evict", "ls_cache_snapshot", "ls_cache_wait", "ls_cache_stats", "ls_layer_status", "ls_kernel_launches",
     "ls_last_error", "ls_version", "ls_timing_enable", "ls_timing_read", "ls_set_option", "ls_topk_select_static", "ls_stack_create",
-    "ls_stack_destroy", "ls_stack_decode",
+    "ls_stack_destroy", "ls_stack_decode", "ls_controller_quantize", "ls_controller_build",
 ]
 
 
@@ -97,6 +97,8 @@ def lib() -> C.CDLL:
         L.ls_stack_decode.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(ls_selection), C.c_int32, C.c_int32,
                                       C.POINTER(ls_selection), C.POINTER(ls_stack_trace), C.c_void_p]
         L.ls_topk_select_static.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.ls_controller_quantize.argtypes = [C.c_double, C.c_double, C.c_int32]
+        L.ls_controller_build.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.ls_timing_enable.argtypes = [C.c_int32]
         L.ls_timing_read.argtypes = [C.c_int32, C.POINTER(C.c_int64), C.POINTER(C.c_double)]
         L.ls_kernel_launches.restype = C.c_int64
@@ -388,3 +390,22 @@ def ls_stack_decode(stack: Stack, x: torch.Tensor, x_out: torch.Tensor, sel_firs
     assert x.dtype == torch.float32 and x.is_cuda and x.is_contiguous() and x_out.is_contiguous()
     _check(lib().ls_stack_decode(stack.handle, x.data_ptr(), x_out.data_ptr(), C.byref(sel_first.c), n_chunks, k_next,
                                  C.byref(sel_out.c), None if trace is None else C.byref(trace.c), _stream(stream)))
+
+
+def ls_controller_quantize(remaining: float, vmax: float, n_states: int) -> int:
+    rc = lib().ls_controller_quantize(remaining, vmax, n_states)
+    if rc < 0:
+        _check(rc)
+    return rc
+
+
+def ls_controller_build(t_bar: np.ndarray, next_state: np.ndarray, horizon: int):
+    """(lut [n_layers, n_states] int32, value [n_layers, n_states]) from host arrays t_bar [N, Q, A] and next_state [N, Q, A, S]."""
+    t = np.ascontiguousarray(t_bar, dtype=np.float64)
+    ns = np.ascontiguousarray(next_state, dtype=np.int32)
+    N, Q, A = t.shape
+    S = ns.shape[3] if ns.ndim == 4 else 0
+    lut = np.full((N, Q), -2, dtype=np.int32)
+    val = np.zeros((N, Q), dtype=np.float64)
+    _check(lib().ls_controller_build(N, Q, A, S, horizon, t.ctypes.data, ns.ctypes.data if S else None, lut.ctypes.data, val.ctypes.data))
+    return lut, val

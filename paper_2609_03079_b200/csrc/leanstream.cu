@@ -4,7 +4,9 @@
 #include <atomic>
 #include <cstdarg>
 #include <cstdio>
+#include <cmath>
 #include <cstring>
+#include <limits>
 #include <mutex>
 #include <new>
 #include <string>
@@ -751,6 +753,53 @@ int32_t ls_topk_select_static(const double* d_scores, int32_t n, int32_t k, int3
   return LS_OK;
 }
 
+
+// ---- streaming controller (host side) -------------------------------------------------------------------------------
+int32_t ls_controller_quantize(double remaining, double vmax, int32_t n_states) {
+  if (n_states < 1 || !(vmax > 0.0)) return fail(LS_ERR_INVALID, "ls_controller_quantize: n_states >= 1 and vmax > 0 are required");
+  if (!(remaining > 0.0)) return 0;
+  const double b = floor(remaining / vmax * (double)n_states);
+  return b >= (double)(n_states - 1) ? n_states - 1 : (int32_t)b;
+}
+
+int32_t ls_controller_build(int32_t N, int32_t Q, int32_t A, int32_t S, int32_t H, const double* t_bar, const int32_t* next_state,
+                            int32_t* lut, double* value) {
+  if (N < 1 || Q < 1 || A < 1 || S < 0 || H < 1 || !t_bar || !lut || (S > 0 && !next_state))
+    return fail(LS_ERR_INVALID, "ls_controller_build: bad argument");
+  for (size_t i = 0; S > 0 && i < (size_t)N * Q * A * S; ++i)
+    if (next_state[i] >= Q) return fail(LS_ERR_INVALID, "ls_controller_build: state sample %d outside [0, %d)", next_state[i], Q);
+  const double INF = std::numeric_limits<double>::infinity();
+  std::vector<double> prev((size_t)(N + 1) * Q, 0.0), cur((size_t)(N + 1) * Q, 0.0);
+  for (int h = 1; h <= H; ++h) {
+    std::fill(cur.begin(), cur.end(), 0.0);
+    for (int n = 0; n < N; ++n)
+      for (int q = 0; q < Q; ++q) {
+        double best = INF;
+        int best_a = -1;
+        for (int a = 0; a < A; ++a) {
+          const double t = t_bar[((size_t)n * Q + q) * A + a];
+          if (!(t >= 0.0) || t == INF) continue;
+          double future = 0.0;
+          if (n + 1 < N && S > 0) {
+            const int32_t* smp = next_state + (((size_t)n * Q + q) * A + a) * S;
+            double sum = 0.0;
+            int cnt = 0;
+            for (int s = 0; s < S; ++s)
+              if (smp[s] >= 0) { sum += prev[(size_t)(n + 1) * Q + smp[s]]; ++cnt; }
+            future = cnt > 0 ? sum / cnt : 0.0;
+          }
+          const double cost = t + future;
+          if (cost < best) { best = cost; best_a = a; }
+        }
+        cur[(size_t)n * Q + q] = best_a >= 0 ? best : INF;
+        if (h == H) lut[(size_t)n * Q + q] = best_a;
+      }
+    prev.swap(cur);
+  }
+  if (value)
+    for (size_t i = 0; i < (size_t)N * Q; ++i) value[i] = prev[i];
+  return LS_OK;
+}
 
 int32_t ls_set_option(int32_t option, int32_t value) {
   if (option == LS_OPT_FUSED) {
