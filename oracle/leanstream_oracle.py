@@ -474,3 +474,63 @@ def controller_lut(t_bar: np.ndarray, next_state: np.ndarray, horizon: int):
                     lut[n, q] = best_a
         V_prev = V
     return lut, V_prev[:N]
+
+
+# ----------------------------------------------------------------------------------------------
+# Stacked learnable hashing predictor, inference only (Section 3.3.1 - 3.3.3)
+# ----------------------------------------------------------------------------------------------
+def sign_pm(v: np.ndarray) -> np.ndarray:
+    """Elementwise sign with values in {-1, +1}; zero counts as +1 (the paper's sign() leaves 0 open)."""
+    return np.where(np.asarray(v) >= 0, 1, -1).astype(np.int64)
+
+
+def hash_index(code: Sequence[int]) -> int:
+    """``phi_tau``: a code in {-1,+1}^tau to its bucket number.  The convention is the one the structured matrix Z of
+    Section 3.3.2 fixes (for tau = 3 its rows run (-1,-1,-1), (-1,-1,+1), (-1,+1,-1), ..., (+1,+1,+1)): -1 is bit 0,
+    +1 is bit 1, and the FIRST component is the most significant bit."""
+    idx = 0
+    for c in code:
+        idx = (idx << 1) | (1 if int(c) > 0 else 0)
+    return idx
+
+
+@dataclass
+class HashPredictor:
+    """Operands of a stack of learnable hashing layers (Eq. ``y_k = T_k[phi_tau(sign(x_k (*) W_k))]``).
+
+    ``pca`` [d_model, r]: the PCA projection applied to the feature first (Section 3.3.3).  ``w1`` [r, tau]: real
+    hyperplanes of the first layer.  ``w[k]`` [d, tau] in {-1,+1}: binary hyperplanes of layer k+2.  ``t[k]`` [2^tau, d]
+    in {-1,+1}: the bucket features of layer k+1.  ``codes`` [F, d] in {-1,+1}: one binary code per hidden neuron; a
+    neuron's priority is the inner product of the last layer's output with its code (an XNOR-and-bitcount product like the
+    inner layers', Section 3.3.1).  The paper does not spell out the output stage for the neuron-activation task; this is
+    the reading taken (it reproduces the predictor size the paper reports: d_ff x d bits per block)."""
+
+    pca: np.ndarray
+    w1: np.ndarray
+    w: List[np.ndarray]
+    t: List[np.ndarray]
+    codes: np.ndarray
+
+    @property
+    def n_layers(self) -> int:
+        return len(self.t)
+
+
+def hash_predictor_trace(P: HashPredictor, v: np.ndarray):
+    """Bucket numbers of every layer and the last layer's output for the feature ``v`` (un-normalised: a hyperplane hash
+    does not see a positive scale, so the norm of Section 2.1 drops out).  Returns ``(indices, y_last, first_dots)``."""
+    z = np.asarray(v, dtype=np.float64) @ P.pca
+    dots = z @ P.w1
+    idx = [hash_index(sign_pm(dots))]
+    y = P.t[0][idx[0]].astype(np.int64)
+    for k, W in enumerate(P.w):
+        code = sign_pm(y @ W.astype(np.int64))  # XNOR-and-bitcount product: an integer inner product of sign vectors
+        idx.append(hash_index(code))
+        y = P.t[k + 1][idx[-1]].astype(np.int64)
+    return idx, y, dots
+
+
+def hash_predictor_scores(P: HashPredictor, v: np.ndarray) -> np.ndarray:
+    """Priority of every neuron: inner product of the last layer's output with the neuron's code (integers, as fp64)."""
+    _, y, _ = hash_predictor_trace(P, v)
+    return (P.codes.astype(np.int64) @ y).astype(np.float64)
