@@ -42,6 +42,7 @@ extern "C" {
 #define LS_ERR_INTERNAL (-7) /* a kernel's self-check failed (reported through ls_layer_status) */
 
 #define LS_ACT_RELU 0
+#define LS_ACT_SILU 1 /* the activation Eq. 1 prints: g * sigmoid(g); no exact zeros, so every selected neuron needs all its rows */
 #define LS_WDTYPE_BF16 0
 #define LS_WDTYPE_FP16 1
 #define LS_NORM_RMS 0
@@ -51,8 +52,8 @@ typedef struct ls_layer ls_layer;
 
 /*
  * Problem statement of one FFN layer: the operands of Eq. 1 plus the layer's neuron predictor.
- *   act(h W_gate) * (h W_up) W_down with act = ReLU (the sparsity source of Section 2.1); gated = 0 gives the
- *   two-matrix form act(h W_fc1 + b) W_fc2 + b_down.  h = rmsnorm(x) without gain (norm = LS_NORM_RMS) or h = x.
+ *   act(h W_gate) * (h W_up) W_down with act = ReLU (the sparsity source of Section 2.1) or SiLU (as Eq. 1 prints it);
+ *   gated = 0 gives the two-matrix form act(h W_fc1 + b) W_fc2 + b_down.  h = rmsnorm(x) without gain (norm = LS_NORM_RMS) or h = x.
  *   Predictor (Section 3.3.3: projection of the feature, then the scorer): s = pred_b^T (pred_a^T h) + pred_c.
  * All weight matrices are 16-bit (wdtype), row-major, HOST memory, copied by ls_layer_create():
  *   w_gate, w_up, w_down_t: [d_ff][d_model] (w_down_t is neuron-major, i.e. the transposed down projection);
@@ -254,7 +255,8 @@ int32_t ls_stack_decode(ls_stack *stack, const float *d_x, float *d_x_out, const
  *   1 <= n <= LS_STATIC_TOPK_MAX_N and 0 <= k <= n, otherwise LS_ERR_INVALID with an explanatory ls_last_error().
  *
  * The first call on a device looks up the array's device address (cudaGetSymbolAddress) and opts the kernel in to its
- * shared memory; make that first call outside any stream capture, with the target device current.  All calls on a
+ * shared memory; make that first call outside any stream capture.  Every call runs on the device that owns d_scores
+ * (d_idx, d_mask and d_count must live there too), whatever device is current.  All calls on a
  * device share the one array: two calls that overlap on the GPU (different streams) race on it, so order them; the
  * array keeps whatever the last call left there, which is harmless because every entry is written before it is read.
  */
@@ -305,6 +307,36 @@ int32_t ls_set_option(int32_t option, int32_t value);
 #define LS_TIMED_STACK 4   /* the whole-token kernel of ls_stack_decode */
 int32_t ls_timing_enable(int32_t on);
 int32_t ls_timing_read(int32_t kind, int64_t *launches, double *total_ms);
+
+/*
+ * Stacked learnable hashing predictor, inference (Section 3.3.1 - 3.3.3): an alternative to the linear predictor of
+ * ls_layer_desc for ranking a layer's neurons.  Layer k computes y_k = T_k[phi_tau(sign(x_k (*) W_k))]: the first layer
+ * hashes the PCA-projected feature with real hyperplanes (decided in fp64), the others are binary (XNOR and bitcount); a
+ * neuron's priority is the XNOR-and-bitcount inner product of the last layer's output with the neuron's binary code.
+ * Sign vectors are packed one bit per component: +1 -> 1, -1 -> 0, component c at bit (c & 31) of word (c >> 5).
+ * phi_tau takes the FIRST component of a code as the most significant bit (the convention of the structured matrix Z of
+ * Section 3.3.2); sign(0) = +1.
+ *   pca     HOST [d_model][rank] 16-bit (wdtype)      w1      HOST float [rank][tau]
+ *   w       HOST uint32 [n_layers-1][tau][d_code/32]   tables  HOST uint32 [n_layers][2^tau][d_code/32]
+ *   codes   HOST uint32 [d_ff][d_code/32]
+ *   d_model, rank multiples of 8; 1 <= tau <= 16; d_code a multiple of 32, at most 1024; 1 <= n_layers <= 16.
+ * ls_hash_predict: scores every neuron from d_feature [d_model] (float, un-normalised: a hyperplane hash does not see a
+ *   positive scale) and selects the k best under the same total order as ls_predict; `out` as there (scores are the
+ *   integer priorities as fp64).  d_layer_idx (nullable, DEVICE int32 [n_layers]) receives every layer's bucket number.
+ */
+typedef struct ls_hash_predictor ls_hash_predictor;
+typedef struct {
+  uint32_t struct_size;
+  int32_t device;
+  int32_t d_model, rank, tau, d_code, n_layers, d_ff, wdtype;
+  const void *pca;
+  const float *w1;
+  const uint32_t *w, *tables, *codes;
+} ls_hash_predictor_desc;
+int32_t ls_hash_predictor_create(const ls_hash_predictor_desc *desc, ls_hash_predictor **out);
+int32_t ls_hash_predictor_destroy(ls_hash_predictor *pred);
+int32_t ls_hash_predict(ls_hash_predictor *pred, const float *d_feature, int32_t k, ls_selection *out, int32_t *d_layer_idx,
+                        void *stream);
 
 /*
  * Streaming controller (Section 3.2.3: state q_n = Q(R_n), coordination plan phi_n, finite-horizon stochastic dynamic

@@ -89,6 +89,7 @@ class OracleLayer:
             pred_bt=np.ascontiguousarray(decode16(la.pred_b, dt).T),
             pred_c=np.zeros(F) if la.pred_c is None else la.pred_c.astype(np.float64),
             eps=float(la.norm_eps),
+            act=SILU if getattr(la, "act", "relu") == "silu" else RELU,
         )
 
 

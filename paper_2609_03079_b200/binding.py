@@ -15,7 +15,7 @@ import torch
 from . import build as _build
 
 LS_OK, LS_ERR_INVALID, LS_ERR_NOMEM, LS_ERR_CUDA, LS_ERR_STATE, LS_ERR_CAPACITY, LS_ERR_TIMEOUT, LS_ERR_INTERNAL = 0, -1, -2, -3, -4, -5, -6, -7
-LS_ACT_RELU = 0
+LS_ACT_RELU, LS_ACT_SILU = 0, 1
 LS_WDTYPE_BF16, LS_WDTYPE_FP16 = 0, 1
 LS_NORM_RMS, LS_NORM_NONE = 0, 1
 
@@ -23,7 +23,8 @@ EXPORTS = [
     "ls_layer_create", "ls_layer_destroy", "ls_predict", "ls_sparse_ffn_step", "ls_cache_lookup", "ls_cache_reserve",
     "ls_cache_evict", "ls_cache_snapshot", "ls_cache_wait", "ls_cache_stats", "ls_layer_status", "ls_kernel_launches",
     "ls_last_error", "ls_version", "ls_timing_enable", "ls_timing_read", "ls_set_option", "ls_topk_select_static", "ls_stack_create",
-    "ls_stack_destroy", "ls_stack_decode", "ls_controller_quantize", "ls_controller_build",
+    "ls_stack_destroy", "ls_stack_decode", "ls_controller_quantize", "ls_controller_build", "ls_hash_predictor_create",
+    "ls_hash_predictor_destroy", "ls_hash_predict",
 ]
 
 
@@ -58,6 +59,12 @@ class ls_stack_trace(C.Structure):
 
 
 LS_STACK_NSTAMP = 12
+
+
+class ls_hash_predictor_desc(C.Structure):
+    _fields_ = [("struct_size", C.c_uint32), ("device", C.c_int32), ("d_model", C.c_int32), ("rank", C.c_int32), ("tau", C.c_int32),
+                ("d_code", C.c_int32), ("n_layers", C.c_int32), ("d_ff", C.c_int32), ("wdtype", C.c_int32), ("pca", C.c_void_p),
+                ("w1", C.c_void_p), ("w", C.c_void_p), ("tables", C.c_void_p), ("codes", C.c_void_p)]
 
 
 class ls_cache_stats_t(C.Structure):
@@ -97,6 +104,9 @@ def lib() -> C.CDLL:
         L.ls_stack_decode.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(ls_selection), C.c_int32, C.c_int32,
                                       C.POINTER(ls_selection), C.POINTER(ls_stack_trace), C.c_void_p]
         L.ls_topk_select_static.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.ls_hash_predictor_create.argtypes = [C.POINTER(ls_hash_predictor_desc), C.POINTER(C.c_void_p)]
+        L.ls_hash_predictor_destroy.argtypes = [C.c_void_p]
+        L.ls_hash_predict.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(ls_selection), C.c_void_p, C.c_void_p]
         L.ls_controller_quantize.argtypes = [C.c_double, C.c_double, C.c_int32]
         L.ls_controller_build.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.ls_timing_enable.argtypes = [C.c_int32]
@@ -219,7 +229,7 @@ def ls_layer_create(arrays, device: int = 0, cache_rows: int = 0, max_batch: int
     d.device = device
     d.d_model, d.d_ff = arrays.d_model, arrays.d_ff
     d.gated = 1 if arrays.gated else 0
-    d.act = LS_ACT_RELU
+    d.act = LS_ACT_SILU if getattr(arrays, "act", "relu") == "silu" else LS_ACT_RELU
     d.wdtype = LS_WDTYPE_BF16 if arrays.wdtype == "bf16" else LS_WDTYPE_FP16
     d.norm = norm
     d.norm_eps = float(arrays.norm_eps)
@@ -409,3 +419,45 @@ def ls_controller_build(t_bar: np.ndarray, next_state: np.ndarray, horizon: int)
     val = np.zeros((N, Q), dtype=np.float64)
     _check(lib().ls_controller_build(N, Q, A, S, horizon, t.ctypes.data, ns.ctypes.data if S else None, lut.ctypes.data, val.ctypes.data))
     return lut, val
+
+
+class HashPredictor:
+    """Owner of one ``ls_hash_predictor*`` handle."""
+
+    def __init__(self, handle: int, d_ff: int, n_layers: int, device: int):
+        self.handle, self.d_ff, self.n_layers, self.device = handle, d_ff, n_layers, device
+
+    def close(self) -> None:
+        if self.handle:
+            lib().ls_hash_predictor_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def ls_hash_predictor_create(arrays, device: int = 0) -> HashPredictor:
+    """Create from host arrays (attributes as produced by ``workload.make_hash_predictor``: packed sign bits)."""
+    keep = [np.ascontiguousarray(arrays.pca), np.ascontiguousarray(arrays.w1, dtype=np.float32), np.ascontiguousarray(arrays.w_bits, dtype=np.uint32),
+            np.ascontiguousarray(arrays.t_bits, dtype=np.uint32), np.ascontiguousarray(arrays.code_bits, dtype=np.uint32)]
+    d = ls_hash_predictor_desc()
+    d.struct_size = C.sizeof(ls_hash_predictor_desc)
+    d.device = device
+    d.d_model, d.rank, d.tau, d.d_code, d.n_layers, d.d_ff = arrays.d_model, arrays.rank, arrays.tau, arrays.d_code, arrays.n_layers, arrays.d_ff
+    d.wdtype = LS_WDTYPE_BF16 if arrays.wdtype == "bf16" else LS_WDTYPE_FP16
+    d.pca, d.w1 = keep[0].ctypes.data, keep[1].ctypes.data
+    d.w = keep[2].ctypes.data if arrays.n_layers > 1 else None
+    d.tables, d.codes = keep[3].ctypes.data, keep[4].ctypes.data
+    out = C.c_void_p()
+    _check(lib().ls_hash_predictor_create(C.byref(d), C.byref(out)))
+    return HashPredictor(out.value, arrays.d_ff, arrays.n_layers, device)
+
+
+def ls_hash_predict(pred: HashPredictor, feature: torch.Tensor, k: int, out: Selection, layer_idx: Optional[torch.Tensor] = None,
+                    stream=None) -> Selection:
+    assert feature.dtype == torch.float32 and feature.is_cuda and feature.is_contiguous()
+    _check(lib().ls_hash_predict(pred.handle, feature.data_ptr(), k, C.byref(out.c), _ptr(layer_idx), _stream(stream)))
+    return out

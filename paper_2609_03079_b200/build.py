@@ -11,7 +11,7 @@ ROOT = os.path.dirname(PKG_DIR)
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libleanstream.so")
 SOURCES = ["leanstream.cu"]
-HEADERS = ["ls_common.cuh", "ls_topk.cuh", "ls_kernels.cuh", "ls_cache.cuh", "ls_token.cuh"]
+HEADERS = ["ls_common.cuh", "ls_topk.cuh", "ls_kernels.cuh", "ls_cache.cuh", "ls_token.cuh", "ls_hash.cuh"]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -13,6 +13,7 @@
 #include <vector>
 
 #include "ls_cache.cuh"
+#include "ls_hash.cuh"
 #include "ls_kernels.cuh"
 #include "ls_token.cuh"
 
@@ -134,6 +135,22 @@ struct ls_layer {
   double* wt_range = nullptr;  // [2] {hi, scale} of the score bins used when a fused step refines THIS layer (carried from call to call)
 
   ls::CacheState cache;  // residency tables, pinned backing store, copy stream
+};
+
+struct ls_hash_predictor {
+  int device = 0, d = 0, r = 0, tau = 0, words = 0, n_layers = 0, F = 0, wd = 0, sm_count = 148;
+  uint16_t* pca_t = nullptr;   // [r][d]
+  float* w1 = nullptr;         // [r][tau]
+  uint32_t* w = nullptr;       // [n_layers - 1][tau][words]
+  uint32_t* tables = nullptr;  // [n_layers][2^tau][words]
+  uint32_t* codes = nullptr;   // [F][words]
+  double* z = nullptr;         // [r]
+  double* sumsq = nullptr;     // [1]
+  uint32_t* y = nullptr;       // [words]
+  double* scores = nullptr;    // [F]
+  unsigned long long* cand_key = nullptr;  // [F]
+  int32_t* cand_idx = nullptr;             // [F]
+  int* status = nullptr;
 };
 
 struct ls_stack {
@@ -438,7 +455,7 @@ int32_t fused_step(ls_layer* L, ls_layer* next, const float* d_x, float* d_x_out
   LS_TRY(device_scratch(L->device, &D));
   ls::WtLayer& a = c.one;
   a.bundles = L->bundles; a.b_gate = L->b_gate; a.b_down = L->b_down;
-  a.n_mat = L->n_mat; a.F = L->F; a.norm = L->norm; a.eps = L->eps;
+  a.n_mat = L->n_mat; a.F = L->F; a.norm = L->norm; a.act = L->act; a.eps = L->eps;
   a.At_sl = next->pred_at_sl; a.Bt_pad = next->pred_bt_pad; a.pc = next->pred_c;
   a.r = next->r; a.Fn = next->F; a.norm_n = next->norm; a.eps_n = next->eps;
   a.range = next->wt_range;
@@ -508,7 +525,7 @@ int32_t launch_stage(ls_layer* L, int B, const int32_t* exec_idx, const int32_t*
     KernelTimer timer(LS_TIMED_GATEUP, st);
     const int grid = std::max(1, std::min((per_stage + 7) / 8, L->sm_count * 4));
     const size_t sm = (size_t)B * d * sizeof(float);
-    ls::ls_gateup_kernel<WD, BT><<<grid, 256, sm, st>>>(L->bundles, L->n_mat, L->gated, slot_of, L->b_gate, L->xin, B, d, L->norm,
+    ls::ls_gateup_kernel<WD, BT><<<grid, 256, sm, st>>>(L->bundles, L->n_mat, L->gated, L->act, slot_of, L->b_gate, L->xin, B, d, L->norm,
                                                         L->eps, exec_idx, count_ptr, K, c, L->F, L->actv, L->max_sel, L->survive,
                                                         L->status, need_seq ? L->cache.d_landed : nullptr, need_seq,
                                                         need_seq ? ls::cache_list_header(L->cache, need_seq) : nullptr);
@@ -670,7 +687,7 @@ int32_t ls_stack_create(ls_layer* const* layers, int32_t n_layers, ls_stack** ou
     ls_layer* next = layers[n + 1 < n_layers ? n + 1 : n];  // the last layer refines a weight-tied copy of itself
     ls::WtLayer& a = h[n];
     a.bundles = L->bundles; a.b_gate = L->b_gate; a.b_down = L->b_down;
-    a.n_mat = L->n_mat; a.F = L->F; a.norm = L->norm; a.eps = L->eps;
+    a.n_mat = L->n_mat; a.F = L->F; a.norm = L->norm; a.act = L->act; a.eps = L->eps;
     a.At_sl = next->pred_at_sl; a.Bt_pad = next->pred_bt_pad; a.pc = next->pred_c;
     a.r = next->r; a.Fn = next->F; a.norm_n = next->norm; a.eps_n = next->eps;
     a.range = S->ranges + 2 * n;
@@ -742,9 +759,13 @@ int32_t ls_topk_select_static(const double* d_scores, int32_t n, int32_t k, int3
     return fail(LS_ERR_INVALID, "ls_topk_select_static: n = %d is outside [1, %d] (the static scratch holds at most %d candidates)", n,
                 LS_STATIC_TOPK_MAX_N, LS_STATIC_TOPK_MAX_N);
   if (k < 0 || k > n) return fail(LS_ERR_INVALID, "ls_topk_select_static: k = %d is outside [0, n = %d]", k, n);
+  // the launch goes to the device that owns the scores (its copy of the static scratch), whatever device is current
   int dev = -1;
-  LS_CUDA(cudaGetDevice(&dev));
+  cudaPointerAttributes at{};
+  if (cudaPointerGetAttributes(&at, d_scores) == cudaSuccess && at.type == cudaMemoryTypeDevice) dev = at.device;
+  else { cudaGetLastError(); LS_CUDA(cudaGetDevice(&dev)); }
   if (dev < 0 || dev >= 64) return fail(LS_ERR_INVALID, "ls_topk_select_static: device ordinal %d not supported", dev);
+  DeviceGuard guard(dev);
   unsigned char* scratch = nullptr;
   LS_TRY(static_topk_setup(dev, &scratch));
   ls_topk_static_kernel<<<1, ls::TK_THREADS, ls::topk_kernel_smem(n), (cudaStream_t)stream>>>(d_scores, n, k, d_idx, d_mask, d_count,
@@ -753,6 +774,87 @@ int32_t ls_topk_select_static(const double* d_scores, int32_t n, int32_t k, int3
   return LS_OK;
 }
 
+
+// ---- stacked hashing predictor ----------------------------------------------------------------------------------------
+int32_t ls_hash_predictor_destroy(ls_hash_predictor* P) {
+  if (!P) return LS_OK;
+  DeviceGuard guard(P->device);
+  cudaDeviceSynchronize();
+  cudaFree(P->pca_t); cudaFree(P->w1); cudaFree(P->w); cudaFree(P->tables); cudaFree(P->codes); cudaFree(P->z); cudaFree(P->sumsq);
+  cudaFree(P->y); cudaFree(P->scores); cudaFree(P->cand_key); cudaFree(P->cand_idx); cudaFree(P->status);
+  delete P;
+  return LS_OK;
+}
+
+int32_t ls_hash_predictor_create(const ls_hash_predictor_desc* D, ls_hash_predictor** out) {
+  if (out) *out = nullptr;
+  if (!D || !out) return fail(LS_ERR_INVALID, "ls_hash_predictor_create: NULL argument");
+  if (D->struct_size != sizeof(ls_hash_predictor_desc))
+    return fail(LS_ERR_INVALID, "ls_hash_predictor_create: struct_size %u, expected %zu", D->struct_size, sizeof(ls_hash_predictor_desc));
+  if (D->d_model < 8 || D->d_model % 8 || D->d_model > 16384 || D->rank < 8 || D->rank % 8 || D->rank > 1024)
+    return fail(LS_ERR_INVALID, "ls_hash_predictor_create: d_model, rank must be multiples of 8 within [8, 16384] / [8, 1024]");
+  if (D->tau < 1 || D->tau > ls::HASH_MAX_TAU || D->d_code < 32 || D->d_code % 32 || D->d_code > 32 * ls::HASH_MAX_WORDS ||
+      D->n_layers < 1 || D->n_layers > ls::HASH_MAX_LAYERS || D->d_ff < 1 || D->d_ff > 32768)
+    return fail(LS_ERR_INVALID, "ls_hash_predictor_create: tau, d_code, n_layers or d_ff out of range");
+  if (D->wdtype != LS_WDTYPE_BF16 && D->wdtype != LS_WDTYPE_FP16) return fail(LS_ERR_INVALID, "unknown wdtype");
+  if (!D->pca || !D->w1 || !D->tables || !D->codes || (D->n_layers > 1 && !D->w)) return fail(LS_ERR_INVALID, "ls_hash_predictor_create: missing table");
+  int ndev = 0;
+  LS_CUDA(cudaGetDeviceCount(&ndev));
+  if (D->device < 0 || D->device >= ndev) return fail(LS_ERR_INVALID, "device %d out of range", D->device);
+  DeviceGuard guard(D->device);
+  ls_hash_predictor* P = new (std::nothrow) ls_hash_predictor();
+  if (!P) return fail(LS_ERR_NOMEM, "host allocation");
+  P->device = D->device; P->d = D->d_model; P->r = D->rank; P->tau = D->tau; P->words = D->d_code / 32; P->n_layers = D->n_layers;
+  P->F = D->d_ff; P->wd = D->wdtype;
+  cudaDeviceProp prop;
+  int32_t rc = LS_OK;
+  auto up = [&](auto** dst, const void* src, size_t n) -> int32_t {
+    LS_TRY(dalloc(dst, n));
+    if (src && n) LS_CUDA(cudaMemcpy(*dst, src, n * sizeof(**dst), cudaMemcpyHostToDevice));
+    return LS_OK;
+  };
+  const size_t W = P->words, nb = (size_t)1 << P->tau;
+  if (cudaGetDeviceProperties(&prop, D->device) == cudaSuccess) P->sm_count = prop.multiProcessorCount;
+  if ((rc = upload_transposed16(&P->pca_t, D->pca, P->d, P->r)) != LS_OK || (rc = up(&P->w1, D->w1, (size_t)P->r * P->tau)) != LS_OK ||
+      (rc = up(&P->w, D->w, (size_t)(P->n_layers - 1) * P->tau * W)) != LS_OK || (rc = up(&P->tables, D->tables, (size_t)P->n_layers * nb * W)) != LS_OK ||
+      (rc = up(&P->codes, D->codes, (size_t)P->F * W)) != LS_OK || (rc = dalloc(&P->z, (size_t)P->r)) != LS_OK ||
+      (rc = dalloc(&P->sumsq, 1)) != LS_OK || (rc = dalloc(&P->y, W)) != LS_OK || (rc = dalloc(&P->scores, (size_t)P->F)) != LS_OK ||
+      (rc = dalloc(&P->cand_key, (size_t)P->F)) != LS_OK || (rc = dalloc(&P->cand_idx, (size_t)P->F)) != LS_OK ||
+      (rc = dalloc(&P->status, 1)) != LS_OK) {
+    const std::string keep = g_err;
+    ls_hash_predictor_destroy(P);
+    g_err = keep;
+    return rc;
+  }
+  cudaMemset(P->status, 0, sizeof(int));
+  cudaFuncSetAttribute(ls::ls_topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  LS_CUDA(cudaDeviceSynchronize());
+  *out = P;
+  return LS_OK;
+}
+
+int32_t ls_hash_predict(ls_hash_predictor* P, const float* d_feature, int32_t k, ls_selection* out, int32_t* d_layer_idx, void* stream) {
+  if (!P || !d_feature || !out || !out->idx || !out->count) return fail(LS_ERR_INVALID, "ls_hash_predict: predictor, feature, out->idx and out->count are required");
+  if (k < 0 || k > P->F) return fail(LS_ERR_INVALID, "ls_hash_predict: k %d outside [0, d_ff]", k);
+  if (out->cap < k) return fail(LS_ERR_INVALID, "ls_hash_predict: out->cap %d < k %d", out->cap, k);
+  DeviceGuard guard(P->device);
+  cudaStream_t st = (cudaStream_t)stream;
+  KernelTimer timer(LS_TIMED_PREDICT, st);
+  {
+    const int wpb = 8, grid = (P->r + wpb - 1) / wpb;
+    if (P->wd == 0) ls::ls_latent_kernel<0><<<grid, 256, 0, st>>>(P->pca_t, d_feature, P->d, P->r, 1, P->z, P->sumsq);
+    else ls::ls_latent_kernel<1><<<grid, 256, 0, st>>>(P->pca_t, d_feature, P->d, P->r, 1, P->z, P->sumsq);
+    LS_LAUNCHED();
+  }
+  ls::ls_hash_layers_kernel<<<1, 256, 0, st>>>(P->z, P->w1, P->r, P->tau, P->words, P->n_layers, P->w, P->tables, P->y, d_layer_idx);
+  LS_LAUNCHED();
+  ls::ls_hash_scores_kernel<<<std::min((P->F + 255) / 256, P->sm_count * 4), 256, 0, st>>>(P->y, P->codes, P->words, P->F, P->scores, out->scores);
+  LS_LAUNCHED();
+  ls::ls_topk_kernel<<<1, ls::TK_THREADS, ls::topk_kernel_smem(P->F), st>>>(P->scores, P->F, k, nullptr, out->idx, out->cap, out->mask, 0, out->count,
+                                                                          P->cand_key, P->cand_idx, P->status);
+  LS_LAUNCHED();
+  return LS_OK;
+}
 
 // ---- streaming controller (host side) -------------------------------------------------------------------------------
 int32_t ls_controller_quantize(double remaining, double vmax, int32_t n_states) {
@@ -853,7 +955,7 @@ int32_t ls_layer_create(const ls_layer_desc* D, ls_layer** out) {
   if (D->d_model < 8 || D->d_model % 8 || D->d_model > 16384) return fail(LS_ERR_INVALID, "d_model must be a multiple of 8 in [8, 16384]");
   if (D->d_ff < 1 || D->d_ff > 32768) return fail(LS_ERR_INVALID, "d_ff must be in [1, 32768]");
   if (D->pred_rank < 8 || D->pred_rank % 8 || D->pred_rank > 1024) return fail(LS_ERR_INVALID, "pred_rank must be a multiple of 8 in [8, 1024]");
-  if (D->act != LS_ACT_RELU) return fail(LS_ERR_INVALID, "only LS_ACT_RELU is implemented");
+  if (D->act != LS_ACT_RELU && D->act != LS_ACT_SILU) return fail(LS_ERR_INVALID, "act must be LS_ACT_RELU or LS_ACT_SILU");
   if (D->wdtype != LS_WDTYPE_BF16 && D->wdtype != LS_WDTYPE_FP16) return fail(LS_ERR_INVALID, "unknown wdtype");
   if (D->norm != LS_NORM_RMS && D->norm != LS_NORM_NONE) return fail(LS_ERR_INVALID, "unknown norm");
   if (!D->w_gate || !D->w_down_t || (D->gated && !D->w_up) || !D->pred_a || !D->pred_b)

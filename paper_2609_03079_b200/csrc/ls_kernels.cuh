@@ -111,11 +111,11 @@ __global__ void __launch_bounds__(256) ls_scores_kernel(const uint16_t* __restri
 // ------------------------------------------------------------------------------------------------------------------
 // Stage c, part 1: gate/up gather-GEMV and activation for the neurons of the stage (Eq. 1, the bracket).
 // One warp per neuron, 128-bit row loads, fp32 accumulation, warp-shuffle reduction.
-// a[b][p] = relu(inv_rms_b * (w_gate[i] . x_b) + b_i) * (inv_rms_b * (w_up[i] . x_b)), p = rank position of neuron i.
+// a[b][p] = act(inv_rms_b * (w_gate[i] . x_b) + b_i) * (inv_rms_b * (w_up[i] . x_b)), p = rank position of neuron i.
 // ------------------------------------------------------------------------------------------------------------------
 template <int WD, int BT>
 __global__ void __launch_bounds__(256)
-    ls_gateup_kernel(const uint16_t* __restrict__ bundles, int n_mat, int gated, const int32_t* __restrict__ slot_of,
+    ls_gateup_kernel(const uint16_t* __restrict__ bundles, int n_mat, int gated, int act_kind, const int32_t* __restrict__ slot_of,
                      const float* __restrict__ b_gate, const float* __restrict__ xin, int B, int d, int norm, float eps,
                      const int32_t* __restrict__ exec_idx, const int32_t* __restrict__ count_ptr, int K, int c, int F,
                      float* __restrict__ act, int act_stride, uint32_t* survive, int* status, const unsigned* landed, unsigned need_seq,
@@ -202,7 +202,7 @@ __global__ void __launch_bounds__(256)
     for (int b = 0; b < BT; ++b) {
       if (b < B) {
         const float g = warp_sum(ag[b]) * s_inv[b] + (b_gate ? b_gate[i] : 0.f);
-        float a = fmaxf(g, 0.f);
+        float a = act_kind == 0 ? fmaxf(g, 0.f) : g / (1.f + expf(-g));  // ReLU, or SiLU as Eq. 1 prints it
         if (gated) a *= warp_sum(au[b]) * s_inv[b];
         if (lane == 0) act[(size_t)b * act_stride + p] = a;
         any |= (a != 0.f);

@@ -77,7 +77,7 @@ __host__ __device__ inline int wt_rows(int E) { return 8 * wt_tiles(E) + wt_plai
 
 struct WtLayer {  // one per layer of the stack (device array)
   const uint16_t* bundles; const float* b_gate; const float* b_down;
-  int n_mat, F, norm; float eps;
+  int n_mat, F, norm, act; float eps;  // act: 0 ReLU, 1 SiLU
   // predictor of the layer this one refines (the next layer; the last layer refines itself)
   const uint16_t* At_sl; const uint16_t* Bt_pad; const float* pc;  // Bt_pad: rows of wt_brow_bytes(r) bytes, zero padded
   int r, Fn, norm_n; float eps_n;
@@ -343,14 +343,17 @@ __device__ __forceinline__ void wt_stream(const WtCall& C, WtShared& sh, const W
     wt_ring_dots<WD>(ring, row_b, ng, s_x, d, C.piece_len, s_gsum + 4 * g0);
     __syncthreads();
   }
-  // activation of the gate branch and the ordered list of survivors (a_i = relu(g_i) u_i: g_i <= 0 needs no other row)
+  // activation of the gate branch and the ordered list of survivors (ReLU: a_i = relu(g_i) u_i, so g_i <= 0 needs no other
+  // row; SiLU has no zeros: every selected neuron goes on)
   {
     float g = 0.f;
+    bool sv = false;
     if (my_idx >= 0) {
       const float4 s4 = *reinterpret_cast<const float4*>(s_gsum + tid * 4);
       g = ((s4.x + s4.y) + (s4.z + s4.w)) * inv + my_b;
+      sv = g > 0.f;
+      if (L.act != 0) { g = g / (1.f + expf(-g)); sv = true; }
     }
-    const bool sv = g > 0.f;
     const unsigned m = __ballot_sync(0xffffffffu, sv);
     if (lane == 0) sh.wcnt[warp] = __popc(m);
     __syncthreads();

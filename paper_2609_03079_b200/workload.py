@@ -34,7 +34,7 @@ import threading
 
 _EIGH_LOCK = threading.Lock()
 
-T_GATE, T_UP, T_DOWN, T_PRED_NOISE, T_TOKENS = 0, 1, 2, 3, 4
+T_GATE, T_UP, T_DOWN, T_PRED_NOISE, T_TOKENS, T_HASH = 0, 1, 2, 3, 4, 5
 
 WEIGHT_STD = 0.02
 PRED_NOISE_STD = 0.01
@@ -121,6 +121,7 @@ class LayerArrays:
     pred_c: np.ndarray  # [d_ff] float32
     b_down: Optional[np.ndarray] = None  # [d_model] float32
     meta: dict = field(default_factory=dict)
+    act: str = "relu"  # "relu" (the sparsity source of the workloads) or "silu" (as Eq. 1 of the paper prints it)
 
 
 def _rng(seed: int, layer: int, tensor_id: int) -> np.random.Generator:
@@ -232,3 +233,49 @@ def tied_duplicate_layer(base: LayerArrays, pairs) -> LayerArrays:
         out.pred_b[:, dst] = out.pred_b[:, src]
         out.pred_c[dst] = out.pred_c[src]
     return out
+
+
+@dataclass
+class HashPredictorArrays:
+    """Host arrays of a stacked hashing predictor with random tables (trained ones do not exist offline), in both forms:
+    sign arrays in {-1,+1} for the oracle and the same signs packed one bit per component for the library
+    (+1 -> 1, component c at bit c % 32 of word c // 32)."""
+
+    d_model: int
+    rank: int
+    tau: int
+    d_code: int
+    n_layers: int
+    d_ff: int
+    wdtype: str
+    pca: np.ndarray        # [d_model, rank] uint16 bit patterns (the layer's PCA projection)
+    w1: np.ndarray         # [rank, tau] float32
+    w_signs: List[np.ndarray]   # n_layers - 1 arrays [d_code, tau] int8
+    t_signs: List[np.ndarray]   # n_layers arrays [2^tau, d_code] int8
+    code_signs: np.ndarray      # [d_ff, d_code] int8
+    w_bits: np.ndarray     # [n_layers - 1, tau, d_code // 32] uint32
+    t_bits: np.ndarray     # [n_layers, 2^tau, d_code // 32] uint32
+    code_bits: np.ndarray  # [d_ff, d_code // 32] uint32
+
+
+def pack_signs(signs: np.ndarray) -> np.ndarray:
+    """[..., d] signs in {-1,+1} -> [..., d // 32] uint32, bit (c % 32) of word (c // 32) set where the sign is +1."""
+    b = np.ascontiguousarray(np.asarray(signs) > 0, dtype=np.uint8)
+    if b.shape[-1] % 32:
+        raise ValueError("the number of components must be a multiple of 32")
+    return np.ascontiguousarray(np.packbits(b, axis=-1, bitorder="little")).view(np.uint32)
+
+
+def make_hash_predictor(base: LayerArrays, seed: int, layer: int, tau: int = 8, d_code: int = 256, n_layers: int = 5) -> HashPredictorArrays:
+    """Random stacked-hashing tables on top of a layer's PCA projection (the paper's default shape: five layers, tau = 8,
+    d = 256).  Random tables serve parity and throughput only: they predict nothing."""
+    rng = _rng(seed, layer, T_HASH)
+    w1 = rng.standard_normal((base.rank, tau)).astype(np.float32)
+    pm = lambda shape: (rng.integers(0, 2, size=shape, dtype=np.int8) * 2 - 1).astype(np.int8)
+    w_signs = [pm((d_code, tau)) for _ in range(n_layers - 1)]
+    t_signs = [pm((2 ** tau, d_code)) for _ in range(n_layers)]
+    code_signs = pm((base.d_ff, d_code))
+    w_bits = np.stack([pack_signs(w.T) for w in w_signs]) if w_signs else np.zeros((0, tau, d_code // 32), dtype=np.uint32)
+    t_bits = np.stack([pack_signs(t) for t in t_signs])
+    return HashPredictorArrays(base.d_model, base.rank, tau, d_code, n_layers, base.d_ff, base.wdtype, base.pred_a, w1, w_signs, t_signs,
+                               code_signs, np.ascontiguousarray(w_bits), np.ascontiguousarray(t_bits), np.ascontiguousarray(pack_signs(code_signs)))

@@ -79,6 +79,9 @@ def check_survive(gpu_survive: set, L: orc.OracleLayer, x: np.ndarray, order: np
     g = L.w_gate[order] @ h + L.b_gate[order]
     a = orc.neuron_activations(L, h, order)
     ref = set(order[a != 0.0].tolist())
+    if L.act == orc.SILU:  # no zeros: every selected neuron survives (an exact zero needs g = 0 or u = 0 exactly)
+        assert gpu_survive == ref
+        return
     tol = 1e-5 * np.linalg.norm(L.w_gate[order], axis=1) * np.linalg.norm(h)
     fuzzy = set(order[np.abs(g) <= tol].tolist())
     assert (gpu_survive ^ ref) <= fuzzy, f"survive mask differs: {sorted((gpu_survive ^ ref) - fuzzy)[:10]}"

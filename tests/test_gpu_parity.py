@@ -307,3 +307,21 @@ def test_llama7b_shaped_layer_wide_selection():
     assert stats.get("band", 0) == 0
     ga.close()
     gb.close()
+
+
+@pytest.mark.parametrize("gated", [True, False])
+def test_silu_layers(gated):
+    """The activation Eq. 1 prints (SiLU): no exact zeros, so every selected neuron contributes its up and down rows;
+    values against the oracle's SiLU branch, sets bit-exact as always, on ragged shapes."""
+    spec, la = custom_arrays(23, 264, 1000, 40, gated=gated, wdtype="bf16" if gated else "fp16")
+    la.act = "silu"
+    if not gated:
+        la.b_down = (0.01 * np.arange(264, dtype=np.float32) - 1.0)
+    OL = orc.OracleLayer.from_arrays(la)
+    assert OL.act == orc.SILU
+    gl = ls.ls_layer_create(la, DEV)
+    stats = {}
+    for x in wl.make_tokens(spec):
+        run_step_and_compare(gl, gl, OL, OL, x, 77, 5, 130, stats)
+    assert stats.get("band", 0) == 0
+    gl.close()

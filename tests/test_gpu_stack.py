@@ -261,3 +261,14 @@ def test_llama7b_full_stack_two_consecutive_tokens():
                 assert S[n, :k].tolist() == order_out.tolist()
         cur = nxt
     assert stats.get("band", 0) == 0
+
+
+def test_tiny4_stack_with_silu_layers():
+    """Whole-token kernel on SiLU layers: every selected neuron's bundle is streamed (several batches of the row ring)."""
+    spec = wl.SPECS["tiny4"]
+    arrays = wl.make_stack(spec, down_scale=50.0)
+    for a in arrays:
+        a.act = "silu"
+    stats = {}
+    decode_and_check(spec, arrays, 4, spec.k, 2, stats)
+    assert stats.get("band", 0) == 0
