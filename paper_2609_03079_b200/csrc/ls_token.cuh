@@ -123,6 +123,7 @@ struct WtCall {
 
 struct WtShared {
   WtLayer L[2];
+  unsigned long long mbar[3];  // transaction barriers of the bulk copies: rows into the ring, the A slices, the B^T rows
   int dead;               // a wait timed out: no more waiting
   int nmine, nsurv;
   int wcnt[WT_WARPS];
@@ -235,65 +236,156 @@ __device__ __forceinline__ void wt_share(int count, int K, int gs, int cta, int&
 }
 
 // ---- S: gate rows, survivors, up and down rows -----------------------------------------------------------------------
-// Rows travel global -> shared memory by cp.async (requested by tiny loops, all in flight at once, no registers held),
-// and every computation is a small rolled loop over shared memory: the phase's code stays a few hundred instructions.
+// Rows travel global -> shared memory as bulk copies (one instruction per row, issued by one lane; the copy engine moves
+// the bytes and counts them off on a transaction barrier in shared memory), all in flight at once, no registers held;
+// every computation is a small rolled loop over shared memory.
+__device__ __forceinline__ uint32_t wt_saddr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void wt_mbar_init(unsigned long long* b, int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(wt_saddr(b)), "r"(count) : "memory");
+}
+// One arrival that also announces `bytes` bytes of copies to come.
+__device__ __forceinline__ void wt_mbar_expect(unsigned long long* b, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(wt_saddr(b)), "r"(bytes) : "memory");
+}
+// Linear copy global -> shared memory (both 16-byte aligned, a multiple of 16 bytes, no multicast).
+__device__ __forceinline__ void wt_bulk_load(void* dst, const void* src, uint32_t bytes, unsigned long long* b) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(wt_saddr(dst)), "l"(src),
+               "r"(bytes), "r"(wt_saddr(b))
+               : "memory");
+}
+// Shared memory that ordinary loads and stores touched is handed to the copy engine.
+__device__ __forceinline__ void wt_fence_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// Wait (bounded) for the phase of parity `parity` to complete; on a timeout the CTA stops waiting for anything.
+__device__ __noinline__ void wt_mbar_wait(WtShared& sh, unsigned long long* b, uint32_t parity) {
+  if (sh.dead) return;
+  const long long t0 = clock64();
+  for (;;) {
+    uint32_t ok;
+    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+                 : "=r"(ok)
+                 : "r"(wt_saddr(b)), "r"(parity)
+                 : "memory");
+    if (ok) return;
+    if (clock64() - t0 > WT_SPIN_CLOCKS) break;
+  }
+  sh.dead = 1;
+  set_status(sh.L[0].status, ST_TIMEOUT);
+}
 
-// `nrow` rows of `bytes` bytes each, row i from src_of(i), to consecutive places in the ring (a warp per row).
+// `nrow` rows of `bytes` bytes each, row i from src_of(i), to consecutive places in the ring: warp w's first lane issues
+// the rows w, w + 16, ... and arrives once on the barrier (16 arrivals complete a phase) with the bytes it asked for.
 template <class SrcFn>
-__device__ __forceinline__ void wt_request_rows(unsigned char* ring, int nrow, int bytes, SrcFn src_of) {
+__device__ __forceinline__ void wt_request_rows(unsigned long long* bar, unsigned char* ring, int nrow, int bytes, SrcFn src_of) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (lane != 0) return;
+  uint32_t total = 0;
+#pragma unroll 1
+  for (int i = warp; i < nrow; i += WT_WARPS) total += src_of(i) != nullptr ? bytes : 0;
+  wt_fence_async();
+  wt_mbar_expect(bar, total);
 #pragma unroll 1
   for (int i = warp; i < nrow; i += WT_WARPS) {
     const unsigned char* src = src_of(i);
-    if (src == nullptr) continue;
-    unsigned char* dst = ring + (size_t)i * bytes;
-#pragma unroll 1
-    for (int o = lane * 16; o < bytes; o += 512) wt_cp_async16(dst + o, src + o);
+    if (src != nullptr) wt_bulk_load(ring + (size_t)i * bytes, src, bytes, bar);
   }
 }
 
-// Dot products of `nrow` rows in the ring (row i at ring + i * stride) with x, a quarter of a row per warp and turn:
-// out[4 i + q] = partial sum of quarter q of row i.
+// Four consecutive 16-bit weights widened exactly to fp32.
 template <int WD>
-__device__ __forceinline__ void wt_ring_dots(const unsigned char* ring, int stride, int nrow, const float* s_x, int d, int piece_len, float* out) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-#pragma unroll 1
-  for (int u = warp; u < 4 * nrow; u += WT_WARPS) {
-    const int c_lo = min(d, (u & 3) * piece_len), c_hi = min(d, c_lo + piece_len);
-    const uint16_t* w = reinterpret_cast<const uint16_t*>(ring + (size_t)(u >> 2) * stride);
-    float acc = 0.f;
-#pragma unroll 1
-    for (int c = c_lo + lane * 8; c < c_hi; c += 256) {
-      float f[8];
-      unpack8<WD>(*reinterpret_cast<const uint4*>(w + c), f);
-      const float4 x0 = *reinterpret_cast<const float4*>(s_x + c), x1 = *reinterpret_cast<const float4*>(s_x + c + 4);
-      acc = fmaf(f[0], x0.x, acc); acc = fmaf(f[1], x0.y, acc); acc = fmaf(f[2], x0.z, acc); acc = fmaf(f[3], x0.w, acc);
-      acc = fmaf(f[4], x1.x, acc); acc = fmaf(f[5], x1.y, acc); acc = fmaf(f[6], x1.z, acc); acc = fmaf(f[7], x1.w, acc);
-    }
-    acc = warp_sum(acc);
-    if (lane == 0) out[u] = acc;
+__device__ __forceinline__ void wt_unpack4(const uint2& v, float (&f)[4]) {
+  if (WD == WD_BF16) {
+    f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xffff0000u);
+    f[2] = __uint_as_float(v.y << 16); f[3] = __uint_as_float(v.y & 0xffff0000u);
+  } else {
+    const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&v.x)), b = __half22float2(*reinterpret_cast<const __half2*>(&v.y));
+    f[0] = a.x; f[1] = a.y; f[2] = b.x; f[3] = b.y;
   }
 }
 
-// This CTA's slices of the next layer's predictor matrix A, its rows of B^T (stored padded, so both are plain linear
-// copies) and its score offsets: asynchronously to shared memory; needed in P1 and P3.
-__device__ __forceinline__ void wt_fetch_predictor(const WtCall& C, const WtLayer& L, unsigned char* smem) {
-  const int tid = threadIdx.x, G = gridDim.x, d = C.d;
-  const int nsl = (d + 31) >> 5, per_slice = L.r * 4;  // 16-byte pieces per slice
-  unsigned char* s_a = smem + C.lay.u_off;
+// Dot products of `nrow` rows in the ring (row i at ring + i * stride) with x: out[4 i + p] = partial sum of quarter p of
+// row i.  Warp (p, q) = (warp % 4, warp / 4) takes quarter p of the rows q, q + 4, ...; its part of x stays in registers
+// across the rows (x is fp32, twice the bytes of a row: reading it once per row would double the shared-memory traffic).
+// A lane owns columns 4 lane .. 4 lane + 3 of each run of 128 columns: every load is free of bank conflicts.
+template <int WD>
+__device__ __noinline__ void wt_ring_dots(const unsigned char* ring, int stride, int nrow, const float* s_x, int d, int piece_len, float* out) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int p = warp & 3, q = warp >> 2;
+  const int c_lo = min(d, p * piece_len), c_hi = min(d, c_lo + piece_len);
+  if (q >= nrow) return;
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};  // rows r0, r0 + 4, r0 + 8, r0 + 12
 #pragma unroll 1
-  for (int s = blockIdx.x, si = 0; s < nsl; s += G, ++si) {
-    const unsigned char* src = reinterpret_cast<const unsigned char*>(L.At_sl) + (size_t)s * per_slice * 16;
+  for (int r0 = q; r0 < nrow; r0 += 16) {
 #pragma unroll 1
-    for (int i = tid; i < per_slice; i += WT_THREADS) wt_cp_async16(s_a + (si * per_slice + i) * 16, src + i * 16);
+    for (int cb = c_lo + lane * 4; cb < c_hi; cb += 1024) {
+      float4 xv[8];
+#pragma unroll
+      for (int it = 0; it < 8; ++it) {
+        const int c = cb + it * 128;
+        xv[it] = c < c_hi ? *reinterpret_cast<const float4*>(s_x + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int r = r0 + 4 * j;
+        if (r < nrow) {
+          const uint16_t* w = reinterpret_cast<const uint16_t*>(ring + (size_t)r * stride);
+          float a0 = acc[j], a1 = 0.f;
+#pragma unroll
+          for (int it = 0; it < 8; it += 2) {
+            const int c = cb + it * 128;
+            float f[4], g[4];
+            if (c < c_hi) {
+              wt_unpack4<WD>(*reinterpret_cast<const uint2*>(w + c), f);
+              a0 = fmaf(f[0], xv[it].x, a0); a0 = fmaf(f[1], xv[it].y, a0); a0 = fmaf(f[2], xv[it].z, a0); a0 = fmaf(f[3], xv[it].w, a0);
+            }
+            if (c + 128 < c_hi) {
+              wt_unpack4<WD>(*reinterpret_cast<const uint2*>(w + c + 128), g);
+              a1 = fmaf(g[0], xv[it + 1].x, a1); a1 = fmaf(g[1], xv[it + 1].y, a1); a1 = fmaf(g[2], xv[it + 1].z, a1); a1 = fmaf(g[3], xv[it + 1].w, a1);
+            }
+          }
+          acc[j] = a0 + a1;
+        }
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int r = r0 + 4 * j;
+      if (r < nrow) {  // (uniform over the warp)
+        const float v = warp_sum(acc[j]);
+        if (lane == 0) out[4 * r + p] = v;
+      }
+      acc[j] = 0.f;
+    }
   }
+}
+
+// This CTA's slices of the next layer's predictor matrix A and its rows of B^T (stored padded, so both are plain linear
+// copies: bulk copies by thread 0, each on a barrier of its own that completes exactly one phase per layer, also when
+// there is nothing to copy) and its score offsets (4-byte asynchronous copies): needed in P1 and P3.  Called after a
+// __syncthreads that ends the ring's use.
+__device__ __forceinline__ void wt_fetch_predictor(const WtCall& C, WtShared& sh, const WtLayer& L, unsigned char* smem) {
+  const int tid = threadIdx.x, G = gridDim.x, d = C.d;
+  const int nsl = (d + 31) >> 5, slice_b = L.r * 64;  // bytes per slice: 32 columns of r 16-bit entries
   const int per = (L.Fn + G - 1) / G, n0 = min(L.Fn, (int)blockIdx.x * per), n1 = min(L.Fn, n0 + per);
-  const int RB = wt_brow_bytes(L.r);
-  const int npieces = (((n1 - n0 + 7) >> 3) * 8) * (RB >> 4);
-  unsigned char* s_b = smem + C.lay.u_off + C.lay.b_off;
-  const unsigned char* src = reinterpret_cast<const unsigned char*>(L.Bt_pad) + (size_t)n0 * RB;
+  if (tid == 0) {
+    unsigned char* s_a = smem + C.lay.u_off;
+    wt_fence_async();
+    uint32_t a_bytes = 0;
 #pragma unroll 1
-  for (int i = tid; i < npieces; i += WT_THREADS) wt_cp_async16(s_b + i * 16, src + (size_t)i * 16);
+    for (int s = blockIdx.x; s < nsl; s += G) a_bytes += slice_b;
+    wt_mbar_expect(&sh.mbar[1], a_bytes);
+    if (slice_b > 0) {
+#pragma unroll 1
+      for (int s = blockIdx.x, si = 0; s < nsl; s += G, ++si)
+        wt_bulk_load(s_a + (size_t)si * slice_b, reinterpret_cast<const unsigned char*>(L.At_sl) + (size_t)s * slice_b, slice_b, &sh.mbar[1]);
+    }
+    const int RB = wt_brow_bytes(L.r);
+    const uint32_t b_bytes = (uint32_t)(((n1 - n0 + 7) >> 3) * 8) * RB;
+    wt_mbar_expect(&sh.mbar[2], b_bytes);
+    unsigned char* s_b = smem + C.lay.u_off + C.lay.b_off;
+    const unsigned char* src = reinterpret_cast<const unsigned char*>(L.Bt_pad) + (size_t)n0 * RB;
+#pragma unroll 1
+    for (uint32_t o = 0; o < b_bytes; o += 32768u) wt_bulk_load(s_b + o, src + o, min(32768u, b_bytes - o), &sh.mbar[2]);
+  }
   float* s_pc = reinterpret_cast<float*>(smem + C.lay.pc_off);
 #pragma unroll 1
   for (int i = tid; i < n1 - n0; i += WT_THREADS) {
@@ -302,11 +394,24 @@ __device__ __forceinline__ void wt_fetch_predictor(const WtCall& C, const WtLaye
   }
 }
 
+// The same rows of B^T once more, by ordinary asynchronous copies (after a degenerate selection borrowed their place).
+__device__ __noinline__ void wt_refetch_b(const WtCall& C, const WtLayer& L, unsigned char* smem) {
+  const int G = gridDim.x;
+  const int per = (L.Fn + G - 1) / G, n0 = min(L.Fn, (int)blockIdx.x * per), n1 = min(L.Fn, n0 + per);
+  const int RB = wt_brow_bytes(L.r);
+  const int npieces = (((n1 - n0 + 7) >> 3) * 8) * (RB >> 4);
+  unsigned char* s_b = smem + C.lay.u_off + C.lay.b_off;
+  const unsigned char* src = reinterpret_cast<const unsigned char*>(L.Bt_pad) + (size_t)n0 * RB;
+#pragma unroll 1
+  for (int i = threadIdx.x; i < npieces; i += WT_THREADS) wt_cp_async16(s_b + i * 16, src + (size_t)i * 16);
+  wt_cp_async_wait();
+}
+
 template <int WD>
 __device__ __noinline__ void wt_score_evals(const WtCall& C, WtShared& sh, const WtLayer& L, int e0, int ne, bool last);
 
 template <int WD>
-__device__ __forceinline__ void wt_stream(const WtCall& C, WtShared& sh, const WtLayer& L, unsigned char* smem, bool active) {
+__device__ __forceinline__ void wt_stream(const WtCall& C, WtShared& sh, const WtLayer& L, unsigned char* smem, bool active, uint32_t& ring_phase) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int d = C.d;
   const float* s_x = reinterpret_cast<const float*>(smem + C.lay.x_off);
@@ -334,12 +439,12 @@ __device__ __forceinline__ void wt_stream(const WtCall& C, WtShared& sh, const W
 #pragma unroll 1
   for (int g0 = 0; g0 < nmine; g0 += cap_g) {
     const int ng = min(cap_g, nmine - g0);
-    wt_request_rows(ring, ng, row_b, [&](int i) -> const unsigned char* {
+    wt_request_rows(&sh.mbar[0], ring, ng, row_b, [&](int i) -> const unsigned char* {
       const int v = s_mine[g0 + i];
       return v >= 0 ? wbase + (size_t)v * bundle_b : nullptr;
     });
-    wt_cp_async_wait();
-    __syncthreads();
+    wt_mbar_wait(sh, &sh.mbar[0], ring_phase);
+    ring_phase ^= 1u;
     wt_ring_dots<WD>(ring, row_b, ng, s_x, d, C.piece_len, s_gsum + 4 * g0);
     __syncthreads();
   }
@@ -382,9 +487,9 @@ __device__ __forceinline__ void wt_stream(const WtCall& C, WtShared& sh, const W
 #pragma unroll 1
   for (int b0 = 0; b0 < nsurv; b0 += cap_s) {
     const int nb = min(cap_s, nsurv - b0);
-    wt_request_rows(ring, nb, rest_b, [&](int i) -> const unsigned char* { return wbase + (size_t)s_sidx[b0 + i] * bundle_b + row_b; });
-    wt_cp_async_wait();
-    __syncthreads();
+    wt_request_rows(&sh.mbar[0], ring, nb, rest_b, [&](int i) -> const unsigned char* { return wbase + (size_t)s_sidx[b0 + i] * bundle_b + row_b; });
+    wt_mbar_wait(sh, &sh.mbar[0], ring_phase);
+    ring_phase ^= 1u;
     if (gated) {
       wt_ring_dots<WD>(ring, rest_b, nb, s_x, d, C.piece_len, s_gsum);
       __syncthreads();
@@ -428,7 +533,7 @@ __device__ __forceinline__ void wt_stream(const WtCall& C, WtShared& sh, const W
     __stcg(reinterpret_cast<float4*>(yp + tid * 8), make_float4(acc8[0], acc8[1], acc8[2], acc8[3]));
     __stcg(reinterpret_cast<float4*>(yp + tid * 8 + 4), make_float4(acc8[4], acc8[5], acc8[6], acc8[7]));
   }
-  wt_fetch_predictor(C, L, smem);
+  wt_fetch_predictor(C, sh, L, smem);
 }
 
 // ---- P1: stage sums, partial residual features, x_out, partial latents of this CTA's slices ----------------------------
@@ -460,6 +565,7 @@ __device__ __forceinline__ void wt_feature(const WtCall& C, WtShared& sh, const 
       for (int row = warp; row < n_act; row += WT_WARPS) wt_cp_async16(s_y + row * 32 + lane * 4, yp + (size_t)row * d);
     }
     wt_cp_async_wait();
+    wt_mbar_wait(sh, &sh.mbar[1], (uint32_t)n & 1u);  // (this CTA's slices of A, requested at the end of S)
     __syncthreads();
     {
       const int c = warp / wps, h = warp - c * wps;
@@ -594,8 +700,7 @@ __device__ __noinline__ void wt_score_evals(const WtCall& C, WtShared& sh, const
     const int bv = sh.b_valid;
     __syncthreads();
     if (!bv) {  // (a general top-k borrowed the place of the B^T rows: fetch them again)
-      wt_fetch_predictor(C, L, wt_smem);
-      wt_cp_async_wait();
+      wt_refetch_b(C, L, wt_smem);
       if (tid == 0) sh.b_valid = 1;
       __syncthreads();
     }
@@ -940,7 +1045,15 @@ __global__ void __launch_bounds__(WT_THREADS, 1) ls_token_kernel(const WtLayer* 
   // ---- prologue: arguments of layer 0, x, 1 / rms, this CTA's slice of the first selection
   if (tid < NW)
     reinterpret_cast<uint32_t*>(&sh.L[0])[tid] = g_layers ? reinterpret_cast<const uint32_t*>(&g_layers[0])[tid] : reinterpret_cast<const uint32_t*>(&C.one)[tid];
-  if (tid == 0) { sh.dead = 0; sh.b_valid = 1; }
+  if (tid == 0) {
+    sh.dead = 0;
+    sh.b_valid = 1;
+    wt_mbar_init(&sh.mbar[0], WT_WARPS);  // rows into the ring: one arrival per warp and batch
+    wt_mbar_init(&sh.mbar[1], 1);         // A slices, B^T rows: one phase per layer
+    wt_mbar_init(&sh.mbar[2], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  uint32_t ring_phase = 0;
   {
     double sq = 0.0;
     for (int c = tid * 4; c < d; c += WT_THREADS * 4) {
@@ -975,16 +1088,23 @@ __global__ void __launch_bounds__(WT_THREADS, 1) ls_token_kernel(const WtLayer* 
   }
   __syncthreads();
 
-  // The refined sets of layer m's evaluations j < K: one CTA each, CTAs that own no slice of the feature when there are
-  // enough of them (they have nothing else to do in P1).
-  auto refined_sets = [&](int m, const WtLayer& Lm) {
-    const int nsl = (d + 31) >> 5, keff_m = min(C.k_next, Lm.Fn);
+  // The refined sets of layer m's evaluations j < K (their scores are complete since layer m's last barrier).  `where` 0:
+  // called at the start of the next layer's stream phase, 1: in its P1, 2: after the last layer.  They go to the CTAs
+  // that have no rows to stream (two or so evaluations each: the stream phase is long enough) when there are such CTAs,
+  // otherwise to CTAs that own no slice of the feature, during P1.
+  auto refined_sets = [&](int m, const WtLayer& Lm, int where) {
+    const int nsl = (d + 31) >> 5, keff_m = min(C.k_next, Lm.Fn), n_idle = G - n_act;
+    const bool in_stream = n_idle > 0;
+    if (where != 2 && (where == 0) != in_stream) return;
     unsigned long long* cuts = C.cuts + (size_t)m * E;
 #pragma unroll 1
     for (int j = 0; j < K; ++j) {
-      const int owner = nsl + K <= G ? nsl + j : G - 1 - (j % G);
-      if (cta == owner)
+      const int owner = in_stream ? n_act + j % n_idle : (nsl + K <= G ? nsl + j : G - 1 - (j % G));
+      if (cta == owner) {
+        // (in P1 this CTA's rows of B^T may still be on their way into the work area a degenerate selection borrows)
+        if (where == 1) wt_mbar_wait(sh, &sh.mbar[2], (uint32_t)(m + 1) & 1u);
         wt_refined_set(C, sh, smem, j, Lm.Fn, keff_m, C.tr_masks ? C.tr_masks + ((size_t)m * E + j) * C.tr_words : nullptr, cuts + j);
+      }
     }
   };
 
@@ -995,8 +1115,9 @@ __global__ void __launch_bounds__(WT_THREADS, 1) ls_token_kernel(const WtLayer* 
     const int rz = (L.r + 4) & ~3;
     const int keff = min(C.k_next, L.Fn);
     if (stamps) wt_stamp(C, n, 0);
-    // ---- S
-    wt_stream<WD>(C, sh, L, smem, active);
+    // ---- S (and, on the CTAs without rows, the refined sets of the layer before)
+    if (n > 0 && !active) refined_sets(n - 1, sh.L[(n - 1) & 1], 0);
+    wt_stream<WD>(C, sh, L, smem, active, ring_phase);
     if (stamps) wt_stamp(C, n, 1);
     wt_grid_sync(C, sh, ++epoch * G);
     if (sh.dead) return;
@@ -1004,7 +1125,7 @@ __global__ void __launch_bounds__(WT_THREADS, 1) ls_token_kernel(const WtLayer* 
     // ---- P1 (and the refined sets of the layer before, whose scores are complete now)
     float* x_out = last ? C.x_out : C.xbuf + (size_t)((n + 1) & 1) * d;
     wt_feature<WD>(C, sh, L, smem, n, x_out, E, rz);
-    if (n > 0) refined_sets(n - 1, sh.L[(n - 1) & 1]);
+    if (n > 0) refined_sets(n - 1, sh.L[(n - 1) & 1], 1);
     if (stamps) wt_stamp(C, n, 3);
     // next layer's arguments (the layer before's are not needed any more)
     __syncthreads();
@@ -1035,7 +1156,8 @@ __global__ void __launch_bounds__(WT_THREADS, 1) ls_token_kernel(const WtLayer* 
     if (sh.dead) return;
     if (stamps) wt_stamp(C, n, 6);
     // ---- P3
-    wt_cp_async_wait();  // (this CTA's rows of B^T, requested at the end of S)
+    wt_cp_async_wait();  // (this CTA's score offsets and rows of B^T, requested at the end of S)
+    wt_mbar_wait(sh, &sh.mbar[2], (uint32_t)n & 1u);
     __syncthreads();
     wt_score_evals<WD>(C, sh, L, 0, E, last);
     if (stamps) wt_stamp(C, n, 7);
@@ -1062,7 +1184,7 @@ __global__ void __launch_bounds__(WT_THREADS, 1) ls_token_kernel(const WtLayer* 
     if (stamps) wt_stamp(C, n, 10);
   }
   // ---- the last layer's refined sets
-  refined_sets(C.n_layers - 1, sh.L[(C.n_layers - 1) & 1]);
+  refined_sets(C.n_layers - 1, sh.L[(C.n_layers - 1) & 1], 2);
 }
 
 }  // namespace ls
