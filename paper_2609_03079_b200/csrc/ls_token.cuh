@@ -1089,17 +1089,19 @@ __global__ void __launch_bounds__(WT_THREADS, 1) ls_token_kernel(const WtLayer* 
   __syncthreads();
 
   // The refined sets of layer m's evaluations j < K (their scores are complete since layer m's last barrier).  `where` 0:
-  // called at the start of the next layer's stream phase, 1: in its P1, 2: after the last layer.  They go to the CTAs
-  // that have no rows to stream (two or so evaluations each: the stream phase is long enough) when there are such CTAs,
-  // otherwise to CTAs that own no slice of the feature, during P1.
+  // called at the start of the next layer's stream phase, 1: in its P1, 2: after the last layer.  The CTAs that have no
+  // rows to stream take two evaluations each during the stream phase (it is long enough for two); what is left goes to
+  // CTAs that own no slice of the feature, during P1 (or, when every CTA owns one, behind its slice).
   auto refined_sets = [&](int m, const WtLayer& Lm, int where) {
-    const int nsl = (d + 31) >> 5, keff_m = min(C.k_next, Lm.Fn), n_idle = G - n_act;
-    const bool in_stream = n_idle > 0;
-    if (where != 2 && (where == 0) != in_stream) return;
+    const int n_idle = G - n_act, cap_s = min(K, 2 * n_idle);
+    if ((where == 0 && cap_s == 0) || (where == 1 && cap_s == K)) return;
+    const int nsl = (d + 31) >> 5, keff_m = min(C.k_next, Lm.Fn);
+    const int j0 = where == 1 ? cap_s : 0, j1 = where == 0 ? cap_s : K;
     unsigned long long* cuts = C.cuts + (size_t)m * E;
 #pragma unroll 1
-    for (int j = 0; j < K; ++j) {
-      const int owner = in_stream ? n_act + j % n_idle : (nsl + K <= G ? nsl + j : G - 1 - (j % G));
+    for (int j = j0; j < j1; ++j) {
+      const int q = j - cap_s;
+      const int owner = j < cap_s ? n_act + (j < n_idle ? j : j - n_idle) : (nsl + q < G ? nsl + q : G - 1 - (q % G));
       if (cta == owner) {
         // (in P1 this CTA's rows of B^T may still be on their way into the work area a degenerate selection borrows)
         if (where == 1) wt_mbar_wait(sh, &sh.mbar[2], (uint32_t)(m + 1) & 1u);
