@@ -365,6 +365,8 @@ bool token_layout(const TokenShape* S, int K, ls::WtSmem* out) {
   size_t o = 0;
   auto take = [&](size_t bytes) { const size_t at = o; o += (bytes + 127) & ~(size_t)127; return (unsigned)at; };
   L.x_off = take((size_t)S->d * 4);
+  L.xs_off = take((size_t)((S->d + 15) / 16) * 96);
+  L.part_off = take((size_t)ls::WT_WARPS * ls::WT_MMA_ROWS * 4);
   L.xt_off = take((size_t)(ls::WT_MAXE + 1) * ls::WT_XBLK * 8);
   L.dm_off = take((size_t)ls::WT_WARPS * 32 * 4);
   L.mine_off = take((size_t)ls::WT_MAXMINE * (4 + 16 + 4 + 4) + 32 * 4);
@@ -387,7 +389,7 @@ bool token_layout(const TokenShape* S, int K, ls::WtSmem* out) {
   L.ckey_off = sub((size_t)ls::WT_CANDCAP * 8);
   L.cidx_off = sub((size_t)ls::WT_CANDCAP * 4);
   L.cbin_off = sub((size_t)ls::WT_CANDCAP * 2);
-  const size_t bundle_rest = (size_t)2 * S->d * 2;  // up and down rows of one survivor
+  const size_t bundle_rest = (size_t)2 * S->d * 2 + 16;  // up and down rows of one survivor (rows sit 16 bytes apart modulo 128)
   const size_t u_need = std::max(std::max(q, bundle_rest), ls::topk_smem_bytes(S->f_max));
   if (o + u_need > kTokenSmemBudget) return false;
   L.total = (unsigned)kTokenSmemBudget;  // the rest of the budget lets more rows travel at once
@@ -409,6 +411,7 @@ int32_t launch_token(const TokenShape* shp, int device, int wd, const ls::WtLaye
   if (!token_layout(shp, K, &c.lay)) return fail(LS_ERR_STATE, "%s: %d stages do not fit the whole-token kernel's shared memory", who, K);
   c.n_layers = n_layers; c.d = shp->d; c.K = K; c.k_next = k_next; c.gs = gs;
   c.piece_len = ((shp->d + 3) / 4 + 255) / 256 * 256;
+  c.mma = shp->d % 16 == 0 ? 1 : 0;
   c.ring_bytes = (int)(c.lay.total - c.lay.u_off);
   c.inv_d = 1.0 / (double)shp->d;
   c.x_in = d_x; c.x_out = d_x_out;

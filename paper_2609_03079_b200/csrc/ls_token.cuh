@@ -86,7 +86,7 @@ struct WtLayer {  // one per layer of the stack (device array)
 };
 
 struct WtSmem {  // byte offsets into dynamic shared memory (computed on the host)
-  unsigned x_off, xt_off, dm_off, mine_off, bits_off, pc_off, hist_off, u_off;
+  unsigned x_off, xs_off, part_off, xt_off, dm_off, mine_off, bits_off, pc_off, hist_off, u_off;
   // region u: A slices | B^T rows | a slice of the partial outputs (P1) or latents (P3) | raw scores | selection lists.
   // While the layer streams the whole region is the ring of the rows in flight (the predictor operands are requested
   // when the stream is over); the general top-k also takes it from its start.
@@ -98,6 +98,7 @@ struct WtSmem {  // byte offsets into dynamic shared memory (computed on the hos
 struct WtCall {
   double inv_d;  // 1 / d
   int n_layers, d, K, k_next, piece_len, gs, ring_bytes;  // gs: CTAs per stage; ring_bytes: room for rows in shared memory
+  int mma;  // d is a multiple of 16: the dot products of the stream phase run on the 16-bit tensor cores
   const float* x_in; float* x_out;
   const int32_t* sel_idx; const int32_t* sel_count; int sel_cap;
   int32_t* out_idx; int32_t* out_count; uint32_t* out_mask; double* out_scores; int out_cap;
@@ -272,10 +273,10 @@ __device__ __noinline__ void wt_mbar_wait(WtShared& sh, unsigned long long* b, u
   set_status(sh.L[0].status, ST_TIMEOUT);
 }
 
-// `nrow` rows of `bytes` bytes each, row i from src_of(i), to consecutive places in the ring: warp w's first lane issues
+// `nrow` rows of `bytes` bytes each, row i from src_of(i), to ring + i * stride: warp w's first lane issues
 // the rows w, w + 16, ... and arrives once on the barrier (16 arrivals complete a phase) with the bytes it asked for.
 template <class SrcFn>
-__device__ __forceinline__ void wt_request_rows(unsigned long long* bar, unsigned char* ring, int nrow, int bytes, SrcFn src_of) {
+__device__ __forceinline__ void wt_request_rows(unsigned long long* bar, unsigned char* ring, int stride, int nrow, int bytes, SrcFn src_of) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   if (lane != 0) return;
   uint32_t total = 0;
@@ -286,7 +287,7 @@ __device__ __forceinline__ void wt_request_rows(unsigned long long* bar, unsigne
 #pragma unroll 1
   for (int i = warp; i < nrow; i += WT_WARPS) {
     const unsigned char* src = src_of(i);
-    if (src != nullptr) wt_bulk_load(ring + (size_t)i * bytes, src, bytes, bar);
+    if (src != nullptr) wt_bulk_load(ring + (size_t)i * stride, src, bytes, bar);
   }
 }
 
@@ -355,6 +356,107 @@ __device__ __noinline__ void wt_ring_dots(const unsigned char* ring, int stride,
       }
       acc[j] = 0.f;
     }
+  }
+}
+
+// ---- the same dot products on the 16-bit tensor cores ---------------------------------------------------------------------
+// A row-times-x product has one output column, but the kernel is bound by instructions, not by arithmetic, and one
+// m16n8k16 MMA replaces 16 x 16 multiply-adds of 32 lanes.  Exactness: x (fp32) is cut into three 16-bit terms,
+// x = t0 + 2^-S t1 + 2^-2S t2 (S = 8 for bf16, 11 for fp16; every cut is an exact fp32 subtraction), which become three
+// columns of the B operand; products of 16-bit values are exact in the fp32 accumulator, so the result differs from the
+// fp32 FMA loop only by the order and rounding of the additions.
+constexpr int WT_MMA_ROWS = 32;  // rows per batch (two m-tiles)
+
+template <int WD>
+__device__ __forceinline__ uint32_t wt_to16(float v) {
+  if (WD == WD_BF16) {
+    unsigned short h;
+    asm("cvt.rn.bf16.f32 %0, %1;" : "=h"(h) : "f"(v));
+    return (uint32_t)h;
+  }
+  return (uint32_t)__half_as_ushort(__float2half_rn(v));
+}
+template <int WD>
+__device__ __forceinline__ float wt_from16(uint32_t h) {
+  if (WD == WD_BF16) return __uint_as_float(h << 16);
+  return __half2float(__ushort_as_half((unsigned short)h));
+}
+// Four consecutive components of x (c a multiple of 4) to the fp32 copy and to the three 16-bit terms, the latter in the
+// order the MMA's B operand wants: [k-step of 16][term][t = 0..3][x[2t], x[2t+1], x[8+2t], x[8+2t+1]].
+template <int WD>
+__device__ __forceinline__ void wt_store_x4(float* s_x, uint16_t* s_xs, int c, const float4& v) {
+  *reinterpret_cast<float4*>(s_x + c) = v;
+  if (s_xs == nullptr) return;
+  constexpr float SC = WD == WD_BF16 ? 256.f : 2048.f;
+  const float x[4] = {v.x, v.y, v.z, v.w};
+  uint32_t term[3][4];
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const uint32_t h0 = wt_to16<WD>(x[e]);
+    const float r1 = (x[e] - wt_from16<WD>(h0)) * SC;
+    const uint32_t h1 = wt_to16<WD>(r1);
+    const float r2 = (r1 - wt_from16<WD>(h1)) * SC;
+    term[0][e] = h0; term[1][e] = h1; term[2][e] = wt_to16<WD>(r2);
+  }
+  const int ks = c >> 4, w = c & 15, t0 = (w & 7) >> 1, j0 = (w >> 3) * 2;
+#pragma unroll
+  for (int g = 0; g < 3; ++g) {
+    uint16_t* base = s_xs + ((ks * 3 + g) * 4 + t0) * 4 + j0;
+    *reinterpret_cast<uint32_t*>(base) = term[g][0] | (term[g][1] << 16);
+    *reinterpret_cast<uint32_t*>(base + 4) = term[g][2] | (term[g][3] << 16);
+  }
+}
+
+// Dot products of `nrow` <= 32 rows in the ring (row i at ring + i * stride, stride = 16 mod 128 bytes so that the matrix
+// loads are free of bank conflicts) with x: warp w takes the k-steps [w * per, (w + 1) * per) of every m-tile and leaves
+// its partial sums in part[w][row]; the caller adds the sixteen partials in a fixed order.
+template <int WD>
+__device__ __noinline__ void wt_ring_mma(const unsigned char* ring, int stride, int nrow, const uint16_t* s_xs, int d, float* part) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, g = lane >> 2, t = lane & 3;
+  const int nks = d >> 4, per = (nks + WT_WARPS - 1) / WT_WARPS;
+  const int k0 = min(nks, warp * per), k1 = min(nks, k0 + per);
+  constexpr float M1 = WD == WD_BF16 ? 1.f / 256.f : 1.f / 2048.f;
+  const int n_mt = (nrow + 15) >> 4;
+#pragma unroll 1
+  for (int mt = 0; mt < n_mt; ++mt) {
+    // this lane's row of the four 8 x 8 matrices of an A tile: matrix lane / 8 = (rows 0-7 | 8-15) x (k 0-7 | 8-15)
+    const int row = min(nrow - 1, mt * 16 + ((lane >> 3) & 1) * 8 + (lane & 7));
+    uint32_t a_addr = wt_saddr(ring + (size_t)row * stride) + (uint32_t)(k0 * 32 + (lane >> 4) * 16);
+    const uint16_t* xb = s_xs + ((k0 * 3 + g) * 4 + t) * 4;
+    float c0 = 0.f, c1 = 0.f, c2 = 0.f, c3 = 0.f;
+#pragma unroll 2
+    for (int ks = k0; ks < k1; ++ks, a_addr += 32, xb += 48) {
+      uint32_t a0, a1, a2, a3, b0 = 0u, b1 = 0u;
+      asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(a0), "=r"(a1), "=r"(a2), "=r"(a3) : "r"(a_addr));
+      if (g < 3) {
+        const uint2 b = *reinterpret_cast<const uint2*>(xb);
+        b0 = b.x; b1 = b.y;
+      }
+      if (WD == WD_BF16)
+        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                     : "+f"(c0), "+f"(c1), "+f"(c2), "+f"(c3) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+      else
+        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                     : "+f"(c0), "+f"(c1), "+f"(c2), "+f"(c3) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+    }
+    // columns 0, 1, 2 of the tile are the three terms: lane t = 0 holds columns 0 and 1, lane t = 1 column 2
+    float lo8 = t == 0 ? c0 + M1 * c1 : (M1 * M1) * c0, hi8 = t == 0 ? c2 + M1 * c3 : (M1 * M1) * c2;
+    lo8 += __shfl_down_sync(0xffffffffu, lo8, 1);
+    hi8 += __shfl_down_sync(0xffffffffu, hi8, 1);
+    if (t == 0) {
+      part[warp * WT_MMA_ROWS + mt * 16 + g] = lo8;
+      part[warp * WT_MMA_ROWS + mt * 16 + g + 8] = hi8;
+    }
+  }
+}
+// (after a __syncthreads) the sixteen partial sums of row i, added in a fixed order, as the first of the row's four places
+__device__ __forceinline__ void wt_fold_parts(const float* part, int nrow, float* out) {
+  const int i = threadIdx.x;
+  if (i < nrow) {
+    float v = 0.f;
+#pragma unroll
+    for (int w = 0; w < WT_WARPS; ++w) v += part[w * WT_MMA_ROWS + i];
+    *reinterpret_cast<float4*>(out + 4 * i) = make_float4(v, 0.f, 0.f, 0.f);
   }
 }
 
@@ -434,18 +536,27 @@ __device__ __forceinline__ void wt_stream(const WtCall& C, WtShared& sh, const W
     my_idx = s_mine[tid];
     if (my_idx >= 0 && L.b_gate) my_b = __ldg(L.b_gate + my_idx);
   }
-  // gate rows: as many at a time as the ring holds (all of them in the usual case)
-  const int cap_g = C.ring_bytes / row_b;
+  const uint16_t* s_xs = reinterpret_cast<const uint16_t*>(smem + C.lay.xs_off);
+  float* s_part = reinterpret_cast<float*>(smem + C.lay.part_off);
+  // gate rows: as many at a time as the ring holds (all of them in the usual case); rows sit 16 bytes apart modulo 128
+  const int gstride = row_b + 16;
+  const int cap_g = min(WT_MMA_ROWS, C.ring_bytes / gstride);
 #pragma unroll 1
   for (int g0 = 0; g0 < nmine; g0 += cap_g) {
     const int ng = min(cap_g, nmine - g0);
-    wt_request_rows(&sh.mbar[0], ring, ng, row_b, [&](int i) -> const unsigned char* {
+    wt_request_rows(&sh.mbar[0], ring, gstride, ng, row_b, [&](int i) -> const unsigned char* {
       const int v = s_mine[g0 + i];
       return v >= 0 ? wbase + (size_t)v * bundle_b : nullptr;
     });
     wt_mbar_wait(sh, &sh.mbar[0], ring_phase);
     ring_phase ^= 1u;
-    wt_ring_dots<WD>(ring, row_b, ng, s_x, d, C.piece_len, s_gsum + 4 * g0);
+    if (C.mma) {
+      wt_ring_mma<WD>(ring, gstride, ng, s_xs, d, s_part);
+      __syncthreads();
+      wt_fold_parts(s_part, ng, s_gsum + 4 * g0);
+    } else {
+      wt_ring_dots<WD>(ring, gstride, ng, s_x, d, C.piece_len, s_gsum + 4 * g0);
+    }
     __syncthreads();
   }
   // activation of the gate branch and the ordered list of survivors (ReLU: a_i = relu(g_i) u_i, so g_i <= 0 needs no other
@@ -476,7 +587,8 @@ __device__ __forceinline__ void wt_stream(const WtCall& C, WtShared& sh, const W
   const int nsurv = sh.nsurv;
   // survivors: the rest of their bundles (up and down rows are adjacent: one linear copy), as many as the ring holds
   const int rest_b = (L.n_mat - 1) * row_b;
-  const int cap_s = C.ring_bytes / rest_b;
+  const int rstride = rest_b + 16;
+  const int cap_s = min(WT_MMA_ROWS, C.ring_bytes / rstride);
   float acc8[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};  // (d <= 4096: one column group per thread; beyond: see below)
   float* yp = C.ypart + (size_t)blockIdx.x * d;
   const bool wide = d > WT_THREADS * 8;
@@ -487,11 +599,17 @@ __device__ __forceinline__ void wt_stream(const WtCall& C, WtShared& sh, const W
 #pragma unroll 1
   for (int b0 = 0; b0 < nsurv; b0 += cap_s) {
     const int nb = min(cap_s, nsurv - b0);
-    wt_request_rows(&sh.mbar[0], ring, nb, rest_b, [&](int i) -> const unsigned char* { return wbase + (size_t)s_sidx[b0 + i] * bundle_b + row_b; });
+    wt_request_rows(&sh.mbar[0], ring, rstride, nb, rest_b, [&](int i) -> const unsigned char* { return wbase + (size_t)s_sidx[b0 + i] * bundle_b + row_b; });
     wt_mbar_wait(sh, &sh.mbar[0], ring_phase);
     ring_phase ^= 1u;
     if (gated) {
-      wt_ring_dots<WD>(ring, rest_b, nb, s_x, d, C.piece_len, s_gsum);
+      if (C.mma) {
+        wt_ring_mma<WD>(ring, rstride, nb, s_xs, d, s_part);
+        __syncthreads();
+        wt_fold_parts(s_part, nb, s_gsum);
+      } else {
+        wt_ring_dots<WD>(ring, rstride, nb, s_x, d, C.piece_len, s_gsum);
+      }
       __syncthreads();
       if (tid < nb) {
         const float4 u4 = *reinterpret_cast<const float4*>(s_gsum + tid * 4);
@@ -511,7 +629,7 @@ __device__ __forceinline__ void wt_stream(const WtCall& C, WtShared& sh, const W
       for (int s0 = 0; s0 < nb; ++s0) {
         const float a = s_sact[b0 + s0];
         float f[8];
-        unpack8<WD>(*reinterpret_cast<const uint4*>(dn + (size_t)s0 * rest_b + col * 2), f);
+        unpack8<WD>(*reinterpret_cast<const uint4*>(dn + (size_t)s0 * rstride + col * 2), f);
 #pragma unroll
         for (int e = 0; e < 8; ++e) a8[e] = fmaf(a, f[e], a8[e]);
       }
@@ -1035,6 +1153,7 @@ __global__ void __launch_bounds__(WT_THREADS, 1) ls_token_kernel(const WtLayer* 
   const int tid = threadIdx.x, cta = blockIdx.x, G = gridDim.x;
   const int d = C.d, K = C.K, E = K + 1;
   float* s_x = reinterpret_cast<float*>(smem + C.lay.x_off);
+  uint16_t* s_xs = C.mma ? reinterpret_cast<uint16_t*>(smem + C.lay.xs_off) : nullptr;  // x as three 16-bit terms (tensor-core operand)
   int* s_mine = reinterpret_cast<int*>(smem + C.lay.mine_off);
   constexpr int NW = sizeof(WtLayer) / 4;
   const int n_act = C.gs * K;
@@ -1058,7 +1177,7 @@ __global__ void __launch_bounds__(WT_THREADS, 1) ls_token_kernel(const WtLayer* 
     double sq = 0.0;
     for (int c = tid * 4; c < d; c += WT_THREADS * 4) {
       const float4 v = __ldcg(reinterpret_cast<const float4*>(C.x_in + c));
-      *reinterpret_cast<float4*>(s_x + c) = v;
+      wt_store_x4<WD>(s_x, s_xs, c, v);
       sq += (double)v.x * v.x + (double)v.y * v.y + (double)v.z * v.z + (double)v.w * v.w;
       if (C.tr_x && cta == 0) *reinterpret_cast<float4*>(C.tr_x + c) = v;
     }
@@ -1139,7 +1258,7 @@ __global__ void __launch_bounds__(WT_THREADS, 1) ls_token_kernel(const WtLayer* 
     wt_latent_sums(C, L.r, E, rz);
     if (!last) {
 #pragma unroll 1
-      for (int c = tid * 4; c < d; c += WT_THREADS * 4) *reinterpret_cast<float4*>(s_x + c) = __ldcg(reinterpret_cast<const float4*>(x_out + c));
+      for (int c = tid * 4; c < d; c += WT_THREADS * 4) wt_store_x4<WD>(s_x, s_xs, c, __ldcg(reinterpret_cast<const float4*>(x_out + c)));
     }
     if (tid == 32) {
       const double bh = L.range[0], bs = L.range[1];
