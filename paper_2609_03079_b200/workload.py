@@ -189,7 +189,8 @@ def make_layer(spec: StackSpec, layer: int, svd_device: str = "cpu", down_scale:
     w_down_t = _normal_bits(spec.seed, layer, T_DOWN, (F, d), WEIGHT_STD * down_scale, spec.wdtype)
     b = np.full((F,), gate_bias(spec.activity, d), dtype=np.float32)
     pa, pb = _svd_predictor(bits16_to_f32(w_gate, spec.wdtype), spec.rank, spec.seed, layer, spec.wdtype, svd_device)
-    return LayerArrays(d, F, spec.gated, spec.wdtype, spec.rank, spec.norm_eps, w_gate, w_up, w_down_t, b, pa, pb,
+    # (eps as the fp32 value the C ABI's `float` field carries, so that the oracle and the library see the same number)
+    return LayerArrays(d, F, spec.gated, spec.wdtype, spec.rank, float(np.float32(spec.norm_eps)), w_gate, w_up, w_down_t, b, pa, pb,
                        b.copy(), None, {"spec": spec.name, "layer": layer})
 
 

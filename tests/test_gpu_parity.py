@@ -222,6 +222,31 @@ def test_fp16_non_gated_layer():
     gl.close()
 
 
+def test_fp16_gated_layer_on_the_tensor_core_dot_products():
+    """fp16 weights, gated, d a multiple of 16: the whole-token kernel's gate and up dot products run as fp16 MMAs on x cut
+    into three fp16 terms (scaled by 2^11 per term); tokens of very different magnitudes exercise the scaling."""
+    spec, la = custom_arrays(24, 512, 2048, 64, gated=True, wdtype="fp16", activity=0.15)
+    gl = ls.ls_layer_create(la, DEV)
+    OL = orc.OracleLayer.from_arrays(la)
+    stats = {}
+    toks = wl.make_tokens(spec)
+    for x, scale in zip(toks[:3], (1.0, 1e-3, 300.0)):
+        run_step_and_compare(gl, gl, OL, OL, (x * scale).astype(np.float32), 320, 4, 320, stats)
+    gl.close()
+
+
+def test_feature_wider_than_one_pass_of_the_block():
+    """d = 6144 > 4096 columns: a thread owns more than one group of eight output columns, so the partial output is
+    accumulated in the CTA's global row instead of registers; rows of 12 KB, several ring batches."""
+    spec, la = custom_arrays(25, 6144, 2048, 64, activity=0.2)
+    gl = ls.ls_layer_create(la, DEV)
+    OL = orc.OracleLayer.from_arrays(la)
+    stats = {}
+    for x in wl.make_tokens(spec)[:2]:
+        run_step_and_compare(gl, gl, OL, OL, x, 448, 8, 448, stats)
+    gl.close()
+
+
 def test_batch_union(tiny):
     spec, la, OL, gl, toks = tiny
     stats = {}
