@@ -164,7 +164,9 @@ int32_t ls_sparse_ffn_step(ls_layer *layer, ls_layer *next, const float *d_x, fl
  *   *h_nmiss (nullable, HOST) receives the number of misses: for it the call waits on the calling thread for the decision
  *   (not for the copies), at most LS_OPT_HOST_WAIT_MS (LS_ERR_TIMEOUT otherwise; the request stays enqueued).
  *   LS_ERR_CAPACITY if wanted + protected exceed cache_rows (nothing changes).
- *   (ls_sparse_ffn_step reserves through the same machinery without waiting on the host at all.)
+ *   (ls_sparse_ffn_step reserves through the same machinery without waiting on the host at all; with the gather
+ *   transport its refine-driven requests for the next layer are decided on that layer's copy stream, and every entry
+ *   point here first makes its stream wait for such pending decisions, so callers see them as if they had run in order.)
  *
  * ls_cache_evict: evicts lowest-priority unprotected residents until at least min_free slots are free (fewer when
  *   only protected ones remain); d_evicted (nullable, [cache_rows]) and d_nevicted (nullable) receive them.  Asynchronous.

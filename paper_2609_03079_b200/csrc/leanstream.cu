@@ -487,6 +487,9 @@ int32_t predict_impl(ls_layer* L, const float* d_feature, int B, int k, double* 
     else ls::ls_latent_kernel<1><<<grid, 256, 0, st>>>(L->pred_at, d_feature, d, r, B, L->z, L->sumsq);
     LS_LAUNCHED();
   }
+  // (a cache decision enqueued on the copy stream may still be reading the priorities and the list of the evaluation
+  //  before: the stream joins it here, behind the latents, so that the decision overlaps with whatever ran since)
+  if (L->cache_rows > 0) LS_TRY(ls::cache_join(L->cache, st, g_err));
   {
     const int grid = std::min((F + 7) / 8, L->sm_count * 8);
     const size_t sm = (size_t)B * r * sizeof(double);
@@ -1082,7 +1085,7 @@ int32_t ls_sparse_ffn_step(ls_layer* L, ls_layer* next, const float* d_x, float*
       // fetch rule: the first ceil(count (j+1)/(K+1)) ranks of C^(j) are admitted
       LS_TRY(cache_rc(ls::cache_reserve_async(next->cache, miss_path, next->prio, next->F, idx_out, cnt_out, 0, j + 1, K + 1, next->max_sel,
                                               nullptr, next->status, st, nullptr, g_opt_host_wait_ms.load(std::memory_order_relaxed) * 1e-3,
-                                              g_err, g_launches)));
+                                              g_err, g_launches, /*side=*/true)));
     }
     return LS_OK;
   };

@@ -57,6 +57,8 @@ struct CacheState {
   int32_t* h_res = nullptr;         // pinned [CACHE_HDR]: counters of a request, for the calls that report them
   cudaStream_t copy_stream = nullptr;
   cudaEvent_t ev_list = nullptr, ev_res = nullptr;
+  cudaEvent_t ev_want = nullptr, ev_decided = nullptr;  // a decision kernel on the copy stream: its inputs are ready / it has run
+  bool side_pending = false;        // a decision kernel was enqueued on the copy stream since the last join
   unsigned seq_issued = 0;          // requests enqueued by the calling thread
   unsigned seq_lane = 0;            // requests the I/O lane has taken over (lane thread only)
   std::atomic<long long> lane_copies{0};
@@ -166,11 +168,13 @@ inline void cache_destroy(CacheState& c) {
   cudaFree(c.d_stats); cudaFree(c.d_key); cudaFree(c.d_idx);
   if (c.ev_list) cudaEventDestroy(c.ev_list);
   if (c.ev_res) cudaEventDestroy(c.ev_res);
+  if (c.ev_want) cudaEventDestroy(c.ev_want);
+  if (c.ev_decided) cudaEventDestroy(c.ev_decided);
   if (c.copy_stream) cudaStreamDestroy(c.copy_stream);
   c.h_bundles = c.h_bundles_dev = nullptr; c.h_list = c.h_list_dev = nullptr; c.h_ack = c.h_ack_dev = nullptr; c.h_seq = nullptr; c.h_res = nullptr;
   c.d_slot_of = c.d_neuron_of = nullptr; c.d_nres = nullptr; c.d_exec_idx = c.d_miss_neuron = c.d_victim_slot = c.d_free_list = c.d_list = nullptr;
   c.d_landed = c.d_gdone = nullptr; c.d_stats = nullptr; c.d_key = nullptr; c.d_idx = nullptr;
-  c.ev_list = c.ev_res = nullptr; c.copy_stream = nullptr;
+  c.ev_list = c.ev_res = c.ev_want = c.ev_decided = nullptr; c.copy_stream = nullptr;
 }
 
 inline int32_t cache_create(CacheState& c, int device, int F, int C, size_t bundle_bytes, int max_sel, void* bundles_dev, std::string& err) {
@@ -211,6 +215,8 @@ inline int32_t cache_create(CacheState& c, int device, int F, int C, size_t bund
   LS_CACHE_CUDA(cudaStreamCreateWithFlags(&c.copy_stream, cudaStreamNonBlocking));
   LS_CACHE_CUDA(cudaEventCreateWithFlags(&c.ev_list, cudaEventDisableTiming));
   LS_CACHE_CUDA(cudaEventCreateWithFlags(&c.ev_res, cudaEventDisableTiming));
+  LS_CACHE_CUDA(cudaEventCreateWithFlags(&c.ev_want, cudaEventDisableTiming));
+  LS_CACHE_CUDA(cudaEventCreateWithFlags(&c.ev_decided, cudaEventDisableTiming));
   CopyLane::get().add(&c);
   return 0;
 }
@@ -496,27 +502,60 @@ inline int32_t cache_lane_wait(CacheState& c, unsigned seq, double limit_s, std:
   return 0;
 }
 
+// Makes `st` wait for the decision kernels that were enqueued on the copy stream (`side` requests): everything that reads
+// or changes the cache's tables, its priorities or a request's input list on `st` joins first.
+inline int32_t cache_join(CacheState& c, cudaStream_t st, std::string& err) {
+  if (c.side_pending) {
+    LS_CACHE_CUDA(cudaStreamWaitEvent(st, c.ev_decided, 0));
+    c.side_pending = false;
+  }
+  return 0;
+}
+
+// Enqueues one request: the decision kernel and the transport of its misses.  side = false: the decision kernel runs on
+// `st` (whatever follows on `st` sees its tables).  side = true (gather transport only): `st` only marks the point at
+// which the request's inputs (priorities, wanted list) are ready; the decision kernel runs on the copy stream, off the
+// path of the kernels that follow on `st`, and the caller joins (cache_join) before `st` changes those inputs again or
+// touches the tables.
 inline int32_t cache_reserve_async(CacheState& c, int miss_path, const double* prio, int F, const int32_t* want, const int32_t* count_ptr,
                                    int admit_ranks, int admit_num, int admit_den, int cap, const uint32_t* protect, int* status,
-                                   cudaStream_t st, unsigned* seq_out, double limit_s, std::string& err, std::atomic<int64_t>& launches) {
+                                   cudaStream_t st, unsigned* seq_out, double limit_s, std::string& err, std::atomic<int64_t>& launches,
+                                   bool side = false) {
   const bool lane = miss_path == MISS_PATH_LANE;
+  if (lane) side = false;
   if (lane && c.seq_issued >= 2) {
     const int32_t rc = cache_lane_wait(c, c.seq_issued - 1, limit_s, err);
+    if (rc != 0) return rc;
+  }
+  if (!side) {
+    const int32_t rc = cache_join(c, st, err);
     if (rc != 0) return rc;
   }
   const unsigned seq = ++c.seq_issued;
   const size_t list_ints = CACHE_HDR + 2 * (size_t)c.max_sel;
   int32_t* h_list = lane ? c.h_list_dev + (size_t)(seq & 1u) * list_ints : nullptr;
   int32_t* d_list = c.d_list + (size_t)(seq & 1u) * list_ints;
-  ls_cache_reserve_kernel<<<1, TK_THREADS, cache_kernel_smem(F, cap), st>>>(
+  cudaStream_t dst = st;
+  if (side) {
+    LS_CACHE_CUDA(cudaEventRecord(c.ev_want, st));
+    LS_CACHE_CUDA(cudaStreamWaitEvent(c.copy_stream, c.ev_want, 0));
+    dst = c.copy_stream;
+  }
+  ls_cache_reserve_kernel<<<1, TK_THREADS, cache_kernel_smem(F, cap), dst>>>(
       prio, F, c.C, want, count_ptr, admit_ranks, admit_num, admit_den, cap, protect, c.d_slot_of, c.d_neuron_of, c.d_nres, c.d_exec_idx,
       c.d_miss_neuron, c.d_victim_slot, c.d_free_list, d_list, c.d_stats, seq, h_list, lane ? c.h_ack_dev : c.d_landed, c.bundle_bytes,
       c.d_key, c.d_idx, status);
   launches.fetch_add(1, std::memory_order_relaxed);
   LS_CACHE_CUDA(cudaPeekAtLastError());
+  if (side) {
+    LS_CACHE_CUDA(cudaEventRecord(c.ev_decided, c.copy_stream));
+    c.side_pending = true;
+  }
   if (!lane) {
-    LS_CACHE_CUDA(cudaEventRecord(c.ev_list, st));
-    LS_CACHE_CUDA(cudaStreamWaitEvent(c.copy_stream, c.ev_list, 0));
+    if (!side) {
+      LS_CACHE_CUDA(cudaEventRecord(c.ev_list, st));
+      LS_CACHE_CUDA(cudaStreamWaitEvent(c.copy_stream, c.ev_list, 0));
+    }
     ls_cache_gather_kernel<<<128, 256, 0, c.copy_stream>>>(d_list, static_cast<const unsigned char*>(c.h_bundles_dev),
                                                            static_cast<unsigned char*>(c.bundles_dev), c.bundle_bytes, c.d_landed, c.d_gdone,
                                                            c.d_stats, seq);
@@ -551,6 +590,7 @@ inline const int32_t* cache_list_header(const CacheState& c, unsigned seq) {
 // Makes `st` wait (on the device, bounded) until the rows of every request enqueued so far are in their slots.
 inline int32_t cache_wait(CacheState& c, int* status, cudaStream_t st, std::string& err, std::atomic<int64_t>& launches) {
   if (c.seq_issued == 0) return 0;
+  { const int32_t rc = cache_join(c, st, err); if (rc != 0) return rc; }
   ls_cache_wait_kernel<<<1, 32, 0, st>>>(c.d_landed, c.seq_issued, status);
   launches.fetch_add(1, std::memory_order_relaxed);
   LS_CACHE_CUDA(cudaPeekAtLastError());
@@ -559,6 +599,7 @@ inline int32_t cache_wait(CacheState& c, int* status, cudaStream_t st, std::stri
 
 inline int32_t cache_evict(CacheState& c, const double* prio, int F, int min_free, const uint32_t* protect, int32_t* d_evicted,
                            int32_t* d_nevicted, int* /*status*/, cudaStream_t st, std::string& err, std::atomic<int64_t>& launches) {
+  { const int32_t rc = cache_join(c, st, err); if (rc != 0) return rc; }
   ls_cache_evict_kernel<<<1, TK_THREADS, cache_kernel_smem(F, 0), st>>>(prio, F, c.C, min_free, protect, c.d_slot_of, c.d_neuron_of,
                                                                          c.d_nres, d_evicted, d_nevicted, c.d_stats, c.d_key, c.d_idx);
   launches.fetch_add(1, std::memory_order_relaxed);
@@ -576,6 +617,7 @@ inline int32_t cache_stats(CacheState& c, long long out[8], std::string& err) {
 
 inline int32_t cache_lookup(CacheState& c, int F, const int32_t* d_idx, int n, int32_t* d_slot, int32_t* d_nhit, int* status,
                             cudaStream_t st, std::string& err, std::atomic<int64_t>& launches) {
+  { const int32_t rc = cache_join(c, st, err); if (rc != 0) return rc; }
   ls_cache_lookup_kernel<<<1, 1024, 0, st>>>(c.d_slot_of, F, d_idx, n, d_slot, d_nhit, status);
   launches.fetch_add(1, std::memory_order_relaxed);
   LS_CACHE_CUDA(cudaPeekAtLastError());
@@ -583,6 +625,7 @@ inline int32_t cache_lookup(CacheState& c, int F, const int32_t* d_idx, int n, i
 }
 
 inline int32_t cache_snapshot(CacheState& c, int F, uint32_t* mask, cudaStream_t st, std::string& err, std::atomic<int64_t>& launches) {
+  { const int32_t rc = cache_join(c, st, err); if (rc != 0) return rc; }
   ls_cache_snapshot_kernel<<<8, 256, 0, st>>>(c.d_slot_of, F, mask);
   launches.fetch_add(1, std::memory_order_relaxed);
   LS_CACHE_CUDA(cudaPeekAtLastError());
