@@ -461,6 +461,7 @@ int32_t fused_step(ls_layer* L, ls_layer* next, const float* d_x, float* d_x_out
   a.n_mat = L->n_mat; a.F = L->F; a.norm = L->norm; a.act = L->act; a.eps = L->eps;
   a.At_sl = next->pred_at_sl; a.Bt_pad = next->pred_bt_pad; a.pc = next->pred_c;
   a.r = next->r; a.Fn = next->F; a.norm_n = next->norm; a.eps_n = next->eps;
+  a.per = (next->F + L->sm_count - 1) / L->sm_count;
   a.range = next->wt_range;
   a.status = L->status;
   c.cuts = D->cuts1; c.sellist = next->tmp_idx; c.xbuf = nullptr;
@@ -696,6 +697,7 @@ int32_t ls_stack_create(ls_layer* const* layers, int32_t n_layers, ls_stack** ou
     a.n_mat = L->n_mat; a.F = L->F; a.norm = L->norm; a.act = L->act; a.eps = L->eps;
     a.At_sl = next->pred_at_sl; a.Bt_pad = next->pred_bt_pad; a.pc = next->pred_c;
     a.r = next->r; a.Fn = next->F; a.norm_n = next->norm; a.eps_n = next->eps;
+    a.per = (next->F + L->sm_count - 1) / L->sm_count;
     a.range = S->ranges + 2 * n;
     a.status = L->status;
     hr[2 * n] = 1.0;                          // scores binned over [-1, 1] until a launch has observed their range

@@ -81,6 +81,7 @@ struct WtLayer {  // one per layer of the stack (device array)
   // predictor of the layer this one refines (the next layer; the last layer refines itself)
   const uint16_t* At_sl; const uint16_t* Bt_pad; const float* pc;  // Bt_pad: rows of wt_brow_bytes(r) bytes, zero padded
   int r, Fn, norm_n; float eps_n;
+  int per;  // ceil(Fn / CTAs): the neurons of that predictor one CTA scores (computed on the host: no division on the device)
   double* range;  // [2] {hi, scale} of the score bins, refreshed by every launch for the next one
   int* status;
 };
@@ -127,6 +128,7 @@ struct WtShared {
   unsigned long long mbar[3];  // transaction barriers of the bulk copies: rows into the ring, the A slices, the B^T rows
   int dead;               // a wait timed out: no more waiting
   int nmine, nsurv;
+  int my_lo, my_hi, keff_shared;  // this CTA's ranks [my_lo, my_hi) of a selection of keff_shared neurons
   int wcnt[WT_WARPS];
   int blo, bhi, ncand, slow, found;
   float inv_x;            // 1 / rms of the layer's input
@@ -467,7 +469,7 @@ __device__ __forceinline__ void wt_fold_parts(const float* part, int nrow, float
 __device__ __forceinline__ void wt_fetch_predictor(const WtCall& C, WtShared& sh, const WtLayer& L, unsigned char* smem) {
   const int tid = threadIdx.x, G = gridDim.x, d = C.d;
   const int nsl = (d + 31) >> 5, slice_b = L.r * 64;  // bytes per slice: 32 columns of r 16-bit entries
-  const int per = (L.Fn + G - 1) / G, n0 = min(L.Fn, (int)blockIdx.x * per), n1 = min(L.Fn, n0 + per);
+  const int per = L.per, n0 = min(L.Fn, (int)blockIdx.x * per), n1 = min(L.Fn, n0 + per);
   if (tid == 0) {
     unsigned char* s_a = smem + C.lay.u_off;
     wt_fence_async();
@@ -499,7 +501,7 @@ __device__ __forceinline__ void wt_fetch_predictor(const WtCall& C, WtShared& sh
 // The same rows of B^T once more, by ordinary asynchronous copies (after a degenerate selection borrowed their place).
 __device__ __noinline__ void wt_refetch_b(const WtCall& C, const WtLayer& L, unsigned char* smem) {
   const int G = gridDim.x;
-  const int per = (L.Fn + G - 1) / G, n0 = min(L.Fn, (int)blockIdx.x * per), n1 = min(L.Fn, n0 + per);
+  const int per = L.per, n0 = min(L.Fn, (int)blockIdx.x * per), n1 = min(L.Fn, n0 + per);
   const int RB = wt_brow_bytes(L.r);
   const int npieces = (((n1 - n0 + 7) >> 3) * 8) * (RB >> 4);
   unsigned char* s_b = smem + C.lay.u_off + C.lay.b_off;
@@ -811,7 +813,7 @@ __device__ __noinline__ void wt_score_evals(const WtCall& C, WtShared& sh, const
   const int RS = wt_feat_stride(r), RB = wt_brow_bytes(r);
   const int ntile = wt_tiles(ne), nplain = wt_plain(ne), rows = wt_rows(ne);
   const int nblk = (r + 31) >> 5;
-  const int per = (Fn + G - 1) / G, n0 = min(Fn, (int)blockIdx.x * per), n1 = min(Fn, n0 + per);
+  const int per = L.per, n0 = min(Fn, (int)blockIdx.x * per), n1 = min(Fn, n0 + per);
   const int n_mt = (n1 - n0 + 7) >> 3, per8 = n_mt * 8;
   if (ne <= 0) return;
   {
@@ -829,6 +831,7 @@ __device__ __noinline__ void wt_score_evals(const WtCall& C, WtShared& sh, const
     for (int i = tid; i < rows * RS; i += WT_THREADS) s_z[i] = 0.0;
     __syncthreads();
   }
+  const double ss = tid < ne ? __ldcg(C.z + (e0 + tid) * rz + r) : 0.0;  // (requested before the latents: one round trip, not two)
 #pragma unroll 1
   for (int e = warp; e < ne; e += WT_WARPS) {  // (plain loads: an asynchronous copy would also wait for the rows in flight)
     const double* zr = C.z + (e0 + e) * rz;
@@ -845,10 +848,7 @@ __device__ __noinline__ void wt_score_evals(const WtCall& C, WtShared& sh, const
       }
     }
   }
-  if (tid < ne) {
-    const double ss = __ldcg(C.z + (e0 + tid) * rz + r);
-    sh.inv[e0 + tid] = L.norm_n == 0 ? wt_rsqrt(ss * C.inv_d + (double)L.eps_n) : 1.0;
-  }
+  if (tid < ne) sh.inv[e0 + tid] = L.norm_n == 0 ? wt_rsqrt(ss * C.inv_d + (double)L.eps_n) : 1.0;
   if (tid == 0) { sh.kmin = 0xffffffffffffffffULL; sh.kmax = 0ULL; }
   __syncthreads();
   // raw dot products: a warp per m-tile of eight neurons, all blocks of the rank
@@ -1229,6 +1229,7 @@ __global__ void __launch_bounds__(WT_THREADS, 1) ls_token_kernel(const WtLayer* 
     }
   };
 
+  if (tid == 0) sh.keff_shared = -1;  // (this CTA's ranks of the next selection are kept for as long as its size stays the same)
 #pragma unroll 1
   for (int n = 0; n < C.n_layers; ++n) {
     const WtLayer& L = sh.L[n & 1];
@@ -1286,8 +1287,14 @@ __global__ void __launch_bounds__(WT_THREADS, 1) ls_token_kernel(const WtLayer* 
     if (sh.dead) return;
     if (stamps) wt_stamp(C, n, 8);
     // ---- P4
-    int lo, hi;
-    wt_share(keff, K, C.gs, cta, lo, hi);
+    if (keff != sh.keff_shared) {  // (three integer divisions: once per launch unless the layers differ in size)
+      int l0, h0;
+      wt_share(keff, K, C.gs, cta, l0, h0);
+      __syncthreads();
+      if (tid == 0) { sh.my_lo = l0; sh.my_hi = h0; sh.keff_shared = keff; }
+      __syncthreads();
+    }
+    const int lo = sh.my_lo, hi = sh.my_hi;
     if (tid == 0) sh.inv_x = (float)sh.inv[K];
     unsigned long long* cuts = C.cuts + (size_t)n * E;  // the keys of the last members of this layer's refined sets
     if (!wt_select(C, sh, K, L.Fn, keff, lo, hi, C.lay.mine_off, false, cuts + K)) {
