@@ -514,8 +514,24 @@ __device__ __noinline__ void wt_refetch_b(const WtCall& C, const WtLayer& L, uns
 template <int WD>
 __device__ __noinline__ void wt_score_evals(const WtCall& C, WtShared& sh, const WtLayer& L, int e0, int ne, bool last);
 
+// Requests the gate rows of this CTA's neurons g0, g0 + 1, ... (as many as a ring batch holds) of layer L.  Called by the
+// stream phase, and for the first batch already at the end of the selection that produced the list, so that the rows
+// travel while the layer's bookkeeping is done.
+__device__ __forceinline__ void wt_request_gate(const WtCall& C, WtShared& sh, const WtLayer& L, unsigned char* smem, int g0, int nmine) {
+  const int* s_mine = reinterpret_cast<const int*>(smem + C.lay.mine_off);
+  const int row_b = C.d * 2, gstride = row_b + 16;
+  const int cap_g = min(WT_MMA_ROWS, C.ring_bytes / gstride);
+  const size_t bundle_b = (size_t)L.n_mat * row_b;
+  const unsigned char* wbase = reinterpret_cast<const unsigned char*>(L.bundles);
+  wt_request_rows(&sh.mbar[0], smem + C.lay.u_off, gstride, min(cap_g, nmine - g0), row_b, [&](int i) -> const unsigned char* {
+    const int v = s_mine[g0 + i];
+    return v >= 0 ? wbase + (size_t)v * bundle_b : nullptr;
+  });
+}
+
 template <int WD>
-__device__ __forceinline__ void wt_stream(const WtCall& C, WtShared& sh, const WtLayer& L, unsigned char* smem, bool active, uint32_t& ring_phase) {
+__device__ __forceinline__ void wt_stream(const WtCall& C, WtShared& sh, const WtLayer& L, unsigned char* smem, bool active, uint32_t& ring_phase,
+                                          bool first_requested) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int d = C.d;
   const float* s_x = reinterpret_cast<const float*>(smem + C.lay.x_off);
@@ -546,10 +562,7 @@ __device__ __forceinline__ void wt_stream(const WtCall& C, WtShared& sh, const W
 #pragma unroll 1
   for (int g0 = 0; g0 < nmine; g0 += cap_g) {
     const int ng = min(cap_g, nmine - g0);
-    wt_request_rows(&sh.mbar[0], ring, gstride, ng, row_b, [&](int i) -> const unsigned char* {
-      const int v = s_mine[g0 + i];
-      return v >= 0 ? wbase + (size_t)v * bundle_b : nullptr;
-    });
+    if (g0 > 0 || !first_requested) wt_request_gate(C, sh, L, smem, g0, nmine);
     wt_mbar_wait(sh, &sh.mbar[0], ring_phase);
     ring_phase ^= 1u;
     if (C.mma) {
@@ -1239,7 +1252,7 @@ __global__ void __launch_bounds__(WT_THREADS, 1) ls_token_kernel(const WtLayer* 
     if (stamps) wt_stamp(C, n, 0);
     // ---- S (and, on the CTAs without rows, the refined sets of the layer before)
     if (n > 0 && !active) refined_sets(n - 1, sh.L[(n - 1) & 1], 0);
-    wt_stream<WD>(C, sh, L, smem, active, ring_phase);
+    wt_stream<WD>(C, sh, L, smem, active, ring_phase, n > 0);
     if (stamps) wt_stamp(C, n, 1);
     wt_grid_sync(C, sh, ++epoch * G);
     if (sh.dead) return;
@@ -1256,10 +1269,17 @@ __global__ void __launch_bounds__(WT_THREADS, 1) ls_token_kernel(const WtLayer* 
     if (sh.dead) return;
     if (stamps) wt_stamp(C, n, 4);
     // ---- P2
+    // (the next layer's input is requested before the sums, so that the two round trips to L2 overlap)
+    const int xc0 = tid * 4, xc1 = xc0 + WT_THREADS * 4;
+    float4 xv0 = make_float4(0.f, 0.f, 0.f, 0.f), xv1 = xv0;
+    if (!last && xc0 < d) xv0 = __ldcg(reinterpret_cast<const float4*>(x_out + xc0));
+    if (!last && xc1 < d) xv1 = __ldcg(reinterpret_cast<const float4*>(x_out + xc1));
     wt_latent_sums(C, L.r, E, rz);
     if (!last) {
+      if (xc0 < d) wt_store_x4<WD>(s_x, s_xs, xc0, xv0);
+      if (xc1 < d) wt_store_x4<WD>(s_x, s_xs, xc1, xv1);
 #pragma unroll 1
-      for (int c = tid * 4; c < d; c += WT_THREADS * 4) wt_store_x4<WD>(s_x, s_xs, c, __ldcg(reinterpret_cast<const float4*>(x_out + c)));
+      for (int c = xc1 + WT_THREADS * 4; c < d; c += WT_THREADS * 4) wt_store_x4<WD>(s_x, s_xs, c, __ldcg(reinterpret_cast<const float4*>(x_out + c)));
     }
     if (tid == 32) {
       const double bh = L.range[0], bs = L.range[1];
@@ -1305,6 +1325,7 @@ __global__ void __launch_bounds__(WT_THREADS, 1) ls_token_kernel(const WtLayer* 
       __syncthreads();
     }
     if (stamps) wt_stamp(C, n, 9);
+    if (!last && hi > lo) wt_request_gate(C, sh, sh.L[(n + 1) & 1], smem, 0, hi - lo);  // (the next layer's first gate rows: on their way)
     if (tid == 0) sh.nmine = hi - lo;
     if (last || C.tr_sel || C.tr_masks || C.tr_counts) wt_export_selection(C, s_mine, n, lo, hi - lo, keff, last);
     if (cta == 0 && tid < 32) wt_update_range(C, L);
