@@ -52,6 +52,9 @@ def parse_args():
     ap.add_argument("--no-graph", action="store_true", help="launch every call from the host instead of one CUDA graph per token")
     ap.add_argument("--per-layer", action="store_true", help="one kernel per layer (ls_sparse_ffn_step) instead of one per token")
     ap.add_argument("--phases", action="store_true", help="also print the per-phase timeline of the whole-token kernel (stderr)")
+    ap.add_argument("--predictors", action="store_true",
+                    help="also time one ranking of a layer's neurons by the linear predictor (ls_predict) and by a stacked hashing "
+                         "predictor of the paper's default shape with random tables (ls_hash_predict); stderr")
     ap.add_argument("--miss-path", default="gather", choices=["gather", "lane"],
                     help="cached workloads: misses by a gather kernel reading pinned host memory, or by the host I/O lane (cudaMemcpyAsync)")
     ap.add_argument("--cpu-sample-layers", type=int, default=2)
@@ -282,6 +285,31 @@ def phase_table(ls, stack, layers, x_buf, X0, sels, K, k):
     return rows
 
 
+def predictor_times(ls, wl, torch, spec, la, layer, x_buf, k, local, reps=200):
+    """One ranking of a layer's neurons (scores of all d_ff neurons + exact top-k) by each predictor, CUDA events around
+    `reps` back-to-back calls on the current stream.  The hashing predictor has the paper's default shape (five layers,
+    tau = 8, 256-bit codes) and random tables: same arithmetic and memory traffic as a trained one, no predictive value."""
+    ha = wl.make_hash_predictor(la, spec.seed, 0)
+    hp = ls.ls_hash_predictor_create(ha, local)
+    sel = ls.Selection(spec.d_ff, k, local)
+    out = {}
+    for name, call in (("ls_predict (rank-%d linear, fp64)" % spec.rank, lambda: ls.ls_predict(layer, x_buf, k, sel)),
+                       ("ls_hash_predict (5 layers, tau 8, 256-bit codes)", lambda: ls.ls_hash_predict(hp, x_buf.view(-1), k, sel))):
+        for _ in range(10):
+            call()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(reps):
+            call()
+        e1.record()
+        torch.cuda.synchronize()
+        out[name] = e0.elapsed_time(e1) / reps * 1e3
+        print(f"  {name:52s} {out[name]:8.2f} us per ranking of {spec.d_ff} neurons (k = {k})", file=sys.stderr)
+    hp.close()
+    return out
+
+
 def run_resident(args, ls, wl, replicas, torch, dist, world, rank, local, dev, spec):
     n_layers = args.layers or spec.n_layers
     K, k, d = args.chunks, args.k or spec.k, spec.d_model
@@ -428,6 +456,9 @@ def run_resident(args, ls, wl, replicas, torch, dist, world, rank, local, dev, s
             for nm, med, mx in phases:
                 print(f"  {nm:42s} median {med:7.2f} us   slowest CTA {mx:7.2f} us", file=sys.stderr)
 
+        if args.predictors and keep_host:
+            predictor_times(ls, wl, torch, spec, keep_host[0], layers[0], x_buf, k, local)
+
         arrays = [keep_host[l] for l in sorted(keep_host)]
         cpu = cpu_baseline(arrays, spec, K, n_layers, 48 * len(arrays), k=k)  # fifteen to twenty seconds of CPU work
 
@@ -528,14 +559,31 @@ def run_cached(args, ls, wl, replicas, torch, dist, world, rank, local, dev, spe
     x_buf = torch.zeros(B, d, dtype=torch.float32, device=dev)
     sels = [ls.Selection(F, max_sel, local) for _ in range(2)]
 
-    def decode_token(t, record=None):
+    nwords = (F + 31) // 32
+    snap = [torch.zeros(nwords, dtype=torch.int32, device=dev) for _ in range(2)]
+
+    def bits(m):
+        return int(np.unpackbits(m.cpu().numpy().view(np.uint8)).sum())
+
+    def decode_token(t, record=None, redund=None):
         x_buf.copy_(X0[t])
         ls.ls_predict(layers[0], x_buf, k, sels[0])
         for n in range(n_layers):
             nxt = layers[n + 1] if n + 1 < n_layers else layers[n]
             if record is not None:
                 record[n].append(sels[n % 2].order().tolist())
+            watch = redund is not None and nxt is not layers[n]
+            if watch:
+                ls.ls_cache_snapshot(nxt, snap[0])  # the next layer's residents before this layer's refinements prefetch
             ls.ls_sparse_ffn_step(layers[n], nxt, x_buf, x_buf, sels[n % 2], K, k, sels[(n + 1) % 2], None)
+            if watch:
+                # loading redundancy (Section 4.3): rows the refinements brought in that the final set does not use, over the
+                # rows the final set truly lacked
+                ls.ls_cache_snapshot(nxt, snap[1])
+                final = sels[(n + 1) % 2].mask
+                fetched = snap[1] & ~snap[0]
+                redund[0] += bits(fetched & ~final)
+                redund[1] += bits(final & ~snap[0])
 
     def stats_sum():
         tot = {}
@@ -577,8 +625,9 @@ def run_cached(args, ls, wl, replicas, torch, dist, world, rank, local, dev, spe
         win = min(16, args.steps)
         record = [[] for _ in range(n_layers)]
         s0 = stats_sum()
+        redund = [0, 0]
         for t in range(warm, warm + win):
-            decode_token(t, record)
+            decode_token(t, record, redund if t < warm + 4 else None)
         torch.cuda.synchronize()
         s1 = stats_sum()
         ours_window = (s1["misses"] - s0["misses"]) / max(1, (s1["hits"] - s0["hits"]) + (s1["misses"] - s0["misses"]))
@@ -646,7 +695,10 @@ def run_cached(args, ls, wl, replicas, torch, dist, world, rank, local, dev, spe
                       "miss_bytes_per_layer": miss_bytes / (args.steps * n_layers),
                       "lru_miss_ratio_same_trace": lru, "miss_ratio_in_that_window": ours_window,
                       "window": f"{win} tokens after the timed region, every {max(1, n_layers // 8)}th layer for the LRU replay",
-                      "loading_redundancy": None, "loading_redundancy_note": "needs the per-stage fetch lists; reported by the tests on the small stacks"},
+                      "loading_redundancy": (redund[0] / redund[1]) if redund[1] else None,
+                      "loading_redundancy_note": "first 4 tokens of that window, every layer boundary: rows the refinements prefetched that the "
+                                                 "final set does not use / rows the final set lacked before them (snapshots of the next "
+                                                 "layer's resident set around each step)"},
             "roofline": {"bound": "host link", "achieved": miss_bytes / t_s / 1e9, "peak": link, "unit": "GB/s", "frac": miss_bytes / t_s / 1e9 / link,
                          "peak_kind": "measured here: one 256 MiB pinned host-to-device copy, best of five", "traffic": None,
                          "hbm": {"selected_row_bytes_gbs": sel_bytes / t_s / 1e9, "peak": peaks["hbm_gbs"], "frac": sel_bytes / t_s / 1e9 / peaks["hbm_gbs"], "peak_kind": peak_kind},

@@ -359,14 +359,25 @@ int32_t create_impl(const ls_layer_desc* D, ls_layer* L) {
 // users have disjoint lifetimes (the A slices, the latents of all evaluations, the selection's work area, the general
 // top-k's work area).
 struct TokenShape { int d, sm_count, r_max, f_max, ns_cta; };
-bool token_layout(const TokenShape* S, int K, ls::WtSmem* out) {
+bool token_layout_try(const TokenShape* S, int K, bool mma, ls::WtSmem* out);
+// The shared-memory plan: with the tensor-core operand copy of x when d allows it and everything fits, else without
+// (the dot products of the stream phase then run as FMA loops).
+bool token_layout(const TokenShape* S, int K, ls::WtSmem* out, int* mma_out = nullptr) {
+  if (S->d % 16 == 0 && token_layout_try(S, K, true, out)) {
+    if (mma_out) *mma_out = 1;
+    return true;
+  }
+  if (mma_out) *mma_out = 0;
+  return token_layout_try(S, K, false, out);
+}
+bool token_layout_try(const TokenShape* S, int K, bool mma, ls::WtSmem* out) {
   const int E = K + 1, G = S->sm_count;
   ls::WtSmem L{};
   size_t o = 0;
   auto take = [&](size_t bytes) { const size_t at = o; o += (bytes + 127) & ~(size_t)127; return (unsigned)at; };
   L.x_off = take((size_t)S->d * 4);
-  L.xs_off = take((size_t)((S->d + 15) / 16) * 96);
-  L.part_off = take((size_t)ls::WT_WARPS * ls::WT_MMA_ROWS * 4);
+  L.xs_off = take(mma ? (size_t)((S->d + 15) / 16) * 96 : 0);
+  L.part_off = take(mma ? (size_t)ls::WT_WARPS * ls::WT_MMA_ROWS * 4 : 0);
   L.xt_off = take((size_t)(ls::WT_MAXE + 1) * ls::WT_XBLK * 8);
   L.dm_off = take((size_t)ls::WT_WARPS * 32 * 4);
   L.mine_off = take((size_t)ls::WT_MAXMINE * (4 + 16 + 4 + 4) + 32 * 4);
@@ -408,10 +419,9 @@ int32_t launch_token(const TokenShape* shp, int device, int wd, const ls::WtLaye
     return fail(LS_ERR_INVALID, "%s: selection too long for the whole-token kernel", who);
   DeviceScratch* D = nullptr;
   LS_TRY(device_scratch(device, &D));
-  if (!token_layout(shp, K, &c.lay)) return fail(LS_ERR_STATE, "%s: %d stages do not fit the whole-token kernel's shared memory", who, K);
+  if (!token_layout(shp, K, &c.lay, &c.mma)) return fail(LS_ERR_STATE, "%s: %d stages do not fit the whole-token kernel's shared memory", who, K);
   c.n_layers = n_layers; c.d = shp->d; c.K = K; c.k_next = k_next; c.gs = gs;
   c.piece_len = ((shp->d + 3) / 4 + 255) / 256 * 256;
-  c.mma = shp->d % 16 == 0 ? 1 : 0;
   c.ring_bytes = (int)(c.lay.total - c.lay.u_off);
   c.inv_d = 1.0 / (double)shp->d;
   c.x_in = d_x; c.x_out = d_x_out;

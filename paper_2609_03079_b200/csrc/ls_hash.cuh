@@ -62,9 +62,12 @@ __global__ void __launch_bounds__(256) ls_hash_layers_kernel(const double* __res
   if (tid < words) y_out[tid] = s_y[tid];
 }
 
-// Priorities: scores[i] = d - 2 * popcount(y XOR codes[i]) for every neuron.
+// Priorities: s_i = d - 2 * popcount(y XOR codes[i]) for every neuron (to scores_user, nullable).  The priorities are
+// small integers with hundreds of neurons per value; the ranking key written to `keys` is s_i * F + (F - 1 - i), an exact
+// integer in fp64 whose order is the library's total order (priority descending, index ascending) without any ties, so
+// the binned top-k that follows meets evenly filled bins instead of a few huge ones.
 __global__ void __launch_bounds__(256) ls_hash_scores_kernel(const uint32_t* __restrict__ y, const uint32_t* __restrict__ codes, int words, int F,
-                                                            double* __restrict__ scores, double* __restrict__ scores_user) {
+                                                            double* __restrict__ keys, double* __restrict__ scores_user) {
   __shared__ uint32_t s_y[HASH_MAX_WORDS];
   if (threadIdx.x < words) s_y[threadIdx.x] = y[threadIdx.x];
   __syncthreads();
@@ -80,7 +83,7 @@ __global__ void __launch_bounds__(256) ls_hash_scores_kernel(const uint32_t* __r
       for (int q = 0; q < words; ++q) diff += __popc(__ldg(c + q) ^ s_y[q]);
     }
     const double s = (double)(words * 32 - 2 * diff);
-    scores[i] = s;
+    keys[i] = s * (double)F + (double)(F - 1 - i);
     if (scores_user) scores_user[i] = s;
   }
 }
