@@ -1,16 +1,19 @@
 // Whole-token kernel: every layer of a resident stack for one decode token in ONE cooperative launch (batch 1).
 //
 // Two costs shape it.  A grid barrier costs about 2,300 SM clocks on this GPU whatever its form (one L2 round trip to
-// arrive, one to see the last arrival), as long as a layer's whole weight traffic takes at full HBM speed; and code that a
-// layer executes once streams into the SM at about six clocks per instruction unless the layer's whole path fits the
-// instruction cache (32 to 48 KB).  So a layer step has FOUR barriers, the fewest the data flow allows, and every phase is
-// a handful of small rolled loops; rare paths (trace export, slow selection) are out of line.
+// arrive, one to see the last arrival), as long as a layer's whole weight traffic takes at full HBM speed; and with one
+// CTA of sixteen warps per SM every instruction on the path that all warps execute costs four to five clocks.  So a layer
+// step has FOUR barriers, the fewest the data flow allows, every phase is a handful of small rolled loops, whatever can
+// be computed once (on the host, or per launch) is, and rare paths (trace export, slow selection) are out of line.
 //
 //   S  stream    The K priority stages of the layer (Eq. 1) run concurrently on K groups of CTAs (the output is a sum over
 //                hidden neurons, Section 3.2.2, so only stage MEMBERSHIP defines the partial features of Eq. 2).  A CTA
-//                owns a contiguous slice of the ranks of one stage.  Rows go straight from global memory to registers with
-//                128-bit loads, a dozen in flight per thread: gate rows first, then the up and down rows of the neurons
-//                that survive the ReLU only.  The CTA's partial output goes to its own row of a scratch array.
+//                owns a contiguous slice of the ranks of one stage.  Rows travel global -> shared memory as bulk copies
+//                (one instruction per row, completion on a transaction barrier): gate rows first (requested as soon as
+//                the selection that lists them exists), then the up and down rows of the neurons that survive the
+//                activation only.  Dot products run on the 16-bit tensor cores with x cut exactly into three 16-bit
+//                terms.  The CTA's partial output goes to its own row of a scratch array.  CTAs without rows establish
+//                the refined sets j < K of the layer before meanwhile.
 //      -- barrier 1 --
 //   P1 feature   The feature is cut into slices of 32 columns, one per CTA.  The owner adds the partial outputs of every
 //                stage's CTAs in a fixed order, forms x~^(j) = x~^(j-1) + dm^(j), j = 0..K (Eq. 2), writes x_out = x~^(K)
@@ -28,7 +31,7 @@
 //                that cover the slice, their members, exact comparison of the members' keys.  Nothing is exchanged, so
 //                the next layer's stream phase starts without a further barrier.  The refined sets of the evaluations
 //                j < K are established by the same routine (the slice being the set's last rank) during the next layer's
-//                P1, on CTAs that own no slice of the feature.
+//                stream phase on the CTAs that have no rows, or during its P1 on CTAs that own no slice of the feature.
 //
 // A selection whose bins are too full for this (ties, a score range that moved) takes a slower, equally exact route
 // through one CTA and an extra barrier; the decision is taken from the same histogram by every CTA alike.
