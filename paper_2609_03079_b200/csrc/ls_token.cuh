@@ -485,6 +485,9 @@ __device__ __forceinline__ void wt_fetch_predictor(const WtCall& C, WtShared& sh
       for (int s = blockIdx.x, si = 0; s < nsl; s += G, ++si)
         wt_bulk_load(s_a + (size_t)si * slice_b, reinterpret_cast<const unsigned char*>(L.At_sl) + (size_t)s * slice_b, slice_b, &sh.mbar[1]);
     }
+  }
+  if (tid == 32) {  // (a thread of another warp: the two requests go out side by side)
+    wt_fence_async();
     const int RB = wt_brow_bytes(L.r);
     const uint32_t b_bytes = (uint32_t)(((n1 - n0 + 7) >> 3) * 8) * RB;
     wt_mbar_expect(&sh.mbar[2], b_bytes);
