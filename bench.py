@@ -244,6 +244,7 @@ def parity_gate_stack(ls, wl, spec, host_arrays, stack, layers, x_buf, X0, sels,
     checked = 0
     idxs = sorted(host_arrays)
     OL = {l: orc.OracleLayer.from_arrays(host_arrays[l]) for l in idxs}
+    quality = {"stage": [f"{j}/{K}" for j in range(K + 1)], "importance_ratio": [], "top10_recall": []}
     for l in idxs:
         order = S[l, :k].astype(np.int64)
         if order.tolist() != orc.topk_order(orc.predictor_scores(OL[l], X[l]), k).tolist():
@@ -257,12 +258,23 @@ def parity_gate_stack(ls, wl, spec, host_arrays, stack, layers, x_buf, X0, sels,
             if not ok:
                 raise RuntimeError(f"parity gate: partial feature {j} of layer {l} off (rel-L2 {rel:.2e})")
         if l + 1 in OL:
+            # what the next layer truly activates on its real input: the yardstick of the paper's validation across
+            # refinement steps (Section 4.3: stages 0/K ... K/K, Importance Ratio and recall of the top 10 %)
+            Ln = OL[l + 1]
+            true_abs = np.abs(orc.neuron_activations(Ln, orc.mlp_input(Ln, X[l + 1]), np.arange(Ln.d_ff)))
             for j in range(K + 1):
-                want = set(orc.topk_order(orc.predictor_scores(OL[l + 1], XT[l, j]), k).tolist())
-                if mask_to_set(M[l, j], spec.d_ff) != want:
+                got = mask_to_set(M[l, j], spec.d_ff)
+                want = set(orc.topk_order(orc.predictor_scores(Ln, XT[l, j]), k).tolist())
+                if got != want:
                     raise RuntimeError(f"parity gate: refined set {j} of layer {l} differs from the oracle")
+                if quality is not None and not quality["importance_ratio"][j:]:
+                    quality["importance_ratio"].append(round(orc.importance_ratio(sorted(got), true_abs), 4))
+                    quality["top10_recall"].append(round(orc.top_fraction_recall(sorted(got), true_abs, 0.10), 4))
         checked += 1
-    return {"layers_checked": checked, "token": 1, "what": "selections and refined sets bit-exact, outputs within rel-L2 1e-3"}
+    out = {"layers_checked": checked, "token": 1, "what": "selections and refined sets bit-exact, outputs within rel-L2 1e-3"}
+    if quality is not None and quality["importance_ratio"]:
+        out["refine_quality_layer0_to_1"] = quality
+    return out
 
 
 def phase_table(ls, stack, layers, x_buf, X0, sels, K, k):
