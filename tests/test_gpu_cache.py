@@ -167,6 +167,51 @@ def test_cached_stack_decode_matches_oracle(K):
         g.close()
 
 
+def test_cached_stack_at_a_mid_size_with_eight_stages():
+    """Three cached layers of a size that spans many tiles (d 1024, d_ff 8192, rank 64, k 640, 25 % cached), K = 8, an
+    AR(1) stream: every step's execution order, the resident sets of both caches after every step (the refinements of the
+    layer before prefetch into the next layer's cache from the copy stream), the next selection and the values."""
+    spec = wl.StackSpec("cache-mid", 36, 3, 1024, 8192, True, "bf16", 64, 0.07, 4, "ar1", ar_rho=0.8)
+    arrays = wl.make_stack(spec, down_scale=20.0)
+    OLs = [orc.OracleLayer.from_arrays(a) for a in arrays]
+    C_ROWS, k, K = 2048, 640, 8
+    GLs = [ls.ls_layer_create(a, DEV, cache_rows=C_ROWS) for a in arrays]
+    caches = [orc.LogicalCache(8192, C_ROWS) for _ in arrays]
+    sels = [ls.Selection(8192, k, DEV) for _ in range(4)]
+    n = len(GLs)
+    for x0 in wl.make_tokens(spec):
+        x = dev_tensor(x0[None, :])
+        ls.ls_predict(GLs[0], x, k, sels[0])
+        caches[0].set_priorities(sels[0].scores.cpu().numpy())
+        for l in range(n):
+            last = l == n - 1
+            gn = GLs[l] if last else GLs[l + 1]
+            sel, sel_next = sels[l], sels[l + 1]
+            order = sel.order()
+            trace = ls.StepTrace(GLs[l], gn, K, 1, k)
+            x_out = torch.empty_like(x)
+            ls.ls_sparse_ffn_step(GLs[l], gn, x, x_out, sel, K, k, sel_next, trace)
+            torch.cuda.synchronize()
+            xt = trace.xtilde.cpu().numpy()
+            res = orc.sparse_ffn_step(OLs[l], OLs[l if last else l + 1], x.cpu().numpy(), order, K, k, cache=caches[l],
+                                      next_cache=None if last else caches[l + 1], xtilde_override=xt)
+            assert trace.exec_idx.cpu().numpy()[:k].tolist() == res["exec_order"].tolist()
+            assert snapshot(GLs[l]) == caches[l].resident
+            if not last:
+                assert snapshot(GLs[l + 1]) == caches[l + 1].resident
+            y_ref = res["xtilde"][K] - x.cpu().numpy()
+            for j in range(K + 1):
+                assert_values_close(xt[j] - x.cpu().numpy(), res["xtilde"][j] - x.cpu().numpy(), scale_ref=y_ref, what=f"xt[{j}]")
+            assert sel_next.order().tolist() == res["refine_orders"][K].tolist()
+            x = x_out
+    for l in range(n):
+        st = ls.ls_cache_stats(GLs[l])
+        assert (st["hits"], st["misses"], st["evictions"]) == (caches[l].hits, caches[l].misses, caches[l].evictions)
+        assert ls.ls_layer_status(GLs[l]) == 0
+    for g in GLs:
+        g.close()
+
+
 def test_reserve_times_out_on_the_host_and_the_layer_stays_usable():
     """Failure path of the one wait the calling thread has: with the compute stream still busy with ordinary earlier work
     and a wait limit of zero, ls_cache_reserve gives up with LS_ERR_TIMEOUT and a useful message.  Nothing is lost: the
