@@ -68,6 +68,49 @@ def decode_and_check(spec, arrays, K, k, n_tokens, stats, tokens=None):
         g.close()
 
 
+def test_stack_of_layers_that_differ_in_width_and_rank():
+    """Layers of one d_model but different d_ff (1024, 776, 1280: one not a multiple of 32) and predictor ranks (32, 24,
+    40): the per-layer shares of the neurons, the score rows and the bins change from layer to layer inside one launch.
+    Every boundary, partial feature and refined set against the oracle, two tokens."""
+    shapes = [(1024, 32), (776, 24), (1280, 40)]
+    specs = [wl.StackSpec(f"mixed{l}", 60 + l, 1, 256, F, True, "bf16", r, 0.2, 4, "iid_rms1") for l, (F, r) in enumerate(shapes)]
+    arrays = [wl.make_layer(sp, 0, down_scale=40.0) for sp in specs]
+    OLs = [orc.OracleLayer.from_arrays(a) for a in arrays]
+    GLs = [ls.ls_layer_create(a, DEV) for a in arrays]
+    stack = ls.ls_stack_create(GLs)
+    n, k, K = len(GLs), 160, 4
+    Fmax = max(F for F, _ in shapes)
+    sel0, sel_out = ls.Selection(shapes[0][0], k, DEV), ls.Selection(shapes[-1][0], k, DEV)
+    trace = ls.StackTrace(stack, k, n_chunks=K)
+    stats = {}
+    for x0 in wl.make_tokens(specs[0])[:2]:
+        x = torch.from_numpy(x0).cuda(DEV)
+        x_out = torch.empty_like(x)
+        ls.ls_predict(GLs[0], x, k, sel0)
+        ls.ls_stack_decode(stack, x, x_out, sel0, K, k, sel_out, trace)
+        torch.cuda.synchronize()
+        assert all(ls.ls_layer_status(g) == 0 for g in GLs)
+        X, S = trace.x.cpu().numpy(), trace.sel_idx.cpu().numpy()
+        XT, M = trace.xtilde.cpu().numpy(), trace.refine_masks.cpu().numpy().view(np.uint32)
+        for layer in range(n):
+            nxt = OLs[min(layer + 1, n - 1)]
+            order = S[layer, :k].astype(np.int64)
+            check_selection(order, orc.predictor_scores(OLs[layer], X[layer]), k, stats)
+            res = orc.sparse_ffn_step(OLs[layer], None, X[layer], order, K)
+            assert_values_close(X[layer + 1] - X[layer], res["y"][0], what=f"layer {layer}")
+            for j in range(K + 1):
+                scores = orc.predictor_scores(nxt, XT[layer, j])
+                got = mask_to_set(M[layer, j], nxt.d_ff)
+                if got != set(orc.topk_order(scores, k).tolist()):
+                    assert_set_in_tie_band(got, scores, k, stats)
+            check_selection(S[layer + 1, :k].astype(np.int64), orc.predictor_scores(nxt, X[layer + 1]), k, stats)
+        assert S[n, :k].tolist() == sel_out.order().tolist()
+    assert Fmax == 1280
+    stack.close()
+    for g in GLs:
+        g.close()
+
+
 @pytest.mark.parametrize("K", [1, 4, 8])
 def test_tiny4_stack_decode(K):
     spec = wl.SPECS["tiny4"]
