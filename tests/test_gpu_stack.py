@@ -111,7 +111,7 @@ def test_stack_of_layers_that_differ_in_width_and_rank():
         g.close()
 
 
-@pytest.mark.parametrize("K", [1, 4, 8])
+@pytest.mark.parametrize("K", [1, 2, 4, 8, 9, 16])  # K + 1 evaluations: 2 plain | 1 tile | 1 tile | 1 tile + 1 | 1 tile + 2 | 2 tiles + 1
 def test_tiny4_stack_decode(K):
     spec = wl.SPECS["tiny4"]
     stats = {}
