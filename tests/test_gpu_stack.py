@@ -68,6 +68,15 @@ def decode_and_check(spec, arrays, K, k, n_tokens, stats, tokens=None):
         g.close()
 
 
+@pytest.mark.parametrize("k,K", [(1, 1), (7, 8), (33, 16), (1024, 3)])
+def test_tiny4_stack_at_the_edges_of_k(k, K):
+    """One selected neuron; fewer neurons than stages (most CTAs and some stages stay empty); a count that no stage divides;
+    every neuron selected (k = d_ff: the sparse step is the dense one and every refined set is the whole layer)."""
+    spec = wl.SPECS["tiny4"]
+    stats = {}
+    decode_and_check(spec, wl.make_stack(spec, down_scale=50.0), K, k, 2, stats)
+
+
 def test_stack_of_layers_that_differ_in_width_and_rank():
     """Layers of one d_model but different d_ff (1024, 776, 1280: one not a multiple of 32) and predictor ranks (32, 24,
     40): the per-layer shares of the neurons, the score rows and the bins change from layer to layer inside one launch.
