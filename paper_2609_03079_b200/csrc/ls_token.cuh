@@ -135,7 +135,6 @@ struct WtShared {
   int wcnt[WT_WARPS];
   int blo, bhi, ncand, slow, found;
   float inv_x;            // 1 / rms of the layer's input
-  float act8[8];          // activations of a batch of survivors
   unsigned long long kmin, kmax;  // key range of this CTA's final scores
   double bin_hi, bin_scale;       // the score bins of the refinement in progress (all its evaluations use the same)
   double pf_thr;                  // final scores from here on: the neuron's gate row is asked into L2 (speculation)
@@ -144,7 +143,6 @@ struct WtShared {
   int b_valid;                    // the B^T rows in shared memory are intact (the general top-k borrows their place)
   double inv[WT_MAXE + 7];
   double redd[WT_WARPS];
-  unsigned long long redk[2 * WT_WARPS];
   unsigned redu[WT_WARPS];
 };
 
