@@ -493,7 +493,7 @@ int32_t predict_impl(ls_layer* L, const float* d_feature, int B, int k, double* 
   const int d = L->d, r = L->r, F = L->F;
   KernelTimer timer(LS_TIMED_PREDICT, st);
   {
-    const int wpb = 8, grid = (r + wpb - 1) / wpb;
+    const int grid = (r + 1) / 2;  // two latent rows per block of eight warps
     if (L->wd == 0) ls::ls_latent_kernel<0><<<grid, 256, 0, st>>>(L->pred_at, d_feature, d, r, B, L->z, L->sumsq);
     else ls::ls_latent_kernel<1><<<grid, 256, 0, st>>>(L->pred_at, d_feature, d, r, B, L->z, L->sumsq);
     LS_LAUNCHED();
@@ -859,7 +859,7 @@ int32_t ls_hash_predict(ls_hash_predictor* P, const float* d_feature, int32_t k,
   cudaStream_t st = (cudaStream_t)stream;
   KernelTimer timer(LS_TIMED_PREDICT, st);
   {
-    const int wpb = 8, grid = (P->r + wpb - 1) / wpb;
+    const int grid = (P->r + 1) / 2;  // two latent rows per block of eight warps
     if (P->wd == 0) ls::ls_latent_kernel<0><<<grid, 256, 0, st>>>(P->pca_t, d_feature, P->d, P->r, 1, P->z, P->sumsq);
     else ls::ls_latent_kernel<1><<<grid, 256, 0, st>>>(P->pca_t, d_feature, P->d, P->r, 1, P->z, P->sumsq);
     LS_LAUNCHED();

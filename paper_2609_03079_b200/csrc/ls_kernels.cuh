@@ -29,37 +29,49 @@ __global__ void ls_step_init_kernel(const float* __restrict__ x, const float* __
 // ------------------------------------------------------------------------------------------------------------------
 // Predictor latent, un-normalised: z[b][j] = sum_i A[i][j] * v[b][i] in fp64 (A stored transposed, one row per j),
 // plus sum of squares of the feature (the RMS norm is a scalar applied by the scores kernel).
-// One warp per latent row.
+// FOUR warps per latent row (a launch of r / 2 blocks keeps more loads in flight than one warp per row did: the kernel is
+// bound by the latency of its row loads): warp q of a row takes the 8-column chunks q, q + 4, ...; the four partial sums
+// are added in a fixed order.
 // ------------------------------------------------------------------------------------------------------------------
 template <int WD>
 __global__ void __launch_bounds__(256) ls_latent_kernel(const uint16_t* __restrict__ At, const float* __restrict__ v, int d,
                                                         int r, int B, double* __restrict__ z, double* __restrict__ sumsq) {
+  __shared__ double s_part[2][4], s_sq[4];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int j = blockIdx.x * (blockDim.x >> 5) + warp;
-  if (j >= r) return;
+  const int jr = warp >> 2, q = warp & 3;  // row of this block, quarter of the row
+  const int j = blockIdx.x * 2 + jr;
   const int nch = d >> 3;
-  const uint16_t* row = At + (size_t)j * d;
+  const uint16_t* row = At + (size_t)min(j, r - 1) * d;
   for (int b = 0; b < B; ++b) {
     const float* vb = v + (size_t)b * d;
     double acc = 0.0, sq = 0.0;
-    for (int ch = lane; ch < nch; ch += 32) {
-      float w[8];
-      unpack8<WD>(ldg128(row + ch * 8), w);
-      const float4 x0 = __ldg(reinterpret_cast<const float4*>(vb + ch * 8));
-      const float4 x1 = __ldg(reinterpret_cast<const float4*>(vb + ch * 8 + 4));
-      const float xs[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+    if (j < r) {
+#pragma unroll 2
+      for (int ch = q * 32 + lane; ch < nch; ch += 128) {
+        float w[8];
+        unpack8<WD>(ldg128(row + ch * 8), w);
+        const float4 x0 = __ldg(reinterpret_cast<const float4*>(vb + ch * 8));
+        const float4 x1 = __ldg(reinterpret_cast<const float4*>(vb + ch * 8 + 4));
+        const float xs[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
 #pragma unroll
-      for (int e = 0; e < 8; ++e) acc = fma((double)w[e], (double)xs[e], acc);
-      if (j == 0) {
+        for (int e = 0; e < 8; ++e) acc = fma((double)w[e], (double)xs[e], acc);
+        if (j == 0) {
 #pragma unroll
-        for (int e = 0; e < 8; ++e) sq = fma((double)xs[e], (double)xs[e], sq);
+          for (int e = 0; e < 8; ++e) sq = fma((double)xs[e], (double)xs[e], sq);
+        }
       }
     }
     acc = warp_sum(acc);
-    if (lane == 0) z[(size_t)b * r + j] = acc;
-    if (j == 0) {
-      sq = warp_sum(sq);
-      if (lane == 0) sumsq[b] = sq;
+    sq = warp_sum(sq);
+    __syncthreads();
+    if (lane == 0) {
+      s_part[jr][q] = acc;
+      if (j == 0) s_sq[q] = sq;
+    }
+    __syncthreads();
+    if (q == 0 && lane == 0 && j < r) {
+      z[(size_t)b * r + j] = (s_part[jr][0] + s_part[jr][1]) + (s_part[jr][2] + s_part[jr][3]);
+      if (j == 0) sumsq[b] = (s_sq[0] + s_sq[1]) + (s_sq[2] + s_sq[3]);
     }
   }
 }
@@ -67,7 +79,8 @@ __global__ void __launch_bounds__(256) ls_latent_kernel(const uint16_t* __restri
 // ------------------------------------------------------------------------------------------------------------------
 // Predictor scores: s[b][i] = sum_j B[j][i] * z[b][j] * inv_rms[b] + c[i], fp64; prio[i] = max_b s[b][i].
 // B stored transposed ([F][r], one row per neuron); one warp per neuron, every neuron reduced in the same order,
-// so equal predictor columns give bit-equal scores.
+// so equal predictor columns give bit-equal scores.  At batch 1 with r <= 512 a lane's (at most two) chunks of the
+// normalised latents stay in registers for all its neurons (the shared-memory reads of z were what the kernel waited for).
 // ------------------------------------------------------------------------------------------------------------------
 template <int WD>
 __global__ void __launch_bounds__(256) ls_scores_kernel(const uint16_t* __restrict__ Bt, const float* __restrict__ c,
@@ -75,15 +88,47 @@ __global__ void __launch_bounds__(256) ls_scores_kernel(const uint16_t* __restri
                                                         int r, int F, int B, int norm, float eps, double* __restrict__ scores,
                                                         double* __restrict__ prio, double* __restrict__ prio_user) {
   extern __shared__ double zs[];  // [B][r], normalised
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int wpb = blockDim.x >> 5;
+  const int nch = r >> 3;
+  if (B == 1 && nch <= 64) {
+    const double inv = norm == 0 ? 1.0 / sqrt(sumsq[0] / (double)d + (double)eps) : 1.0;
+    double z0[8], z1[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      z0[e] = lane < nch ? z[lane * 8 + e] * inv : 0.0;
+      z1[e] = lane + 32 < nch ? z[(lane + 32) * 8 + e] * inv : 0.0;
+    }
+    for (int i = blockIdx.x * wpb + warp; i < F; i += gridDim.x * wpb) {
+      const uint16_t* row = Bt + (size_t)i * r;
+      double acc = 0.0;
+      if (lane < nch) {
+        float w[8];
+        unpack8<WD>(ldg128(row + lane * 8), w);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc = fma((double)w[e], z0[e], acc);
+      }
+      if (lane + 32 < nch) {
+        float w[8];
+        unpack8<WD>(ldg128(row + (lane + 32) * 8), w);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc = fma((double)w[e], z1[e], acc);
+      }
+      acc = warp_sum(acc);
+      const double s = canonical_score(acc + (c ? (double)c[i] : 0.0));
+      if (lane == 0) {
+        prio[i] = s;
+        if (prio_user) prio_user[i] = s;
+      }
+    }
+    return;
+  }
   for (int t = threadIdx.x; t < B * r; t += blockDim.x) {
     const int b = t / r;
     const double inv = norm == 0 ? 1.0 / sqrt(sumsq[b] / (double)d + (double)eps) : 1.0;
     zs[t] = z[t] * inv;
   }
   __syncthreads();
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int wpb = blockDim.x >> 5;
-  const int nch = r >> 3;
   for (int i = blockIdx.x * wpb + warp; i < F; i += gridDim.x * wpb) {
     const uint16_t* row = Bt + (size_t)i * r;
     double best = 0.0;
