@@ -540,7 +540,7 @@ int32_t launch_stage(ls_layer* L, int B, const int32_t* exec_idx, const int32_t*
   const int per_stage = (sel_cap + K - 1) / K;
   {
     KernelTimer timer(LS_TIMED_GATEUP, st);
-    const int grid = std::max(1, std::min((per_stage + 7) / 8, L->sm_count * 4));
+    const int grid = std::max(1, std::min((per_stage + 1) / 2, L->sm_count * 4));  // two neurons per block
     const size_t sm = (size_t)B * d * sizeof(float);
     ls::ls_gateup_kernel<WD, BT><<<grid, 256, sm, st>>>(L->bundles, L->n_mat, L->gated, L->act, slot_of, L->b_gate, L->xin, B, d, L->norm,
                                                         L->eps, exec_idx, count_ptr, K, c, L->F, L->actv, L->max_sel, L->survive,
@@ -1107,7 +1107,7 @@ int32_t ls_sparse_ffn_step(ls_layer* L, ls_layer* next, const float* d_x, float*
     const int32_t splits = launch_stage_dispatch(L, B, exec_idx, sel->count, sel->cap, K, c, st, own_seq);
     if (splits < 0) return splits;
     const bool last = (c + 1 == K);
-    ls::ls_stage_finalize_kernel<<<std::min(64, (int)((bd + 255) / 256)), 256, 0, st>>>(
+    ls::ls_stage_finalize_kernel<<<std::min(4 * L->sm_count, (int)((bd + 31) / 32)), 256, 0, st>>>(
         L->ypart, splits, B, d, L->xt, tr.xtilde ? tr.xtilde + (size_t)(c + 1) * bd : nullptr, last ? d_x_out : nullptr);
     LS_LAUNCHED();
     LS_TRY(refine(c + 1));

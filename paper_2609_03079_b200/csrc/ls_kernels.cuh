@@ -155,7 +155,10 @@ __global__ void __launch_bounds__(256) ls_scores_kernel(const uint16_t* __restri
 
 // ------------------------------------------------------------------------------------------------------------------
 // Stage c, part 1: gate/up gather-GEMV and activation for the neurons of the stage (Eq. 1, the bracket).
-// One warp per neuron, 128-bit row loads, fp32 accumulation, warp-shuffle reduction.
+// FOUR warps per neuron (two neurons per block of eight warps): a stage is a few hundred neurons, and with one warp per
+// neuron the launch was a few dozen blocks waiting for their own row loads.  Warp q of a neuron takes the 8-column chunks
+// q, q + 4, ... of the gate and up rows; 128-bit row loads, fp32 accumulation, warp-shuffle reduction, the four partial
+// sums added in a fixed order.
 // a[b][p] = act(inv_rms_b * (w_gate[i] . x_b) + b_i) * (inv_rms_b * (w_up[i] . x_b)), p = rank position of neuron i.
 // ------------------------------------------------------------------------------------------------------------------
 template <int WD, int BT>
@@ -168,10 +171,11 @@ __global__ void __launch_bounds__(256)
   extern __shared__ __align__(16) float xs[];  // [B][d]
   __shared__ float s_inv[8];
   __shared__ double s_red[8][8];
+  __shared__ float s_acc[2][4][BT][2];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   int lo, hi;
   stage_bounds(*count_ptr, K, c, lo, hi);
-  if (lo + (int)blockIdx.x * 8 >= hi) return;
+  if (lo + (int)blockIdx.x * 2 >= hi) return;
   // Cached layer: the residents come first in the execution order; a stage that reaches into the misses waits (bounded)
   // until the rows of the layer's request have landed in their slots.
   if (landed && threadIdx.x == 0 && hi > list_hdr[1]) {
@@ -201,59 +205,69 @@ __global__ void __launch_bounds__(256)
   __syncthreads();
 
   const int nch = d >> 3;
-  for (int p = lo + blockIdx.x * 8 + warp; p < hi; p += gridDim.x * 8) {
-    const int i = exec_idx[p];
-    if ((unsigned)i >= (unsigned)F) {  // never dereference a bad index
-      if (lane == 0) {
-        set_status(status, ST_BAD_INDEX);
-        for (int b = 0; b < B; ++b) act[(size_t)b * act_stride + p] = 0.f;
-      }
-      continue;
-    }
-    const int slot = slot_of ? slot_of[i] : i;
-    if (slot < 0) {
-      if (lane == 0) {
-        set_status(status, ST_BAD_INDEX);
-        for (int b = 0; b < B; ++b) act[(size_t)b * act_stride + p] = 0.f;
-      }
-      continue;
-    }
-    const uint16_t* grow = bundles + (size_t)slot * n_mat * d;
-    const uint16_t* urow = grow + d;
+  const int jr = warp >> 2, q = warp & 3;  // neuron of this block, quarter of its rows
+  for (int p0 = lo + blockIdx.x * 2; p0 < hi; p0 += gridDim.x * 2) {
+    const int p = p0 + jr;
+    const bool live = p < hi;
+    const int i = live ? exec_idx[p] : 0;
+    const bool in_range = live && (unsigned)i < (unsigned)F;  // never dereference a bad index
+    const int slot = in_range ? (slot_of ? slot_of[i] : i) : -1;
+    const bool ok = in_range && slot >= 0;
     float ag[BT], au[BT];
 #pragma unroll
     for (int b = 0; b < BT; ++b) { ag[b] = 0.f; au[b] = 0.f; }
+    if (ok) {
+      const uint16_t* grow = bundles + (size_t)slot * n_mat * d;
+      const uint16_t* urow = grow + d;
 #pragma unroll 4
-    for (int ch = lane; ch < nch; ch += 32) {
-      float wg[8], wu[8];
-      unpack8<WD>(ld_stream128(grow + ch * 8), wg);
-      if (gated) unpack8<WD>(ld_stream128(urow + ch * 8), wu);
+      for (int ch = q * 32 + lane; ch < nch; ch += 128) {
+        float wg[8], wu[8];
+        unpack8<WD>(ld_stream128(grow + ch * 8), wg);
+        if (gated) unpack8<WD>(ld_stream128(urow + ch * 8), wu);
 #pragma unroll
-      for (int b = 0; b < BT; ++b) {
-        if (b < B) {
-          const float4 x0 = *reinterpret_cast<const float4*>(xs + b * d + ch * 8);
-          const float4 x1 = *reinterpret_cast<const float4*>(xs + b * d + ch * 8 + 4);
-          const float xv[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+        for (int b = 0; b < BT; ++b) {
+          if (b < B) {
+            const float4 x0 = *reinterpret_cast<const float4*>(xs + b * d + ch * 8);
+            const float4 x1 = *reinterpret_cast<const float4*>(xs + b * d + ch * 8 + 4);
+            const float xv[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
 #pragma unroll
-          for (int e = 0; e < 8; ++e) {
-            ag[b] = fmaf(wg[e], xv[e], ag[b]);
-            if (gated) au[b] = fmaf(wu[e], xv[e], au[b]);
+            for (int e = 0; e < 8; ++e) {
+              ag[b] = fmaf(wg[e], xv[e], ag[b]);
+              if (gated) au[b] = fmaf(wu[e], xv[e], au[b]);
+            }
           }
         }
       }
     }
-    bool any = false;
 #pragma unroll
     for (int b = 0; b < BT; ++b) {
       if (b < B) {
-        const float g = warp_sum(ag[b]) * s_inv[b] + (b_gate ? b_gate[i] : 0.f);
-        float a = act_kind == 0 ? fmaxf(g, 0.f) : g / (1.f + expf(-g));  // ReLU, or SiLU as Eq. 1 prints it
-        if (gated) a *= warp_sum(au[b]) * s_inv[b];
-        if (lane == 0) act[(size_t)b * act_stride + p] = a;
-        any |= (a != 0.f);
+        const float g = warp_sum(ag[b]), u = gated ? warp_sum(au[b]) : 0.f;
+        if (lane == 0) { s_acc[jr][q][b][0] = g; s_acc[jr][q][b][1] = u; }
       }
     }
-    if (lane == 0 && any) atomicOr(&survive[i >> 5], 1u << (i & 31));
+    __syncthreads();
+    if (q == 0 && lane == 0 && live) {
+      if (!ok) {
+        set_status(status, ST_BAD_INDEX);
+        for (int b = 0; b < B; ++b) act[(size_t)b * act_stride + p] = 0.f;
+      } else {
+        bool any = false;
+#pragma unroll
+        for (int b = 0; b < BT; ++b) {
+          if (b < B) {
+            const float gs = (s_acc[jr][0][b][0] + s_acc[jr][1][b][0]) + (s_acc[jr][2][b][0] + s_acc[jr][3][b][0]);
+            const float g = gs * s_inv[b] + (b_gate ? b_gate[i] : 0.f);
+            float a = act_kind == 0 ? fmaxf(g, 0.f) : g / (1.f + expf(-g));  // ReLU, or SiLU as Eq. 1 prints it
+            if (gated) a *= ((s_acc[jr][0][b][1] + s_acc[jr][1][b][1]) + (s_acc[jr][2][b][1] + s_acc[jr][3][b][1])) * s_inv[b];
+            act[(size_t)b * act_stride + p] = a;
+            any |= (a != 0.f);
+          }
+        }
+        if (any) atomicOr(&survive[i >> 5], 1u << (i & 31));
+      }
+    }
+    __syncthreads();
   }
 }
 
@@ -309,16 +323,27 @@ __global__ void __launch_bounds__(256)
 }
 
 // x~^(c+1) = x~^(c) + sum over splits (fixed order: deterministic); optional copies to the trace and to x_out.
+// Eight threads per element (the splits dealt over them, their partial sums added by a fixed tree): with one thread per
+// element the kernel was a handful of blocks each waiting for its own chain of loads.  blockDim.x a multiple of 32.
 __global__ void ls_stage_finalize_kernel(const float* __restrict__ ypart, int nsplit, int B, int d, float* xt, float* trace_out,
                                          float* x_out) {
   const int n = B * d;
-  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+  const int part = threadIdx.x & 7;
+  const int per_block = blockDim.x >> 3;
+  for (int i0 = blockIdx.x * per_block; i0 < n; i0 += gridDim.x * per_block) {  // (uniform over the block: shuffles below)
+    const int i = i0 + (threadIdx.x >> 3);
     float s = 0.f;
-    for (int sp = 0; sp < nsplit; ++sp) s += ypart[(size_t)sp * n + i];
-    const float v = xt[i] + s;
-    xt[i] = v;
-    if (trace_out) trace_out[i] = v;
-    if (x_out) x_out[i] = v;
+    if (i < n)
+      for (int sp = part; sp < nsplit; sp += 8) s += ypart[(size_t)sp * n + i];
+    s += __shfl_xor_sync(0xffffffffu, s, 1);
+    s += __shfl_xor_sync(0xffffffffu, s, 2);
+    s += __shfl_xor_sync(0xffffffffu, s, 4);
+    if (part == 0 && i < n) {
+      const float v = xt[i] + s;
+      xt[i] = v;
+      if (trace_out) trace_out[i] = v;
+      if (x_out) x_out[i] = v;
+    }
   }
 }
 
