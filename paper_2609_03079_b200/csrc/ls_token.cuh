@@ -504,7 +504,6 @@ __device__ __forceinline__ void wt_fetch_predictor(const WtCall& C, WtShared& sh
 
 // The same rows of B^T once more, by ordinary asynchronous copies (after a degenerate selection borrowed their place).
 __device__ __noinline__ void wt_refetch_b(const WtCall& C, const WtLayer& L, unsigned char* smem) {
-  const int G = gridDim.x;
   const int per = L.per, n0 = min(L.Fn, (int)blockIdx.x * per), n1 = min(L.Fn, n0 + per);
   const int RB = wt_brow_bytes(L.r);
   const int npieces = (((n1 - n0 + 7) >> 3) * 8) * (RB >> 4);
@@ -821,7 +820,7 @@ template <int WD>
 __device__ __noinline__ void wt_score_evals(const WtCall& C, WtShared& sh, const WtLayer& L, int e0, int ne, bool last) {
   extern __shared__ __align__(128) unsigned char wt_smem[];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, g = lane >> 2, t = lane & 3;
-  const int r = L.r, Fn = L.Fn, G = gridDim.x, K = C.K;
+  const int r = L.r, Fn = L.Fn, K = C.K;
   const int rz = (r + 4) & ~3;
   double* s_z = reinterpret_cast<double*>(wt_smem + C.lay.u_off + C.lay.yz_off);
   double* s_dot = reinterpret_cast<double*>(wt_smem + C.lay.u_off + C.lay.dot_off);  // [ne][per8] raw dot products
